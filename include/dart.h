@@ -1,0 +1,219 @@
+/*
+ * dart.h -- C ABI of the B200 (sm_100a) implementation of DART's drafting step.
+ *
+ * One call of dart_draft_step followed by one call of dart_build_tree is one "draft step":
+ * target hidden states -> one draft decoder layer over the prefix KV cache plus K query rows
+ * -> LM head -> per-position log-softmax + top-k -> N-gram-scored tree pruning -> a
+ * fixed-budget draft token tree (token ids, parents, tree-attention mask).
+ *
+ * Conventions
+ *   - Every pointer is labelled HOST or DEVICE.  Device buffers are caller-owned unless stated.
+ *   - bf16 tensors are row-major with the last index fastest; weight matrices are [out, in];
+ *     every device pointer must be 16-byte aligned.
+ *   - All GPU work is enqueued on the CUDA stream passed as `void* cuda_stream` (a cudaStream_t;
+ *     NULL = the legacy default stream).  dart_draft_step and dart_build_tree do not
+ *     synchronise, allocate, or copy between host and device.
+ *   - Return value: DART_OK (0) or a negative dart_status.  Argument errors are reported
+ *     synchronously and enqueue nothing.  Errors that only the device can detect (a lookup
+ *     that ran past its probe bound) set a status word read by dart_last_device_status.
+ *   - One handle may be used from one host thread and one stream at a time.
+ *   - There is no CPU fallback: on a machine without an sm_100 device dart_draft_init fails.
+ */
+#ifndef DART_H_
+#define DART_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum dart_status {
+  DART_OK = 0,
+  DART_ERR_INVALID_ARG = -1,      /* NULL/misaligned pointer, shape the kernels do not support */
+  DART_ERR_UNSUPPORTED_ARCH = -2, /* current device is not compute capability 10.x */
+  DART_ERR_CUDA = -3,             /* a CUDA runtime call failed; see dart_last_cuda_error */
+  DART_ERR_CAPACITY = -4,         /* batch > max_batch, or prefix + K > max_prefix */
+  DART_ERR_TIMEOUT = -5,          /* a bounded device-side loop gave up (device status word) */
+  DART_ERR_INTERNAL = -6
+} dart_status;
+
+typedef struct dart_handle dart_handle; /* opaque; owns workspace + the device N-gram table */
+
+/*
+ * Shapes and hyper-parameters, fixed for the lifetime of a handle.
+ * Layer shapes follow Appendix B ("hyperparameters ... aligned with the target model");
+ * topk/beam/tree_budget and the Combine weights are Appendix D's k_i, w, theta+1, w_ng,
+ * 0.9^level, (level+1)^-0.7.
+ */
+typedef struct dart_config {
+  uint32_t struct_size;  /* = sizeof(dart_config); guards against layout mismatch */
+  int32_t hidden;        /* h; multiple of 64 */
+  int32_t n_q_heads;     /* H_q */
+  int32_t n_kv_heads;    /* H_kv; H_q % H_kv == 0 and (H_q/H_kv)*K <= 64 */
+  int32_t head_dim;      /* d_h: 64 or 128 */
+  int32_t mlp_inter;     /* I; multiple of 16 */
+  int32_t vocab;         /* V; multiple of 16, < 2^21 */
+  int32_t feat_in;       /* width of the concatenated target features (3h); multiple of 16 */
+  int32_t max_batch;     /* sequences per call, <= 64 */
+  int32_t max_prefix;    /* P_cap: rows per sequence in the caller's KV cache */
+  int32_t K;             /* query rows per sequence = future positions d (Section 3.2); 1..8 */
+  int32_t topk;          /* k_i: candidates kept per position, 1..32 (Appendix D: 25) */
+  int32_t beam;          /* w: beam width, 1..32 (Appendix D: 20) */
+  int32_t tree_budget;   /* nodes in the output tree including the root, 2..64 (theta + 1 = 60) */
+  int32_t ngram_order;   /* 2 or 3 (Appendix C: 3) */
+  float rope_theta;      /* RoPE base (1e6) */
+  float rms_eps;         /* RMSNorm epsilon (1e-6) */
+  float w_ng;            /* Combine: N-gram weight (0.5) */
+  float logit_decay;     /* Combine: w_logit = logit_decay^level (0.9) */
+  float level_exp;       /* Combine: w_level = (level+1)^-level_exp (0.7) */
+  float eps_logit;       /* epsilon inside s_logit = log(softmax + eps) */
+  float eps_ng;          /* epsilon of a missing N-gram: s_ng = log(eps_ng) */
+  float temperature;     /* 0 = deterministic top-k; > 0 = Gumbel-top-k on logits / temperature */
+  uint64_t philox_seed;  /* key of the Philox4x32-10 stream used when temperature > 0 */
+} dart_config;
+
+/*
+ * Draft-model parameters (Appendix B "Trainable parameters": FC, decoder layer, LM head, mask
+ * representation; the embedding is the target's).  DEVICE pointers to bf16, row-major
+ * [out, in]; caller-owned, never written, must outlive the handle.
+ */
+typedef struct dart_weights {
+  const void* w_fc;       /* [h, feat_in]   fusion of the three target layers' hidden states */
+  const void* embed;      /* [V, h]         target embedding table (shifted token embedding) */
+  const void* mask_vec;   /* [2h]           learned <mask> representation, stands for [g ; e] */
+  const void* norm_g;     /* [h]            RMSNorm gain on g */
+  const void* norm_e;     /* [h]            RMSNorm gain on e */
+  const void* w_q;        /* [H_q*d_h, 2h]  */
+  const void* w_k;        /* [H_kv*d_h, 2h] */
+  const void* w_v;        /* [H_kv*d_h, 2h] */
+  const void* w_o;        /* [h, H_q*d_h]   */
+  const void* norm_post;  /* [h]            RMSNorm gain before the MLP */
+  const void* w_gate;     /* [I, h] */
+  const void* w_up;       /* [I, h] */
+  const void* w_down;     /* [h, I] */
+  const void* norm_final; /* [h]            RMSNorm gain before the LM head */
+  const void* w_lm;       /* [V, h]         the drafter's own LM head */
+} dart_weights;
+
+/*
+ * N-gram rows (Appendix C), HOST arrays of length n_rows, copied into a library-owned
+ * device hash table by dart_draft_init.  Row i says: after context (ctx0[i], ctx1[i]) the
+ * token next[i] has continuity score score[i] = log(Pr(next | context) + eps), Appendix D's
+ * s_ng.  order[i] is 3 (trigram) or 2 (bigram; ctx0[i] ignored).  Of duplicate rows the first wins.
+ */
+typedef struct dart_ngram_host {
+  int64_t n_rows;
+  const uint8_t* order;
+  const int32_t* ctx0;
+  const int32_t* ctx1;
+  const int32_t* next;
+  const float* score;
+} dart_ngram_host;
+
+/*
+ * Inputs of one forward pass (Section 3.2).  Per sequence b the K query rows are
+ * r = 0..K-1 at absolute positions P_b + r, P_b = seq_lens[b]; rows r < n_fresh carry fresh
+ * target features and the id of the token that follows them (shifted embedding), the rest
+ * are <mask> rows.  The canonical step is n_fresh = 1: the last prefix position plus d-1 masks.
+ */
+typedef struct dart_step_in {
+  int32_t batch;          /* B <= max_batch */
+  int32_t n_fresh;        /* F, 0..K (0: K mask rows, feats/tokens unused) */
+  const void* feats;      /* DEVICE bf16 [B, F, feat_in] */
+  const int32_t* tokens;  /* DEVICE i32  [B, F] next-token ids, 0 <= id < V */
+  const int32_t* seq_lens;      /* DEVICE i32 [B]  P_b: rows already in the cache */
+  const int32_t* seq_lens_host; /* HOST   i32 [B]  same values; used for capacity checks and launch sizing */
+  void* k_cache;          /* DEVICE bf16 [max_batch, H_kv, max_prefix, d_h], post-RoPE keys */
+  void* v_cache;          /* DEVICE bf16, same layout.  The call writes rows P_b .. P_b+K-1 of both:
+                             rows < P_b+F are the fresh positions' k, v (a valid append; the caller
+                             advances seq_lens), rows >= P_b+F are scratch that the next call overwrites. */
+  uint64_t step_counter;  /* Philox counter word; change it every call when temperature > 0 */
+} dart_step_in;
+
+/*
+ * Outputs of one forward pass: Algorithm 1 lines 6-8 for every logit row.  Row r predicts
+ * the token after position P_b + r (shifted logits); rows r >= max(F,1)-1 are the d logit
+ * rows of Section 3.2, earlier rows are computed as well.
+ */
+typedef struct dart_step_out {
+  int32_t* topk_ids;      /* DEVICE i32 [B, K, topk]  S_i, by selection value desc, ties lower id */
+  float* topk_slogit;     /* DEVICE f32 [B, K, topk]  s_logit = log(softmax(logits/T) + eps_logit) */
+  float* logits;          /* DEVICE f32 [B, K, V] or NULL.  Full logits (before 1/T), for checking only */
+} dart_step_out;
+
+/* Inputs of Algorithm 1 for B sequences. */
+typedef struct dart_tree_in {
+  int32_t batch;
+  int32_t first_row;          /* first logit row used as level 0 (= max(F,1)-1) */
+  int32_t n_levels;           /* d = number of levels, first_row + n_levels <= K */
+  const int32_t* topk_ids;    /* DEVICE i32 [B, K, topk] as written by dart_draft_step */
+  const float* topk_slogit;   /* DEVICE f32 [B, K, topk] */
+  const int32_t* ctx_tail;    /* DEVICE i32 [B, 2]: the last two known tokens (c_-2, c_-1); -1 = absent */
+} dart_tree_in;
+
+/*
+ * The pruned draft tree per sequence.  Slot 0 is the root (token c_-1, parent -1, depth 0);
+ * slots 1..n_nodes-1 are the selected nodes by score descending.  parents[x] < x.
+ * mask[x][y] = 1 iff y == x or y is an ancestor of x (the tree-attention mask).
+ * Unused slots: token -1, parent -1, depth -1, mask row 0.
+ */
+typedef struct dart_tree_out {
+  int32_t* tokens;   /* DEVICE i32 [B, tree_budget] */
+  int32_t* parents;  /* DEVICE i32 [B, tree_budget] */
+  int32_t* depth;    /* DEVICE i32 [B, tree_budget] */
+  uint8_t* mask;     /* DEVICE u8  [B, tree_budget, tree_budget] */
+  int32_t* n_nodes;  /* DEVICE i32 [B] */
+  float* scores;     /* DEVICE f32 [B, tree_budget] or NULL: the (ancestor-clamped) node scores */
+} dart_tree_out;
+
+/*
+ * Create a handle (Section 3.2 + Section 4 set-up): validates cfg, records the weight
+ * pointers, builds the device N-gram hash table from the host rows (ngram may be NULL or
+ * empty: every lookup then misses), allocates the workspace (the only allocation the library
+ * ever makes) and precomputes Appendix D's per-level weights.  Synchronous.
+ * Errors: INVALID_ARG, UNSUPPORTED_ARCH, CUDA.  *out is NULL on failure.
+ */
+int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const dart_ngram_host* ngram,
+                    dart_handle** out);
+
+/*
+ * One forward pass of the draft layer and LM head with fused log-softmax/top-k
+ * (Section 3.2; Algorithm 1 lines 6-8; Appendix D s_logit).  Asynchronous on `cuda_stream`.
+ * Errors: INVALID_ARG (NULL pointers, n_fresh out of range), CAPACITY (batch > max_batch or
+ * seq_lens_host[b] + K > max_prefix).
+ */
+int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out* out, void* cuda_stream);
+
+/*
+ * Continuity-aware tree pruning (Algorithm 1, Appendix D) for B sequences, one thread block
+ * per sequence.  Asynchronous on `cuda_stream`.  Bit-exact with a sequential fp32 evaluation
+ * of Algorithm 1 that breaks ties by generation order.  Errors: INVALID_ARG, CAPACITY.
+ */
+int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out* out, void* cuda_stream);
+
+/* Free the workspace and the N-gram table.  The caller's buffers are untouched. */
+int dart_draft_destroy(dart_handle* h);
+
+/* Device-side status word since the last call of this function: DART_OK or DART_ERR_TIMEOUT.
+ * Synchronises `cuda_stream`. */
+int dart_last_device_status(dart_handle* h, void* cuda_stream);
+
+/* The cudaError_t (as int) behind the last DART_ERR_CUDA of this handle (or of init when h is NULL). */
+int dart_last_cuda_error(const dart_handle* h);
+
+/* Human-readable name of a dart_status. */
+const char* dart_status_string(int status);
+
+/* Bytes of device workspace a handle for `cfg` allocates (excluding the N-gram table); 0 if cfg is invalid. */
+size_t dart_workspace_bytes(const dart_config* cfg);
+
+/* Number of kernels one dart_draft_step / dart_build_tree call enqueues for this batch size
+ * (used by benchmarks to report launch counts). */
+int dart_step_launch_count(const dart_handle* h, int batch, int n_fresh);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DART_H_ */

@@ -1,0 +1,203 @@
+"""Thin ctypes binding of ``libdart.so`` (the C ABI declared in ``include/dart.h``).
+
+Argument marshalling only: torch provides device memory and streams, every step of the
+drafting path runs in the library's CUDA kernels.  There is no fallback: if the shared
+library is missing or fails to load, importing callers get an exception.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdart.so")
+
+DART_OK = 0
+DART_ERR_INVALID_ARG = -1
+DART_ERR_UNSUPPORTED_ARCH = -2
+DART_ERR_CUDA = -3
+DART_ERR_CAPACITY = -4
+DART_ERR_TIMEOUT = -5
+DART_ERR_INTERNAL = -6
+
+EXPORTS = [
+    "dart_draft_init", "dart_draft_step", "dart_build_tree", "dart_draft_destroy", "dart_last_device_status",
+    "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_step_launch_count",
+]
+
+
+class DartConfig(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("hidden", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("mlp_inter", C.c_int32), ("vocab", C.c_int32), ("feat_in", C.c_int32),
+        ("max_batch", C.c_int32), ("max_prefix", C.c_int32), ("K", C.c_int32), ("topk", C.c_int32),
+        ("beam", C.c_int32), ("tree_budget", C.c_int32), ("ngram_order", C.c_int32),
+        ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("w_ng", C.c_float), ("logit_decay", C.c_float),
+        ("level_exp", C.c_float), ("eps_logit", C.c_float), ("eps_ng", C.c_float), ("temperature", C.c_float),
+        ("philox_seed", C.c_uint64),
+    ]
+
+
+WEIGHT_NAMES = ["w_fc", "embed", "mask_vec", "norm_g", "norm_e", "w_q", "w_k", "w_v", "w_o", "norm_post",
+                "w_gate", "w_up", "w_down", "norm_final", "w_lm"]
+
+
+class DartWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
+
+
+class DartNgramHost(C.Structure):
+    _fields_ = [("n_rows", C.c_int64), ("order", C.c_void_p), ("ctx0", C.c_void_p), ("ctx1", C.c_void_p),
+                ("next", C.c_void_p), ("score", C.c_void_p)]
+
+
+class DartStepIn(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_fresh", C.c_int32), ("feats", C.c_void_p), ("tokens", C.c_void_p),
+                ("seq_lens", C.c_void_p), ("seq_lens_host", C.c_void_p), ("k_cache", C.c_void_p),
+                ("v_cache", C.c_void_p), ("step_counter", C.c_uint64)]
+
+
+class DartStepOut(C.Structure):
+    _fields_ = [("topk_ids", C.c_void_p), ("topk_slogit", C.c_void_p), ("logits", C.c_void_p)]
+
+
+class DartTreeIn(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("first_row", C.c_int32), ("n_levels", C.c_int32), ("topk_ids", C.c_void_p),
+                ("topk_slogit", C.c_void_p), ("ctx_tail", C.c_void_p)]
+
+
+class DartTreeOut(C.Structure):
+    _fields_ = [("tokens", C.c_void_p), ("parents", C.c_void_p), ("depth", C.c_void_p), ("mask", C.c_void_p),
+                ("n_nodes", C.c_void_p), ("scores", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libdart.so (once).  Raises if it has not been built: there is no CPU fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_19278_b200.build` "
+                               "(the drafting step has no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.dart_draft_init.argtypes = [C.POINTER(DartConfig), C.POINTER(DartWeights), C.POINTER(DartNgramHost),
+                                      C.POINTER(C.c_void_p)]
+        L.dart_draft_init.restype = C.c_int
+        L.dart_draft_step.argtypes = [C.c_void_p, C.POINTER(DartStepIn), C.POINTER(DartStepOut), C.c_void_p]
+        L.dart_draft_step.restype = C.c_int
+        L.dart_build_tree.argtypes = [C.c_void_p, C.POINTER(DartTreeIn), C.POINTER(DartTreeOut), C.c_void_p]
+        L.dart_build_tree.restype = C.c_int
+        L.dart_draft_destroy.argtypes = [C.c_void_p]
+        L.dart_draft_destroy.restype = C.c_int
+        L.dart_last_device_status.argtypes = [C.c_void_p, C.c_void_p]
+        L.dart_last_device_status.restype = C.c_int
+        L.dart_last_cuda_error.argtypes = [C.c_void_p]
+        L.dart_last_cuda_error.restype = C.c_int
+        L.dart_status_string.argtypes = [C.c_int]
+        L.dart_status_string.restype = C.c_char_p
+        L.dart_workspace_bytes.argtypes = [C.POINTER(DartConfig)]
+        L.dart_workspace_bytes.restype = C.c_size_t
+        L.dart_step_launch_count.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        L.dart_step_launch_count.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+class DartError(RuntimeError):
+    def __init__(self, status: int, where: str, cuda_error: int = 0):
+        self.status = status
+        name = lib().dart_status_string(status).decode()
+        extra = f" (cudaError {cuda_error})" if cuda_error else ""
+        super().__init__(f"{where}: {name}{extra}")
+
+
+def make_config(w, **over) -> DartConfig:
+    """dart_config from a synthetic.Workload (Appendix D defaults for the pruning constants)."""
+    cfg = DartConfig()
+    cfg.struct_size = C.sizeof(DartConfig)
+    vals = dict(hidden=w.hidden, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                mlp_inter=w.mlp_inter, vocab=w.vocab, feat_in=w.feat_in, max_batch=w.batch,
+                max_prefix=w.max_prefix, K=w.K, topk=w.topk, beam=w.beam, tree_budget=w.tree_budget,
+                ngram_order=3, rope_theta=1e6, rms_eps=1e-6, w_ng=0.5, logit_decay=0.9, level_exp=0.7,
+                eps_logit=1e-10, eps_ng=1e-10, temperature=w.temperature, philox_seed=1234)
+    vals.update(over)
+    for k, v in vals.items():
+        setattr(cfg, k, v)
+    return cfg
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+class DartDraft:
+    """Owner of a dart_handle.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, cfg: DartConfig, weights: Dict[str, torch.Tensor], ngram: Optional[Dict[str, np.ndarray]] = None):
+        self._h = C.c_void_p()
+        self.cfg = cfg
+        self._weights = {n: weights[n] for n in WEIGHT_NAMES}      # keep the device tensors alive
+        for n, t in self._weights.items():
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous(), n
+        ws = DartWeights(**{n: t.data_ptr() for n, t in self._weights.items()})
+        ng = None
+        if ngram is not None and len(ngram["next"]):
+            self._ng = {k: np.ascontiguousarray(v) for k, v in ngram.items()}
+            assert self._ng["order"].dtype == np.uint8 and self._ng["score"].dtype == np.float32
+            ng = DartNgramHost(len(self._ng["next"]), self._ng["order"].ctypes.data, self._ng["ctx0"].ctypes.data,
+                               self._ng["ctx1"].ctypes.data, self._ng["next"].ctypes.data, self._ng["score"].ctypes.data)
+        rc = lib().dart_draft_init(C.byref(cfg), C.byref(ws), C.byref(ng) if ng is not None else None, C.byref(self._h))
+        if rc != DART_OK:
+            raise DartError(rc, "dart_draft_init", lib().dart_last_cuda_error(None))
+
+    def close(self):
+        if self._h:
+            lib().dart_draft_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @staticmethod
+    def _stream(stream) -> int:
+        return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+
+    def draft_step(self, *, feats, tokens, seq_lens, seq_lens_host: np.ndarray, k_cache, v_cache, n_fresh: int,
+                   topk_ids, topk_slogit, logits=None, step_counter: int = 0, stream=None) -> None:
+        """dart_draft_step: all tensors are caller-owned device tensors; seq_lens_host is a host int32 array."""
+        slh = np.ascontiguousarray(seq_lens_host, dtype=np.int32)
+        sin = DartStepIn(len(slh), n_fresh, _ptr(feats), _ptr(tokens), _ptr(seq_lens), slh.ctypes.data,
+                         _ptr(k_cache), _ptr(v_cache), step_counter)
+        sout = DartStepOut(_ptr(topk_ids), _ptr(topk_slogit), _ptr(logits))
+        rc = lib().dart_draft_step(self._h, C.byref(sin), C.byref(sout), self._stream(stream))
+        if rc != DART_OK:
+            raise DartError(rc, "dart_draft_step", lib().dart_last_cuda_error(self._h))
+
+    def build_tree(self, *, batch: int, topk_ids, topk_slogit, ctx_tail, tokens, parents, depth, mask, n_nodes,
+                   scores=None, first_row: int = 0, n_levels: Optional[int] = None, stream=None) -> None:
+        """dart_build_tree on caller-owned device tensors."""
+        tin = DartTreeIn(batch, first_row, self.cfg.K - first_row if n_levels is None else n_levels,
+                         _ptr(topk_ids), _ptr(topk_slogit), _ptr(ctx_tail))
+        tout = DartTreeOut(_ptr(tokens), _ptr(parents), _ptr(depth), _ptr(mask), _ptr(n_nodes), _ptr(scores))
+        rc = lib().dart_build_tree(self._h, C.byref(tin), C.byref(tout), self._stream(stream))
+        if rc != DART_OK:
+            raise DartError(rc, "dart_build_tree", lib().dart_last_cuda_error(self._h))
+
+    def device_status(self, stream=None) -> int:
+        return lib().dart_last_device_status(self._h, self._stream(stream))
+
+    def launch_count(self, batch: int, n_fresh: int) -> int:
+        return lib().dart_step_launch_count(self._h, batch, n_fresh)
+
+
+def workspace_bytes(cfg: DartConfig) -> int:
+    return lib().dart_workspace_bytes(C.byref(cfg))

@@ -1,0 +1,496 @@
+// C ABI of the DART drafting step: handle management, argument validation, launch planning.
+// Every arithmetic step of the path runs in the kernels of this directory; this file only
+// validates, sizes and enqueues.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <vector>
+
+#include "../../include/dart.h"
+#include "kernels.h"
+
+using namespace dart;
+
+namespace {
+
+int g_init_cuda_error = 0;
+
+struct Workspace {
+  void* base = nullptr;
+  size_t bytes = 0;
+  float* part = nullptr;        // split partials of the current projection
+  float* res = nullptr;         // [Mmax, h] residual stream
+  bf16 *z_hi = nullptr, *z_lo = nullptr;   // [Mmax, 2h]
+  bf16* q = nullptr;            // [Mmax, Hq*dh]
+  bf16 *a_hi = nullptr, *a_lo = nullptr;   // [Mmax, Hq*dh]
+  bf16 *n_hi = nullptr, *n_lo = nullptr;   // [Mmax, h]
+  bf16 *u_hi = nullptr, *u_lo = nullptr;   // [Mmax, I]
+  float *o_part = nullptr, *ml_part = nullptr;
+  float *lm_stats = nullptr, *lm_key = nullptr, *lm_y = nullptr;
+  int32_t* lm_id = nullptr;
+  int* status = nullptr;
+};
+
+}  // namespace
+
+struct dart_handle {
+  dart_config cfg;
+  dart_weights w;
+  int device = 0;
+  int n_sm = 0;
+  int last_cuda_error = 0;
+  GemmPlan plan_fc, plan_qkv, plan_o, plan_gu, plan_down;
+  int lm_grid = 0;
+  int attn_pairs_cap = 0;  // capacity of the attention partial buffers in (sequence, chunk) pairs
+  Workspace ws;
+  NgramSlot* ng_slots = nullptr;
+  uint32_t ng_mask = 0, ng_max_probe = 0;
+  float wl[8], wv[8], wn, miss;
+  std::vector<int*> owned;  // small device arrays (plan tables)
+};
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+bool aligned16(const void* p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool config_ok(const dart_config* c) {
+  if (c == nullptr || c->struct_size != sizeof(dart_config)) return false;
+  if (c->hidden < 64 || c->hidden % 64 != 0) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads != 0) return false;
+  if (c->K < 1 || c->K > 8) return false;
+  if ((c->n_q_heads / c->n_kv_heads) * c->K > 64) return false;
+  if (c->mlp_inter < 16 || c->mlp_inter % 16 != 0) return false;
+  if (c->vocab < 16 || c->vocab % 16 != 0 || c->vocab >= (1 << 21) - 1) return false;
+  if (c->feat_in < 16 || c->feat_in % 16 != 0) return false;
+  if (c->max_batch < 1 || c->max_batch > 32 || c->max_batch * c->K > 128) return false;
+  if (c->max_prefix < c->K) return false;
+  if (c->topk < 1 || c->topk > 32 || c->topk > c->vocab) return false;
+  if (c->beam < 1 || c->beam > 32) return false;
+  if (c->tree_budget < 2 || c->tree_budget > 64) return false;
+  if (c->ngram_order != 2 && c->ngram_order != 3) return false;
+  if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f) || !(c->temperature >= 0.f)) return false;
+  if (!(c->eps_ng > 0.f) || !(c->eps_logit >= 0.f)) return false;
+  return true;
+}
+
+// Cut the flattened (tile, k-step) space of a projection into `grid_target` equal ranges.
+void make_plan_host(GemmPlan& p, const GemmSeg* segs, int nseg, int Kd, int grid_target, std::vector<int>& clo,
+                    std::vector<int>& chi) {
+  p.nseg = nseg;
+  int tiles = 0;
+  for (int i = 0; i < 3; ++i) {
+    if (i < nseg) {
+      p.seg[i] = segs[i];
+      p.seg[i].tile0 = tiles;
+      tiles += (segs[i].rows + 127) / 128;
+    } else {
+      p.seg[i] = p.seg[0];
+    }
+  }
+  p.Kd = Kd;
+  p.SK = (Kd + 63) / 64;
+  p.n_tiles = tiles;
+  p.U = (long long)tiles * p.SK;
+  p.grid = (int)((long long)grid_target < p.U ? grid_target : p.U);
+  clo.assign(tiles, 0x7fffffff);
+  chi.assign(tiles, -1);
+  p.slots = 1;
+  for (int c = 0; c < p.grid; ++c) {
+    const long long u0 = ((long long)c * p.U) / p.grid, u1 = ((long long)(c + 1) * p.U) / p.grid;
+    if (u0 >= u1) continue;
+    const int t0 = (int)(u0 / p.SK), t1 = (int)((u1 - 1) / p.SK);
+    if (t1 - t0 + 1 > p.slots) p.slots = t1 - t0 + 1;
+    for (int t = t0; t <= t1; ++t) {
+      if (c < clo[t]) clo[t] = c;
+      if (c > chi[t]) chi[t] = c;
+    }
+  }
+}
+
+size_t part_floats(const GemmPlan& p, int MP) { return (size_t)p.grid * p.slots * 128 * MP; }
+
+struct Layout {
+  size_t total = 0;
+  size_t take(size_t bytes) {
+    const size_t off = total;
+    total += align_up(bytes, 256);
+    return off;
+  }
+};
+
+// Sizes every workspace region; with base != nullptr also assigns the pointers.
+size_t layout_workspace(const dart_config& c, int n_sm, size_t part_max_floats, int attn_pairs_cap, int lm_grid,
+                        char* base, Workspace* ws) {
+  Layout L;
+  const size_t Mmax = (size_t)c.max_batch * c.K;
+  const size_t MPmax = padded_tokens((int)Mmax);
+  const size_t dq = (size_t)c.n_q_heads * c.head_dim;
+  size_t o;
+#define TAKE(field, type, bytes) \
+  o = L.take(bytes);             \
+  if (base) ws->field = reinterpret_cast<type>(base + o);
+  TAKE(part, float*, part_max_floats * sizeof(float));
+  TAKE(res, float*, Mmax * c.hidden * sizeof(float));
+  TAKE(z_hi, bf16*, Mmax * 2 * c.hidden * sizeof(bf16));
+  TAKE(z_lo, bf16*, Mmax * 2 * c.hidden * sizeof(bf16));
+  TAKE(q, bf16*, Mmax * dq * sizeof(bf16));
+  TAKE(a_hi, bf16*, Mmax * dq * sizeof(bf16));
+  TAKE(a_lo, bf16*, Mmax * dq * sizeof(bf16));
+  TAKE(n_hi, bf16*, Mmax * c.hidden * sizeof(bf16));
+  TAKE(n_lo, bf16*, Mmax * c.hidden * sizeof(bf16));
+  TAKE(u_hi, bf16*, Mmax * c.mlp_inter * sizeof(bf16));
+  TAKE(u_lo, bf16*, Mmax * c.mlp_inter * sizeof(bf16));
+  TAKE(o_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * c.head_dim * sizeof(float));
+  TAKE(ml_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * 2 * sizeof(float));
+  TAKE(lm_stats, float*, (size_t)lm_grid * MPmax * 2 * sizeof(float));
+  TAKE(lm_key, float*, (size_t)lm_grid * MPmax * 32 * sizeof(float));
+  TAKE(lm_y, float*, (size_t)lm_grid * MPmax * 32 * sizeof(float));
+  TAKE(lm_id, int32_t*, (size_t)lm_grid * MPmax * 32 * sizeof(int32_t));
+  TAKE(status, int*, 256);
+#undef TAKE
+  (void)n_sm;
+  return L.total;
+}
+
+struct PlanSet {
+  GemmPlan fc, qkv, o, gu, down;
+  std::vector<int> clo[5], chi[5];
+  size_t part_max = 0;
+};
+
+void build_plans(const dart_config& c, const dart_weights* w, int n_sm, PlanSet& ps) {
+  const int grid = 2 * n_sm;
+  const int h = c.hidden, dq = c.n_q_heads * c.head_dim, dkv = c.n_kv_heads * c.head_dim;
+  const bf16* nul = nullptr;
+  auto W = [&](const void* p) { return w ? static_cast<const bf16*>(p) : nul; };
+  GemmSeg s[3];
+  s[0] = {W(w ? w->w_fc : nullptr), h, 0};
+  make_plan_host(ps.fc, s, 1, c.feat_in, grid, ps.clo[0], ps.chi[0]);
+  s[0] = {W(w ? w->w_q : nullptr), dq, 0};
+  s[1] = {W(w ? w->w_k : nullptr), dkv, 0};
+  s[2] = {W(w ? w->w_v : nullptr), dkv, 0};
+  make_plan_host(ps.qkv, s, 3, 2 * h, grid, ps.clo[1], ps.chi[1]);
+  s[0] = {W(w ? w->w_o : nullptr), h, 0};
+  make_plan_host(ps.o, s, 1, dq, grid, ps.clo[2], ps.chi[2]);
+  s[0] = {W(w ? w->w_gate : nullptr), c.mlp_inter, 0};
+  s[1] = {W(w ? w->w_up : nullptr), c.mlp_inter, 0};
+  make_plan_host(ps.gu, s, 2, h, grid, ps.clo[3], ps.chi[3]);
+  s[0] = {W(w ? w->w_down : nullptr), h, 0};
+  make_plan_host(ps.down, s, 1, c.mlp_inter, grid, ps.clo[4], ps.chi[4]);
+  const int MPmax = padded_tokens(c.max_batch * c.K);
+  const GemmPlan* all[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
+  ps.part_max = 0;
+  for (int i = 0; i < 5; ++i) {
+    const size_t f = part_floats(*all[i], MPmax);
+    if (f > ps.part_max) ps.part_max = f;
+  }
+}
+
+int attn_pairs_capacity(const dart_config& c, int n_sm) { return (2 * n_sm) / c.n_kv_heads + c.max_batch + 2; }
+
+int fail_cuda(dart_handle* h, cudaError_t e) {
+  if (h) h->last_cuda_error = (int)e; else g_init_cuda_error = (int)e;
+  return DART_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* dart_status_string(int status) {
+  switch (status) {
+    case DART_OK: return "DART_OK";
+    case DART_ERR_INVALID_ARG: return "DART_ERR_INVALID_ARG";
+    case DART_ERR_UNSUPPORTED_ARCH: return "DART_ERR_UNSUPPORTED_ARCH";
+    case DART_ERR_CUDA: return "DART_ERR_CUDA";
+    case DART_ERR_CAPACITY: return "DART_ERR_CAPACITY";
+    case DART_ERR_TIMEOUT: return "DART_ERR_TIMEOUT";
+    case DART_ERR_INTERNAL: return "DART_ERR_INTERNAL";
+    default: return "DART_ERR_UNKNOWN";
+  }
+}
+
+size_t dart_workspace_bytes(const dart_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  const int n_sm = 148;  // sized for a B200; dart_draft_init uses the device's own count
+  PlanSet ps;
+  build_plans(*cfg, nullptr, n_sm, ps);
+  return layout_workspace(*cfg, n_sm, ps.part_max, attn_pairs_capacity(*cfg, n_sm), 2 * n_sm, nullptr, nullptr);
+}
+
+int dart_last_cuda_error(const dart_handle* h) { return h ? h->last_cuda_error : g_init_cuda_error; }
+
+int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const dart_ngram_host* ngram, dart_handle** out) {
+  if (out == nullptr) return DART_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_ok(cfg) || weights == nullptr) return DART_ERR_INVALID_ARG;
+  const void* wp[15] = {weights->w_fc, weights->embed, weights->mask_vec, weights->norm_g, weights->norm_e,
+                        weights->w_q, weights->w_k, weights->w_v, weights->w_o, weights->norm_post,
+                        weights->w_gate, weights->w_up, weights->w_down, weights->norm_final, weights->w_lm};
+  for (int i = 0; i < 15; ++i)
+    if (!aligned16(wp[i])) return DART_ERR_INVALID_ARG;
+  if (ngram != nullptr && ngram->n_rows > 0 &&
+      (ngram->order == nullptr || ngram->ctx0 == nullptr || ngram->ctx1 == nullptr || ngram->next == nullptr ||
+       ngram->score == nullptr))
+    return DART_ERR_INVALID_ARG;
+
+  int dev = 0, major = 0, n_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail_cuda(nullptr, e);
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (e != cudaSuccess) return fail_cuda(nullptr, e);
+  if (major != 10) return DART_ERR_UNSUPPORTED_ARCH;
+  e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return fail_cuda(nullptr, e);
+
+  dart_handle* h = new dart_handle();
+  h->cfg = *cfg;
+  h->w = *weights;
+  h->device = dev;
+  h->n_sm = n_sm;
+
+  auto bail = [&](int code) {
+    dart_draft_destroy(h);
+    return code;
+  };
+
+  PlanSet ps;
+  build_plans(*cfg, weights, n_sm, ps);
+  GemmPlan* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
+  for (int i = 0; i < 5; ++i) {
+    int *dlo = nullptr, *dhi = nullptr;
+    const size_t nb = ps.clo[i].size() * sizeof(int);
+    if ((e = cudaMalloc(&dlo, nb)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+    h->owned.push_back(dlo);
+    if ((e = cudaMalloc(&dhi, nb)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+    h->owned.push_back(dhi);
+    if ((e = cudaMemcpy(dlo, ps.clo[i].data(), nb, cudaMemcpyHostToDevice)) != cudaSuccess ||
+        (e = cudaMemcpy(dhi, ps.chi[i].data(), nb, cudaMemcpyHostToDevice)) != cudaSuccess) {
+      g_init_cuda_error = (int)e;
+      return bail(DART_ERR_CUDA);
+    }
+    plans[i]->d_tile_clo = dlo;
+    plans[i]->d_tile_chi = dhi;
+  }
+  h->plan_fc = ps.fc; h->plan_qkv = ps.qkv; h->plan_o = ps.o; h->plan_gu = ps.gu; h->plan_down = ps.down;
+  h->lm_grid = 2 * n_sm;
+  if (h->lm_grid > cfg->vocab / 16) h->lm_grid = cfg->vocab / 16;
+  h->attn_pairs_cap = attn_pairs_capacity(*cfg, n_sm);
+
+  h->ws.bytes = layout_workspace(*cfg, n_sm, ps.part_max, h->attn_pairs_cap, 2 * n_sm, nullptr, nullptr);
+  if ((e = cudaMalloc(&h->ws.base, h->ws.bytes)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+  layout_workspace(*cfg, n_sm, ps.part_max, h->attn_pairs_cap, 2 * n_sm, static_cast<char*>(h->ws.base), &h->ws);
+  if ((e = cudaMemset(h->ws.base, 0, h->ws.bytes)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+
+  // Appendix D's per-level weights: fp64 from the fp32 settings, rounded once to fp32
+  for (int i = 0; i < 8; ++i) {
+    h->wl[i] = (float)pow((double)cfg->logit_decay, (double)i);
+    h->wv[i] = (float)pow((double)(i + 1), -(double)cfg->level_exp);
+  }
+  h->wn = cfg->w_ng;
+  h->miss = (float)log((double)cfg->eps_ng);
+
+  // N-gram rows -> open-addressing table (linear probing, load <= 0.5, first duplicate wins)
+  const long long n_rows = ngram ? ngram->n_rows : 0;
+  if (n_rows > 0) {
+    size_t cap = 16;
+    while (cap < (size_t)(2 * n_rows)) cap <<= 1;
+    if (cap > (1ull << 31)) return bail(DART_ERR_INVALID_ARG);
+    std::vector<NgramSlot> tab(cap);
+    memset(tab.data(), 0, cap * sizeof(NgramSlot));
+    const uint32_t mask = (uint32_t)(cap - 1);
+    uint32_t max_probe = 0;
+    for (long long i = 0; i < n_rows; ++i) {
+      const int ord = ngram->order[i];
+      const int c0 = ngram->ctx0[i], c1 = ngram->ctx1[i], nx = ngram->next[i];
+      if ((ord != 2 && ord != 3) || c1 < 0 || nx < 0 || c1 >= cfg->vocab || nx >= cfg->vocab ||
+          (ord == 3 && (c0 < 0 || c0 >= cfg->vocab)))
+        return bail(DART_ERR_INVALID_ARG);
+      if (ord == 3 && cfg->ngram_order < 3) continue;
+      const unsigned long long key = ngram_key(ord, c0, c1, nx);
+      uint32_t pos = (uint32_t)ngram_hash(key) & mask, d = 0;
+      while (tab[pos].key != 0ull && tab[pos].key != key) { pos = (pos + 1) & mask; ++d; }
+      if (tab[pos].key == key) continue;
+      tab[pos].key = key;
+      tab[pos].score = ngram->score[i];
+      if (d > max_probe) max_probe = d;
+    }
+    if ((e = cudaMalloc(&h->ng_slots, cap * sizeof(NgramSlot))) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+    if ((e = cudaMemcpy(h->ng_slots, tab.data(), cap * sizeof(NgramSlot), cudaMemcpyHostToDevice)) != cudaSuccess) {
+      g_init_cuda_error = (int)e;
+      return bail(DART_ERR_CUDA);
+    }
+    h->ng_mask = mask;
+    h->ng_max_probe = max_probe;
+  }
+
+  if ((e = attention_setup()) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+  if ((e = tree_setup(cfg->topk, cfg->beam, cfg->tree_budget, cfg->K)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+  if ((e = cudaDeviceSynchronize()) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+  *out = h;
+  return DART_OK;
+}
+
+int dart_draft_destroy(dart_handle* h) {
+  if (h == nullptr) return DART_OK;
+  for (int* p : h->owned) cudaFree(p);
+  if (h->ws.base) cudaFree(h->ws.base);
+  if (h->ng_slots) cudaFree(h->ng_slots);
+  delete h;
+  return DART_OK;
+}
+
+int dart_step_launch_count(const dart_handle* h, int batch, int n_fresh) {
+  (void)batch;
+  if (h == nullptr) return 0;
+  // fc, stage, qkv, qkv_finalize, attention, combine, o, res_norm, gate_up gemm, gate_up, down, res_norm, lm, merge, tree
+  return (n_fresh > 0 ? 15 : 14);
+}
+
+int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out* out, void* cuda_stream) {
+  if (h == nullptr || in == nullptr || out == nullptr) return DART_ERR_INVALID_ARG;
+  const dart_config& c = h->cfg;
+  const int B = in->batch, F = in->n_fresh, K = c.K;
+  if (B < 1 || F < 0 || F > K) return DART_ERR_INVALID_ARG;
+  if (B > c.max_batch) return DART_ERR_CAPACITY;
+  if (in->seq_lens == nullptr || in->seq_lens_host == nullptr || !aligned16(in->k_cache) || !aligned16(in->v_cache))
+    return DART_ERR_INVALID_ARG;
+  if (F > 0 && (!aligned16(in->feats) || in->tokens == nullptr)) return DART_ERR_INVALID_ARG;
+  if (out->topk_ids == nullptr || out->topk_slogit == nullptr) return DART_ERR_INVALID_ARG;
+  long long total_keys = 0;
+  for (int b = 0; b < B; ++b) {
+    const int P = in->seq_lens_host[b];
+    if (P < 0) return DART_ERR_INVALID_ARG;
+    if ((long long)P + K > c.max_prefix) return DART_ERR_CAPACITY;
+    total_keys += P + K;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int M = B * K, MP = padded_tokens(M);
+  const int hdim = c.hidden, dq = c.n_q_heads * c.head_dim;
+  Workspace& ws = h->ws;
+  cudaError_t e;
+
+  // S0: feature fusion FC on the fresh rows, then z = [RMSNorm(g); RMSNorm(e)]
+  StageParams sp;
+  memset(&sp, 0, sizeof(sp));
+  if (F > 0) {
+    if ((e = launch_gemm_rows(h->plan_fc, static_cast<const bf16*>(in->feats), nullptr, c.feat_in, B * F, ws.part, st)) != cudaSuccess)
+      return fail_cuda(h, e);
+    sp.fc = make_view(h->plan_fc, ws.part, padded_tokens(B * F));
+  }
+  sp.B = B; sp.K = K; sp.F = F; sp.h = hdim; sp.tokens = in->tokens; sp.vocab = c.vocab;
+  sp.embed = static_cast<const bf16*>(h->w.embed); sp.mask_vec = static_cast<const bf16*>(h->w.mask_vec);
+  sp.norm_g = static_cast<const bf16*>(h->w.norm_g); sp.norm_e = static_cast<const bf16*>(h->w.norm_e);
+  sp.eps = c.rms_eps; sp.res = ws.res; sp.z_hi = ws.z_hi; sp.z_lo = ws.z_lo;
+  if ((e = launch_stage_inputs(sp, st)) != cudaSuccess) return fail_cuda(h, e);
+
+  // S1: QKV projection + RoPE + cache rows
+  if ((e = launch_gemm_rows(h->plan_qkv, ws.z_hi, ws.z_lo, 2 * hdim, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
+  QkvParams qp;
+  qp.qkv = make_view(h->plan_qkv, ws.part, MP);
+  qp.q_tile0 = h->plan_qkv.seg[0].tile0; qp.k_tile0 = h->plan_qkv.seg[1].tile0; qp.v_tile0 = h->plan_qkv.seg[2].tile0;
+  qp.B = B; qp.K = K; qp.Hq = c.n_q_heads; qp.Hkv = c.n_kv_heads; qp.dh = c.head_dim;
+  qp.seq_lens = in->seq_lens; qp.rope_theta = c.rope_theta; qp.q_out = ws.q;
+  qp.k_cache = static_cast<bf16*>(in->k_cache); qp.v_cache = static_cast<bf16*>(in->v_cache); qp.P_cap = c.max_prefix;
+  if ((e = launch_qkv_finalize(qp, st)) != cudaSuccess) return fail_cuda(h, e);
+
+  // S2: split-KV attention over cache rows 0 .. P_b+K-1
+  AttnParams ap;
+  ap.B = B; ap.K = K; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.dh = c.head_dim;
+  ap.seq_lens = in->seq_lens; ap.q = ws.q;
+  ap.k_cache = static_cast<const bf16*>(in->k_cache); ap.v_cache = static_cast<const bf16*>(in->v_cache); ap.P_cap = c.max_prefix;
+  {
+    long long per = (total_keys * c.n_kv_heads + 2 * h->n_sm - 1) / (2 * h->n_sm);
+    long long chunk = ((per + 63) / 64) * 64;
+    if (chunk < 64) chunk = 64;
+    ap.chunk_keys = (int)chunk;
+  }
+  ap.o_part = ws.o_part; ap.ml_part = ws.ml_part; ap.a_hi = ws.a_hi; ap.a_lo = ws.a_lo;
+  {
+    long long pairs = 0;
+    for (int b = 0; b < B; ++b) pairs += (in->seq_lens_host[b] + K + ap.chunk_keys - 1) / ap.chunk_keys;
+    if (pairs > h->attn_pairs_cap) return DART_ERR_INTERNAL;
+  }
+  if ((e = launch_attention(ap, in->seq_lens_host, st)) != cudaSuccess) return fail_cuda(h, e);
+
+  // S3: o_proj + residual + RMSNorm
+  if ((e = launch_gemm_rows(h->plan_o, ws.a_hi, ws.a_lo, dq, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
+  ResNormParams rp;
+  rp.proj = make_view(h->plan_o, ws.part, MP);
+  rp.M = M; rp.h = hdim; rp.gamma = static_cast<const bf16*>(h->w.norm_post); rp.eps = c.rms_eps;
+  rp.res = ws.res; rp.n_hi = ws.n_hi; rp.n_lo = ws.n_lo;
+  if ((e = launch_res_norm(rp, st)) != cudaSuccess) return fail_cuda(h, e);
+
+  // S4: gate/up + SiLU * mul
+  if ((e = launch_gemm_rows(h->plan_gu, ws.n_hi, ws.n_lo, hdim, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
+  GateUpParams gp;
+  gp.gu = make_view(h->plan_gu, ws.part, MP);
+  gp.up_tile0 = h->plan_gu.seg[1].tile0; gp.M = M; gp.I = c.mlp_inter; gp.u_hi = ws.u_hi; gp.u_lo = ws.u_lo;
+  if ((e = launch_gate_up(gp, st)) != cudaSuccess) return fail_cuda(h, e);
+
+  // S5: down + residual + final RMSNorm
+  if ((e = launch_gemm_rows(h->plan_down, ws.u_hi, ws.u_lo, c.mlp_inter, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
+  rp.proj = make_view(h->plan_down, ws.part, MP);
+  rp.gamma = static_cast<const bf16*>(h->w.norm_final);
+  if ((e = launch_res_norm(rp, st)) != cudaSuccess) return fail_cuda(h, e);
+
+  // S6 + S7: LM head with fused log-softmax / top-k, then the merge
+  LmParams lp;
+  lp.W = static_cast<const bf16*>(h->w.w_lm); lp.V = c.vocab; lp.Kd = hdim;
+  lp.x_hi = ws.n_hi; lp.x_lo = ws.n_lo; lp.ldx = hdim; lp.M = M; lp.K = K;
+  lp.topk = c.topk;
+  lp.inv_temp = c.temperature > 0.f ? 1.f / c.temperature : 1.f;
+  lp.gumbel = c.temperature > 0.f ? 1 : 0;
+  lp.seed_lo = (uint32_t)(c.philox_seed & 0xffffffffull); lp.seed_hi = (uint32_t)(c.philox_seed >> 32);
+  lp.step = (uint32_t)(in->step_counter & 0xffffffffull);
+  lp.eps_logit = c.eps_logit;
+  lp.grid = (MP <= 32) ? h->lm_grid : (h->lm_grid + 1) / 2;
+  lp.logits_out = out->logits;
+  lp.part_stats = ws.lm_stats; lp.part_key = ws.lm_key; lp.part_y = ws.lm_y; lp.part_id = ws.lm_id;
+  lp.out_ids = out->topk_ids; lp.out_slogit = out->topk_slogit;
+  if ((e = launch_lm_head(lp, st)) != cudaSuccess) return fail_cuda(h, e);
+  if ((e = launch_topk_merge(lp, st)) != cudaSuccess) return fail_cuda(h, e);
+  return DART_OK;
+}
+
+int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out* out, void* cuda_stream) {
+  if (h == nullptr || in == nullptr || out == nullptr) return DART_ERR_INVALID_ARG;
+  const dart_config& c = h->cfg;
+  if (in->batch < 1 || in->first_row < 0 || in->n_levels < 1 || in->first_row + in->n_levels > c.K) return DART_ERR_INVALID_ARG;
+  if (in->batch > c.max_batch) return DART_ERR_CAPACITY;
+  if (in->topk_ids == nullptr || in->topk_slogit == nullptr || in->ctx_tail == nullptr) return DART_ERR_INVALID_ARG;
+  if (out->tokens == nullptr || out->parents == nullptr || out->depth == nullptr || out->mask == nullptr || out->n_nodes == nullptr)
+    return DART_ERR_INVALID_ARG;
+  if (in->n_levels * (c.tree_budget - 1) > 1024) return DART_ERR_INVALID_ARG;
+  TreeParams tp;
+  tp.B = in->batch; tp.K = c.K; tp.topk = c.topk; tp.beam = c.beam; tp.budget = c.tree_budget;
+  tp.first_row = in->first_row; tp.n_levels = in->n_levels; tp.ngram_order = c.ngram_order;
+  tp.ids = in->topk_ids; tp.slogit = in->topk_slogit; tp.ctx_tail = in->ctx_tail;
+  tp.table.slots = h->ng_slots; tp.table.mask = h->ng_mask; tp.table.max_probe = h->ng_max_probe;
+  for (int i = 0; i < 8; ++i) { tp.wl[i] = h->wl[i]; tp.wv[i] = h->wv[i]; }
+  tp.wn = h->wn; tp.miss = h->miss;
+  tp.tokens = out->tokens; tp.parents = out->parents; tp.depth = out->depth; tp.mask = out->mask;
+  tp.n_nodes = out->n_nodes; tp.scores = out->scores; tp.status = h->ws.status;
+  cudaError_t e = launch_tree(tp, static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return fail_cuda(h, e);
+  return DART_OK;
+}
+
+int dart_last_device_status(dart_handle* h, void* cuda_stream) {
+  if (h == nullptr) return DART_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int v = 0;
+  cudaError_t e = cudaMemcpyAsync(&v, h->ws.status, sizeof(int), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail_cuda(h, e);
+  if (v != 0) {
+    cudaMemsetAsync(h->ws.status, 0, sizeof(int), st);
+    cudaStreamSynchronize(st);
+  }
+  return v == 0 ? DART_OK : DART_ERR_TIMEOUT;
+}
+
+}  // extern "C"

@@ -1,0 +1,125 @@
+"""GPU parity at sizes the oracle finishes in seconds: the tiny reference config and odd
+shapes that span several tiles with ragged tails, every batch-size code path (8, 32, 128
+padded token rows), all fresh-row counts, and temperature > 0.  All calls go through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import parity
+from oracle import forward as ofw
+from oracle import tree as otree
+from paper_2601_19278_b200 import runner, synthetic as syn
+
+pytestmark = pytest.mark.gpu
+
+C1 = syn.WORKLOADS["C1"]
+CASES = {
+    "C1": C1,
+    "C1_two_fresh": syn.small_variant(C1, n_fresh=2),
+    "C1_all_mask": syn.small_variant(C1, n_fresh=0),
+    "ragged_b2": syn.small_variant(C1, batch=2, ragged_lo=40, prefix=200),
+    "b3_k4_pad32": syn.small_variant(C1, batch=3, ragged_lo=1, prefix=90, vocab=2064),
+    "dh128_k8": syn.small_variant(C1, hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, mlp_inter=1376,
+                                  vocab=4112, prefix=333, K=8, tree_budget=60),
+    "gqa5_k8": syn.small_variant(C1, hidden=640, n_q_heads=5, n_kv_heads=1, head_dim=128, mlp_inter=1040,
+                                 vocab=3088, prefix=150, K=8, tree_budget=60, batch=2, ragged_lo=3),
+    "b16_k8_pad128": syn.small_variant(C1, batch=16, K=8, ragged_lo=10, prefix=300, vocab=2048, tree_budget=60),
+    "empty_prefix": syn.small_variant(C1, prefix=0),
+    "hot_b4": syn.small_variant(C1, batch=4, ragged_lo=20, prefix=160, temperature=1.0),
+}
+
+
+def _run(w, want_tree=True, step_counter=5):
+    wt = syn.make_weights(w)
+    inp = syn.make_step_inputs(w)
+    rows = syn.make_ngram_rows(w.vocab, min(w.ngram_rows, 20000), w.ngram_mode)
+    ses = runner.DraftSession(w, wt, rows, want_logits=True, philox_seed=parity.PHILOX_SEED)
+    ses.load_inputs(inp)
+    ses.step(step_counter=step_counter)
+    if want_tree:
+        ses.tree()
+    torch.cuda.synchronize()
+    assert ses.draft.device_status() == 0
+    return wt, inp, rows, ses
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_forward_topk_and_cache_match_oracle(name):
+    w = CASES[name]
+    wt, inp, rows, ses = _run(w, want_tree=False)
+    ref = parity.oracle_forward(w, wt, inp)
+    stats = parity.check_logits(ses.logits.cpu().numpy(), ref["logits"])
+    ids_g, sl_g = ses.topk_ids.cpu().numpy(), ses.topk_slogit.cpu().numpy()
+    k = ses.cfg.topk
+    for b in range(w.batch):
+        for r in range(w.K):
+            noise = ofw.gumbel_noise(w.vocab, r, b, 5, parity.PHILOX_SEED) if w.temperature > 0 else None
+            parity.check_topk_row(ids_g[b, r], sl_g[b, r], ref["logits"][b, r], k, 1e-10, w.temperature, noise)
+    # cache rows P_b .. P_b+F-1 hold the fresh positions' post-RoPE k, v (bf16-rounded); earlier rows untouched
+    kc, vc = ses.inp["k_cache"].float().cpu().numpy(), ses.inp["v_cache"].float().cpu().numpy()
+    k0, v0 = inp["k_cache"].float().numpy(), inp["v_cache"].float().numpy()
+    for b in range(w.batch):
+        P = int(inp["seq_lens"][b])
+        assert np.array_equal(kc[b, :, :P], k0[b, :, :P]) and np.array_equal(vc[b, :, :P], v0[b, :, :P])
+        for r in range(inp["n_fresh"]):
+            np.testing.assert_allclose(kc[b, :, P + r], ref["k_new"][b, r], rtol=1e-2, atol=2e-2)
+            np.testing.assert_allclose(vc[b, :, P + r], ref["v_new"][b, r], rtol=1e-2, atol=2e-2)
+    assert stats["max_abs"] < parity.TOL_ABS
+    ses.close()
+
+
+@pytest.mark.parametrize("name", ["C1", "ragged_b2", "dh128_k8", "b16_k8_pad128", "hot_b4", "C1_two_fresh"])
+def test_tree_from_gpu_candidates_is_bit_exact(name):
+    """The oracle's Algorithm 1 on the GPU's own (ids, s_logit) must give the GPU's tree."""
+    w = CASES[name]
+    wt, inp, rows, ses = _run(w)
+    tri, bi = otree.tables_from_rows(rows)
+    fr = max(inp["n_fresh"], 1) - 1
+    ids, sl = ses.topk_ids.cpu().numpy()[:, fr:], ses.topk_slogit.cpu().numpy()[:, fr:]
+    ref = parity.oracle_tree_batch(ids, sl, inp["ctx_tail"].numpy(), tri, bi, beam=w.beam, budget=w.tree_budget)
+    parity.assert_tree_equal(ses.tree_outputs(), ref)
+    ses.close()
+
+
+def test_planted_ngram_rows_change_the_tree_and_stay_bit_exact():
+    """Random-init logits almost never meet random table rows, so plant rows on the oracle's own
+    top-k ids: the hit path of the lookup is then exercised end to end."""
+    w = C1
+    wt = syn.make_weights(w)
+    inp = syn.make_step_inputs(w)
+    ref = parity.oracle_forward(w, wt, inp)
+    top = [ofw.topk_candidates(ref["logits"][0, r], w.topk, 1e-10)["ids"] for r in range(w.K)]
+    ctx = inp["ctx_tail"].numpy()[0]
+    extra = [[3, int(ctx[0]), int(ctx[1]), int(top[0][5])], [2, -1, int(ctx[1]), int(top[0][7])]]
+    for r in range(1, w.K):
+        extra += [[3, int(top[r - 1][j]), int(top[r - 1][j + 1]), int(top[r][9 - j])] for j in range(4)]
+        extra += [[2, -1, int(top[r - 1][j]), int(top[r][j + 3])] for j in range(6)]
+        if r >= 2:
+            extra += [[3, int(top[r - 2][j]), int(top[r - 1][2 * j]), int(top[r][j + 1])] for j in range(6)]
+    rows = syn.make_ngram_rows(w.vocab, 20000, w.ngram_mode, extra_rows=np.array(extra))
+    tri, bi = otree.tables_from_rows(rows)
+    ses = runner.DraftSession(w, wt, rows, want_logits=False)
+    ses.load_inputs(inp)
+    ses.step()
+    ses.tree()
+    got = ses.tree_outputs()
+    ids, sl = ses.topk_ids.cpu().numpy(), ses.topk_slogit.cpu().numpy()
+    with_table = parity.oracle_tree_batch(ids, sl, inp["ctx_tail"].numpy(), tri, bi, beam=w.beam, budget=w.tree_budget)
+    without = parity.oracle_tree_batch(ids, sl, inp["ctx_tail"].numpy(), {}, {}, beam=w.beam, budget=w.tree_budget)
+    parity.assert_tree_equal(got, with_table)
+    assert not np.array_equal(with_table["tokens"], without["tokens"])
+    ses.close()
+
+
+def test_runs_are_bitwise_repeatable():
+    w = CASES["dh128_k8"]
+    wt, inp, rows, ses = _run(w)
+    a = (ses.logits.clone(), ses.topk_ids.clone(), ses.topk_slogit.clone(), ses.tokens.clone(), ses.mask.clone())
+    for _ in range(5):
+        ses.step(step_counter=5)
+        ses.tree()
+        torch.cuda.synchronize()
+        b = (ses.logits, ses.topk_ids, ses.topk_slogit, ses.tokens, ses.mask)
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+    ses.close()
