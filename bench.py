@@ -1,0 +1,324 @@
+#!/usr/bin/env python
+"""Benchmark of the DART drafting step (dart_draft_step + dart_build_tree) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C3] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: feature FC,
+draft decoder layer, LM head with fused log-softmax/top-k, N-gram tree pruning.  Prints ONE
+JSON line (rank 0).  With N > 1 every rank runs an independent replica of the step on its
+own GPU (the path has no exchange step: "replicas only", weak scaling); the timed region is
+bracketed by barriers and the time is the max over ranks.
+
+--impl reference times the CPU oracle (oracle/) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "draft_steps_per_second"
+UNIT = "steps/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "200",
+                                          "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[1])); smax.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7), ("sw_power_cap", 8)):
+                if len(r) > col and r[col].lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores.  A full fp64 step takes ~12 s at the Qwen3-14B
+    shape, so each timed step is a bounded sample of it: every matrix product of the step is run
+    by the oracle's own `linear` on the first `frac` of that matrix's output rows (inputs are the
+    step's real activations), attention, top-k and the tree run in full.  `value` counts the
+    fraction of a step each sample covers."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import parity
+    from oracle import forward as ofw, tree as otree
+    from paper_2601_19278_b200 import synthetic as syn
+    w = syn.WORKLOADS[args.workload]
+    wt = syn.make_weights(w)
+    inp = syn.make_step_inputs(w)
+    rows = syn.make_ngram_rows(w.vocab, min(w.ngram_rows, 200_000), w.ngram_mode)
+    tri, bi = otree.tables_from_rows(rows)
+    npw, npi = parity.np_weights(wt), parity.np_inputs(inp)
+    cfg = parity.oracle_cfg(w)
+    t0 = time.perf_counter()
+    full = ofw.draft_forward(cfg, npw, npi, keep_intermediates=True)      # untimed: activations + full-step time
+    t_full = time.perf_counter() - t0
+    frac = min(1.0, 120.0 / ((args.steps + args.warmup) * t_full))
+    feats = ofw.bf16_to_f64(npi["feats"])
+    seq = npi["seq_lens"]
+
+    def part(x, name):
+        r = max(16, int(npw[name].shape[0] * frac))
+        return ofw.linear(x, npw[name][:r])
+
+    def one_step():
+        part(feats, "w_fc")
+        for n in ("w_q", "w_k", "w_v"):
+            part(full["z"], n)
+        for b in range(w.batch):
+            P = int(seq[b])
+            k_all = np.concatenate([ofw.bf16_to_f64(npi["k_cache"][b, :, :P]), full["k_new"][b].transpose(1, 0, 2)], axis=1)
+            v_all = np.concatenate([ofw.bf16_to_f64(npi["v_cache"][b, :, :P]), full["v_new"][b].transpose(1, 0, 2)], axis=1)
+            ofw.attention_rows(full["q"][b], k_all, v_all, P)
+        part(full["attn"], "w_o")
+        ofw.silu(part(full["n2"], "w_gate")) * part(full["n2"], "w_up")
+        r = max(16, int(npw["w_down"].shape[0] * frac))
+        ofw.linear(full["u"], npw["w_down"][:r])
+        logits = part(full["n3"], "w_lm")
+        for b in range(w.batch):
+            c = [ofw.topk_candidates(logits[b, rr], w.topk, 1e-10) for rr in range(w.K)]
+            ids = np.stack([x["ids"] for x in c]); sl = np.stack([x["slogit"] for x in c]).astype(np.float32)
+            otree.build_tree(ids, sl, tuple(inp["ctx_tail"].numpy()[b]), tri, bi, beam=w.beam, budget=w.tree_budget)
+
+    for _ in range(args.warmup):
+        one_step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_step()
+    dt = time.perf_counter() - t0
+    value = frac * args.steps / dt
+    cores = torch.get_num_threads()
+    sample = (f"each of the {args.steps} timed steps = {frac:.4f} of a full step of workload {w.name}: every matrix product on the "
+              f"first {frac:.4f} of its output rows, attention/top-k/tree in full; one untimed full fp64 step took {t_full:.1f} s")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / (args.steps * frac), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": w.name},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2601_19278_b200 import runner, synthetic as syn
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = syn.WORKLOADS[args.workload]
+    wt = syn.make_weights(w)
+    inp = syn.make_step_inputs(w)
+    rows = syn.make_ngram_rows(w.vocab, w.ngram_rows, w.ngram_mode)
+    ses = runner.DraftSession(w, wt, rows, device=f"cuda:{local}", want_logits=False)
+    ses.load_inputs(inp)
+    stream = torch.cuda.current_stream()
+    n_launch = ses.draft.launch_count(w.batch, inp["n_fresh"])
+    hbm_peak, peak_kind = _peaks()
+    bytes_step = syn.algorithmic_bytes(w, inp["seq_lens"].numpy())
+    lm_bytes = 2 * w.vocab * w.hidden
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step(i):
+        ses.step(step_counter=i)
+        ses.tree()
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    lm_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in lm_ev:                       # torch creates the CUDA event lazily, on its first record
+        a.record(stream)
+        b.record(stream)
+    torch.cuda.synchronize()
+    ev[0].record(stream)
+    for i in range(args.steps):
+        ses.draft.set_profile_events(6, lm_ev[i][0], lm_ev[i][1])
+        step(args.warmup + i)
+        ev[i + 1].record(stream)
+    barrier()
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    lm_ms = [a.elapsed_time(b) for a, b in lm_ev]
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the C ABI with host buffers: pinned inputs in, tree out, every step
+    host_in = {k: inp[k].contiguous().pin_memory() for k in ("feats", "tokens", "seq_lens", "ctx_tail")}
+    host_out = {k: torch.empty_like(getattr(ses, k), device="cpu").pin_memory() for k in ("tokens", "parents", "depth", "mask", "n_nodes")}
+    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+    def e2e_step(i):
+        for k, t in host_in.items():
+            ses.inp[k].copy_(t, non_blocking=True)
+        step(i)
+        for k, t in host_out.items():
+            t.copy_(getattr(ses, k), non_blocking=True)
+        stream.synchronize()                     # the caller needs the tree before it can verify
+
+    for i in range(args.warmup):
+        e2e_step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        e2e_step(i)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(t[0]), float(t[1])
+    assert ses.draft.device_status() == 0
+
+    if rank == 0:
+        ms_per_step = total_ms / args.steps
+        value = world * args.steps / (total_ms * 1e-3)
+        lm_avg_ms = sum(lm_ms) / len(lm_ms)
+        achieved = lm_bytes / (lm_avg_ms * 1e-3) / 1e9
+        step_gbs = bytes_step / (ms_per_step * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{w.name}: batch {w.batch}, hidden {w.hidden}, {w.n_q_heads}q/{w.n_kv_heads}kv x{w.head_dim}, "
+                                   f"mlp {w.mlp_inter}, vocab {w.vocab}, prefix {w.prefix}, K={w.K}, n_fresh={inp['n_fresh']}, "
+                                   f"topk {w.topk}, beam {w.beam}, budget {w.tree_budget}, ngram_rows {len(rows['next'])}, T={w.temperature}",
+                       "parallelism": "replicas only" if world > 1 else "1 GPU",
+                       "l2": f"inputs larger than L2: {bytes_step / 1e9:.3f} GB of weights+KV streamed per step",
+                       "feature_fc_in_path": inp["n_fresh"] > 0},
+            "latency_us": {"p50": 1e3 * statistics.median(per_step), "min": 1e3 * min(per_step), "max": 1e3 * max(per_step)},
+            "step_bytes": bytes_step, "step_gbs": step_gbs,
+            "step_frac_of_hbm_peak": step_gbs / hbm_peak, "step_frac_of_8tbs": step_gbs / 8000.0,
+            "roofline": {"bound": "hbm", "kernel": "lm_head_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                         "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}", "traffic": args.lm_traffic,
+                         "bytes_per_launch": lm_bytes, "us_per_launch": 1e3 * lm_avg_ms},
+            "e2e": {"value": world * args.steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
+            "gpu_launches": args.steps * n_launch,
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w, wt, inp, rows)
+        print(json.dumps(line))
+    ses.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(w, wt, inp, rows):
+    """The oracle timed on this machine's host cores on one full step of the same workload."""
+    import torch
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import parity
+    from oracle import forward as ofw, tree as otree
+    sub = {k: v[:200_000] for k, v in rows.items()}
+    tri, bi = otree.tables_from_rows(sub)
+    npw, npi = parity.np_weights(wt), parity.np_inputs(inp)
+    t0 = time.perf_counter()
+    ref = ofw.draft_forward(parity.oracle_cfg(w), npw, npi)
+    t1 = time.perf_counter()
+    for b in range(w.batch):
+        c = [ofw.topk_candidates(ref["logits"][b, r], w.topk, 1e-10) for r in range(w.K)]
+        ids = np.stack([x["ids"] for x in c]); sl = np.stack([x["slogit"] for x in c]).astype(np.float32)
+        otree.build_tree(ids, sl, tuple(inp["ctx_tail"].numpy()[b]), tri, bi, beam=w.beam, budget=w.tree_budget)
+    t2 = time.perf_counter()
+    return {"value": 1.0 / (t2 - t0), "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"1 full step of workload {w.name} (N-gram table cut to 200k rows for the dict build)",
+            "forward_s": t1 - t0, "topk_tree_s": t2 - t1}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="C3")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--lm-traffic", type=float, default=None,
+                    help="DRAM bytes per LM-head launch from the committed ncu capture (profiles/), reported as roofline.traffic")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -56,7 +56,7 @@ typedef struct dart_config {
   int32_t mlp_inter;     /* I; multiple of 16 */
   int32_t vocab;         /* V; multiple of 16, < 2^21 */
   int32_t feat_in;       /* width of the concatenated target features (3h); multiple of 16 */
-  int32_t max_batch;     /* sequences per call, <= 64 */
+  int32_t max_batch;     /* sequences per call; <= 32 and max_batch * K <= 128 */
   int32_t max_prefix;    /* P_cap: rows per sequence in the caller's KV cache */
   int32_t K;             /* query rows per sequence = future positions d (Section 3.2); 1..8 */
   int32_t topk;          /* k_i: candidates kept per position, 1..32 (Appendix D: 25) */
@@ -126,9 +126,9 @@ typedef struct dart_step_in {
   const int32_t* seq_lens;      /* DEVICE i32 [B]  P_b: rows already in the cache */
   const int32_t* seq_lens_host; /* HOST   i32 [B]  same values; used for capacity checks and launch sizing */
   void* k_cache;          /* DEVICE bf16 [max_batch, H_kv, max_prefix, d_h], post-RoPE keys */
-  void* v_cache;          /* DEVICE bf16, same layout.  The call writes rows P_b .. P_b+K-1 of both:
-                             rows < P_b+F are the fresh positions' k, v (a valid append; the caller
-                             advances seq_lens), rows >= P_b+F are scratch that the next call overwrites. */
+  void* v_cache;          /* DEVICE bf16, same layout.  The call appends the fresh positions' k, v: it writes
+                             rows P_b .. P_b+F-1 of both caches and nothing else (the <mask> rows' k, v
+                             are transient); the caller advances seq_lens.  Needs P_b + F <= max_prefix. */
   uint64_t step_counter;  /* Philox counter word; change it every call when temperature > 0 */
 } dart_step_in;
 
@@ -182,7 +182,7 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
  * One forward pass of the draft layer and LM head with fused log-softmax/top-k
  * (Section 3.2; Algorithm 1 lines 6-8; Appendix D s_logit).  Asynchronous on `cuda_stream`.
  * Errors: INVALID_ARG (NULL pointers, n_fresh out of range), CAPACITY (batch > max_batch or
- * seq_lens_host[b] + K > max_prefix).
+ * seq_lens_host[b] + n_fresh > max_prefix).
  */
 int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out* out, void* cuda_stream);
 
@@ -212,6 +212,16 @@ size_t dart_workspace_bytes(const dart_config* cfg);
 /* Number of kernels one dart_draft_step / dart_build_tree call enqueues for this batch size
  * (used by benchmarks to report launch counts). */
 int dart_step_launch_count(const dart_handle* h, int batch, int n_fresh);
+
+/*
+ * Measurement aid (the paper has no counterpart): the next dart_draft_step (stages 0..7) or
+ * dart_build_tree (stage 8) records the caller-owned CUDA events `start_event` / `stop_event`
+ * (cudaEvent_t handles) on the stream immediately before and after the kernels of `stage`,
+ * then forgets them.  Stages: 0 feature FC + input staging, 1 QKV + RoPE, 2 attention,
+ * 3 o_proj + norm, 4 gate/up, 5 down + norm, 6 LM-head kernel alone, 7 top-k merge, 8 tree.
+ * Errors: INVALID_ARG.
+ */
+int dart_set_profile_events(dart_handle* h, int stage, void* start_event, void* stop_event);
 
 #ifdef __cplusplus
 }

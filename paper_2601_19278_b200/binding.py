@@ -27,6 +27,7 @@ DART_ERR_INTERNAL = -6
 EXPORTS = [
     "dart_draft_init", "dart_draft_step", "dart_build_tree", "dart_draft_destroy", "dart_last_device_status",
     "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_step_launch_count",
+    "dart_set_profile_events",
 ]
 
 
@@ -105,6 +106,8 @@ def lib() -> C.CDLL:
         L.dart_workspace_bytes.restype = C.c_size_t
         L.dart_step_launch_count.argtypes = [C.c_void_p, C.c_int, C.c_int]
         L.dart_step_launch_count.restype = C.c_int
+        L.dart_set_profile_events.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        L.dart_set_profile_events.restype = C.c_int
         _lib = L
     return _lib
 
@@ -194,6 +197,12 @@ class DartDraft:
 
     def device_status(self, stream=None) -> int:
         return lib().dart_last_device_status(self._h, self._stream(stream))
+
+    def set_profile_events(self, stage: int, start: torch.cuda.Event, stop: torch.cuda.Event) -> None:
+        """dart_set_profile_events: bracket one stage of the next call with two torch CUDA events."""
+        rc = lib().dart_set_profile_events(self._h, stage, start.cuda_event, stop.cuda_event)
+        if rc != DART_OK:
+            raise DartError(rc, "dart_set_profile_events")
 
     def launch_count(self, batch: int, n_fresh: int) -> int:
         return lib().dart_step_launch_count(self._h, batch, n_fresh)

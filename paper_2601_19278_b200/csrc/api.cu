@@ -22,7 +22,8 @@ struct Workspace {
   float* part = nullptr;        // split partials of the current projection
   float* res = nullptr;         // [Mmax, h] residual stream
   bf16 *z_hi = nullptr, *z_lo = nullptr;   // [Mmax, 2h]
-  bf16* q = nullptr;            // [Mmax, Hq*dh]
+  bf16 *q_hi = nullptr, *q_lo = nullptr;   // [Mmax, Hq*dh]
+  bf16 *k_new = nullptr, *v_new = nullptr; // [max_batch, Hkv, 16, dh]
   bf16 *a_hi = nullptr, *a_lo = nullptr;   // [Mmax, Hq*dh]
   bf16 *n_hi = nullptr, *n_lo = nullptr;   // [Mmax, h]
   bf16 *u_hi = nullptr, *u_lo = nullptr;   // [Mmax, I]
@@ -48,6 +49,8 @@ struct dart_handle {
   uint32_t ng_mask = 0, ng_max_probe = 0;
   float wl[8], wv[8], wn, miss;
   std::vector<int*> owned;  // small device arrays (plan tables)
+  int prof_stage = -1;      // measurement aid: stage whose kernels the next call brackets with events
+  cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
 };
 
 namespace {
@@ -66,7 +69,7 @@ bool config_ok(const dart_config* c) {
   if (c->vocab < 16 || c->vocab % 16 != 0 || c->vocab >= (1 << 21) - 1) return false;
   if (c->feat_in < 16 || c->feat_in % 16 != 0) return false;
   if (c->max_batch < 1 || c->max_batch > 32 || c->max_batch * c->K > 128) return false;
-  if (c->max_prefix < c->K) return false;
+  if (c->max_prefix < 1) return false;
   if (c->topk < 1 || c->topk > 32 || c->topk > c->vocab) return false;
   if (c->beam < 1 || c->beam > 32) return false;
   if (c->tree_budget < 2 || c->tree_budget > 64) return false;
@@ -136,7 +139,10 @@ size_t layout_workspace(const dart_config& c, int n_sm, size_t part_max_floats, 
   TAKE(res, float*, Mmax * c.hidden * sizeof(float));
   TAKE(z_hi, bf16*, Mmax * 2 * c.hidden * sizeof(bf16));
   TAKE(z_lo, bf16*, Mmax * 2 * c.hidden * sizeof(bf16));
-  TAKE(q, bf16*, Mmax * dq * sizeof(bf16));
+  TAKE(q_hi, bf16*, Mmax * dq * sizeof(bf16));
+  TAKE(q_lo, bf16*, Mmax * dq * sizeof(bf16));
+  TAKE(k_new, bf16*, (size_t)c.max_batch * c.n_kv_heads * 16 * c.head_dim * sizeof(bf16));
+  TAKE(v_new, bf16*, (size_t)c.max_batch * c.n_kv_heads * 16 * c.head_dim * sizeof(bf16));
   TAKE(a_hi, bf16*, Mmax * dq * sizeof(bf16));
   TAKE(a_lo, bf16*, Mmax * dq * sizeof(bf16));
   TAKE(n_hi, bf16*, Mmax * c.hidden * sizeof(bf16));
@@ -189,7 +195,7 @@ void build_plans(const dart_config& c, const dart_weights* w, int n_sm, PlanSet&
   }
 }
 
-int attn_pairs_capacity(const dart_config& c, int n_sm) { return (2 * n_sm) / c.n_kv_heads + c.max_batch + 2; }
+int attn_pairs_capacity(const dart_config& c, int n_sm) { return (2 * n_sm) / c.n_kv_heads + 2 * c.max_batch + 2; }
 
 int fail_cuda(dart_handle* h, cudaError_t e) {
   if (h) h->last_cuda_error = (int)e; else g_init_cuda_error = (int)e;
@@ -364,18 +370,22 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   for (int b = 0; b < B; ++b) {
     const int P = in->seq_lens_host[b];
     if (P < 0) return DART_ERR_INVALID_ARG;
-    if ((long long)P + K > c.max_prefix) return DART_ERR_CAPACITY;
-    total_keys += P + K;
+    if ((long long)P + F > c.max_prefix) return DART_ERR_CAPACITY;
+    total_keys += P;
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int M = B * K, MP = padded_tokens(M);
   const int hdim = c.hidden, dq = c.n_q_heads * c.head_dim;
   Workspace& ws = h->ws;
   cudaError_t e;
+  auto mark = [&](int stage, bool begin) {
+    if (h->prof_stage == stage) cudaEventRecord(begin ? h->prof_start : h->prof_stop, st);
+  };
 
   // S0: feature fusion FC on the fresh rows, then z = [RMSNorm(g); RMSNorm(e)]
   StageParams sp;
   memset(&sp, 0, sizeof(sp));
+  mark(0, true);
   if (F > 0) {
     if ((e = launch_gemm_rows(h->plan_fc, static_cast<const bf16*>(in->feats), nullptr, c.feat_in, B * F, ws.part, st)) != cudaSuccess)
       return fail_cuda(h, e);
@@ -386,6 +396,8 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   sp.norm_g = static_cast<const bf16*>(h->w.norm_g); sp.norm_e = static_cast<const bf16*>(h->w.norm_e);
   sp.eps = c.rms_eps; sp.res = ws.res; sp.z_hi = ws.z_hi; sp.z_lo = ws.z_lo;
   if ((e = launch_stage_inputs(sp, st)) != cudaSuccess) return fail_cuda(h, e);
+  mark(0, false);
+  mark(1, true);
 
   // S1: QKV projection + RoPE + cache rows
   if ((e = launch_gemm_rows(h->plan_qkv, ws.z_hi, ws.z_lo, 2 * hdim, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
@@ -393,14 +405,17 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   qp.qkv = make_view(h->plan_qkv, ws.part, MP);
   qp.q_tile0 = h->plan_qkv.seg[0].tile0; qp.k_tile0 = h->plan_qkv.seg[1].tile0; qp.v_tile0 = h->plan_qkv.seg[2].tile0;
   qp.B = B; qp.K = K; qp.Hq = c.n_q_heads; qp.Hkv = c.n_kv_heads; qp.dh = c.head_dim;
-  qp.seq_lens = in->seq_lens; qp.rope_theta = c.rope_theta; qp.q_out = ws.q;
+  qp.seq_lens = in->seq_lens; qp.rope_theta = c.rope_theta; qp.F = F;
+  qp.q_hi = ws.q_hi; qp.q_lo = ws.q_lo; qp.k_new = ws.k_new; qp.v_new = ws.v_new;
   qp.k_cache = static_cast<bf16*>(in->k_cache); qp.v_cache = static_cast<bf16*>(in->v_cache); qp.P_cap = c.max_prefix;
   if ((e = launch_qkv_finalize(qp, st)) != cudaSuccess) return fail_cuda(h, e);
+  mark(1, false);
+  mark(2, true);
 
-  // S2: split-KV attention over cache rows 0 .. P_b+K-1
+  // S2: split-KV attention over cache rows 0 .. P_b-1 and the K new rows
   AttnParams ap;
   ap.B = B; ap.K = K; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.dh = c.head_dim;
-  ap.seq_lens = in->seq_lens; ap.q = ws.q;
+  ap.seq_lens = in->seq_lens; ap.q_hi = ws.q_hi; ap.q_lo = ws.q_lo; ap.k_new = ws.k_new; ap.v_new = ws.v_new;
   ap.k_cache = static_cast<const bf16*>(in->k_cache); ap.v_cache = static_cast<const bf16*>(in->v_cache); ap.P_cap = c.max_prefix;
   {
     long long per = (total_keys * c.n_kv_heads + 2 * h->n_sm - 1) / (2 * h->n_sm);
@@ -411,10 +426,12 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ap.o_part = ws.o_part; ap.ml_part = ws.ml_part; ap.a_hi = ws.a_hi; ap.a_lo = ws.a_lo;
   {
     long long pairs = 0;
-    for (int b = 0; b < B; ++b) pairs += (in->seq_lens_host[b] + K + ap.chunk_keys - 1) / ap.chunk_keys;
+    for (int b = 0; b < B; ++b) pairs += (in->seq_lens_host[b] + ap.chunk_keys - 1) / ap.chunk_keys + 1;
     if (pairs > h->attn_pairs_cap) return DART_ERR_INTERNAL;
   }
   if ((e = launch_attention(ap, in->seq_lens_host, st)) != cudaSuccess) return fail_cuda(h, e);
+  mark(2, false);
+  mark(3, true);
 
   // S3: o_proj + residual + RMSNorm
   if ((e = launch_gemm_rows(h->plan_o, ws.a_hi, ws.a_lo, dq, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
@@ -423,6 +440,8 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   rp.M = M; rp.h = hdim; rp.gamma = static_cast<const bf16*>(h->w.norm_post); rp.eps = c.rms_eps;
   rp.res = ws.res; rp.n_hi = ws.n_hi; rp.n_lo = ws.n_lo;
   if ((e = launch_res_norm(rp, st)) != cudaSuccess) return fail_cuda(h, e);
+  mark(3, false);
+  mark(4, true);
 
   // S4: gate/up + SiLU * mul
   if ((e = launch_gemm_rows(h->plan_gu, ws.n_hi, ws.n_lo, hdim, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
@@ -430,12 +449,15 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   gp.gu = make_view(h->plan_gu, ws.part, MP);
   gp.up_tile0 = h->plan_gu.seg[1].tile0; gp.M = M; gp.I = c.mlp_inter; gp.u_hi = ws.u_hi; gp.u_lo = ws.u_lo;
   if ((e = launch_gate_up(gp, st)) != cudaSuccess) return fail_cuda(h, e);
+  mark(4, false);
+  mark(5, true);
 
   // S5: down + residual + final RMSNorm
   if ((e = launch_gemm_rows(h->plan_down, ws.u_hi, ws.u_lo, c.mlp_inter, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   rp.proj = make_view(h->plan_down, ws.part, MP);
   rp.gamma = static_cast<const bf16*>(h->w.norm_final);
   if ((e = launch_res_norm(rp, st)) != cudaSuccess) return fail_cuda(h, e);
+  mark(5, false);
 
   // S6 + S7: LM head with fused log-softmax / top-k, then the merge
   LmParams lp;
@@ -451,8 +473,13 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   lp.logits_out = out->logits;
   lp.part_stats = ws.lm_stats; lp.part_key = ws.lm_key; lp.part_y = ws.lm_y; lp.part_id = ws.lm_id;
   lp.out_ids = out->topk_ids; lp.out_slogit = out->topk_slogit;
+  mark(6, true);
   if ((e = launch_lm_head(lp, st)) != cudaSuccess) return fail_cuda(h, e);
+  mark(6, false);
+  mark(7, true);
   if ((e = launch_topk_merge(lp, st)) != cudaSuccess) return fail_cuda(h, e);
+  mark(7, false);
+  if (h->prof_stage >= 0 && h->prof_stage <= 7) h->prof_stage = -1;
   return DART_OK;
 }
 
@@ -474,8 +501,19 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
   tp.wn = h->wn; tp.miss = h->miss;
   tp.tokens = out->tokens; tp.parents = out->parents; tp.depth = out->depth; tp.mask = out->mask;
   tp.n_nodes = out->n_nodes; tp.scores = out->scores; tp.status = h->ws.status;
-  cudaError_t e = launch_tree(tp, static_cast<cudaStream_t>(cuda_stream));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (h->prof_stage == 8) cudaEventRecord(h->prof_start, st);
+  cudaError_t e = launch_tree(tp, st);
   if (e != cudaSuccess) return fail_cuda(h, e);
+  if (h->prof_stage == 8) { cudaEventRecord(h->prof_stop, st); h->prof_stage = -1; }
+  return DART_OK;
+}
+
+int dart_set_profile_events(dart_handle* h, int stage, void* start_event, void* stop_event) {
+  if (h == nullptr || stage < 0 || stage > 8 || start_event == nullptr || stop_event == nullptr) return DART_ERR_INVALID_ARG;
+  h->prof_stage = stage;
+  h->prof_start = static_cast<cudaEvent_t>(start_event);
+  h->prof_stop = static_cast<cudaEvent_t>(stop_event);
   return DART_OK;
 }
 

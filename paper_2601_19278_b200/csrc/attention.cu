@@ -2,13 +2,21 @@
 // other (Section 3.1: strictly causal over the prefix and inside the masked block;
 // Appendix B: grouped-query heads, post-RoPE keys in the cache).
 //
-// The new rows' k and v have already been written to cache rows P_b .. P_b+K-1, so a query
-// row r simply reads cache positions s <= P_b + r.  One CTA handles one (sequence, KV head,
-// chunk of keys); its (H_q/H_kv)*K query rows (<= 64) form up to four 16-row MMA tiles, one
-// per warp.  KV tiles of 64 keys are staged in shared memory with cp.async (double buffered,
-// XOR-swizzled 16-byte chunks), scores and P*V run on mma.sync with warp-level online
-// softmax, and the per-chunk (max, sum, unnormalised output) partials are merged by
-// attn_combine_kernel, which also emits the bf16 hi/lo activations for o_proj.
+// One CTA handles one (sequence, KV head, chunk of keys); its (H_q/H_kv)*K query rows (<= 64)
+// form up to four 16-row MMA tiles, one per warp.  Cache chunks cover positions [0, P_b), which
+// every query row may read; one extra chunk per sequence holds the step's own K new rows, read
+// causally (row r reads new rows r' <= r).  KV tiles of 64 keys are staged in shared memory
+// with cp.async (double buffered, XOR-swizzled 16-byte chunks); scores and P*V run on
+// mma.sync.m16n8k16 with a warp-level online softmax; the per-chunk (max, sum, unnormalised
+// output) partials are merged by attn_combine_kernel, which also emits the bf16 hi/lo
+// activations for o_proj.
+//
+// Accuracy: the queries, the softmax weights and the new rows' k, v enter the bf16 MMAs as
+// hi + lo pairs (x ~= hi + lo), so only the cache itself is bf16.  The new rows come from a
+// 16-row side tile per (sequence, KV head): rows 0..7 hold the hi parts, rows 8..15 the lo
+// parts, so the same MMA code produces q.k_hi in score columns 0..7 and q.k_lo in columns
+// 8..15 (same thread, same register slot), which are added before the softmax; for P*V the
+// weights of columns 0..7 are duplicated into 8..15 so that P*(v_hi + v_lo) falls out.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -16,7 +24,7 @@ namespace dart {
 
 struct AttnArgs {
   AttnParams p;
-  int chunk_base[33];  // prefix sums of chunks per sequence
+  int chunk_base[33];  // prefix sums of chunks per sequence (cache chunks + 1 new-rows chunk)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -36,9 +44,12 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-  return *reinterpret_cast<uint32_t*>(&v);
+// (a, b) -> packed bf16 hi parts and packed bf16 lo parts
+__device__ __forceinline__ void pack_hi_lo(float a, float b, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(a - __low2float(h), b - __high2float(h));
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
 // byte offset of 16-byte chunk `chunk` of row `row` in a [rows][DH] bf16 tile, XOR-swizzled
@@ -53,30 +64,36 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const AttnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int TILE_BYTES = 64 * DH * 2;
   constexpr int CH = DH / 8;  // 16-byte chunks per row
-  unsigned char* Qs = smem;
-  unsigned char* Ks = smem + TILE_BYTES;
-  unsigned char* Vs = smem + 3 * TILE_BYTES;
+  unsigned char* Qh = smem;
+  unsigned char* Ql = smem + TILE_BYTES;
+  unsigned char* Ks = smem + 2 * TILE_BYTES;
+  unsigned char* Vs = smem + 4 * TILE_BYTES;
 
   const int ci = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int P = p.seq_lens[b];
-  const int n_keys = P + p.K;
-  const int k_begin = ci * p.chunk_keys;
-  if (k_begin >= n_keys) return;
-  const int k_end = min(n_keys, k_begin + p.chunk_keys);
+  const int n_cc = (P + p.chunk_keys - 1) / p.chunk_keys;  // cache chunks of this sequence
+  if (ci > n_cc) return;
+  const bool is_new = ci == n_cc;
+  const int k_begin = is_new ? 0 : ci * p.chunk_keys;
+  const int k_end = is_new ? 16 : min(P, k_begin + p.chunk_keys);
   const int n_tiles = (k_end - k_begin + 63) >> 6;
   const int G = p.Hq / p.Hkv, R = G * p.K;
   const int n_mt = (R + 15) >> 4;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
 
-  const bf16* qsrc = p.q + ((size_t)b * p.Hq + (size_t)hk * G) * p.K * DH;
-  const bf16* kbase = p.k_cache + ((size_t)b * p.Hkv + hk) * p.P_cap * DH;
-  const bf16* vbase = p.v_cache + ((size_t)b * p.Hkv + hk) * p.P_cap * DH;
+  const size_t qoff = ((size_t)b * p.Hq + (size_t)hk * G) * p.K * DH;
+  const bf16* kbase = is_new ? p.k_new + ((size_t)b * p.Hkv + hk) * 16 * DH
+                             : p.k_cache + ((size_t)b * p.Hkv + hk) * p.P_cap * DH;
+  const bf16* vbase = is_new ? p.v_new + ((size_t)b * p.Hkv + hk) * 16 * DH
+                             : p.v_cache + ((size_t)b * p.Hkv + hk) * p.P_cap * DH;
 
-  // Q tile (rows >= R zero-filled)
+  // Q tiles, hi and lo (rows >= R zero-filled)
   for (int i = tid; i < 64 * CH; i += 128) {
     const int row = i / CH, ch = i % CH;
     const bool ok = row < R;
-    cp_async16(smem_u32(Qs + swz<DH>(row, ch)), ok ? (const void*)(qsrc + (size_t)row * DH + ch * 8) : (const void*)qsrc, ok ? 16 : 0);
+    const size_t off = qoff + (ok ? (size_t)row * DH + ch * 8 : 0);
+    cp_async16(smem_u32(Qh + swz<DH>(row, ch)), p.q_hi + off, ok ? 16 : 0);
+    cp_async16(smem_u32(Ql + swz<DH>(row, ch)), p.q_lo + off, ok ? 16 : 0);
   }
   auto load_tile = [&](int ti, int buf) {
     const int k0 = k_begin + ti * 64;
@@ -97,10 +114,9 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const AttnArgs a) {
 #pragma unroll
   for (int n = 0; n < DH / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-  uint32_t qf[DH / 16][4];
   const bool active = warp < n_mt;
   const int rr0 = warp * 16 + g, rr1 = rr0 + 8;
-  const int lim0 = P + (rr0 % p.K), lim1 = P + (rr1 % p.K);  // last visible key position per row
+  const int r0 = rr0 % p.K, r1 = rr1 % p.K;  // position of the row inside its sequence's K-block
 
   for (int ti = 0; ti < n_tiles; ++ti) {
     const int buf = ti & 1;
@@ -109,40 +125,46 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const AttnArgs a) {
     cp_async_wait<1>();
     __syncthreads();
     if (active) {
-      if (ti == 0) {
-#pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks) {
-          const int mi = lane >> 3;
-          ldmatrix_x4(qf[ks], smem_u32(Qs + swz<DH>(warp * 16 + (mi & 1) * 8 + (lane & 7), 2 * ks + (mi >> 1))));
-        }
-      }
       float s[8][4];
 #pragma unroll
       for (int n = 0; n < 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
       const unsigned char* Kt = Ks + buf * TILE_BYTES;
       const unsigned char* Vt = Vs + buf * TILE_BYTES;
+      const int mi = lane >> 3;
 #pragma unroll
       for (int ks = 0; ks < DH / 16; ++ks) {
+        uint32_t qh[4], ql[4];
+        const uint32_t qa = swz<DH>(warp * 16 + (mi & 1) * 8 + (lane & 7), 2 * ks + (mi >> 1));
+        ldmatrix_x4(qh, smem_u32(Qh + qa));
+        ldmatrix_x4(ql, smem_u32(Ql + qa));
 #pragma unroll
         for (int np = 0; np < 4; ++np) {
+          if (is_new && np > 0) break;  // the new-rows tile has 16 rows only
           uint32_t kb[4];
-          const int mi = lane >> 3;
           ldmatrix_x4(kb, smem_u32(Kt + swz<DH>(16 * np + (mi >> 1) * 8 + (lane & 7), 2 * ks + (mi & 1))));
-          mma_bf16_16816(s[2 * np], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], kb[0], kb[1]);
-          mma_bf16_16816(s[2 * np + 1], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], kb[2], kb[3]);
+          mma_bf16_16816(s[2 * np], qh[0], qh[1], qh[2], qh[3], kb[0], kb[1]);
+          mma_bf16_16816(s[2 * np], ql[0], ql[1], ql[2], ql[3], kb[0], kb[1]);
+          mma_bf16_16816(s[2 * np + 1], qh[0], qh[1], qh[2], qh[3], kb[2], kb[3]);
+          mma_bf16_16816(s[2 * np + 1], ql[0], ql[1], ql[2], ql[3], kb[2], kb[3]);
         }
       }
       // scale, mask, online softmax (rows g and g+8 of this warp's tile)
       const int k0 = k_begin + ti * 64;
       float tmax0 = -INFINITY, tmax1 = -INFINITY;
+      if (is_new) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[0][e] += s[1][e];  // q.k_hi + q.k_lo
+      }
 #pragma unroll
       for (int n = 0; n < 8; ++n) {
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int kk = k0 + n * 8 + 2 * t + e;
-          const bool in = kk < k_end;
-          s[n][e] = (in && kk <= lim0) ? s[n][e] * sl2 : -INFINITY;
-          s[n][2 + e] = (in && kk <= lim1) ? s[n][2 + e] * sl2 : -INFINITY;
+          // cache chunk: every position below P is visible; new chunk: column r' (< K) visible to rows r >= r'
+          const bool v0 = is_new ? (n == 0 && kk < p.K && kk <= r0) : (kk < k_end);
+          const bool v1 = is_new ? (n == 0 && kk < p.K && kk <= r1) : (kk < k_end);
+          s[n][e] = v0 ? s[n][e] * sl2 : -INFINITY;
+          s[n][2 + e] = v1 ? s[n][2 + e] * sl2 : -INFINITY;
           tmax0 = fmaxf(tmax0, s[n][e]);
           tmax1 = fmaxf(tmax1, s[n][2 + e]);
         }
@@ -168,21 +190,30 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const AttnArgs a) {
       }
       l_run[0] = l_run[0] * al0 + sum0;
       l_run[1] = l_run[1] * al1 + sum1;
+      if (is_new) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[1][e] = s[0][e];  // same weights on the v_lo rows
+      }
 #pragma unroll
       for (int n = 0; n < DH / 8; ++n) {
         o[n][0] *= al0; o[n][1] *= al0; o[n][2] *= al1; o[n][3] *= al1;
       }
 #pragma unroll
       for (int kp = 0; kp < 4; ++kp) {
-        const uint32_t a0 = pack_bf16(s[2 * kp][0], s[2 * kp][1]), a1 = pack_bf16(s[2 * kp][2], s[2 * kp][3]);
-        const uint32_t a2 = pack_bf16(s[2 * kp + 1][0], s[2 * kp + 1][1]), a3 = pack_bf16(s[2 * kp + 1][2], s[2 * kp + 1][3]);
+        if (is_new && kp > 0) break;
+        uint32_t ah[4], al[4];
+        pack_hi_lo(s[2 * kp][0], s[2 * kp][1], ah[0], al[0]);
+        pack_hi_lo(s[2 * kp][2], s[2 * kp][3], ah[1], al[1]);
+        pack_hi_lo(s[2 * kp + 1][0], s[2 * kp + 1][1], ah[2], al[2]);
+        pack_hi_lo(s[2 * kp + 1][2], s[2 * kp + 1][3], ah[3], al[3]);
 #pragma unroll
         for (int dp = 0; dp < DH / 16; ++dp) {
           uint32_t vb[4];
-          const int mi = lane >> 3;
           ldmatrix_x4_trans(vb, smem_u32(Vt + swz<DH>(16 * kp + (mi & 1) * 8 + (lane & 7), 2 * dp + (mi >> 1))));
-          mma_bf16_16816(o[2 * dp], a0, a1, a2, a3, vb[0], vb[1]);
-          mma_bf16_16816(o[2 * dp + 1], a0, a1, a2, a3, vb[2], vb[3]);
+          mma_bf16_16816(o[2 * dp], ah[0], ah[1], ah[2], ah[3], vb[0], vb[1]);
+          mma_bf16_16816(o[2 * dp], al[0], al[1], al[2], al[3], vb[0], vb[1]);
+          mma_bf16_16816(o[2 * dp + 1], ah[0], ah[1], ah[2], ah[3], vb[2], vb[3]);
+          mma_bf16_16816(o[2 * dp + 1], al[0], al[1], al[2], al[3], vb[2], vb[3]);
         }
       }
     }
@@ -240,7 +271,7 @@ __global__ void attn_combine_kernel(const AttnArgs a) {
 }
 
 cudaError_t attention_setup() {
-  return cudaFuncSetAttribute(attn_splitkv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 5 * 64 * 128 * 2);
+  return cudaFuncSetAttribute(attn_splitkv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 6 * 64 * 128 * 2);
 }
 
 cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, cudaStream_t st) {
@@ -249,16 +280,16 @@ cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, cuda
   int base = 0, max_chunks = 0;
   for (int b = 0; b < p.B; ++b) {
     a.chunk_base[b] = base;
-    const int n = (seq_lens_host[b] + p.K + p.chunk_keys - 1) / p.chunk_keys;
+    const int n = (seq_lens_host[b] + p.chunk_keys - 1) / p.chunk_keys + 1;  // cache chunks + the new-rows chunk
     base += n;
     if (n > max_chunks) max_chunks = n;
   }
   a.chunk_base[p.B] = base;
   dim3 grid(max_chunks, p.Hkv, p.B);
   if (p.dh == 128)
-    attn_splitkv_kernel<128><<<grid, 128, 5 * 64 * 128 * 2, st>>>(a);
+    attn_splitkv_kernel<128><<<grid, 128, 6 * 64 * 128 * 2, st>>>(a);
   else
-    attn_splitkv_kernel<64><<<grid, 128, 5 * 64 * 64 * 2, st>>>(a);
+    attn_splitkv_kernel<64><<<grid, 128, 6 * 64 * 64 * 2, st>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   dim3 cgrid(p.B * p.K, p.Hq);

@@ -1,7 +1,8 @@
 // Finalize kernels: sum the split partials of a projection in a fixed order and apply the
 // element-wise / row-wise op that follows it in the draft layer (Section 3.2):
 //   stage_inputs : z = [RMSNorm(g) ; RMSNorm(e)], residual = g     (g = FC(features) or <mask>)
-//   qkv_finalize : RoPE on q, k at position P_b + r; write q, and k, v into the cache rows
+//   qkv_finalize : RoPE on q, k at position P_b + r; write q and the new rows' k, v as hi/lo pairs,
+//                  append the fresh rows' k, v to the cache
 //   res_norm     : x = residual + proj ; n = RMSNorm(x)             (after o_proj and after down)
 //   gate_up      : u = SiLU(gate) * up
 // Outputs that feed the next projection are written as bf16 hi + lo pairs.
@@ -73,15 +74,23 @@ __global__ void qkv_finalize_kernel(const QkvParams p) {
     o1 = (float)((double)x1 * cs - (double)x2 * sn);
     o2 = (float)((double)x2 * cs + (double)x1 * sn);
   }
+  bf16 h1, l1, h2, l2;
+  split_bf16(o1, h1, l1);
+  split_bf16(o2, h2, l2);
   if (kind == 0) {
-    bf16* dst = p.q_out + (((size_t)b * p.Hq + hs) * p.K + r) * dh;
-    dst[i] = __float2bfloat16_rn(o1);
-    dst[i + half] = __float2bfloat16_rn(o2);
+    const size_t o = (((size_t)b * p.Hq + hs) * p.K + r) * dh;
+    p.q_hi[o + i] = h1; p.q_hi[o + i + half] = h2;
+    p.q_lo[o + i] = l1; p.q_lo[o + i + half] = l2;
   } else {
     const int hk = (kind == 1) ? hs - p.Hq : hs - p.Hq - p.Hkv;
-    bf16* dst = (kind == 1 ? p.k_cache : p.v_cache) + (((size_t)b * p.Hkv + hk) * p.P_cap + pos) * dh;
-    dst[i] = __float2bfloat16_rn(o1);
-    dst[i + half] = __float2bfloat16_rn(o2);
+    bf16* side = (kind == 1 ? p.k_new : p.v_new) + ((size_t)b * p.Hkv + hk) * 16 * dh;
+    side[(size_t)r * dh + i] = h1; side[(size_t)r * dh + i + half] = h2;
+    side[(size_t)(8 + r) * dh + i] = l1; side[(size_t)(8 + r) * dh + i + half] = l2;
+    if (r < p.F) {  // a fresh position: its k, v become part of the prefix cache
+      bf16* dst = (kind == 1 ? p.k_cache : p.v_cache) + (((size_t)b * p.Hkv + hk) * p.P_cap + pos) * dh;
+      dst[i] = h1;
+      dst[i + half] = h2;
+    }
   }
 }
 

@@ -79,8 +79,10 @@ struct QkvParams {  // S1 epilogue: RoPE + cache write
   int B, K, Hq, Hkv, dh;
   const int32_t* seq_lens;
   float rope_theta;
-  bf16* q_out;       // [B, Hq, K, dh]
-  bf16* k_cache; bf16* v_cache;  // [*, Hkv, P_cap, dh]; rows P_b + r written
+  int F;             // rows r < F are fresh: their k, v are appended to the cache at P_b + r
+  bf16* q_hi; bf16* q_lo;        // [B, Hq, K, dh] post-RoPE queries as hi + lo
+  bf16* k_new; bf16* v_new;      // [B, Hkv, 16, dh]: rows 0..7 hi parts of the K new rows, rows 8..15 lo parts
+  bf16* k_cache; bf16* v_cache;  // [*, Hkv, P_cap, dh]
   long long P_cap;
 };
 cudaError_t launch_qkv_finalize(const QkvParams& p, cudaStream_t st);
@@ -103,12 +105,13 @@ struct GateUpParams {  // u = SiLU(gate) * up
 cudaError_t launch_gate_up(const GateUpParams& p, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
-// Split-KV grouped-query attention over the cache (rows 0 .. P_b+K-1) + combine.
+// Split-KV grouped-query attention over the cache (rows 0 .. P_b-1) and the step's new rows + combine.
 // ---------------------------------------------------------------------------------------------
 struct AttnParams {
   int B, K, Hq, Hkv, dh;
   const int32_t* seq_lens;
-  const bf16* q;        // [B,Hq,K,dh]
+  const bf16* q_hi; const bf16* q_lo;      // [B,Hq,K,dh]
+  const bf16* k_new; const bf16* v_new;    // [B,Hkv,16,dh] hi rows 0..7, lo rows 8..15
   const bf16* k_cache; const bf16* v_cache; long long P_cap;
   int chunk_keys;       // keys per CTA (multiple of 64)
   float* o_part;        // [sum_b chunks_b, Hkv, 64, dh]

@@ -6,13 +6,14 @@ N-gram rows) with the shapes and distributions of the paper's Qwen3 workloads
 arithmetic: both the CUDA library and the CPU oracle consume the arrays it
 returns, and neither is imported here.
 
-Tensor #n is drawn from ``torch.Generator().manual_seed(seed + n)`` so that a
-single tensor can be regenerated without the others.
+Tensor #n derives its generator seeds from ``seed + n`` so that a single tensor can be
+regenerated without the others (large tensors use one generator per 2^24-element chunk).
 """
 from __future__ import annotations
 
 import dataclasses
 import math
+import os
 from typing import Dict, Optional
 
 import numpy as np
@@ -82,18 +83,35 @@ def _gen(seed: int, name: str) -> torch.Generator:
     return g
 
 
-def _randn_bf16(shape, gen, scale=1.0, shift=0.0, chunk=1 << 26) -> torch.Tensor:
-    """N(shift, scale^2) rounded to bf16 (round-to-nearest-even), drawn in chunks."""
+def _randn_bf16(shape, gen, scale=1.0, shift=0.0, chunk=1 << 24) -> torch.Tensor:
+    """N(shift, scale^2) rounded to bf16 (round-to-nearest-even).
+
+    Large tensors are drawn in chunks of 2^24 elements, chunk c from its own generator seeded
+    with ``gen.initial_seed() + 7919 * (c + 1)``, so that the chunks can be drawn by a few
+    threads at once; the result does not depend on the number of threads.
+    """
     n = int(np.prod(shape))
     out = torch.empty(n, dtype=torch.bfloat16)
-    for s in range(0, n, chunk):
-        e = min(n, s + chunk)
-        t = torch.randn(e - s, generator=gen, dtype=torch.float32)
+    base = gen.initial_seed()
+
+    def draw(c: int) -> None:
+        s, e = c * chunk, min(n, (c + 1) * chunk)
+        g = torch.Generator(device="cpu")
+        g.manual_seed(base + 7919 * (c + 1))
+        t = torch.randn(e - s, generator=g, dtype=torch.float32)
         if scale != 1.0:
             t.mul_(scale)
         if shift != 0.0:
             t.add_(shift)
         out[s:e] = t.to(torch.bfloat16)
+
+    n_chunks = (n + chunk - 1) // chunk
+    if n_chunks <= 1:
+        draw(0) if n else None
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+            list(ex.map(draw, range(n_chunks)))
     return out.view(*shape)
 
 
@@ -154,11 +172,10 @@ def make_step_inputs(w: Workload, seed: int = BASE_SEED, n_fresh: Optional[int] 
     P_cap = w.max_prefix
     k_cache = torch.zeros(B, w.n_kv_heads, P_cap, w.head_dim, dtype=torch.bfloat16)
     v_cache = torch.zeros_like(k_cache)
-    gk, gv = _gen(seed, "k_cache"), _gen(seed, "v_cache")
     for b in range(B):
         P = int(seq_lens[b])
-        k_cache[b, :, :P] = _randn_bf16((w.n_kv_heads, P, w.head_dim), gk)
-        v_cache[b, :, :P] = _randn_bf16((w.n_kv_heads, P, w.head_dim), gv)
+        k_cache[b, :, :P] = _randn_bf16((w.n_kv_heads, P, w.head_dim), _gen(seed + 100 * b, "k_cache"))
+        v_cache[b, :, :P] = _randn_bf16((w.n_kv_heads, P, w.head_dim), _gen(seed + 100 * b, "v_cache"))
     ctx_first = zipf.draw(B, _gen(seed, "ctx_tail"))
     ctx_tail = np.empty((B, 2), dtype=np.int32)
     ctx_tail[:, 0] = ctx_first
