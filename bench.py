@@ -169,6 +169,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     w = syn.WORKLOADS[args.workload]
+    if args.vocab:
+        w = syn.small_variant(w, vocab=args.vocab, name=f"{w.name} with vocab cut to {args.vocab}")
     wt = syn.make_weights(w)
     inp = syn.make_step_inputs(w)
     rows = syn.make_ngram_rows(w.vocab, w.ngram_rows, w.ngram_mode)
@@ -309,6 +311,8 @@ def main():
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--vocab", type=int, default=0,
+                    help="override the workload's vocabulary (a smaller case of the same kernels, for ncu captures)")
     ap.add_argument("--lm-traffic", type=float, default=None,
                     help="DRAM bytes per LM-head launch from the committed ncu capture (profiles/), reported as roofline.traffic")
     args = ap.parse_args()

@@ -27,6 +27,18 @@ __device__ __forceinline__ uint4 ld_act16(const void* p) {
   return v;
 }
 
+// Element offsets, inside a 64-wide k-step, of the two 16-byte chunks that lane t (= lane & 3)
+// of a quad loads from a weight row (and, identically, from an activation row).  Mode 0: the
+// quad's four lanes take bytes [32t, 32t+16) in one instruction and [32t+16, 32t+32) in the next,
+// so each instruction touches all four 32-byte sectors of the row's 128-byte line; mode 1: one
+// instruction covers bytes [0,64) contiguously, the next [64,128).  Mode 0 measured faster on
+// B200 (the memory system sees whole-line requests).
+#ifndef DART_CHUNK_MODE
+#define DART_CHUNK_MODE 0
+#endif
+__device__ __forceinline__ int chunk_k0(int t) { return DART_CHUNK_MODE == 0 ? t * 16 : t * 8; }
+__device__ __forceinline__ int chunk_k1(int t) { return DART_CHUNK_MODE == 0 ? t * 16 + 8 : t * 8 + 32; }
+
 // D(16x8,f32) += A(16x16,bf16,row) * B(16x8,bf16,col)
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {

@@ -6,8 +6,9 @@
 //   * weights are the MMA's M-side operand (16 weight rows x 16 k per mma.sync.m16n8k16),
 //     token rows are the 8-wide N side, so M = 8 tokens is an exact fit;
 //   * weight fragments go global -> registers with 128-bit coalesced loads, each quad reading
-//     one full 128-byte line of a weight row per k-step; the k index is permuted identically
-//     on both operands so that a thread's 32 contiguous bytes are exactly its fragment slots;
+//     64 contiguous bytes (two whole sectors) of a weight row per instruction and one full
+//     128-byte line per k-step; the k index is permuted identically on both operands so that
+//     the 2 x 16 bytes a thread loads are exactly its fragment slots;
 //   * activations (a few hundred KB, bf16 hi + lo) are read through L1 by every warp;
 //   * the flattened (128-row tile, k-step) space is cut into gridDim.x equal ranges, so every
 //     CTA streams the same number of bytes (no tail wave); per-tile partials are summed in CTA
@@ -52,7 +53,9 @@ struct RowCursor {
   }
 };
 
-template <int NT, bool HAS_LO, int PF>
+// FULL: Kd is a multiple of 64, every segment's rows a multiple of 128 and all MP token rows are
+// valid, so the streaming loop carries no bounds predicates.
+template <int NT, bool HAS_LO, int PF, bool FULL>
 __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) gemm_rows_kernel(const GemmRowsArgs p) {
   constexpr int MP = 8 * NT;
   const int c = blockIdx.x, G = gridDim.x;
@@ -73,14 +76,19 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) gemm_rows_kernel(const
   cp.set_tile(p, warp, g);
 
   auto issue = [&](uint4(&dst)[4]) {
-    const int k = ld.ks * 64 + t * 16;
-    if (ld.valid && k < p.Kd) {
-      dst[0] = ld_stream16(ld.r0 + k);
-      dst[1] = ld_stream16(ld.r0 + k + 8);
-      dst[2] = ld_stream16(ld.r1 + k);
-      dst[3] = ld_stream16(ld.r1 + k + 8);
+    const int ka = ld.ks * 64 + chunk_k0(t), kb = ld.ks * 64 + chunk_k1(t);
+    if (FULL) {
+      dst[0] = ld_stream16(ld.r0 + ka);
+      dst[1] = ld_stream16(ld.r0 + kb);
+      dst[2] = ld_stream16(ld.r1 + ka);
+      dst[3] = ld_stream16(ld.r1 + kb);
     } else {
-      dst[0] = dst[1] = dst[2] = dst[3] = make_uint4(0, 0, 0, 0);
+      const bool va = ld.valid && ka < p.Kd, vb = ld.valid && kb < p.Kd;
+      const uint4 z = make_uint4(0, 0, 0, 0);
+      dst[0] = va ? ld_stream16(ld.r0 + ka) : z;
+      dst[1] = vb ? ld_stream16(ld.r0 + kb) : z;
+      dst[2] = va ? ld_stream16(ld.r1 + ka) : z;
+      dst[3] = vb ? ld_stream16(ld.r1 + kb) : z;
     }
     ld.advance(p, warp, g);
   };
@@ -93,22 +101,28 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) gemm_rows_kernel(const
 #pragma unroll
     for (int s = 0; s < PF; ++s) {
       if (u + s < u1) {
-        const int k = cp.ks * 64 + t * 16;
-        const bool kval = k < p.Kd;
+        const int ka = cp.ks * 64 + chunk_k0(t), kb = cp.ks * 64 + chunk_k1(t);
+        const bool kval = ka < p.Kd, kval2 = kb < p.Kd;
         const uint32_t w0[8] = {a[s][0].x, a[s][0].y, a[s][0].z, a[s][0].w, a[s][1].x, a[s][1].y, a[s][1].z, a[s][1].w};
         const uint32_t w1[8] = {a[s][2].x, a[s][2].y, a[s][2].z, a[s][2].w, a[s][3].x, a[s][3].y, a[s][3].z, a[s][3].w};
 #pragma unroll
         for (int n = 0; n < NT; ++n) {
           const int tok = n * 8 + g;
           uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0, l0 = h0, l1 = h0;
-          if (kval && tok < p.M) {
-            const bf16* xp = p.x_hi + (size_t)tok * p.ldx + k;
-            h0 = ld_act16(xp);
-            h1 = ld_act16(xp + 8);
-            if (HAS_LO) {
-              const bf16* xl = p.x_lo + (size_t)tok * p.ldx + k;
-              l0 = ld_act16(xl);
-              l1 = ld_act16(xl + 8);
+          const bf16* xp = p.x_hi + (size_t)tok * p.ldx;
+          const bf16* xq = p.x_lo + (size_t)tok * p.ldx;
+          if (FULL) {
+            h0 = ld_act16(xp + ka);
+            h1 = ld_act16(xp + kb);
+            if (HAS_LO) { l0 = ld_act16(xq + ka); l1 = ld_act16(xq + kb); }
+          } else if (tok < p.M) {
+            if (kval) {
+              h0 = ld_act16(xp + ka);
+              if (HAS_LO) l0 = ld_act16(xq + ka);
+            }
+            if (kval2) {
+              h1 = ld_act16(xp + kb);
+              if (HAS_LO) l1 = ld_act16(xq + kb);
             }
           }
           const uint32_t xh[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
@@ -141,8 +155,11 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) gemm_rows_kernel(const
 }
 
 template <int NT, bool HAS_LO, int PF>
-static cudaError_t launch_t(const GemmRowsArgs& a, int grid, cudaStream_t st) {
-  gemm_rows_kernel<NT, HAS_LO, PF><<<grid, 256, 0, st>>>(a);
+static cudaError_t launch_t(const GemmRowsArgs& a, int grid, bool full, cudaStream_t st) {
+  if (full)
+    gemm_rows_kernel<NT, HAS_LO, PF, true><<<grid, 256, 0, st>>>(a);
+  else
+    gemm_rows_kernel<NT, HAS_LO, PF, false><<<grid, 256, 0, st>>>(a);
   return cudaGetLastError();
 }
 
@@ -155,9 +172,11 @@ cudaError_t launch_gemm_rows(const GemmPlan& plan, const bf16* x_hi, const bf16*
   a.x_hi = x_hi; a.x_lo = x_lo; a.ldx = ldx; a.M = M; a.part = part;
   const int MP = padded_tokens(M);
   const bool lo = x_lo != nullptr;
-  if (MP == 8) return lo ? launch_t<1, true, 4>(a, plan.grid, st) : launch_t<1, false, 4>(a, plan.grid, st);
-  if (MP == 32) return lo ? launch_t<4, true, 2>(a, plan.grid, st) : launch_t<4, false, 2>(a, plan.grid, st);
-  return lo ? launch_t<16, true, 2>(a, plan.grid, st) : launch_t<16, false, 2>(a, plan.grid, st);
+  bool full = (plan.Kd % 64 == 0) && (M == MP);
+  for (int i = 0; i < plan.nseg; ++i) full = full && (plan.seg[i].rows % 128 == 0);
+  if (MP == 8) return lo ? launch_t<1, true, 4>(a, plan.grid, full, st) : launch_t<1, false, 4>(a, plan.grid, full, st);
+  if (MP == 32) return lo ? launch_t<4, true, 2>(a, plan.grid, full, st) : launch_t<4, false, 2>(a, plan.grid, full, st);
+  return lo ? launch_t<16, true, 2>(a, plan.grid, full, st) : launch_t<16, false, 2>(a, plan.grid, full, st);
 }
 
 }  // namespace dart

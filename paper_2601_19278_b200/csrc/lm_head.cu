@@ -39,7 +39,9 @@ __device__ __forceinline__ void list_insert(float& lk, float& ly, int& lid, floa
   else if (lane > pos) { lk = pk; ly = py; lid = pid; }
 }
 
-template <int NT, bool HAS_LO, int PF>
+// FULL: Kd is a multiple of 512 (every warp has the same number of whole k-steps) and all MP
+// token rows are valid, so the streaming loop carries no bounds predicates at all.
+template <int NT, bool HAS_LO, int PF, bool FULL>
 __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) lm_head_kernel(const LmParams p) {
   constexpr int MP = 8 * NT;
   constexpr int RB = (NT <= 4) ? 2 : 1;      // reduce buffers
@@ -72,16 +74,21 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) lm_head_kernel(const L
 
   auto issue = [&](uint4(&dst)[4]) {
     const int ks = warp + 8 * ld.i;
-    const int k = ks * 64 + t * 16;
-    if (ks < SK && k < p.Kd) {
-      const bf16* r0 = p.W + (size_t)(ld.mt * 16 + g) * p.Kd + k;
-      const bf16* r1 = r0 + (size_t)8 * p.Kd;
-      dst[0] = ld_stream16(r0);
-      dst[1] = ld_stream16(r0 + 8);
-      dst[2] = ld_stream16(r1);
-      dst[3] = ld_stream16(r1 + 8);
+    const int ka = ks * 64 + chunk_k0(t), kb = ks * 64 + chunk_k1(t);
+    const bf16* r0 = p.W + (size_t)(ld.mt * 16 + g) * p.Kd;
+    const bf16* r1 = r0 + (size_t)8 * p.Kd;
+    if (FULL) {
+      dst[0] = ld_stream16(r0 + ka);
+      dst[1] = ld_stream16(r0 + kb);
+      dst[2] = ld_stream16(r1 + ka);
+      dst[3] = ld_stream16(r1 + kb);
     } else {
-      dst[0] = dst[1] = dst[2] = dst[3] = make_uint4(0, 0, 0, 0);
+      const bool va = ks < SK && ka < p.Kd, vb = ks < SK && kb < p.Kd;
+      const uint4 z = make_uint4(0, 0, 0, 0);
+      dst[0] = va ? ld_stream16(r0 + ka) : z;
+      dst[1] = vb ? ld_stream16(r0 + kb) : z;
+      dst[2] = va ? ld_stream16(r1 + ka) : z;
+      dst[3] = vb ? ld_stream16(r1 + kb) : z;
     }
     if (++ld.i == spw) { ld.i = 0; ++ld.mt; }
   };
@@ -96,22 +103,28 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) lm_head_kernel(const L
     for (int s = 0; s < PF; ++s) {
       if (u + s < nsteps) {
         const int ks = warp + 8 * cp.i;
-        const int k = ks * 64 + t * 16;
-        const bool kval = (ks < SK) && (k < p.Kd);
+        const int ka = ks * 64 + chunk_k0(t), kb = ks * 64 + chunk_k1(t);
+        const bool kval = (ks < SK) && (ka < p.Kd), kval2 = (ks < SK) && (kb < p.Kd);
         const uint32_t w0[8] = {a[s][0].x, a[s][0].y, a[s][0].z, a[s][0].w, a[s][1].x, a[s][1].y, a[s][1].z, a[s][1].w};
         const uint32_t w1[8] = {a[s][2].x, a[s][2].y, a[s][2].z, a[s][2].w, a[s][3].x, a[s][3].y, a[s][3].z, a[s][3].w};
 #pragma unroll
         for (int n = 0; n < NT; ++n) {
           const int tok = n * 8 + g;
           uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0, l0 = h0, l1 = h0;
-          if (kval && tok < p.M) {
-            const bf16* xp = p.x_hi + (size_t)tok * p.ldx + k;
-            h0 = ld_act16(xp);
-            h1 = ld_act16(xp + 8);
-            if (HAS_LO) {
-              const bf16* xl = p.x_lo + (size_t)tok * p.ldx + k;
-              l0 = ld_act16(xl);
-              l1 = ld_act16(xl + 8);
+          const bf16* xp = p.x_hi + (size_t)tok * p.ldx;
+          const bf16* xq = p.x_lo + (size_t)tok * p.ldx;
+          if (FULL) {
+            h0 = ld_act16(xp + ka);
+            h1 = ld_act16(xp + kb);
+            if (HAS_LO) { l0 = ld_act16(xq + ka); l1 = ld_act16(xq + kb); }
+          } else if (tok < p.M) {
+            if (kval) {
+              h0 = ld_act16(xp + ka);
+              if (HAS_LO) l0 = ld_act16(xq + ka);
+            }
+            if (kval2) {
+              h1 = ld_act16(xp + kb);
+              if (HAS_LO) l1 = ld_act16(xq + kb);
             }
           }
           const uint32_t xh[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
@@ -297,23 +310,24 @@ static size_t lm_smem_bytes() {
   return sizeof(float) * ((size_t)RB * 8 * 16 * MP + (size_t)MP * 129 + 3 * (size_t)MP * 32 + 2 * (size_t)MP);
 }
 
-template <int NT, bool HAS_LO, int PF>
+template <int NT, int PF, bool FULL>
 static cudaError_t launch_lm_t(const LmParams& p, cudaStream_t st) {
   const size_t smem = lm_smem_bytes<NT>();
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(lm_head_kernel<NT, HAS_LO, PF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(lm_head_kernel<NT, true, PF, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  lm_head_kernel<NT, HAS_LO, PF><<<p.grid, 256, smem, st>>>(p);
+  lm_head_kernel<NT, true, PF, FULL><<<p.grid, 256, smem, st>>>(p);
   return cudaGetLastError();
 }
 
 cudaError_t launch_lm_head(const LmParams& p, cudaStream_t st) {
   const int MP = padded_tokens(p.M);
-  const bool lo = p.x_lo != nullptr;
-  if (MP == 8) return lo ? launch_lm_t<1, true, 4>(p, st) : launch_lm_t<1, false, 4>(p, st);
-  if (MP == 32) return lo ? launch_lm_t<4, true, 2>(p, st) : launch_lm_t<4, false, 2>(p, st);
-  return lo ? launch_lm_t<16, true, 2>(p, st) : launch_lm_t<16, false, 2>(p, st);
+  if (p.x_lo == nullptr) return cudaErrorInvalidValue;  // the LM head always takes hi + lo activations
+  const bool full = (p.Kd % 512 == 0) && (p.M == MP);
+  if (MP == 8) return full ? launch_lm_t<1, 4, true>(p, st) : launch_lm_t<1, 4, false>(p, st);
+  if (MP == 32) return full ? launch_lm_t<4, 2, true>(p, st) : launch_lm_t<4, 2, false>(p, st);
+  return full ? launch_lm_t<16, 2, true>(p, st) : launch_lm_t<16, 2, false>(p, st);
 }
 
 cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st) {
