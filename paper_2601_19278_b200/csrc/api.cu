@@ -333,6 +333,7 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
     h->ng_max_probe = max_probe;
   }
 
+  if ((e = topk_merge_setup(2 * n_sm)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
   if ((e = attention_setup()) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
   if ((e = tree_setup(cfg->topk, cfg->beam, cfg->tree_budget, cfg->K)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
   if ((e = cudaDeviceSynchronize()) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }

@@ -136,6 +136,7 @@ struct LmParams {
   int32_t* out_ids; float* out_slogit;  // [M, topk]
 };
 cudaError_t launch_lm_head(const LmParams& p, cudaStream_t st);
+cudaError_t topk_merge_setup(int max_grid);  // once per device
 cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------

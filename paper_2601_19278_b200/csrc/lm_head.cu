@@ -9,7 +9,7 @@
 // through shared memory.  Complete logits never leave the SM: every 128 vocab rows a warp per
 // token row folds them into a running (max, sum-exp) pair and an exact top-32 list held one
 // entry per lane.  The CTA writes (max, sum-exp, list) per token row; topk_merge_kernel
-// combines the CTAs' results and emits the k best ids with s_logit = log(softmax + eps).
+// (topk_merge.cu) combines the CTAs' results and emits the k best ids with s_logit = log(softmax + eps).
 //
 // With temperature > 0 the list is ordered by logit/T + Gumbel noise (Gumbel-top-k = sampling
 // without replacement); the noise of token v in row (b, r) is word v&3 of
@@ -229,81 +229,6 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) lm_head_kernel(const L
   for (int i = tid; i < MP * 2; i += 256) p.part_stats[(size_t)c * MP * 2 + i] = st_ms[i];
 }
 
-// One block per token row: combine the CTAs' (max, sum-exp) pairs and top lists.
-__global__ void __launch_bounds__(256) topk_merge_kernel(const LmParams p) {
-  __shared__ float sh[32];
-  __shared__ float wk[8][32], wy[8][32];
-  __shared__ int wi[8][32];
-  const int tk = blockIdx.x, MP = padded_tokens(p.M), G = p.grid;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  float mx = -INFINITY;
-  for (int c = tid; c < G; c += 256) mx = fmaxf(mx, p.part_stats[((size_t)c * MP + tk) * 2]);
-  mx = warp_max(mx);
-  __syncthreads();
-  if (lane == 0) sh[warp] = mx;
-  __syncthreads();
-  mx = sh[0];
-  for (int i = 1; i < 8; ++i) mx = fmaxf(mx, sh[i]);
-  float sum = 0.f;
-  for (int c = tid; c < G; c += 256) {
-    const float mc = p.part_stats[((size_t)c * MP + tk) * 2];
-    if (mc != -INFINITY) sum += p.part_stats[((size_t)c * MP + tk) * 2 + 1] * expf(mc - mx);
-  }
-  sum = block_sum(sum, sh);
-  const float lse = mx + logf(sum);
-
-  // each warp scans a strided slice of the G*32 candidates
-  float lk = -INFINITY, ly = 0.f;
-  int lid = 0x7fffffff;
-  float thr_k = -INFINITY;
-  int thr_id = 0x7fffffff;
-  const int total = G * 32;
-  for (int base = warp * 32; base < total; base += 256) {
-    const int idx = base + lane;
-    const int c = idx >> 5, e = idx & 31;
-    const size_t o = ((size_t)c * MP + tk) * 32 + e;
-    const bool ok = idx < total && e < p.topk;
-    const float ck = ok ? p.part_key[o] : -INFINITY, cy = ok ? p.part_y[o] : 0.f;
-    const int cid = ok ? p.part_id[o] : 0x7fffffff;
-    auto better = [&](float k, int id) { return k > thr_k || (k == thr_k && id < thr_id); };
-    unsigned mask = __ballot_sync(0xffffffffu, ok && ck > -INFINITY && better(ck, cid));
-    while (mask) {
-      const int src = __ffs(mask) - 1;
-      list_insert(lk, ly, lid, __shfl_sync(0xffffffffu, ck, src), __shfl_sync(0xffffffffu, cy, src),
-                  __shfl_sync(0xffffffffu, cid, src), lane);
-      thr_k = __shfl_sync(0xffffffffu, lk, p.topk - 1);
-      thr_id = __shfl_sync(0xffffffffu, lid, p.topk - 1);
-      mask &= mask - 1;
-      mask &= __ballot_sync(0xffffffffu, ok && ck > -INFINITY && better(ck, cid));
-    }
-  }
-  wk[warp][lane] = lk; wy[warp][lane] = ly; wi[warp][lane] = lid;
-  __syncthreads();
-  if (warp == 0) {
-    for (int w = 1; w < 8; ++w) {
-      const float ck = wk[w][lane], cy = wy[w][lane];
-      const int cid = wi[w][lane];
-      const bool ok = lane < p.topk && ck > -INFINITY;
-      auto better = [&](float k, int id) { return k > thr_k || (k == thr_k && id < thr_id); };
-      unsigned mask = __ballot_sync(0xffffffffu, ok && better(ck, cid));
-      while (mask) {
-        const int src = __ffs(mask) - 1;
-        list_insert(lk, ly, lid, __shfl_sync(0xffffffffu, ck, src), __shfl_sync(0xffffffffu, cy, src),
-                    __shfl_sync(0xffffffffu, cid, src), lane);
-        thr_k = __shfl_sync(0xffffffffu, lk, p.topk - 1);
-        thr_id = __shfl_sync(0xffffffffu, lid, p.topk - 1);
-        mask &= mask - 1;
-        mask &= __ballot_sync(0xffffffffu, ok && better(ck, cid));
-      }
-    }
-    if (lane < p.topk) {
-      const bool have = lk > -INFINITY;
-      p.out_ids[(size_t)tk * p.topk + lane] = have ? lid : -1;
-      p.out_slogit[(size_t)tk * p.topk + lane] = have ? logf(expf(ly - lse) + p.eps_logit) : -INFINITY;
-    }
-  }
-}
-
 template <int NT>
 static size_t lm_smem_bytes() {
   constexpr int MP = 8 * NT, RB = (NT <= 4) ? 2 : 1;
@@ -328,11 +253,6 @@ cudaError_t launch_lm_head(const LmParams& p, cudaStream_t st) {
   if (MP == 8) return full ? launch_lm_t<1, 4, true>(p, st) : launch_lm_t<1, 4, false>(p, st);
   if (MP == 32) return full ? launch_lm_t<4, 2, true>(p, st) : launch_lm_t<4, 2, false>(p, st);
   return full ? launch_lm_t<16, 2, true>(p, st) : launch_lm_t<16, 2, false>(p, st);
-}
-
-cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st) {
-  topk_merge_kernel<<<p.M, 256, 0, st>>>(p);
-  return cudaGetLastError();
 }
 
 }  // namespace dart
