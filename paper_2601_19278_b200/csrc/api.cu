@@ -20,13 +20,16 @@ struct Workspace {
   void* base = nullptr;
   size_t bytes = 0;
   float* part = nullptr;        // split partials of the current projection
-  float* res = nullptr;         // [Mmax, h] residual stream
-  bf16 *z_hi = nullptr, *z_lo = nullptr;   // [Mmax, 2h]
+  float* res0 = nullptr;        // [max_batch*K, h]  g of the fresh rows (first residual)
+  float* x1 = nullptr;          // [Mmax, h] residual stream after attention
+  bf16 *z_hi = nullptr, *z_lo = nullptr;   // [Mmax + 1, 2h]: fresh rows' z, last row = the <mask> row
   bf16 *q_hi = nullptr, *q_lo = nullptr;   // [Mmax, Hq*dh]
   bf16 *k_new = nullptr, *v_new = nullptr; // [max_batch, Hkv, 16, dh]
   bf16 *a_hi = nullptr, *a_lo = nullptr;   // [Mmax, Hq*dh]
-  bf16 *n_hi = nullptr, *n_lo = nullptr;   // [Mmax, h]
+  bf16 *n_hi = nullptr, *n_lo = nullptr;   // [Mmax, h]  gain-scaled residual (not yet divided by its rms)
   bf16 *u_hi = nullptr, *u_lo = nullptr;   // [Mmax, I]
+  float *ss_g = nullptr, *ss_1 = nullptr, *ss_2 = nullptr;  // [h/128 tiles][MP] sums of squares per tile
+  float* rstd_mask = nullptr;
   float *o_part = nullptr, *ml_part = nullptr;
   float *lm_stats = nullptr, *lm_key = nullptr, *lm_y = nullptr;
   int32_t* lm_id = nullptr;
@@ -44,12 +47,13 @@ struct dart_handle {
   GemmPlan plan_fc, plan_qkv, plan_o, plan_gu, plan_down;
   int lm_grid = 0;
   int attn_pairs_cap = 0;  // capacity of the attention partial buffers in (sequence, chunk) pairs
+  int h_tiles = 0;         // 128-row tiles of a hidden-sized row
   Workspace ws;
   NgramSlot* ng_slots = nullptr;
   uint32_t ng_mask = 0, ng_max_probe = 0;
   float wl[8], wv[8], wn, miss;
-  std::vector<int*> owned;  // small device arrays (plan tables)
-  int prof_stage = -1;      // measurement aid: stage whose kernels the next call brackets with events
+  std::vector<void*> owned;  // small device arrays (plan tables, counters)
+  int prof_stage = -1;       // measurement aid: stage whose kernels the next call brackets with events
   cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
 };
 
@@ -79,12 +83,18 @@ bool config_ok(const dart_config* c) {
   return true;
 }
 
+struct PlanHost {
+  GemmPlan plan;
+  std::vector<int> clo, chi, first, expected;
+};
+
 // Cut the flattened (tile, k-step) space of a projection into `grid_target` equal ranges.
-void make_plan_host(GemmPlan& p, const GemmSeg* segs, int nseg, int Kd, int grid_target, std::vector<int>& clo,
-                    std::vector<int>& chi) {
+void make_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int grid_target, int pair_offset) {
+  GemmPlan& p = ph.plan;
+  memset(&p, 0, sizeof(p));
   p.nseg = nseg;
   int tiles = 0;
-  for (int i = 0; i < 3; ++i) {
+  for (int i = 0; i < 6; ++i) {
     if (i < nseg) {
       p.seg[i] = segs[i];
       p.seg[i].tile0 = tiles;
@@ -98,19 +108,25 @@ void make_plan_host(GemmPlan& p, const GemmSeg* segs, int nseg, int Kd, int grid
   p.n_tiles = tiles;
   p.U = (long long)tiles * p.SK;
   p.grid = (int)((long long)grid_target < p.U ? grid_target : p.U);
-  clo.assign(tiles, 0x7fffffff);
-  chi.assign(tiles, -1);
+  p.pair_offset = pair_offset;
+  p.n_groups = pair_offset > 0 ? pair_offset : tiles;
+  ph.clo.assign(tiles, 0x7fffffff);
+  ph.chi.assign(tiles, -1);
+  ph.first.assign(p.grid, 0);
   p.slots = 1;
   for (int c = 0; c < p.grid; ++c) {
     const long long u0 = ((long long)c * p.U) / p.grid, u1 = ((long long)(c + 1) * p.U) / p.grid;
     if (u0 >= u1) continue;
     const int t0 = (int)(u0 / p.SK), t1 = (int)((u1 - 1) / p.SK);
+    ph.first[c] = t0;
     if (t1 - t0 + 1 > p.slots) p.slots = t1 - t0 + 1;
     for (int t = t0; t <= t1; ++t) {
-      if (c < clo[t]) clo[t] = c;
-      if (c > chi[t]) chi[t] = c;
+      if (c < ph.clo[t]) ph.clo[t] = c;
+      if (c > ph.chi[t]) ph.chi[t] = c;
     }
   }
+  ph.expected.assign(p.n_groups, 0);
+  for (int t = 0; t < tiles; ++t) ph.expected[pair_offset > 0 ? t % pair_offset : t] += ph.chi[t] - ph.clo[t] + 1;
 }
 
 size_t part_floats(const GemmPlan& p, int MP) { return (size_t)p.grid * p.slots * 128 * MP; }
@@ -125,20 +141,21 @@ struct Layout {
 };
 
 // Sizes every workspace region; with base != nullptr also assigns the pointers.
-size_t layout_workspace(const dart_config& c, int n_sm, size_t part_max_floats, int attn_pairs_cap, int lm_grid,
-                        char* base, Workspace* ws) {
+size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_pairs_cap, int lm_grid, char* base, Workspace* ws) {
   Layout L;
   const size_t Mmax = (size_t)c.max_batch * c.K;
   const size_t MPmax = padded_tokens((int)Mmax);
   const size_t dq = (size_t)c.n_q_heads * c.head_dim;
+  const size_t ht = (c.hidden + 127) / 128;
   size_t o;
 #define TAKE(field, type, bytes) \
   o = L.take(bytes);             \
   if (base) ws->field = reinterpret_cast<type>(base + o);
   TAKE(part, float*, part_max_floats * sizeof(float));
-  TAKE(res, float*, Mmax * c.hidden * sizeof(float));
-  TAKE(z_hi, bf16*, Mmax * 2 * c.hidden * sizeof(bf16));
-  TAKE(z_lo, bf16*, Mmax * 2 * c.hidden * sizeof(bf16));
+  TAKE(res0, float*, Mmax * c.hidden * sizeof(float));
+  TAKE(x1, float*, Mmax * c.hidden * sizeof(float));
+  TAKE(z_hi, bf16*, (Mmax + 1) * 2 * c.hidden * sizeof(bf16));
+  TAKE(z_lo, bf16*, (Mmax + 1) * 2 * c.hidden * sizeof(bf16));
   TAKE(q_hi, bf16*, Mmax * dq * sizeof(bf16));
   TAKE(q_lo, bf16*, Mmax * dq * sizeof(bf16));
   TAKE(k_new, bf16*, (size_t)c.max_batch * c.n_kv_heads * 16 * c.head_dim * sizeof(bf16));
@@ -149,6 +166,10 @@ size_t layout_workspace(const dart_config& c, int n_sm, size_t part_max_floats, 
   TAKE(n_lo, bf16*, Mmax * c.hidden * sizeof(bf16));
   TAKE(u_hi, bf16*, Mmax * c.mlp_inter * sizeof(bf16));
   TAKE(u_lo, bf16*, Mmax * c.mlp_inter * sizeof(bf16));
+  TAKE(ss_g, float*, ht * MPmax * sizeof(float));
+  TAKE(ss_1, float*, ht * MPmax * sizeof(float));
+  TAKE(ss_2, float*, ht * MPmax * sizeof(float));
+  TAKE(rstd_mask, float*, 256);
   TAKE(o_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * c.head_dim * sizeof(float));
   TAKE(ml_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * 2 * sizeof(float));
   TAKE(lm_stats, float*, (size_t)lm_grid * MPmax * 2 * sizeof(float));
@@ -157,40 +178,43 @@ size_t layout_workspace(const dart_config& c, int n_sm, size_t part_max_floats, 
   TAKE(lm_id, int32_t*, (size_t)lm_grid * MPmax * 32 * sizeof(int32_t));
   TAKE(status, int*, 256);
 #undef TAKE
-  (void)n_sm;
   return L.total;
 }
 
 struct PlanSet {
-  GemmPlan fc, qkv, o, gu, down;
-  std::vector<int> clo[5], chi[5];
+  PlanHost fc, qkv, o, gu, down;
   size_t part_max = 0;
 };
 
 void build_plans(const dart_config& c, const dart_weights* w, int n_sm, PlanSet& ps) {
   const int grid = 2 * n_sm;
   const int h = c.hidden, dq = c.n_q_heads * c.head_dim, dkv = c.n_kv_heads * c.head_dim;
-  const bf16* nul = nullptr;
-  auto W = [&](const void* p) { return w ? static_cast<const bf16*>(p) : nul; };
-  GemmSeg s[3];
-  s[0] = {W(w ? w->w_fc : nullptr), h, 0};
-  make_plan_host(ps.fc, s, 1, c.feat_in, grid, ps.clo[0], ps.chi[0]);
-  s[0] = {W(w ? w->w_q : nullptr), dq, 0};
-  s[1] = {W(w ? w->w_k : nullptr), dkv, 0};
-  s[2] = {W(w ? w->w_v : nullptr), dkv, 0};
-  make_plan_host(ps.qkv, s, 3, 2 * h, grid, ps.clo[1], ps.chi[1]);
-  s[0] = {W(w ? w->w_o : nullptr), h, 0};
-  make_plan_host(ps.o, s, 1, dq, grid, ps.clo[2], ps.chi[2]);
-  s[0] = {W(w ? w->w_gate : nullptr), c.mlp_inter, 0};
-  s[1] = {W(w ? w->w_up : nullptr), c.mlp_inter, 0};
-  make_plan_host(ps.gu, s, 2, h, grid, ps.clo[3], ps.chi[3]);
-  s[0] = {W(w ? w->w_down : nullptr), h, 0};
-  make_plan_host(ps.down, s, 1, c.mlp_inter, grid, ps.clo[4], ps.chi[4]);
+  auto W = [&](const void* p, long long off) { return w ? static_cast<const bf16*>(p) + off : nullptr; };
+  GemmSeg s[6];
+  s[0] = {W(w ? w->w_fc : nullptr, 0), h, 0, c.feat_in, 0};
+  make_plan_host(ps.fc, s, 1, c.feat_in, grid, 0);
+  // QKV reads z = [g-half | e-half] (2h wide); the two halves carry different 1/rms factors, so each
+  // weight matrix is split into its g-half and e-half columns and the halves are finalized in pairs
+  const int qt = (dq + 127) / 128, kt = (dkv + 127) / 128;
+  s[0] = {W(w ? w->w_q : nullptr, 0), dq, 0, 2 * h, 0};
+  s[1] = {W(w ? w->w_k : nullptr, 0), dkv, 0, 2 * h, 0};
+  s[2] = {W(w ? w->w_v : nullptr, 0), dkv, 0, 2 * h, 0};
+  s[3] = {W(w ? w->w_q : nullptr, h), dq, 0, 2 * h, h};
+  s[4] = {W(w ? w->w_k : nullptr, h), dkv, 0, 2 * h, h};
+  s[5] = {W(w ? w->w_v : nullptr, h), dkv, 0, 2 * h, h};
+  make_plan_host(ps.qkv, s, 6, h, grid, qt + 2 * kt);
+  s[0] = {W(w ? w->w_o : nullptr, 0), h, 0, dq, 0};
+  make_plan_host(ps.o, s, 1, dq, grid, 0);
+  s[0] = {W(w ? w->w_gate : nullptr, 0), c.mlp_inter, 0, h, 0};
+  s[1] = {W(w ? w->w_up : nullptr, 0), c.mlp_inter, 0, h, 0};
+  make_plan_host(ps.gu, s, 2, h, grid, (c.mlp_inter + 127) / 128);
+  s[0] = {W(w ? w->w_down : nullptr, 0), h, 0, c.mlp_inter, 0};
+  make_plan_host(ps.down, s, 1, c.mlp_inter, grid, 0);
   const int MPmax = padded_tokens(c.max_batch * c.K);
-  const GemmPlan* all[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
+  const PlanHost* all[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
   ps.part_max = 0;
   for (int i = 0; i < 5; ++i) {
-    const size_t f = part_floats(*all[i], MPmax);
+    const size_t f = part_floats(all[i]->plan, MPmax);
     if (f > ps.part_max) ps.part_max = f;
   }
 }
@@ -200,6 +224,18 @@ int attn_pairs_capacity(const dart_config& c, int n_sm) { return (2 * n_sm) / c.
 int fail_cuda(dart_handle* h, cudaError_t e) {
   if (h) h->last_cuda_error = (int)e; else g_init_cuda_error = (int)e;
   return DART_ERR_CUDA;
+}
+
+template <typename T>
+cudaError_t upload(dart_handle* h, const std::vector<T>& v, T** out) {
+  T* d = nullptr;
+  const size_t nb = (v.size() ? v.size() : 1) * sizeof(T);
+  cudaError_t e = cudaMalloc(&d, nb);
+  if (e != cudaSuccess) return e;
+  h->owned.push_back(d);
+  if (v.size()) e = cudaMemcpy(d, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice);
+  *out = d;
+  return e;
 }
 
 }  // namespace
@@ -224,7 +260,7 @@ size_t dart_workspace_bytes(const dart_config* cfg) {
   const int n_sm = 148;  // sized for a B200; dart_draft_init uses the device's own count
   PlanSet ps;
   build_plans(*cfg, nullptr, n_sm, ps);
-  return layout_workspace(*cfg, n_sm, ps.part_max, attn_pairs_capacity(*cfg, n_sm), 2 * n_sm, nullptr, nullptr);
+  return layout_workspace(*cfg, ps.part_max, attn_pairs_capacity(*cfg, n_sm), 2 * n_sm, nullptr, nullptr);
 }
 
 int dart_last_cuda_error(const dart_handle* h) { return h ? h->last_cuda_error : g_init_cuda_error; }
@@ -257,39 +293,44 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   h->w = *weights;
   h->device = dev;
   h->n_sm = n_sm;
+  h->h_tiles = (cfg->hidden + 127) / 128;
 
-  auto bail = [&](int code) {
-    dart_draft_destroy(h);
-    return code;
-  };
+#define INIT_CHECK(expr)                                 \
+  if ((e = (expr)) != cudaSuccess) {                     \
+    g_init_cuda_error = (int)e;                          \
+    dart_draft_destroy(h);                               \
+    return DART_ERR_CUDA;                                \
+  }
 
   PlanSet ps;
   build_plans(*cfg, weights, n_sm, ps);
-  GemmPlan* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
+  PlanHost* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
   for (int i = 0; i < 5; ++i) {
-    int *dlo = nullptr, *dhi = nullptr;
-    const size_t nb = ps.clo[i].size() * sizeof(int);
-    if ((e = cudaMalloc(&dlo, nb)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
-    h->owned.push_back(dlo);
-    if ((e = cudaMalloc(&dhi, nb)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
-    h->owned.push_back(dhi);
-    if ((e = cudaMemcpy(dlo, ps.clo[i].data(), nb, cudaMemcpyHostToDevice)) != cudaSuccess ||
-        (e = cudaMemcpy(dhi, ps.chi[i].data(), nb, cudaMemcpyHostToDevice)) != cudaSuccess) {
-      g_init_cuda_error = (int)e;
-      return bail(DART_ERR_CUDA);
-    }
-    plans[i]->d_tile_clo = dlo;
-    plans[i]->d_tile_chi = dhi;
+    PlanHost& ph = *plans[i];
+    INIT_CHECK(upload(h, ph.clo, &ph.plan.d_tile_clo));
+    INIT_CHECK(upload(h, ph.chi, &ph.plan.d_tile_chi));
+    INIT_CHECK(upload(h, ph.first, &ph.plan.d_first_tile));
+    INIT_CHECK(upload(h, ph.expected, &ph.plan.d_expected));
+    std::vector<int> zeros(ph.plan.n_groups, 0);
+    INIT_CHECK(upload(h, zeros, &ph.plan.d_ctr));
   }
-  h->plan_fc = ps.fc; h->plan_qkv = ps.qkv; h->plan_o = ps.o; h->plan_gu = ps.gu; h->plan_down = ps.down;
+  h->plan_fc = ps.fc.plan; h->plan_qkv = ps.qkv.plan; h->plan_o = ps.o.plan; h->plan_gu = ps.gu.plan; h->plan_down = ps.down.plan;
   h->lm_grid = 2 * n_sm;
   if (h->lm_grid > cfg->vocab / 16) h->lm_grid = cfg->vocab / 16;
   h->attn_pairs_cap = attn_pairs_capacity(*cfg, n_sm);
 
-  h->ws.bytes = layout_workspace(*cfg, n_sm, ps.part_max, h->attn_pairs_cap, 2 * n_sm, nullptr, nullptr);
-  if ((e = cudaMalloc(&h->ws.base, h->ws.bytes)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
-  layout_workspace(*cfg, n_sm, ps.part_max, h->attn_pairs_cap, 2 * n_sm, static_cast<char*>(h->ws.base), &h->ws);
-  if ((e = cudaMemset(h->ws.base, 0, h->ws.bytes)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+  h->ws.bytes = layout_workspace(*cfg, ps.part_max, h->attn_pairs_cap, 2 * n_sm, nullptr, nullptr);
+  INIT_CHECK(cudaMalloc(&h->ws.base, h->ws.bytes));
+  layout_workspace(*cfg, ps.part_max, h->attn_pairs_cap, 2 * n_sm, static_cast<char*>(h->ws.base), &h->ws);
+  INIT_CHECK(cudaMemset(h->ws.base, 0, h->ws.bytes));
+
+  // the <mask> rows' z (last row of the z buffers) and the 1/rms of their g half: constants of the model
+  {
+    const size_t mrow = (size_t)cfg->max_batch * cfg->K * 2 * cfg->hidden;
+    INIT_CHECK(launch_mask_row(static_cast<const bf16*>(weights->mask_vec), static_cast<const bf16*>(weights->norm_g),
+                               static_cast<const bf16*>(weights->norm_e), cfg->hidden, cfg->rms_eps, h->ws.z_hi + mrow,
+                               h->ws.z_lo + mrow, h->ws.rstd_mask, nullptr));
+  }
 
   // Appendix D's per-level weights: fp64 from the fp32 settings, rounded once to fp32
   for (int i = 0; i < 8; ++i) {
@@ -304,7 +345,7 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   if (n_rows > 0) {
     size_t cap = 16;
     while (cap < (size_t)(2 * n_rows)) cap <<= 1;
-    if (cap > (1ull << 31)) return bail(DART_ERR_INVALID_ARG);
+    if (cap > (1ull << 31)) { dart_draft_destroy(h); return DART_ERR_INVALID_ARG; }
     std::vector<NgramSlot> tab(cap);
     memset(tab.data(), 0, cap * sizeof(NgramSlot));
     const uint32_t mask = (uint32_t)(cap - 1);
@@ -313,8 +354,10 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
       const int ord = ngram->order[i];
       const int c0 = ngram->ctx0[i], c1 = ngram->ctx1[i], nx = ngram->next[i];
       if ((ord != 2 && ord != 3) || c1 < 0 || nx < 0 || c1 >= cfg->vocab || nx >= cfg->vocab ||
-          (ord == 3 && (c0 < 0 || c0 >= cfg->vocab)))
-        return bail(DART_ERR_INVALID_ARG);
+          (ord == 3 && (c0 < 0 || c0 >= cfg->vocab))) {
+        dart_draft_destroy(h);
+        return DART_ERR_INVALID_ARG;
+      }
       if (ord == 3 && cfg->ngram_order < 3) continue;
       const unsigned long long key = ngram_key(ord, c0, c1, nx);
       uint32_t pos = (uint32_t)ngram_hash(key) & mask, d = 0;
@@ -324,26 +367,24 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
       tab[pos].score = ngram->score[i];
       if (d > max_probe) max_probe = d;
     }
-    if ((e = cudaMalloc(&h->ng_slots, cap * sizeof(NgramSlot))) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
-    if ((e = cudaMemcpy(h->ng_slots, tab.data(), cap * sizeof(NgramSlot), cudaMemcpyHostToDevice)) != cudaSuccess) {
-      g_init_cuda_error = (int)e;
-      return bail(DART_ERR_CUDA);
-    }
+    INIT_CHECK(cudaMalloc(&h->ng_slots, cap * sizeof(NgramSlot)));
+    INIT_CHECK(cudaMemcpy(h->ng_slots, tab.data(), cap * sizeof(NgramSlot), cudaMemcpyHostToDevice));
     h->ng_mask = mask;
     h->ng_max_probe = max_probe;
   }
 
-  if ((e = topk_merge_setup(2 * n_sm)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
-  if ((e = attention_setup()) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
-  if ((e = tree_setup(cfg->topk, cfg->beam, cfg->tree_budget, cfg->K)) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
-  if ((e = cudaDeviceSynchronize()) != cudaSuccess) { g_init_cuda_error = (int)e; return bail(DART_ERR_CUDA); }
+  INIT_CHECK(topk_merge_setup(2 * n_sm));
+  INIT_CHECK(attention_setup());
+  INIT_CHECK(tree_setup(cfg->topk, cfg->beam, cfg->tree_budget, cfg->K));
+  INIT_CHECK(cudaDeviceSynchronize());
+#undef INIT_CHECK
   *out = h;
   return DART_OK;
 }
 
 int dart_draft_destroy(dart_handle* h) {
   if (h == nullptr) return DART_OK;
-  for (int* p : h->owned) cudaFree(p);
+  for (void* p : h->owned) cudaFree(p);
   if (h->ws.base) cudaFree(h->ws.base);
   if (h->ng_slots) cudaFree(h->ng_slots);
   delete h;
@@ -353,8 +394,8 @@ int dart_draft_destroy(dart_handle* h) {
 int dart_step_launch_count(const dart_handle* h, int batch, int n_fresh) {
   (void)batch;
   if (h == nullptr) return 0;
-  // fc, stage, qkv, qkv_finalize, attention, combine, o, res_norm, gate_up gemm, gate_up, down, res_norm, lm, merge, tree
-  return (n_fresh > 0 ? 15 : 14);
+  // fc, qkv, attention, combine, o_proj, gate/up, down, lm head, merge (+ tree)
+  return (n_fresh > 0 ? 10 : 9);
 }
 
 int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out* out, void* cuda_stream) {
@@ -377,43 +418,44 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int M = B * K, MP = padded_tokens(M);
   const int hdim = c.hidden, dq = c.n_q_heads * c.head_dim;
+  const long long mask_row = (long long)c.max_batch * K;
   Workspace& ws = h->ws;
   cudaError_t e;
   auto mark = [&](int stage, bool begin) {
     if (h->prof_stage == stage) cudaEventRecord(begin ? h->prof_start : h->prof_stop, st);
   };
+  EpiArgs ep;
+  GemmInput gi;
 
-  // S0: feature fusion FC on the fresh rows, then z = [RMSNorm(g); RMSNorm(e)]
-  StageParams sp;
-  memset(&sp, 0, sizeof(sp));
+  // S0: feature-fusion FC on the fresh rows; epilogue: residual g, z g-half (gain-scaled), sums of squares;
+  // prologue: z e-half = RMSNorm(embedding of the next token)
   mark(0, true);
   if (F > 0) {
-    if ((e = launch_gemm_rows(h->plan_fc, static_cast<const bf16*>(in->feats), nullptr, c.feat_in, B * F, ws.part, st)) != cudaSuccess)
-      return fail_cuda(h, e);
-    sp.fc = make_view(h->plan_fc, ws.part, padded_tokens(B * F));
+    memset(&ep, 0, sizeof(ep));
+    ep.mode = EPI_FC; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
+    ep.res0 = ws.res0; ep.gamma = static_cast<const bf16*>(h->w.norm_g);
+    ep.out_hi = ws.z_hi; ep.out_lo = ws.z_lo; ep.ld_out = 2 * hdim; ep.ss_out = ws.ss_g;
+    ep.tokens = in->tokens; ep.vocab = c.vocab; ep.embed = static_cast<const bf16*>(h->w.embed);
+    ep.gamma_e = static_cast<const bf16*>(h->w.norm_e);
+    gi = {static_cast<const bf16*>(in->feats), nullptr, c.feat_in, B * F, 0, 0, 0};
+    if ((e = launch_gemm_rows(h->plan_fc, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   }
-  sp.B = B; sp.K = K; sp.F = F; sp.h = hdim; sp.tokens = in->tokens; sp.vocab = c.vocab;
-  sp.embed = static_cast<const bf16*>(h->w.embed); sp.mask_vec = static_cast<const bf16*>(h->w.mask_vec);
-  sp.norm_g = static_cast<const bf16*>(h->w.norm_g); sp.norm_e = static_cast<const bf16*>(h->w.norm_e);
-  sp.eps = c.rms_eps; sp.res = ws.res; sp.z_hi = ws.z_hi; sp.z_lo = ws.z_lo;
-  if ((e = launch_stage_inputs(sp, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(0, false);
-  mark(1, true);
 
-  // S1: QKV projection + RoPE + cache rows
-  if ((e = launch_gemm_rows(h->plan_qkv, ws.z_hi, ws.z_lo, 2 * hdim, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
-  QkvParams qp;
-  qp.qkv = make_view(h->plan_qkv, ws.part, MP);
-  qp.q_tile0 = h->plan_qkv.seg[0].tile0; qp.k_tile0 = h->plan_qkv.seg[1].tile0; qp.v_tile0 = h->plan_qkv.seg[2].tile0;
-  qp.B = B; qp.K = K; qp.Hq = c.n_q_heads; qp.Hkv = c.n_kv_heads; qp.dh = c.head_dim;
-  qp.seq_lens = in->seq_lens; qp.rope_theta = c.rope_theta; qp.F = F;
-  qp.q_hi = ws.q_hi; qp.q_lo = ws.q_lo; qp.k_new = ws.k_new; qp.v_new = ws.v_new;
-  qp.k_cache = static_cast<bf16*>(in->k_cache); qp.v_cache = static_cast<bf16*>(in->v_cache); qp.P_cap = c.max_prefix;
-  if ((e = launch_qkv_finalize(qp, st)) != cudaSuccess) return fail_cuda(h, e);
+  // S1: QKV projection; epilogue: 1/rms of g, RoPE, q and new k/v as hi/lo, cache append
+  mark(1, true);
+  memset(&ep, 0, sizeof(ep));
+  ep.mode = EPI_QKV; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
+  ep.ss_in = ws.ss_g; ep.ss_tiles = h->h_tiles; ep.ss_mp = padded_tokens(B * (F > 0 ? F : 1)); ep.rstd_mask = ws.rstd_mask;
+  ep.Hq = c.n_q_heads; ep.Hkv = c.n_kv_heads; ep.dh = c.head_dim; ep.seq_lens = in->seq_lens; ep.rope_theta = c.rope_theta;
+  ep.q_hi = ws.q_hi; ep.q_lo = ws.q_lo; ep.k_new = ws.k_new; ep.v_new = ws.v_new;
+  ep.k_cache = static_cast<bf16*>(in->k_cache); ep.v_cache = static_cast<bf16*>(in->v_cache); ep.P_cap = c.max_prefix;
+  gi = {ws.z_hi, ws.z_lo, 2 * hdim, M, K, F, mask_row};
+  if ((e = launch_gemm_rows(h->plan_qkv, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(1, false);
-  mark(2, true);
 
   // S2: split-KV attention over cache rows 0 .. P_b-1 and the K new rows
+  mark(2, true);
   AttnParams ap;
   ap.B = B; ap.K = K; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.dh = c.head_dim;
   ap.seq_lens = in->seq_lens; ap.q_hi = ws.q_hi; ap.q_lo = ws.q_lo; ap.k_new = ws.k_new; ap.v_new = ws.v_new;
@@ -432,38 +474,43 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   }
   if ((e = launch_attention(ap, in->seq_lens_host, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(2, false);
+
+  // S3: o_proj; epilogue: x1 = residual + proj, gain-scaled hi/lo, sums of squares
   mark(3, true);
-
-  // S3: o_proj + residual + RMSNorm
-  if ((e = launch_gemm_rows(h->plan_o, ws.a_hi, ws.a_lo, dq, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
-  ResNormParams rp;
-  rp.proj = make_view(h->plan_o, ws.part, MP);
-  rp.M = M; rp.h = hdim; rp.gamma = static_cast<const bf16*>(h->w.norm_post); rp.eps = c.rms_eps;
-  rp.res = ws.res; rp.n_hi = ws.n_hi; rp.n_lo = ws.n_lo;
-  if ((e = launch_res_norm(rp, st)) != cudaSuccess) return fail_cuda(h, e);
+  memset(&ep, 0, sizeof(ep));
+  ep.mode = EPI_RES; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
+  ep.res0 = ws.res0; ep.res_in = nullptr; ep.res_out = ws.x1; ep.mask_vec = static_cast<const bf16*>(h->w.mask_vec);
+  ep.gamma = static_cast<const bf16*>(h->w.norm_post);
+  ep.out_hi = ws.n_hi; ep.out_lo = ws.n_lo; ep.ld_out = hdim; ep.ss_out = ws.ss_1;
+  gi = {ws.a_hi, ws.a_lo, dq, M, 0, 0, 0};
+  if ((e = launch_gemm_rows(h->plan_o, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(3, false);
+
+  // S4: gate/up; epilogue: u = SiLU(rstd1 * gate) * (rstd1 * up)
   mark(4, true);
-
-  // S4: gate/up + SiLU * mul
-  if ((e = launch_gemm_rows(h->plan_gu, ws.n_hi, ws.n_lo, hdim, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
-  GateUpParams gp;
-  gp.gu = make_view(h->plan_gu, ws.part, MP);
-  gp.up_tile0 = h->plan_gu.seg[1].tile0; gp.M = M; gp.I = c.mlp_inter; gp.u_hi = ws.u_hi; gp.u_lo = ws.u_lo;
-  if ((e = launch_gate_up(gp, st)) != cudaSuccess) return fail_cuda(h, e);
+  memset(&ep, 0, sizeof(ep));
+  ep.mode = EPI_GATE_UP; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
+  ep.ss_in = ws.ss_1; ep.ss_tiles = h->h_tiles; ep.ss_mp = MP;
+  ep.out_hi = ws.u_hi; ep.out_lo = ws.u_lo; ep.ld_out = c.mlp_inter;
+  gi = {ws.n_hi, ws.n_lo, hdim, M, 0, 0, 0};
+  if ((e = launch_gemm_rows(h->plan_gu, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(4, false);
-  mark(5, true);
 
-  // S5: down + residual + final RMSNorm
-  if ((e = launch_gemm_rows(h->plan_down, ws.u_hi, ws.u_lo, c.mlp_inter, M, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
-  rp.proj = make_view(h->plan_down, ws.part, MP);
-  rp.gamma = static_cast<const bf16*>(h->w.norm_final);
-  if ((e = launch_res_norm(rp, st)) != cudaSuccess) return fail_cuda(h, e);
+  // S5: down; epilogue: x2 = x1 + proj, gain-scaled hi/lo for the LM head, sums of squares
+  mark(5, true);
+  memset(&ep, 0, sizeof(ep));
+  ep.mode = EPI_RES; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
+  ep.res_in = ws.x1; ep.res_out = nullptr; ep.gamma = static_cast<const bf16*>(h->w.norm_final);
+  ep.out_hi = ws.n_hi; ep.out_lo = ws.n_lo; ep.ld_out = hdim; ep.ss_out = ws.ss_2;
+  gi = {ws.u_hi, ws.u_lo, c.mlp_inter, M, 0, 0, 0};
+  if ((e = launch_gemm_rows(h->plan_down, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(5, false);
 
   // S6 + S7: LM head with fused log-softmax / top-k, then the merge
   LmParams lp;
   lp.W = static_cast<const bf16*>(h->w.w_lm); lp.V = c.vocab; lp.Kd = hdim;
   lp.x_hi = ws.n_hi; lp.x_lo = ws.n_lo; lp.ldx = hdim; lp.M = M; lp.K = K;
+  lp.ss_in = ws.ss_2; lp.ss_tiles = h->h_tiles; lp.ss_mp = MP; lp.rms_eps = c.rms_eps;
   lp.topk = c.topk;
   lp.inv_temp = c.temperature > 0.f ? 1.f / c.temperature : 1.f;
   lp.gumbel = c.temperature > 0.f ? 1 : 0;

@@ -9,100 +9,88 @@ namespace dart {
 typedef __nv_bfloat16 bf16;
 
 // ---------------------------------------------------------------------------------------------
-// Weight-streaming small-M GEMM, "rows" mode:  part = W[rows, Kd] * x[M, Kd]^T, split over the
-// flattened (128-row tile, 64-wide k-step) space so that every CTA streams the same number of
-// weight bytes.  A CTA writes one fp32 partial per tile it touches; a finalize kernel sums the
-// partials of a tile in CTA order (deterministic) and applies the op that follows the GEMM.
+// Weight-streaming small-M GEMM:  y = W[rows, Kd] * x[M, Kd]^T, split over the flattened
+// (128-row tile, 64-wide k-step) space so that every CTA streams the same number of weight bytes.
+// A CTA writes one fp32 partial per tile it touches; the CTA that completes a tile (or a pair of
+// tiles) sums the partials in CTA order and applies the op that follows the projection.
 // ---------------------------------------------------------------------------------------------
 struct GemmSeg {
-  const bf16* W;  // [rows, Kd] row-major
+  const bf16* W;  // first element of the segment's sub-matrix (row 0, first column used)
   int rows;       // multiple of 16
   int tile0;      // index of this segment's first 128-row tile in the launch
+  int ld;         // row stride of W in elements
+  int xoff;       // column offset into the activation rows for this segment
 };
 
 struct GemmPlan {
   int nseg;
-  GemmSeg seg[3];
-  int Kd;         // reduction length, multiple of 16
-  int SK;         // ceil(Kd / 64) k-steps per tile
-  int n_tiles;    // 128-row tiles over all segments
-  int grid;       // CTAs
-  int slots;      // max tiles a CTA touches
-  long long U;    // n_tiles * SK
-  int* d_tile_clo;  // DEVICE [n_tiles] first CTA contributing to a tile
-  int* d_tile_chi;  // DEVICE [n_tiles] last CTA contributing to a tile
+  GemmSeg seg[6];
+  int Kd;           // reduction length per segment, multiple of 16
+  int SK;           // ceil(Kd / 64) k-steps per tile
+  int n_tiles;      // 128-row tiles over all segments
+  int grid;         // CTAs
+  int slots;        // max tiles a CTA touches
+  long long U;      // n_tiles * SK
+  int pair_offset;  // > 0: tiles T and T + pair_offset are finalized together (group = T % pair_offset)
+  int n_groups;
+  int* d_tile_clo;    // DEVICE [n_tiles] first CTA contributing to a tile
+  int* d_tile_chi;    // DEVICE [n_tiles] last CTA contributing to a tile
+  int* d_first_tile;  // DEVICE [grid]    first tile of a CTA's range
+  int* d_ctr;         // DEVICE [n_groups] tickets taken (zero between launches)
+  int* d_expected;    // DEVICE [n_groups] tickets that complete a group
 };
-
-// What a finalize kernel needs to sum a tile's partials.
-struct PartView {
-  const float* part;  // [grid][slots][128][MP]
-  const int* clo;
-  const int* chi;
-  int SK;
-  long long U;
-  int G;
-  int slots;
-  int MP;  // padded token count (8, 32 or 128)
-};
-
-inline PartView make_view(const GemmPlan& p, const float* part, int MP) {
-  PartView v;
-  v.part = part; v.clo = p.d_tile_clo; v.chi = p.d_tile_chi; v.SK = p.SK; v.U = p.U; v.G = p.grid;
-  v.slots = p.slots; v.MP = MP;
-  return v;
-}
 
 __host__ __device__ inline int padded_tokens(int M) { return M <= 8 ? 8 : (M <= 32 ? 32 : 128); }
 
-// x_hi/x_lo: bf16 [>=M, ldx] activations (lo may be NULL: plain bf16 input).  M valid tokens.
-cudaError_t launch_gemm_rows(const GemmPlan& plan, const bf16* x_hi, const bf16* x_lo, long long ldx, int M,
-                             float* part, cudaStream_t st);
+struct GemmInput {
+  const bf16* x_hi; const bf16* x_lo;  // [rows, ldx] activations as hi (+ lo, may be NULL)
+  long long ldx;
+  int M;              // valid tokens
+  int x_K, x_F;       // x_K > 0: token (b, r) reads row b*x_F + r if r < x_F, else row x_mask_row
+  long long x_mask_row;
+};
 
-// ---------------------------------------------------------------------------------------------
-// Finalize kernels (one CTA per token row).
-// ---------------------------------------------------------------------------------------------
-struct StageParams {  // S0: z = [RMSNorm(g); RMSNorm(e)], residual = g
-  PartView fc;        // FC partials, token index = b*F + r (only when F > 0)
-  int B, K, F, h;
-  const int32_t* tokens;  // [B,F]
-  int vocab;
-  const bf16* embed; const bf16* mask_vec; const bf16* norm_g; const bf16* norm_e;
+enum EpiMode : int { EPI_FC = 0, EPI_QKV = 1, EPI_RES = 2, EPI_GATE_UP = 3 };
+
+// Everything the fused epilogues need (unused fields stay zero).
+struct EpiArgs {
+  int mode;
+  int K, F, h;        // rows per sequence, fresh rows per sequence, hidden
   float eps;
-  float* res;      // [M, h] fp32 residual stream (out)
-  bf16* z_hi; bf16* z_lo;  // [M, 2h]
+  // EPI_FC: g -> res0 [B*F, h], z g-half (gain-scaled, hi/lo, row stride ld_out), ss_out [tile][MP]
+  // EPI_RES: x = res + proj -> res_out, out_hi/lo = x * gamma, ss_out
+  float* res0;            // FC: out; RES with res_in == NULL: the fresh rows' g
+  const float* res_in;    // RES: residual in (NULL: first residual = g or <mask>)
+  float* res_out;         // RES: residual out (may be NULL)
+  const bf16* mask_vec;   // <mask> representation [2h]
+  const bf16* gamma;      // gain applied to the hi/lo output
+  bf16* out_hi; bf16* out_lo; long long ld_out;
+  float* ss_out;
+  // rstd of the *input* of this projection, applied to its output: per-tile sums of squares
+  const float* ss_in; int ss_tiles; int ss_mp;
+  const float* rstd_mask;  // QKV: 1/rms of the <mask> row's g half
+  // EPI_FC prologue: shifted token embedding of the fresh rows
+  const int32_t* tokens; int vocab; const bf16* embed; const bf16* gamma_e;
+  // EPI_QKV
+  int Hq, Hkv, dh; const int32_t* seq_lens; float rope_theta;
+  bf16* q_hi; bf16* q_lo; bf16* k_new; bf16* v_new; bf16* k_cache; bf16* v_cache; long long P_cap;
 };
-cudaError_t launch_stage_inputs(const StageParams& p, cudaStream_t st);
 
-struct QkvParams {  // S1 epilogue: RoPE + cache write
-  PartView qkv;     // rows: [q heads | k heads | v heads] (three segments)
-  int q_tile0, k_tile0, v_tile0;
-  int B, K, Hq, Hkv, dh;
-  const int32_t* seq_lens;
-  float rope_theta;
-  int F;             // rows r < F are fresh: their k, v are appended to the cache at P_b + r
-  bf16* q_hi; bf16* q_lo;        // [B, Hq, K, dh] post-RoPE queries as hi + lo
-  bf16* k_new; bf16* v_new;      // [B, Hkv, 16, dh]: rows 0..7 hi parts of the K new rows, rows 8..15 lo parts
-  bf16* k_cache; bf16* v_cache;  // [*, Hkv, P_cap, dh]
-  long long P_cap;
+struct GemmArgs {
+  GemmSeg seg[6];
+  int nseg, Kd, SK, slots;
+  long long U;
+  const bf16* x_hi; const bf16* x_lo; long long ldx; int M;
+  int x_K, x_F; long long x_mask_row;
+  float* part; const int* first_tile; const int* clo; const int* chi;
+  int* ctr; const int* expected; int pair_offset;
+  EpiArgs epi;
 };
-cudaError_t launch_qkv_finalize(const QkvParams& p, cudaStream_t st);
 
-struct ResNormParams {  // x_out = res + sum(parts); n = RMSNorm(x_out) * gamma
-  PartView proj;
-  int M, h;
-  const bf16* gamma; float eps;
-  float* res;          // [M,h] in/out (updated in place)
-  bf16* n_hi; bf16* n_lo;  // [M,h]
-};
-cudaError_t launch_res_norm(const ResNormParams& p, cudaStream_t st);
-
-struct GateUpParams {  // u = SiLU(gate) * up
-  PartView gu;  // two segments: gate rows then up rows
-  int up_tile0;
-  int M, I;
-  bf16* u_hi; bf16* u_lo;  // [M, I]
-};
-cudaError_t launch_gate_up(const GateUpParams& p, cudaStream_t st);
+cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const EpiArgs& epi, float* part, cudaStream_t st);
+// z row of the <mask> rows and the 1/rms of its g half (once, at init)
+cudaError_t launch_mask_row(const bf16* mask_vec, const bf16* norm_g, const bf16* norm_e, int h, float eps, bf16* z_hi,
+                            bf16* z_lo, float* rstd_mask, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
 // Split-KV grouped-query attention over the cache (rows 0 .. P_b-1) and the step's new rows + combine.
@@ -128,6 +116,7 @@ cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, cuda
 struct LmParams {
   const bf16* W; int V; int Kd;
   const bf16* x_hi; const bf16* x_lo; long long ldx; int M; int K;  // token m = b*K + r
+  const float* ss_in; int ss_tiles; int ss_mp; float rms_eps;  // final RMSNorm's 1/rms, applied to the logits
   int topk; float inv_temp; int gumbel; uint32_t seed_lo, seed_hi, step; float eps_logit;
   int grid;
   float* logits_out;       // nullable [M,V]

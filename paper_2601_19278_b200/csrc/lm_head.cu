@@ -53,6 +53,7 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) lm_head_kernel(const L
   float* st_y = st_key + MP * 32;
   int* st_id = reinterpret_cast<int*>(st_y + MP * 32);
   float* st_ms = reinterpret_cast<float*>(st_id + MP * 32);  // [MP][2]
+  float* s_rstd = st_ms + 2 * MP;                            // [MP] 1/rms of the final RMSNorm per token row
 
   const int c = blockIdx.x, G = gridDim.x;
   const int n_mt = p.V >> 4;
@@ -62,7 +63,14 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) lm_head_kernel(const L
   const int spw = (SK + 7) >> 3;  // k-steps per warp per tile
 
   for (int i = tid; i < MP * 32; i += 256) { st_key[i] = -INFINITY; st_y[i] = 0.f; st_id[i] = 0x7fffffff; }
-  for (int i = tid; i < MP; i += 256) { st_ms[2 * i] = -INFINITY; st_ms[2 * i + 1] = 0.f; }
+  for (int i = tid; i < MP; i += 256) {
+    st_ms[2 * i] = -INFINITY;
+    st_ms[2 * i + 1] = 0.f;
+    float ssq = 0.f;  // the activations are x * gain; their 1/rms multiplies the logits (same fixed order everywhere)
+    if (i < p.M)
+      for (int tl = 0; tl < p.ss_tiles; ++tl) ssq += p.ss_in[(size_t)tl * p.ss_mp + i];
+    s_rstd[i] = i < p.M ? 1.f / sqrtf(ssq / (float)p.Kd + p.rms_eps) : 0.f;
+  }
   __syncthreads();
 
   float acc[NT][4];
@@ -154,6 +162,7 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) lm_head_kernel(const L
             float v = 0.f;
 #pragma unroll
             for (int w = 0; w < 8; ++w) v += red[((size_t)buf * 8 + w) * 16 * MP + row * MP + tok];
+            v *= s_rstd[tok];
             stage[tok * SROW + slot * 16 + row] = v;
             if (p.logits_out != nullptr && tok < p.M) p.logits_out[(size_t)tok * p.V + cp.mt * 16 + row] = v;
           }
@@ -232,7 +241,7 @@ __global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) lm_head_kernel(const L
 template <int NT>
 static size_t lm_smem_bytes() {
   constexpr int MP = 8 * NT, RB = (NT <= 4) ? 2 : 1;
-  return sizeof(float) * ((size_t)RB * 8 * 16 * MP + (size_t)MP * 129 + 3 * (size_t)MP * 32 + 2 * (size_t)MP);
+  return sizeof(float) * ((size_t)RB * 8 * 16 * MP + (size_t)MP * 129 + 3 * (size_t)MP * 32 + 3 * (size_t)MP);
 }
 
 template <int NT, int PF, bool FULL>
