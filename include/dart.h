@@ -223,6 +223,27 @@ int dart_step_launch_count(const dart_handle* h, int batch, int n_fresh);
  */
 int dart_set_profile_events(dart_handle* h, int stage, void* start_event, void* stop_event);
 
+/*
+ * Per-row log-softmax + top-k of caller-provided logits without any allocation (the paper has no
+ * counterpart: this is the candidate selection of Algorithm 1 lines 6-8 at temperature 0, offered to
+ * callers that cannot allocate device memory -- a process whose own pool already owns all of HBM, a
+ * latency-critical loop where cudaMalloc's implicit synchronisation is not allowed, a plug-in without a
+ * dart_handle to hold a workspace).  Needs no handle.
+ *   logits      DEVICE f32 [rows, vocab], row-major            (in)
+ *   out_ids     DEVICE i32 [rows, topk]   value desc, ties to the lower id   (out)
+ *   out_slogit  DEVICE f32 [rows, topk]   log(softmax(logits)[id] + eps_logit) (out)
+ * Limits: 1 <= rows <= 128 (more: DART_ERR_CAPACITY), 1 <= topk <= min(32, vocab).
+ * Scratch: a fixed 1.6 MB array inside the library's device image, one per GPU, which every GPU that
+ * loads the library holds until the process exits.  All calls on a GPU share it and it keeps the last
+ * call's contents (every call overwrites what it reads, nothing needs clearing): calls that overlap on
+ * the same GPU -- different streams or host threads -- race; serialise them.
+ * The first call on each device (made with that device current) looks up the array's device address;
+ * make that first call before any CUDA stream capture.  Calls cudaMalloc/cudaFree never.
+ * Asynchronous on `cuda_stream`.  Errors: INVALID_ARG, CAPACITY, CUDA.
+ */
+int dart_topk_rows_noalloc(const float* logits, int32_t rows, int32_t vocab, int32_t topk, float eps_logit,
+                           int32_t* out_ids, float* out_slogit, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

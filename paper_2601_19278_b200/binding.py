@@ -27,7 +27,7 @@ DART_ERR_INTERNAL = -6
 EXPORTS = [
     "dart_draft_init", "dart_draft_step", "dart_build_tree", "dart_draft_destroy", "dart_last_device_status",
     "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_step_launch_count",
-    "dart_set_profile_events",
+    "dart_set_profile_events", "dart_topk_rows_noalloc",
 ]
 
 
@@ -108,6 +108,9 @@ def lib() -> C.CDLL:
         L.dart_step_launch_count.restype = C.c_int
         L.dart_set_profile_events.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         L.dart_set_profile_events.restype = C.c_int
+        L.dart_topk_rows_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
+                                             C.c_void_p, C.c_void_p]
+        L.dart_topk_rows_noalloc.restype = C.c_int
         _lib = L
     return _lib
 
@@ -206,6 +209,20 @@ class DartDraft:
 
     def launch_count(self, batch: int, n_fresh: int) -> int:
         return lib().dart_step_launch_count(self._h, batch, n_fresh)
+
+
+def topk_rows_noalloc(logits: torch.Tensor, topk: int, eps_logit: float, out_ids: torch.Tensor, out_slogit: torch.Tensor,
+                      stream=None) -> None:
+    """dart_topk_rows_noalloc: log-softmax + top-k of fp32 logits [rows, vocab] into caller-owned outputs.
+    For callers that may not allocate device memory: the library uses a fixed scratch array of its own
+    (at most 128 rows; calls on one GPU must not overlap)."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous() and logits.dim() == 2
+    rows, vocab = logits.shape
+    st = (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+    rc = lib().dart_topk_rows_noalloc(logits.data_ptr(), rows, vocab, topk, eps_logit, out_ids.data_ptr(),
+                                      out_slogit.data_ptr(), st)
+    if rc != DART_OK:
+        raise DartError(rc, "dart_topk_rows_noalloc")
 
 
 def workspace_bytes(cfg: DartConfig) -> int:
