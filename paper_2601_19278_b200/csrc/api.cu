@@ -88,7 +88,7 @@ struct PlanHost {
   std::vector<int> clo, chi, first, expected;
 };
 
-// Cut the flattened (tile, k-step) space of a projection into `grid_target` equal ranges.
+// Cut the flattened (16-row tile, k-round) space of a projection into `grid_target` equal ranges.
 void make_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int grid_target, int pair_offset) {
   GemmPlan& p = ph.plan;
   memset(&p, 0, sizeof(p));
@@ -105,19 +105,21 @@ void make_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int gri
   }
   p.Kd = Kd;
   p.SK = (Kd + 63) / 64;
+  p.KR = (p.SK + 15) / 16;
   p.n_tiles = tiles;
-  p.U = (long long)tiles * p.SK;
+  const int n_mt = tiles * 8;
+  p.U = (long long)n_mt * p.KR;
   p.grid = (int)((long long)grid_target < p.U ? grid_target : p.U);
   p.pair_offset = pair_offset;
   p.n_groups = pair_offset > 0 ? pair_offset : tiles;
-  ph.clo.assign(tiles, 0x7fffffff);
-  ph.chi.assign(tiles, -1);
+  ph.clo.assign(n_mt, 0x7fffffff);
+  ph.chi.assign(n_mt, -1);
   ph.first.assign(p.grid, 0);
   p.slots = 1;
   for (int c = 0; c < p.grid; ++c) {
     const long long u0 = ((long long)c * p.U) / p.grid, u1 = ((long long)(c + 1) * p.U) / p.grid;
     if (u0 >= u1) continue;
-    const int t0 = (int)(u0 / p.SK), t1 = (int)((u1 - 1) / p.SK);
+    const int t0 = (int)(u0 / p.KR), t1 = (int)((u1 - 1) / p.KR);
     ph.first[c] = t0;
     if (t1 - t0 + 1 > p.slots) p.slots = t1 - t0 + 1;
     for (int t = t0; t <= t1; ++t) {
@@ -126,10 +128,13 @@ void make_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int gri
     }
   }
   ph.expected.assign(p.n_groups, 0);
-  for (int t = 0; t < tiles; ++t) ph.expected[pair_offset > 0 ? t % pair_offset : t] += ph.chi[t] - ph.clo[t] + 1;
+  for (int t = 0; t < n_mt; ++t) {
+    const int tile = t >> 3;
+    ph.expected[pair_offset > 0 ? tile % pair_offset : tile] += ph.chi[t] - ph.clo[t] + 1;
+  }
 }
 
-size_t part_floats(const GemmPlan& p, int MP) { return (size_t)p.grid * p.slots * 128 * MP; }
+size_t part_floats(const GemmPlan& p, int MP) { return (size_t)p.grid * p.slots * 16 * MP; }
 
 struct Layout {
   size_t total = 0;
@@ -307,9 +312,9 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   PlanHost* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
   for (int i = 0; i < 5; ++i) {
     PlanHost& ph = *plans[i];
-    INIT_CHECK(upload(h, ph.clo, &ph.plan.d_tile_clo));
-    INIT_CHECK(upload(h, ph.chi, &ph.plan.d_tile_chi));
-    INIT_CHECK(upload(h, ph.first, &ph.plan.d_first_tile));
+    INIT_CHECK(upload(h, ph.clo, &ph.plan.d_mt_clo));
+    INIT_CHECK(upload(h, ph.chi, &ph.plan.d_mt_chi));
+    INIT_CHECK(upload(h, ph.first, &ph.plan.d_first_mt));
     INIT_CHECK(upload(h, ph.expected, &ph.plan.d_expected));
     std::vector<int> zeros(ph.plan.n_groups, 0);
     INIT_CHECK(upload(h, zeros, &ph.plan.d_ctr));

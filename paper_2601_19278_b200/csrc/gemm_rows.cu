@@ -3,102 +3,112 @@
 // into its epilogue.
 //
 // The op is HBM-bound: M = batch*K token rows (8..128) against weight matrices of 10^7..10^8
-// elements, i.e. M flop per weight byte.  Design:
-//   * weights are the MMA's M-side operand (16 weight rows x 16 k per mma.sync.m16n8k16),
-//     token rows are the 8-wide N side, so M = 8 tokens is an exact fit;
-//   * weight fragments go global -> registers with 128-bit loads; the k index is permuted
-//     identically on both operands so that the 2 x 16 bytes a thread loads are exactly its
-//     fragment slots;
-//   * activations (a few hundred KB, bf16 hi + lo) are read through L1 by every warp;
-//   * the flattened (128-row tile, 64-wide k-step) space is cut into gridDim.x equal ranges,
-//     so every CTA streams the same number of bytes (no tail wave).  A CTA writes one fp32
-//     partial per tile it touches and takes a ticket on the tile's counter; the CTA that takes
-//     the last ticket sums the tile's partials in CTA order (deterministic, no float atomics)
-//     and applies the fused op: residual add, RMSNorm gain + sum of squares, RoPE + cache
-//     append, or SiLU-gate.
+// elements, i.e. M flop per weight byte.  The streaming loop is the shared core of
+// stream_core.cuh (16 warps per CTA interleave k-steps over one 16-row tile; 2 CTAs per SM).
+// What this file adds:
+//   * stream-K: the flattened (16-row tile, k-round) space is cut into gridDim.x equal ranges, so
+//     every CTA streams the same number of bytes (no tail wave).  A CTA writes one fp32 partial per
+//     16-row tile it touches and takes tickets on the counter of the tile's 128-row group; the CTA
+//     that takes the last ticket sums the group's partials in CTA order (deterministic, no float
+//     atomics) and applies the fused op: residual add, RMSNorm gain + sum of squares, RoPE + cache
+//     append, or SiLU-gate;
 //   * RMSNorm's 1/rms is a per-token scalar, so it is applied *after* the next projection
 //     (W (x*gain) * rstd): no row-wide reduction ever sits between two kernels.  A finalizer
-//     only emits its tile's partial sum of squares; whoever needs rstd adds up the tiles'.
+//     only emits its group's partial sum of squares; whoever needs rstd adds up the groups'.
 #include "common.cuh"
 #include "kernels.h"
+#include "stream_core.cuh"
 
 namespace dart {
-
-struct RowCursor {
-  int tile, ks;
-  const bf16* r0;
-  const bf16* r1;
-  int xoff;
-  bool valid;
-  __device__ __forceinline__ void set_tile(const GemmArgs& p, int warp, int g) {
-    int s = 0;
-#pragma unroll
-    for (int i = 1; i < 6; ++i)
-      if (i < p.nseg && tile >= p.seg[i].tile0) s = i;
-    const GemmSeg sg = p.seg[s];
-    const int row0 = (tile - sg.tile0) * 128 + warp * 16;
-    valid = row0 < sg.rows;
-    r0 = sg.W + (size_t)(valid ? row0 + g : 0) * sg.ld;
-    r1 = r0 + (size_t)(valid ? 8 : 0) * sg.ld;
-    xoff = sg.xoff;
-  }
-  __device__ __forceinline__ void advance(const GemmArgs& p, int warp, int g) {
-    if (++ks == p.SK) {
-      ks = 0;
-      ++tile;
-      set_tile(p, warp, g);
-    }
-  }
-};
 
 // ------------------------------------------------------------------------------------------
 // Fused epilogues, run by the CTA that completes a tile (or a pair of tiles).
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ float piece_sum(const GemmArgs& p, int tile, int row, int tok, int MP) {
+// Shared-memory description of one group: for each of its (up to 16) 16-row tiles, the partial pieces
+// to add up, as offsets into `part` in units of one 16 x MP piece, in CTA order.
+constexpr int kMaxPieces = 33;
+struct GroupMeta {
+  int cnt[16];
+  unsigned off[16][kMaxPieces];
+};
+
+__device__ __forceinline__ void load_group_meta(const GemmArgs& p, int Ta, int Tb, bool paired, GroupMeta* gm) {
+  const int j = threadIdx.x;
+  if (j < 16 && (j < 8 || paired)) {
+    const int mt = (j < 8 ? Ta : Tb) * 8 + (j & 7);
+    const int lo = p.clo[mt], hi = p.chi[mt];
+    int n = 0;
+    for (int c = lo; c <= hi && n < kMaxPieces; ++c) gm->off[j][n++] = (unsigned)(c * p.slots + (mt - p.first_mt[c]));
+    gm->cnt[j] = n;
+  }
+  __syncthreads();
+}
+
+// which: 0 = tile Ta, 1 = tile Tb of the group
+__device__ __forceinline__ float piece_sum(const GemmArgs& p, const GroupMeta* gm, int which, int row, int tok, int MP) {
   float s = 0.f;
-  const int lo = p.clo[tile], hi = p.chi[tile];
-  for (int c = lo; c <= hi; ++c)
-    s += p.part[(((size_t)c * p.slots + (tile - p.first_tile[c])) * 128 + row) * MP + tok];
+  const int j = which * 8 + (row >> 4), r = row & 15;
+  const int n = gm->cnt[j];
+  for (int i = 0; i < n; ++i) s += p.part[((size_t)gm->off[j][i] * 16 + r) * MP + tok];
   return s;
 }
 
-// rstd of a token from per-tile sums of squares ss[tile][mp] over `ntile` tiles of a width-`h` row
-__device__ __forceinline__ float rstd_from(const float* ss, int ntile, int mp, int col, int h, float eps) {
-  float s = 0.f;
-  for (int t = 0; t < ntile; ++t) s += ss[(size_t)t * mp + col];
-  return 1.f / sqrtf(s / (float)h + eps);
+// 1/rms of every token row from per-tile sums of squares ss[tile][mp] (tiles of a width-`h` row), into
+// s_rstd[0..M).  Four threads per token add up interleaved tiles, then their four partials are added in a
+// fixed order.  col(tok) maps a token to its column of ss.  Needs M <= 128 and blockDim >= 512.
+template <class ColFn>
+__device__ __forceinline__ void rstd_all(const float* ss, int ntile, int mp, int M, int h, float eps, float* s_part,
+                                         float* s_rstd, ColFn col) {
+  const int tid = threadIdx.x;
+  if (tid < 4 * M) {
+    const int tok = tid >> 2, q = tid & 3;
+    const int cidx = col(tok);
+    float s = 0.f;
+    if (cidx >= 0)
+      for (int t = q; t < ntile; t += 4) s += ss[(size_t)t * mp + cidx];
+    s_part[tid] = s;
+  }
+  __syncthreads();
+  if (tid < M) {
+    const float s = s_part[4 * tid] + s_part[4 * tid + 1] + s_part[4 * tid + 2] + s_part[4 * tid + 3];
+    if (col(tid) >= 0) s_rstd[tid] = 1.f / sqrtf(s / (float)h + eps);
+  }
+  __syncthreads();
 }
 
-// sum over the tile's 128 rows of v (one value per thread: row = tid & 127, token parity = tid >> 7),
-// result valid in every thread; fixed order.  sh: 8 floats.
+// sum over the group's 128 rows of v (one value per thread: row = tid & 127, token class = tid >> 7),
+// result valid in every thread; fixed order.  sh: one float per warp.
 __device__ __forceinline__ float tile_rows_sum(float v, float* sh) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   v = warp_sum(v);
   __syncthreads();
   if (lane == 0) sh[warp] = v;
   __syncthreads();
-  const int half = warp >> 2;  // warps 0..3 hold token parity 0, warps 4..7 parity 1
-  return sh[half * 4] + sh[half * 4 + 1] + sh[half * 4 + 2] + sh[half * 4 + 3];
+  const int cls = warp >> 2;  // warps 4*cls .. 4*cls+3 hold the 128 rows of token class cls
+  return sh[cls * 4] + sh[cls * 4 + 1] + sh[cls * 4 + 2] + sh[cls * 4 + 3];
 }
 
-__device__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, float* s_rstd) {
+__device__ __noinline__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, float* s_rstd, GroupMeta* gm,
+                                            float* s_part) {
   const EpiArgs& e = p.epi;
   const int tid = threadIdx.x;
   const int Ta = group, Tb = group + p.pair_offset;
+  load_group_meta(p, Ta, Tb, p.pair_offset > 0, gm);
   int s = 0;  // segment of tile Ta
   for (int i = 1; i < 6; ++i)
-    if (i < p.nseg && Ta >= p.seg[i].tile0) s = i;
-  const int row_base = (Ta - p.seg[s].tile0) * 128;       // first row of the tile inside its matrix
-  const int rows_valid = min(128, p.seg[s].rows - row_base);
-  const int row = tid & 127, par = tid >> 7;               // thread -> (row, token parity)
+    if (i < p.s.nseg && Ta >= p.s.seg[i].tile0) s = i;
+  const int row_base = (Ta - p.s.seg[s].tile0) * 128;       // first row of the tile inside its matrix
+  const int rows_valid = min(128, p.s.seg[s].rows - row_base);
+  const int row = tid & 127, par = tid >> 7;               // thread -> (row, token class)
+  const int npar = blockDim.x >> 7;
 
   if (e.mode == EPI_FC) {
     // g = FC(features) on the fresh rows: residual stream, gain-scaled hi/lo, tile sum of squares
-    for (int tok = par; tok < MP; tok += 2) {
+    for (int tok = par; tok < MP; tok += npar) {
       float g = 0.f;
-      if (row < rows_valid && tok < p.M) g = piece_sum(p, Ta, row, tok, MP);
+      if (row < rows_valid && tok < p.s.M) g = piece_sum(p, gm, 0, row, tok, MP);
       const float ssq = tile_rows_sum(g * g, sh);
-      if (row < rows_valid && tok < p.M) {
+      if (row < rows_valid && tok < p.s.M) {
         const int n = row_base + row;
         e.res0[(size_t)tok * e.h + n] = g;
         bf16 hi, lo;
@@ -106,13 +116,13 @@ __device__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, 
         e.out_hi[(size_t)tok * e.ld_out + n] = hi;
         e.out_lo[(size_t)tok * e.ld_out + n] = lo;
       }
-      if (row == 0 && tok < p.M) e.ss_out[(size_t)Ta * MP + tok] = ssq;
+      if (row == 0 && tok < p.s.M) e.ss_out[(size_t)Ta * MP + tok] = ssq;
     }
   } else if (e.mode == EPI_RES) {
     // x = residual + proj; gain-scaled hi/lo for the next projection; tile sum of squares
-    for (int tok = par; tok < MP; tok += 2) {
+    for (int tok = par; tok < MP; tok += npar) {
       float x = 0.f;
-      if (row < rows_valid && tok < p.M) {
+      if (row < rows_valid && tok < p.s.M) {
         const int n = row_base + row;
         float r;
         if (e.res_in != nullptr) r = e.res_in[(size_t)tok * e.h + n];
@@ -120,10 +130,10 @@ __device__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, 
           const int b = tok / e.K, rr = tok % e.K;
           r = rr < e.F ? e.res0[(size_t)(b * e.F + rr) * e.h + n] : __bfloat162float(e.mask_vec[n]);
         }
-        x = r + piece_sum(p, Ta, row, tok, MP);
+        x = r + piece_sum(p, gm, 0, row, tok, MP);
       }
       const float ssq = tile_rows_sum(x * x, sh);
-      if (row < rows_valid && tok < p.M) {
+      if (row < rows_valid && tok < p.s.M) {
         const int n = row_base + row;
         if (e.res_out != nullptr) e.res_out[(size_t)tok * e.h + n] = x;
         bf16 hi, lo;
@@ -131,17 +141,16 @@ __device__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, 
         e.out_hi[(size_t)tok * e.ld_out + n] = hi;
         e.out_lo[(size_t)tok * e.ld_out + n] = lo;
       }
-      if (row == 0 && tok < p.M) e.ss_out[(size_t)Ta * MP + tok] = ssq;
+      if (row == 0 && tok < p.s.M) e.ss_out[(size_t)Ta * MP + tok] = ssq;
     }
   } else if (e.mode == EPI_GATE_UP) {
     // u = SiLU(rstd * gate) * (rstd * up): the previous RMSNorm's 1/rms is applied here
-    if (tid < p.M) s_rstd[tid] = rstd_from(e.ss_in, e.ss_tiles, e.ss_mp, tid, e.h, e.eps);
-    __syncthreads();
-    for (int tok = par; tok < p.M; tok += 2) {
+    rstd_all(e.ss_in, e.ss_tiles, e.ss_mp, p.s.M, e.h, e.eps, s_part, s_rstd, [](int tok) { return tok; });
+    for (int tok = par; tok < p.s.M; tok += npar) {
       if (row < rows_valid) {
         const int n = row_base + row;
-        const float gt = s_rstd[tok] * piece_sum(p, Ta, row, tok, MP);
-        const float up = s_rstd[tok] * piece_sum(p, Tb, row, tok, MP);
+        const float gt = s_rstd[tok] * piece_sum(p, gm, 0, row, tok, MP);
+        const float up = s_rstd[tok] * piece_sum(p, gm, 1, row, tok, MP);
         bf16 hi, lo;
         split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
         e.out_hi[(size_t)tok * e.ld_out + n] = hi;
@@ -151,20 +160,22 @@ __device__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, 
   } else if (e.mode == EPI_QKV) {
     // y = rstd_g * (W[:, :h] z_g) + W[:, h:] z_e ; RoPE on q, k at position P_b + r ; q and the new rows'
     // k, v as hi/lo pairs ; the fresh rows' k, v appended to the cache
-    if (tid < p.M) {
-      const int b = tid / e.K, rr = tid % e.K;
-      s_rstd[tid] = rr < e.F ? rstd_from(e.ss_in, e.ss_tiles, e.ss_mp, b * e.F + rr, e.h, e.eps) : e.rstd_mask[0];
-    }
+    if (tid < p.s.M) s_rstd[tid] = e.rstd_mask[0];  // <mask> rows; fresh rows are overwritten below
     __syncthreads();
+    {
+      const int K = e.K, F = e.F;
+      rstd_all(e.ss_in, e.ss_tiles, e.ss_mp, p.s.M, e.h, e.eps, s_part, s_rstd,
+               [K, F](int tok) { const int b = tok / K, rr = tok % K; return rr < F ? b * F + rr : -1; });
+    }
     const int kind = s;  // segment 0,1,2 = q,k,v (g half); the e half is the paired tile
     const int dh = e.dh, half = dh >> 1;
     const int pairs = (rows_valid / dh) * half;  // (head, i) pairs in this tile
-    for (int idx = tid; idx < pairs * p.M; idx += 256) {
+    for (int idx = tid; idx < pairs * p.s.M; idx += blockDim.x) {
       const int tok = idx / pairs, pi = idx - tok * pairs;
       const int hl = pi / half, i = pi - hl * half;
       const int ra = hl * dh + i, rb = ra + half;
-      const float x1 = s_rstd[tok] * piece_sum(p, Ta, ra, tok, MP) + piece_sum(p, Tb, ra, tok, MP);
-      const float x2 = s_rstd[tok] * piece_sum(p, Ta, rb, tok, MP) + piece_sum(p, Tb, rb, tok, MP);
+      const float x1 = s_rstd[tok] * piece_sum(p, gm, 0, ra, tok, MP) + piece_sum(p, gm, 1, ra, tok, MP);
+      const float x2 = s_rstd[tok] * piece_sum(p, gm, 0, rb, tok, MP) + piece_sum(p, gm, 1, rb, tok, MP);
       const int b = tok / e.K, r = tok % e.K;
       const long long pos = (long long)e.seq_lens[b] + r;
       float o1 = x1, o2 = x2;
@@ -199,7 +210,7 @@ __device__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, 
 
 // Shifted token embedding of the fresh rows (Section 3.2): e = E[token], normalised (its 1/rms needs
 // nothing else) and written as the second half of the fresh row's z.  One CTA per fresh row.
-__device__ void embed_rows(const GemmArgs& p, float* sh) {
+__device__ __noinline__ void embed_rows(const GemmArgs& p, float* sh) {
   const EpiArgs& e = p.epi;
   const int ftok = blockIdx.x;
   const int id = min(max(e.tokens[ftok], 0), e.vocab - 1);
@@ -219,134 +230,68 @@ __device__ void embed_rows(const GemmArgs& p, float* sh) {
   }
 }
 
-// FULL: Kd is a multiple of 64, every segment's rows a multiple of 128 and all MP token rows are
-// valid, so the streaming loop carries no bounds predicates.
+// Epilogue functor of the streaming core: partial write and tickets.  A CTA that takes the last ticket of
+// a group only records the group; it runs the fused finalize after it has streamed its whole range, so the
+// streaming loop stays free of the finalize's registers and latency.
+template <int NT, int NW>
+struct GemmEpi {
+  static constexpr int MP = 8 * NT;
+  const GemmArgs& p;
+  const float* red;
+  int* s_done;   // [0] = count, [1..] = completed groups
+  int c, first_mt, pending;
+
+  __device__ __forceinline__ int group_of(int mt) const {
+    const int tile = mt >> 3;
+    return p.pair_offset > 0 ? tile % p.pair_offset : tile;
+  }
+  __device__ __forceinline__ void mtile_done(int mt, int buf, bool last) {
+    float* dst = p.part + ((size_t)c * p.slots + (mt - first_mt)) * 16 * MP;
+    for (int e = threadIdx.x; e < 16 * MP; e += blockDim.x) dst[e] = red_sum<NW, MP>(red, buf, e / MP, e % MP);
+    ++pending;
+    const int group = group_of(mt);
+    if (last || group_of(mt + 1) != group) {
+      // this CTA's last piece of the group: take its tickets
+      __threadfence();
+      __syncthreads();
+      if (threadIdx.x == 0 && atomicAdd(&p.ctr[group], pending) + pending == p.expected[group]) s_done[++s_done[0]] = group;
+      pending = 0;
+    }
+  }
+};
+
+constexpr int kMaxDone = 62;
+
+// FULL: Kd is a multiple of 1024, every segment's rows a multiple of 128, so the streaming loop carries
+// no bounds predicates (padded token rows read row 0 and are never used).
 template <int NT, bool HAS_LO, int PF, bool FULL>
-__global__ void __launch_bounds__(256, (NT <= 4 ? 2 : 1)) gemm_rows_kernel(const GemmArgs p) {
-  constexpr int MP = 8 * NT;
+__global__ void __launch_bounds__(512, (NT == 1 ? 2 : 1)) gemm_rows_kernel(const __grid_constant__ GemmArgs p) {
+  constexpr int NW = 16, RB = (NT <= 4) ? 2 : 1;
+  extern __shared__ __align__(16) float red[];  // [RB][NW][16][MP]
   __shared__ float sh[32];
   __shared__ float s_rstd[128];
-  __shared__ int s_last;
+  __shared__ int s_done[kMaxDone + 2];
   const int c = blockIdx.x, G = gridDim.x;
-  if (p.epi.mode == EPI_FC && c < p.M) embed_rows(p, sh);
+  if (threadIdx.x == 0) s_done[0] = 0;
+  if (p.epi.mode == EPI_FC && c < p.s.M) embed_rows(p, sh);
   const long long u0 = ((long long)c * p.U) / G, u1 = ((long long)(c + 1) * p.U) / G;
   if (u0 >= u1) return;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-  const int tile_first = (int)(u0 / p.SK);
-
-  float acc[NT][4];
-#pragma unroll
-  for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-  uint4 a[PF][4];
-
-  // activation row of each token this thread feeds to the MMA (token n*8+g); with x_K > 0 the rows
-  // r >= x_F of every sequence all read the shared <mask> row
-  const bf16* xh[NT];
-  const long long xlo_delta = p.x_lo - p.x_hi;
-#pragma unroll
-  for (int n = 0; n < NT; ++n) {
-    const int tok = n * 8 + g;
-    long long rowi = tok;
-    if (p.x_K > 0) {
-      const int b = tok / p.x_K, r = tok % p.x_K;
-      rowi = r < p.x_F ? (long long)b * p.x_F + r : p.x_mask_row;
-    }
-    xh[n] = p.x_hi + rowi * p.ldx;
+  __syncthreads();
+  {
+    GemmEpi<NT, NW> epi{p, red, s_done, c, (int)(u0 / p.s.KR), 0};
+    stream_units<NT, HAS_LO, PF, NW, RB, FULL>(p.s, u0, u1, red, epi);
   }
-
-  RowCursor ld, cp;
-  ld.tile = cp.tile = tile_first;
-  ld.ks = cp.ks = (int)(u0 - (long long)tile_first * p.SK);
-  ld.set_tile(p, warp, g);
-  cp.set_tile(p, warp, g);
-
-  auto issue = [&](uint4(&dst)[4]) {
-    const int ka = ld.ks * 64 + chunk_k0(t), kb = ld.ks * 64 + chunk_k1(t);
-    if (FULL) {
-      dst[0] = ld_stream16(ld.r0 + ka);
-      dst[1] = ld_stream16(ld.r0 + kb);
-      dst[2] = ld_stream16(ld.r1 + ka);
-      dst[3] = ld_stream16(ld.r1 + kb);
-    } else {
-      const bool va = ld.valid && ka < p.Kd, vb = ld.valid && kb < p.Kd;
-      const uint4 z = make_uint4(0, 0, 0, 0);
-      dst[0] = va ? ld_stream16(ld.r0 + ka) : z;
-      dst[1] = vb ? ld_stream16(ld.r0 + kb) : z;
-      dst[2] = va ? ld_stream16(ld.r1 + ka) : z;
-      dst[3] = vb ? ld_stream16(ld.r1 + kb) : z;
-    }
-    ld.advance(p, warp, g);
-  };
-
-#pragma unroll
-  for (int s = 0; s < PF; ++s)
-    if (u0 + s < u1) issue(a[s]);
-
-  for (long long u = u0; u < u1; u += PF) {
-#pragma unroll
-    for (int s = 0; s < PF; ++s) {
-      if (u + s < u1) {
-        const int ka = cp.ks * 64 + chunk_k0(t), kb = cp.ks * 64 + chunk_k1(t);
-        const bool kval = ka < p.Kd, kval2 = kb < p.Kd;
-        const uint32_t w0[8] = {a[s][0].x, a[s][0].y, a[s][0].z, a[s][0].w, a[s][1].x, a[s][1].y, a[s][1].z, a[s][1].w};
-        const uint32_t w1[8] = {a[s][2].x, a[s][2].y, a[s][2].z, a[s][2].w, a[s][3].x, a[s][3].y, a[s][3].z, a[s][3].w};
-#pragma unroll
-        for (int n = 0; n < NT; ++n) {
-          const int tok = n * 8 + g;
-          uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0, l0 = h0, l1 = h0;
-          const bf16* xp = xh[n] + cp.xoff;
-          const bf16* xq = xp + xlo_delta;
-          if (FULL) {
-            h0 = ld_act16(xp + ka);
-            h1 = ld_act16(xp + kb);
-            if (HAS_LO) { l0 = ld_act16(xq + ka); l1 = ld_act16(xq + kb); }
-          } else if (tok < p.M) {
-            if (kval) {
-              h0 = ld_act16(xp + ka);
-              if (HAS_LO) l0 = ld_act16(xq + ka);
-            }
-            if (kval2) {
-              h1 = ld_act16(xp + kb);
-              if (HAS_LO) l1 = ld_act16(xq + kb);
-            }
-          }
-          const uint32_t xhv[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
-          const uint32_t xlv[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            mma_bf16_16816(acc[n], w0[2 * j], w1[2 * j], w0[2 * j + 1], w1[2 * j + 1], xhv[2 * j], xhv[2 * j + 1]);
-            if (HAS_LO)
-              mma_bf16_16816(acc[n], w0[2 * j], w1[2 * j], w0[2 * j + 1], w1[2 * j + 1], xlv[2 * j], xlv[2 * j + 1]);
-          }
-        }
-        if (u + s + PF < u1) issue(a[s]);
-        const bool tile_end = (cp.ks == p.SK - 1) || (u + s == u1 - 1);
-        if (tile_end) {
-          if (cp.valid) {
-            float* dst = p.part + (((size_t)c * p.slots + (cp.tile - tile_first)) * 128 + warp * 16) * MP;
-#pragma unroll
-            for (int n = 0; n < NT; ++n) {
-              *reinterpret_cast<float2*>(dst + (size_t)g * MP + n * 8 + 2 * t) = make_float2(acc[n][0], acc[n][1]);
-              *reinterpret_cast<float2*>(dst + (size_t)(g + 8) * MP + n * 8 + 2 * t) = make_float2(acc[n][2], acc[n][3]);
-            }
-          }
-#pragma unroll
-          for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-          // ticket: the CTA that completes the tile (pair) runs the fused epilogue
-          const int group = p.pair_offset > 0 ? cp.tile % p.pair_offset : cp.tile;
-          __threadfence();
-          __syncthreads();
-          if (threadIdx.x == 0) s_last = (atomicAdd(&p.ctr[group], 1) == p.expected[group] - 1);
-          __syncthreads();
-          if (s_last) {
-            __threadfence();
-            finalize_group(p, group, MP, sh, s_rstd);
-            if (threadIdx.x == 0) p.ctr[group] = 0;
-          }
-        }
-        cp.advance(p, warp, g);
-      }
-    }
+  __syncthreads();
+  // fused finalize of the groups this CTA completed (the streaming buffers are free now)
+  const int n_done = s_done[0];
+  GroupMeta* gm = reinterpret_cast<GroupMeta*>(red);
+  float* s_part = reinterpret_cast<float*>(gm + 1);
+  for (int i = 0; i < n_done; ++i) {
+    const int group = s_done[1 + i];
+    __threadfence();
+    finalize_group(p, group, 8 * NT, sh, s_rstd, gm, s_part);
+    if (threadIdx.x == 0) p.ctr[group] = 0;
+    __syncthreads();
   }
 }
 
@@ -382,30 +327,39 @@ cudaError_t launch_mask_row(const bf16* mask_vec, const bf16* norm_g, const bf16
 
 template <int NT, bool HAS_LO, int PF>
 static cudaError_t launch_t(const GemmArgs& a, int grid, bool full, cudaStream_t st) {
-  if (full)
-    gemm_rows_kernel<NT, HAS_LO, PF, true><<<grid, 256, 0, st>>>(a);
-  else
-    gemm_rows_kernel<NT, HAS_LO, PF, false><<<grid, 256, 0, st>>>(a);
+  constexpr int RB = (NT <= 4) ? 2 : 1;
+  const size_t smem = (size_t)RB * 16 * 16 * 8 * NT * sizeof(float);
+  cudaError_t e;
+  if (full) {
+    if (smem > 48 * 1024 && (e = cudaFuncSetAttribute(gemm_rows_kernel<NT, HAS_LO, PF, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    gemm_rows_kernel<NT, HAS_LO, PF, true><<<grid, 512, smem, st>>>(a);
+  } else {
+    if (smem > 48 * 1024 && (e = cudaFuncSetAttribute(gemm_rows_kernel<NT, HAS_LO, PF, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    gemm_rows_kernel<NT, HAS_LO, PF, false><<<grid, 512, smem, st>>>(a);
+  }
   return cudaGetLastError();
 }
 
 cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const EpiArgs& epi, float* part, cudaStream_t st) {
   GemmArgs a;
-  for (int i = 0; i < 6; ++i) a.seg[i] = plan.seg[i < plan.nseg ? i : 0];
-  a.nseg = plan.nseg;
-  a.Kd = plan.Kd; a.SK = plan.SK; a.slots = plan.slots; a.U = plan.U;
-  a.x_hi = in.x_hi; a.x_lo = in.x_lo != nullptr ? in.x_lo : in.x_hi; a.ldx = in.ldx; a.M = in.M;
-  a.x_K = in.x_K; a.x_F = in.x_F; a.x_mask_row = in.x_mask_row;
-  a.part = part; a.first_tile = plan.d_first_tile; a.clo = plan.d_tile_clo; a.chi = plan.d_tile_chi;
+  for (int i = 0; i < 6; ++i) a.s.seg[i] = plan.seg[i < plan.nseg ? i : 0];
+  a.s.nseg = plan.nseg;
+  a.s.Kd = plan.Kd; a.s.SK = plan.SK; a.s.KR = plan.KR; a.slots = plan.slots; a.U = plan.U;
+  a.s.x_hi = in.x_hi; a.s.x_lo = in.x_lo != nullptr ? in.x_lo : in.x_hi; a.s.ldx = in.ldx; a.s.M = in.M;
+  a.s.x_K = in.x_K; a.s.x_F = in.x_F; a.s.x_mask_row = in.x_mask_row;
+  a.part = part; a.first_mt = plan.d_first_mt; a.clo = plan.d_mt_clo; a.chi = plan.d_mt_chi;
   a.ctr = plan.d_ctr; a.expected = plan.d_expected; a.pair_offset = plan.pair_offset;
   a.epi = epi;
   const int MP = padded_tokens(in.M);
   const bool lo = in.x_lo != nullptr;
-  bool full = (plan.Kd % 64 == 0) && (in.M == MP);
+  bool full = (plan.Kd % 1024 == 0);   // padded token rows are harmless: they read row 0 and are never used
   for (int i = 0; i < plan.nseg; ++i) full = full && (plan.seg[i].rows % 128 == 0);
-  if (MP == 8) return lo ? launch_t<1, true, 4>(a, plan.grid, full, st) : launch_t<1, false, 4>(a, plan.grid, full, st);
+  #ifndef DART_GEMM_PF
+#define DART_GEMM_PF 1
+#endif
+  if (MP == 8) return lo ? launch_t<1, true, DART_GEMM_PF>(a, plan.grid, full, st) : launch_t<1, false, DART_GEMM_PF>(a, plan.grid, full, st);
   if (MP == 32) return lo ? launch_t<4, true, 2>(a, plan.grid, full, st) : launch_t<4, false, 2>(a, plan.grid, full, st);
-  return lo ? launch_t<16, true, 2>(a, plan.grid, full, st) : launch_t<16, false, 2>(a, plan.grid, full, st);
+  return lo ? launch_t<16, true, 1>(a, plan.grid, full, st) : launch_t<16, false, 1>(a, plan.grid, full, st);
 }
 
 }  // namespace dart

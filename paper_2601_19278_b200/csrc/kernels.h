@@ -26,16 +26,17 @@ struct GemmPlan {
   int nseg;
   GemmSeg seg[6];
   int Kd;           // reduction length per segment, multiple of 16
-  int SK;           // ceil(Kd / 64) k-steps per tile
-  int n_tiles;      // 128-row tiles over all segments
+  int SK;           // ceil(Kd / 64) k-steps per row
+  int KR;           // ceil(SK / 16) k-rounds per 16-row tile (16 warps take one k-step each)
+  int n_tiles;      // 128-row tiles over all segments (8 16-row tiles each)
   int grid;         // CTAs
-  int slots;        // max tiles a CTA touches
-  long long U;      // n_tiles * SK
+  int slots;        // max 16-row tiles a CTA touches
+  long long U;      // n_tiles * 8 * KR work units
   int pair_offset;  // > 0: tiles T and T + pair_offset are finalized together (group = T % pair_offset)
   int n_groups;
-  int* d_tile_clo;    // DEVICE [n_tiles] first CTA contributing to a tile
-  int* d_tile_chi;    // DEVICE [n_tiles] last CTA contributing to a tile
-  int* d_first_tile;  // DEVICE [grid]    first tile of a CTA's range
+  int* d_mt_clo;      // DEVICE [n_tiles*8] first CTA contributing to a 16-row tile
+  int* d_mt_chi;      // DEVICE [n_tiles*8] last CTA contributing to a 16-row tile
+  int* d_first_mt;    // DEVICE [grid]      first 16-row tile of a CTA's range
   int* d_ctr;         // DEVICE [n_groups] tickets taken (zero between launches)
   int* d_expected;    // DEVICE [n_groups] tickets that complete a group
 };
@@ -76,13 +77,26 @@ struct EpiArgs {
   bf16* q_hi; bf16* q_lo; bf16* k_new; bf16* v_new; bf16* k_cache; bf16* v_cache; long long P_cap;
 };
 
+// What the shared streaming core (stream_core.cuh) needs to know about a launch.
+struct StreamArgs {
+  GemmSeg seg[6];     // sub-matrices streamed by this launch; tile0 in 128-row tiles
+  int nseg;
+  int Kd;             // reduction length (multiple of 16)
+  int SK;             // 64-wide k-steps per row
+  int KR;             // k-rounds per 16-row tile = ceil(SK / warps per CTA)
+  const bf16* x_hi;   // activations [rows, ldx] hi part
+  const bf16* x_lo;   // lo part (== x_hi when the input is plain bf16)
+  long long ldx;
+  int M;              // valid token rows
+  int x_K, x_F;       // x_K > 0: token (b, r) reads row b*x_F + r if r < x_F, else row x_mask_row
+  long long x_mask_row;
+};
+
 struct GemmArgs {
-  GemmSeg seg[6];
-  int nseg, Kd, SK, slots;
+  StreamArgs s;
+  int slots;
   long long U;
-  const bf16* x_hi; const bf16* x_lo; long long ldx; int M;
-  int x_K, x_F; long long x_mask_row;
-  float* part; const int* first_tile; const int* clo; const int* chi;
+  float* part; const int* first_mt; const int* clo; const int* chi;
   int* ctr; const int* expected; int pair_offset;
   EpiArgs epi;
 };
@@ -114,6 +128,7 @@ cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, cuda
 // LM head with fused log-softmax / top-k partials, and the merge that finishes them.
 // ---------------------------------------------------------------------------------------------
 struct LmParams {
+  StreamArgs s;  // filled by launch_lm_head
   const bf16* W; int V; int Kd;
   const bf16* x_hi; const bf16* x_lo; long long ldx; int M; int K;  // token m = b*K + r
   const float* ss_in; int ss_tiles; int ss_mp; float rms_eps;  // final RMSNorm's 1/rms, applied to the logits
