@@ -59,7 +59,7 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 }
 
 template <int DH>
-__global__ void __launch_bounds__(128) attn_splitkv_kernel(const AttnArgs a) {
+__global__ void __launch_bounds__(128) attn_splitkv_kernel(const __grid_constant__ AttnArgs a) {
   const AttnParams& p = a.p;
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int TILE_BYTES = 64 * DH * 2;
@@ -70,6 +70,7 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const AttnArgs a) {
   unsigned char* Vs = smem + 4 * TILE_BYTES;
 
   const int ci = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  pdl_wait();
   const int P = p.seq_lens[b];
   const int n_cc = (P + p.chunk_keys - 1) / p.chunk_keys;  // cache chunks of this sequence
   if (ci > n_cc) return;
@@ -246,6 +247,7 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const AttnArgs a) {
 __global__ void attn_combine_kernel(const AttnArgs a) {
   const AttnParams& p = a.p;
   const int m = blockIdx.x, j = blockIdx.y, d = threadIdx.x, dh = p.dh;
+  pdl_wait();
   const int b = m / p.K, r = m % p.K, G = p.Hq / p.Hkv, hk = j / G, rr = (j % G) * p.K + r;
   const int n_chunks = a.chunk_base[b + 1] - a.chunk_base[b];
   float mx = -INFINITY;
@@ -286,15 +288,14 @@ cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, cuda
   }
   a.chunk_base[p.B] = base;
   dim3 grid(max_chunks, p.Hkv, p.B);
+  cudaError_t e;
   if (p.dh == 128)
-    attn_splitkv_kernel<128><<<grid, 128, 6 * 64 * 128 * 2, st>>>(a);
+    e = launch_pdl(attn_splitkv_kernel<128>, grid, dim3(128), (size_t)6 * 64 * 128 * 2, st, a);
   else
-    attn_splitkv_kernel<64><<<grid, 128, 6 * 64 * 64 * 2, st>>>(a);
-  cudaError_t e = cudaGetLastError();
+    e = launch_pdl(attn_splitkv_kernel<64>, grid, dim3(128), (size_t)6 * 64 * 64 * 2, st, a);
   if (e != cudaSuccess) return e;
   dim3 cgrid(p.B * p.K, p.Hq);
-  attn_combine_kernel<<<cgrid, p.dh, 0, st>>>(a);
-  return cudaGetLastError();
+  return launch_pdl(attn_combine_kernel, cgrid, dim3(p.dh), 0, st, a);
 }
 
 }  // namespace dart

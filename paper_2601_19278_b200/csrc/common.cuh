@@ -91,6 +91,18 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1
   return c;
 }
 
+// Programmatic dependent launch.  Every kernel of the step is launched with the programmatic-stream-
+// serialization attribute.  A kernel calls pdl_wait() before it touches anything an earlier kernel
+// produced or may still be reading -- in the streaming kernels that is after the first weight loads have
+// been issued -- and pdl_trigger() once its main work is done (before its epilogue), so that the next
+// kernel's blocks are scheduled onto SMs as they drain and start their own weight stream early.
+// pdl_wait() returns once the predecessor grid has completed and its writes are visible; since every
+// kernel waits before it completes, completion is transitive along the stream.
+// (Measured on B200: triggering at kernel *start* instead doubled the step time -- the early-launched
+// successors crowd the running kernel -- so the trigger comes late.)
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Device status word values (mirrors dart_status for the device-detectable errors).
 enum : int { DEV_OK = 0, DEV_TIMEOUT = -5 };
 

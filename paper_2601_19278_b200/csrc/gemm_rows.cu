@@ -245,6 +245,7 @@ struct GemmEpi {
     const int tile = mt >> 3;
     return p.pair_offset > 0 ? tile % p.pair_offset : tile;
   }
+  __device__ __forceinline__ void after_wait() {}
   __device__ __forceinline__ void mtile_done(int mt, int buf, bool last) {
     float* dst = p.part + ((size_t)c * p.slots + (mt - first_mt)) * 16 * MP;
     for (int e = threadIdx.x; e < 16 * MP; e += blockDim.x) dst[e] = red_sum<NW, MP>(red, buf, e / MP, e % MP);
@@ -273,15 +274,17 @@ __global__ void __launch_bounds__(512, (NT == 1 ? 2 : 1)) gemm_rows_kernel(const
   __shared__ int s_done[kMaxDone + 2];
   const int c = blockIdx.x, G = gridDim.x;
   if (threadIdx.x == 0) s_done[0] = 0;
-  if (p.epi.mode == EPI_FC && c < p.s.M) embed_rows(p, sh);
   const long long u0 = ((long long)c * p.U) / G, u1 = ((long long)(c + 1) * p.U) / G;
-  if (u0 >= u1) return;
   __syncthreads();
-  {
+  if (u0 < u1) {
     GemmEpi<NT, NW> epi{p, red, s_done, c, (int)(u0 / p.s.KR), 0};
     stream_units<NT, HAS_LO, PF, NW, RB, FULL>(p.s, u0, u1, red, epi);
+  } else {
+    pdl_wait();
   }
+  pdl_trigger();
   __syncthreads();
+  if (p.epi.mode == EPI_FC && c < p.s.M) embed_rows(p, sh);
   // fused finalize of the groups this CTA completed (the streaming buffers are free now)
   const int n_done = s_done[0];
   GroupMeta* gm = reinterpret_cast<GroupMeta*>(red);
@@ -332,12 +335,11 @@ static cudaError_t launch_t(const GemmArgs& a, int grid, bool full, cudaStream_t
   cudaError_t e;
   if (full) {
     if (smem > 48 * 1024 && (e = cudaFuncSetAttribute(gemm_rows_kernel<NT, HAS_LO, PF, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    gemm_rows_kernel<NT, HAS_LO, PF, true><<<grid, 512, smem, st>>>(a);
+    return launch_pdl(gemm_rows_kernel<NT, HAS_LO, PF, true>, dim3(grid), dim3(512), smem, st, a);
   } else {
     if (smem > 48 * 1024 && (e = cudaFuncSetAttribute(gemm_rows_kernel<NT, HAS_LO, PF, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    gemm_rows_kernel<NT, HAS_LO, PF, false><<<grid, 512, smem, st>>>(a);
+    return launch_pdl(gemm_rows_kernel<NT, HAS_LO, PF, false>, dim3(grid), dim3(512), smem, st, a);
   }
-  return cudaGetLastError();
 }
 
 cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const EpiArgs& epi, float* part, cudaStream_t st) {

@@ -8,6 +8,22 @@ namespace dart {
 
 typedef __nv_bfloat16 bf16;
 
+// Launch with programmatic stream serialization (see pdl_wait / pdl_trigger in common.cuh).
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Weight-streaming small-M GEMM:  y = W[rows, Kd] * x[M, Kd]^T, split over the flattened
 // (128-row tile, 64-wide k-step) space so that every CTA streams the same number of weight bytes.

@@ -45,8 +45,19 @@ struct LmEpi {
   const LmParams& p;
   const float* red;
   float* stage;   // [MP][SROW]
-  float* st_key; float* st_y; int* st_id; float* st_ms; const float* s_rstd;
+  float* st_key; float* st_y; int* st_id; float* st_ms; float* s_rstd;
   int mt0;
+
+  // the final RMSNorm's per-token 1/rms comes from the previous kernel's sums of squares
+  __device__ __forceinline__ void after_wait() {
+    for (int i = threadIdx.x; i < MP; i += NW * 32) {
+      float ssq = 0.f;  // the activations are x * gain; their 1/rms multiplies the logits (same fixed order everywhere)
+      if (i < p.M)
+        for (int tl = 0; tl < p.ss_tiles; ++tl) ssq += p.ss_in[(size_t)tl * p.ss_mp + i];
+      s_rstd[i] = i < p.M ? 1.f / sqrtf(ssq / (float)p.Kd + p.rms_eps) : 0.f;
+    }
+    __syncthreads();
+  }
 
   __device__ __forceinline__ void mtile_done(int mt, int buf, bool last) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -116,7 +127,7 @@ struct LmEpi {
 // FULL: Kd is a multiple of 64*NW and all rows/tokens are in range, so the streaming loop carries no
 // bounds predicates at all.
 template <int NT, int PF, int NW, bool FULL>
-__global__ void __launch_bounds__(NW * 32, (NT == 1 ? 2 : 1)) lm_head_kernel(const LmParams p) {
+__global__ void __launch_bounds__(NW * 32, (NT == 1 ? 2 : 1)) lm_head_kernel(const __grid_constant__ LmParams p) {
   constexpr int MP = 8 * NT;
   constexpr int RB = (NT <= 4) ? 2 : 1;      // reduce buffers
   constexpr int SROW = 128 + 1;
@@ -137,17 +148,16 @@ __global__ void __launch_bounds__(NW * 32, (NT == 1 ? 2 : 1)) lm_head_kernel(con
   for (int i = tid; i < MP; i += NW * 32) {
     st_ms[2 * i] = -INFINITY;
     st_ms[2 * i + 1] = 0.f;
-    float ssq = 0.f;  // the activations are x * gain; their 1/rms multiplies the logits (same fixed order everywhere)
-    if (i < p.M)
-      for (int tl = 0; tl < p.ss_tiles; ++tl) ssq += p.ss_in[(size_t)tl * p.ss_mp + i];
-    s_rstd[i] = i < p.M ? 1.f / sqrtf(ssq / (float)p.Kd + p.rms_eps) : 0.f;
   }
   __syncthreads();
 
   if (mt1 > mt0) {
     LmEpi<NT, NW> epi{p, red, stage, st_key, st_y, st_id, st_ms, s_rstd, mt0};
     stream_units<NT, true, PF, NW, RB, FULL>(p.s, (long long)mt0 * p.s.KR, (long long)mt1 * p.s.KR, red, epi);
+  } else {
+    pdl_wait();
   }
+  pdl_trigger();
   __syncthreads();
   for (int i = tid; i < MP * 32; i += NW * 32) {
     const size_t o = (size_t)c * MP * 32 + i;
@@ -172,8 +182,7 @@ static cudaError_t launch_lm_t(LmParams& p, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(lm_head_kernel<NT, PF, NW, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  lm_head_kernel<NT, PF, NW, FULL><<<p.grid, NW * 32, smem, st>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(lm_head_kernel<NT, PF, NW, FULL>, dim3(p.grid), dim3(NW * 32), smem, st, p);
 }
 
 cudaError_t launch_lm_head(const LmParams& pin, cudaStream_t st) {

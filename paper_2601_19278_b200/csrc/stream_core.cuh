@@ -41,7 +41,8 @@ struct UnitCursor {
   }
 };
 
-// Streams units [u0, u1) of the flattened (m-tile, k-round) space.  `epi.mtile_done(mt, buf, last)` is
+// Streams units [u0, u1) of the flattened (m-tile, k-round) space.  `epi.after_wait()` is called by every
+// thread once the predecessor kernel has completed (it may contain CTA-wide barriers).  `epi.mtile_done(mt, buf, last)` is
 // called by every thread of the CTA after the partial tiles of m-tile `mt` have been written to
 // red[buf] = [NW][16 rows][MP tokens] (RB buffers) and a __syncthreads(); it may contain further CTA-wide barriers.
 // FULL: Kd is a multiple of 64*NW, every m-tile is valid and all MP token rows exist.
@@ -106,6 +107,9 @@ __device__ __forceinline__ void stream_units(const StreamArgs& a, long long u0, 
 #pragma unroll
   for (int s = 0; s < PF; ++s)
     if (s < n) issue(wreg[s]);
+  // the weights above depend on no earlier kernel; everything below (activations, partials) does
+  pdl_wait();
+  epi.after_wait();
 
   int buf = 0;
   for (int u = 0; u < n; u += PF) {

@@ -29,6 +29,7 @@ __global__ void __launch_bounds__(1024) topk_merge_kernel(const LmParams p) {
   __shared__ float s_thr_key;
   __shared__ int s_thr_id, s_nsurv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
+  pdl_wait();
 
   for (int i = tid; i < G * 32; i += nthr) {
     const int c = i >> 5, e = i & 31;
@@ -114,8 +115,7 @@ cudaError_t topk_merge_setup(int max_grid) {
 }
 
 cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st) {
-  topk_merge_kernel<<<p.M, 1024, merge_smem(p.grid), st>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(topk_merge_kernel, dim3(p.M), dim3(1024), merge_smem(p.grid), st, p);
 }
 
 }  // namespace dart

@@ -12,16 +12,15 @@
 //     so all of them are looked up in one parallel sweep before the level loop; inside the
 //     loop each candidate needs one trigram probe, whose context only exists once the
 //     previous level's beam is known;
-//   * top-w and top-theta use ranks, not sorts.  Every warp sorts its 32 candidates with a
-//     shuffle bitonic network (total order: score desc, generation index asc).  A threshold
-//     entry T is then taken from the runs' p-th entries: T = the m-th best of them with
-//     m * (p + 1) >= theta, so at least theta candidates are not after T.  Only those
-//     "survivors" (each run contributes a prefix; typically ~90 of 500) are ranked, by
-//     counting the survivors that precede each one.  Ranks are unique, so "rank r < w" *is*
-//     beam slot r and "rank r < theta" is the level's r-th finalist, with no dependence on
-//     thread timing;
-//   * the final top-theta only needs each level's theta best nodes (by ancestor-clamped
-//     score): at most levels * theta finalists, ranked by the same counting.
+//   * selection is a bitonic merge tree held in registers.  Every warp sorts its 32 candidates
+//     with a shuffle network (total order: score desc, generation index asc); pairs of warps
+//     then merge their runs, keeping the best 64 (two per lane): C[p] = better(A[p], B[63-p])
+//     is a bitonic sequence holding the best 64 of A and B, which six compare-exchange stages
+//     sort.  After log2(warps) rounds warp 0 holds the level's best 64 in order: the first w
+//     are the next beam (w <= 32).  There are no data-dependent loops and the result does
+//     not depend on thread timing;
+//   * the final top-theta (theta <= 63) is kept the same way: warp 0 merges each level's best
+//     64 (by ancestor-clamped score, node index asc) into a running global best 64.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -46,72 +45,120 @@ __device__ __forceinline__ bool probe_rest(const NgramTable& T, unsigned long lo
   return false;
 }
 
-// (score, index) total order: a strictly precedes b
-__device__ __forceinline__ bool before(float sa, int ia, float sb, int ib) { return sa > sb || (sa == sb && ia < ib); }
+// A candidate as one 64-bit key whose unsigned order is the total order (score desc, index asc):
+// high word = the score's bits mapped so that larger floats give larger integers (-0 is first folded
+// into +0, so that equal scores compare equal), low word = ~index.  The larger key precedes.
+typedef unsigned long long Key;
+constexpr Key kPadKey = 0ull;  // below every real key: (-inf score would map above 0; index bits of a pad are 0)
 
-// Sort one value per lane so that lane 0 holds the entry that precedes all others.
-__device__ __forceinline__ void warp_sort(float& s, int& c, int lane) {
+__device__ __forceinline__ Key make_key(float s, int c) {
+  uint32_t u = __float_as_uint(s + 0.0f);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return ((Key)u << 32) | (Key)(~(uint32_t)c);
+}
+__device__ __forceinline__ int key_index(Key k) { return (int)(~(uint32_t)k); }
+__device__ __forceinline__ Key shfl_key(Key k, int src) { return __shfl_sync(0xffffffffu, k, src); }
+__device__ __forceinline__ Key kmax(Key a, Key b) { return a > b ? a : b; }
+__device__ __forceinline__ Key kmin(Key a, Key b) { return a > b ? b : a; }
+
+// Sort one key per lane so that lane 0 holds the largest.
+__device__ __forceinline__ void warp_sort(Key& x, int lane) {
 #pragma unroll
   for (int k = 2; k <= 32; k <<= 1) {
 #pragma unroll
     for (int j = k >> 1; j > 0; j >>= 1) {
-      const float os = __shfl_xor_sync(0xffffffffu, s, j);
-      const int oc = __shfl_xor_sync(0xffffffffu, c, j);
+      const Key o = shfl_key(x, lane ^ j);
       const bool up = (lane & k) == 0, lower = (lane & j) == 0;
-      const bool mine_first = before(s, c, os, oc);
-      const bool keep = (lower == up) ? mine_first : !mine_first;
-      if (!keep) { s = os; c = oc; }
+      x = (lower == up) ? kmax(x, o) : kmin(x, o);
     }
   }
 }
 
-// number of entries of a sorted 32-entry run that precede (s, c)
-__device__ __forceinline__ int count_before(const float* rs, const int* rc, float s, int c) {
-  int cnt = 0;
+// (x0, x1) hold a bitonic sequence of 64 keys (position p = 32*reg + lane); sort it, largest first.
+__device__ __forceinline__ void bitonic_merge64(Key& x0, Key& x1, int lane) {
+  const Key hi = kmax(x0, x1), lo = kmin(x0, x1);
+  x0 = hi;
+  x1 = lo;
 #pragma unroll
-  for (int step = 32; step > 0; step >>= 1)
-    if (cnt + step <= 32 && before(rs[cnt + step - 1], rc[cnt + step - 1], s, c)) cnt += step;
-  return cnt;
+  for (int j = 16; j > 0; j >>= 1) {
+    const bool lower = (lane & j) == 0;
+    const Key o0 = shfl_key(x0, lane ^ j), o1 = shfl_key(x1, lane ^ j);
+    x0 = lower ? kmax(x0, o0) : kmin(x0, o0);
+    x1 = lower ? kmax(x1, o1) : kmin(x1, o1);
+  }
+}
+
+// Merge the sorted 64-key run (y0, y1) of the same warp into (x0, x1), keeping the best 64 sorted.
+__device__ __forceinline__ void merge_keep64(Key& x0, Key& x1, Key y0, Key y1, int lane) {
+  const Key r0 = shfl_key(y1, 31 - lane), r1 = shfl_key(y0, 31 - lane);  // y reversed: y[63 - p]
+  x0 = kmax(x0, r0);
+  x1 = kmax(x1, r1);
+  bitonic_merge64(x0, x1, lane);
 }
 
 struct TreeSmem {
   float* n_score; float* n_clamp; int* n_tok; int* n_par; unsigned char* n_j;
-  float* bg; float* run_s; int* run_c; float* sv_s; int* sv_c; int* beam_a; int* beam_b; int* fin; int* sel; int* par_out; int* lvl_base;
+  float* bg; Key* xk; int* beam_a; int* beam_b; int* sel; int* par_out; int* lvl_base;
 };
 
 __host__ __device__ inline size_t tree_layout(int k, int w, int budget, int L, unsigned char* base, TreeSmem* t) {
   const int n_max = 1 + k + (L - 1) * w * k;
-  const int theta = budget - 1;
   size_t o = 0;
   auto take = [&](size_t bytes) { const size_t r = o; o += (bytes + 15) & ~size_t(15); return r; };
   const size_t o_score = take((size_t)n_max * 4), o_clamp = take((size_t)n_max * 4), o_tok = take((size_t)n_max * 4),
                o_par = take((size_t)n_max * 4), o_j = take((size_t)n_max), o_bg = take((size_t)(k + (L - 1) * k * k) * 4),
-               o_rs = take(32 * 32 * 4), o_rc = take(32 * 32 * 4), o_ss = take(1024 * 4), o_sc = take(1024 * 4), o_ba = take((size_t)w * 4), o_bb = take((size_t)w * 4),
-               o_fin = take((size_t)L * theta * 4), o_sel = take((size_t)budget * 4), o_po = take((size_t)budget * 4),
-               o_lb = take((size_t)(L + 1) * 4);
+               o_xk = take(32 * 64 * 8), o_ba = take((size_t)w * 4), o_bb = take((size_t)w * 4),
+               o_sel = take((size_t)(budget + 1) * 4), o_po = take((size_t)budget * 4), o_lb = take((size_t)(L + 1) * 4);
   if (t != nullptr) {
     t->n_score = reinterpret_cast<float*>(base + o_score); t->n_clamp = reinterpret_cast<float*>(base + o_clamp);
     t->n_tok = reinterpret_cast<int*>(base + o_tok); t->n_par = reinterpret_cast<int*>(base + o_par);
     t->n_j = base + o_j; t->bg = reinterpret_cast<float*>(base + o_bg);
-    t->run_s = reinterpret_cast<float*>(base + o_rs); t->run_c = reinterpret_cast<int*>(base + o_rc);
-    t->sv_s = reinterpret_cast<float*>(base + o_ss); t->sv_c = reinterpret_cast<int*>(base + o_sc);
+    t->xk = reinterpret_cast<Key*>(base + o_xk);
     t->beam_a = reinterpret_cast<int*>(base + o_ba); t->beam_b = reinterpret_cast<int*>(base + o_bb);
-    t->fin = reinterpret_cast<int*>(base + o_fin); t->sel = reinterpret_cast<int*>(base + o_sel);
+    t->sel = reinterpret_cast<int*>(base + o_sel);
     t->par_out = reinterpret_cast<int*>(base + o_po); t->lvl_base = reinterpret_cast<int*>(base + o_lb);
   }
   return o;
 }
 
-__global__ void __launch_bounds__(1024) tree_kernel(const TreeParams p) {
+// Best 64 of the block's candidates (one key per thread; pads are kPadKey), sorted, in warp 0's (x0, x1).
+// `pred` is OR-reduced over the block in the first barrier and returned.  nruns = warps that hold
+// candidates.  All threads of the block must call this.
+__device__ __forceinline__ int block_best64(Key key, int nruns, const TreeSmem& m, int pred, Key& x0, Key& x1) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  warp_sort(key, lane);
+  x0 = key;
+  x1 = kPadKey;
+  int any = 0;
+  bool first = true;
+  for (int stride = 1; stride < nruns || first; stride <<= 1) {
+    const bool donor = (warp & (2 * stride - 1)) == stride && warp < nruns;
+    if (donor) {
+      m.xk[warp * 64 + lane] = x0;
+      m.xk[warp * 64 + 32 + lane] = x1;
+    }
+    if (first) { any = __syncthreads_or(pred); first = false; } else __syncthreads();
+    if ((warp & (2 * stride - 1)) == 0 && warp + stride < nruns) {
+      const int pw = (warp + stride) * 64;
+      x0 = kmax(x0, m.xk[pw + 63 - lane]);
+      x1 = kmax(x1, m.xk[pw + 31 - lane]);
+      bitonic_merge64(x0, x1, lane);
+    }
+  }
+  return any;
+}
+
+// MAXT: launch bound (512 leaves the compiler twice the registers; 1024 covers beam * topk up to 1024)
+template <int MAXT>
+__global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
   extern __shared__ __align__(16) unsigned char tsm[];
   const int k = p.topk, w = p.beam, L = p.n_levels, theta = p.budget - 1;
   TreeSmem m;
   tree_layout(k, w, p.budget, L, tsm, &m);
-  __shared__ int s_nsurv, s_thr_c;
-  __shared__ float s_thr_s;
   __shared__ unsigned long long s_bits[64];
 
-  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
+  pdl_wait();
   const int* ids = p.ids + ((size_t)b * p.K + p.first_row) * k;
   const float* sl = p.slogit + ((size_t)b * p.K + p.first_row) * k;
   const int ctx0 = p.ctx_tail[2 * b], ctx1 = p.ctx_tail[2 * b + 1];
@@ -122,42 +169,42 @@ __global__ void __launch_bounds__(1024) tree_kernel(const TreeParams p) {
     m.n_score[0] = 0.f; m.n_clamp[0] = INFINITY; m.n_tok[0] = ctx1; m.n_par[0] = -1; m.n_j[0] = 0;
     m.beam_a[0] = 0; m.lvl_base[0] = 1;
   }
-  // ---- every bigram any level can ask for: bg[0][0][jt] = (ctx1, S_0[jt]); bg[i][jb][jt] = (S_{i-1}[jb], S_i[jt])
+  // ---- every bigram any level can ask for: bg[jt] = (ctx1, S_0[jt]); bg[k + (i-1)k^2 + jb*k + jt] = (S_{i-1}[jb], S_i[jt]).
+  // A thread issues the first probe of all its lookups (up to 12) before it resolves any of them.
   {
     const int n_bg = k + (L - 1) * k * k;
-    for (int base = 0; base < n_bg; base += 8 * 1024) {
-      unsigned long long key[8];
-      uint32_t hh[8];
-      NgramSlot first[8];
-      bool want[8];
+    for (int e0 = 0; e0 < n_bg; e0 += 12 * nthr) {
+      Key key[12];
+      uint32_t hh[12];
+      NgramSlot first[12];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int e = base + u * 1024 + tid;
-        want[u] = false;
-        if (e < n_bg && have_table) {
-          int tb, tt;
+      for (int u = 0; u < 12; ++u) {
+        const int e = e0 + u * nthr + tid;
+        int tb = -1, tt = 0;
+        if (e < n_bg) {
           if (e < k) { tb = ctx1; tt = ids[e]; }
-          else { const int r = e - k, i = 1 + r / (k * k), q = r % (k * k); tb = ids[(i - 1) * k + q / k]; tt = ids[i * k + q % k]; }
-          if (tb >= 0) {
-            key[u] = ngram_key(2, -1, tb, tt);
-            hh[u] = (uint32_t)ngram_hash(key[u]) & T.mask;
-            first[u] = load_slot(T.slots + hh[u]);
-            want[u] = true;
-          }
+          else { const int r = e - k, i = r / (k * k), q = r - i * k * k, jb = q / k; tb = ids[i * k + jb]; tt = ids[(i + 1) * k + q - jb * k]; }
         }
+        const bool want = have_table && tb >= 0;
+        key[u] = want ? ngram_key(2, -1, tb, tt) : 0ull;
+        hh[u] = (uint32_t)ngram_hash(key[u]) & T.mask;
+        first[u] = want ? load_slot(T.slots + hh[u]) : NgramSlot{0ull, 0.f, 0u};
       }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int e = base + u * 1024 + tid;
+      for (int u = 0; u < 12; ++u) {
+        const int e = e0 + u * nthr + tid;
         if (e < n_bg) {
-          float sc = p.miss;
-          if (want[u]) { float v; if (probe_rest(T, key[u], hh[u], first[u], v)) sc = v; }
+          float sc = p.miss, v;
+          if (key[u] != 0ull && probe_rest(T, key[u], hh[u], first[u], v)) sc = v;
           m.bg[e] = sc;
         }
       }
     }
   }
   __syncthreads();
+
+  // running global best 64 by (clamped score desc, node index asc); lives in warp 0's registers
+  Key g0 = kPadKey, g1 = kPadKey;
 
   int nb = 1;
   int* beam = m.beam_a;
@@ -187,101 +234,30 @@ __global__ void __launch_bounds__(1024) tree_kernel(const TreeParams p) {
       const int n = base + tid;
       m.n_score[n] = s; m.n_clamp[n] = cl; m.n_tok[n] = t; m.n_par[n] = node; m.n_j[n] = (unsigned char)j;
     }
-    // does any candidate's clamped score differ from its score?  (never, when increments are <= 0)
-    const int differs = __syncthreads_or(tid < ncand && cl != s);
-
-    // ---- ranks by (score desc, generation asc); a second pass on the clamped scores only if they differ
-    const int n_want = theta > w ? theta : w;
-    for (int pass = 0; pass < (differs ? 2 : 1); ++pass) {
-      float key = (pass == 0) ? s : cl;
-      int c = (tid < ncand) ? tid : 0x7fffffff;
-      if (warp < nruns) {
-        warp_sort(key, c, lane);
-        m.run_s[warp * 32 + lane] = key;
-        m.run_c[warp * 32 + lane] = c;
-      }
-      if (tid == 0) s_nsurv = 0;
+    // keys carry the node index base + tid, which orders candidates of one level like tid does
+    // best 64 by score -> next beam; `differs`: some clamped score is not its score (never, when increments <= 0)
+    Key x0, x1;
+    const int differs = block_best64(tid < ncand ? make_key(s, base + tid) : kPadKey, nruns, m, tid < ncand && cl != s, x0, x1);
+    if (warp == 0 && lane < w && x0 != kPadKey) beam_next[lane] = key_index(x0);
+    if (differs) {  // the level's best 64 by clamped score are a different set: select again
       __syncthreads();
-      // threshold: the m-th best of the runs' p-th entries, m * (p + 1) >= n_want
-      // (with too few runs for that, T is the sentinel that nothing is after: everything survives)
-      int mm = (nruns + 1) >> 1;
-      if (mm < ((n_want + 31) >> 5)) mm = (n_want + 31) >> 5;
-      const int pp = (n_want + mm - 1) / mm - 1;
-      if (warp == 0) {
-        float tk = (lane < nruns) ? m.run_s[lane * 32 + pp] : -INFINITY;
-        int tc = (lane < nruns) ? m.run_c[lane * 32 + pp] : 0x7fffffff;
-        warp_sort(tk, tc, lane);
-        if (mm > nruns) { tk = -INFINITY; tc = 0x7fffffff; }
-        if (lane == (mm > nruns ? 0 : mm - 1)) { s_thr_s = tk; s_thr_c = tc; }
-      }
-      __syncthreads();
-      const float ts = s_thr_s;
-      const int tc = s_thr_c;
-      // survivors: entries that are not after T (a prefix of every run)
-      const bool surv = warp < nruns && c != 0x7fffffff && !before(ts, tc, key, c);
-      const unsigned bal = __ballot_sync(0xffffffffu, surv);
-      int off = 0;
-      if (lane == 0 && bal) off = atomicAdd(&s_nsurv, __popc(bal));
-      off = __shfl_sync(0xffffffffu, off, 0);
-      if (surv) {
-        const int slot = off + __popc(bal & ((1u << lane) - 1));
-        m.sv_s[slot] = key;
-        m.sv_c[slot] = c;
-      }
-      __syncthreads();
-      const int ns = s_nsurv;
-      if (surv) {
-        int rank = 0;
-        for (int o = 0; o < ns; ++o) rank += before(m.sv_s[o], m.sv_c[o], key, c);
-        if (pass == 0) {
-          if (rank < w) beam_next[rank] = base + c;
-          if (!differs && rank < theta) m.fin[i * theta + rank] = base + c;
-        } else if (rank < theta) {
-          m.fin[i * theta + rank] = base + c;
-        }
-      }
-      __syncthreads();
+      block_best64(tid < ncand ? make_key(cl, base + tid) : kPadKey, nruns, m, 0, x0, x1);
     }
+    if (warp == 0) merge_keep64(g0, g1, x0, x1, lane);
     if (tid == 0) m.lvl_base[i + 1] = base + ncand;
     __syncthreads();
     nb = ncand < w ? ncand : w;
     int* tmp = beam; beam = beam_next; beam_next = tmp;
   }
 
-  // ---- global top-theta over the per-level finalists (clamped score desc, node index asc)
+  // ---- the selected nodes: the first n_sel entries of the global best 64
   const int total = m.lvl_base[L] - 1;
   const int n_sel = total < theta ? total : theta;
-  {
-    // compact the finalists: level i contributes min(ncand_i, theta) nodes
-    const int i = tid / theta, q = tid - i * theta;
-    bool mine = false;
-    int me = 0;
-    if (i < L) {
-      const int ncand_i = m.lvl_base[i + 1] - m.lvl_base[i];
-      if (q < (ncand_i < theta ? ncand_i : theta)) { mine = true; me = m.fin[tid]; }
-    }
-    if (tid == 0) s_nsurv = 0;
-    __syncthreads();
-    const unsigned bal = __ballot_sync(0xffffffffu, mine);
-    int off = 0;
-    if (lane == 0 && bal) off = atomicAdd(&s_nsurv, __popc(bal));
-    off = __shfl_sync(0xffffffffu, off, 0);
-    float mc = 0.f;
-    if (mine) {
-      const int slot = off + __popc(bal & ((1u << lane) - 1));
-      mc = m.n_clamp[me];
-      m.sv_s[slot] = mc;
-      m.sv_c[slot] = me;
-    }
-    __syncthreads();
-    const int ns = s_nsurv;
-    if (mine) {
-      int rank = 0;
-      for (int o = 0; o < ns; ++o) rank += before(m.sv_s[o], m.sv_c[o], mc, me);
-      if (rank < n_sel) m.sel[rank + 1] = me;
-    }
+  if (warp == 0) {
+    if (lane < n_sel) m.sel[1 + lane] = key_index(g0);
+    if (32 + lane < n_sel) m.sel[33 + lane] = key_index(g1);
+    if (lane == 0) m.sel[0] = 0;
   }
-  if (tid == 0) m.sel[0] = 0;
   __syncthreads();
 
   // ---- outputs
@@ -323,7 +299,7 @@ __global__ void __launch_bounds__(1024) tree_kernel(const TreeParams p) {
   if (tid == 0) p.n_nodes[b] = 1 + n_sel;
   __syncthreads();
   uint8_t* mbase = p.mask + (size_t)b * budget * budget;
-  for (int e = tid; e < budget * budget; e += 1024) {
+  for (int e = tid; e < budget * budget; e += nthr) {
     const int x = e / budget, y = e - x * budget;
     mbase[e] = (uint8_t)((s_bits[x] >> y) & 1ull);
   }
@@ -336,14 +312,23 @@ size_t tree_smem_bytes(int topk, int beam, int budget, int n_levels) {
 cudaError_t tree_setup(int topk, int beam, int budget, int max_levels) {
   const size_t smem = tree_smem_bytes(topk, beam, budget, max_levels);
   if (smem > 48 * 1024)
-    return cudaFuncSetAttribute(tree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  {
+    cudaError_t e = cudaFuncSetAttribute(tree_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(tree_kernel<1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  }
   return cudaSuccess;
 }
 
 cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
   const size_t smem = tree_smem_bytes(p.topk, p.beam, p.budget, p.n_levels);
-  tree_kernel<<<p.B, 1024, smem, st>>>(p);
-  return cudaGetLastError();
+  // one thread per (beam entry, candidate) pair; a smaller block makes every barrier cheaper
+  int need = p.beam * p.topk;
+  if (p.budget > need) need = p.budget;
+  int threads = (need + 31) / 32 * 32;
+  if (threads > 1024) threads = 1024;
+  if (threads <= 512) return launch_pdl(tree_kernel<512>, dim3(p.B), dim3(threads), smem, st, p);
+  return launch_pdl(tree_kernel<1024>, dim3(p.B), dim3(threads), smem, st, p);
 }
 
 }  // namespace dart
