@@ -9,7 +9,8 @@
  * Conventions
  *   - Every pointer is labelled HOST or DEVICE.  Device buffers are caller-owned unless stated.
  *   - bf16 tensors are row-major with the last index fastest; weight matrices are [out, in];
- *     every device pointer must be 16-byte aligned.
+ *     weight pointers and `feats` must be 32-byte aligned (they are read with 256-bit loads), every
+ *     other device pointer 16-byte aligned.
  *   - All GPU work is enqueued on the CUDA stream passed as `void* cuda_stream` (a cudaStream_t;
  *     NULL = the legacy default stream).  dart_draft_step and dart_build_tree do not
  *     synchronise, allocate, or copy between host and device.

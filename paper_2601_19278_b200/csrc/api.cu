@@ -61,6 +61,7 @@ namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 bool aligned16(const void* p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned32(const void* p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 
 bool config_ok(const dart_config* c) {
   if (c == nullptr || c->struct_size != sizeof(dart_config)) return false;
@@ -278,7 +279,7 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
                         weights->w_q, weights->w_k, weights->w_v, weights->w_o, weights->norm_post,
                         weights->w_gate, weights->w_up, weights->w_down, weights->norm_final, weights->w_lm};
   for (int i = 0; i < 15; ++i)
-    if (!aligned16(wp[i])) return DART_ERR_INVALID_ARG;
+    if (!aligned32(wp[i])) return DART_ERR_INVALID_ARG;  // the matrices are streamed with 32-byte loads
   if (ngram != nullptr && ngram->n_rows > 0 &&
       (ngram->order == nullptr || ngram->ctx0 == nullptr || ngram->ctx1 == nullptr || ngram->next == nullptr ||
        ngram->score == nullptr))
@@ -411,7 +412,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   if (B > c.max_batch) return DART_ERR_CAPACITY;
   if (in->seq_lens == nullptr || in->seq_lens_host == nullptr || !aligned16(in->k_cache) || !aligned16(in->v_cache))
     return DART_ERR_INVALID_ARG;
-  if (F > 0 && (!aligned16(in->feats) || in->tokens == nullptr)) return DART_ERR_INVALID_ARG;
+  if (F > 0 && (!aligned32(in->feats) || in->tokens == nullptr)) return DART_ERR_INVALID_ARG;
   if (out->topk_ids == nullptr || out->topk_slogit == nullptr) return DART_ERR_INVALID_ARG;
   long long total_keys = 0;
   for (int b = 0; b < B; ++b) {

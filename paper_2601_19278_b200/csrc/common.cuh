@@ -27,6 +27,24 @@ __device__ __forceinline__ uint4 ld_act16(const void* p) {
   return v;
 }
 
+// 32-byte (256-bit) loads, sm_100: a lane's two 16-byte chunks of a k-step are adjacent (see chunk_k0/1),
+// so one instruction fetches both.  Addresses must be 32-byte aligned.
+struct U8 { uint32_t v[8]; };
+__device__ __forceinline__ U8 ld_stream32(const void* p) {
+  U8 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]), "=r"(r.v[4]), "=r"(r.v[5]), "=r"(r.v[6]), "=r"(r.v[7])
+               : "l"(p));
+  return r;
+}
+__device__ __forceinline__ U8 ld_act32(const void* p) {
+  U8 r;
+  asm volatile("ld.global.ca.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]), "=r"(r.v[4]), "=r"(r.v[5]), "=r"(r.v[6]), "=r"(r.v[7])
+               : "l"(p));
+  return r;
+}
+
 // Element offsets, inside a 64-wide k-step, of the two 16-byte chunks that lane t (= lane & 3)
 // of a quad loads from a weight row (and, identically, from an activation row).  Mode 0: the
 // quad's four lanes take bytes [32t, 32t+16) in one instruction and [32t+16, 32t+32) in the next,

@@ -83,7 +83,7 @@ def test_argument_errors_are_reported_without_a_gpu(binding):
     w = binding.DartWeights()                                          # all NULL pointers
     assert lib.dart_draft_init(C.byref(cfg), C.byref(w), None, C.byref(h)) == binding.DART_ERR_INVALID_ARG
     for n in binding.WEIGHT_NAMES:
-        setattr(w, n, 0x1008)                                          # 8-byte aligned only
+        setattr(w, n, 0x1010)                                          # 16-byte aligned only: 32 are needed
     assert lib.dart_draft_init(C.byref(cfg), C.byref(w), None, C.byref(h)) == binding.DART_ERR_INVALID_ARG
     assert lib.dart_draft_step(None, None, None, None) == binding.DART_ERR_INVALID_ARG
     assert lib.dart_build_tree(None, None, None, None) == binding.DART_ERR_INVALID_ARG
