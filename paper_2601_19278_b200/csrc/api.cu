@@ -30,6 +30,7 @@ struct Workspace {
   bf16 *u_hi = nullptr, *u_lo = nullptr;   // [Mmax, I]
   float *ss_g = nullptr, *ss_1 = nullptr, *ss_2 = nullptr;  // [h/128 tiles][MP] sums of squares per tile
   float* rstd_mask = nullptr;
+  float* bg = nullptr;          // [max_batch][topk + (K-1)*topk^2] bigram scores of the tree builder
   float *o_part = nullptr, *ml_part = nullptr;
   float *lm_stats = nullptr, *lm_key = nullptr, *lm_y = nullptr;
   int32_t* lm_id = nullptr;
@@ -176,6 +177,7 @@ size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_p
   TAKE(ss_1, float*, ht * MPmax * sizeof(float));
   TAKE(ss_2, float*, ht * MPmax * sizeof(float));
   TAKE(rstd_mask, float*, 256);
+  TAKE(bg, float*, (size_t)c.max_batch * (c.topk + (size_t)(c.K - 1) * c.topk * c.topk) * sizeof(float));
   TAKE(o_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * c.head_dim * sizeof(float));
   TAKE(ml_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * 2 * sizeof(float));
   TAKE(lm_stats, float*, (size_t)lm_grid * MPmax * 2 * sizeof(float));
@@ -400,8 +402,8 @@ int dart_draft_destroy(dart_handle* h) {
 int dart_step_launch_count(const dart_handle* h, int batch, int n_fresh) {
   (void)batch;
   if (h == nullptr) return 0;
-  // fc, qkv, attention, combine, o_proj, gate/up, down, lm head, merge (+ tree)
-  return (n_fresh > 0 ? 10 : 9);
+  // fc, qkv, attention, combine, o_proj, gate/up, down, lm head, merge (+ bigram sweep, tree)
+  return (n_fresh > 0 ? 11 : 10);
 }
 
 int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out* out, void* cuda_stream) {
@@ -552,7 +554,7 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
   tp.ids = in->topk_ids; tp.slogit = in->topk_slogit; tp.ctx_tail = in->ctx_tail;
   tp.table.slots = h->ng_slots; tp.table.mask = h->ng_mask; tp.table.max_probe = h->ng_max_probe;
   for (int i = 0; i < 8; ++i) { tp.wl[i] = h->wl[i]; tp.wv[i] = h->wv[i]; }
-  tp.wn = h->wn; tp.miss = h->miss;
+  tp.wn = h->wn; tp.miss = h->miss; tp.bg = h->ws.bg;
   tp.tokens = out->tokens; tp.parents = out->parents; tp.depth = out->depth; tp.mask = out->mask;
   tp.n_nodes = out->n_nodes; tp.scores = out->scores; tp.status = h->ws.status;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

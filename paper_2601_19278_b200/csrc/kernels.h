@@ -169,6 +169,7 @@ struct TreeParams {
   int B, K, topk, beam, budget, first_row, n_levels, ngram_order;
   const int32_t* ids; const float* slogit; const int32_t* ctx_tail;
   NgramTable table;
+  float* bg;   // [B][topk + (n_levels-1)*topk^2] bigram scores (workspace, written by the sweep kernel)
   float wl[8]; float wv[8]; float wn; float miss;
   int32_t* tokens; int32_t* parents; int32_t* depth; uint8_t* mask; int32_t* n_nodes; float* scores;
   int* status;

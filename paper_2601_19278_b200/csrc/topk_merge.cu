@@ -5,107 +5,151 @@
 // (selection key, plain logit y, token id), sorted by (key desc, id asc).  One block per token row:
 //   1. log-sum-exp over the slices (fixed-order reductions, deterministic);
 //   2. all G lists are copied to shared memory with coalesced loads;
-//   3. a threshold T = the topk-th best of the G list *heads* (at least topk entries are >= T, so
-//      the global top-k lies among the entries >= T; each sorted list contributes a prefix);
-//   4. the survivors (typically a few dozen) are ranked by counting how many survivors precede
-//      each one in the total order (key desc, id asc); rank r < topk is output slot r.
+//   3. a threshold T taken from the list *heads*: the heads are warp-sorted and T = the m-th best of
+//      the runs' p-th entries with m * (p + 1) >= topk, so at least topk heads are not after T and the
+//      global top-k lies among the entries that are not after T; each sorted list contributes a prefix;
+//   4. the survivors (typically a few dozen) go through the register merge tree of select.cuh, whose
+//      first topk entries are the answer in order.  More than 1024 survivors (massive ties) fall back
+//      to rank counting.
 // Nothing here depends on the order in which threads run.
 #include "common.cuh"
 #include "kernels.h"
+#include "select.cuh"
 
 namespace dart {
 
-__device__ __forceinline__ bool cand_before(float ka, int ia, float kb, int ib) {  // a strictly precedes b
-  return ka > kb || (ka == kb && ia < ib);
-}
+constexpr int kMergeThreads = 512;
 
-__global__ void __launch_bounds__(1024) topk_merge_kernel(const LmParams p) {
+__global__ void __launch_bounds__(kMergeThreads) topk_merge_kernel(const LmParams p) {
   extern __shared__ __align__(16) unsigned char msm[];
   const int G = p.grid, MP = padded_tokens(p.M), tk = blockIdx.x, topk = p.topk;
-  float* keys = reinterpret_cast<float*>(msm);        // [G*32]
-  int* ids = reinterpret_cast<int*>(keys + G * 32);   // [G*32]
-  int* surv = ids + G * 32;                           // [G*32]
-  __shared__ float sh[32];
-  __shared__ float s_thr_key;
-  __shared__ int s_thr_id, s_nsurv;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
+  float* keys = reinterpret_cast<float*>(msm);                 // [G*32]
+  int* ids = reinterpret_cast<int*>(keys + G * 32);            // [G*32]
+  Key* skey = reinterpret_cast<Key*>(ids + G * 32);            // [G*32] survivors' keys
+  int* ssrc = reinterpret_cast<int*>(skey + G * 32);           // [G*32] survivors' positions c*32+e
+  Key* xk = reinterpret_cast<Key*>(ssrc + G * 32);             // [16 warps][64] merge-tree scratch
+  Key* hr = xk + 16 * 64;                                      // [32 runs][32] sorted heads
+  __shared__ float sh_m[16], sh_s[16];
+  __shared__ float s_lse;
+  __shared__ Key s_thr;
+  __shared__ int s_nsurv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_wait();
 
-  for (int i = tid; i < G * 32; i += nthr) {
-    const int c = i >> 5, e = i & 31;
-    const size_t o = ((size_t)c * MP + tk) * 32 + e;
-    keys[i] = (e < topk) ? p.part_key[o] : -INFINITY;
-    ids[i] = p.part_id[o];
-  }
-  if (tid == 0) { s_thr_key = -INFINITY; s_thr_id = 0x7fffffff; s_nsurv = 0; }
-
-  // ---- log-sum-exp over the slices
-  float mx = -INFINITY;
-  for (int c = tid; c < G; c += nthr) mx = fmaxf(mx, p.part_stats[((size_t)c * MP + tk) * 2]);
-  mx = warp_max(mx);
-  __syncthreads();
-  if (lane == 0) sh[warp] = mx;
-  __syncthreads();
-  mx = sh[0];
-  for (int i = 1; i < (nthr >> 5); ++i) mx = fmaxf(mx, sh[i]);
-  float sum = 0.f;
-  for (int c = tid; c < G; c += nthr) {
-    const float mc = p.part_stats[((size_t)c * MP + tk) * 2];
-    if (mc != -INFINITY) sum += p.part_stats[((size_t)c * MP + tk) * 2 + 1] * expf(mc - mx);
-  }
-  sum = block_sum(sum, sh);
-  const float lse = mx + logf(sum);
-
-  // ---- threshold from the list heads
-  if (G >= topk) {
-    for (int c = tid; c < G; c += nthr) {
-      const float mk = keys[c * 32];
-      const int mi = ids[c * 32];
-      int rank = 0;
-      for (int o = 0; o < G; ++o) rank += cand_before(keys[o * 32], ids[o * 32], mk, mi);
-      if (rank == topk - 1) { s_thr_key = mk; s_thr_id = mi; }
+  {  // coalesced copy of the G lists of this token row: 32 keys and 32 ids per list
+    const float4* ksrc = reinterpret_cast<const float4*>(p.part_key);
+    const int4* isrc = reinterpret_cast<const int4*>(p.part_id);
+    for (int i = tid; i < G * 8; i += kMergeThreads) {
+      const int c = i >> 3, q = i & 7;
+      const size_t o = ((size_t)c * MP + tk) * 8 + q;
+      reinterpret_cast<float4*>(keys)[i] = ksrc[o];
+      reinterpret_cast<int4*>(ids)[i] = isrc[o];
     }
   }
-  __syncthreads();
-  const float tkey = s_thr_key;
-  const int tidx = s_thr_id;
+  if (tid == 0) s_nsurv = 0;
 
-  // ---- survivors: the prefix of every sorted list that is not after the threshold entry
-  for (int c = tid; c < G; c += nthr) {
+  // ---- log-sum-exp over the slices: per-thread online (max, sum), combined in a fixed order
+  float m = -INFINITY, s = 0.f;
+  for (int c = tid; c < G; c += kMergeThreads) {
+    const float mc = p.part_stats[((size_t)c * MP + tk) * 2], sc = p.part_stats[((size_t)c * MP + tk) * 2 + 1];
+    if (mc != -INFINITY) {
+      const float mn = fmaxf(m, mc);
+      s = s * expf(m - mn) + sc * expf(mc - mn);
+      m = mn;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float mo = __shfl_xor_sync(0xffffffffu, m, o), so = __shfl_xor_sync(0xffffffffu, s, o);
+    const float mn = fmaxf(m, mo);
+    const float a = (m == -INFINITY) ? 0.f : s * expf(m - mn), b = (mo == -INFINITY) ? 0.f : so * expf(mo - mn);
+    // both lanes of a pair compute the same value (addition is commutative)
+    s = a + b;
+    m = mn;
+  }
+  if (lane == 0) { sh_m[warp] = m; sh_s[warp] = s; }
+  __syncthreads();   // also publishes keys/ids
+  if (tid == 0) {
+    float mm = -INFINITY;
+    for (int i = 0; i < kMergeThreads / 32; ++i) mm = fmaxf(mm, sh_m[i]);
+    float ss = 0.f;
+    for (int i = 0; i < kMergeThreads / 32; ++i)
+      if (sh_m[i] != -INFINITY) ss += sh_s[i] * expf(sh_m[i] - mm);
+    s_lse = mm + logf(ss);
+  }
+
+  // ---- threshold from the list heads
+  const int nruns = (G + 31) >> 5;  // <= 32
+  Key hk = kPadKey;
+  if (tid < nruns * 32) {
+    const int c = tid;
+    if (c < G && keys[c * 32] != -INFINITY) hk = make_key(keys[c * 32], ids[c * 32]);
+    warp_sort(hk, lane);
+    hr[warp * 32 + lane] = hk;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    int mm = (nruns + 1) >> 1;
+    const int pp = (topk + mm - 1) / mm - 1;   // <= 31 because topk <= 32
+    Key t = (lane < nruns) ? hr[lane * 32 + pp] : kPadKey;
+    warp_sort(t, lane);
+    t = shfl_key(t, mm - 1);
+    if (lane == 0) s_thr = t;
+  }
+  __syncthreads();
+  const Key thr = s_thr;
+
+  // ---- survivors: the prefix of every sorted list that is not after the threshold
+  for (int c = tid; c < G; c += kMergeThreads) {
     for (int e = 0; e < topk; ++e) {
       const float k = keys[c * 32 + e];
-      if (k == -INFINITY || cand_before(tkey, tidx, k, ids[c * 32 + e])) break;
-      surv[atomicAdd(&s_nsurv, 1)] = c * 32 + e;
+      if (k == -INFINITY) break;
+      const Key kk = make_key(k, ids[c * 32 + e]);
+      if (kk < thr) break;
+      const int slot = atomicAdd(&s_nsurv, 1);
+      skey[slot] = kk;
+      ssrc[slot] = c * 32 + e;
     }
   }
   __syncthreads();
   const int ns = s_nsurv;
+  const float lse = s_lse;
+  const int filled = ns < topk ? ns : topk;
 
-  // ---- rank the survivors; rank r < topk is output slot r
-  for (int s = tid; s < ns; s += nthr) {
-    const int me = surv[s];
-    const float mk = keys[me];
-    const int mi = ids[me];
-    int rank = 0;
-    for (int o = 0; o < ns; ++o) {
-      const int ot = surv[o];
-      rank += cand_before(keys[ot], ids[ot], mk, mi);
-    }
-    if (rank < topk) {
-      const int c = me >> 5, e = me & 31;
+  if (ns <= kMergeThreads) {
+    // ---- best 64 of the survivors, in order, via the register merge tree
+    Key x0, x1;
+    block_best64(tid < ns ? skey[tid] : kPadKey, (ns + 31) >> 5, xk, 0, x0, x1);
+    if (warp == 0 && lane < filled) {
+      int src = -1;
+      for (int o = 0; o < ns; ++o)
+        if (skey[o] == x0) { src = ssrc[o]; break; }
+      const int c = src >> 5, e = src & 31;
       const float y = p.part_y[((size_t)c * MP + tk) * 32 + e];
-      p.out_ids[(size_t)tk * topk + rank] = mi;
-      p.out_slogit[(size_t)tk * topk + rank] = logf(expf(y - lse) + p.eps_logit);
+      p.out_ids[(size_t)tk * topk + lane] = ids[src];
+      p.out_slogit[(size_t)tk * topk + lane] = logf(expf(y - lse) + p.eps_logit);
+    }
+  } else {
+    // ---- massive ties: rank every survivor by counting the survivors that precede it
+    for (int sidx = tid; sidx < ns; sidx += kMergeThreads) {
+      const Key me = skey[sidx];
+      int rank = 0;
+      for (int o = 0; o < ns; ++o) rank += skey[o] > me;
+      if (rank < topk) {
+        const int src = ssrc[sidx], c = src >> 5, e = src & 31;
+        const float y = p.part_y[((size_t)c * MP + tk) * 32 + e];
+        p.out_ids[(size_t)tk * topk + rank] = ids[src];
+        p.out_slogit[(size_t)tk * topk + rank] = logf(expf(y - lse) + p.eps_logit);
+      }
     }
   }
-  const int filled = ns < topk ? ns : topk;
   if (tid >= filled && tid < topk) {
     p.out_ids[(size_t)tk * topk + tid] = -1;
     p.out_slogit[(size_t)tk * topk + tid] = -INFINITY;
   }
 }
 
-static size_t merge_smem(int G) { return (size_t)G * 32 * 12; }
+static size_t merge_smem(int G) { return (size_t)G * 32 * (4 + 4 + 8 + 4) + (16 * 64 + 32 * 32) * 8 + 64; }
 
 cudaError_t topk_merge_setup(int max_grid) {
   const size_t smem = merge_smem(max_grid);
@@ -115,7 +159,7 @@ cudaError_t topk_merge_setup(int max_grid) {
 }
 
 cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st) {
-  return launch_pdl(topk_merge_kernel, dim3(p.M), dim3(1024), merge_smem(p.grid), st, p);
+  return launch_pdl(topk_merge_kernel, dim3(p.M), dim3(kMergeThreads), merge_smem(p.grid), st, p);
 }
 
 }  // namespace dart
