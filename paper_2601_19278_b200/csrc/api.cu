@@ -30,6 +30,8 @@ struct Workspace {
   bf16 *u_hi = nullptr, *u_lo = nullptr;   // [Mmax, I]
   float *ss_g = nullptr, *ss_1 = nullptr, *ss_2 = nullptr;  // [h/128 tiles][MP] sums of squares per tile
   float* rstd_mask = nullptr;
+  float* mask_res = nullptr;    // [h] g half of the <mask> representation as fp32
+  float2* rope_tab = nullptr;   // [max_prefix + K][dh/2] (cos, sin)
   float* bg = nullptr;          // [max_batch][topk + (K-1)*topk^2] bigram scores of the tree builder
   float *o_part = nullptr, *ml_part = nullptr;
   float *lm_stats = nullptr, *lm_key = nullptr, *lm_y = nullptr;
@@ -87,7 +89,7 @@ bool config_ok(const dart_config* c) {
 
 struct PlanHost {
   GemmPlan plan;
-  std::vector<int> clo, chi, first, expected;
+  std::vector<int> expected, meta;
 };
 
 // Cut the flattened (16-row tile, k-round) space of a projection into `grid_target` equal ranges.
@@ -114,25 +116,30 @@ void make_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int gri
   p.grid = (int)((long long)grid_target < p.U ? grid_target : p.U);
   p.pair_offset = pair_offset;
   p.n_groups = pair_offset > 0 ? pair_offset : tiles;
-  ph.clo.assign(n_mt, 0x7fffffff);
-  ph.chi.assign(n_mt, -1);
-  ph.first.assign(p.grid, 0);
+  // CTA c streams units [c*U/grid, (c+1)*U/grid): every 16-row tile it touches gets one piece (one ticket).
+  // The piece table holds at most kMetaStride-1 pieces per tile; a tile of KR k-rounds is cut into at most
+  // ceil(KR / (U / grid)) + 1 of them, so (for very long reductions only) the grid shrinks until that fits.
+  while (p.grid > 1 && (p.KR + (p.U / p.grid) - 1) / (p.U / p.grid) + 1 > kMetaStride - 1) p.grid /= 2;
   p.slots = 1;
+  p.meta_stride = kMetaStride;
+  ph.expected.assign(p.n_groups, 0);
+  ph.meta.assign((size_t)n_mt * kMetaStride, 0);
   for (int c = 0; c < p.grid; ++c) {
     const long long u0 = ((long long)c * p.U) / p.grid, u1 = ((long long)(c + 1) * p.U) / p.grid;
     if (u0 >= u1) continue;
     const int t0 = (int)(u0 / p.KR), t1 = (int)((u1 - 1) / p.KR);
-    ph.first[c] = t0;
     if (t1 - t0 + 1 > p.slots) p.slots = t1 - t0 + 1;
-    for (int t = t0; t <= t1; ++t) {
-      if (c < ph.clo[t]) ph.clo[t] = c;
-      if (c > ph.chi[t]) ph.chi[t] = c;
-    }
   }
-  ph.expected.assign(p.n_groups, 0);
-  for (int t = 0; t < n_mt; ++t) {
-    const int tile = t >> 3;
-    ph.expected[pair_offset > 0 ? tile % pair_offset : tile] += ph.chi[t] - ph.clo[t] + 1;
+  for (int c = 0; c < p.grid; ++c) {
+    const long long u0 = ((long long)c * p.U) / p.grid, u1 = ((long long)(c + 1) * p.U) / p.grid;
+    if (u0 >= u1) continue;
+    const int t0 = (int)(u0 / p.KR), t1 = (int)((u1 - 1) / p.KR);
+    for (int t = t0; t <= t1; ++t) {
+      const int tile = t >> 3;
+      ph.expected[pair_offset > 0 ? tile % pair_offset : tile] += 1;
+      int& n = ph.meta[(size_t)t * kMetaStride];
+      if (n < kMetaStride - 1) ph.meta[(size_t)t * kMetaStride + 1 + n++] = c * p.slots + (t - t0);
+    }
   }
 }
 
@@ -177,6 +184,8 @@ size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_p
   TAKE(ss_1, float*, ht * MPmax * sizeof(float));
   TAKE(ss_2, float*, ht * MPmax * sizeof(float));
   TAKE(rstd_mask, float*, 256);
+  TAKE(mask_res, float*, (size_t)c.hidden * sizeof(float));
+  TAKE(rope_tab, float2*, (size_t)(c.max_prefix + c.K) * (c.head_dim / 2) * sizeof(float2));
   TAKE(bg, float*, (size_t)c.max_batch * (c.topk + (size_t)(c.K - 1) * c.topk * c.topk) * sizeof(float));
   TAKE(o_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * c.head_dim * sizeof(float));
   TAKE(ml_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * 2 * sizeof(float));
@@ -315,10 +324,8 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   PlanHost* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
   for (int i = 0; i < 5; ++i) {
     PlanHost& ph = *plans[i];
-    INIT_CHECK(upload(h, ph.clo, &ph.plan.d_mt_clo));
-    INIT_CHECK(upload(h, ph.chi, &ph.plan.d_mt_chi));
-    INIT_CHECK(upload(h, ph.first, &ph.plan.d_first_mt));
     INIT_CHECK(upload(h, ph.expected, &ph.plan.d_expected));
+    INIT_CHECK(upload(h, ph.meta, &ph.plan.d_meta));
     std::vector<int> zeros(ph.plan.n_groups, 0);
     INIT_CHECK(upload(h, zeros, &ph.plan.d_ctr));
   }
@@ -337,8 +344,10 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
     const size_t mrow = (size_t)cfg->max_batch * cfg->K * 2 * cfg->hidden;
     INIT_CHECK(launch_mask_row(static_cast<const bf16*>(weights->mask_vec), static_cast<const bf16*>(weights->norm_g),
                                static_cast<const bf16*>(weights->norm_e), cfg->hidden, cfg->rms_eps, h->ws.z_hi + mrow,
-                               h->ws.z_lo + mrow, h->ws.rstd_mask, nullptr));
+                               h->ws.z_lo + mrow, h->ws.rstd_mask, h->ws.mask_res, nullptr));
   }
+
+  INIT_CHECK(launch_rope_table(h->ws.rope_tab, cfg->max_prefix + cfg->K, cfg->head_dim, cfg->rope_theta, nullptr));
 
   // Appendix D's per-level weights: fp64 from the fp32 settings, rounded once to fp32
   for (int i = 0; i < 8; ++i) {
@@ -455,7 +464,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   memset(&ep, 0, sizeof(ep));
   ep.mode = EPI_QKV; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
   ep.ss_in = ws.ss_g; ep.ss_tiles = h->h_tiles; ep.ss_mp = padded_tokens(B * (F > 0 ? F : 1)); ep.rstd_mask = ws.rstd_mask;
-  ep.Hq = c.n_q_heads; ep.Hkv = c.n_kv_heads; ep.dh = c.head_dim; ep.seq_lens = in->seq_lens; ep.rope_theta = c.rope_theta;
+  ep.Hq = c.n_q_heads; ep.Hkv = c.n_kv_heads; ep.dh = c.head_dim; ep.seq_lens = in->seq_lens; ep.rope_tab = ws.rope_tab;
   ep.q_hi = ws.q_hi; ep.q_lo = ws.q_lo; ep.k_new = ws.k_new; ep.v_new = ws.v_new;
   ep.k_cache = static_cast<bf16*>(in->k_cache); ep.v_cache = static_cast<bf16*>(in->v_cache); ep.P_cap = c.max_prefix;
   gi = {ws.z_hi, ws.z_lo, 2 * hdim, M, K, F, mask_row};
@@ -487,7 +496,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   mark(3, true);
   memset(&ep, 0, sizeof(ep));
   ep.mode = EPI_RES; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
-  ep.res0 = ws.res0; ep.res_in = nullptr; ep.res_out = ws.x1; ep.mask_vec = static_cast<const bf16*>(h->w.mask_vec);
+  ep.res0 = ws.res0; ep.res_in = nullptr; ep.res_out = ws.x1; ep.mask_res = ws.mask_res;
   ep.gamma = static_cast<const bf16*>(h->w.norm_post);
   ep.out_hi = ws.n_hi; ep.out_lo = ws.n_lo; ep.ld_out = hdim; ep.ss_out = ws.ss_1;
   gi = {ws.a_hi, ws.a_lo, dq, M, 0, 0, 0};

@@ -24,187 +24,241 @@ namespace dart {
 // ------------------------------------------------------------------------------------------
 // Fused epilogues, run by the CTA that completes a tile (or a pair of tiles).
 // ------------------------------------------------------------------------------------------
-// Shared-memory description of one group: for each of its (up to 16) 16-row tiles, the partial pieces
-// to add up, as offsets into `part` in units of one 16 x MP piece, in CTA order.
-constexpr int kMaxPieces = 33;
-struct GroupMeta {
-  int cnt[16];
-  unsigned off[16][kMaxPieces];
+// Shared-memory working set of one finalize.
+struct FinSmem {
+  float rpart[512];      // partial sums of squares for the 1/rms
+  float xs[2][128][9];   // summed pieces: [tile of the pair][row][token of the chunk], padded against conflicts
 };
+static_assert(sizeof(FinSmem) <= 2 * 16 * 16 * 8 * sizeof(float), "the finalize working set must fit the streaming buffers");
 
-__device__ __forceinline__ void load_group_meta(const GemmArgs& p, int Ta, int Tb, bool paired, GroupMeta* gm) {
-  const int j = threadIdx.x;
-  if (j < 16 && (j < 8 || paired)) {
-    const int mt = (j < 8 ? Ta : Tb) * 8 + (j & 7);
-    const int lo = p.clo[mt], hi = p.chi[mt];
-    int n = 0;
-    for (int c = lo; c <= hi && n < kMaxPieces; ++c) gm->off[j][n++] = (unsigned)(c * p.slots + (mt - p.first_mt[c]));
-    gm->cnt[j] = n;
+// Piece table of one group in shared memory: for each of its (up to 16) 16-row tiles the count and the
+// offsets (units of one 16 x MP piece, CTA order) of the pieces to add up.  The table is plan data, so a
+// CTA copies the rows of the groups it may end up finalizing (those its range touches) with cp.async
+// right at its start; by the time a finalize runs they have long arrived.
+struct GroupMeta { int row[16][kMetaStride]; };
+constexpr int kMetaSlots = 2;
+
+__device__ __forceinline__ void meta_prefetch(const GemmArgs& p, int group, GroupMeta* gm) {
+  const int Ta = group, Tb = group + p.pair_offset;
+  const int nrow = p.pair_offset > 0 ? 16 : 8;
+  for (int i = threadIdx.x; i < nrow * kMetaStride; i += blockDim.x) {
+    const int j = i / kMetaStride, q = i - j * kMetaStride;
+    const int* src = p.meta + (size_t)((j < 8 ? Ta : Tb) * 8 + (j & 7)) * kMetaStride + q;
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(&gm->row[j][q]);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
   }
-  __syncthreads();
+  asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
-// which: 0 = tile Ta, 1 = tile Tb of the group
-__device__ __forceinline__ float piece_sum(const GemmArgs& p, const GroupMeta* gm, int which, int row, int tok, int MP) {
+// Partial sum of squares of token row tid / TPT over the tiles q, q + TPT, ... (TPT = blockDim / MP threads
+// per token); col(tok) maps a token to its column of ss[tile][mp], or -1.
+template <class ColFn>
+__device__ __forceinline__ float rstd_issue(const float* ss, int ntile, int mp, int M, int MP, ColFn col) {
+  const int TPT = blockDim.x / MP, tok = threadIdx.x / TPT, q = threadIdx.x % TPT;
+  const int cidx = tok < M ? col(tok) : -1;
   float s = 0.f;
-  const int j = which * 8 + (row >> 4), r = row & 15;
-  const int n = gm->cnt[j];
-  for (int i = 0; i < n; ++i) s += p.part[((size_t)gm->off[j][i] * 16 + r) * MP + tok];
+  if (cidx >= 0) {
+#pragma unroll 4
+    for (int t = q; t < ntile; t += TPT) s += __ldcg(ss + (size_t)t * mp + cidx);
+  }
   return s;
 }
-
-// 1/rms of every token row from per-tile sums of squares ss[tile][mp] (tiles of a width-`h` row), into
-// s_rstd[0..M).  Four threads per token add up interleaved tiles, then their four partials are added in a
-// fixed order.  col(tok) maps a token to its column of ss.  Needs M <= 128 and blockDim >= 512.
+// Fixed-order reduction of those partials to s_rstd[tok] = 1/rms.  Two barriers.
 template <class ColFn>
-__device__ __forceinline__ void rstd_all(const float* ss, int ntile, int mp, int M, int h, float eps, float* s_part,
-                                         float* s_rstd, ColFn col) {
-  const int tid = threadIdx.x;
-  if (tid < 4 * M) {
-    const int tok = tid >> 2, q = tid & 3;
-    const int cidx = col(tok);
-    float s = 0.f;
-    if (cidx >= 0)
-      for (int t = q; t < ntile; t += 4) s += ss[(size_t)t * mp + cidx];
-    s_part[tid] = s;
-  }
+__device__ __forceinline__ void rstd_finish(float s, int M, int MP, int h, float eps, FinSmem* fs, float* s_rstd, ColFn col) {
+  const int TPT = blockDim.x / MP, width = TPT < 32 ? TPT : 32, nsub = TPT < 32 ? 1 : TPT / 32;
+  for (int o = width >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if ((threadIdx.x % width) == 0) fs->rpart[threadIdx.x / width] = s;
   __syncthreads();
-  if (tid < M) {
-    const float s = s_part[4 * tid] + s_part[4 * tid + 1] + s_part[4 * tid + 2] + s_part[4 * tid + 3];
-    if (col(tid) >= 0) s_rstd[tid] = 1.f / sqrtf(s / (float)h + eps);
+  if (threadIdx.x < M && col(threadIdx.x) >= 0) {
+    float t = 0.f;
+    for (int k = 0; k < nsub; ++k) t += fs->rpart[threadIdx.x * nsub + k];
+    s_rstd[threadIdx.x] = 1.f / sqrtf(t / (float)h + eps);
   }
   __syncthreads();
 }
 
-// sum over the group's 128 rows of v (one value per thread: row = tid & 127, token class = tid >> 7),
-// result valid in every thread; fixed order.  sh: one float per warp.
-__device__ __forceinline__ float tile_rows_sum(float v, float* sh) {
+// Piece sums of the group's tile(s) for the 8 tokens tok0 .. tok0+7, pieces in CTA order.  The thread ->
+// element mapping follows the pieces' memory layout (coalesced), and the first four pieces of every
+// element are requested before any is used.
+template <int NTILE>
+struct Gather {
+  static constexpr int Q = NTILE * 2;   // elements per thread (512 threads, 1024 elements per tile)
+  float v[Q][4];
+  __device__ __forceinline__ void issue(const GemmArgs& p, const GroupMeta* gm, int tok0, int MP) {
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+      const int e = threadIdx.x + 512 * q, row = (e >> 3) & 127;
+      const int* m = gm->row[(e >> 10) * 8 + (row >> 4)];
+      const float* src = p.part + (size_t)(row & 15) * MP + tok0 + (e & 7);
+      const int n = m[0];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[q][u] = u < n ? __ldcg(src + (size_t)m[1 + u] * 16 * MP) : 0.f;
+    }
+  }
+  __device__ __forceinline__ void finish(const GemmArgs& p, const GroupMeta* gm, int tok0, int MP, FinSmem* fs) {
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+      const int e = threadIdx.x + 512 * q, row = (e >> 3) & 127;
+      const int* m = gm->row[(e >> 10) * 8 + (row >> 4)];
+      float acc = (((0.f + v[q][0]) + v[q][1]) + v[q][2]) + v[q][3];
+      for (int u = 4; u < m[0]; ++u)  // rare: long reductions cut into many short ranges
+        acc += __ldcg(p.part + ((size_t)m[1 + u] * 16 + (row & 15)) * MP + tok0 + (e & 7));
+      fs->xs[e >> 10][row][e & 7] = acc;
+    }
+  }
+};
+
+// Sums v0 and v1 over the 128 rows of a tile (thread -> row = tid & 127, token class = tid >> 7);
+// results valid in every thread; fixed order.  sh: two floats per warp.
+__device__ __forceinline__ void tile_rows_sum2(float v0, float v1, float* sh, float& r0, float& r1) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  v = warp_sum(v);
+  v0 = warp_sum(v0);
+  v1 = warp_sum(v1);
   __syncthreads();
-  if (lane == 0) sh[warp] = v;
+  if (lane == 0) { sh[warp] = v0; sh[16 + warp] = v1; }
   __syncthreads();
-  const int cls = warp >> 2;  // warps 4*cls .. 4*cls+3 hold the 128 rows of token class cls
-  return sh[cls * 4] + sh[cls * 4 + 1] + sh[cls * 4 + 2] + sh[cls * 4 + 3];
+  const int c4 = (warp >> 2) * 4;  // warps c4 .. c4+3 hold the 128 rows of this token class
+  r0 = sh[c4] + sh[c4 + 1] + sh[c4 + 2] + sh[c4 + 3];
+  r1 = sh[16 + c4] + sh[16 + c4 + 1] + sh[16 + c4 + 2] + sh[16 + c4 + 3];
 }
 
-__device__ __noinline__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, float* s_rstd, GroupMeta* gm,
-                                            float* s_part) {
+// The fused epilogue of one completed group (one 128-row tile, or a pair of tiles).  It sits on the
+// kernel's tail, so it is built around a single round trip to memory: every load it needs (pieces,
+// residual, gain, sums of squares, RoPE entry) is requested up front, from addresses that depend on
+// nothing loaded here (the piece table is already in shared memory); then come the reductions through shared memory and the stores.
+// Needs blockDim.x == 512.  s_pos[tok] = P_b + r (EPI_QKV), s_rstd preset to the <mask> rows' 1/rms.
+__device__ __noinline__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, float* s_rstd, const int* s_pos,
+                                            const GroupMeta* gm, FinSmem* fs) {
   const EpiArgs& e = p.epi;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, M = p.s.M;
   const int Ta = group, Tb = group + p.pair_offset;
-  load_group_meta(p, Ta, Tb, p.pair_offset > 0, gm);
+  const bool paired = p.pair_offset > 0;
   int s = 0;  // segment of tile Ta
   for (int i = 1; i < 6; ++i)
     if (i < p.s.nseg && Ta >= p.s.seg[i].tile0) s = i;
   const int row_base = (Ta - p.s.seg[s].tile0) * 128;       // first row of the tile inside its matrix
   const int rows_valid = min(128, p.s.seg[s].rows - row_base);
-  const int row = tid & 127, par = tid >> 7;               // thread -> (row, token class)
-  const int npar = blockDim.x >> 7;
+  const int row = tid & 127, par = tid >> 7;               // thread -> (row, token class 0..3)
+  const int n = row_base + row;
+  const int K = e.K, F = e.F;
+  const auto col_id = [](int tok) { return tok; };
+  const auto col_fresh = [K, F](int tok) { const int b = tok / K, rr = tok % K; return rr < F ? b * F + rr : -1; };
+  const bool rowmode = e.mode == EPI_FC || e.mode == EPI_RES;
+  const int dh = e.dh, half = dh >> 1;
+  const int pairs = e.mode == EPI_QKV ? (rows_valid / dh) * half : 1;   // (head, i) pairs of this tile
 
-  if (e.mode == EPI_FC) {
-    // g = FC(features) on the fresh rows: residual stream, gain-scaled hi/lo, tile sum of squares
-    for (int tok = par; tok < MP; tok += npar) {
-      float g = 0.f;
-      if (row < rows_valid && tok < p.s.M) g = piece_sum(p, gm, 0, row, tok, MP);
-      const float ssq = tile_rows_sum(g * g, sh);
-      if (row < rows_valid && tok < p.s.M) {
-        const int n = row_base + row;
-        e.res0[(size_t)tok * e.h + n] = g;
-        bf16 hi, lo;
-        split_bf16(g * __bfloat162float(e.gamma[n]), hi, lo);
-        e.out_hi[(size_t)tok * e.ld_out + n] = hi;
-        e.out_lo[(size_t)tok * e.ld_out + n] = lo;
-      }
-      if (row == 0 && tok < p.s.M) e.ss_out[(size_t)Ta * MP + tok] = ssq;
+  for (int tok0 = 0; tok0 < M; tok0 += 8) {
+    const int t0 = tok0 + par, t1 = tok0 + par + 4;  // this thread's tokens in the row-major modes
+    const bool ok0 = row < rows_valid && t0 < M, ok1 = row < rows_valid && t1 < M;
+    const int ptok = tok0 + tid / pairs, pi = tid % pairs;    // this thread's (token, pair) in EPI_QKV
+    // ---- every load, before any use
+    Gather<2> g2;
+    Gather<1> g1;
+    if (paired) g2.issue(p, gm, tok0, MP); else g1.issue(p, gm, tok0, MP);
+    unsigned short gam_raw = 0;
+    if (rowmode && row < rows_valid) gam_raw = reinterpret_cast<const unsigned short*>(e.gamma)[n];
+    float r0 = 0.f, r1 = 0.f;
+    if (e.mode == EPI_RES) {
+      // residual: the stream so far, or (first projection) g of a fresh row / the <mask> representation
+      const float* s0 = e.res_in != nullptr ? e.res_in + (size_t)t0 * e.h
+                                            : ((t0 % K) < F ? e.res0 + (size_t)((t0 / K) * F + t0 % K) * e.h : e.mask_res);
+      const float* s1 = e.res_in != nullptr ? e.res_in + (size_t)t1 * e.h
+                                            : ((t1 % K) < F ? e.res0 + (size_t)((t1 / K) * F + t1 % K) * e.h : e.mask_res);
+      if (ok0) r0 = __ldcg(s0 + n);
+      if (ok1) r1 = __ldcg(s1 + n);
     }
-  } else if (e.mode == EPI_RES) {
-    // x = residual + proj; gain-scaled hi/lo for the next projection; tile sum of squares
-    for (int tok = par; tok < MP; tok += npar) {
-      float x = 0.f;
-      if (row < rows_valid && tok < p.s.M) {
-        const int n = row_base + row;
-        float r;
-        if (e.res_in != nullptr) r = e.res_in[(size_t)tok * e.h + n];
-        else {  // first residual: g of a fresh row, or the <mask> representation
-          const int b = tok / e.K, rr = tok % e.K;
-          r = rr < e.F ? e.res0[(size_t)(b * e.F + rr) * e.h + n] : __bfloat162float(e.mask_vec[n]);
-        }
-        x = r + piece_sum(p, gm, 0, row, tok, MP);
-      }
-      const float ssq = tile_rows_sum(x * x, sh);
-      if (row < rows_valid && tok < p.s.M) {
-        const int n = row_base + row;
-        if (e.res_out != nullptr) e.res_out[(size_t)tok * e.h + n] = x;
-        bf16 hi, lo;
-        split_bf16(x * __bfloat162float(e.gamma[n]), hi, lo);
-        e.out_hi[(size_t)tok * e.ld_out + n] = hi;
-        e.out_lo[(size_t)tok * e.ld_out + n] = lo;
-      }
-      if (row == 0 && tok < p.s.M) e.ss_out[(size_t)Ta * MP + tok] = ssq;
+    float2 cs = make_float2(1.f, 0.f);
+    if (e.mode == EPI_QKV && s < 2 && tid < pairs * 8 && ptok < M)
+      cs = e.rope_tab[(size_t)s_pos[ptok] * half + (pi % half)];  // (cos, sin) of pos * theta^(-2i/d_h)
+    float rs = 0.f;
+    if (tok0 == 0) {
+      if (e.mode == EPI_GATE_UP) rs = rstd_issue(e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_id);
+      if (e.mode == EPI_QKV) rs = rstd_issue(e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_fresh);
     }
-  } else if (e.mode == EPI_GATE_UP) {
-    // u = SiLU(rstd * gate) * (rstd * up): the previous RMSNorm's 1/rms is applied here
-    rstd_all(e.ss_in, e.ss_tiles, e.ss_mp, p.s.M, e.h, e.eps, s_part, s_rstd, [](int tok) { return tok; });
-    for (int tok = par; tok < p.s.M; tok += npar) {
-      if (row < rows_valid) {
-        const int n = row_base + row;
-        const float gt = s_rstd[tok] * piece_sum(p, gm, 0, row, tok, MP);
-        const float up = s_rstd[tok] * piece_sum(p, gm, 1, row, tok, MP);
-        bf16 hi, lo;
-        split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
-        e.out_hi[(size_t)tok * e.ld_out + n] = hi;
-        e.out_lo[(size_t)tok * e.ld_out + n] = lo;
-      }
+    // ---- reductions through shared memory
+    if (tok0 == 0) {
+      if (e.mode == EPI_GATE_UP) rstd_finish(rs, M, MP, e.h, e.eps, fs, s_rstd, col_id);
+      if (e.mode == EPI_QKV) rstd_finish(rs, M, MP, e.h, e.eps, fs, s_rstd, col_fresh);
     }
-  } else if (e.mode == EPI_QKV) {
-    // y = rstd_g * (W[:, :h] z_g) + W[:, h:] z_e ; RoPE on q, k at position P_b + r ; q and the new rows'
-    // k, v as hi/lo pairs ; the fresh rows' k, v appended to the cache
-    if (tid < p.s.M) s_rstd[tid] = e.rstd_mask[0];  // <mask> rows; fresh rows are overwritten below
+    if (paired) g2.finish(p, gm, tok0, MP, fs); else g1.finish(p, gm, tok0, MP, fs);
     __syncthreads();
-    {
-      const int K = e.K, F = e.F;
-      rstd_all(e.ss_in, e.ss_tiles, e.ss_mp, p.s.M, e.h, e.eps, s_part, s_rstd,
-               [K, F](int tok) { const int b = tok / K, rr = tok % K; return rr < F ? b * F + rr : -1; });
-    }
-    const int kind = s;  // segment 0,1,2 = q,k,v (g half); the e half is the paired tile
-    const int dh = e.dh, half = dh >> 1;
-    const int pairs = (rows_valid / dh) * half;  // (head, i) pairs in this tile
-    for (int idx = tid; idx < pairs * p.s.M; idx += blockDim.x) {
-      const int tok = idx / pairs, pi = idx - tok * pairs;
-      const int hl = pi / half, i = pi - hl * half;
-      const int ra = hl * dh + i, rb = ra + half;
-      const float x1 = s_rstd[tok] * piece_sum(p, gm, 0, ra, tok, MP) + piece_sum(p, gm, 1, ra, tok, MP);
-      const float x2 = s_rstd[tok] * piece_sum(p, gm, 0, rb, tok, MP) + piece_sum(p, gm, 1, rb, tok, MP);
-      const int b = tok / e.K, r = tok % e.K;
-      const long long pos = (long long)e.seq_lens[b] + r;
-      float o1 = x1, o2 = x2;
-      if (kind < 2) {
-        const double inv = pow((double)e.rope_theta, -2.0 * (double)i / (double)dh);
-        double sn, cs;
-        sincos((double)pos * inv, &sn, &cs);
-        o1 = (float)((double)x1 * cs - (double)x2 * sn);
-        o2 = (float)((double)x2 * cs + (double)x1 * sn);
+
+    // ---- the mode's arithmetic and stores
+    if (rowmode) {
+      // FC: g = FC(features) on the fresh rows.  RES: x = residual + projection.  Both: residual stream,
+      // gain-scaled hi/lo for the next projection, the tile's sum of squares for the next 1/rms.
+      const float gam = __bfloat162float(__ushort_as_bfloat16(gam_raw));
+      const float x0 = ok0 ? r0 + fs->xs[0][row][par] : 0.f, x1 = ok1 ? r1 + fs->xs[0][row][par + 4] : 0.f;
+      float q0, q1;
+      tile_rows_sum2(x0 * x0, x1 * x1, sh, q0, q1);
+      float* res = e.mode == EPI_FC ? e.res0 : e.res_out;
+      bf16 hi, lo;
+      if (ok0) {
+        if (res != nullptr) res[(size_t)t0 * e.h + n] = x0;
+        split_bf16(x0 * gam, hi, lo);
+        e.out_hi[(size_t)t0 * e.ld_out + n] = hi;
+        e.out_lo[(size_t)t0 * e.ld_out + n] = lo;
       }
-      bf16 h1, l1, h2, l2;
-      split_bf16(o1, h1, l1);
-      split_bf16(o2, h2, l2);
-      const int head = (row_base / dh) + hl;
-      if (kind == 0) {
-        const size_t o = (((size_t)b * e.Hq + head) * e.K + r) * dh;
-        e.q_hi[o + i] = h1; e.q_hi[o + i + half] = h2;
-        e.q_lo[o + i] = l1; e.q_lo[o + i + half] = l2;
-      } else {
-        bf16* side = (kind == 1 ? e.k_new : e.v_new) + ((size_t)b * e.Hkv + head) * 16 * dh;
-        side[(size_t)r * dh + i] = h1; side[(size_t)r * dh + i + half] = h2;
-        side[(size_t)(8 + r) * dh + i] = l1; side[(size_t)(8 + r) * dh + i + half] = l2;
-        if (r < e.F) {
-          bf16* dst = (kind == 1 ? e.k_cache : e.v_cache) + (((size_t)b * e.Hkv + head) * e.P_cap + pos) * dh;
-          dst[i] = h1;
-          dst[i + half] = h2;
+      if (ok1) {
+        if (res != nullptr) res[(size_t)t1 * e.h + n] = x1;
+        split_bf16(x1 * gam, hi, lo);
+        e.out_hi[(size_t)t1 * e.ld_out + n] = hi;
+        e.out_lo[(size_t)t1 * e.ld_out + n] = lo;
+      }
+      if (row == 0 && t0 < M) e.ss_out[(size_t)Ta * MP + t0] = q0;
+      if (row == 0 && t1 < M) e.ss_out[(size_t)Ta * MP + t1] = q1;
+    } else if (e.mode == EPI_GATE_UP) {
+      // u = SiLU(rstd * gate) * (rstd * up): the previous RMSNorm's 1/rms is applied here
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const int tl = par + 4 * k, tok = tok0 + tl;
+        if (row < rows_valid && tok < M) {
+          const float gt = s_rstd[tok] * fs->xs[0][row][tl], up = s_rstd[tok] * fs->xs[1][row][tl];
+          bf16 hi, lo;
+          split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
+          e.out_hi[(size_t)tok * e.ld_out + n] = hi;
+          e.out_lo[(size_t)tok * e.ld_out + n] = lo;
+        }
+      }
+    } else if (e.mode == EPI_QKV) {
+      // y = rstd_g * (W[:, :h] z_g) + W[:, h:] z_e ; RoPE on q, k at position P_b + r ; q and the new rows'
+      // k, v as hi/lo pairs ; the fresh rows' k, v appended to the cache.  segment 0,1,2 = q,k,v (g half);
+      // the e half is the paired tile.
+      const int kind = s;
+      if (tid < pairs * 8 && ptok < M) {
+        const int tl = ptok - tok0, tok = ptok;
+        const int hl = pi / half, i = pi - hl * half;
+        const int ra = hl * dh + i, rb = ra + half;
+        const float x1 = s_rstd[tok] * fs->xs[0][ra][tl] + fs->xs[1][ra][tl];
+        const float x2 = s_rstd[tok] * fs->xs[0][rb][tl] + fs->xs[1][rb][tl];
+        const int b = tok / K, r = tok % K;
+        float o1 = x1, o2 = x2;
+        if (kind < 2) {
+          o1 = x1 * cs.x - x2 * cs.y;
+          o2 = x2 * cs.x + x1 * cs.y;
+        }
+        bf16 h1, l1, h2, l2;
+        split_bf16(o1, h1, l1);
+        split_bf16(o2, h2, l2);
+        const int head = (row_base / dh) + hl;
+        if (kind == 0) {
+          const size_t o = (((size_t)b * e.Hq + head) * K + r) * dh;
+          e.q_hi[o + i] = h1; e.q_hi[o + i + half] = h2;
+          e.q_lo[o + i] = l1; e.q_lo[o + i + half] = l2;
+        } else {
+          bf16* side = (kind == 1 ? e.k_new : e.v_new) + ((size_t)b * e.Hkv + head) * 16 * dh;
+          side[(size_t)r * dh + i] = h1; side[(size_t)r * dh + i + half] = h2;
+          side[(size_t)(8 + r) * dh + i] = l1; side[(size_t)(8 + r) * dh + i + half] = l2;
+          if (r < F) {
+            bf16* dst = (kind == 1 ? e.k_cache : e.v_cache) + (((size_t)b * e.Hkv + head) * e.P_cap + s_pos[tok]) * dh;
+            dst[i] = h1;
+            dst[i + half] = h2;
+          }
         }
       }
     }
+    __syncthreads();
   }
 }
 
@@ -252,10 +306,14 @@ struct GemmEpi {
     ++pending;
     const int group = group_of(mt);
     if (last || group_of(mt + 1) != group) {
-      // this CTA's last piece of the group: take its tickets
+      // this CTA's last piece of the group: take its tickets.  (Taking them one tile later, when the fence
+      // would be free, was measured slower: it delays the finalize of every group.)
       __threadfence();
       __syncthreads();
-      if (threadIdx.x == 0 && atomicAdd(&p.ctr[group], pending) + pending == p.expected[group]) s_done[++s_done[0]] = group;
+      if (threadIdx.x == 0 && atomicAdd(&p.ctr[group], pending) + pending == p.expected[group]) {
+        __threadfence();  // acquire: the other CTAs' pieces are visible to whatever follows the next barrier
+        s_done[++s_done[0]] = group;
+      }
       pending = 0;
     }
   }
@@ -272,9 +330,24 @@ __global__ void __launch_bounds__(512, (NT == 1 ? 2 : 1)) gemm_rows_kernel(const
   __shared__ float sh[32];
   __shared__ float s_rstd[128];
   __shared__ int s_done[kMaxDone + 2];
+  __shared__ int s_pos[128];
+  __shared__ GroupMeta s_meta[kMetaSlots];
   const int c = blockIdx.x, G = gridDim.x;
   if (threadIdx.x == 0) s_done[0] = 0;
+  if (p.epi.mode == EPI_QKV && threadIdx.x < p.s.M) {
+    // inputs of the step and init-time constants: nothing an earlier kernel of this step writes
+    s_pos[threadIdx.x] = p.epi.seq_lens[threadIdx.x / p.epi.K] + threadIdx.x % p.epi.K;
+    s_rstd[threadIdx.x] = p.epi.rstd_mask[0];  // <mask> rows; fresh rows are overwritten in the finalize
+  }
   const long long u0 = ((long long)c * p.U) / G, u1 = ((long long)(c + 1) * p.U) / G;
+  int cand[kMetaSlots] = {-1, -1};  // groups whose piece tables sit in s_meta
+  if (u0 < u1) {
+    const int t0 = (int)(u0 / p.s.KR) >> 3, t1 = (int)((u1 - 1) / p.s.KR) >> 3;
+    cand[0] = p.pair_offset > 0 ? t0 % p.pair_offset : t0;
+    cand[1] = p.pair_offset > 0 ? t1 % p.pair_offset : t1;
+    meta_prefetch(p, cand[0], &s_meta[0]);
+    if (cand[1] != cand[0]) meta_prefetch(p, cand[1], &s_meta[1]);
+  }
   __syncthreads();
   if (u0 < u1) {
     GemmEpi<NT, NW> epi{p, red, s_done, c, (int)(u0 / p.s.KR), 0};
@@ -287,12 +360,20 @@ __global__ void __launch_bounds__(512, (NT == 1 ? 2 : 1)) gemm_rows_kernel(const
   if (p.epi.mode == EPI_FC && c < p.s.M) embed_rows(p, sh);
   // fused finalize of the groups this CTA completed (the streaming buffers are free now)
   const int n_done = s_done[0];
-  GroupMeta* gm = reinterpret_cast<GroupMeta*>(red);
-  float* s_part = reinterpret_cast<float*>(gm + 1);
+  FinSmem* fs = reinterpret_cast<FinSmem*>(red);
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
   for (int i = 0; i < n_done; ++i) {
     const int group = s_done[1 + i];
-    __threadfence();
-    finalize_group(p, group, 8 * NT, sh, s_rstd, gm, s_part);
+    int slot = group == cand[0] ? 0 : (group == cand[1] ? 1 : -1);
+    if (slot < 0) {  // a range that touches more than two groups (short reductions): fetch the table now
+      slot = 0;
+      cand[0] = group;
+      meta_prefetch(p, group, &s_meta[0]);
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      __syncthreads();
+    }
+    finalize_group(p, group, 8 * NT, sh, s_rstd, s_pos, &s_meta[slot], fs);
     if (threadIdx.x == 0) p.ctr[group] = 0;
     __syncthreads();
   }
@@ -301,7 +382,7 @@ __global__ void __launch_bounds__(512, (NT == 1 ? 2 : 1)) gemm_rows_kernel(const
 // The <mask> rows are the same for every sequence and every step: their z row ([m_g * gain_g (not yet
 // normalised) ; RMSNorm(m_e)]) and the 1/rms of m_g are computed once, at init.
 __global__ void __launch_bounds__(256) mask_row_kernel(const bf16* mask_vec, const bf16* norm_g, const bf16* norm_e, int h,
-                                                       float eps, bf16* z_hi, bf16* z_lo, float* rstd_mask) {
+                                                       float eps, bf16* z_hi, bf16* z_lo, float* rstd_mask, float* mask_res) {
   __shared__ float sh[32];
   float sg = 0.f, se = 0.f;
   for (int n = threadIdx.x; n < h; n += blockDim.x) {
@@ -317,14 +398,32 @@ __global__ void __launch_bounds__(256) mask_row_kernel(const bf16* mask_vec, con
     bf16 hi, lo;
     split_bf16(__bfloat162float(mask_vec[n]) * __bfloat162float(norm_g[n]), hi, lo);
     z_hi[n] = hi; z_lo[n] = lo;
+    mask_res[n] = __bfloat162float(mask_vec[n]);
     split_bf16(__bfloat162float(mask_vec[h + n]) * re * __bfloat162float(norm_e[n]), hi, lo);
     z_hi[h + n] = hi; z_lo[h + n] = lo;
   }
 }
 
+// (cos, sin) of every (position, frequency) pair the cache can hold, computed once in double precision.
+__global__ void rope_table_kernel(float2* tab, int n_pos, int half, double theta, int dh) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)n_pos * half) return;
+  const int pos = (int)(idx / half), i = (int)(idx % half);
+  const double inv = pow(theta, -2.0 * (double)i / (double)dh);
+  double sn, cs;
+  sincos((double)pos * inv, &sn, &cs);
+  tab[idx] = make_float2((float)cs, (float)sn);
+}
+
+cudaError_t launch_rope_table(float2* tab, int n_pos, int dh, float theta, cudaStream_t st) {
+  const long long n = (long long)n_pos * (dh / 2);
+  rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(tab, n_pos, dh / 2, (double)theta, dh);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_mask_row(const bf16* mask_vec, const bf16* norm_g, const bf16* norm_e, int h, float eps, bf16* z_hi,
-                            bf16* z_lo, float* rstd_mask, cudaStream_t st) {
-  mask_row_kernel<<<1, 256, 0, st>>>(mask_vec, norm_g, norm_e, h, eps, z_hi, z_lo, rstd_mask);
+                            bf16* z_lo, float* rstd_mask, float* mask_res, cudaStream_t st) {
+  mask_row_kernel<<<1, 256, 0, st>>>(mask_vec, norm_g, norm_e, h, eps, z_hi, z_lo, rstd_mask, mask_res);
   return cudaGetLastError();
 }
 
@@ -349,7 +448,7 @@ cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const Ep
   a.s.Kd = plan.Kd; a.s.SK = plan.SK; a.s.KR = plan.KR; a.slots = plan.slots; a.U = plan.U;
   a.s.x_hi = in.x_hi; a.s.x_lo = in.x_lo != nullptr ? in.x_lo : in.x_hi; a.s.ldx = in.ldx; a.s.M = in.M;
   a.s.x_K = in.x_K; a.s.x_F = in.x_F; a.s.x_mask_row = in.x_mask_row;
-  a.part = part; a.first_mt = plan.d_first_mt; a.clo = plan.d_mt_clo; a.chi = plan.d_mt_chi;
+  a.part = part; a.meta = plan.d_meta; a.meta_stride = plan.meta_stride;
   a.ctr = plan.d_ctr; a.expected = plan.d_expected; a.pair_offset = plan.pair_offset;
   a.epi = epi;
   const int MP = padded_tokens(in.M);

@@ -38,6 +38,8 @@ struct GemmSeg {
   int xoff;       // column offset into the activation rows for this segment
 };
 
+constexpr int kMetaStride = 36;   // ints per 16-row tile in the piece table: count + up to 35 offsets
+
 struct GemmPlan {
   int nseg;
   GemmSeg seg[6];
@@ -50,11 +52,10 @@ struct GemmPlan {
   long long U;      // n_tiles * 8 * KR work units
   int pair_offset;  // > 0: tiles T and T + pair_offset are finalized together (group = T % pair_offset)
   int n_groups;
-  int* d_mt_clo;      // DEVICE [n_tiles*8] first CTA contributing to a 16-row tile
-  int* d_mt_chi;      // DEVICE [n_tiles*8] last CTA contributing to a 16-row tile
-  int* d_first_mt;    // DEVICE [grid]      first 16-row tile of a CTA's range
   int* d_ctr;         // DEVICE [n_groups] tickets taken (zero between launches)
   int* d_expected;    // DEVICE [n_groups] tickets that complete a group
+  int* d_meta;        // DEVICE [n_tiles*8][meta_stride]: piece count, then piece offsets (CTA order) per 16-row tile
+  int meta_stride;    // <= kMetaStride
 };
 
 __host__ __device__ inline int padded_tokens(int M) { return M <= 8 ? 8 : (M <= 32 ? 32 : 128); }
@@ -79,7 +80,7 @@ struct EpiArgs {
   float* res0;            // FC: out; RES with res_in == NULL: the fresh rows' g
   const float* res_in;    // RES: residual in (NULL: first residual = g or <mask>)
   float* res_out;         // RES: residual out (may be NULL)
-  const bf16* mask_vec;   // <mask> representation [2h]
+  const float* mask_res;  // g half of the <mask> representation as fp32 [h]: the <mask> rows' first residual
   const bf16* gamma;      // gain applied to the hi/lo output
   bf16* out_hi; bf16* out_lo; long long ld_out;
   float* ss_out;
@@ -89,7 +90,7 @@ struct EpiArgs {
   // EPI_FC prologue: shifted token embedding of the fresh rows
   const int32_t* tokens; int vocab; const bf16* embed; const bf16* gamma_e;
   // EPI_QKV
-  int Hq, Hkv, dh; const int32_t* seq_lens; float rope_theta;
+  int Hq, Hkv, dh; const int32_t* seq_lens; const float2* rope_tab;  // [positions][dh/2] (cos, sin)
   bf16* q_hi; bf16* q_lo; bf16* k_new; bf16* v_new; bf16* k_cache; bf16* v_cache; long long P_cap;
 };
 
@@ -112,15 +113,18 @@ struct GemmArgs {
   StreamArgs s;
   int slots;
   long long U;
-  float* part; const int* first_mt; const int* clo; const int* chi;
+  float* part;        // [grid][slots] pieces of 16 x MP floats
   int* ctr; const int* expected; int pair_offset;
+  const int* meta; int meta_stride;
   EpiArgs epi;
 };
 
 cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const EpiArgs& epi, float* part, cudaStream_t st);
+// (cos, sin) table of RoPE for positions 0 .. n_pos-1 (once, at init)
+cudaError_t launch_rope_table(float2* tab, int n_pos, int dh, float theta, cudaStream_t st);
 // z row of the <mask> rows and the 1/rms of its g half (once, at init)
 cudaError_t launch_mask_row(const bf16* mask_vec, const bf16* norm_g, const bf16* norm_e, int h, float eps, bf16* z_hi,
-                            bf16* z_lo, float* rstd_mask, cudaStream_t st);
+                            bf16* z_lo, float* rstd_mask, float* mask_res, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
 // Split-KV grouped-query attention over the cache (rows 0 .. P_b-1) and the step's new rows + combine.
