@@ -266,7 +266,10 @@ def run_ours(args):
             "step_bytes": bytes_step, "step_gbs": step_gbs,
             "step_frac_of_hbm_peak": step_gbs / hbm_peak, "step_frac_of_8tbs": step_gbs / 8000.0,
             "roofline": {"bound": "hbm", "kernel": "lm_head_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                         "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}", "traffic": args.lm_traffic,
+                         "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
+                         "traffic": args.lm_traffic if args.lm_traffic is not None else lm_bytes * LM_READ_RATIO + LM_WRITE_BYTES,
+                         "traffic_source": "ncu capture of a vocab-32768 launch (profiles/lm_head_kernel_C3_vocab32768.txt), reads "
+                                           "scaled by the bytes streamed, writes taken as measured",
                          "bytes_per_launch": lm_bytes, "us_per_launch": 1e3 * lm_avg_ms},
             "e2e": {"value": world * args.steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
@@ -301,6 +304,12 @@ def cpu_baseline(w, wt, inp, rows):
     return {"value": 1.0 / (t2 - t0), "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
             "sample": f"1 full step of workload {w.name} (N-gram table cut to 200k rows for the dict build)",
             "forward_s": t1 - t0, "topk_tree_s": t2 - t1}
+
+
+# DRAM traffic of one LM-head launch, from the committed ncu capture of the vocab-32768 case of the same
+# kernel: dram__bytes_read / algorithmic bytes, and dram__bytes_write (per-CTA results, independent of vocab).
+LM_READ_RATIO = 335.762e6 / 335.544e6
+LM_WRITE_BYTES = 3.7e6
 
 
 def main():
