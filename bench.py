@@ -157,16 +157,12 @@ def run_reference(args):
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
-    from paper_2601_19278_b200 import runner, synthetic as syn
+    from paper_2601_19278_b200 import replicas, runner, synthetic as syn
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = replicas.env()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init(world, "nccl", dev)
 
     w = syn.WORKLOADS[args.workload]
     if args.vocab:
@@ -183,9 +179,7 @@ def run_ours(args):
     lm_bytes = 2 * w.vocab * w.hidden
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(world, torch.cuda.synchronize)
 
     def step(i):
         ses.step(step_counter=i)
@@ -240,15 +234,12 @@ def run_ours(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], world, dev)
     assert ses.draft.device_status() == 0
 
     if rank == 0:
         ms_per_step = total_ms / args.steps
-        value = world * args.steps / (total_ms * 1e-3)
+        value = replicas.job_steps_per_second(world, args.steps, total_ms)
         lm_avg_ms = sum(lm_ms) / len(lm_ms)
         achieved = lm_bytes / (lm_avg_ms * 1e-3) / 1e9
         step_gbs = bytes_step / (ms_per_step * 1e-3) / 1e9
@@ -271,7 +262,7 @@ def run_ours(args):
                          "traffic_source": "ncu capture of a vocab-32768 launch (profiles/lm_head_kernel_C3_vocab32768.txt), reads "
                                            "scaled by the bytes streamed, writes taken as measured",
                          "bytes_per_launch": lm_bytes, "us_per_launch": 1e3 * lm_avg_ms},
-            "e2e": {"value": world * args.steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": replicas.job_steps_per_second(world, args.steps, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
             "gpu_launches": args.steps * n_launch,
             "clocks": clocks,
@@ -280,8 +271,7 @@ def run_ours(args):
             line["cpu_baseline"] = cpu_baseline(w, wt, inp, rows)
         print(json.dumps(line))
     ses.close()
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.finish(world)
 
 
 def cpu_baseline(w, wt, inp, rows):
