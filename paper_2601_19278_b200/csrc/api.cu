@@ -22,7 +22,8 @@ struct Workspace {
   float* part = nullptr;        // split partials of the current projection
   float* res0 = nullptr;        // [max_batch*K, h]  g of the fresh rows (first residual)
   float* x1 = nullptr;          // [Mmax, h] residual stream after attention
-  bf16 *z_hi = nullptr, *z_lo = nullptr;   // [Mmax + 1, 2h]: fresh rows' z, last row = the <mask> row
+  bf16 *z_hi = nullptr, *z_lo = nullptr;   // [Mmax, 2h]: z row of every token row (b, r); <mask> rows are copies of zmask
+  bf16 *zmask_hi = nullptr, *zmask_lo = nullptr;   // [2h] the <mask> row, written once at init
   bf16 *q_hi = nullptr, *q_lo = nullptr;   // [Mmax, Hq*dh]
   bf16 *k_new = nullptr, *v_new = nullptr; // [max_batch, Hkv, 16, dh]
   bf16 *a_hi = nullptr, *a_lo = nullptr;   // [Mmax, Hq*dh]
@@ -56,6 +57,7 @@ struct dart_handle {
   uint32_t ng_mask = 0, ng_max_probe = 0;
   float wl[8], wv[8], wn, miss;
   std::vector<void*> owned;  // small device arrays (plan tables, counters)
+  int z_B = -1, z_F = -1;    // row pattern (batch, fresh rows) the <mask> rows of z were last written for
   int prof_stage = -1;       // measurement aid: stage whose kernels the next call brackets with events
   cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
 };
@@ -168,8 +170,10 @@ size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_p
   TAKE(part, float*, part_max_floats * sizeof(float));
   TAKE(res0, float*, Mmax * c.hidden * sizeof(float));
   TAKE(x1, float*, Mmax * c.hidden * sizeof(float));
-  TAKE(z_hi, bf16*, (Mmax + 1) * 2 * c.hidden * sizeof(bf16));
-  TAKE(z_lo, bf16*, (Mmax + 1) * 2 * c.hidden * sizeof(bf16));
+  TAKE(z_hi, bf16*, Mmax * 2 * c.hidden * sizeof(bf16));
+  TAKE(z_lo, bf16*, Mmax * 2 * c.hidden * sizeof(bf16));
+  TAKE(zmask_hi, bf16*, (size_t)2 * c.hidden * sizeof(bf16));
+  TAKE(zmask_lo, bf16*, (size_t)2 * c.hidden * sizeof(bf16));
   TAKE(q_hi, bf16*, Mmax * dq * sizeof(bf16));
   TAKE(q_lo, bf16*, Mmax * dq * sizeof(bf16));
   TAKE(k_new, bf16*, (size_t)c.max_batch * c.n_kv_heads * 16 * c.head_dim * sizeof(bf16));
@@ -341,10 +345,9 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
 
   // the <mask> rows' z (last row of the z buffers) and the 1/rms of their g half: constants of the model
   {
-    const size_t mrow = (size_t)cfg->max_batch * cfg->K * 2 * cfg->hidden;
     INIT_CHECK(launch_mask_row(static_cast<const bf16*>(weights->mask_vec), static_cast<const bf16*>(weights->norm_g),
-                               static_cast<const bf16*>(weights->norm_e), cfg->hidden, cfg->rms_eps, h->ws.z_hi + mrow,
-                               h->ws.z_lo + mrow, h->ws.rstd_mask, h->ws.mask_res, nullptr));
+                               static_cast<const bf16*>(weights->norm_e), cfg->hidden, cfg->rms_eps, h->ws.zmask_hi,
+                               h->ws.zmask_lo, h->ws.rstd_mask, h->ws.mask_res, nullptr));
   }
 
   INIT_CHECK(launch_rope_table(h->ws.rope_tab, cfg->max_prefix + cfg->K, cfg->head_dim, cfg->rope_theta, nullptr));
@@ -435,7 +438,6 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int M = B * K, MP = padded_tokens(M);
   const int hdim = c.hidden, dq = c.n_q_heads * c.head_dim;
-  const long long mask_row = (long long)c.max_batch * K;
   Workspace& ws = h->ws;
   cudaError_t e;
   auto mark = [&](int stage, bool begin) {
@@ -443,6 +445,12 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   };
   EpiArgs ep;
   GemmInput gi;
+
+  // the <mask> rows of z are constant; they are (re)written only when the row pattern changes
+  if (h->z_B != B || h->z_F != F) {
+    if ((e = launch_fill_mask_rows(ws.z_hi, ws.z_lo, ws.zmask_hi, ws.zmask_lo, B, K, F, 2 * hdim, st)) != cudaSuccess) return fail_cuda(h, e);
+    h->z_B = B; h->z_F = F;
+  }
 
   // S0: feature-fusion FC on the fresh rows; epilogue: residual g, z g-half (gain-scaled), sums of squares;
   // prologue: z e-half = RMSNorm(embedding of the next token)
@@ -454,7 +462,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
     ep.out_hi = ws.z_hi; ep.out_lo = ws.z_lo; ep.ld_out = 2 * hdim; ep.ss_out = ws.ss_g;
     ep.tokens = in->tokens; ep.vocab = c.vocab; ep.embed = static_cast<const bf16*>(h->w.embed);
     ep.gamma_e = static_cast<const bf16*>(h->w.norm_e);
-    gi = {static_cast<const bf16*>(in->feats), nullptr, c.feat_in, B * F, 0, 0, 0};
+    gi = {static_cast<const bf16*>(in->feats), nullptr, c.feat_in, B * F};
     if ((e = launch_gemm_rows(h->plan_fc, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   }
   mark(0, false);
@@ -467,7 +475,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ep.Hq = c.n_q_heads; ep.Hkv = c.n_kv_heads; ep.dh = c.head_dim; ep.seq_lens = in->seq_lens; ep.rope_tab = ws.rope_tab;
   ep.q_hi = ws.q_hi; ep.q_lo = ws.q_lo; ep.k_new = ws.k_new; ep.v_new = ws.v_new;
   ep.k_cache = static_cast<bf16*>(in->k_cache); ep.v_cache = static_cast<bf16*>(in->v_cache); ep.P_cap = c.max_prefix;
-  gi = {ws.z_hi, ws.z_lo, 2 * hdim, M, K, F, mask_row};
+  gi = {ws.z_hi, ws.z_lo, 2 * hdim, M};
   if ((e = launch_gemm_rows(h->plan_qkv, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(1, false);
 
@@ -499,7 +507,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ep.res0 = ws.res0; ep.res_in = nullptr; ep.res_out = ws.x1; ep.mask_res = ws.mask_res;
   ep.gamma = static_cast<const bf16*>(h->w.norm_post);
   ep.out_hi = ws.n_hi; ep.out_lo = ws.n_lo; ep.ld_out = hdim; ep.ss_out = ws.ss_1;
-  gi = {ws.a_hi, ws.a_lo, dq, M, 0, 0, 0};
+  gi = {ws.a_hi, ws.a_lo, dq, M};
   if ((e = launch_gemm_rows(h->plan_o, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(3, false);
 
@@ -509,7 +517,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ep.mode = EPI_GATE_UP; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
   ep.ss_in = ws.ss_1; ep.ss_tiles = h->h_tiles; ep.ss_mp = MP;
   ep.out_hi = ws.u_hi; ep.out_lo = ws.u_lo; ep.ld_out = c.mlp_inter;
-  gi = {ws.n_hi, ws.n_lo, hdim, M, 0, 0, 0};
+  gi = {ws.n_hi, ws.n_lo, hdim, M};
   if ((e = launch_gemm_rows(h->plan_gu, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(4, false);
 
@@ -519,7 +527,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ep.mode = EPI_RES; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
   ep.res_in = ws.x1; ep.res_out = nullptr; ep.gamma = static_cast<const bf16*>(h->w.norm_final);
   ep.out_hi = ws.n_hi; ep.out_lo = ws.n_lo; ep.ld_out = hdim; ep.ss_out = ws.ss_2;
-  gi = {ws.u_hi, ws.u_lo, c.mlp_inter, M, 0, 0, 0};
+  gi = {ws.u_hi, ws.u_lo, c.mlp_inter, M};
   if ((e = launch_gemm_rows(h->plan_down, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(5, false);
 

@@ -193,18 +193,20 @@ __device__ __noinline__ void finalize_group(const GemmArgs& p, int group, int MP
       float q0, q1;
       tile_rows_sum2(x0 * x0, x1 * x1, sh, q0, q1);
       float* res = e.mode == EPI_FC ? e.res0 : e.res_out;
+      // the FC's token index counts fresh rows only; its z row is the step's row (b, r)
+      const int o0 = e.mode == EPI_FC ? (t0 / F) * K + t0 % F : t0, o1 = e.mode == EPI_FC ? (t1 / F) * K + t1 % F : t1;
       bf16 hi, lo;
       if (ok0) {
         if (res != nullptr) res[(size_t)t0 * e.h + n] = x0;
         split_bf16(x0 * gam, hi, lo);
-        e.out_hi[(size_t)t0 * e.ld_out + n] = hi;
-        e.out_lo[(size_t)t0 * e.ld_out + n] = lo;
+        e.out_hi[(size_t)o0 * e.ld_out + n] = hi;
+        e.out_lo[(size_t)o0 * e.ld_out + n] = lo;
       }
       if (ok1) {
         if (res != nullptr) res[(size_t)t1 * e.h + n] = x1;
         split_bf16(x1 * gam, hi, lo);
-        e.out_hi[(size_t)t1 * e.ld_out + n] = hi;
-        e.out_lo[(size_t)t1 * e.ld_out + n] = lo;
+        e.out_hi[(size_t)o1 * e.ld_out + n] = hi;
+        e.out_lo[(size_t)o1 * e.ld_out + n] = lo;
       }
       if (row == 0 && t0 < M) e.ss_out[(size_t)Ta * MP + t0] = q0;
       if (row == 0 && t1 < M) e.ss_out[(size_t)Ta * MP + t1] = q1;
@@ -267,6 +269,7 @@ __device__ __noinline__ void finalize_group(const GemmArgs& p, int group, int MP
 __device__ __noinline__ void embed_rows(const GemmArgs& p, float* sh) {
   const EpiArgs& e = p.epi;
   const int ftok = blockIdx.x;
+  const int orow = (ftok / e.F) * e.K + ftok % e.F;   // z row of fresh row (b, r)
   const int id = min(max(e.tokens[ftok], 0), e.vocab - 1);
   const bf16* row = e.embed + (size_t)id * e.h;
   float ss = 0.f;
@@ -279,8 +282,8 @@ __device__ __noinline__ void embed_rows(const GemmArgs& p, float* sh) {
   for (int n = threadIdx.x; n < e.h; n += blockDim.x) {
     bf16 hi, lo;
     split_bf16(__bfloat162float(row[n]) * rs * __bfloat162float(e.gamma_e[n]), hi, lo);
-    e.out_hi[(size_t)ftok * e.ld_out + e.h + n] = hi;
-    e.out_lo[(size_t)ftok * e.ld_out + e.h + n] = lo;
+    e.out_hi[(size_t)orow * e.ld_out + e.h + n] = hi;
+    e.out_lo[(size_t)orow * e.ld_out + e.h + n] = lo;
   }
 }
 
@@ -421,6 +424,22 @@ cudaError_t launch_rope_table(float2* tab, int n_pos, int dh, float theta, cudaS
   return cudaGetLastError();
 }
 
+__global__ void fill_mask_rows_kernel(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int K, int F, int width) {
+  const int tok = blockIdx.x;
+  if (tok % K < F) return;
+  const uint4* sh = reinterpret_cast<const uint4*>(zmask_hi);
+  const uint4* sl = reinterpret_cast<const uint4*>(zmask_lo);
+  uint4* dh = reinterpret_cast<uint4*>(z_hi + (size_t)tok * width);
+  uint4* dl = reinterpret_cast<uint4*>(z_lo + (size_t)tok * width);
+  for (int i = threadIdx.x; i < width / 8; i += blockDim.x) { dh[i] = sh[i]; dl[i] = sl[i]; }
+}
+
+cudaError_t launch_fill_mask_rows(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int B, int K, int F, int width,
+                                  cudaStream_t st) {
+  fill_mask_rows_kernel<<<B * K, 256, 0, st>>>(z_hi, z_lo, zmask_hi, zmask_lo, K, F, width);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_mask_row(const bf16* mask_vec, const bf16* norm_g, const bf16* norm_e, int h, float eps, bf16* z_hi,
                             bf16* z_lo, float* rstd_mask, float* mask_res, cudaStream_t st) {
   mask_row_kernel<<<1, 256, 0, st>>>(mask_vec, norm_g, norm_e, h, eps, z_hi, z_lo, rstd_mask, mask_res);
@@ -447,7 +466,6 @@ cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const Ep
   a.s.nseg = plan.nseg;
   a.s.Kd = plan.Kd; a.s.SK = plan.SK; a.s.KR = plan.KR; a.slots = plan.slots; a.U = plan.U;
   a.s.x_hi = in.x_hi; a.s.x_lo = in.x_lo != nullptr ? in.x_lo : in.x_hi; a.s.ldx = in.ldx; a.s.M = in.M;
-  a.s.x_K = in.x_K; a.s.x_F = in.x_F; a.s.x_mask_row = in.x_mask_row;
   a.part = part; a.meta = plan.d_meta; a.meta_stride = plan.meta_stride;
   a.ctr = plan.d_ctr; a.expected = plan.d_expected; a.pair_offset = plan.pair_offset;
   a.epi = epi;

@@ -64,8 +64,6 @@ struct GemmInput {
   const bf16* x_hi; const bf16* x_lo;  // [rows, ldx] activations as hi (+ lo, may be NULL)
   long long ldx;
   int M;              // valid tokens
-  int x_K, x_F;       // x_K > 0: token (b, r) reads row b*x_F + r if r < x_F, else row x_mask_row
-  long long x_mask_row;
 };
 
 enum EpiMode : int { EPI_FC = 0, EPI_QKV = 1, EPI_RES = 2, EPI_GATE_UP = 3 };
@@ -105,8 +103,6 @@ struct StreamArgs {
   const bf16* x_lo;   // lo part (== x_hi when the input is plain bf16)
   long long ldx;
   int M;              // valid token rows
-  int x_K, x_F;       // x_K > 0: token (b, r) reads row b*x_F + r if r < x_F, else row x_mask_row
-  long long x_mask_row;
 };
 
 struct GemmArgs {
@@ -122,6 +118,9 @@ struct GemmArgs {
 cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const EpiArgs& epi, float* part, cudaStream_t st);
 // (cos, sin) table of RoPE for positions 0 .. n_pos-1 (once, at init)
 cudaError_t launch_rope_table(float2* tab, int n_pos, int dh, float theta, cudaStream_t st);
+// Copies the <mask> row into every z row (b, r) with r >= F (when the batch size or F changes)
+cudaError_t launch_fill_mask_rows(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int B, int K, int F, int width,
+                                  cudaStream_t st);
 // z row of the <mask> rows and the 1/rms of its g half (once, at init)
 cudaError_t launch_mask_row(const bf16* mask_vec, const bf16* norm_g, const bf16* norm_e, int h, float eps, bf16* z_hi,
                             bf16* z_lo, float* rstd_mask, float* mask_res, cudaStream_t st);

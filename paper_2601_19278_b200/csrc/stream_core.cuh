@@ -60,12 +60,7 @@ __device__ __forceinline__ void stream_units(const StreamArgs& a, long long u0, 
   for (int i = 0; i < NT; ++i) {
     int tok = i * 8 + g;
     if (tok >= a.M) tok = 0;  // padded token rows read row 0; their results are never used
-    long long rowi = tok;
-    if (a.x_K > 0) {
-      const int b = tok / a.x_K, r = tok % a.x_K;
-      rowi = r < a.x_F ? (long long)b * a.x_F + r : a.x_mask_row;
-    }
-    xh[i] = a.x_hi + rowi * a.ldx;
+    xh[i] = a.x_hi + (long long)tok * a.ldx;
   }
 
   float acc[NT][4];
