@@ -38,6 +38,8 @@ struct Workspace {
   float *lm_stats = nullptr, *lm_key = nullptr, *lm_y = nullptr;
   int32_t* lm_id = nullptr;
   int* status = nullptr;
+  float* lm_pieces = nullptr;   // [SMs][128][MPmax] partial logits of vocabulary tiles cut between CTAs
+  int* lm_flags = nullptr;      // [SMs] launch tag of each CTA's piece
 };
 
 }  // namespace
@@ -49,6 +51,12 @@ struct dart_handle {
   int n_sm = 0;
   int last_cuda_error = 0;
   GemmPlan plan_fc, plan_qkv, plan_o, plan_gu, plan_down;
+  bool umma = false;         // projections run on the tcgen05 / TMA kernels (tensor maps could be encoded)
+  UmmaMaps maps_fc, maps_qkv, maps_o, maps_gu, maps_down;
+  CUtensorMap map_lm;        // the LM head's weight matrix
+  int lm_tag = 0;            // launch counter of the LM head (marks its cross-CTA pieces)
+  int maps_M = -1;           // token rows the activation tensor maps were encoded for
+  const void* maps_feats = nullptr; int maps_fc_M = -1;
   int lm_grid = 0;
   int attn_pairs_cap = 0;  // capacity of the attention partial buffers in (sequence, chunk) pairs
   int h_tiles = 0;         // 128-row tiles of a hidden-sized row
@@ -145,7 +153,58 @@ void make_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int gri
   }
 }
 
-size_t part_floats(const GemmPlan& p, int MP) { return (size_t)p.grid * p.slots * 16 * MP; }
+// The same cut for the tcgen05 kernel: units are (128-row tile, 64-k block), one persistent CTA per SM, a
+// CTA's piece of a tile holds all 128 rows.  The piece table keeps the 16-row granularity of the fused
+// finalize: the j-th 16 rows of a 128-row piece at slot s are "piece" 8 s + j.
+void make_umma_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int grid_target, int pair_offset) {
+  GemmPlan& p = ph.plan;
+  memset(&p, 0, sizeof(p));
+  p.nseg = nseg;
+  p.umma = 1;
+  int tiles = 0;
+  for (int i = 0; i < 6; ++i) {
+    if (i < nseg) {
+      p.seg[i] = segs[i];
+      p.seg[i].tile0 = tiles;
+      tiles += (segs[i].rows + 127) / 128;
+    } else {
+      p.seg[i] = p.seg[0];
+    }
+  }
+  p.Kd = Kd;
+  p.SK = (Kd + 63) / 64;
+  p.KR = p.SK;
+  p.n_tiles = tiles;
+  p.U = (long long)tiles * p.KR;
+  p.grid = (int)((long long)grid_target < p.U ? grid_target : p.U);
+  while (p.grid > 1 && (p.KR + (p.U / p.grid) - 1) / (p.U / p.grid) + 1 > kMetaStride - 1) p.grid /= 2;
+  p.pair_offset = pair_offset;
+  p.n_groups = pair_offset > 0 ? pair_offset : tiles;
+  p.slots = 1;
+  p.meta_stride = kMetaStride;
+  ph.expected.assign(p.n_groups, 0);
+  ph.meta.assign((size_t)tiles * 8 * kMetaStride, 0);
+  for (int c = 0; c < p.grid; ++c) {
+    const long long u0 = ((long long)c * p.U) / p.grid, u1 = ((long long)(c + 1) * p.U) / p.grid;
+    if (u0 >= u1) continue;
+    const int t0 = (int)(u0 / p.KR), t1 = (int)((u1 - 1) / p.KR);
+    if (t1 - t0 + 1 > p.slots) p.slots = t1 - t0 + 1;
+  }
+  for (int c = 0; c < p.grid; ++c) {
+    const long long u0 = ((long long)c * p.U) / p.grid, u1 = ((long long)(c + 1) * p.U) / p.grid;
+    if (u0 >= u1) continue;
+    const int t0 = (int)(u0 / p.KR), t1 = (int)((u1 - 1) / p.KR);
+    for (int t = t0; t <= t1; ++t) {
+      ph.expected[pair_offset > 0 ? t % pair_offset : t] += 1;
+      for (int j = 0; j < 8; ++j) {
+        int& n = ph.meta[(size_t)(t * 8 + j) * kMetaStride];
+        if (n < kMetaStride - 1) ph.meta[(size_t)(t * 8 + j) * kMetaStride + 1 + n++] = (c * p.slots + (t - t0)) * 8 + j;
+      }
+    }
+  }
+}
+
+size_t part_floats(const GemmPlan& p, int MP) { return (size_t)p.grid * p.slots * (p.umma ? 128 : 16) * MP; }
 
 struct Layout {
   size_t total = 0;
@@ -193,6 +252,8 @@ size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_p
   TAKE(bg, float*, (size_t)c.max_batch * (c.topk + (size_t)(c.K - 1) * c.topk * c.topk) * sizeof(float));
   TAKE(o_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * c.head_dim * sizeof(float));
   TAKE(ml_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * 2 * sizeof(float));
+  TAKE(lm_pieces, float*, (size_t)lm_grid * 128 * MPmax * sizeof(float));
+  TAKE(lm_flags, int*, (size_t)lm_grid * sizeof(int));
   TAKE(lm_stats, float*, (size_t)lm_grid * MPmax * 2 * sizeof(float));
   TAKE(lm_key, float*, (size_t)lm_grid * MPmax * 32 * sizeof(float));
   TAKE(lm_y, float*, (size_t)lm_grid * MPmax * 32 * sizeof(float));
@@ -207,8 +268,11 @@ struct PlanSet {
   size_t part_max = 0;
 };
 
-void build_plans(const dart_config& c, const dart_weights* w, int n_sm, PlanSet& ps) {
-  const int grid = 2 * n_sm;
+void build_plans(const dart_config& c, const dart_weights* w, int n_sm, bool umma, PlanSet& ps) {
+  const int grid = umma ? n_sm : 2 * n_sm;
+  auto make_plan_host = [&](PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int g, int pair) {
+    if (umma) make_umma_plan_host(ph, segs, nseg, Kd, g, pair); else ::make_plan_host(ph, segs, nseg, Kd, g, pair);
+  };
   const int h = c.hidden, dq = c.n_q_heads * c.head_dim, dkv = c.n_kv_heads * c.head_dim;
   auto W = [&](const void* p, long long off) { return w ? static_cast<const bf16*>(p) + off : nullptr; };
   GemmSeg s[6];
@@ -238,6 +302,14 @@ void build_plans(const dart_config& c, const dart_weights* w, int n_sm, PlanSet&
     const size_t f = part_floats(all[i]->plan, MPmax);
     if (f > ps.part_max) ps.part_max = f;
   }
+}
+
+// Piece area that serves either kernel family (the choice is made at init, the size must not depend on it).
+size_t part_capacity(const dart_config& c, int n_sm) {
+  PlanSet a, b;
+  build_plans(c, nullptr, n_sm, false, a);
+  build_plans(c, nullptr, n_sm, true, b);
+  return a.part_max > b.part_max ? a.part_max : b.part_max;
 }
 
 int attn_pairs_capacity(const dart_config& c, int n_sm) { return (2 * n_sm) / c.n_kv_heads + 2 * c.max_batch + 2; }
@@ -279,9 +351,7 @@ const char* dart_status_string(int status) {
 size_t dart_workspace_bytes(const dart_config* cfg) {
   if (!config_ok(cfg)) return 0;
   const int n_sm = 148;  // sized for a B200; dart_draft_init uses the device's own count
-  PlanSet ps;
-  build_plans(*cfg, nullptr, n_sm, ps);
-  return layout_workspace(*cfg, ps.part_max, attn_pairs_capacity(*cfg, n_sm), 2 * n_sm, nullptr, nullptr);
+  return layout_workspace(*cfg, part_capacity(*cfg, n_sm), attn_pairs_capacity(*cfg, n_sm), 2 * n_sm, nullptr, nullptr);
 }
 
 int dart_last_cuda_error(const dart_handle* h) { return h ? h->last_cuda_error : g_init_cuda_error; }
@@ -323,9 +393,24 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
     return DART_ERR_CUDA;                                \
   }
 
+#ifndef DART_FORCE_LEGACY
+  {
+    CUtensorMap probe;   // the encoder is there and accepts a weight matrix: use the tcgen05 / TMA kernels
+    h->umma = tmap_encode_bf16(&probe, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 128) == cudaSuccess;
+  }
+#endif
   PlanSet ps;
-  build_plans(*cfg, weights, n_sm, ps);
+  build_plans(*cfg, weights, n_sm, h->umma, ps);
   PlanHost* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
+  if (h->umma) {
+    INIT_CHECK(tmap_encode_bf16(&h->map_lm, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 128));
+    UmmaMaps* maps[5] = {&h->maps_fc, &h->maps_qkv, &h->maps_o, &h->maps_gu, &h->maps_down};
+    for (int i = 0; i < 5; ++i) {
+      const GemmPlan& pl = plans[i]->plan;
+      for (int sg = 0; sg < pl.nseg; ++sg)
+        INIT_CHECK(tmap_encode_bf16(&maps[i]->W[sg], pl.seg[sg].W, pl.Kd, pl.seg[sg].rows, (unsigned long long)pl.seg[sg].ld * 2, 64, 128));
+    }
+  }
   for (int i = 0; i < 5; ++i) {
     PlanHost& ph = *plans[i];
     INIT_CHECK(upload(h, ph.expected, &ph.plan.d_expected));
@@ -338,9 +423,10 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   if (h->lm_grid > cfg->vocab / 16) h->lm_grid = cfg->vocab / 16;
   h->attn_pairs_cap = attn_pairs_capacity(*cfg, n_sm);
 
-  h->ws.bytes = layout_workspace(*cfg, ps.part_max, h->attn_pairs_cap, 2 * n_sm, nullptr, nullptr);
+  const size_t part_cap = part_capacity(*cfg, n_sm);
+  h->ws.bytes = layout_workspace(*cfg, part_cap, h->attn_pairs_cap, 2 * n_sm, nullptr, nullptr);
   INIT_CHECK(cudaMalloc(&h->ws.base, h->ws.bytes));
-  layout_workspace(*cfg, ps.part_max, h->attn_pairs_cap, 2 * n_sm, static_cast<char*>(h->ws.base), &h->ws);
+  layout_workspace(*cfg, part_cap, h->attn_pairs_cap, 2 * n_sm, static_cast<char*>(h->ws.base), &h->ws);
   INIT_CHECK(cudaMemset(h->ws.base, 0, h->ws.bytes));
 
   // the <mask> rows' z (last row of the z buffers) and the 1/rms of their g half: constants of the model
@@ -445,6 +531,21 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   };
   EpiArgs ep;
   GemmInput gi;
+  if (h->umma && h->maps_M != M) {
+    // activation tensor maps: [M rows][width], box = 64 k x MP rows; rows past M read as zeros
+    struct { UmmaMaps* m; const bf16* hi; const bf16* lo; int width; } xin[4] = {
+        {&h->maps_qkv, ws.z_hi, ws.z_lo, 2 * hdim}, {&h->maps_o, ws.a_hi, ws.a_lo, dq},
+        {&h->maps_gu, ws.n_hi, ws.n_lo, hdim}, {&h->maps_down, ws.u_hi, ws.u_lo, c.mlp_inter}};
+    for (int i = 0; i < 4; ++i) {
+      if ((e = tmap_encode_bf16(&xin[i].m->Xhi, xin[i].hi, xin[i].width, M, (unsigned long long)xin[i].width * 2, 64, MP)) != cudaSuccess ||
+          (e = tmap_encode_bf16(&xin[i].m->Xlo, xin[i].lo, xin[i].width, M, (unsigned long long)xin[i].width * 2, 64, MP)) != cudaSuccess)
+        return fail_cuda(h, e);
+    }
+    h->maps_M = M;
+  }
+  auto project = [&](const GemmPlan& plan, const UmmaMaps& maps) -> cudaError_t {
+    return h->umma ? launch_umma_rows(plan, maps, gi, ep, ws.part, ws.status, st) : launch_gemm_rows(plan, gi, ep, ws.part, st);
+  };
 
   // the <mask> rows of z are constant; they are (re)written only when the row pattern changes
   if (h->z_B != B || h->z_F != F) {
@@ -463,7 +564,15 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
     ep.tokens = in->tokens; ep.vocab = c.vocab; ep.embed = static_cast<const bf16*>(h->w.embed);
     ep.gamma_e = static_cast<const bf16*>(h->w.norm_e);
     gi = {static_cast<const bf16*>(in->feats), nullptr, c.feat_in, B * F};
-    if ((e = launch_gemm_rows(h->plan_fc, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
+    if (h->umma && (h->maps_feats != in->feats || h->maps_fc_M != B * F)) {
+      // plain bf16 input: one box of 2 * MP rows, the rows past B * F (the "lo" half among them) read as zeros
+      if ((e = tmap_encode_bf16(&h->maps_fc.Xhi, in->feats, c.feat_in, B * F, (unsigned long long)c.feat_in * 2, 64,
+                                2 * padded_tokens(B * F))) != cudaSuccess)
+        return fail_cuda(h, e);
+      h->maps_fc.Xlo = h->maps_fc.Xhi;
+      h->maps_feats = in->feats; h->maps_fc_M = B * F;
+    }
+    if ((e = project(h->plan_fc, h->maps_fc)) != cudaSuccess) return fail_cuda(h, e);
   }
   mark(0, false);
 
@@ -476,7 +585,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ep.q_hi = ws.q_hi; ep.q_lo = ws.q_lo; ep.k_new = ws.k_new; ep.v_new = ws.v_new;
   ep.k_cache = static_cast<bf16*>(in->k_cache); ep.v_cache = static_cast<bf16*>(in->v_cache); ep.P_cap = c.max_prefix;
   gi = {ws.z_hi, ws.z_lo, 2 * hdim, M};
-  if ((e = launch_gemm_rows(h->plan_qkv, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
+  if ((e = project(h->plan_qkv, h->maps_qkv)) != cudaSuccess) return fail_cuda(h, e);
   mark(1, false);
 
   // S2: split-KV attention over cache rows 0 .. P_b-1 and the K new rows
@@ -508,7 +617,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ep.gamma = static_cast<const bf16*>(h->w.norm_post);
   ep.out_hi = ws.n_hi; ep.out_lo = ws.n_lo; ep.ld_out = hdim; ep.ss_out = ws.ss_1;
   gi = {ws.a_hi, ws.a_lo, dq, M};
-  if ((e = launch_gemm_rows(h->plan_o, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
+  if ((e = project(h->plan_o, h->maps_o)) != cudaSuccess) return fail_cuda(h, e);
   mark(3, false);
 
   // S4: gate/up; epilogue: u = SiLU(rstd1 * gate) * (rstd1 * up)
@@ -518,7 +627,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ep.ss_in = ws.ss_1; ep.ss_tiles = h->h_tiles; ep.ss_mp = MP;
   ep.out_hi = ws.u_hi; ep.out_lo = ws.u_lo; ep.ld_out = c.mlp_inter;
   gi = {ws.n_hi, ws.n_lo, hdim, M};
-  if ((e = launch_gemm_rows(h->plan_gu, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
+  if ((e = project(h->plan_gu, h->maps_gu)) != cudaSuccess) return fail_cuda(h, e);
   mark(4, false);
 
   // S5: down; epilogue: x2 = x1 + proj, gain-scaled hi/lo for the LM head, sums of squares
@@ -528,7 +637,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ep.res_in = ws.x1; ep.res_out = nullptr; ep.gamma = static_cast<const bf16*>(h->w.norm_final);
   ep.out_hi = ws.n_hi; ep.out_lo = ws.n_lo; ep.ld_out = hdim; ep.ss_out = ws.ss_2;
   gi = {ws.u_hi, ws.u_lo, c.mlp_inter, M};
-  if ((e = launch_gemm_rows(h->plan_down, gi, ep, ws.part, st)) != cudaSuccess) return fail_cuda(h, e);
+  if ((e = project(h->plan_down, h->maps_down)) != cudaSuccess) return fail_cuda(h, e);
   mark(5, false);
 
   // S6 + S7: LM head with fused log-softmax / top-k, then the merge
@@ -547,7 +656,15 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   lp.part_stats = ws.lm_stats; lp.part_key = ws.lm_key; lp.part_y = ws.lm_y; lp.part_id = ws.lm_id;
   lp.out_ids = out->topk_ids; lp.out_slogit = out->topk_slogit;
   mark(6, true);
-  if ((e = launch_lm_head(lp, st)) != cudaSuccess) return fail_cuda(h, e);
+  if (h->umma) {
+    // one CTA per SM at most: the CTAs of this kernel wait on one another's pieces, so all must be resident
+    const long long units = (long long)((c.vocab + 127) / 128) * ((hdim + 63) / 64);
+    lp.grid = (int)(units < h->n_sm ? units : h->n_sm);
+    e = launch_lm_head_umma(lp, h->map_lm, h->maps_gu.Xhi, h->maps_gu.Xlo, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
+  } else {
+    e = launch_lm_head(lp, st);
+  }
+  if (e != cudaSuccess) return fail_cuda(h, e);
   mark(6, false);
   mark(7, true);
   if ((e = launch_topk_merge(lp, st)) != cudaSuccess) return fail_cuda(h, e);

@@ -1,6 +1,7 @@
 // Internal interface between the C-ABI layer (api.cu) and the kernel translation units.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -8,9 +9,22 @@ namespace dart {
 
 typedef __nv_bfloat16 bf16;
 
+// All kernels of the step ask for the same (largest) shared-memory carve-out: the streaming kernels need
+// ~200 KB per SM, and an SM whose L1 / shared-memory split differs from what the next kernel wants has to
+// drain and reconfigure first, which serialises consecutive kernels and costs tens of microseconds a switch.
+inline void prefer_max_shared(const void* fn) {
+  static const void* seen[64];
+  static int n = 0;
+  for (int i = 0; i < n; ++i)
+    if (seen[i] == fn) return;
+  if (n < 64) seen[n++] = fn;
+  cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+}
+
 // Launch with programmatic stream serialization (see pdl_wait / pdl_trigger in common.cuh).
 template <class... KArgs, class... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  prefer_max_shared(reinterpret_cast<const void*>(kernel));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -51,6 +65,7 @@ struct GemmPlan {
   int slots;        // max 16-row tiles a CTA touches
   long long U;      // n_tiles * 8 * KR work units
   int pair_offset;  // > 0: tiles T and T + pair_offset are finalized together (group = T % pair_offset)
+  int umma;         // 1: units are (128-row tile, 64-k block) for the tcgen05 kernel (KR = k-blocks per tile), pieces hold 128 rows
   int n_groups;
   int* d_ctr;         // DEVICE [n_groups] tickets taken (zero between launches)
   int* d_expected;    // DEVICE [n_groups] tickets that complete a group
@@ -115,6 +130,26 @@ struct GemmArgs {
   EpiArgs epi;
 };
 
+// The same projections on the tcgen05 / TMA path (umma_gemm.cu): plan units are (128-row tile, 64-k block),
+// one persistent CTA per SM.  Tensor maps: one per weight segment, one each for the hi and lo activations
+// (box = 64 k x MP rows; a plain-bf16 input uses Xhi alone with a box of 2*MP rows, whose missing rows read 0).
+struct UmmaMaps {
+  CUtensorMap W[6];
+  CUtensorMap Xhi, Xlo;
+};
+struct UmmaGemmArgs {
+  GemmArgs g;
+  CUtensorMap mapW[6];
+  CUtensorMap mapXhi, mapXlo;
+  int has_lo;
+  int* status;   // device status word (DEV_TIMEOUT when a bounded wait ran out)
+};
+cudaError_t launch_umma_rows(const GemmPlan& plan, const UmmaMaps& maps, const GemmInput& in, const EpiArgs& epi, float* part,
+                             int* status, cudaStream_t st);
+// 2-D bf16 tensor map [outer][inner] (row stride ld_bytes), box {box_inner, box_outer}, 128-byte swizzle, zero fill.
+cudaError_t tmap_encode_bf16(CUtensorMap* m, const void* base, unsigned long long inner, unsigned long long outer,
+                             unsigned long long ld_bytes, unsigned box_inner, unsigned box_outer);
+
 cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const EpiArgs& epi, float* part, cudaStream_t st);
 // (cos, sin) table of RoPE for positions 0 .. n_pos-1 (once, at init)
 cudaError_t launch_rope_table(float2* tab, int n_pos, int dh, float theta, cudaStream_t st);
@@ -159,6 +194,18 @@ struct LmParams {
   int32_t* out_ids; float* out_slogit;  // [M, topk]
 };
 cudaError_t launch_lm_head(const LmParams& p, cudaStream_t st);
+// The tcgen05 / TMA LM head (p.grid CTAs, at most one per SM so that all of them are resident at once).
+// pieces: [grid][128][MP] fp32 partial logits of tiles cut between CTAs; flags: [grid] ints, a CTA's piece is
+// complete when its flag equals `tag` (a value no earlier launch used).
+struct LmUmmaArgs {
+  LmParams p;
+  CUtensorMap mapW, mapXhi, mapXlo;
+  int KB; long long U;
+  float* pieces; int* flags; int tag;
+  int* status;
+};
+cudaError_t launch_lm_head_umma(const LmParams& p, const CUtensorMap& mapW, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
+                                float* pieces, int* flags, int tag, int* status, cudaStream_t st);
 cudaError_t topk_merge_setup(int max_grid);  // once per device
 cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st);
 

@@ -17,6 +17,7 @@
 #include "common.cuh"
 #include "kernels.h"
 #include "stream_core.cuh"
+#include "umma.cuh"
 
 namespace dart {
 
@@ -34,6 +35,57 @@ __device__ __forceinline__ void list_insert(float& lk, float& ly, int& lid, floa
   const int pid = __shfl_up_sync(0xffffffffu, lid, 1);
   if (lane == pos) { lk = nk; ly = ny; lid = nid; }
   else if (lane > pos) { lk = pk; ly = py; lid = pid; }
+}
+
+// Folds `nrows` (<= 128) complete logits of token row tk (srow[0 .. nrows), vocabulary ids id0 + index) into
+// the CTA's running softmax statistics and its exact top list of that row (Algorithm 1 lines 6-8).  One warp.
+__device__ __forceinline__ void fold_token(const LmParams& p, const float* srow, int nrows, int id0, int tk, int lane,
+                                           float* st_key, float* st_y, int* st_id, float* st_ms) {
+  float lk = st_key[tk * 32 + lane], ly = st_y[tk * 32 + lane];
+  int lid = st_id[tk * 32 + lane];
+  float m_run = st_ms[2 * tk], s_run = st_ms[2 * tk + 1];
+  float yv[4], kv[4];
+  float tmax = -INFINITY;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int idx = lane + 32 * q;
+    const bool ok = idx < nrows;
+    yv[q] = ok ? srow[idx] * p.inv_temp : -INFINITY;
+    kv[q] = yv[q];
+    if (p.gumbel && ok) {
+      const uint32_t v = (uint32_t)(id0 + idx);
+      const uint4 rnd = philox4x32_10(make_uint4(v >> 2, (uint32_t)(tk % p.K), (uint32_t)(tk / p.K), p.step), p.seed_lo, p.seed_hi);
+      const uint32_t wsel = (v & 3) == 0 ? rnd.x : ((v & 3) == 1 ? rnd.y : ((v & 3) == 2 ? rnd.z : rnd.w));
+      kv[q] = yv[q] + gumbel_from_bits(wsel);
+    }
+    tmax = fmaxf(tmax, yv[q]);
+  }
+  tmax = warp_max(tmax);
+  const float m_new = fmaxf(m_run, tmax);
+  float part = 0.f;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) part += (lane + 32 * q < nrows) ? expf(yv[q] - m_new) : 0.f;
+  part = warp_sum(part);
+  s_run = s_run * expf(m_run - m_new) + part;
+  m_run = m_new;
+  float thr = __shfl_sync(0xffffffffu, lk, p.topk - 1);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const bool ok = lane + 32 * q < nrows;
+    unsigned mask = __ballot_sync(0xffffffffu, ok && kv[q] > thr);
+    while (mask) {
+      const int src = __ffs(mask) - 1;
+      const float nk = __shfl_sync(0xffffffffu, kv[q], src), ny = __shfl_sync(0xffffffffu, yv[q], src);
+      list_insert(lk, ly, lid, nk, ny, id0 + src + 32 * q, lane);
+      thr = __shfl_sync(0xffffffffu, lk, p.topk - 1);
+      mask &= mask - 1;
+      mask &= __ballot_sync(0xffffffffu, ok && kv[q] > thr);
+    }
+  }
+  st_key[tk * 32 + lane] = lk;
+  st_y[tk * 32 + lane] = ly;
+  st_id[tk * 32 + lane] = lid;
+  if (lane == 0) { st_ms[2 * tk] = m_run; st_ms[2 * tk + 1] = s_run; }
 }
 
 // Epilogue functor of the streaming core: complete logits of a 16-row vocab tile -> stage; every 128
@@ -72,54 +124,7 @@ struct LmEpi {
       __syncthreads();
       const int nrows = (slot + 1) * 16;
       const int id0 = (mt - slot) * 16;
-      for (int tk = warp; tk < p.M; tk += NW) {
-        float lk = st_key[tk * 32 + lane], ly = st_y[tk * 32 + lane];
-        int lid = st_id[tk * 32 + lane];
-        float m_run = st_ms[2 * tk], s_run = st_ms[2 * tk + 1];
-        float yv[4], kv[4];
-        float tmax = -INFINITY;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int idx = lane + 32 * q;
-          const bool ok = idx < nrows;
-          yv[q] = ok ? stage[tk * SROW + idx] * p.inv_temp : -INFINITY;
-          kv[q] = yv[q];
-          if (p.gumbel && ok) {
-            const uint32_t v = (uint32_t)(id0 + idx);
-            const uint4 rnd = philox4x32_10(make_uint4(v >> 2, (uint32_t)(tk % p.K), (uint32_t)(tk / p.K), p.step),
-                                            p.seed_lo, p.seed_hi);
-            const uint32_t wsel = (v & 3) == 0 ? rnd.x : ((v & 3) == 1 ? rnd.y : ((v & 3) == 2 ? rnd.z : rnd.w));
-            kv[q] = yv[q] + gumbel_from_bits(wsel);
-          }
-          tmax = fmaxf(tmax, yv[q]);
-        }
-        tmax = warp_max(tmax);
-        const float m_new = fmaxf(m_run, tmax);
-        float part = 0.f;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) part += (lane + 32 * q < nrows) ? expf(yv[q] - m_new) : 0.f;
-        part = warp_sum(part);
-        s_run = s_run * expf(m_run - m_new) + part;
-        m_run = m_new;
-        float thr = __shfl_sync(0xffffffffu, lk, p.topk - 1);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const bool ok = lane + 32 * q < nrows;
-          unsigned mask = __ballot_sync(0xffffffffu, ok && kv[q] > thr);
-          while (mask) {
-            const int src = __ffs(mask) - 1;
-            const float nk = __shfl_sync(0xffffffffu, kv[q], src), ny = __shfl_sync(0xffffffffu, yv[q], src);
-            list_insert(lk, ly, lid, nk, ny, id0 + src + 32 * q, lane);
-            thr = __shfl_sync(0xffffffffu, lk, p.topk - 1);
-            mask &= mask - 1;
-            mask &= __ballot_sync(0xffffffffu, ok && kv[q] > thr);
-          }
-        }
-        st_key[tk * 32 + lane] = lk;
-        st_y[tk * 32 + lane] = ly;
-        st_id[tk * 32 + lane] = lid;
-        if (lane == 0) { st_ms[2 * tk] = m_run; st_ms[2 * tk + 1] = s_run; }
-      }
+      for (int tk = warp; tk < p.M; tk += NW) fold_token(p, stage + tk * SROW, nrows, id0, tk, lane, st_key, st_y, st_id, st_ms);
     }
   }
 };
@@ -166,6 +171,266 @@ __global__ void __launch_bounds__(NW * 32, (NT == 1 ? 2 : 1)) lm_head_kernel(con
     p.part_id[o] = st_id[i];
   }
   for (int i = tid; i < MP * 2; i += NW * 32) p.part_stats[(size_t)c * MP * 2 + i] = st_ms[i];
+}
+
+// ------------------------------------------------------------------------------------------------------
+// The same LM head on the Blackwell data path: weights and activation slices arrive by TMA in a ring of
+// shared-memory stages, tcgen05.mma multiplies them straight from there (M = 128 vocabulary rows, N = hi and
+// lo token rows), the fp32 logits of a tile sit in tensor memory until four warps read them out and fold them.
+//
+// Work split: the flattened (128-row vocabulary tile, 64-k block) space is cut into gridDim.x equal ranges
+// (one persistent CTA per SM), so every CTA streams the same number of bytes even though V / 128 is no
+// multiple of the SM count.  A tile cut between CTAs belongs to the CTA that holds its first k-block: the
+// others (for which it is the *first* thing they do) write their partial logits to a piece slot and raise a
+// flag; the owner (for which it is the *last* thing it does) adds them in CTA order and folds.  Ownership
+// is static, so the per-CTA statistics and lists - and with them every output bit - do not depend on timing.
+// The owner's wait on the flags is bounded like every other wait here.
+// ------------------------------------------------------------------------------------------------------
+using namespace umma;
+
+constexpr int kLmUmmaThreads = 256;
+
+template <int MP>
+struct LmUmmaCfg {
+  static constexpr int N = 2 * MP;
+  static constexpr int XBytes = N * 64 * 2;
+  static constexpr int StageBytes = 128 * 64 * 2 + XBytes;
+  static constexpr int TmemCols = 2 * N < 32 ? 32 : 2 * N;
+  // epilogue shared memory: stage [8][129] floats, lists 3 x [MP][32], statistics [MP][2], 1/rms [MP]
+  static constexpr size_t EpiBytes = sizeof(float) * (8 * 129 + 3 * MP * 32 + 3 * MP);
+  static constexpr int Stages = MP == 8 ? 11 : (MP == 32 ? 7 : 3);
+  static constexpr size_t SmemBytes = (size_t)Stages * StageBytes + 1024 + EpiBytes;
+};
+
+template <int MP>
+__global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const __grid_constant__ LmUmmaArgs a) {
+  using C = LmUmmaCfg<MP>;
+  constexpr int SROW = 129;
+  const LmParams& p = a.p;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  float* stage = reinterpret_cast<float*>(ring + (size_t)C::Stages * C::StageBytes);   // [8][SROW]
+  float* st_key = stage + 8 * SROW;          // [MP][32]
+  float* st_y = st_key + MP * 32;
+  int* st_id = reinterpret_cast<int*>(st_y + MP * 32);
+  float* st_ms = reinterpret_cast<float*>(st_id + MP * 32);  // [MP][2]
+  float* s_rstd = st_ms + 2 * MP;                            // [MP]
+  __shared__ uint64_t full[C::Stages], empty[C::Stages], acc_full[2], acc_empty[2];
+  __shared__ uint32_t tmem_base;
+  __shared__ int abort_flag, s_bad;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int c = blockIdx.x, G = gridDim.x;
+  const int KB = a.KB;
+  const long long u0 = ((long long)c * a.U) / G, u1 = ((long long)(c + 1) * a.U) / G;
+
+  if (tid == 0) {
+    for (int s = 0; s < C::Stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+    abort_flag = 0;
+    s_bad = 0;
+    fence_barrier_init();
+  }
+  if (warp == 2) tmem_alloc(&tmem_base, C::TmemCols);
+  for (int i = tid; i < MP * 32; i += kLmUmmaThreads) { st_key[i] = -INFINITY; st_y[i] = 0.f; st_id[i] = 0x7fffffff; }
+  for (int i = tid; i < MP; i += kLmUmmaThreads) { st_ms[2 * i] = -INFINITY; st_ms[2 * i + 1] = 0.f; }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base;
+
+  if (warp == 0 && lane == 0) {
+    // ---- producer: weights do not depend on the previous kernel, activations do
+    const int n = (int)(u1 - u0);
+    const int pre = n < C::Stages ? n : C::Stages;
+    int tile = (int)(u0 / KB), kb = (int)(u0 % KB);
+    for (int it = 0; it < pre; ++it) {
+      mbar_expect_tx(&full[it], C::StageBytes);
+      tma_load_2d(ring + (size_t)it * C::StageBytes, &a.mapW, &full[it], kb * 64, tile * 128);
+      if (++kb == KB) { kb = 0; ++tile; }
+    }
+    pdl_wait();
+    tile = (int)(u0 / KB); kb = (int)(u0 % KB);
+    for (int it = 0; it < pre; ++it) {
+      uint8_t* xs = ring + (size_t)it * C::StageBytes + 128 * 64 * 2;
+      tma_load_2d(xs, &a.mapXhi, &full[it], kb * 64, 0);
+      tma_load_2d(xs + C::XBytes / 2, &a.mapXlo, &full[it], kb * 64, 0);
+      if (++kb == KB) { kb = 0; ++tile; }
+    }
+    int s = pre == C::Stages ? 0 : pre, ph = pre == C::Stages ? 1 : 0;
+    for (int it = pre; it < n; ++it) {
+      if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
+      uint8_t* st = ring + (size_t)s * C::StageBytes;
+      mbar_expect_tx(&full[s], C::StageBytes);
+      tma_load_2d(st, &a.mapW, &full[s], kb * 64, tile * 128);
+      tma_load_2d(st + 128 * 64 * 2, &a.mapXhi, &full[s], kb * 64, 0);
+      tma_load_2d(st + 128 * 64 * 2 + C::XBytes / 2, &a.mapXlo, &full[s], kb * 64, 0);
+      if (++s == C::Stages) { s = 0; ++ph; }
+      if (++kb == KB) { kb = 0; ++tile; }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer
+    constexpr uint32_t idesc = idesc_bf16(128, C::N);
+    const int n = (int)(u1 - u0);
+    int visit = -1, buf = 0, tile = -1;
+    int t = (int)(u0 / KB), kb = (int)(u0 % KB), s = 0, ph = 0;
+    bool ok = true;
+    for (int it = 0; it < n && ok; ++it) {
+      bool first = false;
+      if (t != tile) {
+        if (tile >= 0) mma_commit(&acc_full[buf]);
+        tile = t;
+        first = true;
+        ++visit;
+        buf = visit & 1;
+        if (visit >= 2) {
+          if (!mbar_wait(&acc_empty[buf], ((visit >> 1) - 1) & 1, &abort_flag)) { ok = false; break; }
+          tc_fence_after();
+        }
+      }
+      if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t wa = smem_u32(ring + (size_t)s * C::StageBytes);
+      const uint64_t ad = desc_sw128(wa), bd = desc_sw128(wa + 128 * 64 * 2);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) mma_f16(tmem + buf * C::N, ad + 2 * k, bd + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+      mma_commit(&empty[s]);
+      if (++s == C::Stages) { s = 0; ++ph; }
+      if (++kb == KB) { kb = 0; ++t; }
+    }
+    if (ok && tile >= 0) mma_commit(&acc_full[buf]);
+  } else if (warp >= 4) {
+    // ---- read-out and fold: TMEM lane = vocabulary row of the tile.  The four warps agree on every exit
+    // through s_bad before a barrier of their own (id 1), so a wait that ran out cannot strand the others.
+    const int wq = warp & 3, row = wq * 32 + lane, et = tid - 128;
+    pdl_wait();
+    // the final RMSNorm's per-token 1/rms comes from the previous kernel's sums of squares
+    for (int i = et; i < MP; i += 128) {
+      float ssq = 0.f;
+      if (i < p.M)
+        for (int tl = 0; tl < p.ss_tiles; ++tl) ssq += p.ss_in[(size_t)tl * p.ss_mp + i];
+      s_rstd[i] = i < p.M ? 1.f / sqrtf(ssq / (float)p.Kd + p.rms_eps) : 0.f;
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    int visit = 0;
+    long long u = u0;
+    while (u < u1) {
+      const int tile = (int)(u / KB);
+      const int ka = (int)(u - (long long)tile * KB);
+      long long ue = (long long)(tile + 1) * KB;
+      if (ue > u1) ue = u1;
+      const bool owner = ka == 0, whole = owner && ue == (long long)(tile + 1) * KB;
+      const int buf = visit & 1;
+      if (!mbar_wait(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) s_bad = 1;
+      if (owner && !whole && et == 0) {
+        // the rest of this tile comes from the next CTAs, for which it was the first thing to do
+        for (int cc = c + 1; cc < G && ((long long)cc * a.U) / G < (long long)(tile + 1) * KB; ++cc) {
+          int it = 0;
+          while (*reinterpret_cast<volatile int*>(a.flags + cc) != a.tag && it < kSpinLimit) { __nanosleep(200); ++it; }
+          if (it >= kSpinLimit) { s_bad = 1; abort_flag = 1; }
+        }
+        __threadfence();
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (s_bad) break;
+      tc_fence_after();
+      const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + buf * C::N;
+      const int rows_here = min(128, p.V - tile * 128);
+#pragma unroll 1
+      for (int ch = 0; ch < MP / 8; ++ch) {
+        uint32_t hi[8], lo[8];
+        tmem_ld8(tbase + ch * 8, hi);
+        tmem_ld8(tbase + MP + ch * 8, lo);
+        tmem_ld_wait();
+        float y[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) y[j] = __uint_as_float(hi[j]) + __uint_as_float(lo[j]);
+        if (ch == MP / 8 - 1) {  // the accumulator buffer is free once its last columns are in registers
+          tc_fence_before();
+          mbar_arrive(&acc_empty[buf]);
+        }
+        if (!owner) {
+          float* dst = a.pieces + (((size_t)c * 128 + row) * MP + ch * 8);
+          reinterpret_cast<float4*>(dst)[0] = make_float4(y[0], y[1], y[2], y[3]);
+          reinterpret_cast<float4*>(dst)[1] = make_float4(y[4], y[5], y[6], y[7]);
+          continue;
+        }
+        if (!whole) {
+          for (int cc = c + 1; cc < G && ((long long)cc * a.U) / G < (long long)(tile + 1) * KB; ++cc) {
+            const float* src = a.pieces + (((size_t)cc * 128 + row) * MP + ch * 8);
+            const float4 q0 = __ldcg(reinterpret_cast<const float4*>(src)), q1 = __ldcg(reinterpret_cast<const float4*>(src) + 1);
+            y[0] += q0.x; y[1] += q0.y; y[2] += q0.z; y[3] += q0.w;
+            y[4] += q1.x; y[5] += q1.y; y[6] += q1.z; y[7] += q1.w;
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int tok = ch * 8 + j;
+          const float v = y[j] * s_rstd[tok];
+          stage[j * SROW + row] = v;
+          if (p.logits_out != nullptr && tok < p.M && row < rows_here) p.logits_out[(size_t)tok * p.V + tile * 128 + row] = v;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        for (int j = wq; j < 8; j += 4) {
+          const int tk = ch * 8 + j;
+          if (tk < p.M) fold_token(p, stage + j * SROW, rows_here, tile * 128, tk, lane, st_key, st_y, st_id, st_ms);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
+      if (!owner) {
+        // release the piece: every thread fences its part, then one thread raises this CTA's flag
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et == 0) *reinterpret_cast<volatile int*>(a.flags + c) = a.tag;
+      }
+      ++visit;
+      u = ue;
+    }
+  }
+  pdl_wait();
+  pdl_trigger();
+  __syncthreads();
+  if (warp == 2) { tc_fence_after(); tmem_dealloc(tmem, C::TmemCols); }
+  if (abort_flag || s_bad) {
+    if (tid == 0) {
+      atomicExch(a.status, DEV_TIMEOUT);
+      for (int i = 0; i < 100; ++i) __nanosleep(1000);
+    }
+    __syncthreads();
+  }
+  for (int i = tid; i < MP * 32; i += kLmUmmaThreads) {
+    const size_t o = (size_t)c * MP * 32 + i;
+    p.part_key[o] = st_key[i];
+    p.part_y[o] = st_y[i];
+    p.part_id[o] = st_id[i];
+  }
+  for (int i = tid; i < MP * 2; i += kLmUmmaThreads) p.part_stats[(size_t)c * MP * 2 + i] = st_ms[i];
+}
+
+template <int MP>
+static cudaError_t launch_lm_umma_t(const LmUmmaArgs& a, cudaStream_t st) {
+  using C = LmUmmaCfg<MP>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(lm_head_umma_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  return launch_pdl(lm_head_umma_kernel<MP>, dim3(a.p.grid), dim3(kLmUmmaThreads), C::SmemBytes, st, a);
+}
+
+cudaError_t launch_lm_head_umma(const LmParams& pin, const CUtensorMap& mapW, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
+                                float* pieces, int* flags, int tag, int* status, cudaStream_t st) {
+  LmUmmaArgs a;
+  memset(&a, 0, sizeof(a));
+  a.p = pin;
+  a.mapW = mapW; a.mapXhi = mapXhi; a.mapXlo = mapXlo;
+  a.KB = (pin.Kd + 63) / 64;
+  a.U = (long long)((pin.V + 127) / 128) * a.KB;
+  a.pieces = pieces; a.flags = flags; a.tag = tag; a.status = status;
+  const int MP = padded_tokens(pin.M);
+  if (MP == 8) return launch_lm_umma_t<8>(a, st);
+  if (MP == 32) return launch_lm_umma_t<32>(a, st);
+  return launch_lm_umma_t<128>(a, st);
 }
 
 template <int NT, int NW>
