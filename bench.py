@@ -256,10 +256,10 @@ def run_ours(args):
             "latency_us": {"p50": 1e3 * statistics.median(per_step), "min": 1e3 * min(per_step), "max": 1e3 * max(per_step)},
             "step_bytes": bytes_step, "step_gbs": step_gbs,
             "step_frac_of_hbm_peak": step_gbs / hbm_peak, "step_frac_of_8tbs": step_gbs / 8000.0,
-            "roofline": {"bound": "hbm", "kernel": "lm_head_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+            "roofline": {"bound": "hbm", "kernel": "lm_head_umma_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                          "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
                          "traffic": args.lm_traffic if args.lm_traffic is not None else lm_bytes * LM_READ_RATIO + LM_WRITE_BYTES,
-                         "traffic_source": "ncu capture of a vocab-32768 launch (profiles/lm_head_kernel_C3_vocab32768.txt), reads "
+                         "traffic_source": "ncu capture of a vocab-32768 launch (profiles/lm_head_umma_kernel_C3_vocab32768.txt), reads "
                                            "scaled by the bytes streamed, writes taken as measured",
                          "bytes_per_launch": lm_bytes, "us_per_launch": 1e3 * lm_avg_ms},
             "e2e": {"value": replicas.job_steps_per_second(world, args.steps, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -298,8 +298,8 @@ def cpu_baseline(w, wt, inp, rows):
 
 # DRAM traffic of one LM-head launch, from the committed ncu capture of the vocab-32768 case of the same
 # kernel: dram__bytes_read / algorithmic bytes, and dram__bytes_write (per-CTA results, independent of vocab).
-LM_READ_RATIO = 335.762e6 / 335.544e6
-LM_WRITE_BYTES = 3.7e6
+LM_READ_RATIO = 336.96e6 / 335.544e6
+LM_WRITE_BYTES = 3.5e6
 
 
 def main():

@@ -242,10 +242,11 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
     // ---- producer: weights do not depend on the previous kernel, activations do
     const int n = (int)(u1 - u0);
     const int pre = n < C::Stages ? n : C::Stages;
+    const uint64_t wpol = l2_policy_evict_first();
     int tile = (int)(u0 / KB), kb = (int)(u0 % KB);
     for (int it = 0; it < pre; ++it) {
       mbar_expect_tx(&full[it], C::StageBytes);
-      tma_load_2d(ring + (size_t)it * C::StageBytes, &a.mapW, &full[it], kb * 64, tile * 128);
+      tma_load_2d_hint(ring + (size_t)it * C::StageBytes, &a.mapW, &full[it], kb * 64, tile * 128, wpol);
       if (++kb == KB) { kb = 0; ++tile; }
     }
     pdl_wait();
@@ -261,7 +262,7 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
       if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
       uint8_t* st = ring + (size_t)s * C::StageBytes;
       mbar_expect_tx(&full[s], C::StageBytes);
-      tma_load_2d(st, &a.mapW, &full[s], kb * 64, tile * 128);
+      tma_load_2d_hint(st, &a.mapW, &full[s], kb * 64, tile * 128, wpol);
       tma_load_2d(st + 128 * 64 * 2, &a.mapXhi, &full[s], kb * 64, 0);
       tma_load_2d(st + 128 * 64 * 2 + C::XBytes / 2, &a.mapXlo, &full[s], kb * 64, 0);
       if (++s == C::Stages) { s = 0; ++ph; }

@@ -111,11 +111,12 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
     // ---- producer: weights do not depend on the previous kernel, activations do
     const int n = (int)(u1 - u0);
     const int pre = n < C::Stages ? n : C::Stages;
+    const uint64_t wpol = l2_policy_evict_first();
     UnitPos q;
     q.set(p.s, u0);
     for (int it = 0; it < pre; ++it, q.next(p.s)) {
       mbar_expect_tx(&full[it], C::StageBytes);
-      tma_load_2d(ring + (size_t)it * C::StageBytes, &a.mapW[q.seg], &full[it], q.kb * 64, q.row0);
+      tma_load_2d_hint(ring + (size_t)it * C::StageBytes, &a.mapW[q.seg], &full[it], q.kb * 64, q.row0, wpol);
     }
     pdl_wait();
     q.set(p.s, u0);
@@ -129,7 +130,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
       uint8_t* st = ring + (size_t)s * C::StageBytes;
       mbar_expect_tx(&full[s], C::StageBytes);
-      tma_load_2d(st, &a.mapW[q.seg], &full[s], q.kb * 64, q.row0);
+      tma_load_2d_hint(st, &a.mapW[q.seg], &full[s], q.kb * 64, q.row0, wpol);
       tma_load_2d(st + kWBytes, &a.mapXhi, &full[s], q.xoff + q.kb * 64, 0);
       if (a.has_lo) tma_load_2d(st + kWBytes + C::XBytes / 2, &a.mapXlo, &full[s], q.xoff + q.kb * 64, 0);
       if (++s == C::Stages) { s = 0; ++ph; }
