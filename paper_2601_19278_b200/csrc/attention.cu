@@ -243,33 +243,58 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const __grid_constant
   }
 }
 
-// One block per (token row, query head): merge the chunk partials, normalise, emit hi/lo.
+// One block per (token row, query head): merge the chunk partials, normalise, emit hi/lo.  The block is
+// four groups of d_h threads; the (max, sum) pairs of all chunks are fetched in one round of loads, the
+// groups then add up interleaved quarters of the chunks' outputs (independent loads, one more round) and
+// their four partial sums are added in a fixed order.
+constexpr int kMaxChunks = 192;   // chunks per sequence the combine can hold (host checks)
+
 __global__ void attn_combine_kernel(const AttnArgs a) {
   const AttnParams& p = a.p;
-  const int m = blockIdx.x, j = blockIdx.y, d = threadIdx.x, dh = p.dh;
-  pdl_wait();
+  __shared__ float s_m[kMaxChunks], s_w[kMaxChunks];
+  __shared__ float s_o[4][128];
+  __shared__ float s_L;
+  const int m = blockIdx.x, j = blockIdx.y, dh = p.dh, tid = threadIdx.x, g = tid / dh, d = tid - g * dh;
   const int b = m / p.K, r = m % p.K, G = p.Hq / p.Hkv, hk = j / G, rr = (j % G) * p.K + r;
   const int n_chunks = a.chunk_base[b + 1] - a.chunk_base[b];
+  const size_t slot0 = ((size_t)a.chunk_base[b] * p.Hkv + hk) * 64 + rr, slot_step = (size_t)p.Hkv * 64;
+  pdl_wait();
+  float l_c = 0.f;
+  if (tid < n_chunks) {
+    const float2 ml = *reinterpret_cast<const float2*>(p.ml_part + (slot0 + (size_t)tid * slot_step) * 2);
+    s_m[tid] = ml.x;
+    l_c = ml.y;
+  }
+  __syncthreads();
   float mx = -INFINITY;
-  for (int c = 0; c < n_chunks; ++c) {
-    const size_t slot = ((size_t)(a.chunk_base[b] + c) * p.Hkv + hk) * 64 + rr;
-    mx = fmaxf(mx, p.ml_part[slot * 2]);
+  for (int c = 0; c < n_chunks; ++c) mx = fmaxf(mx, s_m[c]);
+  if (tid < n_chunks) s_w[tid] = s_m[tid] == -INFINITY ? 0.f : exp2f(s_m[tid] - mx);
+  __syncthreads();
+  // L = sum of l_c * w_c in chunk order: the products go through s_m (its maxima are no longer needed)
+  if (tid < n_chunks) s_m[tid] = l_c * s_w[tid];
+  __syncthreads();
+  if (tid == 0) {
+    float L = 0.f;
+    for (int c = 0; c < n_chunks; ++c) L += s_m[c];
+    s_L = L;
   }
-  float L = 0.f, O = 0.f;
-  for (int c = 0; c < n_chunks; ++c) {
-    const size_t slot = ((size_t)(a.chunk_base[b] + c) * p.Hkv + hk) * 64 + rr;
-    const float mc = p.ml_part[slot * 2];
-    if (mc == -INFINITY) continue;
-    const float wgt = exp2f(mc - mx);
-    L += p.ml_part[slot * 2 + 1] * wgt;
-    O += p.o_part[slot * dh + d] * wgt;
+  float O = 0.f;
+  const float* op = p.o_part + slot0 * dh + d;
+#pragma unroll 4
+  for (int c = g; c < n_chunks; c += 4) {
+    const float w = s_w[c];
+    if (w != 0.f) O += op[(size_t)c * slot_step * dh] * w;
   }
-  const float v = O / L;
-  bf16 hi, lo;
-  split_bf16(v, hi, lo);
-  const size_t idx = (size_t)m * p.Hq * dh + (size_t)j * dh + d;
-  p.a_hi[idx] = hi;
-  p.a_lo[idx] = lo;
+  s_o[g][d] = O;
+  __syncthreads();
+  if (g == 0) {
+    const float v = (((s_o[0][d] + s_o[1][d]) + s_o[2][d]) + s_o[3][d]) / s_L;
+    bf16 hi, lo;
+    split_bf16(v, hi, lo);
+    const size_t idx = (size_t)m * p.Hq * dh + (size_t)j * dh + d;
+    p.a_hi[idx] = hi;
+    p.a_lo[idx] = lo;
+  }
 }
 
 cudaError_t attention_setup() {
@@ -287,6 +312,7 @@ cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, cuda
     if (n > max_chunks) max_chunks = n;
   }
   a.chunk_base[p.B] = base;
+  if (max_chunks > kMaxChunks) return cudaErrorInvalidValue;
   dim3 grid(max_chunks, p.Hkv, p.B);
   cudaError_t e;
   if (p.dh == 128)
@@ -295,7 +321,7 @@ cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, cuda
     e = launch_pdl(attn_splitkv_kernel<64>, grid, dim3(128), (size_t)6 * 64 * 64 * 2, st, a);
   if (e != cudaSuccess) return e;
   dim3 cgrid(p.B * p.K, p.Hq);
-  return launch_pdl(attn_combine_kernel, cgrid, dim3(p.dh), 0, st, a);
+  return launch_pdl(attn_combine_kernel, cgrid, dim3(4 * p.dh), 0, st, a);
 }
 
 }  // namespace dart
