@@ -114,8 +114,11 @@ __device__ __forceinline__ void tile_rows_sum2(float v0, float v1, float* sh, fl
 // residual, gain, sums of squares, RoPE entry) is requested up front, from addresses that depend on
 // nothing loaded here (the piece table is already in shared memory); then come the reductions through shared memory and the stores.
 // Needs blockDim.x == 512.  s_pos[tok] = P_b + r (EPI_QKV), s_rstd preset to the <mask> rows' 1/rms.
-static __device__ __noinline__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, float* s_rstd, const int* s_pos,
-                                            const GroupMeta* gm, FinSmem* fs) {
+// One instantiation per epilogue mode: the tail of a kernel executes this code cold, so each mode only
+// carries its own instructions.
+template <int MODE>
+static __device__ __noinline__ void finalize_group_t(const GemmArgs& p, int group, int MP, float* sh, float* s_rstd, const int* s_pos,
+                                              const GroupMeta* gm, FinSmem* fs) {
   const EpiArgs& e = p.epi;
   const int tid = threadIdx.x, M = p.s.M;
   const int Ta = group, Tb = group + p.pair_offset;
@@ -130,9 +133,9 @@ static __device__ __noinline__ void finalize_group(const GemmArgs& p, int group,
   const int K = e.K, F = e.F;
   const auto col_id = [](int tok) { return tok; };
   const auto col_fresh = [K, F](int tok) { const int b = tok / K, rr = tok % K; return rr < F ? b * F + rr : -1; };
-  const bool rowmode = e.mode == EPI_FC || e.mode == EPI_RES;
+  const bool rowmode = MODE == EPI_FC || MODE == EPI_RES;
   const int dh = e.dh, half = dh >> 1;
-  const int pairs = e.mode == EPI_QKV ? (rows_valid / dh) * half : 1;   // (head, i) pairs of this tile
+  const int pairs = MODE == EPI_QKV ? (rows_valid / dh) * half : 1;   // (head, i) pairs of this tile
 
   for (int tok0 = 0; tok0 < M; tok0 += 8) {
     const int t0 = tok0 + par, t1 = tok0 + par + 4;  // this thread's tokens in the row-major modes
@@ -145,7 +148,7 @@ static __device__ __noinline__ void finalize_group(const GemmArgs& p, int group,
     unsigned short gam_raw = 0;
     if (rowmode && row < rows_valid) gam_raw = reinterpret_cast<const unsigned short*>(e.gamma)[n];
     float r0 = 0.f, r1 = 0.f;
-    if (e.mode == EPI_RES) {
+    if (MODE == EPI_RES) {
       // residual: the stream so far, or (first projection) g of a fresh row / the <mask> representation
       const float* s0 = e.res_in != nullptr ? e.res_in + (size_t)t0 * e.h
                                             : ((t0 % K) < F ? e.res0 + (size_t)((t0 / K) * F + t0 % K) * e.h : e.mask_res);
@@ -155,17 +158,17 @@ static __device__ __noinline__ void finalize_group(const GemmArgs& p, int group,
       if (ok1) r1 = __ldcg(s1 + n);
     }
     float2 cs = make_float2(1.f, 0.f);
-    if (e.mode == EPI_QKV && s < 2 && tid < pairs * 8 && ptok < M)
+    if (MODE == EPI_QKV && s < 2 && tid < pairs * 8 && ptok < M)
       cs = e.rope_tab[(size_t)s_pos[ptok] * half + (pi % half)];  // (cos, sin) of pos * theta^(-2i/d_h)
     float rs = 0.f;
     if (tok0 == 0) {
-      if (e.mode == EPI_GATE_UP) rs = rstd_issue(e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_id);
-      if (e.mode == EPI_QKV) rs = rstd_issue(e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_fresh);
+      if (MODE == EPI_GATE_UP) rs = rstd_issue(e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_id);
+      if (MODE == EPI_QKV) rs = rstd_issue(e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_fresh);
     }
     // ---- reductions through shared memory
     if (tok0 == 0) {
-      if (e.mode == EPI_GATE_UP) rstd_finish(rs, M, MP, e.h, e.eps, fs, s_rstd, col_id);
-      if (e.mode == EPI_QKV) rstd_finish(rs, M, MP, e.h, e.eps, fs, s_rstd, col_fresh);
+      if (MODE == EPI_GATE_UP) rstd_finish(rs, M, MP, e.h, e.eps, fs, s_rstd, col_id);
+      if (MODE == EPI_QKV) rstd_finish(rs, M, MP, e.h, e.eps, fs, s_rstd, col_fresh);
     }
     if (paired) g2.finish(p, gm, tok0, MP, fs); else g1.finish(p, gm, tok0, MP, fs);
     __syncthreads();
@@ -178,9 +181,9 @@ static __device__ __noinline__ void finalize_group(const GemmArgs& p, int group,
       const float x0 = ok0 ? r0 + fs->xs[0][row][par] : 0.f, x1 = ok1 ? r1 + fs->xs[0][row][par + 4] : 0.f;
       float q0, q1;
       tile_rows_sum2(x0 * x0, x1 * x1, sh, q0, q1);
-      float* res = e.mode == EPI_FC ? e.res0 : e.res_out;
+      float* res = MODE == EPI_FC ? e.res0 : e.res_out;
       // the FC's token index counts fresh rows only; its z row is the step's row (b, r)
-      const int o0 = e.mode == EPI_FC ? (t0 / F) * K + t0 % F : t0, o1 = e.mode == EPI_FC ? (t1 / F) * K + t1 % F : t1;
+      const int o0 = MODE == EPI_FC ? (t0 / F) * K + t0 % F : t0, o1 = MODE == EPI_FC ? (t1 / F) * K + t1 % F : t1;
       bf16 hi, lo;
       if (ok0) {
         if (res != nullptr) res[(size_t)t0 * e.h + n] = x0;
@@ -196,7 +199,7 @@ static __device__ __noinline__ void finalize_group(const GemmArgs& p, int group,
       }
       if (row == 0 && t0 < M) e.ss_out[(size_t)Ta * MP + t0] = q0;
       if (row == 0 && t1 < M) e.ss_out[(size_t)Ta * MP + t1] = q1;
-    } else if (e.mode == EPI_GATE_UP) {
+    } else if (MODE == EPI_GATE_UP) {
       // u = SiLU(rstd * gate) * (rstd * up): the previous RMSNorm's 1/rms is applied here
 #pragma unroll
       for (int k = 0; k < 2; ++k) {
@@ -209,7 +212,7 @@ static __device__ __noinline__ void finalize_group(const GemmArgs& p, int group,
           e.out_lo[(size_t)tok * e.ld_out + n] = lo;
         }
       }
-    } else if (e.mode == EPI_QKV) {
+    } else if (MODE == EPI_QKV) {
       // y = rstd_g * (W[:, :h] z_g) + W[:, h:] z_e ; RoPE on q, k at position P_b + r ; q and the new rows'
       // k, v as hi/lo pairs ; the fresh rows' k, v appended to the cache.  segment 0,1,2 = q,k,v (g half);
       // the e half is the paired tile.
@@ -247,6 +250,16 @@ static __device__ __noinline__ void finalize_group(const GemmArgs& p, int group,
       }
     }
     __syncthreads();
+  }
+}
+
+static __device__ __forceinline__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, float* s_rstd, const int* s_pos,
+                                                      const GroupMeta* gm, FinSmem* fs) {
+  switch (p.epi.mode) {
+    case EPI_FC: finalize_group_t<EPI_FC>(p, group, MP, sh, s_rstd, s_pos, gm, fs); break;
+    case EPI_QKV: finalize_group_t<EPI_QKV>(p, group, MP, sh, s_rstd, s_pos, gm, fs); break;
+    case EPI_RES: finalize_group_t<EPI_RES>(p, group, MP, sh, s_rstd, s_pos, gm, fs); break;
+    default: finalize_group_t<EPI_GATE_UP>(p, group, MP, sh, s_rstd, s_pos, gm, fs); break;
   }
 }
 
