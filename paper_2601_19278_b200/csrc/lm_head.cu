@@ -44,39 +44,39 @@ __device__ __forceinline__ void fold_token(const LmParams& p, const float* srow,
   float lk = st_key[tk * 32 + lane], ly = st_y[tk * 32 + lane];
   int lid = st_id[tk * 32 + lane];
   float m_run = st_ms[2 * tk], s_run = st_ms[2 * tk + 1];
+  // lane owns the four consecutive vocabulary rows 4*lane .. 4*lane+3 of the 128: one Philox call covers them
   float yv[4], kv[4];
   float tmax = -INFINITY;
+  uint4 rnd = make_uint4(0, 0, 0, 0);
+  if (p.gumbel && 4 * lane < nrows)
+    rnd = philox4x32_10(make_uint4((uint32_t)(id0 >> 2) + lane, (uint32_t)(tk % p.K), (uint32_t)(tk / p.K), p.step), p.seed_lo, p.seed_hi);
+  const uint32_t rw[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    const int idx = lane + 32 * q;
+    const int idx = 4 * lane + q;
     const bool ok = idx < nrows;
     yv[q] = ok ? srow[idx] * p.inv_temp : -INFINITY;
     kv[q] = yv[q];
-    if (p.gumbel && ok) {
-      const uint32_t v = (uint32_t)(id0 + idx);
-      const uint4 rnd = philox4x32_10(make_uint4(v >> 2, (uint32_t)(tk % p.K), (uint32_t)(tk / p.K), p.step), p.seed_lo, p.seed_hi);
-      const uint32_t wsel = (v & 3) == 0 ? rnd.x : ((v & 3) == 1 ? rnd.y : ((v & 3) == 2 ? rnd.z : rnd.w));
-      kv[q] = yv[q] + gumbel_from_bits(wsel);
-    }
+    if (p.gumbel && ok) kv[q] = yv[q] + gumbel_from_bits(rw[q]);
     tmax = fmaxf(tmax, yv[q]);
   }
   tmax = warp_max(tmax);
   const float m_new = fmaxf(m_run, tmax);
   float part = 0.f;
 #pragma unroll
-  for (int q = 0; q < 4; ++q) part += (lane + 32 * q < nrows) ? expf(yv[q] - m_new) : 0.f;
+  for (int q = 0; q < 4; ++q) part += (4 * lane + q < nrows) ? expf(yv[q] - m_new) : 0.f;
   part = warp_sum(part);
   s_run = s_run * expf(m_run - m_new) + part;
   m_run = m_new;
   float thr = __shfl_sync(0xffffffffu, lk, p.topk - 1);
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    const bool ok = lane + 32 * q < nrows;
+    const bool ok = 4 * lane + q < nrows;
     unsigned mask = __ballot_sync(0xffffffffu, ok && kv[q] > thr);
     while (mask) {
       const int src = __ffs(mask) - 1;
       const float nk = __shfl_sync(0xffffffffu, kv[q], src), ny = __shfl_sync(0xffffffffu, yv[q], src);
-      list_insert(lk, ly, lid, nk, ny, id0 + src + 32 * q, lane);
+      list_insert(lk, ly, lid, nk, ny, id0 + 4 * src + q, lane);
       thr = __shfl_sync(0xffffffffu, lk, p.topk - 1);
       mask &= mask - 1;
       mask &= __ballot_sync(0xffffffffu, ok && kv[q] > thr);
