@@ -36,11 +36,20 @@ __device__ __forceinline__ void meta_prefetch(const GemmArgs& p, int group, Grou
   asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
-// Partial sum of squares of token row tid / TPT over the tiles q, q + TPT, ... (TPT = blockDim / MP threads
+// The finalize runs on a team of NTHR threads that synchronises on barrier BAR (0 = __syncthreads, NTHR = the
+// whole CTA: what both kernel families use; a 256-thread team of otherwise idle warps was measured slower).
+// ft is the thread's index in the team.
+template <int NTHR, int BAR>
+__device__ __forceinline__ void team_sync() {
+  if (BAR == 0) __syncthreads();
+  else asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(NTHR) : "memory");
+}
+
+// Partial sum of squares of token row ft / TPT over the tiles q, q + TPT, ... (TPT = NTHR / MP threads
 // per token); col(tok) maps a token to its column of ss[tile][mp], or -1.
-template <class ColFn>
-__device__ __forceinline__ float rstd_issue(const float* ss, int ntile, int mp, int M, int MP, ColFn col) {
-  const int TPT = blockDim.x / MP, tok = threadIdx.x / TPT, q = threadIdx.x % TPT;
+template <int NTHR, class ColFn>
+__device__ __forceinline__ float rstd_issue(int ft, const float* ss, int ntile, int mp, int M, int MP, ColFn col) {
+  const int TPT = NTHR / MP, tok = ft / TPT, q = ft % TPT;
   const int cidx = tok < M ? col(tok) : -1;
   float s = 0.f;
   if (cidx >= 0) {
@@ -50,31 +59,31 @@ __device__ __forceinline__ float rstd_issue(const float* ss, int ntile, int mp, 
   return s;
 }
 // Fixed-order reduction of those partials to s_rstd[tok] = 1/rms.  Two barriers.
-template <class ColFn>
-__device__ __forceinline__ void rstd_finish(float s, int M, int MP, int h, float eps, FinSmem* fs, float* s_rstd, ColFn col) {
-  const int TPT = blockDim.x / MP, width = TPT < 32 ? TPT : 32, nsub = TPT < 32 ? 1 : TPT / 32;
+template <int NTHR, int BAR, class ColFn>
+__device__ __forceinline__ void rstd_finish(int ft, float s, int M, int MP, int h, float eps, FinSmem* fs, float* s_rstd, ColFn col) {
+  const int TPT = NTHR / MP, width = TPT < 32 ? TPT : 32, nsub = TPT < 32 ? 1 : TPT / 32;
   for (int o = width >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  if ((threadIdx.x % width) == 0) fs->rpart[threadIdx.x / width] = s;
-  __syncthreads();
-  if (threadIdx.x < M && col(threadIdx.x) >= 0) {
+  if ((ft % width) == 0) fs->rpart[ft / width] = s;
+  team_sync<NTHR, BAR>();
+  if (ft < M && col(ft) >= 0) {
     float t = 0.f;
-    for (int k = 0; k < nsub; ++k) t += fs->rpart[threadIdx.x * nsub + k];
-    s_rstd[threadIdx.x] = 1.f / sqrtf(t / (float)h + eps);
+    for (int k = 0; k < nsub; ++k) t += fs->rpart[ft * nsub + k];
+    s_rstd[ft] = 1.f / sqrtf(t / (float)h + eps);
   }
-  __syncthreads();
+  team_sync<NTHR, BAR>();
 }
 
 // Piece sums of the group's tile(s) for the 8 tokens tok0 .. tok0+7, pieces in CTA order.  The thread ->
 // element mapping follows the pieces' memory layout (coalesced), and the first four pieces of every
 // element are requested before any is used.
-template <int NTILE>
+template <int NTILE, int NTHR>
 struct Gather {
-  static constexpr int Q = NTILE * 2;   // elements per thread (512 threads, 1024 elements per tile)
+  static constexpr int Q = NTILE * 1024 / NTHR;   // elements per thread (1024 elements per tile)
   float v[Q][4];
-  __device__ __forceinline__ void issue(const GemmArgs& p, const GroupMeta* gm, int tok0, int MP) {
+  __device__ __forceinline__ void issue(int ft, const GemmArgs& p, const GroupMeta* gm, int tok0, int MP) {
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
-      const int e = threadIdx.x + 512 * q, row = (e >> 3) & 127;
+      const int e = ft + NTHR * q, row = (e >> 3) & 127;
       const int* m = gm->row[(e >> 10) * 8 + (row >> 4)];
       const float* src = p.part + (size_t)(row & 15) * MP + tok0 + (e & 7);
       const int n = m[0];
@@ -82,10 +91,10 @@ struct Gather {
       for (int u = 0; u < 4; ++u) v[q][u] = u < n ? __ldcg(src + (size_t)m[1 + u] * 16 * MP) : 0.f;
     }
   }
-  __device__ __forceinline__ void finish(const GemmArgs& p, const GroupMeta* gm, int tok0, int MP, FinSmem* fs) {
+  __device__ __forceinline__ void finish(int ft, const GemmArgs& p, const GroupMeta* gm, int tok0, int MP, FinSmem* fs) {
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
-      const int e = threadIdx.x + 512 * q, row = (e >> 3) & 127;
+      const int e = ft + NTHR * q, row = (e >> 3) & 127;
       const int* m = gm->row[(e >> 10) * 8 + (row >> 4)];
       float acc = (((0.f + v[q][0]) + v[q][1]) + v[q][2]) + v[q][3];
       for (int u = 4; u < m[0]; ++u)  // rare: long reductions cut into many short ranges
@@ -95,32 +104,42 @@ struct Gather {
   }
 };
 
-// Sums v0 and v1 over the 128 rows of a tile (thread -> row = tid & 127, token class = tid >> 7);
-// results valid in every thread; fixed order.  sh: two floats per warp.
-__device__ __forceinline__ void tile_rows_sum2(float v0, float v1, float* sh, float& r0, float& r1) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  v0 = warp_sum(v0);
-  v1 = warp_sum(v1);
-  __syncthreads();
-  if (lane == 0) { sh[warp] = v0; sh[16 + warp] = v1; }
-  __syncthreads();
+// Sums v[0..NV) over the 128 rows of a tile (thread -> row = ft & 127, token class = ft >> 7); results valid
+// in every thread; fixed order.  sh: NV floats per warp of the team (32 floats in all).
+template <int NTHR, int BAR, int NV>
+__device__ __forceinline__ void tile_rows_sum(int ft, float (&v)[NV], float* sh) {
+  constexpr int NWARP = NTHR / 32;
+  const int lane = ft & 31, warp = ft >> 5;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) v[k] = warp_sum(v[k]);
+  team_sync<NTHR, BAR>();
+  if (lane == 0) {
+#pragma unroll
+    for (int k = 0; k < NV; ++k) sh[k * NWARP + warp] = v[k];
+  }
+  team_sync<NTHR, BAR>();
   const int c4 = (warp >> 2) * 4;  // warps c4 .. c4+3 hold the 128 rows of this token class
-  r0 = sh[c4] + sh[c4 + 1] + sh[c4 + 2] + sh[c4 + 3];
-  r1 = sh[16 + c4] + sh[16 + c4 + 1] + sh[16 + c4 + 2] + sh[16 + c4 + 3];
+#pragma unroll
+  for (int k = 0; k < NV; ++k) v[k] = sh[k * NWARP + c4] + sh[k * NWARP + c4 + 1] + sh[k * NWARP + c4 + 2] + sh[k * NWARP + c4 + 3];
 }
 
 // The fused epilogue of one completed group (one 128-row tile, or a pair of tiles).  It sits on the
 // kernel's tail, so it is built around a single round trip to memory: every load it needs (pieces,
 // residual, gain, sums of squares, RoPE entry) is requested up front, from addresses that depend on
-// nothing loaded here (the piece table is already in shared memory); then come the reductions through shared memory and the stores.
-// Needs blockDim.x == 512.  s_pos[tok] = P_b + r (EPI_QKV), s_rstd preset to the <mask> rows' 1/rms.
-// One instantiation per epilogue mode: the tail of a kernel executes this code cold, so each mode only
-// carries its own instructions.
-template <int MODE>
-static __device__ __noinline__ void finalize_group_t(const GemmArgs& p, int group, int MP, float* sh, float* s_rstd, const int* s_pos,
-                                              const GroupMeta* gm, FinSmem* fs) {
+// nothing loaded here (the piece table is already in shared memory); then come the reductions through
+// shared memory and the stores.  s_pos[tok] = P_b + r (EPI_QKV), s_rstd preset to the <mask> rows' 1/rms.
+// dry = true executes the same instructions without a single store to global memory (a measurement aid: a
+// second call on the same group takes 3 us instead of 5.5, because the pieces, written by SMs all over the
+// chip, are then close by - not because of the code: a dry pass ahead of time does not help).
+// One instantiation per epilogue mode, so each mode only carries its own instructions.
+template <int MODE, int NTHR, int BAR>
+static __device__ __noinline__ void finalize_group_t(int ft, const GemmArgs& p, int group, int MP, float* sh, float* s_rstd,
+                                                     const int* s_pos, const GroupMeta* gm, FinSmem* fs, bool dry) {
+  constexpr int NPAR = NTHR / 128;     // token classes: thread -> (row = ft & 127, class = ft >> 7)
+  constexpr int NV = 8 / NPAR;         // tokens of an 8-token chunk per thread in the row-major modes
+  constexpr int NP = 512 / NTHR;       // (token, pair) items per thread in EPI_QKV
   const EpiArgs& e = p.epi;
-  const int tid = threadIdx.x, M = p.s.M;
+  const int M = p.s.M;
   const int Ta = group, Tb = group + p.pair_offset;
   const bool paired = p.pair_offset > 0;
   int s = 0;  // segment of tile Ta
@@ -128,83 +147,89 @@ static __device__ __noinline__ void finalize_group_t(const GemmArgs& p, int grou
     if (i < p.s.nseg && Ta >= p.s.seg[i].tile0) s = i;
   const int row_base = (Ta - p.s.seg[s].tile0) * 128;       // first row of the tile inside its matrix
   const int rows_valid = min(128, p.s.seg[s].rows - row_base);
-  const int row = tid & 127, par = tid >> 7;               // thread -> (row, token class 0..3)
+  const int row = ft & 127, par = ft >> 7;
   const int n = row_base + row;
   const int K = e.K, F = e.F;
   const auto col_id = [](int tok) { return tok; };
   const auto col_fresh = [K, F](int tok) { const int b = tok / K, rr = tok % K; return rr < F ? b * F + rr : -1; };
-  const bool rowmode = MODE == EPI_FC || MODE == EPI_RES;
+  constexpr bool rowmode = MODE == EPI_FC || MODE == EPI_RES;
   const int dh = e.dh, half = dh >> 1;
   const int pairs = MODE == EPI_QKV ? (rows_valid / dh) * half : 1;   // (head, i) pairs of this tile
 
   for (int tok0 = 0; tok0 < M; tok0 += 8) {
-    const int t0 = tok0 + par, t1 = tok0 + par + 4;  // this thread's tokens in the row-major modes
-    const bool ok0 = row < rows_valid && t0 < M, ok1 = row < rows_valid && t1 < M;
-    const int ptok = tok0 + tid / pairs, pi = tid % pairs;    // this thread's (token, pair) in EPI_QKV
     // ---- every load, before any use
-    Gather<2> g2;
-    Gather<1> g1;
-    if (paired) g2.issue(p, gm, tok0, MP); else g1.issue(p, gm, tok0, MP);
+    Gather<2, NTHR> g2;
+    Gather<1, NTHR> g1;
+    if (paired) g2.issue(ft, p, gm, tok0, MP); else g1.issue(ft, p, gm, tok0, MP);
     unsigned short gam_raw = 0;
     if (rowmode && row < rows_valid) gam_raw = reinterpret_cast<const unsigned short*>(e.gamma)[n];
-    float r0 = 0.f, r1 = 0.f;
-    if (MODE == EPI_RES) {
-      // residual: the stream so far, or (first projection) g of a fresh row / the <mask> representation
-      const float* s0 = e.res_in != nullptr ? e.res_in + (size_t)t0 * e.h
-                                            : ((t0 % K) < F ? e.res0 + (size_t)((t0 / K) * F + t0 % K) * e.h : e.mask_res);
-      const float* s1 = e.res_in != nullptr ? e.res_in + (size_t)t1 * e.h
-                                            : ((t1 % K) < F ? e.res0 + (size_t)((t1 / K) * F + t1 % K) * e.h : e.mask_res);
-      if (ok0) r0 = __ldcg(s0 + n);
-      if (ok1) r1 = __ldcg(s1 + n);
+    float res[NV];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+      res[k] = 0.f;
+      const int t = tok0 + par + NPAR * k;
+      if (MODE == EPI_RES && row < rows_valid && t < M) {
+        // residual: the stream so far, or (first projection) g of a fresh row / the <mask> representation
+        const float* src = e.res_in != nullptr ? e.res_in + (size_t)t * e.h
+                                               : ((t % K) < F ? e.res0 + (size_t)((t / K) * F + t % K) * e.h : e.mask_res);
+        res[k] = __ldcg(src + n);
+      }
     }
-    float2 cs = make_float2(1.f, 0.f);
-    if (MODE == EPI_QKV && s < 2 && tid < pairs * 8 && ptok < M)
-      cs = e.rope_tab[(size_t)s_pos[ptok] * half + (pi % half)];  // (cos, sin) of pos * theta^(-2i/d_h)
+    float2 cs[NP];
+#pragma unroll
+    for (int k = 0; k < NP; ++k) {
+      cs[k] = make_float2(1.f, 0.f);
+      const int idx = ft + NTHR * k, ptok = tok0 + idx / pairs, pi = idx % pairs;
+      if (MODE == EPI_QKV && s < 2 && idx < pairs * 8 && ptok < M)
+        cs[k] = e.rope_tab[(size_t)s_pos[ptok] * half + (pi % half)];  // (cos, sin) of pos * theta^(-2i/d_h)
+    }
     float rs = 0.f;
     if (tok0 == 0) {
-      if (MODE == EPI_GATE_UP) rs = rstd_issue(e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_id);
-      if (MODE == EPI_QKV) rs = rstd_issue(e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_fresh);
+      if (MODE == EPI_GATE_UP) rs = rstd_issue<NTHR>(ft, e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_id);
+      if (MODE == EPI_QKV) rs = rstd_issue<NTHR>(ft, e.ss_in, e.ss_tiles, e.ss_mp, M, MP, col_fresh);
     }
     // ---- reductions through shared memory
     if (tok0 == 0) {
-      if (MODE == EPI_GATE_UP) rstd_finish(rs, M, MP, e.h, e.eps, fs, s_rstd, col_id);
-      if (MODE == EPI_QKV) rstd_finish(rs, M, MP, e.h, e.eps, fs, s_rstd, col_fresh);
+      if (MODE == EPI_GATE_UP) rstd_finish<NTHR, BAR>(ft, rs, M, MP, e.h, e.eps, fs, s_rstd, col_id);
+      if (MODE == EPI_QKV) rstd_finish<NTHR, BAR>(ft, rs, M, MP, e.h, e.eps, fs, s_rstd, col_fresh);
     }
-    if (paired) g2.finish(p, gm, tok0, MP, fs); else g1.finish(p, gm, tok0, MP, fs);
-    __syncthreads();
+    if (paired) g2.finish(ft, p, gm, tok0, MP, fs); else g1.finish(ft, p, gm, tok0, MP, fs);
+    team_sync<NTHR, BAR>();
 
     // ---- the mode's arithmetic and stores
     if (rowmode) {
       // FC: g = FC(features) on the fresh rows.  RES: x = residual + projection.  Both: residual stream,
       // gain-scaled hi/lo for the next projection, the tile's sum of squares for the next 1/rms.
       const float gam = __bfloat162float(__ushort_as_bfloat16(gam_raw));
-      const float x0 = ok0 ? r0 + fs->xs[0][row][par] : 0.f, x1 = ok1 ? r1 + fs->xs[0][row][par + 4] : 0.f;
-      float q0, q1;
-      tile_rows_sum2(x0 * x0, x1 * x1, sh, q0, q1);
-      float* res = MODE == EPI_FC ? e.res0 : e.res_out;
-      // the FC's token index counts fresh rows only; its z row is the step's row (b, r)
-      const int o0 = MODE == EPI_FC ? (t0 / F) * K + t0 % F : t0, o1 = MODE == EPI_FC ? (t1 / F) * K + t1 % F : t1;
-      bf16 hi, lo;
-      if (ok0) {
-        if (res != nullptr) res[(size_t)t0 * e.h + n] = x0;
-        split_bf16(x0 * gam, hi, lo);
-        e.out_hi[(size_t)o0 * e.ld_out + n] = hi;
-        e.out_lo[(size_t)o0 * e.ld_out + n] = lo;
+      float x[NV], q[NV];
+#pragma unroll
+      for (int k = 0; k < NV; ++k) {
+        const int t = tok0 + par + NPAR * k;
+        x[k] = (row < rows_valid && t < M) ? res[k] + fs->xs[0][row][par + NPAR * k] : 0.f;
+        q[k] = x[k] * x[k];
       }
-      if (ok1) {
-        if (res != nullptr) res[(size_t)t1 * e.h + n] = x1;
-        split_bf16(x1 * gam, hi, lo);
-        e.out_hi[(size_t)o1 * e.ld_out + n] = hi;
-        e.out_lo[(size_t)o1 * e.ld_out + n] = lo;
+      tile_rows_sum<NTHR, BAR, NV>(ft, q, sh);
+      float* resw = MODE == EPI_FC ? e.res0 : e.res_out;
+#pragma unroll
+      for (int k = 0; k < NV; ++k) {
+        const int t = tok0 + par + NPAR * k;
+        // the FC's token index counts fresh rows only; its z row is the step's row (b, r)
+        const int o = MODE == EPI_FC ? (t / F) * K + t % F : t;
+        if (row < rows_valid && t < M && !dry) {
+          if (resw != nullptr) resw[(size_t)t * e.h + n] = x[k];
+          bf16 hi, lo;
+          split_bf16(x[k] * gam, hi, lo);
+          e.out_hi[(size_t)o * e.ld_out + n] = hi;
+          e.out_lo[(size_t)o * e.ld_out + n] = lo;
+        }
+        if (row == 0 && t < M && !dry) e.ss_out[(size_t)Ta * MP + t] = q[k];
       }
-      if (row == 0 && t0 < M) e.ss_out[(size_t)Ta * MP + t0] = q0;
-      if (row == 0 && t1 < M) e.ss_out[(size_t)Ta * MP + t1] = q1;
     } else if (MODE == EPI_GATE_UP) {
       // u = SiLU(rstd * gate) * (rstd * up): the previous RMSNorm's 1/rms is applied here
 #pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        const int tl = par + 4 * k, tok = tok0 + tl;
-        if (row < rows_valid && tok < M) {
+      for (int k = 0; k < NV; ++k) {
+        const int tl = par + NPAR * k, tok = tok0 + tl;
+        if (row < rows_valid && tok < M && !dry) {
           const float gt = s_rstd[tok] * fs->xs[0][row][tl], up = s_rstd[tok] * fs->xs[1][row][tl];
           bf16 hi, lo;
           split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
@@ -217,49 +242,54 @@ static __device__ __noinline__ void finalize_group_t(const GemmArgs& p, int grou
       // k, v as hi/lo pairs ; the fresh rows' k, v appended to the cache.  segment 0,1,2 = q,k,v (g half);
       // the e half is the paired tile.
       const int kind = s;
-      if (tid < pairs * 8 && ptok < M) {
-        const int tl = ptok - tok0, tok = ptok;
-        const int hl = pi / half, i = pi - hl * half;
-        const int ra = hl * dh + i, rb = ra + half;
-        const float x1 = s_rstd[tok] * fs->xs[0][ra][tl] + fs->xs[1][ra][tl];
-        const float x2 = s_rstd[tok] * fs->xs[0][rb][tl] + fs->xs[1][rb][tl];
-        const int b = tok / K, r = tok % K;
-        float o1 = x1, o2 = x2;
-        if (kind < 2) {
-          o1 = x1 * cs.x - x2 * cs.y;
-          o2 = x2 * cs.x + x1 * cs.y;
-        }
-        bf16 h1, l1, h2, l2;
-        split_bf16(o1, h1, l1);
-        split_bf16(o2, h2, l2);
-        const int head = (row_base / dh) + hl;
-        if (kind == 0) {
-          const size_t o = (((size_t)b * e.Hq + head) * K + r) * dh;
-          e.q_hi[o + i] = h1; e.q_hi[o + i + half] = h2;
-          e.q_lo[o + i] = l1; e.q_lo[o + i + half] = l2;
-        } else {
-          bf16* side = (kind == 1 ? e.k_new : e.v_new) + ((size_t)b * e.Hkv + head) * 16 * dh;
-          side[(size_t)r * dh + i] = h1; side[(size_t)r * dh + i + half] = h2;
-          side[(size_t)(8 + r) * dh + i] = l1; side[(size_t)(8 + r) * dh + i + half] = l2;
-          if (r < F) {
-            bf16* dst = (kind == 1 ? e.k_cache : e.v_cache) + (((size_t)b * e.Hkv + head) * e.P_cap + s_pos[tok]) * dh;
-            dst[i] = h1;
-            dst[i + half] = h2;
+#pragma unroll
+      for (int k = 0; k < NP; ++k) {
+        const int idx = ft + NTHR * k, ptok = tok0 + idx / pairs, pi = idx % pairs;
+        if (idx < pairs * 8 && ptok < M && !dry) {
+          const int tl = ptok - tok0, tok = ptok;
+          const int hl = pi / half, i = pi - hl * half;
+          const int ra = hl * dh + i, rb = ra + half;
+          const float x1 = s_rstd[tok] * fs->xs[0][ra][tl] + fs->xs[1][ra][tl];
+          const float x2 = s_rstd[tok] * fs->xs[0][rb][tl] + fs->xs[1][rb][tl];
+          const int b = tok / K, r = tok % K;
+          float o1 = x1, o2 = x2;
+          if (kind < 2) {
+            o1 = x1 * cs[k].x - x2 * cs[k].y;
+            o2 = x2 * cs[k].x + x1 * cs[k].y;
+          }
+          bf16 h1, l1, h2, l2;
+          split_bf16(o1, h1, l1);
+          split_bf16(o2, h2, l2);
+          const int head = (row_base / dh) + hl;
+          if (kind == 0) {
+            const size_t o = (((size_t)b * e.Hq + head) * K + r) * dh;
+            e.q_hi[o + i] = h1; e.q_hi[o + i + half] = h2;
+            e.q_lo[o + i] = l1; e.q_lo[o + i + half] = l2;
+          } else {
+            bf16* side = (kind == 1 ? e.k_new : e.v_new) + ((size_t)b * e.Hkv + head) * 16 * dh;
+            side[(size_t)r * dh + i] = h1; side[(size_t)r * dh + i + half] = h2;
+            side[(size_t)(8 + r) * dh + i] = l1; side[(size_t)(8 + r) * dh + i + half] = l2;
+            if (r < F) {
+              bf16* dst = (kind == 1 ? e.k_cache : e.v_cache) + (((size_t)b * e.Hkv + head) * e.P_cap + s_pos[tok]) * dh;
+              dst[i] = h1;
+              dst[i + half] = h2;
+            }
           }
         }
       }
     }
-    __syncthreads();
+    team_sync<NTHR, BAR>();
   }
 }
 
-static __device__ __forceinline__ void finalize_group(const GemmArgs& p, int group, int MP, float* sh, float* s_rstd, const int* s_pos,
-                                                      const GroupMeta* gm, FinSmem* fs) {
+template <int NTHR, int BAR>
+static __device__ __forceinline__ void finalize_group(int ft, const GemmArgs& p, int group, int MP, float* sh, float* s_rstd,
+                                                      const int* s_pos, const GroupMeta* gm, FinSmem* fs, bool dry = false) {
   switch (p.epi.mode) {
-    case EPI_FC: finalize_group_t<EPI_FC>(p, group, MP, sh, s_rstd, s_pos, gm, fs); break;
-    case EPI_QKV: finalize_group_t<EPI_QKV>(p, group, MP, sh, s_rstd, s_pos, gm, fs); break;
-    case EPI_RES: finalize_group_t<EPI_RES>(p, group, MP, sh, s_rstd, s_pos, gm, fs); break;
-    default: finalize_group_t<EPI_GATE_UP>(p, group, MP, sh, s_rstd, s_pos, gm, fs); break;
+    case EPI_FC: finalize_group_t<EPI_FC, NTHR, BAR>(ft, p, group, MP, sh, s_rstd, s_pos, gm, fs, dry); break;
+    case EPI_QKV: finalize_group_t<EPI_QKV, NTHR, BAR>(ft, p, group, MP, sh, s_rstd, s_pos, gm, fs, dry); break;
+    case EPI_RES: finalize_group_t<EPI_RES, NTHR, BAR>(ft, p, group, MP, sh, s_rstd, s_pos, gm, fs, dry); break;
+    default: finalize_group_t<EPI_GATE_UP, NTHR, BAR>(ft, p, group, MP, sh, s_rstd, s_pos, gm, fs, dry); break;
   }
 }
 

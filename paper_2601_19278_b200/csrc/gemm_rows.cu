@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(512, (NT == 1 ? 2 : 1)) gemm_rows_kernel(const
       asm volatile("cp.async.wait_all;" ::: "memory");
       __syncthreads();
     }
-    finalize_group(p, group, 8 * NT, sh, s_rstd, s_pos, &s_meta[slot], fs);
+    finalize_group<512, 0>(threadIdx.x, p, group, 8 * NT, sh, s_rstd, s_pos, &s_meta[slot], fs);
     if (threadIdx.x == 0) p.ctr[group] = 0;
     __syncthreads();
   }

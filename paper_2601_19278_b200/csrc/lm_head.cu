@@ -229,6 +229,16 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
     abort_flag = 0;
     s_bad = 0;
     fence_barrier_init();
+    // this thread is the producer: the ring is filled with weights before anything else of the CTA's setup
+    const int n = (int)(u1 - u0);
+    const int pre = n < C::Stages ? n : C::Stages;
+    const uint64_t wpol = l2_policy_evict_first();
+    int tile = (int)(u0 / KB), kb = (int)(u0 % KB);
+    for (int it = 0; it < pre; ++it) {
+      mbar_expect_tx(&full[it], C::StageBytes);
+      tma_load_2d_hint(ring + (size_t)it * C::StageBytes, &a.mapW, &full[it], kb * 64, tile * 128, wpol);
+      if (++kb == KB) { kb = 0; ++tile; }
+    }
   }
   if (warp == 2) tmem_alloc(&tmem_base, C::TmemCols);
   for (int i = tid; i < MP * 32; i += kLmUmmaThreads) { st_key[i] = -INFINITY; st_y[i] = 0.f; st_id[i] = 0x7fffffff; }
@@ -239,16 +249,11 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
   const uint32_t tmem = tmem_base;
 
   if (warp == 0 && lane == 0) {
-    // ---- producer: weights do not depend on the previous kernel, activations do
+    // ---- producer (the ring already holds the first weights): activations depend on the previous kernel
     const int n = (int)(u1 - u0);
     const int pre = n < C::Stages ? n : C::Stages;
     const uint64_t wpol = l2_policy_evict_first();
-    int tile = (int)(u0 / KB), kb = (int)(u0 % KB);
-    for (int it = 0; it < pre; ++it) {
-      mbar_expect_tx(&full[it], C::StageBytes);
-      tma_load_2d_hint(ring + (size_t)it * C::StageBytes, &a.mapW, &full[it], kb * 64, tile * 128, wpol);
-      if (++kb == KB) { kb = 0; ++tile; }
-    }
+    int tile, kb;
     pdl_wait();
     tile = (int)(u0 / KB); kb = (int)(u0 % KB);
     for (int it = 0; it < pre; ++it) {

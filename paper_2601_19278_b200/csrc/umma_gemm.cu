@@ -87,6 +87,17 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
     s_done[0] = 0;
     s_cnt[0] = s_cnt[1] = s_cnt[2] = s_cnt[3] = 0;
     fence_barrier_init();
+    // this thread is the producer: weights do not depend on the previous kernel, so the ring is filled with
+    // them before anything else of the CTA's setup
+    const int n = (int)(u1 - u0);
+    const int pre = n < C::Stages ? n : C::Stages;
+    const uint64_t wpol = l2_policy_evict_first();
+    UnitPos q;
+    if (n > 0) q.set(p.s, u0);
+    for (int it = 0; it < pre; ++it, q.next(p.s)) {
+      mbar_expect_tx(&full[it], C::StageBytes);
+      tma_load_2d_hint(ring + (size_t)it * C::StageBytes, &a.mapW[q.seg], &full[it], q.kb * 64, q.row0, wpol);
+    }
   }
   if (warp == 2) tmem_alloc(&tmem_base, C::TmemCols);
   if (p.epi.mode == EPI_QKV && threadIdx.x < p.s.M) {
@@ -108,16 +119,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
   const uint32_t tmem = tmem_base;
 
   if (warp == 0 && lane == 0) {
-    // ---- producer: weights do not depend on the previous kernel, activations do
+    // ---- producer (the ring already holds the first weights): activations depend on the previous kernel
     const int n = (int)(u1 - u0);
     const int pre = n < C::Stages ? n : C::Stages;
     const uint64_t wpol = l2_policy_evict_first();
     UnitPos q;
-    q.set(p.s, u0);
-    for (int it = 0; it < pre; ++it, q.next(p.s)) {
-      mbar_expect_tx(&full[it], C::StageBytes);
-      tma_load_2d_hint(ring + (size_t)it * C::StageBytes, &a.mapW[q.seg], &full[it], q.kb * 64, q.row0, wpol);
-    }
     pdl_wait();
     q.set(p.s, u0);
     for (int it = 0; it < pre; ++it, q.next(p.s)) {
@@ -245,7 +251,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       asm volatile("cp.async.wait_all;" ::: "memory");
       __syncthreads();
     }
-    finalize_group(p, group, MP, sh, s_rstd, s_pos, &s_meta[slot], fs);
+    finalize_group<512, 0>(threadIdx.x, p, group, MP, sh, s_rstd, s_pos, &s_meta[slot], fs);
     if (threadIdx.x == 0) p.ctr[group] = 0;
     __syncthreads();
   }
