@@ -42,6 +42,42 @@ class DraftSession:
             "v_cache": inp["v_cache"].to(d), "ctx_tail": inp["ctx_tail"].to(d), "n_fresh": int(inp["n_fresh"]),
         }
 
+    def pack_io(self):
+        """Re-home the step's small inputs (features, tokens, lengths, context tail) in ONE device buffer and
+        the tree outputs in another, each with a pinned host mirror, so that a caller moves a step's inputs
+        and results with one copy each way.  Returns (in_host, in_dev, out_host, out_dev, host_views): the
+        byte buffers and the host-side views of every field."""
+        def layout(fields):
+            off, spec = 0, {}
+            for name, t in fields:
+                off = (off + 255) // 256 * 256
+                spec[name] = (off, t.numel() * t.element_size(), t.dtype, tuple(t.shape))
+                off += t.numel() * t.element_size()
+            return spec, (off + 255) // 256 * 256
+
+        def carve(buf, spec):
+            return {n: buf[o:o + nb].view(dt).view(shape) for n, (o, nb, dt, shape) in spec.items()}
+
+        in_fields = [(n, self.inp[n]) for n in ("feats", "tokens", "seq_lens", "ctx_tail")]
+        out_fields = [(n, getattr(self, n)) for n in ("tokens", "parents", "depth", "mask", "n_nodes")]
+        ispec, ibytes = layout(in_fields)
+        ospec, obytes = layout(out_fields)
+        in_dev = torch.zeros(ibytes, dtype=torch.uint8, device=self.dev)
+        out_dev = torch.zeros(obytes, dtype=torch.uint8, device=self.dev)
+        in_host = torch.zeros(ibytes, dtype=torch.uint8).pin_memory()
+        out_host = torch.zeros(obytes, dtype=torch.uint8).pin_memory()
+        dviews, hviews = carve(in_dev, ispec), carve(in_host, ispec)
+        for n, t in in_fields:
+            hviews[n].copy_(t.cpu())
+            dviews[n].copy_(t)
+            self.inp[n] = dviews[n]
+        oviews = carve(out_dev, ospec)
+        for n, t in out_fields:
+            oviews[n].copy_(t)
+            setattr(self, n, oviews[n])
+        hviews.update({"out_" + n: v for n, v in carve(out_host, ospec).items()})
+        return in_host, in_dev, out_host, out_dev, hviews
+
     def step(self, step_counter: int = 0, stream=None) -> None:
         i = self.inp
         self.draft.draft_step(feats=i["feats"] if i["n_fresh"] else None, tokens=i["tokens"] if i["n_fresh"] else None,

@@ -123,3 +123,23 @@ def test_runs_are_bitwise_repeatable():
         for x, y in zip(a, b):
             assert torch.equal(x, y)
     ses.close()
+
+
+def test_packed_io_moves_a_step_with_one_copy_each_way():
+    """The end-to-end path of the benchmark: inputs in one pinned buffer, one copy in, one copy out."""
+    w = CASES["ragged_b2"]
+    wt, inp, rows, ses = _run(w)
+    ref = {k: getattr(ses, k).clone() for k in ("tokens", "parents", "depth", "mask", "n_nodes")}
+    in_host, in_dev, out_host, out_dev, hv = ses.pack_io()
+    in_dev.zero_()                                    # the inputs must really come from the host mirror
+    for n in ("tokens", "parents", "depth", "mask", "n_nodes"):
+        getattr(ses, n).fill_(3)
+    in_dev.copy_(in_host, non_blocking=True)
+    ses.step(step_counter=5)
+    ses.tree()
+    out_host.copy_(out_dev, non_blocking=True)
+    torch.cuda.synchronize()
+    assert ses.draft.device_status() == 0
+    for n, t in ref.items():
+        assert torch.equal(hv["out_" + n], t.cpu()), n
+    ses.close()
