@@ -9,14 +9,16 @@
  * Conventions
  *   - Every pointer is labelled HOST or DEVICE.  Device buffers are caller-owned unless stated.
  *   - bf16 tensors are row-major with the last index fastest; weight matrices are [out, in];
- *     weight pointers and `feats` must be 32-byte aligned (they are read with 256-bit loads), every
- *     other device pointer 16-byte aligned.
+ *     weight pointers and `feats` must be 32-byte aligned and their row strides multiples of 16 bytes
+ *     (they are read by TMA tile loads, or by 256-bit loads in the fallback kernels), every other device
+ *     pointer 16-byte aligned.
  *   - All GPU work is enqueued on the CUDA stream passed as `void* cuda_stream` (a cudaStream_t;
  *     NULL = the legacy default stream).  dart_draft_step and dart_build_tree do not
  *     synchronise, allocate, or copy between host and device.
  *   - Return value: DART_OK (0) or a negative dart_status.  Argument errors are reported
  *     synchronously and enqueue nothing.  Errors that only the device can detect (a lookup
- *     that ran past its probe bound) set a status word read by dart_last_device_status.
+ *     that ran past its probe bound, a bounded wait on a barrier or on another CTA's flag that ran
+ *     out) set a status word read by dart_last_device_status; the kernels never wait without a limit.
  *   - One handle may be used from one host thread and one stream at a time.
  *   - There is no CPU fallback: on a machine without an sm_100 device dart_draft_init fails.
  */

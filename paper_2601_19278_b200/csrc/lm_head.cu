@@ -1,17 +1,20 @@
 // LM head with fused vocab-sharded log-softmax + per-position top-k
 // (Section 3.2: one logit row per future position; Algorithm 1 lines 6-8; Appendix D s_logit).
 //
-// The LM head is 63 % of the step's bytes at the Qwen3-14B shape, so it is the kernel the
-// roofline is quoted on.  Each CTA owns a contiguous range of 16-row vocab tiles, balanced to
-// within one tile, and streams them with the shared core of stream_core.cuh (16 warps interleave
-// the k-steps of a tile, 2 CTAs per SM; the partial tiles are summed through shared memory).  Complete logits never leave the SM: every 128 vocab rows a warp per
-// token row folds them into a running (max, sum-exp) pair and an exact top-32 list held one
-// entry per lane.  The CTA writes (max, sum-exp, list) per token row; topk_merge_kernel
-// (topk_merge.cu) combines the CTAs' results and emits the k best ids with s_logit = log(softmax + eps).
+// The LM head is 63 % of the step's bytes at the Qwen3-14B shape, so it is the kernel the roofline is
+// quoted on.  Two kernels live here.  lm_head_umma_kernel (further down) is the one the step runs: TMA-fed
+// shared-memory ring, tcgen05.mma, logits in tensor memory.  lm_head_kernel is the mma.sync implementation
+// that came first; it is kept as the fallback for a driver without the tensor-map encoder: each CTA owns a
+// contiguous range of 16-row vocab tiles and streams them with the core of stream_core.cuh (16 warps
+// interleave the k-steps of a tile, 2 CTAs per SM; partial tiles are summed through shared memory).
+// In both, complete logits never leave the SM: every 128 vocab rows a warp per token row folds them into a
+// running (max, sum-exp) pair and an exact top-32 list held one entry per lane.  A CTA writes (max, sum-exp,
+// list) per token row; topk_merge_kernel (topk_merge.cu) combines the CTAs' results and emits the k best
+// ids with s_logit = log(softmax + eps).
 //
 // With temperature > 0 the list is ordered by logit/T + Gumbel noise (Gumbel-top-k = sampling
 // without replacement); the noise of token v in row (b, r) is word v&3 of
-// Philox4x32-10(counter = (v>>2, r, b, step), key = seed).
+// Philox4x32-10(counter = (v>>2, r, b, step), key = seed): a lane folds four consecutive tokens per call.
 #include <string.h>
 
 #include "common.cuh"
