@@ -70,8 +70,7 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const __grid_constant
   unsigned char* Vs = smem + 4 * TILE_BYTES;
 
   const int ci = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
-  pdl_wait();
-  const int P = p.seq_lens[b];
+  const int P = p.seq_lens[b];   // an input of the step: readable before the previous kernel has finished
   const int n_cc = (P + p.chunk_keys - 1) / p.chunk_keys;  // cache chunks of this sequence
   if (ci > n_cc) return;
   const bool is_new = ci == n_cc;
@@ -88,14 +87,6 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const __grid_constant
   const bf16* vbase = is_new ? p.v_new + ((size_t)b * p.Hkv + hk) * 16 * DH
                              : p.v_cache + ((size_t)b * p.Hkv + hk) * p.P_cap * DH;
 
-  // Q tiles, hi and lo (rows >= R zero-filled)
-  for (int i = tid; i < 64 * CH; i += 128) {
-    const int row = i / CH, ch = i % CH;
-    const bool ok = row < R;
-    const size_t off = qoff + (ok ? (size_t)row * DH + ch * 8 : 0);
-    cp_async16(smem_u32(Qh + swz<DH>(row, ch)), p.q_hi + off, ok ? 16 : 0);
-    cp_async16(smem_u32(Ql + swz<DH>(row, ch)), p.q_lo + off, ok ? 16 : 0);
-  }
   auto load_tile = [&](int ti, int buf) {
     const int k0 = k_begin + ti * 64;
     for (int i = tid; i < 64 * CH; i += 128) {
@@ -107,7 +98,20 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const __grid_constant
       cp_async16(smem_u32(Vs + buf * TILE_BYTES + swz<DH>(row, ch)), vbase + off, ok ? 16 : 0);
     }
   };
-  load_tile(0, 0);
+  // Cache rows below P_b were written by earlier steps, so a cache chunk's first tile is requested while the
+  // QKV kernel is still finishing; q and the new rows' side tile are its outputs and wait for it.
+  if (!is_new) load_tile(0, 0);
+  cp_async_commit();
+  pdl_wait();
+  // Q tiles, hi and lo (rows >= R zero-filled)
+  for (int i = tid; i < 64 * CH; i += 128) {
+    const int row = i / CH, ch = i % CH;
+    const bool ok = row < R;
+    const size_t off = qoff + (ok ? (size_t)row * DH + ch * 8 : 0);
+    cp_async16(smem_u32(Qh + swz<DH>(row, ch)), p.q_hi + off, ok ? 16 : 0);
+    cp_async16(smem_u32(Ql + swz<DH>(row, ch)), p.q_lo + off, ok ? 16 : 0);
+  }
+  if (is_new) load_tile(0, 0);
   cp_async_commit();
 
   const float sl2 = rsqrtf((float)DH) * 1.4426950408889634f;  // 1/sqrt(d_h) * log2(e)
