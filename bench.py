@@ -236,6 +236,24 @@ def run_ours(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
+    # ---- per-stage device times (outside both timed regions; each stage bracketed by events on its own steps)
+    stage_names = ["fc", "qkv_rope", "attention", "o_proj", "gate_up", "down", "lm_head", "topk_merge", "tree"]
+    stages_us = {}
+    if rank == 0:
+        for sidx, sname in enumerate(stage_names):
+            if sidx == 0 and inp["n_fresh"] == 0:
+                continue
+            ts = []
+            for i in range(12):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); b.record(stream)
+                stream.synchronize()
+                ses.draft.set_profile_events(sidx, a, b)
+                step(i)
+                stream.synchronize()
+                ts.append(1e3 * a.elapsed_time(b))
+            stages_us[sname] = statistics.median(ts)
+
     total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], world, dev)
     assert ses.draft.device_status() == 0
 
@@ -255,7 +273,9 @@ def run_ours(args):
                        "parallelism": "replicas only" if world > 1 else "1 GPU",
                        "l2": f"inputs larger than L2: {bytes_step / 1e9:.3f} GB of weights+KV streamed per step",
                        "feature_fc_in_path": inp["n_fresh"] > 0},
-            "latency_us": {"p50": 1e3 * statistics.median(per_step), "min": 1e3 * min(per_step), "max": 1e3 * max(per_step)},
+            "latency_us": {"p50": 1e3 * statistics.median(per_step), "p10": 1e3 * float(np.percentile(per_step, 10)),
+                           "p90": 1e3 * float(np.percentile(per_step, 90)), "min": 1e3 * min(per_step), "max": 1e3 * max(per_step)},
+            "stages_us": stages_us,
             "step_bytes": bytes_step, "step_gbs": step_gbs,
             "step_frac_of_hbm_peak": step_gbs / hbm_peak, "step_frac_of_8tbs": step_gbs / 8000.0,
             "roofline": {"bound": "hbm", "kernel": "lm_head_umma_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
