@@ -111,15 +111,17 @@ def draft_forward(cfg: Dict, w: Dict[str, np.ndarray], inp: Dict[str, np.ndarray
        w_q [Hq*dh,2h], w_k, w_v [Hkv*dh,2h], w_o [h,Hq*dh], norm_post, w_gate, w_up [I,h],
        w_down [h,I], norm_final, w_lm [V,h].
     inp: feats bits [B,F,3h], tokens [B,F], seq_lens [B], k_cache/v_cache bits [B,Hkv,Pcap,dh],
-       n_fresh F.
+       n_fresh F.  n_fresh may also be a sequence of B per-sequence counts F_b (the steady-state call after a
+       verification that accepted a different number of tokens per sequence, Section 3.2 / Figure 2); the
+       fresh rows' features and tokens are then packed in sequence order: feats [sum F_b, 3h], tokens [sum F_b].
     Returns logits [B,K,V] (row r predicts the token after absolute position P_b + r: shifted
     logits, Section 3.2) and the new rows' post-RoPE k and v [B,K,Hkv,dh].
     """
     h, Hq, Hkv, dh, K = (cfg[n] for n in ("hidden", "n_q_heads", "n_kv_heads", "head_dim", "K"))
     theta, eps = float(cfg["rope_theta"]), float(cfg["rms_eps"])
-    F = int(inp["n_fresh"])
     seq_lens = np.asarray(inp["seq_lens"]).astype(np.int64)
     B = seq_lens.shape[0]
+    Fb = np.broadcast_to(np.asarray(inp["n_fresh"], dtype=np.int64), (B,))      # fresh rows of each sequence
     gam = {n: bf16_to_f64(w[n]) for n in ("norm_g", "norm_e", "norm_post", "norm_final")}
     m = bf16_to_f64(w["mask_vec"])
 
@@ -127,13 +129,18 @@ def draft_forward(cfg: Dict, w: Dict[str, np.ndarray], inp: Dict[str, np.ndarray
     # 2h-vector stands in for the pre-norm [g ; e] of every mask row)
     g = np.empty((B, K, h), dtype=np.float64)
     e = np.empty((B, K, h), dtype=np.float64)
-    if F > 0:
-        feats = bf16_to_f64(inp["feats"])                       # [B,F,3h]
-        g[:, :F] = linear(feats, w["w_fc"])                     # fused features, no bias (reading)
-        tok = np.asarray(inp["tokens"]).astype(np.int64)
-        e[:, :F] = bf16_to_f64(w["embed"][tok.reshape(-1)]).reshape(B, F, h)  # shifted embedding
-    g[:, F:] = m[:h]
-    e[:, F:] = m[h:]
+    if Fb.sum() > 0:
+        feats = bf16_to_f64(inp["feats"]).reshape(-1, 3 * h)    # fresh rows packed in sequence order
+        gf = linear(feats, w["w_fc"])                           # fused features, no bias (reading)
+        ef = bf16_to_f64(w["embed"][np.asarray(inp["tokens"]).astype(np.int64).reshape(-1)])  # shifted embedding
+    off = 0
+    for b in range(B):
+        F = int(Fb[b])
+        g[b, :F] = gf[off:off + F] if F else 0.0
+        e[b, :F] = ef[off:off + F] if F else 0.0
+        g[b, F:] = m[:h]
+        e[b, F:] = m[h:]
+        off += F
     z = np.concatenate([rmsnorm(g, gam["norm_g"], eps), rmsnorm(e, gam["norm_e"], eps)], axis=-1)
     res = g                                                     # residual = un-normed g (reading)
 

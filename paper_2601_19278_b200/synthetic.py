@@ -161,8 +161,11 @@ def make_seq_lens(w: Workload, seed: int = BASE_SEED) -> np.ndarray:
     return np.full((w.batch,), w.prefix, dtype=np.int32)
 
 
-def make_step_inputs(w: Workload, seed: int = BASE_SEED, n_fresh: Optional[int] = None) -> Dict[str, object]:
-    """Per-step inputs: target features, next-token ids, prefix KV cache, lengths, context tail."""
+def make_step_inputs(w: Workload, seed: int = BASE_SEED, n_fresh=None) -> Dict[str, object]:
+    """Per-step inputs: target features, next-token ids, prefix KV cache, lengths, context tail.
+    n_fresh: one count for every sequence, or a list of per-sequence counts (see make_ragged_step_inputs)."""
+    if n_fresh is not None and not isinstance(n_fresh, (int, np.integer)):
+        return make_ragged_step_inputs(w, list(n_fresh), seed)
     F = w.n_fresh if n_fresh is None else n_fresh
     B = w.batch
     zipf = ZipfSampler(w.vocab)
@@ -185,6 +188,27 @@ def make_step_inputs(w: Workload, seed: int = BASE_SEED, n_fresh: Optional[int] 
         "seq_lens": torch.from_numpy(seq_lens), "k_cache": k_cache, "v_cache": v_cache,
         "ctx_tail": torch.from_numpy(ctx_tail), "n_fresh": F,
     }
+
+
+def make_ragged_step_inputs(w: Workload, fresh_counts, seed: int = BASE_SEED) -> Dict[str, object]:
+    """The steady-state call after a verification that accepted a different number of tokens per sequence:
+    sequence b has fresh_counts[b] fresh rows (0..K).  Every sequence draws K rows of features and tokens
+    exactly as the uniform generator with n_fresh = K would, then keeps its first fresh_counts[b]; the kept
+    rows are packed in sequence order: feats [sum F_b, 3h], tokens [sum F_b].  "n_fresh" is the list."""
+    assert len(fresh_counts) == w.batch and all(0 <= f <= w.K for f in fresh_counts)
+    full = make_step_inputs(w, seed, n_fresh=w.K)
+    keep_f = [full["feats"][b, :f] for b, f in enumerate(fresh_counts)]
+    keep_t = [full["tokens"][b, :f] for b, f in enumerate(fresh_counts)]
+    out = dict(full)
+    out["feats"] = torch.cat(keep_f, 0).contiguous()
+    out["tokens"] = torch.cat(keep_t, 0).contiguous()
+    ctx = full["ctx_tail"].clone()
+    alt = ZipfSampler(w.vocab).draw(w.batch, _gen(seed + 1000, "ctx_tail"))
+    for b, f in enumerate(fresh_counts):
+        ctx[b, 1] = int(full["tokens"][b, f - 1]) if f > 0 else int(alt[b])
+    out["ctx_tail"] = ctx
+    out["n_fresh"] = [int(f) for f in fresh_counts]
+    return out
 
 
 def make_ngram_rows(vocab: int, n_rows: int, mode: str, seed: int = BASE_SEED,

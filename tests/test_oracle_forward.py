@@ -262,3 +262,27 @@ def test_algorithmic_bytes_match_the_closed_form_per_config():
     for name, val in expect.items():
         w = syn.WORKLOADS[name]
         assert syn.algorithmic_bytes(w, syn.make_seq_lens(w)) == val
+
+
+def test_per_sequence_fresh_counts_equal_each_sequence_run_alone():
+    """Ragged fresh rows (the steady-state call after a verification that accepted a different number of
+    tokens per sequence): every sequence of the batch must come out exactly as if it had been run alone with
+    its own uniform count - which pins the packed feature/token offsets against the uniform path, itself
+    pinned by the torch restatement above."""
+    counts = [2, 0, 4, 1]
+    w = syn.small_variant(TINY, batch=4, ragged_lo=7)
+    wt = _np_weights(syn.make_weights(w))
+    inp = syn.make_step_inputs(w, n_fresh=counts)
+    assert inp["feats"].shape[0] == sum(counts) and list(inp["n_fresh"]) == counts
+    cfg = _cfg(w)
+    got = ofw.draft_forward(cfg, wt, _np_inputs(inp))
+    full = syn.make_step_inputs(w, n_fresh=w.K)                   # the rows every sequence drew
+    for b, F in enumerate(counts):
+        solo = {"feats": full["feats"][b:b + 1, :F].contiguous(), "tokens": full["tokens"][b:b + 1, :F].contiguous(),
+                "seq_lens": full["seq_lens"][b:b + 1], "k_cache": full["k_cache"][b:b + 1], "v_cache": full["v_cache"][b:b + 1],
+                "n_fresh": F}
+        ref = ofw.draft_forward(cfg, wt, _np_inputs(solo))
+        np.testing.assert_array_equal(got["logits"][b], ref["logits"][0])
+        np.testing.assert_array_equal(got["k_new"][b], ref["k_new"][0])
+    # the counts matter: a fresh row and a <mask> row at the same place give different logits
+    assert np.abs(got["logits"][0, 1] - got["logits"][1, 1]).max() > 1e-3
