@@ -168,12 +168,13 @@ def run_ours(args):
     if args.vocab:
         w = syn.small_variant(w, vocab=args.vocab, name=f"{w.name} with vocab cut to {args.vocab}")
     wt = syn.make_weights(w)
-    inp = syn.make_step_inputs(w)
+    inp = syn.make_step_inputs(w, n_fresh=syn.draw_fresh_counts(w) if args.ragged_fresh else None)
     rows = syn.make_ngram_rows(w.vocab, w.ngram_rows, w.ngram_mode)
     ses = runner.DraftSession(w, wt, rows, device=f"cuda:{local}", want_logits=False)
     ses.load_inputs(inp)
     stream = torch.cuda.current_stream()
-    n_launch = ses.draft.launch_count(w.batch, inp["n_fresh"])
+    any_fresh = int(np.max(inp["n_fresh"])) > 0
+    n_launch = ses.draft.launch_count(w.batch, 1 if any_fresh else 0)
     hbm_peak, peak_kind = _peaks()
     bytes_step = syn.algorithmic_bytes(w, inp["seq_lens"].numpy())
     lm_bytes = 2 * w.vocab * w.hidden
@@ -241,7 +242,7 @@ def run_ours(args):
     stages_us = {}
     if rank == 0:
         for sidx, sname in enumerate(stage_names):
-            if sidx == 0 and inp["n_fresh"] == 0:
+            if sidx == 0 and not any_fresh:
                 continue
             ts = []
             for i in range(12):
@@ -272,7 +273,7 @@ def run_ours(args):
                                    f"topk {w.topk}, beam {w.beam}, budget {w.tree_budget}, ngram_rows {len(rows['next'])}, T={w.temperature}",
                        "parallelism": "replicas only" if world > 1 else "1 GPU",
                        "l2": f"inputs larger than L2: {bytes_step / 1e9:.3f} GB of weights+KV streamed per step",
-                       "feature_fc_in_path": inp["n_fresh"] > 0},
+                       "feature_fc_in_path": any_fresh},
             "latency_us": {"p50": 1e3 * statistics.median(per_step), "p10": 1e3 * float(np.percentile(per_step, 10)),
                            "p90": 1e3 * float(np.percentile(per_step, 90)), "min": 1e3 * min(per_step), "max": 1e3 * max(per_step)},
             "stages_us": stages_us,
@@ -335,6 +336,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--vocab", type=int, default=0,
                     help="override the workload's vocabulary (a smaller case of the same kernels, for ncu captures)")
+    ap.add_argument("--ragged-fresh", action="store_true",
+                    help="per-sequence fresh-row counts (a steady-state call after a verification that accepted a different "
+                         "number of tokens per sequence) instead of the workload's uniform count")
     ap.add_argument("--lm-traffic", type=float, default=None,
                     help="DRAM bytes per LM-head launch from the committed ncu capture (profiles/), reported as roofline.traffic")
     args = ap.parse_args()

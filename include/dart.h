@@ -120,12 +120,15 @@ typedef struct dart_ngram_host {
  * r = 0..K-1 at absolute positions P_b + r, P_b = seq_lens[b]; rows r < n_fresh carry fresh
  * target features and the id of the token that follows them (shifted embedding), the rest
  * are <mask> rows.  The canonical step is n_fresh = 1: the last prefix position plus d-1 masks.
+ * After a verification that accepted a different number of tokens per sequence the counts differ:
+ * fresh_counts_host[b] = F_b then replaces n_fresh, and the fresh rows' features and token ids are
+ * packed in sequence order (sequence 0's F_0 rows, then sequence 1's, ...).
  */
 typedef struct dart_step_in {
   int32_t batch;          /* B <= max_batch */
   int32_t n_fresh;        /* F, 0..K (0: K mask rows, feats/tokens unused) */
-  const void* feats;      /* DEVICE bf16 [B, F, feat_in] */
-  const int32_t* tokens;  /* DEVICE i32  [B, F] next-token ids, 0 <= id < V */
+  const void* feats;      /* DEVICE bf16 [B, F, feat_in]  (packed [sum F_b, feat_in] with fresh_counts_host) */
+  const int32_t* tokens;  /* DEVICE i32  [B, F] next-token ids, 0 <= id < V  (packed [sum F_b]) */
   const int32_t* seq_lens;      /* DEVICE i32 [B]  P_b: rows already in the cache */
   const int32_t* seq_lens_host; /* HOST   i32 [B]  same values; used for capacity checks and launch sizing */
   void* k_cache;          /* DEVICE bf16 [max_batch, H_kv, max_prefix, d_h], post-RoPE keys */
@@ -133,6 +136,8 @@ typedef struct dart_step_in {
                              rows P_b .. P_b+F-1 of both caches and nothing else (the <mask> rows' k, v
                              are transient); the caller advances seq_lens.  Needs P_b + F <= max_prefix. */
   uint64_t step_counter;  /* Philox counter word; change it every call when temperature > 0 */
+  const int32_t* fresh_counts_host; /* HOST i32 [B] per-sequence fresh-row counts F_b in 0..K, or NULL: every
+                                       sequence has n_fresh.  With it the call appends rows P_b .. P_b+F_b-1. */
 } dart_step_in;
 
 /*
@@ -154,6 +159,8 @@ typedef struct dart_tree_in {
   const int32_t* topk_ids;    /* DEVICE i32 [B, K, topk] as written by dart_draft_step */
   const float* topk_slogit;   /* DEVICE f32 [B, K, topk] */
   const int32_t* ctx_tail;    /* DEVICE i32 [B, 2]: the last two known tokens (c_-2, c_-1); -1 = absent */
+  const int32_t* first_rows_host; /* HOST i32 [B] per-sequence first logit row (= max(F_b,1)-1), or NULL: first_row for
+                                     all.  Sequence b then has min(n_levels, K - first_rows_host[b]) levels. */
 } dart_tree_in;
 
 /*
@@ -184,8 +191,8 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
 /*
  * One forward pass of the draft layer and LM head with fused log-softmax/top-k
  * (Section 3.2; Algorithm 1 lines 6-8; Appendix D s_logit).  Asynchronous on `cuda_stream`.
- * Errors: INVALID_ARG (NULL pointers, n_fresh out of range), CAPACITY (batch > max_batch or
- * seq_lens_host[b] + n_fresh > max_prefix).
+ * Errors: INVALID_ARG (NULL pointers, a fresh-row count out of range), CAPACITY (batch > max_batch or
+ * seq_lens_host[b] + F_b > max_prefix).
  */
 int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out* out, void* cuda_stream);
 

@@ -59,7 +59,7 @@ class DartNgramHost(C.Structure):
 class DartStepIn(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_fresh", C.c_int32), ("feats", C.c_void_p), ("tokens", C.c_void_p),
                 ("seq_lens", C.c_void_p), ("seq_lens_host", C.c_void_p), ("k_cache", C.c_void_p),
-                ("v_cache", C.c_void_p), ("step_counter", C.c_uint64)]
+                ("v_cache", C.c_void_p), ("step_counter", C.c_uint64), ("fresh_counts_host", C.c_void_p)]
 
 
 class DartStepOut(C.Structure):
@@ -68,7 +68,7 @@ class DartStepOut(C.Structure):
 
 class DartTreeIn(C.Structure):
     _fields_ = [("batch", C.c_int32), ("first_row", C.c_int32), ("n_levels", C.c_int32), ("topk_ids", C.c_void_p),
-                ("topk_slogit", C.c_void_p), ("ctx_tail", C.c_void_p)]
+                ("topk_slogit", C.c_void_p), ("ctx_tail", C.c_void_p), ("first_rows_host", C.c_void_p)]
 
 
 class DartTreeOut(C.Structure):
@@ -177,22 +177,28 @@ class DartDraft:
     def _stream(stream) -> int:
         return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
 
-    def draft_step(self, *, feats, tokens, seq_lens, seq_lens_host: np.ndarray, k_cache, v_cache, n_fresh: int,
+    def draft_step(self, *, feats, tokens, seq_lens, seq_lens_host: np.ndarray, k_cache, v_cache, n_fresh,
                    topk_ids, topk_slogit, logits=None, step_counter: int = 0, stream=None) -> None:
-        """dart_draft_step: all tensors are caller-owned device tensors; seq_lens_host is a host int32 array."""
+        """dart_draft_step: all tensors are caller-owned device tensors; seq_lens_host is a host int32 array.
+        n_fresh: one count for all sequences, or a sequence of per-sequence counts (fresh_counts_host)."""
         slh = np.ascontiguousarray(seq_lens_host, dtype=np.int32)
-        sin = DartStepIn(len(slh), n_fresh, _ptr(feats), _ptr(tokens), _ptr(seq_lens), slh.ctypes.data,
-                         _ptr(k_cache), _ptr(v_cache), step_counter)
+        counts = None if isinstance(n_fresh, (int, np.integer)) else np.ascontiguousarray(n_fresh, dtype=np.int32)
+        sin = DartStepIn(len(slh), int(n_fresh) if counts is None else int(counts.max(initial=0)), _ptr(feats), _ptr(tokens),
+                         _ptr(seq_lens), slh.ctypes.data, _ptr(k_cache), _ptr(v_cache), step_counter,
+                         None if counts is None else counts.ctypes.data)
         sout = DartStepOut(_ptr(topk_ids), _ptr(topk_slogit), _ptr(logits))
         rc = lib().dart_draft_step(self._h, C.byref(sin), C.byref(sout), self._stream(stream))
         if rc != DART_OK:
             raise DartError(rc, "dart_draft_step", lib().dart_last_cuda_error(self._h))
 
     def build_tree(self, *, batch: int, topk_ids, topk_slogit, ctx_tail, tokens, parents, depth, mask, n_nodes,
-                   scores=None, first_row: int = 0, n_levels: Optional[int] = None, stream=None) -> None:
-        """dart_build_tree on caller-owned device tensors."""
-        tin = DartTreeIn(batch, first_row, self.cfg.K - first_row if n_levels is None else n_levels,
-                         _ptr(topk_ids), _ptr(topk_slogit), _ptr(ctx_tail))
+                   scores=None, first_row=0, n_levels: Optional[int] = None, stream=None) -> None:
+        """dart_build_tree on caller-owned device tensors.  first_row: one row for all sequences, or a sequence
+        of per-sequence first rows (first_rows_host)."""
+        rows = None if isinstance(first_row, (int, np.integer)) else np.ascontiguousarray(first_row, dtype=np.int32)
+        fr = int(first_row) if rows is None else int(rows.min())
+        tin = DartTreeIn(batch, fr, self.cfg.K - fr if n_levels is None else n_levels,
+                         _ptr(topk_ids), _ptr(topk_slogit), _ptr(ctx_tail), None if rows is None else rows.ctypes.data)
         tout = DartTreeOut(_ptr(tokens), _ptr(parents), _ptr(depth), _ptr(mask), _ptr(n_nodes), _ptr(scores))
         rc = lib().dart_build_tree(self._h, C.byref(tin), C.byref(tout), self._stream(stream))
         if rc != DART_OK:

@@ -65,7 +65,8 @@ struct dart_handle {
   uint32_t ng_mask = 0, ng_max_probe = 0;
   float wl[8], wv[8], wn, miss;
   std::vector<void*> owned;  // small device arrays (plan tables, counters)
-  int z_B = -1, z_F = -1;    // row pattern (batch, fresh rows) the <mask> rows of z were last written for
+  int z_B = -1;              // row pattern (batch, per-sequence fresh rows) the <mask> rows of z were last written for
+  FreshOffsets z_foff = {};
   int prof_stage = -1;       // measurement aid: stage whose kernels the next call brackets with events
   cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
 };
@@ -513,18 +514,28 @@ int dart_step_launch_count(const dart_handle* h, int batch, int n_fresh) {
 int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out* out, void* cuda_stream) {
   if (h == nullptr || in == nullptr || out == nullptr) return DART_ERR_INVALID_ARG;
   const dart_config& c = h->cfg;
-  const int B = in->batch, F = in->n_fresh, K = c.K;
-  if (B < 1 || F < 0 || F > K) return DART_ERR_INVALID_ARG;
+  const int B = in->batch, K = c.K;
+  if (B < 1) return DART_ERR_INVALID_ARG;
   if (B > c.max_batch) return DART_ERR_CAPACITY;
+  // fresh rows per sequence: one count for all, or the caller's per-sequence counts
+  FreshOffsets fo;
+  fo.v[0] = 0;
+  for (int b = 0; b < B; ++b) {
+    const int Fb = in->fresh_counts_host != nullptr ? in->fresh_counts_host[b] : in->n_fresh;
+    if (Fb < 0 || Fb > K) return DART_ERR_INVALID_ARG;
+    fo.v[b + 1] = fo.v[b] + Fb;
+  }
+  for (int b = B + 1; b < 33; ++b) fo.v[b] = fo.v[B];
+  const int NF = fo.v[B];   // fresh rows of the whole batch
   if (in->seq_lens == nullptr || in->seq_lens_host == nullptr || !aligned16(in->k_cache) || !aligned16(in->v_cache))
     return DART_ERR_INVALID_ARG;
-  if (F > 0 && (!aligned32(in->feats) || in->tokens == nullptr)) return DART_ERR_INVALID_ARG;
+  if (NF > 0 && (!aligned32(in->feats) || in->tokens == nullptr)) return DART_ERR_INVALID_ARG;
   if (out->topk_ids == nullptr || out->topk_slogit == nullptr) return DART_ERR_INVALID_ARG;
   long long total_keys = 0;
   for (int b = 0; b < B; ++b) {
     const int P = in->seq_lens_host[b];
     if (P < 0) return DART_ERR_INVALID_ARG;
-    if ((long long)P + F > c.max_prefix) return DART_ERR_CAPACITY;
+    if ((long long)P + (fo.v[b + 1] - fo.v[b]) > c.max_prefix) return DART_ERR_CAPACITY;
     total_keys += P;
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -554,29 +565,33 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   };
 
   // the <mask> rows of z are constant; they are (re)written only when the row pattern changes
-  if (h->z_B != B || h->z_F != F) {
-    if ((e = launch_fill_mask_rows(ws.z_hi, ws.z_lo, ws.zmask_hi, ws.zmask_lo, B, K, F, 2 * hdim, st)) != cudaSuccess) return fail_cuda(h, e);
-    h->z_B = B; h->z_F = F;
+  if (h->z_B != B || memcmp(h->z_foff.v, fo.v, sizeof(fo.v)) != 0) {
+    if ((e = launch_fill_mask_rows(ws.z_hi, ws.z_lo, ws.zmask_hi, ws.zmask_lo, B, K, fo, 2 * hdim, st)) != cudaSuccess) return fail_cuda(h, e);
+    h->z_B = B; h->z_foff = fo;
   }
+  auto set_epi = [&](int mode) {
+    memset(&ep, 0, sizeof(ep));
+    ep.mode = mode; ep.K = K; ep.h = hdim; ep.eps = c.rms_eps; ep.B = B;
+    memcpy(ep.foff, fo.v, sizeof(ep.foff));
+  };
 
   // S0: feature-fusion FC on the fresh rows; epilogue: residual g, z g-half (gain-scaled), sums of squares;
   // prologue: z e-half = RMSNorm(embedding of the next token)
   mark(0, true);
-  if (F > 0) {
-    memset(&ep, 0, sizeof(ep));
-    ep.mode = EPI_FC; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
+  if (NF > 0) {
+    set_epi(EPI_FC);
     ep.res0 = ws.res0; ep.gamma = static_cast<const bf16*>(h->w.norm_g);
     ep.out_hi = ws.z_hi; ep.out_lo = ws.z_lo; ep.ld_out = 2 * hdim; ep.ss_out = ws.ss_g;
     ep.tokens = in->tokens; ep.vocab = c.vocab; ep.embed = static_cast<const bf16*>(h->w.embed);
     ep.gamma_e = static_cast<const bf16*>(h->w.norm_e);
-    gi = {static_cast<const bf16*>(in->feats), nullptr, c.feat_in, B * F};
-    if (h->umma && (h->maps_feats != in->feats || h->maps_fc_M != B * F)) {
-      // plain bf16 input: one box of 2 * MP rows, the rows past B * F (the "lo" half among them) read as zeros
-      if ((e = tmap_encode_bf16(&h->maps_fc.Xhi, in->feats, c.feat_in, B * F, (unsigned long long)c.feat_in * 2, 64,
-                                2 * padded_tokens(B * F))) != cudaSuccess)
+    gi = {static_cast<const bf16*>(in->feats), nullptr, c.feat_in, NF};
+    if (h->umma && (h->maps_feats != in->feats || h->maps_fc_M != NF)) {
+      // plain bf16 input: one box of 2 * MP rows, the rows past the fresh rows (the "lo" half among them) read as zeros
+      if ((e = tmap_encode_bf16(&h->maps_fc.Xhi, in->feats, c.feat_in, NF, (unsigned long long)c.feat_in * 2, 64,
+                                2 * padded_tokens(NF))) != cudaSuccess)
         return fail_cuda(h, e);
       h->maps_fc.Xlo = h->maps_fc.Xhi;
-      h->maps_feats = in->feats; h->maps_fc_M = B * F;
+      h->maps_feats = in->feats; h->maps_fc_M = NF;
     }
     if ((e = project(h->plan_fc, h->maps_fc)) != cudaSuccess) return fail_cuda(h, e);
   }
@@ -584,9 +599,8 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
 
   // S1: QKV projection; epilogue: 1/rms of g, RoPE, q and new k/v as hi/lo, cache append
   mark(1, true);
-  memset(&ep, 0, sizeof(ep));
-  ep.mode = EPI_QKV; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
-  ep.ss_in = ws.ss_g; ep.ss_tiles = h->h_tiles; ep.ss_mp = padded_tokens(B * (F > 0 ? F : 1)); ep.rstd_mask = ws.rstd_mask;
+  set_epi(EPI_QKV);
+  ep.ss_in = ws.ss_g; ep.ss_tiles = h->h_tiles; ep.ss_mp = padded_tokens(NF > 0 ? NF : 1); ep.rstd_mask = ws.rstd_mask;
   ep.Hq = c.n_q_heads; ep.Hkv = c.n_kv_heads; ep.dh = c.head_dim; ep.seq_lens = in->seq_lens; ep.rope_tab = ws.rope_tab;
   ep.q_hi = ws.q_hi; ep.q_lo = ws.q_lo; ep.k_new = ws.k_new; ep.v_new = ws.v_new;
   ep.k_cache = static_cast<bf16*>(in->k_cache); ep.v_cache = static_cast<bf16*>(in->v_cache); ep.P_cap = c.max_prefix;
@@ -618,8 +632,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
 
   // S3: o_proj; epilogue: x1 = residual + proj, gain-scaled hi/lo, sums of squares
   mark(3, true);
-  memset(&ep, 0, sizeof(ep));
-  ep.mode = EPI_RES; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
+  set_epi(EPI_RES);
   ep.res0 = ws.res0; ep.res_in = nullptr; ep.res_out = ws.x1; ep.mask_res = ws.mask_res;
   ep.gamma = static_cast<const bf16*>(h->w.norm_post);
   ep.out_hi = ws.n_hi; ep.out_lo = ws.n_lo; ep.ld_out = hdim; ep.ss_out = ws.ss_1;
@@ -629,8 +642,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
 
   // S4: gate/up; epilogue: u = SiLU(rstd1 * gate) * (rstd1 * up)
   mark(4, true);
-  memset(&ep, 0, sizeof(ep));
-  ep.mode = EPI_GATE_UP; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
+  set_epi(EPI_GATE_UP);
   ep.ss_in = ws.ss_1; ep.ss_tiles = h->h_tiles; ep.ss_mp = MP;
   ep.out_hi = ws.u_hi; ep.out_lo = ws.u_lo; ep.ld_out = c.mlp_inter;
   gi = {ws.n_hi, ws.n_lo, hdim, M};
@@ -639,8 +651,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
 
   // S5: down; epilogue: x2 = x1 + proj, gain-scaled hi/lo for the LM head, sums of squares
   mark(5, true);
-  memset(&ep, 0, sizeof(ep));
-  ep.mode = EPI_RES; ep.K = K; ep.F = F; ep.h = hdim; ep.eps = c.rms_eps;
+  set_epi(EPI_RES);
   ep.res_in = ws.x1; ep.res_out = nullptr; ep.gamma = static_cast<const bf16*>(h->w.norm_final);
   ep.out_hi = ws.n_hi; ep.out_lo = ws.n_lo; ep.ld_out = hdim; ep.ss_out = ws.ss_2;
   gi = {ws.u_hi, ws.u_lo, c.mlp_inter, M};
@@ -692,6 +703,14 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
   TreeParams tp;
   tp.B = in->batch; tp.K = c.K; tp.topk = c.topk; tp.beam = c.beam; tp.budget = c.tree_budget;
   tp.first_row = in->first_row; tp.n_levels = in->n_levels; tp.ngram_order = c.ngram_order;
+  for (int b = 0; b < 32; ++b) {  // per-sequence first logit row (level 0); a sequence has min(n_levels, K - first row) levels
+    int fr = in->first_row;
+    if (in->first_rows_host != nullptr && b < in->batch) {
+      fr = in->first_rows_host[b];
+      if (fr < 0 || fr >= c.K) return DART_ERR_INVALID_ARG;
+    }
+    tp.first_rows[b] = (unsigned char)fr;
+  }
   tp.ids = in->topk_ids; tp.slogit = in->topk_slogit; tp.ctx_tail = in->ctx_tail;
   tp.table.slots = h->ng_slots; tp.table.mask = h->ng_mask; tp.table.max_probe = h->ng_max_probe;
   for (int i = 0; i < 8; ++i) { tp.wl[i] = h->wl[i]; tp.wv[i] = h->wv[i]; }

@@ -7,6 +7,17 @@
 
 namespace dart {
 
+// Packed index of fresh row (b, r), or -1 for a <mask> row.
+__device__ __forceinline__ int fresh_index(const EpiArgs& e, int b, int r) {
+  return r < e.foff[b + 1] - e.foff[b] ? e.foff[b] + r : -1;
+}
+// Step row b*K + r of packed fresh row f (a scan over at most 32 sequences).
+__device__ __forceinline__ int fresh_to_step_row(const EpiArgs& e, int f) {
+  int b = 0;
+  while (b + 1 < e.B && f >= e.foff[b + 1]) ++b;
+  return b * e.K + (f - e.foff[b]);
+}
+
 // ------------------------------------------------------------------------------------------
 // Fused epilogues, run by the CTA that completes a tile (or a pair of tiles).
 // ------------------------------------------------------------------------------------------
@@ -149,9 +160,9 @@ static __device__ __noinline__ void finalize_group_t(int ft, const GemmArgs& p, 
   const int rows_valid = min(128, p.s.seg[s].rows - row_base);
   const int row = ft & 127, par = ft >> 7;
   const int n = row_base + row;
-  const int K = e.K, F = e.F;
+  const int K = e.K;
   const auto col_id = [](int tok) { return tok; };
-  const auto col_fresh = [K, F](int tok) { const int b = tok / K, rr = tok % K; return rr < F ? b * F + rr : -1; };
+  const auto col_fresh = [K, &e](int tok) { return fresh_index(e, tok / K, tok % K); };
   constexpr bool rowmode = MODE == EPI_FC || MODE == EPI_RES;
   const int dh = e.dh, half = dh >> 1;
   const int pairs = MODE == EPI_QKV ? (rows_valid / dh) * half : 1;   // (head, i) pairs of this tile
@@ -170,8 +181,8 @@ static __device__ __noinline__ void finalize_group_t(int ft, const GemmArgs& p, 
       const int t = tok0 + par + NPAR * k;
       if (MODE == EPI_RES && row < rows_valid && t < M) {
         // residual: the stream so far, or (first projection) g of a fresh row / the <mask> representation
-        const float* src = e.res_in != nullptr ? e.res_in + (size_t)t * e.h
-                                               : ((t % K) < F ? e.res0 + (size_t)((t / K) * F + t % K) * e.h : e.mask_res);
+        const int fi = e.res_in != nullptr ? -1 : fresh_index(e, t / K, t % K);
+        const float* src = e.res_in != nullptr ? e.res_in + (size_t)t * e.h : (fi >= 0 ? e.res0 + (size_t)fi * e.h : e.mask_res);
         res[k] = __ldcg(src + n);
       }
     }
@@ -214,7 +225,7 @@ static __device__ __noinline__ void finalize_group_t(int ft, const GemmArgs& p, 
       for (int k = 0; k < NV; ++k) {
         const int t = tok0 + par + NPAR * k;
         // the FC's token index counts fresh rows only; its z row is the step's row (b, r)
-        const int o = MODE == EPI_FC ? (t / F) * K + t % F : t;
+        const int o = MODE == EPI_FC ? fresh_to_step_row(e, t < M ? t : 0) : t;
         if (row < rows_valid && t < M && !dry) {
           if (resw != nullptr) resw[(size_t)t * e.h + n] = x[k];
           bf16 hi, lo;
@@ -269,7 +280,7 @@ static __device__ __noinline__ void finalize_group_t(int ft, const GemmArgs& p, 
             bf16* side = (kind == 1 ? e.k_new : e.v_new) + ((size_t)b * e.Hkv + head) * 16 * dh;
             side[(size_t)r * dh + i] = h1; side[(size_t)r * dh + i + half] = h2;
             side[(size_t)(8 + r) * dh + i] = l1; side[(size_t)(8 + r) * dh + i + half] = l2;
-            if (r < F) {
+            if (fresh_index(e, b, r) >= 0) {
               bf16* dst = (kind == 1 ? e.k_cache : e.v_cache) + (((size_t)b * e.Hkv + head) * e.P_cap + s_pos[tok]) * dh;
               dst[i] = h1;
               dst[i + half] = h2;
@@ -297,7 +308,7 @@ static __device__ __forceinline__ void finalize_group(int ft, const GemmArgs& p,
 // nothing else) and written as the second half of the fresh row's z.  One CTA per fresh row.
 static __device__ __noinline__ void embed_rows(const GemmArgs& p, float* sh, int ftok) {
   const EpiArgs& e = p.epi;
-  const int orow = (ftok / e.F) * e.K + ftok % e.F;   // z row of fresh row (b, r)
+  const int orow = fresh_to_step_row(e, ftok);   // z row of fresh row (b, r)
   const int id = min(max(e.tokens[ftok], 0), e.vocab - 1);
   const bf16* row = e.embed + (size_t)id * e.h;
   float ss = 0.f;

@@ -160,9 +160,10 @@ cudaError_t launch_rope_table(float2* tab, int n_pos, int dh, float theta, cudaS
   return cudaGetLastError();
 }
 
-__global__ void fill_mask_rows_kernel(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int K, int F, int width) {
-  const int tok = blockIdx.x;
-  if (tok % K < F) return;
+__global__ void fill_mask_rows_kernel(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int K, const FreshOffsets foff,
+                                      int width) {
+  const int tok = blockIdx.x, b = tok / K;
+  if (tok % K < foff.v[b + 1] - foff.v[b]) return;
   const uint4* sh = reinterpret_cast<const uint4*>(zmask_hi);
   const uint4* sl = reinterpret_cast<const uint4*>(zmask_lo);
   uint4* dh = reinterpret_cast<uint4*>(z_hi + (size_t)tok * width);
@@ -170,9 +171,9 @@ __global__ void fill_mask_rows_kernel(bf16* z_hi, bf16* z_lo, const bf16* zmask_
   for (int i = threadIdx.x; i < width / 8; i += blockDim.x) { dh[i] = sh[i]; dl[i] = sl[i]; }
 }
 
-cudaError_t launch_fill_mask_rows(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int B, int K, int F, int width,
-                                  cudaStream_t st) {
-  fill_mask_rows_kernel<<<B * K, 256, 0, st>>>(z_hi, z_lo, zmask_hi, zmask_lo, K, F, width);
+cudaError_t launch_fill_mask_rows(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int B, int K,
+                                  const FreshOffsets& foff, int width, cudaStream_t st) {
+  fill_mask_rows_kernel<<<B * K, 256, 0, st>>>(z_hi, z_lo, zmask_hi, zmask_lo, K, foff, width);
   return cudaGetLastError();
 }
 

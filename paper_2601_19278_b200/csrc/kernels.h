@@ -86,7 +86,10 @@ enum EpiMode : int { EPI_FC = 0, EPI_QKV = 1, EPI_RES = 2, EPI_GATE_UP = 3 };
 // Everything the fused epilogues need (unused fields stay zero).
 struct EpiArgs {
   int mode;
-  int K, F, h;        // rows per sequence, fresh rows per sequence, hidden
+  int K, h;           // rows per sequence, hidden
+  // Fresh rows: sequence b's rows r < F_b carry fresh target features, F_b = foff[b+1] - foff[b]; fresh row (b, r)
+  // is row foff[b] + r of the packed fresh arrays (features, tokens, g, sums of squares).  foff[B] = their count.
+  int B; int foff[33];
   float eps;
   // EPI_FC: g -> res0 [B*F, h], z g-half (gain-scaled, hi/lo, row stride ld_out), ss_out [tile][MP]
   // EPI_RES: x = res + proj -> res_out, out_hi/lo = x * gamma, ss_out
@@ -154,8 +157,9 @@ cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const Ep
 // (cos, sin) table of RoPE for positions 0 .. n_pos-1 (once, at init)
 cudaError_t launch_rope_table(float2* tab, int n_pos, int dh, float theta, cudaStream_t st);
 // Copies the <mask> row into every z row (b, r) with r >= F (when the batch size or F changes)
-cudaError_t launch_fill_mask_rows(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int B, int K, int F, int width,
-                                  cudaStream_t st);
+struct FreshOffsets { int v[33]; };   // prefix sums of the per-sequence fresh counts
+cudaError_t launch_fill_mask_rows(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int B, int K,
+                                  const FreshOffsets& foff, int width, cudaStream_t st);
 // z row of the <mask> rows and the 1/rms of its g half (once, at init)
 cudaError_t launch_mask_row(const bf16* mask_vec, const bf16* norm_g, const bf16* norm_e, int h, float eps, bf16* z_hi,
                             bf16* z_lo, float* rstd_mask, float* mask_res, cudaStream_t st);
@@ -217,6 +221,7 @@ struct NgramTable { const NgramSlot* slots; uint32_t mask; uint32_t max_probe; }
 
 struct TreeParams {
   int B, K, topk, beam, budget, first_row, n_levels, ngram_order;
+  unsigned char first_rows[32];   // per sequence: first logit row = level 0; levels = min(n_levels, K - first row)
   const int32_t* ids; const float* slogit; const int32_t* ctx_tail;
   NgramTable table;
   float* bg;   // [B][topk + (n_levels-1)*topk^2] bigram scores (workspace, written by the sweep kernel)

@@ -77,11 +77,12 @@ __host__ __device__ inline size_t tree_layout(int k, int w, int budget, int L, u
 // gives log(eps).
 __global__ void __launch_bounds__(256) bigram_sweep_kernel(const TreeParams p) {
   pdl_wait();
-  const int k = p.topk, L = p.n_levels, b = blockIdx.y;
-  const int n_bg = k + (L - 1) * k * k;
+  const int k = p.topk, b = blockIdx.y;
+  const int fr = p.first_rows[b], Lb = min(p.n_levels, p.K - fr);   // this sequence's level 0 row and levels
+  const int n_bg = k + (p.n_levels - 1) * k * k;                   // layout stride: the launch's maximum
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= n_bg) return;
-  const int* ids = p.ids + ((size_t)b * p.K + p.first_row) * k;
+  if (e >= k + (Lb - 1) * k * k) return;
+  const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
   int tb, tt;
   if (e < k) { tb = p.ctx_tail[2 * b + 1]; tt = ids[e]; }
   else { const int r = e - k, i = r / (k * k), q = r - i * k * k, jb = q / k; tb = ids[i * k + jb]; tt = ids[(i + 1) * k + q - jb * k]; }
@@ -99,15 +100,16 @@ __global__ void __launch_bounds__(256) bigram_sweep_kernel(const TreeParams p) {
 template <int MAXT>
 __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
   extern __shared__ __align__(16) unsigned char tsm[];
-  const int k = p.topk, w = p.beam, L = p.n_levels, theta = p.budget - 1;
+  const int k = p.topk, w = p.beam, theta = p.budget - 1;
+  const int fr = p.first_rows[blockIdx.x], L = min(p.n_levels, p.K - fr);   // this sequence's level 0 row and levels
   TreeSmem m;
-  tree_layout(k, w, p.budget, L, tsm, &m);
+  tree_layout(k, w, p.budget, p.n_levels, tsm, &m);
   __shared__ unsigned long long s_bits[64];
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
   pdl_wait();
-  const int* ids = p.ids + ((size_t)b * p.K + p.first_row) * k;
-  const float* sl = p.slogit + ((size_t)b * p.K + p.first_row) * k;
+  const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
+  const float* sl = p.slogit + ((size_t)b * p.K + fr) * k;
   const int ctx0 = p.ctx_tail[2 * b], ctx1 = p.ctx_tail[2 * b + 1];
   const NgramTable T = p.table;
   const bool have_table = T.slots != nullptr;

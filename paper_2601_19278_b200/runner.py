@@ -39,7 +39,9 @@ class DraftSession:
         self.inp = {
             "feats": inp["feats"].to(d), "tokens": inp["tokens"].to(d), "seq_lens": inp["seq_lens"].to(d),
             "seq_lens_host": inp["seq_lens"].numpy().astype(np.int32), "k_cache": inp["k_cache"].to(d),
-            "v_cache": inp["v_cache"].to(d), "ctx_tail": inp["ctx_tail"].to(d), "n_fresh": int(inp["n_fresh"]),
+            "v_cache": inp["v_cache"].to(d), "ctx_tail": inp["ctx_tail"].to(d),
+            # one count for all sequences, or a list of per-sequence counts
+            "n_fresh": inp["n_fresh"] if isinstance(inp["n_fresh"], (list, tuple, np.ndarray)) else int(inp["n_fresh"]),
         }
 
     def pack_io(self):
@@ -80,13 +82,20 @@ class DraftSession:
 
     def step(self, step_counter: int = 0, stream=None) -> None:
         i = self.inp
-        self.draft.draft_step(feats=i["feats"] if i["n_fresh"] else None, tokens=i["tokens"] if i["n_fresh"] else None,
+        any_fresh = int(np.max(i["n_fresh"])) > 0
+        self.draft.draft_step(feats=i["feats"] if any_fresh else None, tokens=i["tokens"] if any_fresh else None,
                               seq_lens=i["seq_lens"], seq_lens_host=i["seq_lens_host"], k_cache=i["k_cache"],
                               v_cache=i["v_cache"], n_fresh=i["n_fresh"], topk_ids=self.topk_ids,
                               topk_slogit=self.topk_slogit, logits=self.logits, step_counter=step_counter, stream=stream)
 
     def tree(self, stream=None, topk_ids=None, topk_slogit=None, ctx_tail=None, first_row: Optional[int] = None) -> None:
-        fr = max(self.inp["n_fresh"], 1) - 1 if first_row is None else first_row
+        nf = self.inp["n_fresh"]
+        if first_row is not None:
+            fr = first_row
+        elif isinstance(nf, int):
+            fr = max(nf, 1) - 1
+        else:
+            fr = [max(int(f), 1) - 1 for f in nf]      # level 0 of sequence b = its last fresh row
         self.draft.build_tree(batch=self.w.batch, topk_ids=self.topk_ids if topk_ids is None else topk_ids,
                               topk_slogit=self.topk_slogit if topk_slogit is None else topk_slogit,
                               ctx_tail=self.inp["ctx_tail"] if ctx_tail is None else ctx_tail,

@@ -190,6 +190,17 @@ def make_step_inputs(w: Workload, seed: int = BASE_SEED, n_fresh=None) -> Dict[s
     }
 
 
+def draw_fresh_counts(w: Workload, seed: int = BASE_SEED, mean_accept: float = 3.5) -> list:
+    """Per-sequence fresh-row counts of a steady-state call: one row for the token the target just sampled
+    plus the draft tokens the last verification accepted, a geometric number with the given mean (the paper
+    reports mean acceptance lengths of roughly 3 to 4 tokens per step), capped at K rows."""
+    g = _gen(seed + 19, "tokens")
+    u = torch.rand(w.batch, generator=g).numpy()
+    q = 1.0 - 1.0 / max(mean_accept, 1.0)                      # P(accept one more)
+    extra = np.floor(np.log(np.maximum(u, 1e-12)) / np.log(max(q, 1e-12))).astype(np.int64) if q > 0 else np.zeros(w.batch, np.int64)
+    return [int(min(w.K, 1 + e)) for e in extra]
+
+
 def make_ragged_step_inputs(w: Workload, fresh_counts, seed: int = BASE_SEED) -> Dict[str, object]:
     """The steady-state call after a verification that accepted a different number of tokens per sequence:
     sequence b has fresh_counts[b] fresh rows (0..K).  Every sequence draws K rows of features and tokens

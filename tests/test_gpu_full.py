@@ -17,10 +17,11 @@ from paper_2601_19278_b200 import runner, synthetic as syn
 pytestmark = pytest.mark.gpu
 
 
-def _full_case(name, ngram_rows=200_000, step_counter=3):
+def _full_case(name, ngram_rows=200_000, step_counter=3, ragged_fresh=False):
     w = syn.WORKLOADS[name]
     wt = syn.make_weights(w)
-    inp = syn.make_step_inputs(w)
+    inp = syn.make_step_inputs(w, n_fresh=syn.draw_fresh_counts(w) if ragged_fresh else None)
+    counts = list(np.broadcast_to(np.asarray(inp["n_fresh"]), (w.batch,)))
     rows = syn.make_ngram_rows(w.vocab, ngram_rows, w.ngram_mode)
     ses = runner.DraftSession(w, wt, rows, want_logits=True, philox_seed=parity.PHILOX_SEED)
     ses.load_inputs(inp)
@@ -53,8 +54,13 @@ def _full_case(name, ngram_rows=200_000, step_counter=3):
             worst = max(worst, parity.check_topk_row(ids_g[b, r], sl_g[b, r], ref["logits"][b, r], w.topk, 1e-10, w.temperature, noise))
         np.testing.assert_allclose(kc[b], ref["k_new"][b, 0], rtol=1e-2, atol=2e-2)
     tri, bi = otree.tables_from_rows(rows)
-    tref = parity.oracle_tree_batch(ids_g, sl_g, inp["ctx_tail"].numpy(), tri, bi, beam=w.beam, budget=w.tree_budget)
-    parity.assert_tree_equal(tree_g, tref)
+    ctx = inp["ctx_tail"].numpy()
+    for b in range(w.batch):   # every sequence's tree starts at its own last fresh row
+        fr = max(int(counts[b]), 1) - 1
+        t = otree.build_tree(ids_g[b, fr:], sl_g[b, fr:], (int(ctx[b, 0]), int(ctx[b, 1])), tri, bi, beam=w.beam, budget=w.tree_budget)
+        for key in ("n_nodes", "tokens", "parents", "depth", "mask"):
+            assert np.array_equal(tree_g[key][b], np.asarray(t[key])), (b, key)
+        assert np.array_equal(tree_g["scores"][b].view(np.uint32), np.asarray(t["scores"], dtype=np.float32).view(np.uint32))
     print(f"{name}: logits max-abs {stats['max_abs']:.3e} rel-L2 {stats['rel_l2']:.3e} s_logit max-abs {worst:.3e}")
     return stats
 
@@ -73,3 +79,12 @@ def test_c4_qwen3_32b_batch4_full_parity():
 
 def test_c5_ragged_batch16_temperature1_full_parity():
     _full_case("C5")
+
+
+def test_c5_per_sequence_fresh_counts_full_parity():
+    """The steady-state call: every sequence brings its own number of fresh rows (1..K)."""
+    _full_case("C5", ragged_fresh=True)
+
+
+def test_c3_four_fresh_rows_full_parity():
+    _full_case("C3", ragged_fresh=True)

@@ -143,3 +143,48 @@ def test_packed_io_moves_a_step_with_one_copy_each_way():
     for n, t in ref.items():
         assert torch.equal(hv["out_" + n], t.cpu()), n
     ses.close()
+
+
+@pytest.mark.parametrize("name,counts", [("ragged_b2", [2, 1]), ("b3_k4_pad32", [0, 4, 3]), ("hot_b4", [1, 3, 0, 2]),
+                                          ("b16_k8_pad128", [1, 8, 2, 0, 5, 1, 1, 3, 7, 2, 4, 1, 6, 0, 1, 2])])
+def test_per_sequence_fresh_counts_match_oracle(name, counts):
+    """The steady-state call after a verification that accepted a different number of tokens per sequence:
+    packed fresh rows, per-sequence cache append, and trees that start at each sequence's own last fresh row."""
+    w = CASES[name]
+    wt = syn.make_weights(w)
+    inp = syn.make_step_inputs(w, n_fresh=counts)
+    rows = syn.make_ngram_rows(w.vocab, min(w.ngram_rows, 20000), w.ngram_mode)
+    ses = runner.DraftSession(w, wt, rows, want_logits=True, philox_seed=parity.PHILOX_SEED)
+    ses.load_inputs(inp)
+    ses.step(step_counter=5)
+    ses.tree()
+    torch.cuda.synchronize()
+    assert ses.draft.device_status() == 0
+    ref = parity.oracle_forward(w, wt, inp)
+    parity.check_logits(ses.logits.cpu().numpy(), ref["logits"])
+    ids_g, sl_g = ses.topk_ids.cpu().numpy(), ses.topk_slogit.cpu().numpy()
+    for b in range(w.batch):
+        for r in range(w.K):
+            noise = ofw.gumbel_noise(w.vocab, r, b, 5, parity.PHILOX_SEED) if w.temperature > 0 else None
+            parity.check_topk_row(ids_g[b, r], sl_g[b, r], ref["logits"][b, r], w.topk, 1e-10, w.temperature, noise)
+    # the call appends exactly the fresh positions of every sequence
+    kc, vc = ses.inp["k_cache"].float().cpu().numpy(), ses.inp["v_cache"].float().cpu().numpy()
+    k0, v0 = inp["k_cache"].float().numpy(), inp["v_cache"].float().numpy()
+    for b in range(w.batch):
+        P = int(inp["seq_lens"][b])
+        for r in range(counts[b]):
+            np.testing.assert_allclose(kc[b, :, P + r], ref["k_new"][b, r], rtol=1e-2, atol=2e-2)
+            np.testing.assert_allclose(vc[b, :, P + r], ref["v_new"][b, r], rtol=1e-2, atol=2e-2)
+        keep = np.ones(kc.shape[2], dtype=bool)
+        keep[P:P + counts[b]] = False
+        assert np.array_equal(kc[b][:, keep], k0[b][:, keep]) and np.array_equal(vc[b][:, keep], v0[b][:, keep])
+    # every sequence's tree starts at its own last fresh row and is bit-exact from the GPU's candidates
+    tri, bi = otree.tables_from_rows(rows)
+    got = ses.tree_outputs()
+    ctx = inp["ctx_tail"].numpy()
+    for b in range(w.batch):
+        fr = max(counts[b], 1) - 1
+        t = otree.build_tree(ids_g[b, fr:], sl_g[b, fr:], (int(ctx[b, 0]), int(ctx[b, 1])), tri, bi, beam=w.beam, budget=w.tree_budget)
+        for key in ("n_nodes", "tokens", "parents", "depth", "mask"):
+            assert np.array_equal(got[key][b], np.asarray(t[key])), (b, key)
+    ses.close()
