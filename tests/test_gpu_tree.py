@@ -129,5 +129,19 @@ def test_argument_and_capacity_errors():
     with pytest.raises(binding.DartError) as e:
         ses.step()
     assert e.value.status == binding.DART_ERR_INVALID_ARG
+    # per-sequence counts: one out of range, one that overflows its sequence's cache
+    ses.inp["n_fresh"] = [1] * (w.batch - 1) + [w.K + 1]
+    with pytest.raises(binding.DartError) as e:
+        ses.step()
+    assert e.value.status == binding.DART_ERR_INVALID_ARG
+    ses.inp["n_fresh"] = [1] * w.batch
+    ses.inp["seq_lens_host"] = ses.inp["seq_lens_host"].copy()
+    ses.inp["seq_lens_host"][-1] = w.max_prefix
+    with pytest.raises(binding.DartError) as e:
+        ses.step()
+    assert e.value.status == binding.DART_ERR_CAPACITY
+    with pytest.raises(binding.DartError) as e:
+        ses.draft.build_tree(batch=2, first_row=[0, w.K], **kw)
+    assert e.value.status == binding.DART_ERR_INVALID_ARG
     torch.cuda.synchronize()
     ses.close()
