@@ -171,6 +171,25 @@ def draft_forward(cfg: Dict, w: Dict[str, np.ndarray], inp: Dict[str, np.ndarray
     return out
 
 
+def prefill_kv(cfg: Dict, w: Dict[str, np.ndarray], feats: np.ndarray, tokens: np.ndarray, positions: np.ndarray):
+    """Keys and values of the draft layer for new prefix rows (Section 3.2: the layer attends over its own KV
+    cache of the prefix).  A single layer's k and v depend on the layer's input alone, so no attention is needed:
+    row i with target features feats[i] (bf16 bits [n, 3h]), next-token id tokens[i] and absolute position
+    positions[i] gives z = [RMSNorm(W_fc f) ; RMSNorm(E[token])], k = RoPE(W_k z, position), v = W_v z.
+    Returns k, v as fp64 [n, Hkv, dh]."""
+    h, Hkv, dh = cfg["hidden"], cfg["n_kv_heads"], cfg["head_dim"]
+    theta, eps = float(cfg["rope_theta"]), float(cfg["rms_eps"])
+    g = linear(bf16_to_f64(feats).reshape(-1, 3 * h), w["w_fc"])
+    e = bf16_to_f64(w["embed"][np.asarray(tokens).astype(np.int64).reshape(-1)])
+    z = np.concatenate([rmsnorm(g, bf16_to_f64(w["norm_g"]), eps), rmsnorm(e, bf16_to_f64(w["norm_e"]), eps)], axis=-1)
+    n = z.shape[0]
+    k = linear(z, w["w_k"]).reshape(n, Hkv, dh)
+    v = linear(z, w["w_v"]).reshape(n, Hkv, dh)
+    pos = np.asarray(positions).astype(np.int64)
+    k = rope(k.transpose(1, 0, 2), pos, theta).transpose(1, 0, 2)
+    return k, v
+
+
 def log_softmax(y: np.ndarray) -> np.ndarray:
     mx = y.max(axis=-1, keepdims=True)
     return y - (mx + np.log(np.sum(np.exp(y - mx), axis=-1, keepdims=True)))

@@ -286,3 +286,20 @@ def test_per_sequence_fresh_counts_equal_each_sequence_run_alone():
         np.testing.assert_array_equal(got["k_new"][b], ref["k_new"][0])
     # the counts matter: a fresh row and a <mask> row at the same place give different logits
     assert np.abs(got["logits"][0, 1] - got["logits"][1, 1]).max() > 1e-3
+
+
+def test_prefill_keys_and_values_are_the_forward_pass_s_new_rows():
+    """Draft-side prefill: the k, v it stores for a run of new rows are exactly the new rows' k, v of a forward
+    pass in which all those rows are fresh (the forward pass being pinned above)."""
+    w = syn.small_variant(TINY, K=6, n_fresh=6, prefix=9)
+    wt = _np_weights(syn.make_weights(w))
+    inp = _np_inputs(syn.make_step_inputs(w))
+    cfg = _cfg(w)
+    fwd = ofw.draft_forward(cfg, wt, inp)
+    P = int(inp["seq_lens"][0])
+    k, v = ofw.prefill_kv(cfg, wt, inp["feats"][0], inp["tokens"][0], P + np.arange(6))
+    np.testing.assert_allclose(k, fwd["k_new"][0], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(v, fwd["v_new"][0], rtol=1e-12, atol=1e-13)
+    # positions matter for k (RoPE) and not for v
+    k2, v2 = ofw.prefill_kv(cfg, wt, inp["feats"][0], inp["tokens"][0], P + 1 + np.arange(6))
+    assert np.abs(k2 - k).max() > 1e-3 and np.array_equal(v2, v)
