@@ -297,6 +297,61 @@ def run_ours(args):
     replicas.finish(world)
 
 
+def run_prefill(args):
+    """Draft-side prefill (dart_draft_prefill): time to build the draft layer's KV cache for --prefill-rows new
+    prefix rows of one sequence.  The work is two dense projections per row (feature FC and k/v), so its bound is
+    the tensor pipe: 2 * rows * (3h*h + 2h*2*Hkv*dh) flop against the measured bf16 peak."""
+    import torch
+    from paper_2601_19278_b200 import replicas, runner, synthetic as syn
+    world, rank, local = replicas.env()
+    torch.cuda.set_device(local)
+    w = syn.WORKLOADS[args.workload]
+    n = args.prefill_rows
+    assert 0 < n <= w.prefix, "the rows must fit the workload's cache"
+    wt = syn.make_weights(w)
+    inp = syn.make_step_inputs(w)
+    inp["seq_lens"] = torch.zeros(w.batch, dtype=torch.int32)
+    ses = runner.DraftSession(w, wt, None, device=f"cuda:{local}")
+    ses.load_inputs(inp)
+    g = torch.Generator().manual_seed(5)
+    feats = torch.randn(n, 3 * w.hidden, generator=g).to(torch.bfloat16).to(ses.dev)
+    tokens = torch.randint(0, w.vocab, (n,), generator=g, dtype=torch.int32).to(ses.dev)
+    counts = [n] + [0] * (w.batch - 1)
+    stream = torch.cuda.current_stream()
+    for _ in range(max(args.warmup, 3)):
+        ses.prefill(feats, tokens, counts)
+    torch.cuda.synchronize()
+    steps = min(args.steps, 20)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        ses.prefill(feats, tokens, counts)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    assert ses.draft.device_status() == 0
+    ms = e0.elapsed_time(e1) / steps
+    flop = 2.0 * n * (3 * w.hidden * w.hidden + 2 * w.hidden * 2 * w.n_kv_heads * w.head_dim)
+    peak = 1590.0
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    kind = "fallback"
+    if os.path.exists(pk):
+        d = json.load(open(pk))
+        if "bf16_tflops" in d:
+            peak, kind = float(d["bf16_tflops"]), "measured"
+    if rank == 0:
+        print(json.dumps({
+            "metric": "draft_prefill_rows_per_second", "value": n / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1, "steps": steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{w.name}: draft-side prefill of {n} rows of one sequence (hidden {w.hidden}, {w.n_kv_heads} kv heads x {w.head_dim})"},
+            "roofline": {"bound": "tensor", "achieved": flop / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                         "frac": flop / (ms * 1e-3) / 1e12 / peak, "peak_kind": f"of {kind}", "traffic": None,
+                         "note": "first build: the step's streaming kernels run once per 128 rows, so the weights are re-read "
+                                 "for every run of rows; a tile-resident dense GEMM is the next step"},
+        }))
+    ses.close()
+
+
 def cpu_baseline(w, wt, inp, rows):
     """The oracle timed on this machine's host cores on one full step of the same workload."""
     import torch
@@ -336,6 +391,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--vocab", type=int, default=0,
                     help="override the workload's vocabulary (a smaller case of the same kernels, for ncu captures)")
+    ap.add_argument("--prefill-rows", type=int, default=0,
+                    help="time dart_draft_prefill on this many new prefix rows instead of the drafting step")
     ap.add_argument("--ragged-fresh", action="store_true",
                     help="per-sequence fresh-row counts (a steady-state call after a verification that accepted a different "
                          "number of tokens per sequence) instead of the workload's uniform count")
@@ -344,7 +401,9 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.prefill_rows > 0 and args.impl == "ours":
+        run_prefill(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -224,6 +224,28 @@ size_t dart_workspace_bytes(const dart_config* cfg);
 int dart_step_launch_count(const dart_handle* h, int batch, int n_fresh);
 
 /*
+ * Draft-side prefill (Section 3.2: the draft layer attends over its own KV cache of the prefix, which has to
+ * exist before the first drafting step).  A single layer's keys and values depend on nothing but the layer's
+ * input, so building the cache for new prefix positions needs no attention: for every new row the call
+ * computes z = [RMSNorm(W_fc f) ; RMSNorm(E[token])], k = RoPE(W_k z) and v = W_v z at the row's absolute
+ * position and stores them.  Sequence b gets new_rows_host[b] rows at positions seq_lens_host[b] ..; their
+ * features and next-token ids are packed in sequence order.  The caller then advances its sequence lengths and
+ * runs dart_draft_step as usual (whose own fresh rows are appended by that call).  No logits are produced.
+ * Asynchronous on `cuda_stream`; rows are processed in runs of up to 128 per pair of kernel launches.
+ * Errors: INVALID_ARG, CAPACITY (batch > max_batch or seq_lens_host[b] + new_rows_host[b] > max_prefix).
+ */
+typedef struct dart_prefill_in {
+  int32_t batch;                  /* B <= max_batch */
+  const void* feats;              /* DEVICE bf16 [sum N_b, feat_in], 32-byte aligned */
+  const int32_t* tokens;          /* DEVICE i32  [sum N_b] id of the token that follows each row */
+  const int32_t* seq_lens_host;   /* HOST i32 [B] rows already in the cache */
+  const int32_t* new_rows_host;   /* HOST i32 [B] N_b >= 0 rows to add */
+  void* k_cache;                  /* DEVICE bf16 [max_batch, H_kv, max_prefix, d_h]; rows P_b .. P_b+N_b-1 are written */
+  void* v_cache;                  /* DEVICE bf16, same layout */
+} dart_prefill_in;
+int dart_draft_prefill(dart_handle* h, const dart_prefill_in* in, void* cuda_stream);
+
+/*
  * Measurement aid (the paper has no counterpart): the next dart_draft_step (stages 0..7) or
  * dart_build_tree (stage 8) records the caller-owned CUDA events `start_event` / `stop_event`
  * (cudaEvent_t handles) on the stream immediately before and after the kernels of `stage`,

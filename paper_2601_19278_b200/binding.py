@@ -26,7 +26,7 @@ DART_ERR_INTERNAL = -6
 
 EXPORTS = [
     "dart_draft_init", "dart_draft_step", "dart_build_tree", "dart_draft_destroy", "dart_last_device_status",
-    "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_step_launch_count",
+    "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_step_launch_count", "dart_draft_prefill",
     "dart_set_profile_events", "dart_topk_rows_noalloc",
 ]
 
@@ -60,6 +60,11 @@ class DartStepIn(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_fresh", C.c_int32), ("feats", C.c_void_p), ("tokens", C.c_void_p),
                 ("seq_lens", C.c_void_p), ("seq_lens_host", C.c_void_p), ("k_cache", C.c_void_p),
                 ("v_cache", C.c_void_p), ("step_counter", C.c_uint64), ("fresh_counts_host", C.c_void_p)]
+
+
+class DartPrefillIn(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("feats", C.c_void_p), ("tokens", C.c_void_p), ("seq_lens_host", C.c_void_p),
+                ("new_rows_host", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p)]
 
 
 class DartStepOut(C.Structure):
@@ -104,6 +109,8 @@ def lib() -> C.CDLL:
         L.dart_status_string.restype = C.c_char_p
         L.dart_workspace_bytes.argtypes = [C.POINTER(DartConfig)]
         L.dart_workspace_bytes.restype = C.c_size_t
+        L.dart_draft_prefill.argtypes = [C.c_void_p, C.POINTER(DartPrefillIn), C.c_void_p]
+        L.dart_draft_prefill.restype = C.c_int
         L.dart_step_launch_count.argtypes = [C.c_void_p, C.c_int, C.c_int]
         L.dart_step_launch_count.restype = C.c_int
         L.dart_set_profile_events.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
@@ -190,6 +197,15 @@ class DartDraft:
         rc = lib().dart_draft_step(self._h, C.byref(sin), C.byref(sout), self._stream(stream))
         if rc != DART_OK:
             raise DartError(rc, "dart_draft_step", lib().dart_last_cuda_error(self._h))
+
+    def prefill(self, *, feats, tokens, seq_lens_host, new_rows_host, k_cache, v_cache, stream=None) -> None:
+        """dart_draft_prefill: append the k, v of new prefix rows (packed features / next-token ids) to the caches."""
+        slh = np.ascontiguousarray(seq_lens_host, dtype=np.int32)
+        nrh = np.ascontiguousarray(new_rows_host, dtype=np.int32)
+        pin = DartPrefillIn(len(slh), _ptr(feats), _ptr(tokens), slh.ctypes.data, nrh.ctypes.data, _ptr(k_cache), _ptr(v_cache))
+        rc = lib().dart_draft_prefill(self._h, C.byref(pin), self._stream(stream))
+        if rc != DART_OK:
+            raise DartError(rc, "dart_draft_prefill", lib().dart_last_cuda_error(self._h))
 
     def build_tree(self, *, batch: int, topk_ids, topk_slogit, ctx_tail, tokens, parents, depth, mask, n_nodes,
                    scores=None, first_row=0, n_levels: Optional[int] = None, stream=None) -> None:

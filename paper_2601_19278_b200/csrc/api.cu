@@ -50,9 +50,10 @@ struct dart_handle {
   int device = 0;
   int n_sm = 0;
   int last_cuda_error = 0;
-  GemmPlan plan_fc, plan_qkv, plan_o, plan_gu, plan_down;
+  GemmPlan plan_fc, plan_qkv, plan_o, plan_gu, plan_down, plan_kv;
   bool umma = false;         // projections run on the tcgen05 / TMA kernels (tensor maps could be encoded)
-  UmmaMaps maps_fc, maps_qkv, maps_o, maps_gu, maps_down;
+  UmmaMaps maps_fc, maps_qkv, maps_o, maps_gu, maps_down, maps_kv;
+  int maps_kv_M = -1;        // token rows the prefill's activation maps were encoded for
   CUtensorMap map_lm;        // the LM head's weight matrix
   int lm_tag = 0;            // launch counter of the LM head (marks its cross-CTA pieces)
   int maps_M = -1;           // token rows the activation tensor maps were encoded for
@@ -216,10 +217,18 @@ struct Layout {
   }
 };
 
+// Token rows the workspace is sized for.
+int prefill_run_rows(const dart_config& c) { return 32 * c.K < 128 ? 32 * c.K : 128; }
+int token_rows_capacity(const dart_config& c) {
+  const int step = c.max_batch * c.K, pre = prefill_run_rows(c);
+  return step > pre ? step : pre;
+}
+
 // Sizes every workspace region; with base != nullptr also assigns the pointers.
 size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_pairs_cap, int lm_grid, char* base, Workspace* ws) {
   Layout L;
-  const size_t Mmax = (size_t)c.max_batch * c.K;
+  // token rows of a launch: a step has max_batch * K, a prefill run up to 128 (32 runs of K rows at most)
+  const size_t Mmax = (size_t)token_rows_capacity(c);
   const size_t MPmax = padded_tokens((int)Mmax);
   const size_t dq = (size_t)c.n_q_heads * c.head_dim;
   const size_t ht = (c.hidden + 127) / 128;
@@ -265,7 +274,7 @@ size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_p
 }
 
 struct PlanSet {
-  PlanHost fc, qkv, o, gu, down;
+  PlanHost fc, qkv, o, gu, down, kv;
   size_t part_max = 0;
 };
 
@@ -289,6 +298,9 @@ void build_plans(const dart_config& c, const dart_weights* w, int n_sm, bool umm
   s[4] = {W(w ? w->w_k : nullptr, h), dkv, 0, 2 * h, h};
   s[5] = {W(w ? w->w_v : nullptr, h), dkv, 0, 2 * h, h};
   make_plan_host(ps.qkv, s, 6, h, grid, qt + 2 * kt);
+  // the prefill's projection: k and v only (g-half and e-half columns paired as above)
+  GemmSeg skv[4] = {s[1], s[2], s[4], s[5]};
+  make_plan_host(ps.kv, skv, 4, h, grid, 2 * kt);
   s[0] = {W(w ? w->w_o : nullptr, 0), h, 0, dq, 0};
   make_plan_host(ps.o, s, 1, dq, grid, 0);
   s[0] = {W(w ? w->w_gate : nullptr, 0), c.mlp_inter, 0, h, 0};
@@ -296,10 +308,10 @@ void build_plans(const dart_config& c, const dart_weights* w, int n_sm, bool umm
   make_plan_host(ps.gu, s, 2, h, grid, (c.mlp_inter + 127) / 128);
   s[0] = {W(w ? w->w_down : nullptr, 0), h, 0, c.mlp_inter, 0};
   make_plan_host(ps.down, s, 1, c.mlp_inter, grid, 0);
-  const int MPmax = padded_tokens(c.max_batch * c.K);
-  const PlanHost* all[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
+  const int MPmax = padded_tokens(token_rows_capacity(c));
+  const PlanHost* all[6] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down, &ps.kv};
   ps.part_max = 0;
-  for (int i = 0; i < 5; ++i) {
+  for (int i = 0; i < 6; ++i) {
     const size_t f = part_floats(all[i]->plan, MPmax);
     if (f > ps.part_max) ps.part_max = f;
   }
@@ -408,23 +420,24 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
 #endif
   PlanSet ps;
   build_plans(*cfg, weights, n_sm, h->umma, ps);
-  PlanHost* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
+  PlanHost* plans[6] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down, &ps.kv};
   if (h->umma) {
     INIT_CHECK(tmap_encode_bf16(&h->map_lm, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 128));
-    UmmaMaps* maps[5] = {&h->maps_fc, &h->maps_qkv, &h->maps_o, &h->maps_gu, &h->maps_down};
-    for (int i = 0; i < 5; ++i) {
+    UmmaMaps* maps[6] = {&h->maps_fc, &h->maps_qkv, &h->maps_o, &h->maps_gu, &h->maps_down, &h->maps_kv};
+    for (int i = 0; i < 6; ++i) {
       const GemmPlan& pl = plans[i]->plan;
       for (int sg = 0; sg < pl.nseg; ++sg)
         INIT_CHECK(tmap_encode_bf16(&maps[i]->W[sg], pl.seg[sg].W, pl.Kd, pl.seg[sg].rows, (unsigned long long)pl.seg[sg].ld * 2, 64, 128));
     }
   }
-  for (int i = 0; i < 5; ++i) {
+  for (int i = 0; i < 6; ++i) {
     PlanHost& ph = *plans[i];
     INIT_CHECK(upload(h, ph.expected, &ph.plan.d_expected));
     INIT_CHECK(upload(h, ph.meta, &ph.plan.d_meta));
     std::vector<int> zeros(ph.plan.n_groups, 0);
     INIT_CHECK(upload(h, zeros, &ph.plan.d_ctr));
   }
+  h->plan_kv = ps.kv.plan;
   h->plan_fc = ps.fc.plan; h->plan_qkv = ps.qkv.plan; h->plan_o = ps.o.plan; h->plan_gu = ps.gu.plan; h->plan_down = ps.down.plan;
   h->lm_grid = 2 * n_sm;
   if (h->lm_grid > cfg->vocab / 16) h->lm_grid = cfg->vocab / 16;
@@ -688,6 +701,97 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   if ((e = launch_topk_merge(lp, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(7, false);
   if (h->prof_stage >= 0 && h->prof_stage <= 7) h->prof_stage = -1;
+  return DART_OK;
+}
+
+int dart_draft_prefill(dart_handle* h, const dart_prefill_in* in, void* cuda_stream) {
+  if (h == nullptr || in == nullptr) return DART_ERR_INVALID_ARG;
+  const dart_config& c = h->cfg;
+  const int B = in->batch, K = c.K, hdim = c.hidden;
+  if (B < 1) return DART_ERR_INVALID_ARG;
+  if (B > c.max_batch) return DART_ERR_CAPACITY;
+  if (in->seq_lens_host == nullptr || in->new_rows_host == nullptr || !aligned16(in->k_cache) || !aligned16(in->v_cache))
+    return DART_ERR_INVALID_ARG;
+  if (c.feat_in <= 0) return DART_ERR_INVALID_ARG;
+  long long total = 0;
+  for (int b = 0; b < B; ++b) {
+    const int P = in->seq_lens_host[b], N = in->new_rows_host[b];
+    if (P < 0 || N < 0) return DART_ERR_INVALID_ARG;
+    if ((long long)P + N > c.max_prefix) return DART_ERR_CAPACITY;
+    total += N;
+  }
+  if (total == 0) return DART_OK;
+  if (!aligned32(in->feats) || in->tokens == nullptr) return DART_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  Workspace& ws = h->ws;
+  const int run_rows = prefill_run_rows(c), max_runs = run_rows / K;   // runs * K token rows per launch pair, at most 128
+  const bf16* feats = static_cast<const bf16*>(in->feats);
+  cudaError_t e;
+  int b = 0, done_b = 0;      // next sequence with rows left, rows of it already taken
+  long long done = 0;         // packed rows already processed
+  while (done < total) {
+    // one launch pair covers up to max_runs runs of at most K consecutive rows each, taken in packed order (a run
+    // shorter than K still occupies K token rows of the launch, so the runs, not the rows, bound a launch)
+    EpiArgs ep;
+    memset(&ep, 0, sizeof(ep));
+    FreshOffsets fo;
+    int runs = 0, rows = 0;
+    fo.v[0] = 0;
+    while (b < B && runs < max_runs && rows < run_rows) {
+      const int left = in->new_rows_host[b] - done_b;
+      if (left == 0) { ++b; done_b = 0; continue; }
+      int take = left < K ? left : K;
+      if (take > run_rows - rows) take = run_rows - rows;
+      ep.pos0[runs] = in->seq_lens_host[b] + done_b;
+      ep.slab[runs] = (unsigned char)b;
+      fo.v[runs + 1] = fo.v[runs] + take;
+      ++runs; rows += take; done_b += take;
+    }
+    for (int i = runs + 1; i < 33; ++i) fo.v[i] = fo.v[runs];
+    const int M = runs * K, MP = padded_tokens(M);
+    // <mask> rows pad the runs that are shorter than K (their k, v are not stored)
+    if ((e = launch_fill_mask_rows(ws.z_hi, ws.z_lo, ws.zmask_hi, ws.zmask_lo, runs, K, fo, 2 * hdim, st)) != cudaSuccess) return fail_cuda(h, e);
+    h->z_B = -1;   // the next step rewrites its own <mask> rows
+    ep.K = K; ep.h = hdim; ep.eps = c.rms_eps; ep.B = runs;
+    memcpy(ep.foff, fo.v, sizeof(ep.foff));
+    EpiArgs kv = ep;   // (run bookkeeping shared by both launches)
+    // feature FC on the new rows: g, z g-half, sums of squares; prologue: z e-half from the next tokens' embeddings
+    ep.mode = EPI_FC;
+    ep.res0 = ws.res0; ep.gamma = static_cast<const bf16*>(h->w.norm_g);
+    ep.out_hi = ws.z_hi; ep.out_lo = ws.z_lo; ep.ld_out = 2 * hdim; ep.ss_out = ws.ss_g;
+    ep.tokens = in->tokens + done; ep.vocab = c.vocab; ep.embed = static_cast<const bf16*>(h->w.embed);
+    ep.gamma_e = static_cast<const bf16*>(h->w.norm_e);
+    GemmInput gi = {feats + (size_t)done * c.feat_in, nullptr, c.feat_in, rows};
+    if (h->umma) {
+      if ((e = tmap_encode_bf16(&h->maps_fc.Xhi, gi.x_hi, c.feat_in, rows, (unsigned long long)c.feat_in * 2, 64, 2 * padded_tokens(rows))) != cudaSuccess)
+        return fail_cuda(h, e);
+      h->maps_fc.Xlo = h->maps_fc.Xhi;
+      h->maps_feats = nullptr; h->maps_fc_M = -1;   // the step re-encodes its own
+      e = launch_umma_rows(h->plan_fc, h->maps_fc, gi, ep, ws.part, ws.status, st);
+    } else {
+      e = launch_gemm_rows(h->plan_fc, gi, ep, ws.part, st);
+    }
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    // k, v projections of the runs' rows with RoPE at their positions, stored straight into the cache
+    kv.mode = EPI_QKV; kv.prefill = 1; kv.kind0 = 1;
+    kv.ss_in = ws.ss_g; kv.ss_tiles = h->h_tiles; kv.ss_mp = padded_tokens(rows); kv.rstd_mask = ws.rstd_mask;
+    kv.Hq = c.n_q_heads; kv.Hkv = c.n_kv_heads; kv.dh = c.head_dim; kv.rope_tab = ws.rope_tab;
+    kv.k_cache = static_cast<bf16*>(in->k_cache); kv.v_cache = static_cast<bf16*>(in->v_cache); kv.P_cap = c.max_prefix;
+    gi = {ws.z_hi, ws.z_lo, 2 * hdim, M};
+    if (h->umma) {
+      if (h->maps_kv_M != M) {
+        if ((e = tmap_encode_bf16(&h->maps_kv.Xhi, ws.z_hi, 2 * hdim, M, (unsigned long long)hdim * 4, 64, MP)) != cudaSuccess ||
+            (e = tmap_encode_bf16(&h->maps_kv.Xlo, ws.z_lo, 2 * hdim, M, (unsigned long long)hdim * 4, 64, MP)) != cudaSuccess)
+          return fail_cuda(h, e);
+        h->maps_kv_M = M;
+      }
+      e = launch_umma_rows(h->plan_kv, h->maps_kv, gi, kv, ws.part, ws.status, st);
+    } else {
+      e = launch_gemm_rows(h->plan_kv, gi, kv, ws.part, st);
+    }
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    done += rows;
+  }
   return DART_OK;
 }
 

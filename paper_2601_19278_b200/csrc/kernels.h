@@ -108,6 +108,10 @@ struct EpiArgs {
   // EPI_QKV
   int Hq, Hkv, dh; const int32_t* seq_lens; const float2* rope_tab;  // [positions][dh/2] (cos, sin)
   bf16* q_hi; bf16* q_lo; bf16* k_new; bf16* v_new; bf16* k_cache; bf16* v_cache; long long P_cap;
+  // Draft-side prefill (dart_draft_prefill): the launch covers up to 32 runs of at most K consecutive new rows;
+  // run b holds rows pos0[b] .. of cache slab slab[b]; only k and v are projected (segment s is kind s + kind0:
+  // 0 = q, 1 = k, 2 = v) and nothing but the cache is written.
+  int prefill, kind0; int pos0[32]; unsigned char slab[32];
 };
 
 // What the shared streaming core (stream_core.cuh) needs to know about a launch.

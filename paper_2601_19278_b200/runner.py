@@ -88,6 +88,13 @@ class DraftSession:
                               v_cache=i["v_cache"], n_fresh=i["n_fresh"], topk_ids=self.topk_ids,
                               topk_slogit=self.topk_slogit, logits=self.logits, step_counter=step_counter, stream=stream)
 
+    def prefill(self, feats: torch.Tensor, tokens: torch.Tensor, new_rows, stream=None) -> None:
+        """dart_draft_prefill on this session's caches: new_rows[b] rows are appended after the current lengths,
+        which the caller then advances (self.inp["seq_lens"], self.inp["seq_lens_host"])."""
+        self.draft.prefill(feats=feats.to(self.dev), tokens=tokens.to(self.dev), seq_lens_host=self.inp["seq_lens_host"],
+                           new_rows_host=np.asarray(new_rows, dtype=np.int32), k_cache=self.inp["k_cache"],
+                           v_cache=self.inp["v_cache"], stream=stream)
+
     def tree(self, stream=None, topk_ids=None, topk_slogit=None, ctx_tail=None, first_row: Optional[int] = None) -> None:
         nf = self.inp["n_fresh"]
         if first_row is not None:
