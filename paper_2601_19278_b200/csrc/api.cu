@@ -38,6 +38,8 @@ struct Workspace {
   float *lm_stats = nullptr, *lm_key = nullptr, *lm_y = nullptr;
   int32_t* lm_id = nullptr;
   int* status = nullptr;
+  bf16* pz = nullptr;           // prefill: z of one pass [kPrefillPassRows, 2h] bf16
+  float* pss = nullptr;         // prefill: per-row partial sums of squares of g [kPrefillPassRows, h/256]
   float* lm_pieces = nullptr;   // [SMs][128][MPmax] partial logits of vocabulary tiles cut between CTAs
   int* lm_flags = nullptr;      // [SMs] launch tag of each CTA's piece
 };
@@ -50,10 +52,10 @@ struct dart_handle {
   int device = 0;
   int n_sm = 0;
   int last_cuda_error = 0;
-  GemmPlan plan_fc, plan_qkv, plan_o, plan_gu, plan_down, plan_kv;
+  GemmPlan plan_fc, plan_qkv, plan_o, plan_gu, plan_down;
   bool umma = false;         // projections run on the tcgen05 / TMA kernels (tensor maps could be encoded)
-  UmmaMaps maps_fc, maps_qkv, maps_o, maps_gu, maps_down, maps_kv;
-  int maps_kv_M = -1;        // token rows the prefill's activation maps were encoded for
+  UmmaMaps maps_fc, maps_qkv, maps_o, maps_gu, maps_down;
+  CUtensorMap pmap_fc, pmap_kv[4];   // prefill: W_fc, and the g-/e-half columns of W_k and W_v (boxes of 256 rows)
   CUtensorMap map_lm;        // the LM head's weight matrix
   int lm_tag = 0;            // launch counter of the LM head (marks its cross-CTA pieces)
   int maps_M = -1;           // token rows the activation tensor maps were encoded for
@@ -218,16 +220,14 @@ struct Layout {
 };
 
 // Token rows the workspace is sized for.
-int prefill_run_rows(const dart_config& c) { return 32 * c.K < 128 ? 32 * c.K : 128; }
-int token_rows_capacity(const dart_config& c) {
-  const int step = c.max_batch * c.K, pre = prefill_run_rows(c);
-  return step > pre ? step : pre;
-}
+int token_rows_capacity(const dart_config& c) { return c.max_batch * c.K; }
+// Rows one pass of the draft-side prefill handles (its z and sums-of-squares buffers are sized for this).
+constexpr int kPrefillPassRows = 4096;
+int prefill_fc_tiles(const dart_config& c) { return (c.hidden + 255) / 256; }
 
 // Sizes every workspace region; with base != nullptr also assigns the pointers.
 size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_pairs_cap, int lm_grid, char* base, Workspace* ws) {
   Layout L;
-  // token rows of a launch: a step has max_batch * K, a prefill run up to 128 (32 runs of K rows at most)
   const size_t Mmax = (size_t)token_rows_capacity(c);
   const size_t MPmax = padded_tokens((int)Mmax);
   const size_t dq = (size_t)c.n_q_heads * c.head_dim;
@@ -269,12 +269,16 @@ size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_p
   TAKE(lm_y, float*, (size_t)lm_grid * MPmax * 32 * sizeof(float));
   TAKE(lm_id, int32_t*, (size_t)lm_grid * MPmax * 32 * sizeof(int32_t));
   TAKE(status, int*, 256);
+  if (c.feat_in > 0) {
+    TAKE(pz, bf16*, (size_t)kPrefillPassRows * 2 * c.hidden * sizeof(bf16));
+    TAKE(pss, float*, (size_t)kPrefillPassRows * prefill_fc_tiles(c) * sizeof(float));
+  }
 #undef TAKE
   return L.total;
 }
 
 struct PlanSet {
-  PlanHost fc, qkv, o, gu, down, kv;
+  PlanHost fc, qkv, o, gu, down;
   size_t part_max = 0;
 };
 
@@ -298,9 +302,6 @@ void build_plans(const dart_config& c, const dart_weights* w, int n_sm, bool umm
   s[4] = {W(w ? w->w_k : nullptr, h), dkv, 0, 2 * h, h};
   s[5] = {W(w ? w->w_v : nullptr, h), dkv, 0, 2 * h, h};
   make_plan_host(ps.qkv, s, 6, h, grid, qt + 2 * kt);
-  // the prefill's projection: k and v only (g-half and e-half columns paired as above)
-  GemmSeg skv[4] = {s[1], s[2], s[4], s[5]};
-  make_plan_host(ps.kv, skv, 4, h, grid, 2 * kt);
   s[0] = {W(w ? w->w_o : nullptr, 0), h, 0, dq, 0};
   make_plan_host(ps.o, s, 1, dq, grid, 0);
   s[0] = {W(w ? w->w_gate : nullptr, 0), c.mlp_inter, 0, h, 0};
@@ -309,9 +310,9 @@ void build_plans(const dart_config& c, const dart_weights* w, int n_sm, bool umm
   s[0] = {W(w ? w->w_down : nullptr, 0), h, 0, c.mlp_inter, 0};
   make_plan_host(ps.down, s, 1, c.mlp_inter, grid, 0);
   const int MPmax = padded_tokens(token_rows_capacity(c));
-  const PlanHost* all[6] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down, &ps.kv};
+  const PlanHost* all[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
   ps.part_max = 0;
-  for (int i = 0; i < 6; ++i) {
+  for (int i = 0; i < 5; ++i) {
     const size_t f = part_floats(all[i]->plan, MPmax);
     if (f > ps.part_max) ps.part_max = f;
   }
@@ -420,24 +421,33 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
 #endif
   PlanSet ps;
   build_plans(*cfg, weights, n_sm, h->umma, ps);
-  PlanHost* plans[6] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down, &ps.kv};
+  PlanHost* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
   if (h->umma) {
     INIT_CHECK(tmap_encode_bf16(&h->map_lm, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 128));
-    UmmaMaps* maps[6] = {&h->maps_fc, &h->maps_qkv, &h->maps_o, &h->maps_gu, &h->maps_down, &h->maps_kv};
-    for (int i = 0; i < 6; ++i) {
+    if (cfg->feat_in > 0) {
+      const unsigned long long hh = cfg->hidden, kvr = (unsigned long long)cfg->n_kv_heads * cfg->head_dim;
+      const bf16* wk = static_cast<const bf16*>(weights->w_k);
+      const bf16* wv = static_cast<const bf16*>(weights->w_v);
+      INIT_CHECK(tmap_encode_bf16(&h->pmap_fc, weights->w_fc, cfg->feat_in, hh, (unsigned long long)cfg->feat_in * 2, 64, 256));
+      INIT_CHECK(tmap_encode_bf16(&h->pmap_kv[0], wk, hh, kvr, hh * 4, 64, 256));
+      INIT_CHECK(tmap_encode_bf16(&h->pmap_kv[1], wk + hh, hh, kvr, hh * 4, 64, 256));
+      INIT_CHECK(tmap_encode_bf16(&h->pmap_kv[2], wv, hh, kvr, hh * 4, 64, 256));
+      INIT_CHECK(tmap_encode_bf16(&h->pmap_kv[3], wv + hh, hh, kvr, hh * 4, 64, 256));
+    }
+    UmmaMaps* maps[5] = {&h->maps_fc, &h->maps_qkv, &h->maps_o, &h->maps_gu, &h->maps_down};
+    for (int i = 0; i < 5; ++i) {
       const GemmPlan& pl = plans[i]->plan;
       for (int sg = 0; sg < pl.nseg; ++sg)
         INIT_CHECK(tmap_encode_bf16(&maps[i]->W[sg], pl.seg[sg].W, pl.Kd, pl.seg[sg].rows, (unsigned long long)pl.seg[sg].ld * 2, 64, 128));
     }
   }
-  for (int i = 0; i < 6; ++i) {
+  for (int i = 0; i < 5; ++i) {
     PlanHost& ph = *plans[i];
     INIT_CHECK(upload(h, ph.expected, &ph.plan.d_expected));
     INIT_CHECK(upload(h, ph.meta, &ph.plan.d_meta));
     std::vector<int> zeros(ph.plan.n_groups, 0);
     INIT_CHECK(upload(h, zeros, &ph.plan.d_ctr));
   }
-  h->plan_kv = ps.kv.plan;
   h->plan_fc = ps.fc.plan; h->plan_qkv = ps.qkv.plan; h->plan_o = ps.o.plan; h->plan_gu = ps.gu.plan; h->plan_down = ps.down.plan;
   h->lm_grid = 2 * n_sm;
   if (h->lm_grid > cfg->vocab / 16) h->lm_grid = cfg->vocab / 16;
@@ -722,75 +732,51 @@ int dart_draft_prefill(dart_handle* h, const dart_prefill_in* in, void* cuda_str
   }
   if (total == 0) return DART_OK;
   if (!aligned32(in->feats) || in->tokens == nullptr) return DART_ERR_INVALID_ARG;
+  if (!h->umma) return DART_ERR_UNSUPPORTED_ARCH;   // the dense kernels need the tensor-map encoder
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   Workspace& ws = h->ws;
-  const int run_rows = prefill_run_rows(c), max_runs = run_rows / K;   // runs * K token rows per launch pair, at most 128
   const bf16* feats = static_cast<const bf16*>(in->feats);
   cudaError_t e;
-  int b = 0, done_b = 0;      // next sequence with rows left, rows of it already taken
-  long long done = 0;         // packed rows already processed
-  while (done < total) {
-    // one launch pair covers up to max_runs runs of at most K consecutive rows each, taken in packed order (a run
-    // shorter than K still occupies K token rows of the launch, so the runs, not the rows, bound a launch)
-    EpiArgs ep;
-    memset(&ep, 0, sizeof(ep));
-    FreshOffsets fo;
-    int runs = 0, rows = 0;
-    fo.v[0] = 0;
-    while (b < B && runs < max_runs && rows < run_rows) {
-      const int left = in->new_rows_host[b] - done_b;
-      if (left == 0) { ++b; done_b = 0; continue; }
-      int take = left < K ? left : K;
-      if (take > run_rows - rows) take = run_rows - rows;
-      ep.pos0[runs] = in->seq_lens_host[b] + done_b;
-      ep.slab[runs] = (unsigned char)b;
-      fo.v[runs + 1] = fo.v[runs] + take;
-      ++runs; rows += take; done_b += take;
+  // passes of up to kPrefillPassRows packed rows: embeddings -> z e-half, feature FC -> z g-half, k / v -> caches
+  for (long long done = 0; done < total; done += kPrefillPassRows) {
+    const int T = (int)(total - done < kPrefillPassRows ? total - done : kPrefillPassRows);
+    DenseArgs a;
+    memset(&a, 0, sizeof(a));
+    a.T = T; a.h = hdim; a.eps = c.rms_eps; a.status = ws.status;
+    a.z = ws.pz; a.ldz = 2 * hdim; a.ss = ws.pss; a.ss_ld = prefill_fc_tiles(c); a.ss_n = prefill_fc_tiles(c);
+    // where the pass's rows go: sequence b contributes rows [lo, hi) of its new rows
+    a.B = B;
+    long long off = 0;
+    for (int b = 0; b < B; ++b) {
+      const long long lo = done > off ? done - off : 0;                       // first of b's new rows in this pass
+      long long hi = done + T - off;                                           // one past the last
+      if (hi > in->new_rows_host[b]) hi = in->new_rows_host[b];
+      if (hi < lo) hi = lo;
+      a.seq_off[b] = (int)(off + lo - done < 0 ? 0 : off + lo - done);
+      a.seq_P[b] = in->seq_lens_host[b] + (int)lo;
+      off += in->new_rows_host[b];
+      a.seq_off[b + 1] = (int)(a.seq_off[b] + (hi - lo));
     }
-    for (int i = runs + 1; i < 33; ++i) fo.v[i] = fo.v[runs];
-    const int M = runs * K, MP = padded_tokens(M);
-    // <mask> rows pad the runs that are shorter than K (their k, v are not stored)
-    if ((e = launch_fill_mask_rows(ws.z_hi, ws.z_lo, ws.zmask_hi, ws.zmask_lo, runs, K, fo, 2 * hdim, st)) != cudaSuccess) return fail_cuda(h, e);
-    h->z_B = -1;   // the next step rewrites its own <mask> rows
-    ep.K = K; ep.h = hdim; ep.eps = c.rms_eps; ep.B = runs;
-    memcpy(ep.foff, fo.v, sizeof(ep.foff));
-    EpiArgs kv = ep;   // (run bookkeeping shared by both launches)
-    // feature FC on the new rows: g, z g-half, sums of squares; prologue: z e-half from the next tokens' embeddings
-    ep.mode = EPI_FC;
-    ep.res0 = ws.res0; ep.gamma = static_cast<const bf16*>(h->w.norm_g);
-    ep.out_hi = ws.z_hi; ep.out_lo = ws.z_lo; ep.ld_out = 2 * hdim; ep.ss_out = ws.ss_g;
-    ep.tokens = in->tokens + done; ep.vocab = c.vocab; ep.embed = static_cast<const bf16*>(h->w.embed);
-    ep.gamma_e = static_cast<const bf16*>(h->w.norm_e);
-    GemmInput gi = {feats + (size_t)done * c.feat_in, nullptr, c.feat_in, rows};
-    if (h->umma) {
-      if ((e = tmap_encode_bf16(&h->maps_fc.Xhi, gi.x_hi, c.feat_in, rows, (unsigned long long)c.feat_in * 2, 64, 2 * padded_tokens(rows))) != cudaSuccess)
-        return fail_cuda(h, e);
-      h->maps_fc.Xlo = h->maps_fc.Xhi;
-      h->maps_feats = nullptr; h->maps_fc_M = -1;   // the step re-encodes its own
-      e = launch_umma_rows(h->plan_fc, h->maps_fc, gi, ep, ws.part, ws.status, st);
-    } else {
-      e = launch_gemm_rows(h->plan_fc, gi, ep, ws.part, st);
-    }
-    if (e != cudaSuccess) return fail_cuda(h, e);
-    // k, v projections of the runs' rows with RoPE at their positions, stored straight into the cache
-    kv.mode = EPI_QKV; kv.prefill = 1; kv.kind0 = 1;
-    kv.ss_in = ws.ss_g; kv.ss_tiles = h->h_tiles; kv.ss_mp = padded_tokens(rows); kv.rstd_mask = ws.rstd_mask;
-    kv.Hq = c.n_q_heads; kv.Hkv = c.n_kv_heads; kv.dh = c.head_dim; kv.rope_tab = ws.rope_tab;
+    for (int b = B + 1; b < 33; ++b) a.seq_off[b] = a.seq_off[B];
+    if ((e = launch_prefill_embed(in->tokens + done, T, c.vocab, static_cast<const bf16*>(h->w.embed),
+                                  static_cast<const bf16*>(h->w.norm_e), hdim, c.rms_eps, ws.pz, 2 * hdim, st)) != cudaSuccess)
+      return fail_cuda(h, e);
+    DenseArgs fc = a;
+    fc.mode = 0; fc.n_w = 1; fc.n_tiles_per_w = prefill_fc_tiles(c); fc.n_out = hdim;
+    fc.KB[0] = (c.feat_in + 63) / 64; fc.KB[1] = 0; fc.a_koff[0] = 0; fc.a_koff[1] = 0;
+    fc.gain = static_cast<const bf16*>(h->w.norm_g);
+    fc.mapW[0] = h->pmap_fc;
+    if ((e = tmap_encode_bf16(&fc.mapA, feats + (size_t)done * c.feat_in, c.feat_in, T, (unsigned long long)c.feat_in * 2, 64, 128)) != cudaSuccess)
+      return fail_cuda(h, e);
+    if ((e = launch_umma_dense(fc, h->n_sm, st)) != cudaSuccess) return fail_cuda(h, e);
+    DenseArgs kv = a;
+    kv.mode = 1; kv.n_w = 2; kv.n_tiles_per_w = (c.n_kv_heads * c.head_dim + 255) / 256; kv.n_out = c.n_kv_heads * c.head_dim;
+    kv.KB[0] = kv.KB[1] = (hdim + 63) / 64; kv.a_koff[0] = 0; kv.a_koff[1] = hdim;
+    kv.Hkv = c.n_kv_heads; kv.dh = c.head_dim; kv.rope_tab = ws.rope_tab;
     kv.k_cache = static_cast<bf16*>(in->k_cache); kv.v_cache = static_cast<bf16*>(in->v_cache); kv.P_cap = c.max_prefix;
-    gi = {ws.z_hi, ws.z_lo, 2 * hdim, M};
-    if (h->umma) {
-      if (h->maps_kv_M != M) {
-        if ((e = tmap_encode_bf16(&h->maps_kv.Xhi, ws.z_hi, 2 * hdim, M, (unsigned long long)hdim * 4, 64, MP)) != cudaSuccess ||
-            (e = tmap_encode_bf16(&h->maps_kv.Xlo, ws.z_lo, 2 * hdim, M, (unsigned long long)hdim * 4, 64, MP)) != cudaSuccess)
-          return fail_cuda(h, e);
-        h->maps_kv_M = M;
-      }
-      e = launch_umma_rows(h->plan_kv, h->maps_kv, gi, kv, ws.part, ws.status, st);
-    } else {
-      e = launch_gemm_rows(h->plan_kv, gi, kv, ws.part, st);
-    }
-    if (e != cudaSuccess) return fail_cuda(h, e);
-    done += rows;
+    for (int i = 0; i < 4; ++i) kv.mapW[i] = h->pmap_kv[i];
+    if ((e = tmap_encode_bf16(&kv.mapA, ws.pz, 2 * hdim, T, (unsigned long long)hdim * 4, 64, 128)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = launch_umma_dense(kv, h->n_sm, st)) != cudaSuccess) return fail_cuda(h, e);
   }
   return DART_OK;
 }

@@ -191,7 +191,7 @@ static __device__ __noinline__ void finalize_group_t(int ft, const GemmArgs& p, 
     for (int k = 0; k < NP; ++k) {
       cs[k] = make_float2(1.f, 0.f);
       const int idx = ft + NTHR * k, ptok = tok0 + idx / pairs, pi = idx % pairs;
-      if (MODE == EPI_QKV && s + e.kind0 < 2 && idx < pairs * 8 && ptok < M)
+      if (MODE == EPI_QKV && s < 2 && idx < pairs * 8 && ptok < M)
         cs[k] = e.rope_tab[(size_t)s_pos[ptok] * half + (pi % half)];  // (cos, sin) of pos * theta^(-2i/d_h)
     }
     float rs = 0.f;
@@ -252,7 +252,7 @@ static __device__ __noinline__ void finalize_group_t(int ft, const GemmArgs& p, 
       // y = rstd_g * (W[:, :h] z_g) + W[:, h:] z_e ; RoPE on q, k at position P_b + r ; q and the new rows'
       // k, v as hi/lo pairs ; the fresh rows' k, v appended to the cache.  segment 0,1,2 = q,k,v (g half);
       // the e half is the paired tile.
-      const int kind = s + e.kind0;
+      const int kind = s;
 #pragma unroll
       for (int k = 0; k < NP; ++k) {
         const int idx = ft + NTHR * k, ptok = tok0 + idx / pairs, pi = idx % pairs;
@@ -277,14 +277,11 @@ static __device__ __noinline__ void finalize_group_t(int ft, const GemmArgs& p, 
             e.q_hi[o + i] = h1; e.q_hi[o + i + half] = h2;
             e.q_lo[o + i] = l1; e.q_lo[o + i + half] = l2;
           } else {
-            if (!e.prefill) {   // the step's attention reads its own rows from the hi/lo side tile
-              bf16* side = (kind == 1 ? e.k_new : e.v_new) + ((size_t)b * e.Hkv + head) * 16 * dh;
-              side[(size_t)r * dh + i] = h1; side[(size_t)r * dh + i + half] = h2;
-              side[(size_t)(8 + r) * dh + i] = l1; side[(size_t)(8 + r) * dh + i + half] = l2;
-            }
+            bf16* side = (kind == 1 ? e.k_new : e.v_new) + ((size_t)b * e.Hkv + head) * 16 * dh;
+            side[(size_t)r * dh + i] = h1; side[(size_t)r * dh + i + half] = h2;
+            side[(size_t)(8 + r) * dh + i] = l1; side[(size_t)(8 + r) * dh + i + half] = l2;
             if (fresh_index(e, b, r) >= 0) {
-              const int cb = e.prefill ? e.slab[b] : b;   // cache slab of this run
-              bf16* dst = (kind == 1 ? e.k_cache : e.v_cache) + (((size_t)cb * e.Hkv + head) * e.P_cap + s_pos[tok]) * dh;
+              bf16* dst = (kind == 1 ? e.k_cache : e.v_cache) + (((size_t)b * e.Hkv + head) * e.P_cap + s_pos[tok]) * dh;
               dst[i] = h1;
               dst[i + half] = h2;
             }

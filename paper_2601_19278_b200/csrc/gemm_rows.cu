@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(512, (NT == 1 ? 2 : 1)) gemm_rows_kernel(const
   if (threadIdx.x == 0) s_done[0] = 0;
   if (p.epi.mode == EPI_QKV && threadIdx.x < p.s.M) {
     // inputs of the step and init-time constants: nothing an earlier kernel of this step writes
-    s_pos[threadIdx.x] = (p.epi.prefill ? p.epi.pos0[threadIdx.x / p.epi.K] : p.epi.seq_lens[threadIdx.x / p.epi.K]) + threadIdx.x % p.epi.K;
+    s_pos[threadIdx.x] = p.epi.seq_lens[threadIdx.x / p.epi.K] + threadIdx.x % p.epi.K;
     s_rstd[threadIdx.x] = p.epi.rstd_mask[0];  // <mask> rows; fresh rows are overwritten in the finalize
   }
   const long long u0 = ((long long)c * p.U) / G, u1 = ((long long)(c + 1) * p.U) / G;

@@ -108,10 +108,6 @@ struct EpiArgs {
   // EPI_QKV
   int Hq, Hkv, dh; const int32_t* seq_lens; const float2* rope_tab;  // [positions][dh/2] (cos, sin)
   bf16* q_hi; bf16* q_lo; bf16* k_new; bf16* v_new; bf16* k_cache; bf16* v_cache; long long P_cap;
-  // Draft-side prefill (dart_draft_prefill): the launch covers up to 32 runs of at most K consecutive new rows;
-  // run b holds rows pos0[b] .. of cache slab slab[b]; only k and v are projected (segment s is kind s + kind0:
-  // 0 = q, 1 = k, 2 = v) and nothing but the cache is written.
-  int prefill, kind0; int pos0[32]; unsigned char slab[32];
 };
 
 // What the shared streaming core (stream_core.cuh) needs to know about a launch.
@@ -153,6 +149,26 @@ struct UmmaGemmArgs {
 };
 cudaError_t launch_umma_rows(const GemmPlan& plan, const UmmaMaps& maps, const GemmInput& in, const EpiArgs& epi, float* part,
                              int* status, cudaStream_t st);
+// Dense projections of the draft-side prefill (umma_dense.cu): C[T, n_out] = A[T, k] W^T with 128 token rows per
+// tile on the MMA's M side and 256 output features on its N side.  mode 0: feature FC (A = features, one weight
+// matrix, one reduction range) -> z g-half = bf16(g * gain), ss[T][n_tiles] partial sums of squares.  mode 1:
+// k / v (A = z; weight matrices W_k, W_v, each as its g-half and e-half columns: mapW[2*w + half]) ->
+// y = rstd_g * (g half) + (e half), RoPE on k, bf16 into the caches.
+struct DenseArgs {
+  CUtensorMap mapA, mapW[4];
+  int T, mode, n_w, n_tiles_per_w, n_out;
+  int KB[2], a_koff[2];
+  int h; float eps;
+  const bf16* gain; bf16* z; long long ldz;       // mode 0 outputs
+  float* ss; int ss_ld, ss_n;                      // [T][ss_ld] partial sums of squares (ss_n of them per row)
+  int Hkv, dh; const float2* rope_tab; bf16* k_cache; bf16* v_cache; long long P_cap;
+  int B; int seq_off[33]; int seq_P[32];          // packed row t of sequence b sits at position seq_P[b] + t - seq_off[b]
+  int* status;
+};
+cudaError_t launch_umma_dense(const DenseArgs& a, int n_sm, cudaStream_t st);
+cudaError_t launch_prefill_embed(const int32_t* tokens, int T, int vocab, const bf16* embed, const bf16* gain_e, int h, float eps,
+                                 bf16* z, long long ldz, cudaStream_t st);
+
 // 2-D bf16 tensor map [outer][inner] (row stride ld_bytes), box {box_inner, box_outer}, 128-byte swizzle, zero fill.
 cudaError_t tmap_encode_bf16(CUtensorMap* m, const void* base, unsigned long long inner, unsigned long long outer,
                              unsigned long long ld_bytes, unsigned box_inner, unsigned box_outer);

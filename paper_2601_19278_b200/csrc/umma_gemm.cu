@@ -102,7 +102,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
   if (warp == 2) tmem_alloc(&tmem_base, C::TmemCols);
   if (p.epi.mode == EPI_QKV && threadIdx.x < p.s.M) {
     // inputs of the step and init-time constants: nothing an earlier kernel of this step writes
-    s_pos[threadIdx.x] = (p.epi.prefill ? p.epi.pos0[threadIdx.x / p.epi.K] : p.epi.seq_lens[threadIdx.x / p.epi.K]) + threadIdx.x % p.epi.K;
+    s_pos[threadIdx.x] = p.epi.seq_lens[threadIdx.x / p.epi.K] + threadIdx.x % p.epi.K;
     s_rstd[threadIdx.x] = p.epi.rstd_mask[0];  // <mask> rows; fresh rows are overwritten in the finalize
   }
   int cand[kMetaSlots] = {-1, -1};  // groups whose piece tables sit in s_meta
