@@ -114,3 +114,35 @@ def build_tree(ids: np.ndarray, slogit: np.ndarray, ctx: Tuple[int, int], tri: D
             p = par[p]
     return {"tokens": tokens, "parents": parents, "depth": depth, "mask": mask,
             "n_nodes": np.int32(1 + len(order)), "scores": scores, "n_scored": n_all - 1}
+
+
+def verification_inputs(parents: np.ndarray, depth: np.ndarray, n_nodes: int, root_pos: int, max_levels: int) -> Dict[str, np.ndarray]:
+    """What the target model needs to verify a draft tree in one forward pass with tree attention (Section 3,
+    Figure 2: the draft tree is verified "with Tree Attention"; the tree-attention mask itself is build_tree's
+    `mask`).  Reading (the paper names the step, not its encoding): node x sits at absolute position
+    root_pos + depth[x], root_pos being the position of the root token c_-1; a candidate continuation is a
+    root-to-leaf path, listed as the slots of its nodes.
+      position_ids [budget]           root_pos + depth[x] for the n_nodes used slots, -1 elsewhere
+      retrieve     [budget, L+1]      row j = the slots of the j-th leaf's path, root first, padded with -1;
+                                      leaves in ascending slot order; unused rows all -1
+      n_leaves                        number of leaves (used slots that are nobody's parent)"""
+    budget = parents.shape[0]
+    pos = np.full((budget,), -1, dtype=np.int32)
+    pos[:n_nodes] = root_pos + depth[:n_nodes]
+    is_parent = np.zeros((budget,), dtype=bool)
+    for x in range(1, n_nodes):
+        is_parent[parents[x]] = True
+    retrieve = np.full((budget, max_levels + 1), -1, dtype=np.int32)
+    n_leaves = 0
+    for x in range(n_nodes):
+        if is_parent[x]:
+            continue
+        path = []
+        y = x
+        while y >= 0:
+            path.append(y)
+            y = int(parents[y])
+        path.reverse()
+        retrieve[n_leaves, :len(path)] = path
+        n_leaves += 1
+    return {"position_ids": pos, "retrieve": retrieve, "n_leaves": np.int32(n_leaves)}

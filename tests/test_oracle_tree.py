@@ -205,3 +205,35 @@ def test_ngram_rows_are_normalised_log_probabilities():
         assert abs(np.exp(rows["score"][key == c].astype(np.float64)).sum() - 1.0) < 1e-5
     full = key * 1000 + rows["next"]
     assert len(np.unique(full)) == len(full)
+
+
+def test_verification_inputs_cover_the_tree_with_root_to_leaf_paths():
+    """Pins of the verification glue: every path is a parent chain from the root, depths count up by one along
+    it, the paths' union is the whole tree, a slot is a leaf iff nobody names it as parent, and the number of
+    ancestors-or-self in build_tree's attention mask is the position offset plus one."""
+    rng = np.random.default_rng(3)
+    V, d, k = 50, 5, 6
+    ids = np.stack([rng.choice(V, size=k, replace=False) for _ in range(d)]).astype(np.int32)
+    sl = np.sort(rng.normal(-3, 1.5, size=(d, k)).astype(np.float32))[:, ::-1].copy()
+    t = otree.build_tree(ids, sl, (3, 7), {}, {}, beam=4, budget=24)
+    n = int(t["n_nodes"])
+    g = otree.verification_inputs(np.asarray(t["parents"]), np.asarray(t["depth"]), n, root_pos=100, max_levels=d)
+    par, dep, mask = np.asarray(t["parents"]), np.asarray(t["depth"]), np.asarray(t["mask"])
+    assert np.array_equal(g["position_ids"][:n], 100 + dep[:n]) and np.all(g["position_ids"][n:] == -1)
+    assert np.array_equal(mask[:n].sum(axis=1) - 1, dep[:n])                      # ancestors-or-self = depth + 1
+    leaves = sorted(set(range(n)) - set(int(p) for p in par[1:n]))
+    assert int(g["n_leaves"]) == len(leaves) and n > 5 and len(leaves) > 1
+    seen = set()
+    for j, leaf in enumerate(leaves):
+        path = [int(x) for x in g["retrieve"][j] if x >= 0]
+        assert path[0] == 0 and path[-1] == leaf
+        for a, b in zip(path[:-1], path[1:]):
+            assert par[b] == a and dep[b] == dep[a] + 1
+        assert np.all(g["retrieve"][j, len(path):] == -1)
+        seen.update(path)
+    assert seen == set(range(n))
+    assert np.all(g["retrieve"][len(leaves):] == -1)
+    # a chain (beam 1, one candidate per level) has exactly one leaf and one path through every node
+    t1 = otree.build_tree(ids[:, :1], sl[:, :1], (3, 7), {}, {}, beam=1, budget=24)
+    g1 = otree.verification_inputs(np.asarray(t1["parents"]), np.asarray(t1["depth"]), int(t1["n_nodes"]), root_pos=0, max_levels=d)
+    assert int(g1["n_leaves"]) == 1 and [int(x) for x in g1["retrieve"][0]] == list(range(d + 1))
