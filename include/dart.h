@@ -224,6 +224,30 @@ size_t dart_workspace_bytes(const dart_config* cfg);
 int dart_step_launch_count(const dart_handle* h, int batch, int n_fresh);
 
 /*
+ * Verification inputs of a draft tree (Section 3, Figure 2: the tree is verified by the target model in one
+ * forward pass with tree attention; the attention mask is dart_tree_out.mask).  The paper names the step, not
+ * its encoding; this one is the usual pair: node x sits at absolute position root_pos[b] + depth[x] (root_pos =
+ * position of the root token c_-1), and a candidate continuation is a root-to-leaf path given as the slots of its
+ * nodes.  retrieve row j = path of the j-th leaf (leaves in ascending slot order), root first, padded with -1;
+ * rows past n_leaves and position ids of unused slots are -1.  One small kernel, asynchronous on `cuda_stream`.
+ * Errors: INVALID_ARG, CAPACITY (batch > max_batch).
+ */
+typedef struct dart_verify_in {
+  int32_t batch;
+  int32_t max_levels;         /* columns of retrieve minus one: >= the deepest node's depth (K is always enough) */
+  const int32_t* parents;     /* DEVICE i32 [B, tree_budget] as written by dart_build_tree */
+  const int32_t* depth;       /* DEVICE i32 [B, tree_budget] */
+  const int32_t* n_nodes;     /* DEVICE i32 [B] */
+  const int32_t* root_pos;    /* DEVICE i32 [B] absolute position of each sequence's root token */
+} dart_verify_in;
+typedef struct dart_verify_out {
+  int32_t* position_ids;      /* DEVICE i32 [B, tree_budget] */
+  int32_t* retrieve;          /* DEVICE i32 [B, tree_budget, max_levels + 1] */
+  int32_t* n_leaves;          /* DEVICE i32 [B] */
+} dart_verify_out;
+int dart_tree_verify_inputs(dart_handle* h, const dart_verify_in* in, const dart_verify_out* out, void* cuda_stream);
+
+/*
  * Draft-side prefill (Section 3.2: the draft layer attends over its own KV cache of the prefix, which has to
  * exist before the first drafting step).  A single layer's keys and values depend on nothing but the layer's
  * input, so building the cache for new prefix positions needs no attention: for every new row the call

@@ -26,7 +26,7 @@ DART_ERR_INTERNAL = -6
 
 EXPORTS = [
     "dart_draft_init", "dart_draft_step", "dart_build_tree", "dart_draft_destroy", "dart_last_device_status",
-    "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_step_launch_count", "dart_draft_prefill",
+    "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_step_launch_count", "dart_draft_prefill", "dart_tree_verify_inputs",
     "dart_set_profile_events", "dart_topk_rows_noalloc",
 ]
 
@@ -65,6 +65,15 @@ class DartStepIn(C.Structure):
 class DartPrefillIn(C.Structure):
     _fields_ = [("batch", C.c_int32), ("feats", C.c_void_p), ("tokens", C.c_void_p), ("seq_lens_host", C.c_void_p),
                 ("new_rows_host", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p)]
+
+
+class DartVerifyIn(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("max_levels", C.c_int32), ("parents", C.c_void_p), ("depth", C.c_void_p),
+                ("n_nodes", C.c_void_p), ("root_pos", C.c_void_p)]
+
+
+class DartVerifyOut(C.Structure):
+    _fields_ = [("position_ids", C.c_void_p), ("retrieve", C.c_void_p), ("n_leaves", C.c_void_p)]
 
 
 class DartStepOut(C.Structure):
@@ -109,6 +118,8 @@ def lib() -> C.CDLL:
         L.dart_status_string.restype = C.c_char_p
         L.dart_workspace_bytes.argtypes = [C.POINTER(DartConfig)]
         L.dart_workspace_bytes.restype = C.c_size_t
+        L.dart_tree_verify_inputs.argtypes = [C.c_void_p, C.POINTER(DartVerifyIn), C.POINTER(DartVerifyOut), C.c_void_p]
+        L.dart_tree_verify_inputs.restype = C.c_int
         L.dart_draft_prefill.argtypes = [C.c_void_p, C.POINTER(DartPrefillIn), C.c_void_p]
         L.dart_draft_prefill.restype = C.c_int
         L.dart_step_launch_count.argtypes = [C.c_void_p, C.c_int, C.c_int]
@@ -206,6 +217,15 @@ class DartDraft:
         rc = lib().dart_draft_prefill(self._h, C.byref(pin), self._stream(stream))
         if rc != DART_OK:
             raise DartError(rc, "dart_draft_prefill", lib().dart_last_cuda_error(self._h))
+
+    def verify_inputs(self, *, batch: int, max_levels: int, parents, depth, n_nodes, root_pos, position_ids, retrieve, n_leaves,
+                      stream=None) -> None:
+        """dart_tree_verify_inputs: position ids and root-to-leaf paths of the trees dart_build_tree wrote."""
+        vin = DartVerifyIn(batch, max_levels, _ptr(parents), _ptr(depth), _ptr(n_nodes), _ptr(root_pos))
+        vout = DartVerifyOut(_ptr(position_ids), _ptr(retrieve), _ptr(n_leaves))
+        rc = lib().dart_tree_verify_inputs(self._h, C.byref(vin), C.byref(vout), self._stream(stream))
+        if rc != DART_OK:
+            raise DartError(rc, "dart_tree_verify_inputs", lib().dart_last_cuda_error(self._h))
 
     def build_tree(self, *, batch: int, topk_ids, topk_slogit, ctx_tail, tokens, parents, depth, mask, n_nodes,
                    scores=None, first_row=0, n_levels: Optional[int] = None, stream=None) -> None:

@@ -714,6 +714,19 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   return DART_OK;
 }
 
+int dart_tree_verify_inputs(dart_handle* h, const dart_verify_in* in, const dart_verify_out* out, void* cuda_stream) {
+  if (h == nullptr || in == nullptr || out == nullptr) return DART_ERR_INVALID_ARG;
+  const dart_config& c = h->cfg;
+  if (in->batch < 1 || in->max_levels < 1 || in->max_levels > 64 || c.tree_budget > 64) return DART_ERR_INVALID_ARG;
+  if (in->batch > c.max_batch) return DART_ERR_CAPACITY;
+  if (in->parents == nullptr || in->depth == nullptr || in->n_nodes == nullptr || in->root_pos == nullptr ||
+      out->position_ids == nullptr || out->retrieve == nullptr || out->n_leaves == nullptr)
+    return DART_ERR_INVALID_ARG;
+  const cudaError_t e = launch_verify_inputs(in->batch, c.tree_budget, in->max_levels, in->parents, in->depth, in->n_nodes, in->root_pos,
+                                             out->position_ids, out->retrieve, out->n_leaves, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? DART_OK : fail_cuda(h, e);
+}
+
 int dart_draft_prefill(dart_handle* h, const dart_prefill_in* in, void* cuda_stream) {
   if (h == nullptr || in == nullptr) return DART_ERR_INVALID_ARG;
   const dart_config& c = h->cfg;

@@ -250,6 +250,9 @@ struct TreeParams {
   int* status;
 };
 cudaError_t tree_setup(int topk, int beam, int budget, int max_levels);  // once per device
+// Position ids and root-to-leaf paths of the trees (verification inputs); budget <= 64.
+cudaError_t launch_verify_inputs(int B, int budget, int max_levels, const int32_t* parents, const int32_t* depth, const int32_t* n_nodes,
+                                 const int32_t* root_pos, int32_t* position_ids, int32_t* retrieve, int32_t* n_leaves, cudaStream_t st);
 size_t tree_smem_bytes(int topk, int beam, int budget, int n_levels);
 cudaError_t launch_tree(const TreeParams& p, cudaStream_t st);
 

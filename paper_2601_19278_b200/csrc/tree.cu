@@ -221,6 +221,52 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
   }
 }
 
+// Verification inputs of one tree per block: thread x owns slot x (budget <= 64 threads' worth of slots).
+__global__ void __launch_bounds__(64) verify_inputs_kernel(int budget, int max_levels, const int32_t* parents, const int32_t* depth,
+                                                           const int32_t* n_nodes, const int32_t* root_pos, int32_t* position_ids,
+                                                           int32_t* retrieve, int32_t* n_leaves) {
+  __shared__ int s_par[64], s_dep[64], s_isp[64];
+  const int b = blockIdx.x, x = threadIdx.x, W = max_levels + 1;
+  pdl_wait();
+  const int n = n_nodes[b];
+  const bool used = x < n && x < budget;
+  s_par[x] = used ? parents[(size_t)b * budget + x] : -1;
+  s_dep[x] = used ? depth[(size_t)b * budget + x] : -1;
+  s_isp[x] = 0;
+  __syncthreads();
+  if (used && x >= 1 && s_par[x] >= 0 && s_par[x] < 64) s_isp[s_par[x]] = 1;   // benign race: every writer stores 1
+  __syncthreads();
+  if (x < budget) position_ids[(size_t)b * budget + x] = used ? root_pos[b] + s_dep[x] : -1;
+  const bool leaf = used && !s_isp[x];
+  int rank = 0, total = 0;
+  for (int y = 0; y < budget && y < 64; ++y) {
+    const int l = (y < n && !s_isp[y]) ? 1 : 0;
+    total += l;
+    if (y < x) rank += l;
+  }
+  int32_t* rows = retrieve + (size_t)b * budget * W;
+  if (x < budget && x >= total)   // rows past the last leaf are all -1: row x is cleared by thread x
+    for (int c = 0; c < W; ++c) rows[(size_t)x * W + c] = -1;
+  if (leaf) {
+    int32_t* row = rows + (size_t)rank * W;
+    const int d = s_dep[x];
+    for (int c = d + 1; c < W; ++c) row[c] = -1;
+    int y = x;
+    for (int guard = 0; guard <= max_levels && y >= 0; ++guard) {   // bounded walk up the parent chain
+      const int dy = s_dep[y];
+      if (dy >= 0 && dy < W) row[dy] = y;
+      y = s_par[y];
+    }
+  }
+  if (x == 0) n_leaves[b] = total;
+}
+
+cudaError_t launch_verify_inputs(int B, int budget, int max_levels, const int32_t* parents, const int32_t* depth, const int32_t* n_nodes,
+                                 const int32_t* root_pos, int32_t* position_ids, int32_t* retrieve, int32_t* n_leaves, cudaStream_t st) {
+  return launch_pdl(verify_inputs_kernel, dim3(B), dim3(64), 0, st, budget, max_levels, parents, depth, n_nodes, root_pos, position_ids,
+                    retrieve, n_leaves);
+}
+
 size_t tree_smem_bytes(int topk, int beam, int budget, int n_levels) {
   return tree_layout(topk, beam, budget, n_levels, nullptr, nullptr) + 16;
 }

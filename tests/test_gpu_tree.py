@@ -145,3 +145,26 @@ def test_argument_and_capacity_errors():
     assert e.value.status == binding.DART_ERR_INVALID_ARG
     torch.cuda.synchronize()
     ses.close()
+
+
+@pytest.mark.parametrize("topk,beam,budget,K", [(25, 20, 60, 8), (3, 2, 60, 4), (1, 1, 16, 6), (32, 32, 64, 8)])
+def test_verification_inputs_match_the_oracle(topk, beam, budget, K):
+    """Position ids and root-to-leaf paths of the GPU's own trees, bit for bit."""
+    rows = syn.make_ngram_rows(VOCAB, 50_000, "zipf_mixed", seed=8)
+    w, ses = _session(2, K, topk=topk, beam=beam, budget=budget, rows=rows)
+    t = syn.make_tree_inputs(VOCAB, 2, K, topk, seed=11)
+    got = _gpu_tree(ses, t["ids"], t["slogit"], t["ctx_tail"])
+    dev = ses.dev
+    root_pos = torch.tensor([1000, 17], dtype=torch.int32, device=dev)
+    pos = torch.full((2, budget), 7, dtype=torch.int32, device=dev)
+    ret = torch.full((2, budget, K + 1), 7, dtype=torch.int32, device=dev)
+    nl = torch.zeros((2,), dtype=torch.int32, device=dev)
+    ses.draft.verify_inputs(batch=2, max_levels=K, parents=ses.parents, depth=ses.depth, n_nodes=ses.n_nodes, root_pos=root_pos,
+                            position_ids=pos, retrieve=ret, n_leaves=nl)
+    torch.cuda.synchronize()
+    for b in range(2):
+        ref = otree.verification_inputs(got["parents"][b], got["depth"][b], int(got["n_nodes"][b]), int(root_pos[b]), K)
+        assert np.array_equal(pos[b].cpu().numpy(), ref["position_ids"])
+        assert np.array_equal(ret[b].cpu().numpy(), ref["retrieve"])
+        assert int(nl[b]) == int(ref["n_leaves"]) and int(nl[b]) >= 1
+    ses.close()
