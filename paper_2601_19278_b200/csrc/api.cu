@@ -572,14 +572,16 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   EpiArgs ep;
   GemmInput gi;
   if (h->umma && h->maps_M != M) {
-    // activation tensor maps: [M rows][width], box = 64 k x MP rows; rows past M read as zeros
+    // activation tensor maps: hi and lo buffers as one [M rows][2][width] tensor, box = 64 k x 2 x MP rows; rows past M
+    // read as zeros
     struct { UmmaMaps* m; const bf16* hi; const bf16* lo; int width; } xin[4] = {
         {&h->maps_qkv, ws.z_hi, ws.z_lo, 2 * hdim}, {&h->maps_o, ws.a_hi, ws.a_lo, dq},
         {&h->maps_gu, ws.n_hi, ws.n_lo, hdim}, {&h->maps_down, ws.u_hi, ws.u_lo, c.mlp_inter}};
     for (int i = 0; i < 4; ++i) {
-      if ((e = tmap_encode_bf16(&xin[i].m->Xhi, xin[i].hi, xin[i].width, M, (unsigned long long)xin[i].width * 2, 64, MP)) != cudaSuccess ||
-          (e = tmap_encode_bf16(&xin[i].m->Xlo, xin[i].lo, xin[i].width, M, (unsigned long long)xin[i].width * 2, 64, MP)) != cudaSuccess)
+      const unsigned long long pair = (unsigned long long)(reinterpret_cast<const char*>(xin[i].lo) - reinterpret_cast<const char*>(xin[i].hi));
+      if ((e = tmap_encode_bf16_pair(&xin[i].m->Xhi, xin[i].hi, pair, xin[i].width, M, (unsigned long long)xin[i].width * 2, MP)) != cudaSuccess)
         return fail_cuda(h, e);
+      xin[i].m->Xlo = xin[i].m->Xhi;
     }
     h->maps_M = M;
   }

@@ -134,8 +134,9 @@ struct GemmArgs {
 };
 
 // The same projections on the tcgen05 / TMA path (umma_gemm.cu): plan units are (128-row tile, 64-k block),
-// one persistent CTA per SM.  Tensor maps: one per weight segment, one each for the hi and lo activations
-// (box = 64 k x MP rows; a plain-bf16 input uses Xhi alone with a box of 2*MP rows, whose missing rows read 0).
+// one persistent CTA per SM.  Tensor maps: one per weight segment; Xhi = the activations: hi + lo inputs as one
+// 3-D map (box = 64 k x (hi, lo) x MP rows: accumulator column 2t is token t's hi part, 2t+1 its lo part); a
+// plain-bf16 input as a 2-D map with a box of 2*MP rows whose missing rows read 0 (column t is token t).
 struct UmmaMaps {
   CUtensorMap W[6];
   CUtensorMap Xhi, Xlo;
@@ -172,6 +173,9 @@ cudaError_t launch_prefill_embed(const int32_t* tokens, int T, int vocab, const 
 // 2-D bf16 tensor map [outer][inner] (row stride ld_bytes), box {box_inner, box_outer}, 128-byte swizzle, zero fill.
 cudaError_t tmap_encode_bf16(CUtensorMap* m, const void* base, unsigned long long inner, unsigned long long outer,
                              unsigned long long ld_bytes, unsigned box_inner, unsigned box_outer);
+// hi + lo activation buffers (lo = hi + pair_bytes) as one 3-D map; a box of box_rows tokens arrives as (hi, lo) row pairs.
+cudaError_t tmap_encode_bf16_pair(CUtensorMap* m, const void* hi, unsigned long long pair_bytes, unsigned long long inner,
+                                  unsigned long long rows, unsigned long long ld_bytes, unsigned box_rows);
 
 cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const EpiArgs& epi, float* part, cudaStream_t st);
 // (cos, sin) table of RoPE for positions 0 .. n_pos-1 (once, at init)

@@ -261,8 +261,7 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
     tile = (int)(u0 / KB); kb = (int)(u0 % KB);
     for (int it = 0; it < pre; ++it) {
       uint8_t* xs = ring + (size_t)it * C::StageBytes + 128 * 64 * 2;
-      tma_load_2d(xs, &a.mapXhi, &full[it], kb * 64, 0);
-      tma_load_2d(xs + C::XBytes / 2, &a.mapXlo, &full[it], kb * 64, 0);
+      tma_load_3d(xs, &a.mapXhi, &full[it], kb * 64, 0, 0);
       if (++kb == KB) { kb = 0; ++tile; }
     }
     int s = pre == C::Stages ? 0 : pre, ph = pre == C::Stages ? 1 : 0;
@@ -271,8 +270,7 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
       uint8_t* st = ring + (size_t)s * C::StageBytes;
       mbar_expect_tx(&full[s], C::StageBytes);
       tma_load_2d_hint(st, &a.mapW, &full[s], kb * 64, tile * 128, wpol);
-      tma_load_2d(st + 128 * 64 * 2, &a.mapXhi, &full[s], kb * 64, 0);
-      tma_load_2d(st + 128 * 64 * 2 + C::XBytes / 2, &a.mapXlo, &full[s], kb * 64, 0);
+      tma_load_3d(st + 128 * 64 * 2, &a.mapXhi, &full[s], kb * 64, 0, 0);
       if (++s == C::Stages) { s = 0; ++ph; }
       if (++kb == KB) { kb = 0; ++tile; }
     }
@@ -346,13 +344,12 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
       const int rows_here = min(128, p.V - tile * 128);
 #pragma unroll 1
       for (int ch = 0; ch < MP / 8; ++ch) {
-        uint32_t hi[8], lo[8];
-        tmem_ld8(tbase + ch * 8, hi);
-        tmem_ld8(tbase + MP + ch * 8, lo);
+        uint32_t r[16];   // columns (2t, 2t+1) are token t's hi and lo parts
+        tmem_ld16(tbase + ch * 16, r);
         tmem_ld_wait();
         float y[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) y[j] = __uint_as_float(hi[j]) + __uint_as_float(lo[j]);
+        for (int j = 0; j < 8; ++j) y[j] = __uint_as_float(r[2 * j]) + __uint_as_float(r[2 * j + 1]);
         if (ch == MP / 8 - 1) {  // the accumulator buffer is free once its last columns are in registers
           tc_fence_before();
           mbar_arrive(&acc_empty[buf]);

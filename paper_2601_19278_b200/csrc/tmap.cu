@@ -39,4 +39,24 @@ cudaError_t tmap_encode_bf16(CUtensorMap* m, const void* base, unsigned long lon
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// hi and lo parts of an activation matrix as ONE 3-D tensor [rows][2][inner]: the lo buffer lies `pair_bytes` after
+// the hi buffer, rows are ld_bytes apart.  A box {64, 2, box_rows} lands in shared memory as rows (hi, lo) of token
+// 0, (hi, lo) of token 1, ...: one copy instead of two per stage.
+cudaError_t tmap_encode_bf16_pair(CUtensorMap* m, const void* hi, unsigned long long pair_bytes, unsigned long long inner,
+                                  unsigned long long rows, unsigned long long ld_bytes, unsigned box_rows) {
+  EncodeTiledFn enc = encoder();
+  if (enc == nullptr) return cudaErrorNotSupported;
+  if ((reinterpret_cast<uintptr_t>(hi) & 15u) != 0 || (ld_bytes & 15u) != 0 || (pair_bytes & 15u) != 0 || pair_bytes == 0 || box_rows > 256 ||
+      inner == 0 || rows == 0)
+    return cudaErrorInvalidValue;
+  cuuint64_t dims[3] = {inner, 2, rows};
+  cuuint64_t strides[2] = {pair_bytes, ld_bytes};
+  cuuint32_t box[3] = {64, 2, box_rows};
+  cuuint32_t elem[3] = {1, 1, 1};
+  const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(hi), dims, strides, box, elem,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 }  // namespace dart

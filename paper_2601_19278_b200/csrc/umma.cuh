@@ -52,6 +52,13 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, u
                : "memory");
 }
 
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
+                   smem_u32(dst)),
+               "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+
 // The same load with an L2 eviction policy: weights are read once per step, so they are marked evict-first
 // and do not push the step's small re-used data (activations, pieces, tables, code) out of L2.
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {

@@ -128,8 +128,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
     q.set(p.s, u0);
     for (int it = 0; it < pre; ++it, q.next(p.s)) {
       uint8_t* xs = ring + (size_t)it * C::StageBytes + kWBytes;
-      tma_load_2d(xs, &a.mapXhi, &full[it], q.xoff + q.kb * 64, 0);
-      if (a.has_lo) tma_load_2d(xs + C::XBytes / 2, &a.mapXlo, &full[it], q.xoff + q.kb * 64, 0);
+      if (a.has_lo) tma_load_3d(xs, &a.mapXhi, &full[it], q.xoff + q.kb * 64, 0, 0);
+      else tma_load_2d(xs, &a.mapXhi, &full[it], q.xoff + q.kb * 64, 0);
     }
     int s = pre == C::Stages ? 0 : pre, ph = pre == C::Stages ? 1 : 0;
     for (int it = pre; it < n; ++it, q.next(p.s)) {
@@ -137,8 +137,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       uint8_t* st = ring + (size_t)s * C::StageBytes;
       mbar_expect_tx(&full[s], C::StageBytes);
       tma_load_2d_hint(st, &a.mapW[q.seg], &full[s], q.kb * 64, q.row0, wpol);
-      tma_load_2d(st + kWBytes, &a.mapXhi, &full[s], q.xoff + q.kb * 64, 0);
-      if (a.has_lo) tma_load_2d(st + kWBytes + C::XBytes / 2, &a.mapXlo, &full[s], q.xoff + q.kb * 64, 0);
+      if (a.has_lo) tma_load_3d(st + kWBytes, &a.mapXhi, &full[s], q.xoff + q.kb * 64, 0, 0);
+      else tma_load_2d(st + kWBytes, &a.mapXhi, &full[s], q.xoff + q.kb * 64, 0);
       if (++s == C::Stages) { s = 0; ++ph; }
     }
   } else if (warp == 1 && lane == 0) {
@@ -190,14 +190,22 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + buf * C::N;
 #pragma unroll
       for (int ch = 0; ch < MP / 8; ++ch) {
-        uint32_t hi[8], lo[8];
-        tmem_ld8(tbase + ch * 8, hi);
-        tmem_ld8(tbase + MP + ch * 8, lo);
-        tmem_ld_wait();
-        const float4 v0 = make_float4(__uint_as_float(hi[0]) + __uint_as_float(lo[0]), __uint_as_float(hi[1]) + __uint_as_float(lo[1]),
-                                      __uint_as_float(hi[2]) + __uint_as_float(lo[2]), __uint_as_float(hi[3]) + __uint_as_float(lo[3]));
-        const float4 v1 = make_float4(__uint_as_float(hi[4]) + __uint_as_float(lo[4]), __uint_as_float(hi[5]) + __uint_as_float(lo[5]),
-                                      __uint_as_float(hi[6]) + __uint_as_float(lo[6]), __uint_as_float(hi[7]) + __uint_as_float(lo[7]));
+        // hi + lo inputs: columns (2t, 2t+1) are token t's two parts; a plain input: column t is token t
+        uint32_t r[16];
+        float y[8];
+        if (a.has_lo) {
+          tmem_ld16(tbase + ch * 16, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) y[j] = __uint_as_float(r[2 * j]) + __uint_as_float(r[2 * j + 1]);
+        } else {
+          uint32_t q8[8];
+          tmem_ld8(tbase + ch * 8, q8);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) y[j] = __uint_as_float(q8[j]);
+        }
+        const float4 v0 = make_float4(y[0], y[1], y[2], y[3]), v1 = make_float4(y[4], y[5], y[6], y[7]);
         reinterpret_cast<float4*>(dst + ch * 8)[0] = v0;
         reinterpret_cast<float4*>(dst + ch * 8)[1] = v1;
       }
