@@ -56,7 +56,9 @@ struct dart_handle {
   bool umma = false;         // projections run on the tcgen05 / TMA kernels (tensor maps could be encoded)
   UmmaMaps maps_fc, maps_qkv, maps_o, maps_gu, maps_down;
   CUtensorMap pmap_fc, pmap_kv[4];   // prefill: W_fc, and the g-/e-half columns of W_k and W_v (boxes of 256 rows)
-  CUtensorMap map_lm;        // the LM head's weight matrix
+  CUtensorMap map_lm;        // the LM head's weight matrix (boxes of 128 rows)
+  CUtensorMap map_lm256;     // the same with boxes of 256 rows, for the swapped-operand kernel (33..128 token rows)
+  CUtensorMap lmx_hi, lmx_lo; int lmx_M = -1;   // that kernel's activation maps [M][h], boxes of 128 rows
   int lm_tag = 0;            // launch counter of the LM head (marks its cross-CTA pieces)
   int maps_M = -1;           // token rows the activation tensor maps were encoded for
   const void* maps_feats = nullptr; int maps_fc_M = -1;
@@ -424,6 +426,7 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   PlanHost* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
   if (h->umma) {
     INIT_CHECK(tmap_encode_bf16(&h->map_lm, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 128));
+    INIT_CHECK(tmap_encode_bf16(&h->map_lm256, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 256));
     if (cfg->feat_in > 0) {
       const unsigned long long hh = cfg->hidden, kvr = (unsigned long long)cfg->n_kv_heads * cfg->head_dim;
       const bf16* wk = static_cast<const bf16*>(weights->w_k);
@@ -701,9 +704,20 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   mark(6, true);
   if (h->umma) {
     // one CTA per SM at most: the CTAs of this kernel wait on one another's pieces, so all must be resident
-    const long long units = (long long)((c.vocab + 127) / 128) * ((hdim + 63) / 64);
+    const bool dense = MP == 128;   // many token rows: tokens on the MMA's M side, 256 vocabulary rows per tile
+    const long long units = (long long)((c.vocab + (dense ? 255 : 127)) / (dense ? 256 : 128)) * ((hdim + 63) / 64);
     lp.grid = (int)(units < h->n_sm ? units : h->n_sm);
-    e = launch_lm_head_umma(lp, h->map_lm, h->maps_gu.Xhi, h->maps_gu.Xlo, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
+    if (dense) {
+      if (h->lmx_M != M) {
+        if ((e = tmap_encode_bf16(&h->lmx_hi, ws.n_hi, hdim, M, (unsigned long long)hdim * 2, 64, 128)) != cudaSuccess ||
+            (e = tmap_encode_bf16(&h->lmx_lo, ws.n_lo, hdim, M, (unsigned long long)hdim * 2, 64, 128)) != cudaSuccess)
+          return fail_cuda(h, e);
+        h->lmx_M = M;
+      }
+      e = launch_lm_head_dense(lp, h->map_lm256, h->lmx_hi, h->lmx_lo, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
+    } else {
+      e = launch_lm_head_umma(lp, h->map_lm, h->maps_gu.Xhi, h->maps_gu.Xlo, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
+    }
   } else {
     e = launch_lm_head(lp, st);
   }

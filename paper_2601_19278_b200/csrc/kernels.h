@@ -234,6 +234,11 @@ struct LmUmmaArgs {
 };
 cudaError_t launch_lm_head_umma(const LmParams& p, const CUtensorMap& mapW, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st);
+// The LM head for 33..128 token rows with the operands swapped (token rows on the MMA's M side; lm_head.cu).
+// mapW256: the weight matrix with boxes of 256 rows; mapXhi / mapXlo: 2-D maps [M][Kd], boxes of 128 rows;
+// pieces: [grid][128][256] fp32.  The per-CTA results are laid out for MP = 128 token rows.
+cudaError_t launch_lm_head_dense(const LmParams& p, const CUtensorMap& mapW256, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
+                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st);
 cudaError_t topk_merge_setup(int max_grid);  // once per device
 cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st);
 

@@ -25,9 +25,14 @@
 namespace dart {
 
 __device__ __forceinline__ float gumbel_from_bits(uint32_t x) {
-  // u = ((x >> 8) + 0.5) * 2^-24 in (0,1); fp64 so that u never rounds to 1
-  const double u = ((double)(x >> 8) + 0.5) * (1.0 / 16777216.0);
-  return (float)(-log(-log(u)));
+  // u = ((x >> 8) + 0.5) * 2^-24 in (0, 1); G = -log(-log u).  fp32 throughout (two fp64 logarithms per logit
+  // were the LM head's largest cost at temperature > 0: 690 of 1330 us at 128 token rows).  Near u = 1 the
+  // inner logarithm goes through log1p of the exact distance to 1, so the top bits of x keep their say.
+  const uint32_t m = x >> 8;
+  float t;
+  if (m >= (1u << 23)) t = -log1pf(-(((float)((1u << 24) - m) - 0.5f) * (1.f / 16777216.f)));
+  else t = -logf(((float)m + 0.5f) * (1.f / 16777216.f));
+  return -logf(t);
 }
 
 // Insert (key, y, id) into the warp-resident list (lane j holds the j-th best; order: key desc, id asc).
@@ -437,6 +442,296 @@ cudaError_t launch_lm_head_umma(const LmParams& pin, const CUtensorMap& mapW, co
   if (MP == 8) return launch_lm_umma_t<8>(a, st);
   if (MP == 32) return launch_lm_umma_t<32>(a, st);
   return launch_lm_umma_t<128>(a, st);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// LM head for 33..128 token rows: the operands swap sides.  With that many tokens the activation slice of a
+// 64-k block (hi and lo rows of every token) is as large as the weight tile it meets, and re-reading it from L2
+// for every 128 vocabulary rows is what bounds the kernel above (3 bytes through L2 per weight byte).  Here the
+// token rows are the M side of tcgen05.mma (hi and lo as two MMAs into one accumulator) and 256 vocabulary rows
+// its N side, so a stage carries 32 KB of activations for 32 KB of weights.  The accumulator row of a token
+// is one TMEM lane, i.e. one read-out thread: that thread keeps the token's running (max, sum-exp) in registers
+// and its best-`topk` candidates in a shared-memory row of its own (replace-the-worst; sorted once at the end),
+// so the fold needs no cross-thread step at all.  Work split, ownership of tiles cut between CTAs, flags and
+// bounded waits are those of lm_head_umma_kernel, with 256-row tiles.
+// ------------------------------------------------------------------------------------------------------
+constexpr int kLmDenseStages = 3;
+constexpr int kLmDenseStageBytes = 2 * 128 * 64 * 2 + 256 * 64 * 2;   // hi tokens, lo tokens, 256 vocabulary rows
+constexpr int kLmDenseListStride = 33;                                  // floats per token row of the lists (no bank conflicts)
+constexpr size_t kLmDenseSmem = (size_t)kLmDenseStages * kLmDenseStageBytes + 1024 + 2 * 128 * kLmDenseListStride * 4;
+
+// (key, id) a precedes (key, id) b in the candidate order: larger key first, then smaller id
+__device__ __forceinline__ bool cand_before(float ka, int ia, float kb, int ib) { return ka > kb || (ka == kb && ia < ib); }
+
+__global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const __grid_constant__ LmUmmaArgs a) {
+  const LmParams& p = a.p;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  float* l_key = reinterpret_cast<float*>(ring + (size_t)kLmDenseStages * kLmDenseStageBytes);   // [128][33]
+  int* l_id = reinterpret_cast<int*>(l_key + 128 * kLmDenseListStride);                           // [128][33]
+  __shared__ uint64_t full[kLmDenseStages], empty[kLmDenseStages], acc_full[2], acc_empty[2];
+  __shared__ uint32_t tmem_base;
+  __shared__ int abort_flag, s_bad;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int c = blockIdx.x, G = gridDim.x;
+  const int KB = a.KB;
+  const long long u0 = ((long long)c * a.U) / G, u1 = ((long long)(c + 1) * a.U) / G;
+  constexpr int kXBytes = 128 * 64 * 2;
+
+  if (tid == 0) {
+    for (int s = 0; s < kLmDenseStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+    abort_flag = 0;
+    s_bad = 0;
+    fence_barrier_init();
+    // the producer fills the ring's weight slots before anything else of the CTA's setup
+    const int n = (int)(u1 - u0);
+    const int pre = n < kLmDenseStages ? n : kLmDenseStages;
+    const uint64_t wpol = l2_policy_evict_first();
+    int tile = (int)(u0 / KB), kb = (int)(u0 % KB);
+    for (int it = 0; it < pre; ++it) {
+      mbar_expect_tx(&full[it], kLmDenseStageBytes);
+      tma_load_2d_hint(ring + (size_t)it * kLmDenseStageBytes + 2 * kXBytes, &a.mapW, &full[it], kb * 64, tile * 256, wpol);
+      if (++kb == KB) { kb = 0; ++tile; }
+    }
+  }
+  if (warp == 2) tmem_alloc(&tmem_base, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base;
+
+  if (warp == 0 && lane == 0) {
+    // ---- producer
+    const int n = (int)(u1 - u0);
+    const int pre = n < kLmDenseStages ? n : kLmDenseStages;
+    const uint64_t wpol = l2_policy_evict_first();
+    int tile, kb;
+    pdl_wait();
+    tile = (int)(u0 / KB); kb = (int)(u0 % KB);
+    for (int it = 0; it < pre; ++it) {
+      uint8_t* st = ring + (size_t)it * kLmDenseStageBytes;
+      tma_load_2d(st, &a.mapXhi, &full[it], kb * 64, 0);
+      tma_load_2d(st + kXBytes, &a.mapXlo, &full[it], kb * 64, 0);
+      if (++kb == KB) { kb = 0; ++tile; }
+    }
+    int s = pre == kLmDenseStages ? 0 : pre, ph = pre == kLmDenseStages ? 1 : 0;
+    for (int it = pre; it < n; ++it) {
+      if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
+      uint8_t* st = ring + (size_t)s * kLmDenseStageBytes;
+      mbar_expect_tx(&full[s], kLmDenseStageBytes);
+      tma_load_2d_hint(st + 2 * kXBytes, &a.mapW, &full[s], kb * 64, tile * 256, wpol);
+      tma_load_2d(st, &a.mapXhi, &full[s], kb * 64, 0);
+      tma_load_2d(st + kXBytes, &a.mapXlo, &full[s], kb * 64, 0);
+      if (++s == kLmDenseStages) { s = 0; ++ph; }
+      if (++kb == KB) { kb = 0; ++tile; }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer: D[token, vocabulary row] += (X_hi + X_lo)[token, k] * W[vocabulary row, k]
+    constexpr uint32_t idesc = idesc_bf16(128, 256);
+    const int n = (int)(u1 - u0);
+    int visit = -1, buf = 0, tile = -1;
+    int t = (int)(u0 / KB), kb = (int)(u0 % KB), s = 0, ph = 0;
+    bool ok = true;
+    for (int it = 0; it < n && ok; ++it) {
+      bool first = false;
+      if (t != tile) {
+        if (tile >= 0) mma_commit(&acc_full[buf]);
+        tile = t;
+        first = true;
+        ++visit;
+        buf = visit & 1;
+        if (visit >= 2) {
+          if (!mbar_wait(&acc_empty[buf], ((visit >> 1) - 1) & 1, &abort_flag)) { ok = false; break; }
+          tc_fence_after();
+        }
+      }
+      if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t sa = smem_u32(ring + (size_t)s * kLmDenseStageBytes);
+      const uint64_t hd = desc_sw128(sa), ld = desc_sw128(sa + kXBytes), wd = desc_sw128(sa + 2 * kXBytes);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        mma_f16(tmem + buf * 256, hd + 2 * k, wd + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+        mma_f16(tmem + buf * 256, ld + 2 * k, wd + 2 * k, idesc, 1u);
+      }
+      mma_commit(&empty[s]);
+      if (++s == kLmDenseStages) { s = 0; ++ph; }
+      if (++kb == KB) { kb = 0; ++t; }
+    }
+    if (ok && tile >= 0) mma_commit(&acc_full[buf]);
+  } else if (warp >= 4) {
+    // ---- read-out and fold: TMEM lane = token row; this thread owns the token's statistics and list
+    const int wq = warp & 3, tok = wq * 32 + lane, et = tid - 128;
+    const bool live = tok < p.M;
+    float* my_key = l_key + tok * kLmDenseListStride;
+    int* my_id = l_id + tok * kLmDenseListStride;
+    pdl_wait();
+    float rstd = 0.f;
+    if (live) {  // the final RMSNorm's 1/rms from the previous kernel's sums of squares (same order everywhere)
+      float ssq = 0.f;
+      for (int tl = 0; tl < p.ss_tiles; ++tl) ssq += p.ss_in[(size_t)tl * p.ss_mp + tok];
+      rstd = 1.f / sqrtf(ssq / (float)p.Kd + p.rms_eps);
+    }
+    float m_run = -INFINITY, s_run = 0.f;
+    int n_list = 0, worst = 0;                 // entries in the list, slot of its last-ranked entry
+    float w_key = INFINITY; int w_id = -1;     // that entry (valid once the list is full)
+    const int topk = p.topk;
+    int visit = 0;
+    long long u = u0;
+    while (u < u1) {
+      const int tile = (int)(u / KB);
+      const int ka = (int)(u - (long long)tile * KB);
+      long long ue = (long long)(tile + 1) * KB;
+      if (ue > u1) ue = u1;
+      const bool owner = ka == 0, whole = owner && ue == (long long)(tile + 1) * KB;
+      const int buf = visit & 1;
+      if (!mbar_wait(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) s_bad = 1;
+      if (owner && !whole && et == 0) {
+        for (int cc = c + 1; cc < G && ((long long)cc * a.U) / G < (long long)(tile + 1) * KB; ++cc) {
+          int it = 0;
+          while (*reinterpret_cast<volatile int*>(a.flags + cc) != a.tag && it < kSpinLimit) { __nanosleep(200); ++it; }
+          if (it >= kSpinLimit) { s_bad = 1; abort_flag = 1; }
+        }
+        __threadfence();
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (s_bad) break;
+      tc_fence_after();
+      const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + buf * 256;
+#pragma unroll 1
+      for (int cb = 0; cb < 256; cb += 16) {
+        uint32_t r[16];
+        tmem_ld16(tbase + cb, r);
+        tmem_ld_wait();
+        if (cb == 240) {  // the accumulator buffer is free once its last columns are in registers
+          tc_fence_before();
+          mbar_arrive(&acc_empty[buf]);
+        }
+        float y[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) y[j] = __uint_as_float(r[j]);
+        if (!owner) {
+          float4* dst = reinterpret_cast<float4*>(a.pieces + (((size_t)c * 128 + tok) * 256 + cb));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) dst[j] = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
+          continue;
+        }
+        if (!whole) {
+          for (int cc = c + 1; cc < G && ((long long)cc * a.U) / G < (long long)(tile + 1) * KB; ++cc) {
+            const float4* src = reinterpret_cast<const float4*>(a.pieces + (((size_t)cc * 128 + tok) * 256 + cb));
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float4 q = __ldcg(src + j);
+              y[4 * j] += q.x; y[4 * j + 1] += q.y; y[4 * j + 2] += q.z; y[4 * j + 3] += q.w;
+            }
+          }
+        }
+        const int v0 = tile * 256 + cb;             // vocabulary id of column 0 of this chunk (a multiple of 16)
+        if (!live || v0 >= p.V) continue;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) y[j] *= rstd;
+        if (p.logits_out != nullptr) {
+          float4* lo = reinterpret_cast<float4*>(p.logits_out + (size_t)tok * p.V + v0);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) lo[j] = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
+        }
+#pragma unroll 1
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint4 rnd = make_uint4(0, 0, 0, 0);
+          if (p.gumbel)
+            rnd = philox4x32_10(make_uint4((uint32_t)((v0 >> 2) + q4), (uint32_t)(tok % p.K), (uint32_t)(tok / p.K), p.step), p.seed_lo, p.seed_hi);
+          const uint32_t rw[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int v = v0 + 4 * q4 + q;
+            const float z = y[4 * q4 + q] * p.inv_temp;
+            // running log-sum-exp of this token row
+            if (z > m_run) { s_run = s_run * expf(m_run - z) + 1.f; m_run = z; }
+            else s_run += expf(z - m_run);
+            const float key = p.gumbel ? z + gumbel_from_bits(rw[q]) : z;
+            if (n_list < topk) {
+              my_key[n_list] = key; my_id[n_list] = v;
+              if (n_list == 0 || cand_before(w_key, w_id, key, v)) { w_key = key; w_id = v; worst = n_list; }
+              ++n_list;
+            } else if (cand_before(key, v, w_key, w_id)) {
+              my_key[worst] = key; my_id[worst] = v;
+              w_key = my_key[0]; w_id = my_id[0]; worst = 0;          // find the new last-ranked entry
+              for (int e = 1; e < topk; ++e) {
+                const float ke = my_key[e]; const int ie = my_id[e];
+                if (cand_before(w_key, w_id, ke, ie)) { w_key = ke; w_id = ie; worst = e; }
+              }
+            }
+          }
+        }
+      }
+      if (!owner) {
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et == 0) *reinterpret_cast<volatile int*>(a.flags + c) = a.tag;
+      }
+      ++visit;
+      u = ue;
+    }
+    // ---- this token's list, sorted (key desc, id asc), and its statistics
+    if (live) {
+      for (int i = 1; i < n_list; ++i) {            // insertion sort of at most 32 entries
+        const float ki = my_key[i]; const int ii = my_id[i];
+        int j = i - 1;
+        while (j >= 0 && cand_before(ki, ii, my_key[j], my_id[j])) { my_key[j + 1] = my_key[j]; my_id[j + 1] = my_id[j]; --j; }
+        my_key[j + 1] = ki; my_id[j + 1] = ii;
+      }
+      const size_t o = ((size_t)c * 128 + tok) * 32;
+      for (int e = 0; e < 32; ++e) {
+        const bool have = e < n_list;
+        const float key = have ? my_key[e] : -INFINITY;
+        const int id = have ? my_id[e] : 0x7fffffff;
+        float yv = key;                                   // the un-perturbed logit / T of the entry
+        if (have && p.gumbel) {
+          const uint4 rnd = philox4x32_10(make_uint4((uint32_t)id >> 2, (uint32_t)(tok % p.K), (uint32_t)(tok / p.K), p.step), p.seed_lo, p.seed_hi);
+          const uint32_t wsel = (id & 3) == 0 ? rnd.x : ((id & 3) == 1 ? rnd.y : ((id & 3) == 2 ? rnd.z : rnd.w));
+          yv = key - gumbel_from_bits(wsel);
+        }
+        p.part_key[o + e] = key;
+        p.part_y[o + e] = have ? yv : 0.f;
+        p.part_id[o + e] = id;
+      }
+      p.part_stats[((size_t)c * 128 + tok) * 2] = m_run;
+      p.part_stats[((size_t)c * 128 + tok) * 2 + 1] = s_run;
+    }
+  }
+  pdl_wait();
+  pdl_trigger();
+  __syncthreads();
+  if (warp == 2) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+  if ((abort_flag || s_bad) && tid == 0) {
+    atomicExch(a.status, DEV_TIMEOUT);
+    for (int i = 0; i < 100; ++i) __nanosleep(1000);
+  }
+  // token rows past M leave empty lists (the merge reads MP = 128 rows per CTA)
+  for (int i = tid; i < (128 - p.M) * 32; i += kLmUmmaThreads) {
+    const size_t o = ((size_t)c * 128 + p.M) * 32 + i;
+    p.part_key[o] = -INFINITY; p.part_y[o] = 0.f; p.part_id[o] = 0x7fffffff;
+  }
+  for (int i = tid; i < (128 - p.M) * 2; i += kLmUmmaThreads) p.part_stats[((size_t)c * 128 + p.M) * 2 + i] = (i & 1) ? 0.f : -INFINITY;
+}
+
+cudaError_t launch_lm_head_dense(const LmParams& pin, const CUtensorMap& mapW256, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
+                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st) {
+  LmUmmaArgs a;
+  memset(&a, 0, sizeof(a));
+  a.p = pin;
+  a.mapW = mapW256; a.mapXhi = mapXhi; a.mapXlo = mapXlo;
+  a.KB = (pin.Kd + 63) / 64;
+  a.U = (long long)((pin.V + 255) / 256) * a.KB;
+  a.pieces = pieces; a.flags = flags; a.tag = tag; a.status = status;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(lm_head_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDenseSmem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  return launch_pdl(lm_head_dense_kernel, dim3(a.p.grid), dim3(kLmUmmaThreads), kLmDenseSmem, st, a);
 }
 
 template <int NT, int NW>
