@@ -584,7 +584,6 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
       const unsigned long long pair = (unsigned long long)(reinterpret_cast<const char*>(xin[i].lo) - reinterpret_cast<const char*>(xin[i].hi));
       if ((e = tmap_encode_bf16_pair(&xin[i].m->Xhi, xin[i].hi, pair, xin[i].width, M, (unsigned long long)xin[i].width * 2, MP)) != cudaSuccess)
         return fail_cuda(h, e);
-      xin[i].m->Xlo = xin[i].m->Xhi;
     }
     h->maps_M = M;
   }
@@ -618,7 +617,6 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
       if ((e = tmap_encode_bf16(&h->maps_fc.Xhi, in->feats, c.feat_in, NF, (unsigned long long)c.feat_in * 2, 64,
                                 2 * padded_tokens(NF))) != cudaSuccess)
         return fail_cuda(h, e);
-      h->maps_fc.Xlo = h->maps_fc.Xhi;
       h->maps_feats = in->feats; h->maps_fc_M = NF;
     }
     if ((e = project(h->plan_fc, h->maps_fc)) != cudaSuccess) return fail_cuda(h, e);
@@ -716,7 +714,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
       }
       e = launch_lm_head_dense(lp, h->map_lm256, h->lmx_hi, h->lmx_lo, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
     } else {
-      e = launch_lm_head_umma(lp, h->map_lm, h->maps_gu.Xhi, h->maps_gu.Xlo, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
+      e = launch_lm_head_umma(lp, h->map_lm, h->maps_gu.Xhi, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
     }
   } else {
     e = launch_lm_head(lp, st);

@@ -5,20 +5,38 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 namespace dart {
 
 typedef __nv_bfloat16 bf16;
+
+// Function attributes are per device: a (device, function) pair is configured the first time it is launched.
+// Process-wide table behind a mutex (handles on different devices or threads may launch the same kernel).
+inline bool first_launch_on_device(const void* fn, int what) {
+  static std::mutex mu;
+  static struct { const void* fn; int dev, what; } seen[256];
+  static int n = 0;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  std::lock_guard<std::mutex> lock(mu);
+  for (int i = 0; i < n; ++i)
+    if (seen[i].fn == fn && seen[i].dev == dev && seen[i].what == what) return false;
+  if (n < 256) { seen[n].fn = fn; seen[n].dev = dev; seen[n].what = what; ++n; }
+  return true;
+}
 
 // All kernels of the step ask for the same (largest) shared-memory carve-out: the streaming kernels need
 // ~200 KB per SM, and an SM whose L1 / shared-memory split differs from what the next kernel wants has to
 // drain and reconfigure first, which serialises consecutive kernels and costs tens of microseconds a switch.
 inline void prefer_max_shared(const void* fn) {
-  static const void* seen[64];
-  static int n = 0;
-  for (int i = 0; i < n; ++i)
-    if (seen[i] == fn) return;
-  if (n < 64) seen[n++] = fn;
-  cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+  if (first_launch_on_device(fn, 0))
+    cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+}
+// Opt-in to more than 48 KB of dynamic shared memory, once per device.
+inline cudaError_t allow_dynamic_smem(const void* fn, size_t bytes) {
+  if (!first_launch_on_device(fn, 1)) return cudaSuccess;
+  return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
 // Launch with programmatic stream serialization (see pdl_wait / pdl_trigger in common.cuh).
@@ -139,12 +157,12 @@ struct GemmArgs {
 // plain-bf16 input as a 2-D map with a box of 2*MP rows whose missing rows read 0 (column t is token t).
 struct UmmaMaps {
   CUtensorMap W[6];
-  CUtensorMap Xhi, Xlo;
+  CUtensorMap Xhi;   // the activations (see above)
 };
 struct UmmaGemmArgs {
   GemmArgs g;
   CUtensorMap mapW[6];
-  CUtensorMap mapXhi, mapXlo;
+  CUtensorMap mapXhi;
   int has_lo;
   int* status;   // device status word (DEV_TIMEOUT when a bounded wait ran out)
 };
@@ -232,7 +250,7 @@ struct LmUmmaArgs {
   float* pieces; int* flags; int tag;
   int* status;
 };
-cudaError_t launch_lm_head_umma(const LmParams& p, const CUtensorMap& mapW, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
+cudaError_t launch_lm_head_umma(const LmParams& p, const CUtensorMap& mapW, const CUtensorMap& mapX,
                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st);
 // The LM head for 33..128 token rows with the operands swapped (token rows on the MMA's M side; lm_head.cu).
 // mapW256: the weight matrix with boxes of 256 rows; mapXhi / mapXlo: 2-D maps [M][Kd], boxes of 128 rows;

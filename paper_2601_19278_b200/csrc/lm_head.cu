@@ -420,21 +420,17 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
 template <int MP>
 static cudaError_t launch_lm_umma_t(const LmUmmaArgs& a, cudaStream_t st) {
   using C = LmUmmaCfg<MP>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(lm_head_umma_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SmemBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(lm_head_umma_kernel<MP>), C::SmemBytes);
+  if (e != cudaSuccess) return e;
   return launch_pdl(lm_head_umma_kernel<MP>, dim3(a.p.grid), dim3(kLmUmmaThreads), C::SmemBytes, st, a);
 }
 
-cudaError_t launch_lm_head_umma(const LmParams& pin, const CUtensorMap& mapW, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
+cudaError_t launch_lm_head_umma(const LmParams& pin, const CUtensorMap& mapW, const CUtensorMap& mapX,
                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st) {
   LmUmmaArgs a;
   memset(&a, 0, sizeof(a));
   a.p = pin;
-  a.mapW = mapW; a.mapXhi = mapXhi; a.mapXlo = mapXlo;
+  a.mapW = mapW; a.mapXhi = mapX;
   a.KB = (pin.Kd + 63) / 64;
   a.U = (long long)((pin.V + 127) / 128) * a.KB;
   a.pieces = pieces; a.flags = flags; a.tag = tag; a.status = status;
@@ -725,12 +721,8 @@ cudaError_t launch_lm_head_dense(const LmParams& pin, const CUtensorMap& mapW256
   a.KB = (pin.Kd + 63) / 64;
   a.U = (long long)((pin.V + 255) / 256) * a.KB;
   a.pieces = pieces; a.flags = flags; a.tag = tag; a.status = status;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(lm_head_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDenseSmem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(lm_head_dense_kernel), kLmDenseSmem);
+  if (e != cudaSuccess) return e;
   return launch_pdl(lm_head_dense_kernel, dim3(a.p.grid), dim3(kLmUmmaThreads), kLmDenseSmem, st, a);
 }
 

@@ -224,12 +224,8 @@ cudaError_t launch_prefill_embed(const int32_t* tokens, int T, int vocab, const 
 }
 
 cudaError_t launch_umma_dense(const DenseArgs& a, int n_sm, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(umma_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDenseSmem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_dense_kernel), kDenseSmem);
+  if (e != cudaSuccess) return e;
   const int tiles = ((a.T + 127) / 128) * a.n_w * a.n_tiles_per_w;
   const int grid = tiles < n_sm ? tiles : n_sm;
   return launch_pdl(umma_dense_kernel, dim3(grid), dim3(kDenseThreads), kDenseSmem, st, a);

@@ -268,12 +268,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
 template <int MP>
 static cudaError_t launch_umma_t(const UmmaGemmArgs& a, int grid, cudaStream_t st) {
   using C = UmmaCfg<MP>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(umma_rows_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SmemBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_rows_kernel<MP>), C::SmemBytes);
+  if (e != cudaSuccess) return e;
   return launch_pdl(umma_rows_kernel<MP>, dim3(grid), dim3(kUmmaThreads), C::SmemBytes, st, a);
 }
 
@@ -290,7 +286,7 @@ cudaError_t launch_umma_rows(const GemmPlan& plan, const UmmaMaps& maps, const G
   g.ctr = plan.d_ctr; g.expected = plan.d_expected; g.pair_offset = plan.pair_offset;
   g.epi = epi;
   for (int i = 0; i < 6; ++i) a.mapW[i] = maps.W[i < plan.nseg ? i : 0];
-  a.mapXhi = maps.Xhi; a.mapXlo = maps.Xlo; a.has_lo = in.x_lo != nullptr ? 1 : 0;
+  a.mapXhi = maps.Xhi; a.has_lo = in.x_lo != nullptr ? 1 : 0;
   a.status = status;
   const int MP = padded_tokens(in.M);
   if (MP == 8) return launch_umma_t<8>(a, plan.grid, st);
