@@ -75,6 +75,8 @@ typedef struct dart_config {
   float eps_ng;          /* epsilon of a missing N-gram: s_ng = log(eps_ng) */
   float temperature;     /* 0 = deterministic top-k; > 0 = Gumbel-top-k on logits / temperature */
   uint64_t philox_seed;  /* key of the Philox4x32-10 stream used when temperature > 0 */
+  int32_t ngram_layout;  /* device layout of the N-gram: DART_NGRAM_HASH or DART_NGRAM_TRIE (Appendix C) */
+  int32_t reserved0;     /* 0 */
 } dart_config;
 
 /*
@@ -106,6 +108,9 @@ typedef struct dart_weights {
  * token next[i] has continuity score score[i] = log(Pr(next | context) + eps), Appendix D's
  * s_ng.  order[i] is 3 (trigram) or 2 (bigram; ctx0[i] ignored).  Of duplicate rows the first wins.
  */
+#define DART_NGRAM_HASH 0 /* open-addressing table, one 16-byte slot per row at load <= 0.5: one probe per lookup */
+#define DART_NGRAM_TRIE 1 /* child lists (Appendix C): the context's node is located once, its children are then
+                             searched for every candidate; 8 bytes per row plus 8 per distinct 3-gram context */
 typedef struct dart_ngram_host {
   int64_t n_rows;
   const uint8_t* order;
@@ -218,6 +223,9 @@ const char* dart_status_string(int status);
 
 /* Bytes of device workspace a handle for `cfg` allocates (excluding the N-gram table); 0 if cfg is invalid. */
 size_t dart_workspace_bytes(const dart_config* cfg);
+
+/* Bytes of device memory the N-gram of this handle occupies in its layout (0 without an N-gram or handle). */
+size_t dart_ngram_bytes(const dart_handle* h);
 
 /* Number of kernels one dart_draft_step / dart_build_tree call enqueues for this batch size
  * (used by benchmarks to report launch counts). */

@@ -26,7 +26,7 @@ DART_ERR_INTERNAL = -6
 
 EXPORTS = [
     "dart_draft_init", "dart_draft_step", "dart_build_tree", "dart_draft_destroy", "dart_last_device_status",
-    "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_step_launch_count", "dart_draft_prefill", "dart_tree_verify_inputs",
+    "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_ngram_bytes", "dart_step_launch_count", "dart_draft_prefill", "dart_tree_verify_inputs",
     "dart_set_profile_events", "dart_topk_rows_noalloc",
 ]
 
@@ -39,8 +39,11 @@ class DartConfig(C.Structure):
         ("beam", C.c_int32), ("tree_budget", C.c_int32), ("ngram_order", C.c_int32),
         ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("w_ng", C.c_float), ("logit_decay", C.c_float),
         ("level_exp", C.c_float), ("eps_logit", C.c_float), ("eps_ng", C.c_float), ("temperature", C.c_float),
-        ("philox_seed", C.c_uint64),
+        ("philox_seed", C.c_uint64), ("ngram_layout", C.c_int32), ("reserved0", C.c_int32),
     ]
+
+
+NGRAM_HASH, NGRAM_TRIE = 0, 1
 
 
 WEIGHT_NAMES = ["w_fc", "embed", "mask_vec", "norm_g", "norm_e", "w_q", "w_k", "w_v", "w_o", "norm_post",
@@ -118,6 +121,8 @@ def lib() -> C.CDLL:
         L.dart_status_string.restype = C.c_char_p
         L.dart_workspace_bytes.argtypes = [C.POINTER(DartConfig)]
         L.dart_workspace_bytes.restype = C.c_size_t
+        L.dart_ngram_bytes.argtypes = [C.c_void_p]
+        L.dart_ngram_bytes.restype = C.c_size_t
         L.dart_tree_verify_inputs.argtypes = [C.c_void_p, C.POINTER(DartVerifyIn), C.POINTER(DartVerifyOut), C.c_void_p]
         L.dart_tree_verify_inputs.restype = C.c_int
         L.dart_draft_prefill.argtypes = [C.c_void_p, C.POINTER(DartPrefillIn), C.c_void_p]
@@ -149,7 +154,8 @@ def make_config(w, **over) -> DartConfig:
                 mlp_inter=w.mlp_inter, vocab=w.vocab, feat_in=w.feat_in, max_batch=w.batch,
                 max_prefix=w.max_prefix, K=w.K, topk=w.topk, beam=w.beam, tree_budget=w.tree_budget,
                 ngram_order=3, rope_theta=1e6, rms_eps=1e-6, w_ng=0.5, logit_decay=0.9, level_exp=0.7,
-                eps_logit=1e-10, eps_ng=1e-10, temperature=w.temperature, philox_seed=1234)
+                eps_logit=1e-10, eps_ng=1e-10, temperature=w.temperature, philox_seed=1234,
+                ngram_layout=NGRAM_HASH)
     vals.update(over)
     for k, v in vals.items():
         setattr(cfg, k, v)
@@ -251,6 +257,9 @@ class DartDraft:
 
     def launch_count(self, batch: int, n_fresh: int) -> int:
         return lib().dart_step_launch_count(self._h, batch, n_fresh)
+
+    def ngram_bytes(self) -> int:
+        return lib().dart_ngram_bytes(self._h)
 
 
 def topk_rows_noalloc(logits: torch.Tensor, topk: int, eps_logit: float, out_ids: torch.Tensor, out_slogit: torch.Tensor,

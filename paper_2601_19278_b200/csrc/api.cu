@@ -34,6 +34,7 @@ struct Workspace {
   float* mask_res = nullptr;    // [h] g half of the <mask> representation as fp32
   float2* rope_tab = nullptr;   // [max_prefix + K][dh/2] (cos, sin)
   float* bg = nullptr;          // [max_batch][topk + (K-1)*topk^2] bigram scores of the tree builder
+  uint2* cx = nullptr;          // [max_batch][1 + topk + (K-2)*topk^2] child ranges of the 3-gram contexts (trie layout)
   float *o_part = nullptr, *ml_part = nullptr;
   float *lm_stats = nullptr, *lm_key = nullptr, *lm_y = nullptr;
   int32_t* lm_id = nullptr;
@@ -68,6 +69,8 @@ struct dart_handle {
   Workspace ws;
   NgramSlot* ng_slots = nullptr;
   uint32_t ng_mask = 0, ng_max_probe = 0;
+  NgramTrieOwned ng_trie{};     // the child-list layout (ngram_layout = DART_NGRAM_TRIE)
+  size_t ng_bytes = 0;
   float wl[8], wv[8], wn, miss;
   std::vector<void*> owned;  // small device arrays (plan tables, counters)
   int z_B = -1;              // row pattern (batch, per-sequence fresh rows) the <mask> rows of z were last written for
@@ -98,6 +101,7 @@ bool config_ok(const dart_config* c) {
   if (c->beam < 1 || c->beam > 32) return false;
   if (c->tree_budget < 2 || c->tree_budget > 64) return false;
   if (c->ngram_order != 2 && c->ngram_order != 3) return false;
+  if (c->ngram_layout != DART_NGRAM_HASH && c->ngram_layout != DART_NGRAM_TRIE) return false;
   if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f) || !(c->temperature >= 0.f)) return false;
   if (!(c->eps_ng > 0.f) || !(c->eps_logit >= 0.f)) return false;
   return true;
@@ -262,6 +266,7 @@ size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_p
   TAKE(mask_res, float*, (size_t)c.hidden * sizeof(float));
   TAKE(rope_tab, float2*, (size_t)(c.max_prefix + c.K) * (c.head_dim / 2) * sizeof(float2));
   TAKE(bg, float*, (size_t)c.max_batch * (c.topk + (size_t)(c.K - 1) * c.topk * c.topk) * sizeof(float));
+  TAKE(cx, uint2*, (size_t)c.max_batch * (1 + c.topk + (size_t)(c.K > 2 ? c.K - 2 : 0) * c.topk * c.topk) * sizeof(uint2));
   TAKE(o_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * c.head_dim * sizeof(float));
   TAKE(ml_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * 2 * sizeof(float));
   TAKE(lm_pieces, float*, (size_t)lm_grid * 128 * MPmax * sizeof(float));
@@ -376,6 +381,8 @@ size_t dart_workspace_bytes(const dart_config* cfg) {
   return layout_workspace(*cfg, part_capacity(*cfg, n_sm), attn_pairs_capacity(*cfg, n_sm), 2 * n_sm, nullptr, nullptr);
 }
 
+size_t dart_ngram_bytes(const dart_handle* h) { return h ? h->ng_bytes : 0; }
+
 int dart_last_cuda_error(const dart_handle* h) { return h ? h->last_cuda_error : g_init_cuda_error; }
 
 int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const dart_ngram_host* ngram, dart_handle** out) {
@@ -479,9 +486,26 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   h->wn = cfg->w_ng;
   h->miss = (float)log((double)cfg->eps_ng);
 
-  // N-gram rows -> open-addressing table (linear probing, load <= 0.5, first duplicate wins)
+  // N-gram rows -> device table in the configured layout (of duplicate rows the first wins)
   const long long n_rows = ngram ? ngram->n_rows : 0;
   if (n_rows > 0) {
+    if (n_rows >= (1ll << 32) - 1) { dart_draft_destroy(h); return DART_ERR_INVALID_ARG; }
+    for (long long i = 0; i < n_rows; ++i) {
+      const int ord = ngram->order[i];
+      const int c0 = ngram->ctx0[i], c1 = ngram->ctx1[i], nx = ngram->next[i];
+      if ((ord != 2 && ord != 3) || c1 < 0 || nx < 0 || c1 >= cfg->vocab || nx >= cfg->vocab ||
+          (ord == 3 && (c0 < 0 || c0 >= cfg->vocab))) {
+        dart_draft_destroy(h);
+        return DART_ERR_INVALID_ARG;
+      }
+    }
+  }
+  if (n_rows > 0 && cfg->ngram_layout == DART_NGRAM_TRIE) {
+    INIT_CHECK(ngram_trie_build(ngram->order, ngram->ctx0, ngram->ctx1, ngram->next, ngram->score, n_rows, cfg->vocab,
+                                cfg->ngram_order, &h->ng_trie));
+    h->ng_bytes = h->ng_trie.bytes;
+  } else if (n_rows > 0) {
+    // open-addressing table: linear probing, load <= 0.5
     size_t cap = 16;
     while (cap < (size_t)(2 * n_rows)) cap <<= 1;
     if (cap > (1ull << 31)) { dart_draft_destroy(h); return DART_ERR_INVALID_ARG; }
@@ -492,11 +516,6 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
     for (long long i = 0; i < n_rows; ++i) {
       const int ord = ngram->order[i];
       const int c0 = ngram->ctx0[i], c1 = ngram->ctx1[i], nx = ngram->next[i];
-      if ((ord != 2 && ord != 3) || c1 < 0 || nx < 0 || c1 >= cfg->vocab || nx >= cfg->vocab ||
-          (ord == 3 && (c0 < 0 || c0 >= cfg->vocab))) {
-        dart_draft_destroy(h);
-        return DART_ERR_INVALID_ARG;
-      }
       if (ord == 3 && cfg->ngram_order < 3) continue;
       const unsigned long long key = ngram_key(ord, c0, c1, nx);
       uint32_t pos = (uint32_t)ngram_hash(key) & mask, d = 0;
@@ -510,6 +529,7 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
     INIT_CHECK(cudaMemcpy(h->ng_slots, tab.data(), cap * sizeof(NgramSlot), cudaMemcpyHostToDevice));
     h->ng_mask = mask;
     h->ng_max_probe = max_probe;
+    h->ng_bytes = cap * sizeof(NgramSlot);
   }
 
   INIT_CHECK(topk_merge_setup(2 * n_sm));
@@ -526,6 +546,7 @@ int dart_draft_destroy(dart_handle* h) {
   for (void* p : h->owned) cudaFree(p);
   if (h->ws.base) cudaFree(h->ws.base);
   if (h->ng_slots) cudaFree(h->ng_slots);
+  ngram_trie_free(&h->ng_trie);
   delete h;
   return DART_OK;
 }
@@ -819,7 +840,7 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
   if (in->n_levels * (c.tree_budget - 1) > 1024) return DART_ERR_INVALID_ARG;
   TreeParams tp;
   tp.B = in->batch; tp.K = c.K; tp.topk = c.topk; tp.beam = c.beam; tp.budget = c.tree_budget;
-  tp.first_row = in->first_row; tp.n_levels = in->n_levels; tp.ngram_order = c.ngram_order;
+  tp.first_row = in->first_row; tp.n_levels = in->n_levels; tp.ngram_order = c.ngram_order; tp.vocab = c.vocab;
   for (int b = 0; b < 32; ++b) {  // per-sequence first logit row (level 0); a sequence has min(n_levels, K - first row) levels
     int fr = in->first_row;
     if (in->first_rows_host != nullptr && b < in->batch) {
@@ -831,7 +852,9 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
   tp.ids = in->topk_ids; tp.slogit = in->topk_slogit; tp.ctx_tail = in->ctx_tail;
   tp.table.slots = h->ng_slots; tp.table.mask = h->ng_mask; tp.table.max_probe = h->ng_max_probe;
   for (int i = 0; i < 8; ++i) { tp.wl[i] = h->wl[i]; tp.wv[i] = h->wv[i]; }
-  tp.wn = h->wn; tp.miss = h->miss; tp.bg = h->ws.bg;
+  tp.trie.bi_off = h->ng_trie.bi_off; tp.trie.bi_ent = h->ng_trie.bi_ent; tp.trie.tri_off = h->ng_trie.tri_off;
+  tp.trie.tri_node = h->ng_trie.tri_node; tp.trie.tri_ent = h->ng_trie.tri_ent;
+  tp.wn = h->wn; tp.miss = h->miss; tp.bg = h->ws.bg; tp.cx = h->ws.cx;
   tp.tokens = out->tokens; tp.parents = out->parents; tp.depth = out->depth; tp.mask = out->mask;
   tp.n_nodes = out->n_nodes; tp.scores = out->scores; tp.status = h->ws.status;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

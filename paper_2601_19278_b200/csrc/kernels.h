@@ -265,13 +265,28 @@ cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st);
 // ---------------------------------------------------------------------------------------------
 struct NgramSlot { unsigned long long key; float score; uint32_t pad; };  // 16 bytes; key 0 = empty
 struct NgramTable { const NgramSlot* slots; uint32_t mask; uint32_t max_probe; };
+// The same rows as child lists (Appendix C).  Every list is an array of {key, payload} pairs in ascending key
+// order and has at most `vocab` entries:
+//   2-gram context b   -> bi_ent[bi_off[b] .. bi_off[b+1])             {next token, score bits}
+//   first token a      -> tri_node[tri_off[a] .. tri_off[a+1])         {second context token b, first child}
+//   3-gram context j   -> tri_ent[tri_node[j].y .. tri_node[j+1].y)    {next token, score bits}
+// tri_node carries one sentinel entry after the last node.
+struct NgramTrie { const uint32_t* bi_off; const uint2* bi_ent; const uint32_t* tri_off; const uint2* tri_node; const uint2* tri_ent; };
+struct NgramTrieOwned { uint32_t* bi_off; uint2* bi_ent; uint32_t* tri_off; uint2* tri_node; uint2* tri_ent; size_t bytes; };
+// Host rows -> device child lists (rows must have been validated; 3-gram rows are skipped when ngram_order < 3;
+// of duplicate rows the first wins).  Synchronous; on failure everything allocated so far is released.
+cudaError_t ngram_trie_build(const unsigned char* order, const int32_t* c0, const int32_t* c1, const int32_t* nx, const float* score,
+                             long long n_rows, int vocab, int ngram_order, NgramTrieOwned* out);
+void ngram_trie_free(NgramTrieOwned* t);
 
 struct TreeParams {
-  int B, K, topk, beam, budget, first_row, n_levels, ngram_order;
+  int B, K, topk, beam, budget, first_row, n_levels, ngram_order, vocab;
   unsigned char first_rows[32];   // per sequence: first logit row = level 0; levels = min(n_levels, K - first row)
   const int32_t* ids; const float* slogit; const int32_t* ctx_tail;
   NgramTable table;
+  NgramTrie trie;   // used instead of `table` when trie.bi_off != nullptr
   float* bg;   // [B][topk + (n_levels-1)*topk^2] bigram scores (workspace, written by the sweep kernel)
+  uint2* cx;   // [B][1 + topk + (n_levels-2)*topk^2] child ranges of the 3-gram contexts (trie layout only)
   float wl[8]; float wv[8]; float wn; float miss;
   int32_t* tokens; int32_t* parents; int32_t* depth; uint8_t* mask; int32_t* n_nodes; float* scores;
   int* status;

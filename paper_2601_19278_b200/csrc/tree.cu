@@ -47,6 +47,40 @@ __device__ __forceinline__ bool probe_rest(const NgramTable& T, unsigned long lo
   return false;
 }
 
+// Look `key` up in the sorted list ent[lo .. hi) of {key, payload} pairs (a child list of the trie, at most 2^21
+// entries).  A 16-ary search: every round reads 15 evenly spaced keys at once -- their latencies overlap, so a round
+// costs one memory round trip -- and keeps the sixteenth of the list that can hold the key; a list of 16 or fewer is
+// read whole.  1 round trip for the common short list, 5 for a list as long as the vocabulary.  The rounds are
+// bounded and every read stays inside [lo, hi), whatever the list holds.
+__device__ __forceinline__ bool trie_find(const uint2* __restrict__ ent, uint32_t lo, uint32_t hi, int key, uint32_t& payload, uint32_t& index) {
+#pragma unroll 1
+  for (int round = 0; round < 6 && hi - lo > 16u; ++round) {
+    const uint32_t n = hi - lo;
+    int piv[15];
+#pragma unroll
+    for (int q = 0; q < 15; ++q) piv[q] = (int)__ldg(&ent[lo + ((n * (uint32_t)(q + 1)) >> 4)].x);
+    uint32_t c = 0;
+#pragma unroll
+    for (int q = 0; q < 15; ++q) c += piv[q] <= key ? 1u : 0u;
+    const uint32_t nlo = lo + ((n * c) >> 4), nhi = c < 15u ? lo + ((n * (c + 1u)) >> 4) : hi;
+    lo = nlo; hi = nhi;
+  }
+  bool found = false;
+#pragma unroll
+  for (int q = 0; q < 16; ++q) {
+    const uint32_t idx = lo + (uint32_t)q;
+    if (idx < hi) {
+      const uint2 v = __ldg(&ent[idx]);
+      if ((int)v.x == key) { found = true; payload = v.y; index = idx; }
+    }
+  }
+  return found;
+}
+
+// Sizes of the per-sequence sweep outputs: bigram scores and 3-gram context ranges for `levels` levels.
+__host__ __device__ inline int sweep_bigrams(int k, int levels) { return k + (levels - 1) * k * k; }
+__host__ __device__ inline int sweep_contexts(int k, int levels) { return 1 + (levels >= 2 ? k : 0) + (levels > 2 ? (levels - 2) * k * k : 0); }
+
 struct TreeSmem {
   float* n_score; float* n_clamp; int* n_tok; int* n_par; unsigned char* n_j;
   Key* xk; int* beam_a; int* beam_b; int* sel; int* par_out; int* lvl_base;
@@ -96,8 +130,44 @@ __global__ void __launch_bounds__(256) bigram_sweep_kernel(const TreeParams p) {
   p.bg[(size_t)b * n_bg + e] = sc;
 }
 
+// The sweep for the trie layout.  Besides the bigram scores (a search of context b's child list for t) it locates
+// the node of every 3-gram context a level can ask for -- (c_-2, c_-1) for level 0, (c_-1, S_0[j]) for level 1,
+// (S_{i-2}[j'], S_{i-1}[j]) for level i -- once, and leaves the range of its children in cx, laid out like bg:
+// cx[b][0], cx[b][1 + j], cx[b][1 + k + (i-2)k^2 + j'k + j].  A context that is absent gets the empty range.
+__global__ void __launch_bounds__(256) trie_sweep_kernel(const TreeParams p) {
+  pdl_wait();
+  const int k = p.topk, b = blockIdx.y;
+  const int fr = p.first_rows[b], Lb = min(p.n_levels, p.K - fr);
+  const int n_bg = sweep_bigrams(k, p.n_levels), n_cx = sweep_contexts(k, p.n_levels);   // layout strides: the launch's maximum
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
+  const NgramTrie T = p.trie;
+  uint32_t pay, idx;
+  if (e < n_bg) {
+    if (e >= sweep_bigrams(k, Lb)) return;
+    int tb, tt;
+    if (e < k) { tb = p.ctx_tail[2 * b + 1]; tt = ids[e]; }
+    else { const int r = e - k, i = r / (k * k), q = r - i * k * k, jb = q / k; tb = ids[i * k + jb]; tt = ids[(i + 1) * k + q - jb * k]; }
+    float sc = p.miss;
+    if (tb >= 0 && tb < p.vocab && trie_find(T.bi_ent, __ldg(T.bi_off + tb), __ldg(T.bi_off + tb + 1), tt, pay, idx)) sc = __uint_as_float(pay);
+    p.bg[(size_t)b * n_bg + e] = sc;
+    return;
+  }
+  const int c = e - n_bg;
+  if (c >= sweep_contexts(k, Lb)) return;
+  int ta, tb;
+  if (c == 0) { ta = p.ctx_tail[2 * b]; tb = p.ctx_tail[2 * b + 1]; }
+  else if (c < 1 + k) { ta = p.ctx_tail[2 * b + 1]; tb = ids[c - 1]; }
+  else { const int r = c - 1 - k, i2 = r / (k * k), q = r - i2 * k * k, jp = q / k; ta = ids[i2 * k + jp]; tb = ids[(i2 + 1) * k + q - jp * k]; }
+  uint2 range = make_uint2(0u, 0u);
+  if (p.ngram_order >= 3 && ta >= 0 && ta < p.vocab && tb >= 0 && trie_find(T.tri_node, __ldg(T.tri_off + ta), __ldg(T.tri_off + ta + 1), tb, pay, idx))
+    range = make_uint2(pay, __ldg(&T.tri_node[idx + 1]).y);
+  p.cx[(size_t)b * n_cx + c] = range;
+}
+
 // MAXT: launch bound (512 leaves the compiler twice the registers; 1024 covers beam * topk up to 1024)
-template <int MAXT>
+// TRIE: the N-gram is the child-list trie (3-gram scores: search the context's children, located by the sweep).
+template <int MAXT, bool TRIE>
 __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
   extern __shared__ __align__(16) unsigned char tsm[];
   const int k = p.topk, w = p.beam, theta = p.budget - 1;
@@ -113,7 +183,8 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
   const int ctx0 = p.ctx_tail[2 * b], ctx1 = p.ctx_tail[2 * b + 1];
   const NgramTable T = p.table;
   const bool have_table = T.slots != nullptr;
-  const float* bg = p.bg + (size_t)b * (k + (p.n_levels - 1) * k * k);  // bigram scores from bigram_sweep_kernel
+  const float* bg = p.bg + (size_t)b * sweep_bigrams(k, p.n_levels);  // bigram scores from the sweep kernel
+  const uint2* cx = TRIE ? p.cx + (size_t)b * sweep_contexts(k, p.n_levels) : nullptr;
 
   if (tid == 0) {
     m.n_score[0] = 0.f; m.n_clamp[0] = INFINITY; m.n_tok[0] = ctx1; m.n_par[0] = -1; m.n_j[0] = 0;
@@ -137,7 +208,13 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
       const int ta = node == 0 ? ctx0 : m.n_tok[m.n_par[node]];
       const int t = ids[i * k + j];
       float s_ng = __ldg(bg + (i == 0 ? j : k + (i - 1) * k * k + (int)m.n_j[node] * k + j));
-      if (have_table && p.ngram_order >= 3 && ta >= 0 && tb >= 0) {
+      if (TRIE) {
+        const int jn = m.n_j[node];
+        const int c = i == 0 ? 0 : i == 1 ? 1 + jn : 1 + k + (i - 2) * k * k + (int)m.n_j[m.n_par[node]] * k + jn;
+        const uint2 range = __ldg(cx + c);
+        uint32_t pay, idx;
+        if (range.y > range.x && trie_find(p.trie.tri_ent, range.x, range.y, t, pay, idx)) s_ng = __uint_as_float(pay);
+      } else if (have_table && p.ngram_order >= 3 && ta >= 0 && tb >= 0) {
         const unsigned long long k3 = ngram_key(3, ta, tb, t);
         const uint32_t h3 = (uint32_t)ngram_hash(k3) & T.mask;
         float v;
@@ -275,17 +352,21 @@ cudaError_t tree_setup(int topk, int beam, int budget, int max_levels) {
   const size_t smem = tree_smem_bytes(topk, beam, budget, max_levels);
   if (smem > 48 * 1024)
   {
-    cudaError_t e = cudaFuncSetAttribute(tree_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(tree_kernel<1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(tree_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<1024, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<1024, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    return e;
   }
   return cudaSuccess;
 }
 
 cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
+  const bool trie = p.trie.bi_off != nullptr;
   {
-    const int n_bg = p.topk + (p.n_levels - 1) * p.topk * p.topk;
-    cudaError_t e = launch_pdl(bigram_sweep_kernel, dim3((n_bg + 255) / 256, p.B), dim3(256), 0, st, p);
+    const int n_bg = sweep_bigrams(p.topk, p.n_levels), n_cx = sweep_contexts(p.topk, p.n_levels);
+    cudaError_t e = trie ? launch_pdl(trie_sweep_kernel, dim3((n_bg + n_cx + 255) / 256, p.B), dim3(256), 0, st, p)
+                         : launch_pdl(bigram_sweep_kernel, dim3((n_bg + 255) / 256, p.B), dim3(256), 0, st, p);
     if (e != cudaSuccess) return e;
   }
   const size_t smem = tree_smem_bytes(p.topk, p.beam, p.budget, p.n_levels);
@@ -294,8 +375,12 @@ cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
   if (p.budget > need) need = p.budget;
   int threads = (need + 31) / 32 * 32;
   if (threads > 1024) threads = 1024;
-  if (threads <= 512) return launch_pdl(tree_kernel<512>, dim3(p.B), dim3(threads), smem, st, p);
-  return launch_pdl(tree_kernel<1024>, dim3(p.B), dim3(threads), smem, st, p);
+  if (trie) {
+    if (threads <= 512) return launch_pdl(tree_kernel<512, true>, dim3(p.B), dim3(threads), smem, st, p);
+    return launch_pdl(tree_kernel<1024, true>, dim3(p.B), dim3(threads), smem, st, p);
+  }
+  if (threads <= 512) return launch_pdl(tree_kernel<512, false>, dim3(p.B), dim3(threads), smem, st, p);
+  return launch_pdl(tree_kernel<1024, false>, dim3(p.B), dim3(threads), smem, st, p);
 }
 
 }  // namespace dart
