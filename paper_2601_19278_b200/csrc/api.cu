@@ -853,7 +853,7 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
   tp.table.slots = h->ng_slots; tp.table.mask = h->ng_mask; tp.table.max_probe = h->ng_max_probe;
   for (int i = 0; i < 8; ++i) { tp.wl[i] = h->wl[i]; tp.wv[i] = h->wv[i]; }
   tp.trie.bi_off = h->ng_trie.bi_off; tp.trie.bi_ent = h->ng_trie.bi_ent; tp.trie.tri_off = h->ng_trie.tri_off;
-  tp.trie.tri_node = h->ng_trie.tri_node; tp.trie.tri_ent = h->ng_trie.tri_ent;
+  tp.trie.tri_node = h->ng_trie.tri_node; tp.trie.tri_ent = h->ng_trie.tri_ent; tp.trie.nb8 = 8u * (uint32_t)((c.vocab + 479) / 480);
   tp.wn = h->wn; tp.miss = h->miss; tp.bg = h->ws.bg; tp.cx = h->ws.cx;
   tp.tokens = out->tokens; tp.parents = out->parents; tp.depth = out->depth; tp.mask = out->mask;
   tp.n_nodes = out->n_nodes; tp.scores = out->scores; tp.status = h->ws.status;

@@ -265,13 +265,18 @@ cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st);
 // ---------------------------------------------------------------------------------------------
 struct NgramSlot { unsigned long long key; float score; uint32_t pad; };  // 16 bytes; key 0 = empty
 struct NgramTable { const NgramSlot* slots; uint32_t mask; uint32_t max_probe; };
-// The same rows as child lists (Appendix C).  Every list is an array of {key, payload} pairs in ascending key
-// order and has at most `vocab` entries:
+// The same rows as child lists (Appendix C).  Every list is a run of {key, payload} slots in ascending key order:
 //   2-gram context b   -> bi_ent[bi_off[b] .. bi_off[b+1])             {next token, score bits}
-//   first token a      -> tri_node[tri_off[a] .. tri_off[a+1])         {second context token b, first child}
+//   first token a      -> tri_node[tri_off[a] .. tri_off[a+1])         {second context token b, first child}, then a
+//                                                                      sentinel {0x7fffffff, end of the last node's children}
 //   3-gram context j   -> tri_ent[tri_node[j].y .. tri_node[j+1].y)    {next token, score bits}
-// tri_node carries one sentinel entry after the last node.
-struct NgramTrie { const uint32_t* bi_off; const uint2* bi_ent; const uint32_t* tri_off; const uint2* tri_node; const uint2* tri_ent; };
+// A region may end in slots with key 0xffffffff (alignment filler).  A list of more than kTrieLongList slots is
+// long: its region starts on a 64-byte boundary with nb8 / 8 bitmap blocks of 16 words -- {entries before this
+// block, 480 bits: token 480 * block + r is in the list} -- followed by the list, so that the entry of token t is
+// slot nb8 + (entries before its block) + (set bits below r) of the region.  Regions of kTrieLongList + 7 slots or
+// fewer are short lists; anything larger starts with the bitmap.
+constexpr int kTrieLongList = 1016;
+struct NgramTrie { const uint32_t* bi_off; const uint2* bi_ent; const uint32_t* tri_off; const uint2* tri_node; const uint2* tri_ent; uint32_t nb8; };
 struct NgramTrieOwned { uint32_t* bi_off; uint2* bi_ent; uint32_t* tri_off; uint2* tri_node; uint2* tri_ent; size_t bytes; };
 // Host rows -> device child lists (rows must have been validated; 3-gram rows are skipped when ngram_order < 3;
 // of duplicate rows the first wins).  Synchronous; on failure everything allocated so far is released.

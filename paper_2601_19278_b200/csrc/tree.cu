@@ -47,34 +47,90 @@ __device__ __forceinline__ bool probe_rest(const NgramTable& T, unsigned long lo
   return false;
 }
 
-// Look `key` up in the sorted list ent[lo .. hi) of {key, payload} pairs (a child list of the trie, at most 2^21
-// entries).  A 16-ary search: every round reads 15 evenly spaced keys at once -- their latencies overlap, so a round
-// costs one memory round trip -- and keeps the sixteenth of the list that can hold the key; a list of 16 or fewer is
-// read whole.  1 round trip for the common short list, 5 for a list as long as the vocabulary.  The rounds are
-// bounded and every read stays inside [lo, hi), whatever the list holds.
-__device__ __forceinline__ bool trie_find(const uint2* __restrict__ ent, uint32_t lo, uint32_t hi, int key, uint32_t& payload, uint32_t& index) {
+// The entry of token t in a long list (region ent[lo ..), nb8 bitmap slots first): read t's 64-byte bitmap block,
+// test its bit, count the entries before it, read the entry -- two dependent reads whatever the list's length.
+__device__ __forceinline__ bool long_find(const uint2* __restrict__ ent, uint32_t lo, uint32_t nb8, int t, uint32_t& payload, uint32_t& index) {
+  const uint32_t blk = (uint32_t)t / 480u, r = (uint32_t)t - blk * 480u;
+  if (blk * 8u >= nb8) return false;                       // a token beyond the vocabulary
+  const uint4* bp = reinterpret_cast<const uint4*>(ent + lo + blk * 8u);
+  const uint4 q0 = __ldg(bp), q1 = __ldg(bp + 1), q2 = __ldg(bp + 2), q3 = __ldg(bp + 3);
+  const uint32_t w[16] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w, q2.x, q2.y, q2.z, q2.w, q3.x, q3.y, q3.z, q3.w};
+  const uint32_t word = 1u + (r >> 5), bit = r & 31u;
+  uint32_t rank = w[0], mine = 0u;
+#pragma unroll
+  for (uint32_t q = 1; q < 16; ++q) {
+    rank += q < word ? (uint32_t)__popc(w[q]) : 0u;
+    mine = q == word ? w[q] : mine;
+  }
+  if (((mine >> bit) & 1u) == 0u) return false;
+  rank += (uint32_t)__popc(mine & ((1u << bit) - 1u));
+  index = lo + nb8 + rank;
+  payload = __ldg(&ent[index]).y;
+  return true;
+}
+
+// The candidate tokens S_i of one level as a 64-slot open-addressing table in shared memory (k <= 32, so it is at
+// most half full): token -> the first position j that holds it.  Built and read by one warp or, with a barrier
+// between the two, by a block.
+// `filter` is a 2048-bit map of the tokens' low bits: nearly every child of a list is not a candidate, and one
+// read of the map says so.
+struct CandSet { int tok[64]; int j[64]; uint32_t filter[64]; };
+
+__device__ __forceinline__ uint32_t cand_slot(int t) { return ((uint32_t)t * 0x9E3779B1u) >> 26; }
+__device__ __forceinline__ void cand_clear(CandSet& s, int lane) {
+  s.tok[lane] = -1; s.tok[lane + 32] = -1; s.j[lane] = 0x7fffffff; s.j[lane + 32] = 0x7fffffff;
+  s.filter[lane] = 0u; s.filter[lane + 32] = 0u;
+}
+__device__ __forceinline__ bool cand_maybe(const CandSet& s, int t) { return (s.filter[((uint32_t)t >> 5) & 63u] >> ((uint32_t)t & 31u)) & 1u; }
+__device__ __forceinline__ void cand_insert(CandSet& s, int t, int j) {   // t >= 0
+  atomicOr(&s.filter[((uint32_t)t >> 5) & 63u], 1u << ((uint32_t)t & 31u));
+  uint32_t h = cand_slot(t);
+  for (int probe = 0; probe < 64; ++probe, h = (h + 1) & 63u) {
+    const int old = atomicCAS(&s.tok[h], -1, t);
+    if (old == -1 || old == t) { atomicMin(&s.j[h], j); return; }
+  }
+}
+__device__ __forceinline__ int cand_find(const CandSet& s, int t) {       // first j with token t, or -1
+  uint32_t h = cand_slot(t);
+  for (int probe = 0; probe < 64; ++probe, h = (h + 1) & 63u) {
+    const int v = s.tok[h];
+    if (v == t) return s.j[h];
+    if (v == -1) return -1;
+  }
+  return -1;
+}
+
+// One warp intersects the child list in region ent[lo .. hi) with a candidate set (Appendix C: the context's node is
+// reached once, its children are then read for all candidates).  A short list is read whole, 32 consecutive slots
+// per instruction and sixteen instructions in flight together -- as many requests as the list has cache lines,
+// one memory round trip per 512 slots, two at most -- and every child is looked up in the set.  In a long list
+// each candidate's entry is found through the list's bitmap instead: lane j looks for my_t (its candidate's token
+// where j is the token's first position, else -1).
+// emit(j, payload, index) is called once per candidate token found, with j its first position.
+// DEPTH: reads in flight per lane.
+template <int DEPTH, typename Match, typename Emit>
+__device__ __forceinline__ void warp_list_match(const uint2* __restrict__ ent, uint32_t lo, uint32_t hi, uint32_t nb8, Match match, int my_t,
+                                                int lane, Emit emit) {
+  if (hi <= lo) return;
+  if (hi - lo <= (uint32_t)kTrieLongList + 7u) {
 #pragma unroll 1
-  for (int round = 0; round < 6 && hi - lo > 16u; ++round) {
-    const uint32_t n = hi - lo;
-    int piv[15];
+    for (uint32_t base = lo; base < hi; base += 32u * DEPTH) {
+      uint2 v[DEPTH];
 #pragma unroll
-    for (int q = 0; q < 15; ++q) piv[q] = (int)__ldg(&ent[lo + ((n * (uint32_t)(q + 1)) >> 4)].x);
-    uint32_t c = 0;
+      for (int u = 0; u < DEPTH; ++u) {
+        const uint32_t idx = base + (uint32_t)(u * 32 + lane);
+        v[u] = idx < hi ? __ldg(&ent[idx]) : make_uint2(0xffffffffu, 0u);
+      }
 #pragma unroll
-    for (int q = 0; q < 15; ++q) c += piv[q] <= key ? 1u : 0u;
-    const uint32_t nlo = lo + ((n * c) >> 4), nhi = c < 15u ? lo + ((n * (c + 1u)) >> 4) : hi;
-    lo = nlo; hi = nhi;
-  }
-  bool found = false;
-#pragma unroll
-  for (int q = 0; q < 16; ++q) {
-    const uint32_t idx = lo + (uint32_t)q;
-    if (idx < hi) {
-      const uint2 v = __ldg(&ent[idx]);
-      if ((int)v.x == key) { found = true; payload = v.y; index = idx; }
+      for (int u = 0; u < DEPTH; ++u) {
+        const int j = (int)v[u].x >= 0 ? match((int)v[u].x) : -1;
+        if (j >= 0) emit(j, v[u].y, base + (uint32_t)(u * 32 + lane));
+      }
     }
+  } else if (my_t >= 0) {
+    uint32_t pay, idx;
+    if (long_find(ent, lo, nb8, my_t, pay, idx)) emit(lane, pay, idx);
   }
-  return found;
 }
 
 // Sizes of the per-sequence sweep outputs: bigram scores and 3-gram context ranges for `levels` levels.
@@ -84,6 +140,10 @@ __host__ __device__ inline int sweep_contexts(int k, int levels) { return 1 + (l
 struct TreeSmem {
   float* n_score; float* n_clamp; int* n_tok; int* n_par; unsigned char* n_j;
   Key* xk; int* beam_a; int* beam_b; int* sel; int* par_out; int* lvl_base;
+  // trie layout: per level the candidate set and every candidate's first position; per (beam entry, candidate)
+  // the 3-gram score bits and per beam entry the mask of candidates that have one, double-buffered by level
+  CandSet* sets; unsigned char* fj; uint32_t* s3; uint32_t* hit;
+  uint2* cxs;   // [2][k*k] child ranges of the contexts the next level can ask for, copied in one level ahead
 };
 
 __host__ __device__ inline size_t tree_layout(int k, int w, int budget, int L, unsigned char* base, TreeSmem* t) {
@@ -93,8 +153,13 @@ __host__ __device__ inline size_t tree_layout(int k, int w, int budget, int L, u
   const size_t o_score = take((size_t)n_max * 4), o_clamp = take((size_t)n_max * 4), o_tok = take((size_t)n_max * 4),
                o_par = take((size_t)n_max * 4), o_j = take((size_t)n_max),
                o_xk = take(32 * 64 * 8), o_ba = take((size_t)w * 4), o_bb = take((size_t)w * 4),
-               o_sel = take((size_t)(budget + 1) * 4), o_po = take((size_t)budget * 4), o_lb = take((size_t)(L + 1) * 4);
+               o_sel = take((size_t)(budget + 1) * 4), o_po = take((size_t)budget * 4), o_lb = take((size_t)(L + 1) * 4),
+               o_sets = take((size_t)L * sizeof(CandSet)), o_fj = take((size_t)L * k), o_s3 = take((size_t)2 * w * k * 4),
+               o_hit = take(2 * 32 * 4), o_cxs = take((size_t)2 * k * k * 8);
   if (t != nullptr) {
+    t->sets = reinterpret_cast<CandSet*>(base + o_sets); t->fj = base + o_fj;
+    t->s3 = reinterpret_cast<uint32_t*>(base + o_s3); t->hit = reinterpret_cast<uint32_t*>(base + o_hit);
+    t->cxs = reinterpret_cast<uint2*>(base + o_cxs);
     t->n_score = reinterpret_cast<float*>(base + o_score); t->n_clamp = reinterpret_cast<float*>(base + o_clamp);
     t->n_tok = reinterpret_cast<int*>(base + o_tok); t->n_par = reinterpret_cast<int*>(base + o_par);
     t->n_j = base + o_j;
@@ -130,39 +195,67 @@ __global__ void __launch_bounds__(256) bigram_sweep_kernel(const TreeParams p) {
   p.bg[(size_t)b * n_bg + e] = sc;
 }
 
-// The sweep for the trie layout.  Besides the bigram scores (a search of context b's child list for t) it locates
-// the node of every 3-gram context a level can ask for -- (c_-2, c_-1) for level 0, (c_-1, S_0[j]) for level 1,
-// (S_{i-2}[j'], S_{i-1}[j]) for level i -- once, and leaves the range of its children in cx, laid out like bg:
-// cx[b][0], cx[b][1 + j], cx[b][1 + k + (i-2)k^2 + j'k + j].  A context that is absent gets the empty range.
+// The sweep for the trie layout: one warp per (level i, list kind, context position jb).  The context token x is
+// c_-1 for level 0 and S_{i-1}[jb] after it; the warp intersects one of x's two child lists with S_i:
+//   kind 0  the 2-gram children of x        -> bg, the bigram scores (x, S_i[j]);
+//   kind 1  the 3-gram context nodes (x, .) -> cx, the child ranges of the contexts (x, S_i[j]) that level i+1 can
+//           ask for, laid out like bg: cx[b][0] = (c_-2, c_-1), cx[b][1 + j] = (c_-1, S_0[j]),
+//           cx[b][1 + k + (i-1)k^2 + jb k + j] = (S_{i-1}[jb], S_i[j]).  An absent context gets the empty range.
 __global__ void __launch_bounds__(256) trie_sweep_kernel(const TreeParams p) {
+  __shared__ CandSet s_set[8];
   pdl_wait();
-  const int k = p.topk, b = blockIdx.y;
+  const int k = p.topk, b = blockIdx.y, lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int fr = p.first_rows[b], Lb = min(p.n_levels, p.K - fr);
-  const int n_bg = sweep_bigrams(k, p.n_levels), n_cx = sweep_contexts(k, p.n_levels);   // layout strides: the launch's maximum
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  const int task = blockIdx.x * 8 + wib;                 // ((i * 2) + kind) * k + jb
+  const int i = task / (2 * k), kind = (task - i * 2 * k) / k, jb = task - (i * 2 + kind) * k;
+  if (i >= Lb || (i == 0 && jb > 0)) return;
   const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
   const NgramTrie T = p.trie;
-  uint32_t pay, idx;
-  if (e < n_bg) {
-    if (e >= sweep_bigrams(k, Lb)) return;
-    int tb, tt;
-    if (e < k) { tb = p.ctx_tail[2 * b + 1]; tt = ids[e]; }
-    else { const int r = e - k, i = r / (k * k), q = r - i * k * k, jb = q / k; tb = ids[i * k + jb]; tt = ids[(i + 1) * k + q - jb * k]; }
-    float sc = p.miss;
-    if (tb >= 0 && tb < p.vocab && trie_find(T.bi_ent, __ldg(T.bi_off + tb), __ldg(T.bi_off + tb + 1), tt, pay, idx)) sc = __uint_as_float(pay);
-    p.bg[(size_t)b * n_bg + e] = sc;
-    return;
+  float* bg = p.bg + (size_t)b * sweep_bigrams(k, p.n_levels);
+  uint2* cx = p.cx + (size_t)b * sweep_contexts(k, p.n_levels);
+  const bool tri = p.ngram_order >= 3;
+  if (kind == 1 && i == 0) {                             // the context of level 0
+    const int ta = p.ctx_tail[2 * b], tb = p.ctx_tail[2 * b + 1];
+    if (lane == 0) cx[0] = make_uint2(0u, 0u);
+    __syncwarp();
+    if (tri && ta >= 0 && ta < p.vocab && tb >= 0)
+      warp_list_match<16>(T.tri_node, __ldg(T.tri_off + ta), __ldg(T.tri_off + ta + 1), T.nb8, [&](int tok) { return tok == tb ? 0 : -1; },
+                      lane == 0 ? tb : -1, lane, [&](int, uint32_t pay, uint32_t idx) {
+                        const uint2 range = make_uint2(pay, __ldg(&T.tri_node[idx + 1]).y);
+                        cx[0] = range;
+                      });
   }
-  const int c = e - n_bg;
-  if (c >= sweep_contexts(k, Lb)) return;
-  int ta, tb;
-  if (c == 0) { ta = p.ctx_tail[2 * b]; tb = p.ctx_tail[2 * b + 1]; }
-  else if (c < 1 + k) { ta = p.ctx_tail[2 * b + 1]; tb = ids[c - 1]; }
-  else { const int r = c - 1 - k, i2 = r / (k * k), q = r - i2 * k * k, jp = q / k; ta = ids[i2 * k + jp]; tb = ids[(i2 + 1) * k + q - jp * k]; }
-  uint2 range = make_uint2(0u, 0u);
-  if (p.ngram_order >= 3 && ta >= 0 && ta < p.vocab && tb >= 0 && trie_find(T.tri_node, __ldg(T.tri_off + ta), __ldg(T.tri_off + ta + 1), tb, pay, idx))
-    range = make_uint2(pay, __ldg(&T.tri_node[idx + 1]).y);
-  p.cx[(size_t)b * n_cx + c] = range;
+  if (kind == 1 && i + 1 >= Lb) return;                  // no level left to ask for these contexts
+  const int x = i == 0 ? p.ctx_tail[2 * b + 1] : ids[(i - 1) * k + jb];
+  const int t = lane < k ? ids[i * k + lane] : -1;
+  CandSet& set = s_set[wib];
+  cand_clear(set, lane);
+  __syncwarp();
+  if (t >= 0) cand_insert(set, t, lane);
+  __syncwarp();
+  const int fj = t >= 0 ? cand_find(set, t) : lane;      // first position of this lane's token
+  const bool have = x >= 0 && x < p.vocab && (kind == 0 || tri);
+  if (kind == 0) {
+    float* out = bg + (i == 0 ? 0 : k + (i - 1) * k * k + jb * k);
+    if (lane < k) out[lane] = p.miss;
+    __syncwarp();
+    if (have)
+      warp_list_match<16>(T.bi_ent, __ldg(T.bi_off + x), __ldg(T.bi_off + x + 1), T.nb8, [&](int tok) { return cand_maybe(set, tok) ? cand_find(set, tok) : -1; }, fj == lane ? t : -1, lane,
+                                [&](int j, uint32_t pay, uint32_t) { out[j] = __uint_as_float(pay); });
+    __syncwarp();
+    if (lane < k && fj != lane) out[lane] = out[fj];     // a repeated token takes its first position's score
+  } else {
+    uint2* out = cx + (i == 0 ? 1 : 1 + k + (i - 1) * k * k + jb * k);
+    if (lane < k) out[lane] = make_uint2(0u, 0u);
+    __syncwarp();
+    if (have)
+      warp_list_match<16>(T.tri_node, __ldg(T.tri_off + x), __ldg(T.tri_off + x + 1), T.nb8, [&](int tok) { return cand_maybe(set, tok) ? cand_find(set, tok) : -1; }, fj == lane ? t : -1, lane,
+                                [&](int j, uint32_t pay, uint32_t idx) {
+                                  out[j] = make_uint2(pay, __ldg(&T.tri_node[idx + 1]).y);
+                                });
+    __syncwarp();
+    if (lane < k && fj != lane) out[lane] = out[fj];
+  }
 }
 
 // MAXT: launch bound (512 leaves the compiler twice the registers; 1024 covers beam * topk up to 1024)
@@ -190,6 +283,20 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
     m.n_score[0] = 0.f; m.n_clamp[0] = INFINITY; m.n_tok[0] = ctx1; m.n_par[0] = -1; m.n_j[0] = 0;
     m.beam_a[0] = 0; m.lvl_base[0] = 1;
   }
+  if (TRIE) {   // candidate sets of all levels: warp l builds level l's (l, l + warps, ...)
+    const int nwarp = nthr >> 5;
+    for (int l = warp; l < L; l += nwarp) {
+      cand_clear(m.sets[l], lane);
+      __syncwarp();
+      const int t = lane < k ? ids[l * k + lane] : -1;
+      if (t >= 0) cand_insert(m.sets[l], t, lane);
+      __syncwarp();
+      if (lane < k) m.fj[l * k + lane] = (unsigned char)(t >= 0 ? cand_find(m.sets[l], t) : lane);
+    }
+    for (int e = tid; e < 64; e += nthr) m.hit[e] = 0u;
+    if (tid == 0) m.cxs[0] = __ldg(cx);   // level 0's only context
+    __syncthreads();
+  }
   // running global best 64 by (clamped score desc, node index asc); lives in warp 0's registers
   Key g0 = kPadKey, g1 = kPadKey;
 
@@ -201,6 +308,28 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
     const int base = m.lvl_base[i];
     const int nruns = (ncand + 31) >> 5;
     float s = -INFINITY, cl = -INFINITY;
+    uint32_t* s3 = m.s3 + (i & 1) * w * k;
+    uint32_t* hit = m.hit + (i & 1) * 32;
+    // the ranges level i+1 can ask for, on their way to shared memory while this level is scored
+    const int n_pre = !TRIE || i + 1 >= L ? 0 : i == 0 ? k : k * k;
+    const uint2* pre_src = TRIE ? cx + (i == 0 ? 1 : 1 + k + (i - 1) * k * k) : nullptr;
+    uint2 pre0 = make_uint2(0u, 0u), pre1 = pre0;
+    if (tid < n_pre) pre0 = __ldg(pre_src + tid);
+    if (tid + nthr < n_pre) pre1 = __ldg(pre_src + tid + nthr);
+    if (TRIE) {   // one warp per beam entry: the children of its context, located by the sweep, against S_i
+      const int nwarp = nthr >> 5;
+      const uint2* cxs = m.cxs + (i & 1) * k * k;
+      for (int rho = warp; rho < nb; rho += nwarp) {
+        const int node = beam[rho], jn = m.n_j[node];
+        const uint2 range = cxs[i == 0 ? 0 : i == 1 ? jn : (int)m.n_j[m.n_par[node]] * k + jn];
+        const int my_t = (lane < k && m.fj[i * k + lane] == lane) ? ids[i * k + lane] : -1;
+        warp_list_match<16>(p.trie.tri_ent, range.x, range.y, p.trie.nb8, [&](int tok) { return cand_maybe(m.sets[i], tok) ? cand_find(m.sets[i], tok) : -1; }, my_t, lane, [&](int j, uint32_t pay, uint32_t) {
+          s3[rho * k + j] = pay;
+          atomicOr(&hit[rho], 1u << j);
+        });
+      }
+      __syncthreads();
+    }
     if (tid < ncand) {
       const int rho = tid / k, j = tid - rho * k;
       const int node = beam[rho];
@@ -209,11 +338,8 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
       const int t = ids[i * k + j];
       float s_ng = __ldg(bg + (i == 0 ? j : k + (i - 1) * k * k + (int)m.n_j[node] * k + j));
       if (TRIE) {
-        const int jn = m.n_j[node];
-        const int c = i == 0 ? 0 : i == 1 ? 1 + jn : 1 + k + (i - 2) * k * k + (int)m.n_j[m.n_par[node]] * k + jn;
-        const uint2 range = __ldg(cx + c);
-        uint32_t pay, idx;
-        if (range.y > range.x && trie_find(p.trie.tri_ent, range.x, range.y, t, pay, idx)) s_ng = __uint_as_float(pay);
+        const int f = m.fj[i * k + j];
+        if ((hit[rho] >> f) & 1u) s_ng = __uint_as_float(s3[rho * k + f]);
       } else if (have_table && p.ngram_order >= 3 && ta >= 0 && tb >= 0) {
         const unsigned long long k3 = ngram_key(3, ta, tb, t);
         const uint32_t h3 = (uint32_t)ngram_hash(k3) & T.mask;
@@ -226,6 +352,13 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
       cl = s < pc ? s : pc;
       const int n = base + tid;
       m.n_score[n] = s; m.n_clamp[n] = cl; m.n_tok[n] = t; m.n_par[n] = node; m.n_j[n] = (unsigned char)j;
+    }
+    if (TRIE) {
+      if (tid < 32) m.hit[((i + 1) & 1) * 32 + tid] = 0u;   // the next level's masks (read two barriers from now)
+      uint2* nxt = m.cxs + ((i + 1) & 1) * k * k;
+      if (tid < n_pre) nxt[tid] = pre0;
+      if (tid + nthr < n_pre) nxt[tid + nthr] = pre1;
+      for (int e = tid + 2 * nthr; e < n_pre; e += nthr) nxt[e] = __ldg(pre_src + e);
     }
     // keys carry the node index base + tid, which orders candidates of one level like tid does
     // best 64 by score -> next beam; `differs`: some clamped score is not its score (never, when increments <= 0)
@@ -364,8 +497,9 @@ cudaError_t tree_setup(int topk, int beam, int budget, int max_levels) {
 cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
   const bool trie = p.trie.bi_off != nullptr;
   {
-    const int n_bg = sweep_bigrams(p.topk, p.n_levels), n_cx = sweep_contexts(p.topk, p.n_levels);
-    cudaError_t e = trie ? launch_pdl(trie_sweep_kernel, dim3((n_bg + n_cx + 255) / 256, p.B), dim3(256), 0, st, p)
+    const int n_bg = sweep_bigrams(p.topk, p.n_levels);
+    const int n_task = p.n_levels * 2 * p.topk;   // trie layout: one warp per (level, list kind, context position)
+    cudaError_t e = trie ? launch_pdl(trie_sweep_kernel, dim3((n_task + 7) / 8, p.B), dim3(256), 0, st, p)
                          : launch_pdl(bigram_sweep_kernel, dim3((n_bg + 255) / 256, p.B), dim3(256), 0, st, p);
     if (e != cudaSuccess) return e;
   }
@@ -373,6 +507,7 @@ cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
   // one thread per (beam entry, candidate) pair; a smaller block makes every barrier cheaper
   int need = p.beam * p.topk;
   if (p.budget > need) need = p.budget;
+  if (trie && 32 * p.beam > need) need = 32 * p.beam;   // one warp per beam entry reads its context's children
   int threads = (need + 31) / 32 * 32;
   if (threads > 1024) threads = 1024;
   if (trie) {

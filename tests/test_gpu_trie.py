@@ -22,6 +22,11 @@ def _session(batch, K, topk=25, beam=20, budget=60, rows=None, vocab=VOCAB, **cf
 
 def _gpu_tree(ses, ids, sl, ctx, first_row=0, n_levels=None):
     dev = ses.dev
+    # a first call on other candidates, so that nothing a call leaves in the library's workspace can stand in for the next one's work
+    ses.draft.build_tree(batch=ids.shape[0], topk_ids=torch.from_numpy(np.ascontiguousarray(ids[:, ::-1, ::-1])).to(dev),
+                         topk_slogit=torch.from_numpy(sl).to(dev), ctx_tail=torch.from_numpy(np.ascontiguousarray(ctx[:, ::-1])).to(dev),
+                         tokens=ses.tokens, parents=ses.parents, depth=ses.depth, mask=ses.mask, n_nodes=ses.n_nodes, scores=ses.scores,
+                         first_row=first_row, n_levels=n_levels)
     ses.draft.build_tree(batch=ids.shape[0], topk_ids=torch.from_numpy(ids).to(dev), topk_slogit=torch.from_numpy(sl).to(dev),
                          ctx_tail=torch.from_numpy(ctx).to(dev), tokens=ses.tokens, parents=ses.parents, depth=ses.depth,
                          mask=ses.mask, n_nodes=ses.n_nodes, scores=ses.scores, first_row=first_row, n_levels=n_levels)
@@ -43,22 +48,24 @@ def test_paper_settings_bit_exact_and_smaller_than_the_hash(seed, budget, order)
         sizes[name] = ses.draft.ngram_bytes()
         ses.close()
     n_kept = len(bi) + (len(tri) if order == 3 else 0)
-    assert 8 * n_kept <= sizes["trie"] <= 16 * n_kept + 8 * (VOCAB + 2) + 64
+    n_long_max = n_kept // 1017 + 1                      # lists long enough to carry a bitmap (64 bytes per 480 tokens, + filler)
+    assert 8 * n_kept <= sizes["trie"] <= 16 * n_kept + 16 * (VOCAB + 2) + n_long_max * (64 * 5 + 56)
     assert sizes["hash"] >= 32 * n_kept and sizes["trie"] < sizes["hash"] / 2
 
 
 @pytest.mark.parametrize("vocab", [2048, 32768])
 def test_vocabulary_long_child_lists(vocab):
-    """Child lists of every length class of the 16-ary search (1, 16, 17, 300, the whole vocabulary), candidates on
-    their first and last entries and between entries, each row with a score of its own."""
+    """Child lists of every length class (1 entry, a few, both sides of the long-list threshold of 1016, the whole
+    vocabulary), candidates on their first and last entries, between entries and on both sides of the 480-token
+    blocks of a long list's bitmap, each row with a score of its own."""
     rng = np.random.default_rng(vocab)
-    ctxs = [3, 9, 100, 777, vocab - 1]
-    lens = [vocab, 300, 17, 16, 1]
+    ctxs = [3, 9, 100, 777, vocab - 1, 11, 12]
+    lens = [vocab, 300, 17, 1016, 1, 1017, 1024]
     rows = []
     for b, n in zip(ctxs, lens):                        # 2-gram lists under b
         for t in np.sort(rng.choice(vocab, n, replace=False)) if n < vocab else range(vocab):
             rows.append((2, -1, b, int(t)))
-    for a, b, n in [(3, 9, vocab), (9, 3, 300), (100, 100, 17), (777, 3, 16), (vocab - 1, 9, 1)]:   # 3-gram lists under (a, b)
+    for a, b, n in [(3, 9, vocab), (9, 3, 300), (100, 100, 17), (777, 3, 1016), (vocab - 1, 9, 1), (11, 12, 1017), (12, 11, 1500)]:   # 3-gram lists under (a, b)
         for t in np.sort(rng.choice(vocab, n, replace=False)) if n < vocab else range(vocab):
             rows.append((3, a, b, int(t)))
     for b in range(0, vocab, 2):                        # token 9 is the first token of vocab/2 context nodes
@@ -70,7 +77,7 @@ def test_vocabulary_long_child_lists(vocab):
     tri, bi = otree.tables_from_rows(base)
     B, K, k = 3, 8, 25
     ids = np.zeros((B, K, k), dtype=np.int32)
-    pool = np.array(ctxs + [0, 1, 2, 5, vocab - 2, vocab // 2, 15, 16, 17, 299, 300, 301], dtype=np.int32)
+    pool = np.array(ctxs + [0, 1, 5, vocab - 2, vocab // 2, 479, 480, 481, 959, 960, 31, 32], dtype=np.int32)
     for b in range(B):
         for i in range(K):
             rest = rng.choice(np.setdiff1d(np.arange(vocab, dtype=np.int32), pool), k - len(pool), replace=False)
@@ -78,7 +85,7 @@ def test_vocabulary_long_child_lists(vocab):
             rng.shuffle(row)
             ids[b, i] = row
     sl = (-rng.random((B, K, k)) * 3).astype(np.float32)
-    ctx = np.array([[3, 9], [9, 3], [-1, vocab - 1]], dtype=np.int32)
+    ctx = np.array([[3, 9], [11, 12], [-1, vocab - 1]], dtype=np.int32)
     ref = parity.oracle_tree_batch(ids, sl, ctx, tri, bi, beam=20, budget=60)
     for over in (TRIE, {}):
         w, ses = _session(B, K, rows=base, vocab=vocab, **over)
