@@ -169,8 +169,9 @@ def run_ours(args):
         w = syn.small_variant(w, vocab=args.vocab, name=f"{w.name} with vocab cut to {args.vocab}")
     wt = syn.make_weights(w)
     inp = syn.make_step_inputs(w, n_fresh=syn.draw_fresh_counts(w) if args.ragged_fresh else None)
-    rows = syn.make_ngram_rows(w.vocab, w.ngram_rows, w.ngram_mode)
-    ses = runner.DraftSession(w, wt, rows, device=f"cuda:{local}", want_logits=False)
+    rows = syn.make_ngram_rows(w.vocab, args.ngram_rows or w.ngram_rows, w.ngram_mode)
+    ses = runner.DraftSession(w, wt, rows, device=f"cuda:{local}", want_logits=False,
+                              ngram_layout={"hash": 0, "trie": 1}[args.ngram_layout])
     ses.load_inputs(inp)
     stream = torch.cuda.current_stream()
     any_fresh = int(np.max(inp["n_fresh"])) > 0
@@ -273,7 +274,8 @@ def run_ours(args):
                                    f"topk {w.topk}, beam {w.beam}, budget {w.tree_budget}, ngram_rows {len(rows['next'])}, T={w.temperature}",
                        "parallelism": "replicas only" if world > 1 else "1 GPU",
                        "l2": f"inputs larger than L2: {bytes_step / 1e9:.3f} GB of weights+KV streamed per step",
-                       "feature_fc_in_path": any_fresh},
+                       "feature_fc_in_path": any_fresh,
+                       "ngram": f"{args.ngram_layout} layout, {ses.draft.ngram_bytes() / 1e6:.1f} MB in HBM"},
             "latency_us": {"p50": 1e3 * statistics.median(per_step), "p10": 1e3 * float(np.percentile(per_step, 10)),
                            "p90": 1e3 * float(np.percentile(per_step, 90)), "min": 1e3 * min(per_step), "max": 1e3 * max(per_step)},
             "stages_us": stages_us,
@@ -396,6 +398,9 @@ def main():
     ap.add_argument("--ragged-fresh", action="store_true",
                     help="per-sequence fresh-row counts (a steady-state call after a verification that accepted a different "
                          "number of tokens per sequence) instead of the workload's uniform count")
+    ap.add_argument("--ngram-layout", default="hash", choices=["hash", "trie"],
+                    help="device layout of the N-gram: open-addressing hash table, or child lists (Appendix C's trie)")
+    ap.add_argument("--ngram-rows", type=int, default=0, help="generate this many N-gram rows instead of the workload's count")
     ap.add_argument("--lm-traffic", type=float, default=None,
                     help="DRAM bytes per LM-head launch from the committed ncu capture (profiles/), reported as roofline.traffic")
     args = ap.parse_args()
