@@ -224,6 +224,41 @@ const char* dart_status_string(int status);
 /* Bytes of device workspace a handle for `cfg` allocates (excluding the N-gram table); 0 if cfg is invalid. */
 size_t dart_workspace_bytes(const dart_config* cfg);
 
+/*
+ * Forward attention under the prefix-shared training mask (Section 3.3 "Prefix-shared masked training", Appendix B).
+ * A packed row has L = prompt_len * (1 + draft_len) slots: prompt_len clean positions, then one block of draft_len
+ * masked positions per prefix position n.  Clean slot q reads clean slots <= q; block n reads clean slots 0..n and
+ * its own slots up to the reading one; blocks never read each other.  Slots past seq_lens_host[b] (clean slots >= it,
+ * blocks of prefix positions >= it) read nothing and give zero rows.  Grouped-query heads: head j reads KV head
+ * j / (n_q_heads / n_kv_heads).  Softmax scale 1 / sqrt(head_dim).
+ */
+typedef struct dart_train_attn_in {
+  int32_t batch;             /* 1..64 */
+  int32_t n_q_heads, n_kv_heads;
+  int32_t head_dim;          /* 128 */
+  int32_t prompt_len;        /* clean positions per packed row, >= 1 */
+  int32_t draft_len;         /* d, 1..16 */
+  const void* q;             /* DEVICE bf16 [batch, n_q_heads, L, head_dim], 16-byte aligned; RoPE already applied */
+  const void* k;             /* DEVICE bf16 [batch, n_kv_heads, L, head_dim] */
+  const void* v;             /* DEVICE bf16 [batch, n_kv_heads, L, head_dim] */
+  const int32_t* seq_lens_host; /* HOST [batch]: valid prompt slots, 0..prompt_len */
+  void* out;                 /* DEVICE bf16 [batch, n_q_heads, L, head_dim]; every row is written */
+  void* workspace;           /* DEVICE, dart_train_attention_workspace_bytes(...) bytes, 256-byte aligned; holds V^T */
+  size_t workspace_bytes;
+  int32_t* status;           /* DEVICE, may be NULL: set to a negative code if a bounded wait inside the kernel ran out */
+} dart_train_attn_in;
+
+/* Bytes of workspace dart_train_attention_fwd needs; 0 for arguments it does not accept. */
+size_t dart_train_attention_workspace_bytes(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int32_t prompt_len,
+                                            int32_t draft_len);
+
+/*
+ * Enqueues the attention on `cuda_stream` (two kernels: a transpose of v into the workspace, then the attention).
+ * Needs no handle.  Errors: INVALID_ARG (NULL or misaligned pointers, sizes out of range, head_dim != 128),
+ * CAPACITY (workspace too small), UNSUPPORTED_ARCH, CUDA.
+ */
+int dart_train_attention_fwd(const dart_train_attn_in* in, void* cuda_stream);
+
 /* Bytes of device memory the N-gram of this handle occupies in its layout (0 without an N-gram or handle). */
 size_t dart_ngram_bytes(const dart_handle* h);
 
