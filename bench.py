@@ -354,6 +354,61 @@ def run_prefill(args):
     ses.close()
 
 
+def run_train_attn(args):
+    """Forward attention under the prefix-shared training mask (dart_train_attention_fwd) for one packed row of
+    --train-attn-prompt clean positions with the workload's heads and K = draft length.  Compute-bound: the flop
+    count is 4 * head_dim per visible (query, key) pair and query head -- the mask's own work, nothing for the
+    hidden part -- against the measured bf16 peak."""
+    import torch
+    from paper_2601_19278_b200 import binding, replicas, synthetic as syn
+    world, rank, local = replicas.env()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    w = syn.WORKLOADS[args.workload]
+    Lp, d, Hq, Hkv, dh, B = args.train_attn_prompt, w.K, w.n_q_heads, w.n_kv_heads, w.head_dim, 1
+    L = Lp * (1 + d)
+    g = torch.Generator().manual_seed(11)
+    q = torch.randn(B, Hq, L, dh, generator=g).to(torch.bfloat16).to(dev)
+    k = torch.randn(B, Hkv, L, dh, generator=g).to(torch.bfloat16).to(dev)
+    v = torch.randn(B, Hkv, L, dh, generator=g).to(torch.bfloat16).to(dev)
+    out = torch.empty_like(q)
+    ws = torch.empty(binding.train_attention_workspace_bytes(B, Hkv, dh, Lp, d), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    call = lambda: binding.train_attention_fwd(q, k, v, [Lp] * B, Lp, d, out, ws, status)
+    for _ in range(max(args.warmup, 3)):
+        call()
+    torch.cuda.synchronize()
+    steps = min(args.steps, 20)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        call()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ms = e0.elapsed_time(e1) / steps
+    pairs = Lp * (Lp + 1) // 2 + d * Lp * (Lp + 1) // 2 + Lp * d * (d + 1) // 2      # clean causal + blocks x prefix + inside blocks
+    flop = 4.0 * dh * pairs * Hq * B
+    peak, sustained, kind = 1590.0, None, "fallback"
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        dd = json.load(open(pk))
+        if "bf16_tflops" in dd:
+            peak, kind = float(dd["bf16_tflops"]), "measured"
+        sustained = dd.get("bf16_tflops_sustained")
+    if rank == 0:
+        print(json.dumps({
+            "metric": "train_attention_fwd_rows_per_second", "value": B * L / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1, "steps": steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{w.name} heads ({Hq}q/{Hkv}kv x{dh}): one packed training row, {Lp} clean positions + {Lp} blocks of {d} masked positions = {L} slots; inputs larger than L2: {q.numel() * 2 * 2 / 1e6 + k.numel() * 4 / 1e6:.0f} MB"},
+            "roofline": {"bound": "tensor", "achieved": flop / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                         "frac": flop / (ms * 1e-3) / 1e12 / peak, "peak_kind": f"of {kind} (burst; sustained {sustained})",
+                         "traffic": None, "kernel": "train_attn_kernel (+ one transpose of V)", "flop_visible_pairs": flop},
+        }))
+
+
 def cpu_baseline(w, wt, inp, rows):
     """The oracle timed on this machine's host cores on one full step of the same workload."""
     import torch
@@ -395,6 +450,8 @@ def main():
                     help="override the workload's vocabulary (a smaller case of the same kernels, for ncu captures)")
     ap.add_argument("--prefill-rows", type=int, default=0,
                     help="time dart_draft_prefill on this many new prefix rows instead of the drafting step")
+    ap.add_argument("--train-attn-prompt", type=int, default=0,
+                    help="time dart_train_attention_fwd on one packed training row of this many clean positions instead of the drafting step")
     ap.add_argument("--ragged-fresh", action="store_true",
                     help="per-sequence fresh-row counts (a steady-state call after a verification that accepted a different "
                          "number of tokens per sequence) instead of the workload's uniform count")
@@ -408,6 +465,8 @@ def main():
         args.warmup = 3
     if args.prefill_rows > 0 and args.impl == "ours":
         run_prefill(args)
+    elif args.train_attn_prompt > 0 and args.impl == "ours":
+        run_train_attn(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -802,7 +802,7 @@ int dart_train_attention_fwd(const dart_train_attn_in* in, void* cuda_stream) {
   TrainAttnArgs a;
   memset(&a, 0, sizeof(a));
   if ((e = tmap_encode_bf16(&a.mapQ, in->q, 128, (unsigned long long)B * Hq * L, 256, 64, 128)) != cudaSuccess ||
-      (e = tmap_encode_bf16(&a.mapK, in->k, 128, (unsigned long long)B * Hkv * L, 256, 64, 128)) != cudaSuccess ||
+      (e = tmap_encode_bf16(&a.mapK, in->k, 128, (unsigned long long)B * Hkv * L, 256, 64, 64)) != cudaSuccess ||
       (e = tmap_encode_bf16(&a.mapVc, vt_c, ldc, (unsigned long long)B * Hkv * 128, ldc * 2, 64, 128)) != cudaSuccess ||
       (e = tmap_encode_bf16(&a.mapVm, vt_m, ldm, (unsigned long long)B * Hkv * 128, ldm * 2, 64, 128)) != cudaSuccess)
     return e == cudaErrorNotSupported ? DART_ERR_UNSUPPORTED_ARCH : fail_cuda(nullptr, e);

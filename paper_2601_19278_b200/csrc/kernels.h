@@ -267,7 +267,7 @@ cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st);
 // 120 / d, which leaves room for the up-to-7-column shift that aligns the tile's own keys for TMA.
 __host__ __device__ inline int train_attn_positions_per_tile(int d) { return (128 % d == 0 ? 128 : 120) / d; }
 struct TrainAttnArgs {
-  CUtensorMap mapQ, mapK;      // [B*H*L][128] bf16, boxes of 128 rows x 64 columns
+  CUtensorMap mapQ, mapK;      // [B*H*L][128] bf16, boxes of 128 (Q) / 64 (K) rows x 64 columns
   CUtensorMap mapVc, mapVm;    // V^T of the clean / masked slots: [B*Hkv*128][ld] bf16, boxes of 128 rows x 64 slots
   int B, Hq, Hkv, prompt_len, draft_len, n_clean_tiles;
   int seq_len[64];             // valid prompt slots per sequence

@@ -1,28 +1,83 @@
 // Forward attention under the prefix-shared training mask (Section 3.3, Appendix B): a packed row of
 // `prompt_len` clean positions followed by one block of `draft_len` masked positions per prefix position; block n
 // reads prompt slots 0..n and, causally, itself; clean positions read causally.  The mask is block-sparse with a
-// regular structure, so no mask tensor exists: a CTA owns 128 query rows of one head --
+// regular structure, so no mask tensor exists: a CTA owns 128 query rows --
 //   * a clean tile: 128 consecutive prompt slots, or
-//   * a masked tile: the blocks of T = 128 / draft_len consecutive prefix positions (T * draft_len rows) --
-// and walks exactly the key tiles its rows can see: the clean key tiles up to its last prefix position (only the
-// last of them needs a per-row bound) and, for a masked tile, its own 128 slots (same block and causal).
-// Flash-attention dataflow on the 5th-generation tensor cores:
-//   S = Q K^T       tcgen05.mma, operands by TMA (128-byte swizzle), S in tensor memory, two S buffers
-//   P = exp2(S - m) four warps, one query row per thread; bf16 P written to shared memory in the operand layout
-//   O += P V        tcgen05.mma with V^T tiles (a small kernel transposes V once), O accumulates in tensor memory
-// The running reference maximum m only moves when a tile's maximum exceeds it by more than 2^8, so the O rows are
-// rescaled in tensor memory a few times per row instead of once per tile.  Every mbarrier wait is bounded.
+//   * a masked tile: the blocks of T consecutive prefix positions (T * draft_len <= 128 rows) --
+// of TWO query heads that share a KV head (grouped-query attention: one K / V^T tile in shared memory serves both,
+// which halves the L2 -> SM traffic per flop; with one head per CTA the kernel was bound by it), and walks exactly
+// the 64-key tiles its rows can see: the clean key tiles up to its last prefix position (only those that reach past
+// its first position need a per-row bound) and, for a masked tile, its own slots (same block and causal).
+// Flash-attention dataflow on the 5th-generation tensor cores, per head:
+//   S = Q K^T       tcgen05.mma (128 x 64, k = 128), operands by TMA (128-byte swizzle), two S buffers in tensor memory
+//   P = exp2(S - m) four warps per head, one query row per thread; bf16 P written to shared memory in the operand layout
+//   O += P V        tcgen05.mma (128 x 128, k = 64) with V^T tiles (a small kernel transposes V once); O stays in
+//                   tensor memory
+// The reference maximum m only moves when a tile's maximum exceeds it by more than 2^8, so the O rows are rescaled
+// in tensor memory a few times per row instead of once per tile.  The two heads' softmax groups and the single MMA
+// issuer run concurrently: one head's exponentials overlap the other's MMAs.  Every mbarrier wait is bounded.
 #include "common.cuh"
 #include "kernels.h"
 #include "umma.cuh"
+
+#ifndef TA_WAIT
+#define TA_WAIT 0
+#endif
 
 namespace dart {
 
 using namespace umma;
 
-constexpr int kTaThreads = 256;
-constexpr int kTaTile = 128 * 128 * 2;                 // one 128 x 128 bf16 operand tile: two 64-column halves
-constexpr size_t kTaSmem = (size_t)6 * kTaTile + 1024;  // Q, P, 2 x K, 2 x V^T
+constexpr int kTaThreads = 384;                         // producer, MMA issuer, TMEM owner, idle; 4 + 4 softmax warps
+constexpr int kTaStages = 3;
+constexpr int kTaQ = 128 * 128 * 2;                     // a head's Q tile: two 64-column halves
+constexpr int kTaKV = 64 * 128 * 2;                     // 64 keys x 128 (K: two halves of 64 keys x 64; V^T: 128 x 64 keys)
+constexpr int kTaP = 128 * 64 * 2;                      // a head's P tile
+constexpr size_t kTaSmem = (size_t)2 * kTaQ + 4 * kTaP + 2 * kTaStages * kTaKV + 1024;   // 225 KB
+
+// 64 consecutive fp32 columns of this thread's TMEM lane in one instruction (one wait instead of four).
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64]) {
+  uint32_t r[64];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,"
+      "%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%64];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
+        "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]),
+        "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]),
+        "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]),
+        "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]),
+        "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int q = 0; q < 64; ++q) v[q] = __uint_as_float(r[q]);
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Bounded wait for the tight producer/consumer chains of this kernel: polls without a suspend hint.
+__device__ __forceinline__ bool ta_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (int it = 0; it < 20000000; ++it) {
+    uint32_t ok;
+#if TA_WAIT == 1
+    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+#else
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+#endif
+    if (ok) return true;
+    if ((it & 1023) == 1023 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
 
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
@@ -55,15 +110,18 @@ __global__ void __launch_bounds__(256) train_attn_transpose_kernel(const bf16* _
 __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_constant__ TrainAttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = sm;
-  uint8_t* sP = sm + kTaTile;
-  uint8_t* sK = sm + 2 * kTaTile;     // two stages
-  uint8_t* sV = sm + 4 * kTaTile;     // two stages
-  __shared__ uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full, pv_done;
+  uint8_t* sQ = sm;                                   // [2 heads]
+  uint8_t* sP = sm + 2 * kTaQ;                        // [2 heads][2 buffers]
+  uint8_t* sK = sP + 4 * kTaP;                        // [stages]
+  uint8_t* sV = sK + kTaStages * kTaKV;               // [stages]
+  __shared__ uint64_t q_full, k_full[kTaStages], k_empty[kTaStages], v_full[kTaStages], v_empty[kTaStages];
+  __shared__ uint64_t s_full[2][2], s_empty[2][2], p_full[2][2], pv_done[2][2];
   __shared__ uint32_t tmem_base;
   __shared__ int abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.z, hq = blockIdx.y, hk = hq / (a.Hq / a.Hkv);
+  const int G = a.Hq / a.Hkv, pairs = (G + 1) / 2;    // query heads per KV head; CTAs (pairs of heads) per KV head
+  const int b = blockIdx.z, hk = (int)blockIdx.y / pairs, hq0 = hk * G + ((int)blockIdx.y % pairs) * 2;
+  const int nh = hq0 + 1 < (hk + 1) * G ? 2 : 1;      // an odd group's last CTA has one head
   const int Lp = a.prompt_len, d = a.draft_len, L = Lp * (1 + d), T = train_attn_positions_per_tile(d);
   const int n_mask_tiles = (Lp + T - 1) / T, S = a.seq_len[b];
   // heavy tiles first: masked tiles from the last prefix position down, then clean tiles from the last down
@@ -76,22 +134,27 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
   const int own0 = (n0 * d) & ~7, shift = n0 * d - own0;
   const int rows = masked ? min(T, Lp - n0) * d : min(128, Lp - n0);
   const int last_pos = masked ? min(n0 + T, Lp) - 1 : min(n0 + 128, Lp) - 1;
-  const int n_clean = n0 < S ? min(last_pos, S - 1) / 128 + 1 : 0;   // clean key tiles some valid row can see
-  const int n_kt = n0 < S ? n_clean + (masked ? 1 : 0) : 0;          // + the tile's own slots
-  bf16* out = a.out + ((size_t)(b * a.Hq + hq) * L + q_slot0) * 128;
+  const int n_clean = n0 < S ? min(last_pos, S - 1) / 64 + 1 : 0;   // clean 64-key tiles some valid row can see
+  const int n_own = masked ? (shift + rows > 64 ? 2 : 1) : 0;       // 64-key tiles of the tile's own slots
+  const int n_kt = n0 < S ? n_clean + n_own : 0;
 
   if (n_kt == 0) {   // every row lies past the sequence's length: zero rows, nothing to read
-    for (int e = threadIdx.x; e < rows * 16; e += kTaThreads) reinterpret_cast<uint4*>(out)[e] = make_uint4(0u, 0u, 0u, 0u);
+    for (int h = 0; h < nh; ++h) {
+      bf16* out = a.out + ((size_t)(b * a.Hq + hq0 + h) * L + q_slot0) * 128;
+      for (int e = threadIdx.x; e < rows * 16; e += kTaThreads) reinterpret_cast<uint4*>(out)[e] = make_uint4(0u, 0u, 0u, 0u);
+    }
     return;
   }
   if (threadIdx.x == 0) {
     mbar_init(&q_full, 1);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
-      mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 128);
+    for (int s = 0; s < kTaStages; ++s) {
+      mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], nh); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], nh);   // one release per head
     }
-    mbar_init(&p_full, 128);
-    mbar_init(&pv_done, 1);
+    for (int h = 0; h < 2; ++h)
+      for (int s = 0; s < 2; ++s) {
+        mbar_init(&s_full[h][s], 1); mbar_init(&s_empty[h][s], 128);
+        mbar_init(&p_full[h][s], 128); mbar_init(&pv_done[h][s], 1);
+      }
     abort_flag = 0;
     fence_barrier_init();
   }
@@ -99,165 +162,165 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = tmem_base;          // columns 0..255: two S buffers; 256..383: O
+  const uint32_t tmem = tmem_base;          // head h: columns 256 h + {0, 64}: two S buffers; 256 h + 128: O
 
   if (warp == 0 && lane == 0) {
-    // ---- producer: Q once, then per key tile K [128 keys][128] and V^T [128][128 keys]
-    const int q_row = (b * a.Hq + hq) * L + q_slot0;
-    mbar_expect_tx(&q_full, kTaTile);
-    tma_load_2d(sQ, &a.mapQ, &q_full, 0, q_row);
-    tma_load_2d(sQ + kTaTile / 2, &a.mapQ, &q_full, 64, q_row);
-    for (int j = 0; j < n_kt; ++j) {
-      const int s = j & 1;
-      const bool own = masked && j == n_kt - 1;
-      const int k_row = (b * a.Hkv + hk) * L + (own ? Lp + own0 : j * 128);
-      const int v_col = own ? own0 : j * 128, v_row = (b * a.Hkv + hk) * 128;
-      if (j >= 2 && !mbar_wait(&k_empty[s], ((j >> 1) - 1) & 1, &abort_flag)) break;
-      mbar_expect_tx(&k_full[s], kTaTile);
-      tma_load_2d(sK + s * kTaTile, &a.mapK, &k_full[s], 0, k_row);
-      tma_load_2d(sK + s * kTaTile + kTaTile / 2, &a.mapK, &k_full[s], 64, k_row);
-      if (j >= 2 && !mbar_wait(&v_empty[s], ((j >> 1) - 1) & 1, &abort_flag)) break;
-      mbar_expect_tx(&v_full[s], kTaTile);
-      const CUtensorMap* mv = own ? &a.mapVm : &a.mapVc;
-      tma_load_2d(sV + s * kTaTile, mv, &v_full[s], v_col, v_row);
-      tma_load_2d(sV + s * kTaTile + kTaTile / 2, mv, &v_full[s], v_col + 64, v_row);
+    // ---- producer: the heads' Q tiles once, then per key tile K [64 keys][128] and V^T [128][64 keys]
+    mbar_expect_tx(&q_full, nh * kTaQ);
+    for (int h = 0; h < nh; ++h) {
+      const int q_row = (b * a.Hq + hq0 + h) * L + q_slot0;
+      tma_load_2d(sQ + h * kTaQ, &a.mapQ, &q_full, 0, q_row);
+      tma_load_2d(sQ + h * kTaQ + kTaQ / 2, &a.mapQ, &q_full, 64, q_row);
     }
-  } else if (warp == 1 && lane == 0) {
-    // ---- MMA issuer
-    constexpr uint32_t idesc = idesc_bf16(128, 128);
-    const uint64_t dq0 = desc_sw128(smem_u32(sQ)), dq1 = desc_sw128(smem_u32(sQ + kTaTile / 2));
-    const uint64_t dp0 = desc_sw128(smem_u32(sP)), dp1 = desc_sw128(smem_u32(sP + kTaTile / 2));
-    bool ok = mbar_wait(&q_full, 0, &abort_flag);
+    int s = 0, ph = 0;
+    for (int j = 0; j < n_kt; ++j) {
+      const bool own = j >= n_clean;
+      const int key0 = own ? own0 + (j - n_clean) * 64 : j * 64;     // first key: masked-region index / prompt slot
+      const int k_row = (b * a.Hkv + hk) * L + (own ? Lp + key0 : key0), v_row = (b * a.Hkv + hk) * 128;
+      if (ph > 0 && !ta_wait(&k_empty[s], (ph - 1) & 1, &abort_flag)) break;
+      mbar_expect_tx(&k_full[s], kTaKV);
+      tma_load_2d(sK + s * kTaKV, &a.mapK, &k_full[s], 0, k_row);
+      tma_load_2d(sK + s * kTaKV + kTaKV / 2, &a.mapK, &k_full[s], 64, k_row);
+      if (ph > 0 && !ta_wait(&v_empty[s], (ph - 1) & 1, &abort_flag)) break;
+      mbar_expect_tx(&v_full[s], kTaKV);
+      tma_load_2d(sV + s * kTaKV, own ? &a.mapVm : &a.mapVc, &v_full[s], key0, v_row);
+      if (++s == kTaStages) { s = 0; ++ph; }
+    }
+  } else if ((warp == 1 || warp == 3) && lane == 0 && (warp >> 1) < nh) {
+    // ---- MMA issuer of head h (the two heads are independent pipelines that share the K / V^T stages)
+    const int h = warp >> 1;
+    constexpr uint32_t idesc_s = idesc_bf16(128, 64), idesc_o = idesc_bf16(128, 128);
+    const uint64_t dq0 = desc_sw128(smem_u32(sQ + h * kTaQ)), dq1 = desc_sw128(smem_u32(sQ + h * kTaQ + kTaQ / 2));
+    bool ok = ta_wait(&q_full, 0, &abort_flag);
+    int ss = 0, sph = 0;                     // stage / phase of the next S tile's K
     auto issue_s = [&](int j) -> bool {      // S[j & 1] = Q K_j^T
-      const int s = j & 1;
-      if (j >= 2 && !mbar_wait(&s_empty[s], ((j >> 1) - 1) & 1, &abort_flag)) return false;
-      if (!mbar_wait(&k_full[s], (j >> 1) & 1, &abort_flag)) return false;
+      const int sb = j & 1;
+      if (!ta_wait(&k_full[ss], sph & 1, &abort_flag)) return false;
+      if (j >= 2 && !ta_wait(&s_empty[h][sb], ((j >> 1) - 1) & 1, &abort_flag)) return false;
       tc_fence_after();
-      const uint64_t dk0 = desc_sw128(smem_u32(sK + s * kTaTile)), dk1 = desc_sw128(smem_u32(sK + s * kTaTile + kTaTile / 2));
+      const uint64_t dk0 = desc_sw128(smem_u32(sK + ss * kTaKV)), dk1 = desc_sw128(smem_u32(sK + ss * kTaKV + kTaKV / 2));
+      const uint32_t acc = tmem + h * 256 + sb * 64;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + s * 128, dq0 + 2 * k, dk0 + 2 * k, idesc, k > 0 ? 1u : 0u);
+      for (int k = 0; k < 4; ++k) mma_f16(acc, dq0 + 2 * k, dk0 + 2 * k, idesc_s, k > 0 ? 1u : 0u);
 #pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + s * 128, dq1 + 2 * k, dk1 + 2 * k, idesc, 1u);
-      mma_commit(&k_empty[s]);
-      mma_commit(&s_full[s]);
+      for (int k = 0; k < 4; ++k) mma_f16(acc, dq1 + 2 * k, dk1 + 2 * k, idesc_s, 1u);
+      mma_commit(&s_full[h][sb]);
+      mma_commit(&k_empty[ss]);
+      if (++ss == kTaStages) { ss = 0; ++sph; }
       return true;
     };
     if (ok) ok = issue_s(0);
+    int vs = 0, vph = 0;
     for (int j = 0; j < n_kt && ok; ++j) {
-      const int s = j & 1;
+      const int pb = j & 1;
       if (j + 1 < n_kt && !issue_s(j + 1)) break;
-      if (!mbar_wait(&p_full, j & 1, &abort_flag)) break;
-      if (!mbar_wait(&v_full[s], (j >> 1) & 1, &abort_flag)) break;
+      if (!ta_wait(&v_full[vs], vph & 1, &abort_flag)) break;
+      if (!ta_wait(&p_full[h][pb], (j >> 1) & 1, &abort_flag)) break;
       tc_fence_after();
-      const uint64_t dv0 = desc_sw128(smem_u32(sV + s * kTaTile)), dv1 = desc_sw128(smem_u32(sV + s * kTaTile + kTaTile / 2));
+      const uint64_t dv = desc_sw128(smem_u32(sV + vs * kTaKV)), dp = desc_sw128(smem_u32(sP + (h * 2 + pb) * kTaP));
 #pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + 256, dp0 + 2 * k, dv0 + 2 * k, idesc, (j > 0 || k > 0) ? 1u : 0u);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + 256, dp1 + 2 * k, dv1 + 2 * k, idesc, 1u);
-      mma_commit(&v_empty[s]);
-      mma_commit(&pv_done);
+      for (int k = 0; k < 4; ++k) mma_f16(tmem + h * 256 + 128, dp + 2 * k, dv + 2 * k, idesc_o, (j > 0 || k > 0) ? 1u : 0u);
+      mma_commit(&pv_done[h][pb]);
+      mma_commit(&v_empty[vs]);
+      if (++vs == kTaStages) { vs = 0; ++vph; }
     }
-  } else if (warp >= 4) {
-    // ---- softmax: thread = query row of the tile = TMEM lane
-    const int wq = warp & 3, row = wq * 32 + lane;
-    const uint32_t tb = tmem + ((uint32_t)(wq * 32) << 16);
-    // the row's prefix position (masked: its block's; clean: its own slot); rows past the data or the length see nothing
+  } else if (warp >= 4 && (warp - 4) / 4 < nh) {
+    // ---- softmax of head h: thread = query row of the tile = TMEM lane
+    const int h = (warp - 4) / 4, wq = warp & 3, row = wq * 32 + lane;
+    const uint32_t tb = tmem + ((uint32_t)(wq * 32) << 16) + h * 256;
+    // the row's prefix position (masked: its block's; clean: its own slot); rows past the data or the length give zeros
     const int pos = masked ? n0 + row / d : n0 + row;
     const bool live = row < rows && pos < S;
     const float c = a.scale_log2e;
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < n_kt; ++j) {
-      const int s = j & 1;
-      const bool own = masked && j == n_kt - 1;
-      // visible key columns of this tile for this row: [lo, hi]
-      int lo = 0, hi = -1;
-      if (live) {
-        if (own) { lo = shift + (row / d) * d; hi = shift + row; }
-        else hi = min(127, pos - j * 128);
-      }
-      if (!mbar_wait(&s_full[s], (j >> 1) & 1, &abort_flag)) { ok = false; break; }
+      const int sb = j & 1;
+      const bool own = j >= n_clean;
+      // visible key columns of this tile for this row: [lo, hi]; tiles below the tile's first position need no bound
+      const bool bounded = own || j * 64 + 63 > n0;
+      int lo = 0, hi = 63;
+      if (own) { lo = shift + (row / d) * d - (j - n_clean) * 64; hi = shift + row - (j - n_clean) * 64; }
+      else if (bounded) hi = pos - j * 64;
+      if (!ta_wait(&s_full[h][sb], (j >> 1) & 1, &abort_flag)) { ok = false; break; }
       tc_fence_after();
-      float sv[128];
-#pragma unroll
-      for (int cb = 0; cb < 128; cb += 16) {
-        uint32_t r[16];
-        tmem_ld16(tb + s * 128 + cb, r);
-        tmem_ld_wait();
-#pragma unroll
-        for (int q = 0; q < 16; ++q) sv[cb + q] = __uint_as_float(r[q]);
-      }
+      float sv[64];
+      tmem_ld64(tb + sb * 64, sv);
       tc_fence_before();
-      mbar_arrive(&s_empty[s]);
-      float mt = -INFINITY;
+      mbar_arrive(&s_empty[h][sb]);
+      if (bounded) {
 #pragma unroll
-      for (int q = 0; q < 128; ++q) {
-        sv[q] = (q >= lo && q <= hi) ? sv[q] * c : -INFINITY;
-        mt = fmaxf(mt, sv[q]);
+        for (int q = 0; q < 64; ++q) sv[q] = (q >= lo && q <= hi) ? sv[q] : -INFINITY;
       }
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one of 64 dependent maxima
+#pragma unroll
+      for (int q = 0; q < 64; ++q) mx[q & 3] = fmaxf(mx[q & 3], sv[q]);
+      const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;      // c > 0: the scaled maximum
       float alpha = 1.f;
       if (mt > m_ref + 8.f) {               // also the first visible tile (m_ref = -inf)
-        alpha = m_ref == -INFINITY ? 1.f : exp2f(m_ref - mt);
+        alpha = m_ref == -INFINITY ? 1.f : ex2(m_ref - mt);
         m_ref = mt;
         l *= alpha;
       }
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
-      float lsum = 0.f;
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int q = 0; q < 128; ++q) {
-        sv[q] = exp2f(sv[q] - m_use);       // exp2(-inf) = 0 for the hidden columns
-        lsum += sv[q];
+      for (int q = 0; q < 64; ++q) {
+        sv[q] = ex2(fmaf(sv[q], c, -m_use));   // ex2(-inf) = 0 for the hidden columns
+        ls[q & 3] += sv[q];
       }
-      l += lsum;
-      if (j > 0) {
-        if (!mbar_wait(&pv_done, (j - 1) & 1, &abort_flag)) { ok = false; break; }
+      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      const int pb = j & 1;
+      // this P buffer was last read by the MMA of tile j - 2
+      if (j >= 2 && !ta_wait(&pv_done[h][pb], ((j >> 1) - 1) & 1, &abort_flag)) { ok = false; break; }
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rescale this warp's O rows in tensor memory
+        if (!ta_wait(&pv_done[h][pb ^ 1], ((j - 1) >> 1) & 1, &abort_flag)) { ok = false; break; }   // O holds tiles 0..j-1
         tc_fence_after();
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {   // rescale this warp's O rows in tensor memory
+        {
 #pragma unroll 1
           for (int cb = 0; cb < 128; cb += 16) {
             uint32_t r[16];
-            tmem_ld16(tb + 256 + cb, r);
+            tmem_ld16(tb + 128 + cb, r);
             tmem_ld_wait();
 #pragma unroll
             for (int q = 0; q < 16; ++q) r[q] = __float_as_uint(__uint_as_float(r[q]) * alpha);
-            tmem_st16(tb + 256 + cb, r);
+            tmem_st16(tb + 128 + cb, r);
           }
           tmem_st_wait();
         }
       }
-      // P as the A operand of the second MMA: [128 rows][128 keys] in two 64-key halves, rows of 128 bytes,
-      // 16-byte chunk ch of row r stored at chunk ch ^ (r & 7) (the 128-byte swizzle)
+      uint8_t* prow = sP + (h * 2 + pb) * kTaP + row * 128;
+      // P as the A operand of the second MMA: [128 rows][64 keys], rows of 128 bytes, 16-byte chunk ch of row r
+      // stored at chunk ch ^ (r & 7) (the 128-byte swizzle)
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        uint8_t* prow = sP + hf * (kTaTile / 2) + row * 128;
+      for (int ch = 0; ch < 8; ++ch) {
+        uint32_t w[4];
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          uint32_t w[4];
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const __nv_bfloat162 v2 = __floats2bfloat162_rn(sv[hf * 64 + ch * 8 + 2 * q], sv[hf * 64 + ch * 8 + 2 * q + 1]);
-            w[q] = *reinterpret_cast<const uint32_t*>(&v2);
-          }
-          *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        for (int q = 0; q < 4; ++q) {
+          const __nv_bfloat162 v2 = __floats2bfloat162_rn(sv[ch * 8 + 2 * q], sv[ch * 8 + 2 * q + 1]);
+          w[q] = *reinterpret_cast<const uint32_t*>(&v2);
         }
+        *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
       fence_async_smem();
       tc_fence_before();
-      mbar_arrive(&p_full);
+      mbar_arrive(&p_full[h][pb]);
     }
-    if (ok && mbar_wait(&pv_done, (n_kt - 1) & 1, &abort_flag)) {
+    if (ok && ta_wait(&pv_done[h][(n_kt - 1) & 1], ((n_kt - 1) >> 1) & 1, &abort_flag)) {
       tc_fence_after();
-      const float inv = l > 0.f ? 1.f / l : 0.f;
+      const float inv = (live && l > 0.f) ? 1.f / l : 0.f;
+      bf16* out = a.out + ((size_t)(b * a.Hq + hq0 + h) * L + q_slot0) * 128;
 #pragma unroll 1
       for (int cb = 0; cb < 128; cb += 16) {
         uint32_t r[16];
-        tmem_ld16(tb + 256 + cb, r);
+        tmem_ld16(tb + 128 + cb, r);
         tmem_ld_wait();
         if (row < rows) {
           uint32_t w[8];
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
-            const __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(r[2 * q]) * inv, __uint_as_float(r[2 * q + 1]) * inv);
+            const float x0 = live ? __uint_as_float(r[2 * q]) * inv : 0.f, x1 = live ? __uint_as_float(r[2 * q + 1]) * inv : 0.f;
+            const __nv_bfloat162 v2 = __floats2bfloat162_rn(x0, x1);
             w[q] = *reinterpret_cast<const uint32_t*>(&v2);
           }
           uint4* dst = reinterpret_cast<uint4*>(out + (size_t)row * 128 + cb);
@@ -280,7 +343,8 @@ cudaError_t launch_train_attn(const TrainAttnArgs& a, const bf16* v, bf16* vt_c,
   train_attn_transpose_kernel<<<dim3((ldmax + 31) / 32, 2 * (128 / 32), a.B * a.Hkv), 256, 0, st>>>(v, vt_c, vt_m, L, a.prompt_len, 128, ldc, ldm);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   const int T = train_attn_positions_per_tile(a.draft_len), n_mask_tiles = (a.prompt_len + T - 1) / T;
-  train_attn_kernel<<<dim3(n_mask_tiles + a.n_clean_tiles, a.Hq, a.B), kTaThreads, kTaSmem, st>>>(a);
+  const int G = a.Hq / a.Hkv;   // one CTA per pair of query heads of a KV head
+  train_attn_kernel<<<dim3(n_mask_tiles + a.n_clean_tiles, a.Hkv * ((G + 1) / 2), a.B), kTaThreads, kTaSmem, st>>>(a);
   return cudaGetLastError();
 }
 

@@ -52,6 +52,10 @@ def test_d1_and_an_empty_sequence():
     _run(2, 2, 2, 130, 1, [0, 130], seed=2)
 
 
+def test_odd_group_of_query_heads():
+    _run(1, 6, 2, 70, 8, [66], seed=6)          # three query heads per KV head: a pair and a single per CTA row
+
+
 def test_one_prompt_slot():
     _run(1, 2, 1, 1, 8, [1], seed=3)
 
