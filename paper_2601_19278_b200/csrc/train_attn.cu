@@ -20,10 +20,6 @@
 #include "kernels.h"
 #include "umma.cuh"
 
-#ifndef TA_WAIT
-#define TA_WAIT 0
-#endif
-
 namespace dart {
 
 using namespace umma;
@@ -63,15 +59,10 @@ __device__ __forceinline__ float ex2(float x) {
 }
 // Bounded wait for the tight producer/consumer chains of this kernel: polls without a suspend hint.
 __device__ __forceinline__ bool ta_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (int it = 0; it < 20000000; ++it) {
+  for (int it = 0; it < 4000000; ++it) {
     uint32_t ok;
-#if TA_WAIT == 1
-    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-#else
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-#endif
     if (ok) return true;
     if ((it & 1023) == 1023 && *abort_flag) return false;
   }
@@ -152,8 +143,8 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
     }
     for (int h = 0; h < 2; ++h)
       for (int s = 0; s < 2; ++s) {
-        mbar_init(&s_full[h][s], 1); mbar_init(&s_empty[h][s], 128);
-        mbar_init(&p_full[h][s], 128); mbar_init(&pv_done[h][s], 1);
+        mbar_init(&s_full[h][s], 1); mbar_init(&s_empty[h][s], 4);     // one arrival per softmax warp
+        mbar_init(&p_full[h][s], 4); mbar_init(&pv_done[h][s], 1);
       }
     abort_flag = 0;
     fence_barrier_init();
@@ -247,7 +238,8 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
       float sv[64];
       tmem_ld64(tb + sb * 64, sv);
       tc_fence_before();
-      mbar_arrive(&s_empty[h][sb]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[h][sb]);
       if (bounded) {
 #pragma unroll
         for (int q = 0; q < 64; ++q) sv[q] = (q >= lo && q <= hi) ? sv[q] : -INFINITY;
@@ -304,7 +296,8 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
       }
       fence_async_smem();
       tc_fence_before();
-      mbar_arrive(&p_full[h][pb]);
+      __syncwarp();                          // every lane's P chunks and fences precede the warp's one arrival
+      if (lane == 0) mbar_arrive(&p_full[h][pb]);
     }
     if (ok && ta_wait(&pv_done[h][(n_kt - 1) & 1], ((n_kt - 1) >> 1) & 1, &abort_flag)) {
       tc_fence_after();
