@@ -570,9 +570,49 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const 
       rstd = 1.f / sqrtf(ssq / (float)p.Kd + p.rms_eps);
     }
     float m_run = -INFINITY, s_run = 0.f;
-    int n_list = 0, worst = 0;                 // entries in the list, slot of its last-ranked entry
-    float w_key = INFINITY; int w_id = -1;     // that entry (valid once the list is full)
+    // The token's candidate list: up to 33 entries in this thread's shared-memory row.  An entry is appended when
+    // it may precede the threshold (the last-ranked entry kept by the latest compaction); when any row of the warp
+    // is full the whole warp compacts together -- keeps its best `topk`, renews its threshold -- so the 32 rows do
+    // their list work in step instead of one at a time.  An entry appended at temperature > 0 carries the plain
+    // logit and a pending mark: its exact perturbed key is computed at the next compaction.  (Keeping the kept
+    // part sorted and inserting the appended entries was slower: its shift loop is one dependent chain.)
+    int n_list = 0;
+    bool have_thr = false;
+    float t_key = -INFINITY; int t_id = 0x7fffffff;
     const int topk = p.topk;
+    constexpr int kPending = 1 << 30;
+    auto compact = [&]() {
+      if (p.gumbel) {
+        for (int e = 0; e < n_list; ++e) {
+          const int ie = my_id[e];
+          if (ie & kPending) {
+            const int v = ie & ~kPending;
+            const uint4 rnd = philox4x32_10(make_uint4((uint32_t)v >> 2, (uint32_t)(tok % p.K), (uint32_t)(tok / p.K), p.step), p.seed_lo, p.seed_hi);
+            const uint32_t wsel = (v & 3) == 0 ? rnd.x : ((v & 3) == 1 ? rnd.y : ((v & 3) == 2 ? rnd.z : rnd.w));
+            my_key[e] += gumbel_from_bits(wsel);
+            my_id[e] = v;
+          }
+        }
+      }
+      while (n_list > topk) {                  // drop the last-ranked entry until topk are left
+        int worst = 0;
+        float wk = my_key[0]; int wi = my_id[0];
+        for (int e = 1; e < n_list; ++e) {
+          const float ke = my_key[e]; const int ie = my_id[e];
+          if (cand_before(wk, wi, ke, ie)) { wk = ke; wi = ie; worst = e; }
+        }
+        --n_list;
+        my_key[worst] = my_key[n_list]; my_id[worst] = my_id[n_list];
+      }
+      if (n_list == topk) {                    // the threshold: the last-ranked of the kept entries
+        float wk = my_key[0]; int wi = my_id[0];
+        for (int e = 1; e < n_list; ++e) {
+          const float ke = my_key[e]; const int ie = my_id[e];
+          if (cand_before(wk, wi, ke, ie)) { wk = ke; wi = ie; }
+        }
+        t_key = wk; t_id = wi; have_thr = true;
+      }
+    };
     int visit = 0;
     long long u = u0;
     while (u < u1) {
@@ -624,39 +664,70 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const 
           }
         }
         const int v0 = tile * 256 + cb;             // vocabulary id of column 0 of this chunk (a multiple of 16)
-        if (!live || v0 >= p.V) continue;
+        if (v0 >= p.V) continue;                    // the same for every lane: what follows is warp-collective
 #pragma unroll
         for (int j = 0; j < 16; ++j) y[j] *= rstd;
-        if (p.logits_out != nullptr) {
+        if (live && p.logits_out != nullptr) {
           float4* lo = reinterpret_cast<float4*>(p.logits_out + (size_t)tok * p.V + v0);
 #pragma unroll
           for (int j = 0; j < 4; ++j) lo[j] = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
         }
-#pragma unroll 1
-        for (int q4 = 0; q4 < 4; ++q4) {
-          uint4 rnd = make_uint4(0, 0, 0, 0);
-          if (p.gumbel)
-            rnd = philox4x32_10(make_uint4((uint32_t)((v0 >> 2) + q4), (uint32_t)(tok % p.K), (uint32_t)(tok / p.K), p.step), p.seed_lo, p.seed_hi);
-          const uint32_t rw[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int v = v0 + 4 * q4 + q;
-            const float z = y[4 * q4 + q] * p.inv_temp;
-            // running log-sum-exp of this token row
-            if (z > m_run) { s_run = s_run * expf(m_run - z) + 1.f; m_run = z; }
-            else s_run += expf(z - m_run);
-            const float key = p.gumbel ? z + gumbel_from_bits(rw[q]) : z;
-            if (n_list < topk) {
-              my_key[n_list] = key; my_id[n_list] = v;
-              if (n_list == 0 || cand_before(w_key, w_id, key, v)) { w_key = key; w_id = v; worst = n_list; }
-              ++n_list;
-            } else if (cand_before(key, v, w_key, w_id)) {
-              my_key[worst] = key; my_id[worst] = v;
-              w_key = my_key[0]; w_id = my_id[0]; worst = 0;          // find the new last-ranked entry
-              for (int e = 1; e < topk; ++e) {
-                const float ke = my_key[e]; const int ie = my_id[e];
-                if (cand_before(w_key, w_id, ke, ie)) { w_key = ke; w_id = ie; worst = e; }
-              }
+        for (int j = 0; j < 16; ++j) y[j] *= p.inv_temp;
+        {  // running log-sum-exp of this token row, one chunk at a time (independent exponentials overlap)
+          float cm = y[0];
+#pragma unroll
+          for (int j = 1; j < 16; ++j) cm = fmaxf(cm, y[j]);
+          if (cm > m_run) { s_run *= expf(m_run - cm); m_run = cm; }
+          float e4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int j = 0; j < 16; ++j) e4[j & 3] += expf(y[j] - m_run);
+          s_run += (e4[0] + e4[1]) + (e4[2] + e4[3]);
+        }
+        // which of the 16 logits may precede the threshold.  At temperature > 0 the key is y + G(u): a fast
+        // evaluation of G decides with a margin 10x its error bound (u in [2^-14, 1 - 2^-8]: |error| < 1.2e-4;
+        // outside that range the entry is simply kept as a candidate); exact keys come at the compaction.
+        uint32_t may = 0u;
+        if (p.gumbel) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const uint4 rnd = philox4x32_10(make_uint4((uint32_t)((v0 >> 2) + q4), (uint32_t)(tok % p.K), (uint32_t)(tok / p.K), p.step), p.seed_lo, p.seed_hi);
+            const uint32_t rw[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint32_t m = rw[q] >> 8;
+              const float gq = -__logf(-__logf(((float)m + 0.5f) * (1.f / 16777216.f)));
+              const bool safe = m >= 1024u && m <= (1u << 24) - 65536u;
+              if (!have_thr || !safe || y[4 * q4 + q] + gq + 1e-3f >= t_key) may |= 1u << (4 * q4 + q);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (!have_thr || cand_before(y[j], v0 + j, t_key, t_id)) may |= 1u << j;
+        }
+        if (!live) may = 0u;
+#pragma unroll 1
+        while (__any_sync(0xffffffffu, may != 0u)) {
+          if (may != 0u) {
+            const int j = __ffs(may) - 1;
+            may &= may - 1u;
+            float yj = y[0];
+#pragma unroll
+            for (int q = 1; q < 16; ++q) yj = q == j ? y[q] : yj;
+            my_key[n_list] = yj;
+            my_id[n_list] = (v0 + j) | (p.gumbel ? kPending : 0);
+            ++n_list;
+          }
+          if (__any_sync(0xffffffffu, n_list == kLmDenseListStride)) {
+            compact();
+            // entries of this chunk not yet appended are re-checked against the new threshold when keys are exact
+            if (!p.gumbel && have_thr) {
+              uint32_t keep = 0u;
+#pragma unroll
+              for (int q = 0; q < 16; ++q)
+                if (((may >> q) & 1u) && cand_before(y[q], v0 + q, t_key, t_id)) keep |= 1u << q;
+              may = keep;
             }
           }
         }
@@ -670,6 +741,7 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const 
       u = ue;
     }
     // ---- this token's list, sorted (key desc, id asc), and its statistics
+    compact();                                      // exact keys for the pending entries, the best topk kept
     if (live) {
       for (int i = 1; i < n_list; ++i) {            // insertion sort of at most 32 entries
         const float ki = my_key[i]; const int ii = my_id[i];
