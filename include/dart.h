@@ -243,19 +243,12 @@ typedef struct dart_train_attn_in {
   const void* v;             /* DEVICE bf16 [batch, n_kv_heads, L, head_dim] */
   const int32_t* seq_lens_host; /* HOST [batch]: valid prompt slots, 0..prompt_len */
   void* out;                 /* DEVICE bf16 [batch, n_q_heads, L, head_dim]; every row is written */
-  void* workspace;           /* DEVICE, dart_train_attention_workspace_bytes(...) bytes, 256-byte aligned; holds V^T */
-  size_t workspace_bytes;
   int32_t* status;           /* DEVICE, may be NULL: set to a negative code if a bounded wait inside the kernel ran out */
 } dart_train_attn_in;
 
-/* Bytes of workspace dart_train_attention_fwd needs; 0 for arguments it does not accept. */
-size_t dart_train_attention_workspace_bytes(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int32_t prompt_len,
-                                            int32_t draft_len);
-
 /*
- * Enqueues the attention on `cuda_stream` (two kernels: a transpose of v into the workspace, then the attention).
- * Needs no handle.  Errors: INVALID_ARG (NULL or misaligned pointers, sizes out of range, head_dim != 128),
- * CAPACITY (workspace too small), UNSUPPORTED_ARCH, CUDA.
+ * Enqueues the attention on `cuda_stream` (one kernel; no workspace, no handle).  Errors: INVALID_ARG (NULL or
+ * misaligned pointers, sizes out of range, head_dim != 128), UNSUPPORTED_ARCH, CUDA.
  */
 int dart_train_attention_fwd(const dart_train_attn_in* in, void* cuda_stream);
 

@@ -26,7 +26,7 @@ DART_ERR_INTERNAL = -6
 
 EXPORTS = [
     "dart_draft_init", "dart_draft_step", "dart_build_tree", "dart_draft_destroy", "dart_last_device_status",
-    "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_ngram_bytes", "dart_train_attention_workspace_bytes", "dart_train_attention_fwd", "dart_step_launch_count", "dart_draft_prefill", "dart_tree_verify_inputs",
+    "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_ngram_bytes", "dart_train_attention_fwd", "dart_step_launch_count", "dart_draft_prefill", "dart_tree_verify_inputs",
     "dart_set_profile_events", "dart_topk_rows_noalloc",
 ]
 
@@ -49,8 +49,7 @@ NGRAM_HASH, NGRAM_TRIE = 0, 1
 class DartTrainAttnIn(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("prompt_len", C.c_int32), ("draft_len", C.c_int32), ("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p),
-                ("seq_lens_host", C.c_void_p), ("out", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("status", C.c_void_p)]
+                ("seq_lens_host", C.c_void_p), ("out", C.c_void_p), ("status", C.c_void_p)]
 
 
 WEIGHT_NAMES = ["w_fc", "embed", "mask_vec", "norm_g", "norm_e", "w_q", "w_k", "w_v", "w_o", "norm_post",
@@ -128,8 +127,6 @@ def lib() -> C.CDLL:
         L.dart_status_string.restype = C.c_char_p
         L.dart_workspace_bytes.argtypes = [C.POINTER(DartConfig)]
         L.dart_workspace_bytes.restype = C.c_size_t
-        L.dart_train_attention_workspace_bytes.argtypes = [C.c_int32] * 5
-        L.dart_train_attention_workspace_bytes.restype = C.c_size_t
         L.dart_train_attention_fwd.argtypes = [C.POINTER(DartTrainAttnIn), C.c_void_p]
         L.dart_train_attention_fwd.restype = C.c_int
         L.dart_ngram_bytes.argtypes = [C.c_void_p]
@@ -287,19 +284,14 @@ def topk_rows_noalloc(logits: torch.Tensor, topk: int, eps_logit: float, out_ids
         raise DartError(rc, "dart_topk_rows_noalloc")
 
 
-def train_attention_workspace_bytes(batch: int, n_kv_heads: int, head_dim: int, prompt_len: int, draft_len: int) -> int:
-    return lib().dart_train_attention_workspace_bytes(batch, n_kv_heads, head_dim, prompt_len, draft_len)
-
-
 def train_attention_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_lens, prompt_len: int, draft_len: int,
-                        out: torch.Tensor, workspace: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None) -> None:
+                        out: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None) -> None:
     """dart_train_attention_fwd on caller-owned device tensors: q [B, Hq, L, dh], k, v [B, Hkv, L, dh] bf16,
-    L = prompt_len * (1 + draft_len); seq_lens: host ints [B]; workspace: a uint8 device tensor."""
+    L = prompt_len * (1 + draft_len); seq_lens: host ints [B]."""
     lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
     a = DartTrainAttnIn(batch=q.shape[0], n_q_heads=q.shape[1], n_kv_heads=k.shape[1], head_dim=q.shape[3], prompt_len=prompt_len,
                         draft_len=draft_len, q=q.data_ptr(), k=k.data_ptr(), v=v.data_ptr(), seq_lens_host=lens.ctypes.data,
-                        out=out.data_ptr(), workspace=_ptr(workspace), workspace_bytes=0 if workspace is None else workspace.numel(),
-                        status=_ptr(status))
+                        out=out.data_ptr(), status=_ptr(status))
     st = stream if stream is not None else torch.cuda.current_stream(q.device)
     rc = lib().dart_train_attention_fwd(C.byref(a), C.c_void_p(st.cuda_stream))
     if rc != DART_OK:

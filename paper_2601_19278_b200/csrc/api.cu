@@ -763,30 +763,20 @@ int dart_tree_verify_inputs(dart_handle* h, const dart_verify_in* in, const dart
 }
 
 namespace {
-// V^T leading dimensions of the training attention's workspace (slots, padded to whole 128-slot tiles).
-inline size_t ta_ld(long long slots) { return (size_t)((slots + 127) / 128 * 128); }
 bool train_attn_dims_ok(int batch, int n_kv_heads, int head_dim, int prompt_len, int draft_len) {
   return batch >= 1 && batch <= 64 && n_kv_heads >= 1 && head_dim == 128 && prompt_len >= 1 && draft_len >= 1 && draft_len <= 16 &&
          (long long)batch * n_kv_heads * prompt_len * (1 + draft_len) < (1ll << 31) / 128;
 }
 }  // namespace
 
-size_t dart_train_attention_workspace_bytes(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int32_t prompt_len, int32_t draft_len) {
-  if (!train_attn_dims_ok(batch, n_kv_heads, head_dim, prompt_len, draft_len)) return 0;
-  return (size_t)batch * n_kv_heads * 128 * (ta_ld(prompt_len) + ta_ld((long long)prompt_len * draft_len)) * sizeof(bf16);
-}
-
 int dart_train_attention_fwd(const dart_train_attn_in* in, void* cuda_stream) {
   if (in == nullptr) return DART_ERR_INVALID_ARG;
   if (!train_attn_dims_ok(in->batch, in->n_kv_heads, in->head_dim, in->prompt_len, in->draft_len)) return DART_ERR_INVALID_ARG;
   if (in->n_q_heads < 1 || in->n_q_heads % in->n_kv_heads != 0 || in->n_q_heads > 65535) return DART_ERR_INVALID_ARG;
-  if (!aligned16(in->q) || !aligned16(in->k) || !aligned16(in->v) || !aligned16(in->out) || in->seq_lens_host == nullptr ||
-      in->workspace == nullptr || (reinterpret_cast<uintptr_t>(in->workspace) & 255u) != 0)
+  if (!aligned16(in->q) || !aligned16(in->k) || !aligned16(in->v) || !aligned16(in->out) || in->seq_lens_host == nullptr)
     return DART_ERR_INVALID_ARG;
   for (int b = 0; b < in->batch; ++b)
     if (in->seq_lens_host[b] < 0 || in->seq_lens_host[b] > in->prompt_len) return DART_ERR_INVALID_ARG;
-  if (in->workspace_bytes < dart_train_attention_workspace_bytes(in->batch, in->n_kv_heads, in->head_dim, in->prompt_len, in->draft_len))
-    return DART_ERR_CAPACITY;
   int dev = 0, major = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return fail_cuda(nullptr, e);
@@ -796,22 +786,18 @@ int dart_train_attention_fwd(const dart_train_attn_in* in, void* cuda_stream) {
 
   const int B = in->batch, Hq = in->n_q_heads, Hkv = in->n_kv_heads, Lp = in->prompt_len, d = in->draft_len;
   const unsigned long long L = (unsigned long long)Lp * (1 + d);
-  const size_t ldc = ta_ld(Lp), ldm = ta_ld((long long)Lp * d);
-  bf16* vt_c = static_cast<bf16*>(in->workspace);
-  bf16* vt_m = vt_c + (size_t)B * Hkv * 128 * ldc;
   TrainAttnArgs a;
   memset(&a, 0, sizeof(a));
   if ((e = tmap_encode_bf16(&a.mapQ, in->q, 128, (unsigned long long)B * Hq * L, 256, 64, 128)) != cudaSuccess ||
       (e = tmap_encode_bf16(&a.mapK, in->k, 128, (unsigned long long)B * Hkv * L, 256, 64, 64)) != cudaSuccess ||
-      (e = tmap_encode_bf16(&a.mapVc, vt_c, ldc, (unsigned long long)B * Hkv * 128, ldc * 2, 64, 128)) != cudaSuccess ||
-      (e = tmap_encode_bf16(&a.mapVm, vt_m, ldm, (unsigned long long)B * Hkv * 128, ldm * 2, 64, 128)) != cudaSuccess)
+      (e = tmap_encode_bf16(&a.mapV, in->v, 128, (unsigned long long)B * Hkv * L, 256, 64, 64)) != cudaSuccess)
     return e == cudaErrorNotSupported ? DART_ERR_UNSUPPORTED_ARCH : fail_cuda(nullptr, e);
   a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.prompt_len = Lp; a.draft_len = d; a.n_clean_tiles = (Lp + 127) / 128;
   for (int b = 0; b < B; ++b) a.seq_len[b] = in->seq_lens_host[b];
   a.scale_log2e = (float)(1.4426950408889634 / sqrt(128.0));
   a.out = static_cast<bf16*>(in->out);
   a.status = in->status;
-  e = launch_train_attn(a, static_cast<const bf16*>(in->v), vt_c, vt_m, (int)ldc, (int)ldm, static_cast<cudaStream_t>(cuda_stream));
+  e = launch_train_attn(a, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? DART_OK : fail_cuda(nullptr, e);
 }
 

@@ -263,20 +263,17 @@ cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st);
 // ---------------------------------------------------------------------------------------------
 // Forward attention under the prefix-shared training mask (train_attn.cu).  head_dim = 128.
 // ---------------------------------------------------------------------------------------------
-// Prefix positions whose masked blocks share one 128-row query tile: 128 / d where d divides 128; otherwise
-// 120 / d, which leaves room for the up-to-7-column shift that aligns the tile's own keys for TMA.
-__host__ __device__ inline int train_attn_positions_per_tile(int d) { return (128 % d == 0 ? 128 : 120) / d; }
+// Prefix positions whose masked blocks share one 128-row query tile.
+__host__ __device__ inline int train_attn_positions_per_tile(int d) { return 128 / d; }
 struct TrainAttnArgs {
-  CUtensorMap mapQ, mapK;      // [B*H*L][128] bf16, boxes of 128 (Q) / 64 (K) rows x 64 columns
-  CUtensorMap mapVc, mapVm;    // V^T of the clean / masked slots: [B*Hkv*128][ld] bf16, boxes of 128 rows x 64 slots
+  CUtensorMap mapQ, mapK, mapV;   // [B*H*L][128] bf16, boxes of 128 (Q) / 64 (K, V) rows x 64 columns
   int B, Hq, Hkv, prompt_len, draft_len, n_clean_tiles;
   int seq_len[64];             // valid prompt slots per sequence
   float scale_log2e;           // log2(e) / sqrt(head_dim)
   bf16* out;                   // [B][Hq][L][128]
   int* status;                 // may be null
 };
-// Transposes v into vt_c [B*Hkv][128][ldc] and vt_m [B*Hkv][128][ldm] (zero beyond the data), then runs the attention.
-cudaError_t launch_train_attn(const TrainAttnArgs& a, const bf16* v, bf16* vt_c, bf16* vt_m, int ldc, int ldm, cudaStream_t st);
+cudaError_t launch_train_attn(const TrainAttnArgs& a, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
 // N-gram hash table + tree pruning.

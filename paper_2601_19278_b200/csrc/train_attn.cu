@@ -3,7 +3,7 @@
 // reads prompt slots 0..n and, causally, itself; clean positions read causally.  The mask is block-sparse with a
 // regular structure, so no mask tensor exists: a CTA owns 128 query rows --
 //   * a clean tile: 128 consecutive prompt slots, or
-//   * a masked tile: the blocks of T consecutive prefix positions (T * draft_len <= 128 rows) --
+//   * a masked tile: the blocks of T = 128 / draft_len consecutive prefix positions (T * draft_len <= 128 rows) --
 // of TWO query heads that share a KV head (grouped-query attention: one K / V^T tile in shared memory serves both,
 // which halves the L2 -> SM traffic per flop; with one head per CTA the kernel was bound by it), and walks exactly
 // the 64-key tiles its rows can see: the clean key tiles up to its last prefix position (only those that reach past
@@ -11,8 +11,8 @@
 // Flash-attention dataflow on the 5th-generation tensor cores, per head:
 //   S = Q K^T       tcgen05.mma (128 x 64, k = 128), operands by TMA (128-byte swizzle), two S buffers in tensor memory
 //   P = exp2(S - m) four warps per head, one query row per thread; bf16 P written to shared memory in the operand layout
-//   O += P V        tcgen05.mma (128 x 128, k = 64) with V^T tiles (a small kernel transposes V once); O stays in
-//                   tensor memory
+//   O += P V        tcgen05.mma (128 x 128, k = 64); V tiles are used as stored ([keys][d_h]: the MN-major form of the
+//                   B operand), so no transposed copy of V exists; O stays in tensor memory
 // The reference maximum m only moves when a tile's maximum exceeds it by more than 2^8, so the O rows are rescaled
 // in tensor memory a few times per row instead of once per tile.  The two heads' softmax groups and the single MMA
 // issuer run concurrently: one head's exponentials overlap the other's MMAs.  Every mbarrier wait is bounded.
@@ -27,7 +27,7 @@ using namespace umma;
 constexpr int kTaThreads = 384;                         // producer, MMA issuer, TMEM owner, idle; 4 + 4 softmax warps
 constexpr int kTaStages = 3;
 constexpr int kTaQ = 128 * 128 * 2;                     // a head's Q tile: two 64-column halves
-constexpr int kTaKV = 64 * 128 * 2;                     // 64 keys x 128 (K: two halves of 64 keys x 64; V^T: 128 x 64 keys)
+constexpr int kTaKV = 64 * 128 * 2;                     // 64 keys x 128: two halves of 64 keys x 64 columns, for K and for V
 constexpr int kTaP = 128 * 64 * 2;                      // a head's P tile
 constexpr size_t kTaSmem = (size_t)2 * kTaQ + 4 * kTaP + 2 * kTaStages * kTaKV + 1024;   // 225 KB
 
@@ -80,24 +80,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// V [B*Hkv][L][dh] -> V^T of the clean slots [B*Hkv][dh][ldc] and of the masked slots [B*Hkv][dh][ldm], zero beyond.
-__global__ void __launch_bounds__(256) train_attn_transpose_kernel(const bf16* __restrict__ v, bf16* __restrict__ vt_c, bf16* __restrict__ vt_m,
-                                                                   int L, int Lp, int dh, int ldc, int ldm) {
-  __shared__ bf16 tile[32][34];
-  const int head = blockIdx.z, region = blockIdx.y & 1, d0 = (blockIdx.y >> 1) * 32, s0 = blockIdx.x * 32;
-  const int ld = region ? ldm : ldc, n_src = region ? L - Lp : Lp, src0 = region ? Lp : 0;
-  if (s0 >= ld) return;
-  bf16* dst = (region ? vt_m : vt_c) + (size_t)head * dh * ld;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int r = ty; r < 32; r += 8) {
-    const int s = s0 + r;
-    tile[r][tx] = s < n_src ? v[((size_t)head * L + src0 + s) * dh + d0 + tx] : __float2bfloat16(0.f);
-  }
-  __syncthreads();
-  for (int r = ty; r < 32; r += 8)
-    if (s0 + tx < ld) dst[(size_t)(d0 + r) * ld + s0 + tx] = tile[tx][r];
-}
-
 __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_constant__ TrainAttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -120,13 +102,10 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
   const int ti = masked ? n_mask_tiles - 1 - (int)blockIdx.x : a.n_clean_tiles - 1 - ((int)blockIdx.x - n_mask_tiles);
   const int n0 = masked ? ti * T : ti * 128;                       // first prefix position / prompt slot of the tile
   const int q_slot0 = masked ? Lp + n0 * d : n0;                   // first packed slot of the tile's query rows
-  // a TMA load starts on a 16-byte boundary: the tile's own keys are fetched from the 8-slot boundary below its
-  // first masked slot, `shift` columns early
-  const int own0 = (n0 * d) & ~7, shift = n0 * d - own0;
   const int rows = masked ? min(T, Lp - n0) * d : min(128, Lp - n0);
   const int last_pos = masked ? min(n0 + T, Lp) - 1 : min(n0 + 128, Lp) - 1;
   const int n_clean = n0 < S ? min(last_pos, S - 1) / 64 + 1 : 0;   // clean 64-key tiles some valid row can see
-  const int n_own = masked ? (shift + rows > 64 ? 2 : 1) : 0;       // 64-key tiles of the tile's own slots
+  const int n_own = masked ? (rows > 64 ? 2 : 1) : 0;               // 64-key tiles of the tile's own slots
   const int n_kt = n0 < S ? n_clean + n_own : 0;
 
   if (n_kt == 0) {   // every row lies past the sequence's length: zero rows, nothing to read
@@ -156,7 +135,7 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
   const uint32_t tmem = tmem_base;          // head h: columns 256 h + {0, 64}: two S buffers; 256 h + 128: O
 
   if (warp == 0 && lane == 0) {
-    // ---- producer: the heads' Q tiles once, then per key tile K [64 keys][128] and V^T [128][64 keys]
+    // ---- producer: the heads' Q tiles once, then per key tile K and V, [64 keys][128] each
     mbar_expect_tx(&q_full, nh * kTaQ);
     for (int h = 0; h < nh; ++h) {
       const int q_row = (b * a.Hq + hq0 + h) * L + q_slot0;
@@ -166,15 +145,15 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
     int s = 0, ph = 0;
     for (int j = 0; j < n_kt; ++j) {
       const bool own = j >= n_clean;
-      const int key0 = own ? own0 + (j - n_clean) * 64 : j * 64;     // first key: masked-region index / prompt slot
-      const int k_row = (b * a.Hkv + hk) * L + (own ? Lp + key0 : key0), v_row = (b * a.Hkv + hk) * 128;
+      const int k_row = (b * a.Hkv + hk) * L + (own ? q_slot0 + (j - n_clean) * 64 : j * 64);   // first key's packed slot
       if (ph > 0 && !ta_wait(&k_empty[s], (ph - 1) & 1, &abort_flag)) break;
       mbar_expect_tx(&k_full[s], kTaKV);
       tma_load_2d(sK + s * kTaKV, &a.mapK, &k_full[s], 0, k_row);
       tma_load_2d(sK + s * kTaKV + kTaKV / 2, &a.mapK, &k_full[s], 64, k_row);
       if (ph > 0 && !ta_wait(&v_empty[s], (ph - 1) & 1, &abort_flag)) break;
       mbar_expect_tx(&v_full[s], kTaKV);
-      tma_load_2d(sV + s * kTaKV, own ? &a.mapVm : &a.mapVc, &v_full[s], key0, v_row);
+      tma_load_2d(sV + s * kTaKV, &a.mapV, &v_full[s], 0, k_row);
+      tma_load_2d(sV + s * kTaKV + kTaKV / 2, &a.mapV, &v_full[s], 64, k_row);
       if (++s == kTaStages) { s = 0; ++ph; }
     }
   } else if ((warp == 1 || warp == 3) && lane == 0 && (warp >> 1) < nh) {
@@ -208,9 +187,12 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
       if (!ta_wait(&v_full[vs], vph & 1, &abort_flag)) break;
       if (!ta_wait(&p_full[h][pb], (j >> 1) & 1, &abort_flag)) break;
       tc_fence_after();
-      const uint64_t dv = desc_sw128(smem_u32(sV + vs * kTaKV)), dp = desc_sw128(smem_u32(sP + (h * 2 + pb) * kTaP));
+      const uint64_t dp = desc_sw128(smem_u32(sP + (h * 2 + pb) * kTaP));
+      // V as stored ([keys][d_h], d_h contiguous) is the MN-major form of the B operand: 8-key groups 1024 bytes
+      // apart, the two 64-wide halves of d_h kTaKV / 2 bytes apart, the 16 keys of one MMA 2048 bytes on
+      const uint64_t dv = desc_sw128_mn(smem_u32(sV + vs * kTaKV), kTaKV / 2);
 #pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + h * 256 + 128, dp + 2 * k, dv + 2 * k, idesc_o, (j > 0 || k > 0) ? 1u : 0u);
+      for (int k = 0; k < 4; ++k) mma_f16(tmem + h * 256 + 128, dp + 2 * k, dv + 128 * k, idesc_o | kIdescBMnMajor, (j > 0 || k > 0) ? 1u : 0u);
       mma_commit(&pv_done[h][pb]);
       mma_commit(&v_empty[vs]);
       if (++vs == kTaStages) { vs = 0; ++vph; }
@@ -231,7 +213,7 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
       // visible key columns of this tile for this row: [lo, hi]; tiles below the tile's first position need no bound
       const bool bounded = own || j * 64 + 63 > n0;
       int lo = 0, hi = 63;
-      if (own) { lo = shift + (row / d) * d - (j - n_clean) * 64; hi = shift + row - (j - n_clean) * 64; }
+      if (own) { lo = (row / d) * d - (j - n_clean) * 64; hi = row - (j - n_clean) * 64; }
       else if (bounded) hi = pos - j * 64;
       if (!ta_wait(&s_full[h][sb], (j >> 1) & 1, &abort_flag)) { ok = false; break; }
       tc_fence_after();
@@ -329,12 +311,9 @@ __global__ void __launch_bounds__(kTaThreads, 1) train_attn_kernel(const __grid_
   if (abort_flag && threadIdx.x == 0 && a.status != nullptr) atomicExch(a.status, DEV_TIMEOUT);
 }
 
-cudaError_t launch_train_attn(const TrainAttnArgs& a, const bf16* v, bf16* vt_c, bf16* vt_m, int ldc, int ldm, cudaStream_t st) {
+cudaError_t launch_train_attn(const TrainAttnArgs& a, cudaStream_t st) {
   cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(&train_attn_kernel), kTaSmem);
   if (e != cudaSuccess) return e;
-  const int L = a.prompt_len * (1 + a.draft_len), ldmax = ldc > ldm ? ldc : ldm;
-  train_attn_transpose_kernel<<<dim3((ldmax + 31) / 32, 2 * (128 / 32), a.B * a.Hkv), 256, 0, st>>>(v, vt_c, vt_m, L, a.prompt_len, 128, ldc, ldm);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
   const int T = train_attn_positions_per_tile(a.draft_len), n_mask_tiles = (a.prompt_len + T - 1) / T;
   const int G = a.Hq / a.Hkv;   // one CTA per pair of query heads of a KV head
   train_attn_kernel<<<dim3(n_mask_tiles + a.n_clean_tiles, a.Hkv * ((G + 1) / 2), a.B), kTaThreads, kTaSmem, st>>>(a);

@@ -123,6 +123,19 @@ __device__ __forceinline__ uint64_t desc_sw128(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;                         // 128-byte swizzle
   return d;
 }
+// The same for an MN-major operand tile (the M / N dimension contiguous, e.g. V [keys][d_h] as the B operand of P V):
+// rows of 128 bytes = 64 elements along M / N, one row per k, 8-row groups 1024 bytes apart (stride offset), 64-wide
+// slabs along M / N `slab_bytes` apart (leading offset).  16 k-rows (one MMA) are 2048 bytes: start address + 128.
+__device__ __forceinline__ uint64_t desc_sw128_mn(uint32_t smem_addr, uint32_t slab_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)(slab_bytes >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+constexpr uint32_t kIdescBMnMajor = 1u << 16;   // instruction-descriptor bit: the B operand is MN-major
 // Instruction descriptor: bf16 A and B (both K-major), fp32 D, M x N tile.
 __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);

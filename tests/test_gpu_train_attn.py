@@ -22,9 +22,8 @@ def _run(B, Hq, Hkv, Lp, d, seq_lens, seed, q_scale=1.0):
     v = torch.randn(B, Hkv, L, dh, generator=g).to(torch.bfloat16)
     dev = torch.device("cuda:0")
     out = torch.full((B, Hq, L, dh), float("nan"), dtype=torch.bfloat16, device=dev)
-    ws = torch.empty(binding.train_attention_workspace_bytes(B, Hkv, dh, Lp, d), dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    binding.train_attention_fwd(q.to(dev), k.to(dev), v.to(dev), seq_lens, Lp, d, out, ws, status)
+    binding.train_attention_fwd(q.to(dev), k.to(dev), v.to(dev), seq_lens, Lp, d, out, status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     got = out.float().cpu().numpy().astype(np.float64)
@@ -75,15 +74,13 @@ def test_argument_errors():
     q = torch.zeros(B, Hq, L, dh, dtype=torch.bfloat16, device=dev)
     k = torch.zeros(B, Hkv, L, dh, dtype=torch.bfloat16, device=dev)
     out = torch.zeros_like(q)
-    ws = torch.empty(binding.train_attention_workspace_bytes(B, Hkv, dh, Lp, d), dtype=torch.uint8, device=dev)
-    assert binding.train_attention_workspace_bytes(B, Hkv, 64, Lp, d) == 0
     with pytest.raises(binding.DartError) as e:
-        binding.train_attention_fwd(q, k, k, [Lp + 1], Lp, d, out, ws)
+        binding.train_attention_fwd(q, k, k, [Lp + 1], Lp, d, out)
     assert e.value.status == binding.DART_ERR_INVALID_ARG
     with pytest.raises(binding.DartError) as e:
-        binding.train_attention_fwd(q, k, k, [Lp], Lp, d, out, ws[: ws.numel() // 2])
-    assert e.value.status == binding.DART_ERR_CAPACITY
+        binding.train_attention_fwd(q, k, k, [Lp], Lp, 17, out)
+    assert e.value.status == binding.DART_ERR_INVALID_ARG
     with pytest.raises(binding.DartError) as e:
-        binding.train_attention_fwd(q[:, :, :, :64].contiguous(), k, k, [Lp], Lp, d, out, ws)
+        binding.train_attention_fwd(q[:, :, :, :64].contiguous(), k, k, [Lp], Lp, d, out)
     assert e.value.status == binding.DART_ERR_INVALID_ARG
     torch.cuda.synchronize()
