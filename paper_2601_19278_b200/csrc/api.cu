@@ -65,6 +65,9 @@ struct dart_handle {
   const void* maps_feats = nullptr; int maps_fc_M = -1;
   int lm_grid = 0;
   int attn_pairs_cap = 0;  // capacity of the attention partial buffers in (sequence, chunk) pairs
+  AttnUmmaMaps attn_maps;  // q and new-row maps encoded at init; cache maps follow the caller's pointers
+  const void* attn_k_ptr = nullptr;
+  const void* attn_v_ptr = nullptr;
   int h_tiles = 0;         // 128-row tiles of a hidden-sized row
   Workspace ws;
   NgramSlot* ng_slots = nullptr;
@@ -477,6 +480,14 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   }
 
   INIT_CHECK(launch_rope_table(h->ws.rope_tab, cfg->max_prefix + cfg->K, cfg->head_dim, cfg->rope_theta, nullptr));
+  if (h->umma && cfg->head_dim == 128) {   // the attention's maps over the library's own buffers
+    const unsigned long long q_rows = (unsigned long long)cfg->max_batch * cfg->n_q_heads * cfg->K;
+    const unsigned long long n_rows16 = (unsigned long long)cfg->max_batch * cfg->n_kv_heads * 16;
+    INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapQhi, h->ws.q_hi, 128, q_rows, 256, 64, 64));
+    INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapQlo, h->ws.q_lo, 128, q_rows, 256, 64, 64));
+    INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapKn, h->ws.k_new, 128, n_rows16, 256, 64, 64));
+    INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapVn, h->ws.v_new, 128, n_rows16, 256, 64, 64));
+  }
 
   // Appendix D's per-level weights: fp64 from the fp32 settings, rounded once to fp32
   for (int i = 0; i < 8; ++i) {
@@ -674,7 +685,19 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
     for (int b = 0; b < B; ++b) pairs += (in->seq_lens_host[b] + ap.chunk_keys - 1) / ap.chunk_keys + 1;
     if (pairs > h->attn_pairs_cap) return DART_ERR_INTERNAL;
   }
-  if ((e = launch_attention(ap, in->seq_lens_host, st)) != cudaSuccess) return fail_cuda(h, e);
+  const AttnUmmaMaps* amaps = nullptr;
+  if (h->umma && c.head_dim == 128 && (long long)c.max_batch * c.n_kv_heads * c.max_prefix < (1ll << 31)) {
+    // maps over the caller's caches are re-encoded only when the pointers change
+    if (h->attn_k_ptr != in->k_cache || h->attn_v_ptr != in->v_cache) {
+      const unsigned long long rows = (unsigned long long)c.max_batch * c.n_kv_heads * c.max_prefix;
+      if ((e = tmap_encode_bf16(&h->attn_maps.mapK, in->k_cache, 128, rows, 256, 64, 64)) != cudaSuccess ||
+          (e = tmap_encode_bf16(&h->attn_maps.mapV, in->v_cache, 128, rows, 256, 64, 64)) != cudaSuccess)
+        return fail_cuda(h, e);
+      h->attn_k_ptr = in->k_cache; h->attn_v_ptr = in->v_cache;
+    }
+    amaps = &h->attn_maps;
+  }
+  if ((e = launch_attention(ap, in->seq_lens_host, amaps, ws.status, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(2, false);
 
   // S3: o_proj; epilogue: x1 = residual + proj, gain-scaled hi/lo, sums of squares

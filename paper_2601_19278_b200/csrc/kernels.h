@@ -220,9 +220,24 @@ struct AttnParams {
   float* ml_part;       // [sum_b chunks_b, Hkv, 64, 2]
   bf16* a_hi; bf16* a_lo;  // [M, Hq*dh]
 };
-cudaError_t attention_setup();  // once per device: opt in to the kernel's dynamic shared memory
-// seq_lens_host: the same lengths on the host (sizes the grid and the partial layout); B <= 32
-cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, cudaStream_t st);
+struct AttnArgs {
+  AttnParams p;
+  int chunk_base[33];  // prefix sums of chunks per sequence (cache chunks + 1 new-rows chunk)
+};
+// The tensor-core split kernel (attn_umma.cu, d_h = 128): tensor maps over q_hi / q_lo [B*Hq*K][128], the caches
+// [B*Hkv*P_cap][128] and the new rows' side tiles [B*Hkv*16][128]; boxes of 64 rows x 64 columns.
+struct AttnUmmaMaps { CUtensorMap mapQhi, mapQlo, mapK, mapV, mapKn, mapVn; };
+struct AttnUmmaArgs {
+  AttnArgs a;
+  CUtensorMap mapQhi, mapQlo, mapK, mapV, mapKn, mapVn;
+  int* status;
+};
+cudaError_t attn_umma_setup();  // once per device
+cudaError_t launch_attn_umma_split(const AttnUmmaArgs& a, int max_chunks, cudaStream_t st);
+cudaError_t attention_setup();  // once per device: opt in to the kernels' dynamic shared memory
+// seq_lens_host: the same lengths on the host (sizes the grid and the partial layout); B <= 32.  With `maps`
+// (d_h = 128) the split runs on the tcgen05 kernel, otherwise on the mma.sync one; the combine is the same.
+cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, const AttnUmmaMaps* maps, int* status, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
 // LM head with fused log-softmax / top-k partials, and the merge that finishes them.
