@@ -26,6 +26,12 @@ CASES = {
     "b16_k8_pad128": syn.small_variant(C1, batch=16, K=8, ragged_lo=10, prefix=300, vocab=2048, tree_budget=60),
     "empty_prefix": syn.small_variant(C1, prefix=0),
     "hot_b4": syn.small_variant(C1, batch=4, ragged_lo=20, prefix=160, temperature=1.0),
+    # enough 64-key tiles (sum over sequences x KV heads >= 2048) for the tensor-core split-KV attention: ragged
+    # lengths (partial last tiles, sequences with fewer chunks), 16 and 40 query rows per KV head
+    "attn_tiles_g2": syn.small_variant(C1, hidden=512, n_q_heads=32, n_kv_heads=16, head_dim=128, mlp_inter=1376,
+                                       vocab=2064, batch=8, ragged_lo=900, prefix=2000, K=8, tree_budget=60),
+    "attn_tiles_g5": syn.small_variant(C1, hidden=512, n_q_heads=40, n_kv_heads=8, head_dim=128, mlp_inter=1376,
+                                       vocab=2064, batch=8, ragged_lo=2100, prefix=3000, K=8, tree_budget=60),
 }
 
 
