@@ -34,14 +34,22 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// Bounded wait for the tight producer/consumer chains of this kernel: polls without a suspend hint.
+// Bounded wait for the tight producer / consumer chains of these kernels: polls without a suspend hint (a hinted
+// try_wait may sleep past the completion), and gives up after about a second of SM clock cycles whatever one poll
+// costs.  On time-out (or when another role has given up) sets *abort_flag and returns false.
 __device__ __forceinline__ bool ta_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (int it = 0; it < 4000000; ++it) {
+  long long t_start = 0;
+  for (int it = 0;; ++it) {
     uint32_t ok;
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     if (ok) return true;
-    if ((it & 1023) == 1023 && *abort_flag) return false;
+    if ((it & 255) == 255) {
+      if (*abort_flag) return false;
+      const long long now = clock64();
+      if (t_start == 0) t_start = now;
+      else if (now - t_start > 2000000000ll) break;
+    }
   }
   *abort_flag = 1;
   return false;
