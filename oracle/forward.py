@@ -130,8 +130,11 @@ def draft_forward(cfg: Dict, w: Dict[str, np.ndarray], inp: Dict[str, np.ndarray
     g = np.empty((B, K, h), dtype=np.float64)
     e = np.empty((B, K, h), dtype=np.float64)
     if Fb.sum() > 0:
-        feats = bf16_to_f64(inp["feats"]).reshape(-1, 3 * h)    # fresh rows packed in sequence order
-        gf = linear(feats, w["w_fc"])                           # fused features, no bias (reading)
+        if w.get("w_fc") is None:                               # the caller fused the features itself: feats = g [.., h]
+            gf = bf16_to_f64(inp["feats"]).reshape(-1, h)
+        else:
+            feats = bf16_to_f64(inp["feats"]).reshape(-1, 3 * h)    # fresh rows packed in sequence order
+            gf = linear(feats, w["w_fc"])                           # fused features, no bias (reading)
         ef = bf16_to_f64(w["embed"][np.asarray(inp["tokens"]).astype(np.int64).reshape(-1)])  # shifted embedding
     off = 0
     for b in range(B):

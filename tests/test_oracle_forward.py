@@ -303,3 +303,23 @@ def test_prefill_keys_and_values_are_the_forward_pass_s_new_rows():
     # positions matter for k (RoPE) and not for v
     k2, v2 = ofw.prefill_kv(cfg, wt, inp["feats"][0], inp["tokens"][0], P + 1 + np.arange(6))
     assert np.abs(k2 - k).max() > 1e-3 and np.array_equal(v2, v)
+
+
+def test_prefused_features_equal_the_layer_with_an_identity_fusion():
+    """feat_in = 0: the caller hands g itself.  That is the ordinary layer whose fusion matrix is [I | 0 | 0] fed
+    with [g, 0, 0] -- a product with exact zeros and ones, so the two runs agree bit for bit."""
+    w = syn.small_variant(TINY, batch=2, n_fresh=2, K=4, ragged_lo=5, prefix=21)
+    wt = _np_weights(syn.make_weights(w))
+    inp = _np_inputs(syn.make_step_inputs(w))
+    cfg = _cfg(w)
+    h = w.hidden
+    g_bits = inp["feats"].reshape(-1, 3 * h)[:, :h].copy()                      # any bf16 rows serve as g
+    eye = np.zeros((h, 3 * h), dtype=np.float32)
+    eye[np.arange(h), np.arange(h)] = 1.0
+    wt_id = dict(wt, w_fc=syn.bf16_bits(torch.from_numpy(eye).to(torch.bfloat16)))
+    feats3 = np.zeros((g_bits.shape[0], 3 * h), dtype=g_bits.dtype)
+    feats3[:, :h] = g_bits
+    ref = ofw.draft_forward(cfg, wt_id, dict(inp, feats=feats3.reshape(inp["feats"].shape)))
+    got = ofw.draft_forward(cfg, dict(wt, w_fc=None), dict(inp, feats=g_bits.reshape(inp["feats"].shape[:-1] + (h,))))
+    assert np.array_equal(got["logits"], ref["logits"]) and np.array_equal(got["k_new"], ref["k_new"])
+    assert not np.allclose(got["logits"], ofw.draft_forward(cfg, wt, inp)["logits"])   # and it is not the random fusion
