@@ -58,7 +58,8 @@ typedef struct dart_config {
   int32_t head_dim;      /* d_h: 64 or 128 */
   int32_t mlp_inter;     /* I; multiple of 16 */
   int32_t vocab;         /* V; multiple of 16, < 2^21 */
-  int32_t feat_in;       /* width of the concatenated target features (3h); multiple of 16 */
+  int32_t feat_in;       /* width of the concatenated target features (3h); multiple of 16.  0: the caller fuses the
+                            features itself and passes g [.., hidden] as `feats`; w_fc is unused, no prefill */
   int32_t max_batch;     /* sequences per call; <= 32 and max_batch * K <= 128 */
   int32_t max_prefix;    /* P_cap: rows per sequence in the caller's KV cache */
   int32_t K;             /* query rows per sequence = future positions d (Section 3.2); 1..8 */
@@ -132,7 +133,8 @@ typedef struct dart_ngram_host {
 typedef struct dart_step_in {
   int32_t batch;          /* B <= max_batch */
   int32_t n_fresh;        /* F, 0..K (0: K mask rows, feats/tokens unused) */
-  const void* feats;      /* DEVICE bf16 [B, F, feat_in]  (packed [sum F_b, feat_in] with fresh_counts_host) */
+  const void* feats;      /* DEVICE bf16 [B, F, feat_in]  (packed [sum F_b, feat_in] with fresh_counts_host); with
+                             feat_in = 0 the fused features g, [B, F, hidden] */
   const int32_t* tokens;  /* DEVICE i32  [B, F] next-token ids, 0 <= id < V  (packed [sum F_b]) */
   const int32_t* seq_lens;      /* DEVICE i32 [B]  P_b: rows already in the cache */
   const int32_t* seq_lens_host; /* HOST   i32 [B]  same values; used for capacity checks and launch sizing */

@@ -180,7 +180,8 @@ class DartDraft:
     def __init__(self, cfg: DartConfig, weights: Dict[str, torch.Tensor], ngram: Optional[Dict[str, np.ndarray]] = None):
         self._h = C.c_void_p()
         self.cfg = cfg
-        self._weights = {n: weights[n] for n in WEIGHT_NAMES}      # keep the device tensors alive
+        names = [n for n in WEIGHT_NAMES if not (n == "w_fc" and cfg.feat_in == 0)]   # no fusion matrix without a feature FC
+        self._weights = {n: weights[n] for n in names}             # keep the device tensors alive
         for n, t in self._weights.items():
             assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous(), n
         ws = DartWeights(**{n: t.data_ptr() for n, t in self._weights.items()})

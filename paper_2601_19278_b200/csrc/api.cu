@@ -97,7 +97,7 @@ bool config_ok(const dart_config* c) {
   if ((c->n_q_heads / c->n_kv_heads) * c->K > 64) return false;
   if (c->mlp_inter < 16 || c->mlp_inter % 16 != 0) return false;
   if (c->vocab < 16 || c->vocab % 16 != 0 || c->vocab >= (1 << 21) - 1) return false;
-  if (c->feat_in < 16 || c->feat_in % 16 != 0) return false;
+  if (c->feat_in != 0 && (c->feat_in < 16 || c->feat_in % 16 != 0)) return false;   // 0: the caller passes g itself
   if (c->max_batch < 1 || c->max_batch > 32 || c->max_batch * c->K > 128) return false;
   if (c->max_prefix < 1) return false;
   if (c->topk < 1 || c->topk > 32 || c->topk > c->vocab) return false;
@@ -300,8 +300,9 @@ void build_plans(const dart_config& c, const dart_weights* w, int n_sm, bool umm
   const int h = c.hidden, dq = c.n_q_heads * c.head_dim, dkv = c.n_kv_heads * c.head_dim;
   auto W = [&](const void* p, long long off) { return w ? static_cast<const bf16*>(p) + off : nullptr; };
   GemmSeg s[6];
-  s[0] = {W(w ? w->w_fc : nullptr, 0), h, 0, c.feat_in, 0};
-  make_plan_host(ps.fc, s, 1, c.feat_in, grid, 0);
+  // without a feature FC (feat_in = 0) its plan is a stand-in over the first hidden columns of w_q, never launched
+  s[0] = c.feat_in > 0 ? GemmSeg{W(w ? w->w_fc : nullptr, 0), h, 0, c.feat_in, 0} : GemmSeg{W(w ? w->w_q : nullptr, 0), h < dq ? h : dq, 0, 2 * h, 0};
+  make_plan_host(ps.fc, s, 1, c.feat_in > 0 ? c.feat_in : h, grid, 0);
   // QKV reads z = [g-half | e-half] (2h wide); the two halves carry different 1/rms factors, so each
   // weight matrix is split into its g-half and e-half columns and the halves are finalized in pairs
   const int qt = (dq + 127) / 128, kt = (dkv + 127) / 128;
@@ -396,7 +397,7 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
                         weights->w_q, weights->w_k, weights->w_v, weights->w_o, weights->norm_post,
                         weights->w_gate, weights->w_up, weights->w_down, weights->norm_final, weights->w_lm};
   for (int i = 0; i < 15; ++i)
-    if (!aligned32(wp[i])) return DART_ERR_INVALID_ARG;  // the matrices are streamed with 32-byte loads
+    if (!aligned32(wp[i]) && !(i == 0 && cfg->feat_in == 0)) return DART_ERR_INVALID_ARG;  // the matrices are streamed with 32-byte loads
   if (ngram != nullptr && ngram->n_rows > 0 &&
       (ngram->order == nullptr || ngram->ctx0 == nullptr || ngram->ctx1 == nullptr || ngram->next == nullptr ||
        ngram->score == nullptr))
@@ -643,6 +644,9 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
     ep.out_hi = ws.z_hi; ep.out_lo = ws.z_lo; ep.ld_out = 2 * hdim; ep.ss_out = ws.ss_g;
     ep.tokens = in->tokens; ep.vocab = c.vocab; ep.embed = static_cast<const bf16*>(h->w.embed);
     ep.gamma_e = static_cast<const bf16*>(h->w.norm_e);
+    if (c.feat_in == 0) {   // the caller fused the features: feats = g [fresh rows][hidden]
+      if ((e = launch_prefused_rows(ep, static_cast<const bf16*>(in->feats), NF, st)) != cudaSuccess) return fail_cuda(h, e);
+    } else {
     gi = {static_cast<const bf16*>(in->feats), nullptr, c.feat_in, NF};
     if (h->umma && (h->maps_feats != in->feats || h->maps_fc_M != NF)) {
       // plain bf16 input: one box of 2 * MP rows, the rows past the fresh rows (the "lo" half among them) read as zeros
@@ -652,6 +656,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
       h->maps_feats = in->feats; h->maps_fc_M = NF;
     }
     if ((e = project(h->plan_fc, h->maps_fc)) != cudaSuccess) return fail_cuda(h, e);
+    }
   }
   mark(0, false);
 

@@ -177,6 +177,52 @@ cudaError_t launch_fill_mask_rows(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, 
   return cudaGetLastError();
 }
 
+// Pre-fused features (feat_in = 0): the caller hands g [fresh rows][h] itself, so the feature FC is skipped and
+// this kernel does what its prologue and epilogue do for one fresh row per block (Section 3.2): the residual
+// g as fp32, z's g half = hi/lo of g * gain, the sums of squares of g per 128-column tile (the 1/rms is applied
+// after the QKV projection), and z's e half = RMSNorm of the next token's embedding.
+__global__ void __launch_bounds__(128) prefused_rows_kernel(const EpiArgs e, const bf16* __restrict__ g, int MP) {
+  __shared__ float sh[32];
+  const int t = blockIdx.x, tid = threadIdx.x;
+  pdl_wait();
+  const int orow = fresh_to_step_row(e, t);
+  const bf16* grow = g + (size_t)t * e.h;
+  for (int n0 = 0, tile = 0; n0 < e.h; n0 += 128, ++tile) {
+    const int n = n0 + tid;
+    float x = 0.f;
+    if (n < e.h) {
+      x = __bfloat162float(grow[n]);
+      e.res0[(size_t)t * e.h + n] = x;
+      bf16 hi, lo;
+      split_bf16(x * __bfloat162float(e.gamma[n]), hi, lo);
+      e.out_hi[(size_t)orow * e.ld_out + n] = hi;
+      e.out_lo[(size_t)orow * e.ld_out + n] = lo;
+    }
+    const float ss = block_sum(x * x, sh);
+    if (tid == 0) e.ss_out[(size_t)tile * MP + t] = ss;
+  }
+  // the shifted token embedding of this fresh row
+  const int id = min(max(e.tokens[t], 0), e.vocab - 1);
+  const bf16* row = e.embed + (size_t)id * e.h;
+  float ss = 0.f;
+  for (int n = tid; n < e.h; n += 128) {
+    const float v = __bfloat162float(row[n]);
+    ss += v * v;
+  }
+  ss = block_sum(ss, sh);
+  const float rs = 1.f / sqrtf(ss / (float)e.h + e.eps);
+  for (int n = tid; n < e.h; n += 128) {
+    bf16 hi, lo;
+    split_bf16(__bfloat162float(row[n]) * rs * __bfloat162float(e.gamma_e[n]), hi, lo);
+    e.out_hi[(size_t)orow * e.ld_out + e.h + n] = hi;
+    e.out_lo[(size_t)orow * e.ld_out + e.h + n] = lo;
+  }
+}
+
+cudaError_t launch_prefused_rows(const EpiArgs& e, const bf16* g, int n_fresh, cudaStream_t st) {
+  return launch_pdl(prefused_rows_kernel, dim3(n_fresh), dim3(128), 0, st, e, g, padded_tokens(n_fresh));
+}
+
 cudaError_t launch_mask_row(const bf16* mask_vec, const bf16* norm_g, const bf16* norm_e, int h, float eps, bf16* z_hi,
                             bf16* z_lo, float* rstd_mask, float* mask_res, cudaStream_t st) {
   mask_row_kernel<<<1, 256, 0, st>>>(mask_vec, norm_g, norm_e, h, eps, z_hi, z_lo, rstd_mask, mask_res);

@@ -203,6 +203,8 @@ struct FreshOffsets { int v[33]; };   // prefix sums of the per-sequence fresh c
 cudaError_t launch_fill_mask_rows(bf16* z_hi, bf16* z_lo, const bf16* zmask_hi, const bf16* zmask_lo, int B, int K,
                                   const FreshOffsets& foff, int width, cudaStream_t st);
 // z row of the <mask> rows and the 1/rms of its g half (once, at init)
+// feat_in = 0: g [n_fresh][h] given by the caller; writes what the feature FC's prologue and epilogue write.
+cudaError_t launch_prefused_rows(const EpiArgs& e, const bf16* g, int n_fresh, cudaStream_t st);
 cudaError_t launch_mask_row(const bf16* mask_vec, const bf16* norm_g, const bf16* norm_e, int h, float eps, bf16* z_hi,
                             bf16* z_lo, float* rstd_mask, float* mask_res, cudaStream_t st);
 

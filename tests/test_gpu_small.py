@@ -194,3 +194,32 @@ def test_per_sequence_fresh_counts_match_oracle(name, counts):
         for key in ("n_nodes", "tokens", "parents", "depth", "mask"):
             assert np.array_equal(got[key][b], np.asarray(t[key])), (b, key)
     ses.close()
+
+
+def test_prefused_features_skip_the_feature_fc():
+    """feat_in = 0: the caller passes g itself; logits, candidates and the appended cache rows against the oracle."""
+    w = syn.small_variant(C1, batch=3, ragged_lo=9, prefix=70, K=4, n_fresh=2, vocab=2064)
+    wt = syn.make_weights(w)
+    inp = syn.make_step_inputs(w)
+    g = torch.Generator().manual_seed(21)
+    inp["feats"] = torch.randn(w.batch, 2, w.hidden, generator=g).to(torch.bfloat16)     # g instead of 3h features
+    ses = runner.DraftSession(w, wt, None, want_logits=True, philox_seed=parity.PHILOX_SEED, feat_in=0)
+    ses.load_inputs(inp)
+    ses.step(step_counter=5)
+    torch.cuda.synchronize()
+    assert ses.draft.device_status() == 0
+    npw = parity.np_weights(wt)
+    npw["w_fc"] = None
+    ref = ofw.draft_forward(parity.oracle_cfg(w), npw, parity.np_inputs(inp))
+    stats = parity.check_logits(ses.logits.cpu().numpy(), ref["logits"])
+    assert stats["max_abs"] < parity.TOL_ABS
+    ids_g, sl_g = ses.topk_ids.cpu().numpy(), ses.topk_slogit.cpu().numpy()
+    for b in range(w.batch):
+        for r in range(w.K):
+            parity.check_topk_row(ids_g[b, r], sl_g[b, r], ref["logits"][b, r], ses.cfg.topk, 1e-10, 0.0, None)
+    kc = ses.inp["k_cache"].float().cpu().numpy()
+    for b in range(w.batch):
+        P = int(inp["seq_lens"][b])
+        for r in range(2):
+            np.testing.assert_allclose(kc[b, :, P + r], ref["k_new"][b, r], rtol=1e-2, atol=2e-2)
+    ses.close()
