@@ -223,3 +223,25 @@ def test_prefused_features_skip_the_feature_fc():
         for r in range(2):
             np.testing.assert_allclose(kc[b, :, P + r], ref["k_new"][b, r], rtol=1e-2, atol=2e-2)
     ses.close()
+
+
+def test_tensor_core_attention_edge_lengths():
+    """The split-KV attention on tcgen05 with sequences of 0, 63, 64 and 65 cached positions next to long ones: an
+    empty cache (only the new rows), a partial single tile, an exact tile, a one-key second tile."""
+    w = syn.small_variant(C1, hidden=512, n_q_heads=32, n_kv_heads=16, head_dim=128, mlp_inter=1376, vocab=2064,
+                          batch=8, ragged_lo=3000, prefix=4000, K=8, tree_budget=60)
+    wt = syn.make_weights(w)
+    inp = syn.make_step_inputs(w)
+    lens = inp["seq_lens"].clone()
+    lens[:4] = torch.tensor([0, 63, 64, 65], dtype=lens.dtype)
+    inp["seq_lens"] = lens
+    assert sum((int(x) + 63) // 64 for x in lens) * w.n_kv_heads >= 2048     # enough key tiles for that kernel
+    ses = runner.DraftSession(w, wt, None, want_logits=True, philox_seed=parity.PHILOX_SEED)
+    ses.load_inputs(inp)
+    ses.step(step_counter=5)
+    torch.cuda.synchronize()
+    assert ses.draft.device_status() == 0
+    ref = parity.oracle_forward(w, wt, inp)
+    stats = parity.check_logits(ses.logits.cpu().numpy(), ref["logits"])
+    assert stats["max_abs"] < parity.TOL_ABS
+    ses.close()
