@@ -447,24 +447,29 @@ cudaError_t launch_lm_head_umma(const LmParams& pin, const CUtensorMap& mapW, co
 // token rows are the M side of tcgen05.mma (hi and lo as two MMAs into one accumulator) and 256 vocabulary rows
 // its N side, so a stage carries 32 KB of activations for 32 KB of weights.  The accumulator row of a token
 // is one TMEM lane, i.e. one read-out thread: that thread keeps the token's running (max, sum-exp) in registers
-// and its best-`topk` candidates in a shared-memory row of its own (replace-the-worst; sorted once at the end),
-// so the fold needs no cross-thread step at all.  Work split, ownership of tiles cut between CTAs, flags and
+// and its best-`topk` candidates in a shared-memory row of its own (a heap rooted at the last-ranked entry; sorted
+// once at the end), so the fold needs no cross-thread step at all.  Work split, ownership of tiles cut between CTAs, flags and
 // bounded waits are those of lm_head_umma_kernel, with 256-row tiles.
 // ------------------------------------------------------------------------------------------------------
-constexpr int kLmDenseStages = 3;
+// Two read-out threads per token row, one per half of a tile's 256 columns (warps 4-7 and 8-11), each with its own
+// statistics and list: one warp per scheduler ran the fold at several cycles per instruction and was the longest
+// part of the kernel; two halve that.  The second set of lists takes the shared memory of the ring's third stage
+// (three stages without the fold: 320 us; two: 372 us; fold on one warp set: 748 us).
+constexpr int kLmDenseStages = 2;
+constexpr int kLmDenseThreads = 384;
 constexpr int kLmDenseStageBytes = 2 * 128 * 64 * 2 + 256 * 64 * 2;   // hi tokens, lo tokens, 256 vocabulary rows
 constexpr int kLmDenseListStride = 33;                                  // floats per token row of the lists (no bank conflicts)
-constexpr size_t kLmDenseSmem = (size_t)kLmDenseStages * kLmDenseStageBytes + 1024 + 2 * 128 * kLmDenseListStride * 4;
+constexpr size_t kLmDenseSmem = (size_t)kLmDenseStages * kLmDenseStageBytes + 1024 + 2 * 2 * 128 * kLmDenseListStride * 4;
 
 // (key, id) a precedes (key, id) b in the candidate order: larger key first, then smaller id
 __device__ __forceinline__ bool cand_before(float ka, int ia, float kb, int ib) { return ka > kb || (ka == kb && ia < ib); }
 
-__global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const __grid_constant__ LmUmmaArgs a) {
+__global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const __grid_constant__ LmUmmaArgs a) {
   const LmParams& p = a.p;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  float* l_key = reinterpret_cast<float*>(ring + (size_t)kLmDenseStages * kLmDenseStageBytes);   // [128][33]
-  int* l_id = reinterpret_cast<int*>(l_key + 128 * kLmDenseListStride);                           // [128][33]
+  float* l_key = reinterpret_cast<float*>(ring + (size_t)kLmDenseStages * kLmDenseStageBytes);   // [2 halves][128][33]
+  int* l_id = reinterpret_cast<int*>(l_key + 2 * 128 * kLmDenseListStride);                       // [2 halves][128][33]
   __shared__ uint64_t full[kLmDenseStages], empty[kLmDenseStages], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base;
   __shared__ int abort_flag, s_bad;
@@ -476,7 +481,7 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const 
 
   if (tid == 0) {
     for (int s = 0; s < kLmDenseStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 256); }
     abort_flag = 0;
     s_bad = 0;
     fence_barrier_init();
@@ -557,11 +562,12 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const 
     }
     if (ok && tile >= 0) mma_commit(&acc_full[buf]);
   } else if (warp >= 4) {
-    // ---- read-out and fold: TMEM lane = token row; this thread owns the token's statistics and list
-    const int wq = warp & 3, tok = wq * 32 + lane, et = tid - 128;
+    // ---- read-out and fold: TMEM lane = token row; this thread owns one half of the columns of the token's row of
+    // every tile, with statistics and a list of its own (the two halves are merged at the end)
+    const int wq = warp & 3, half = (warp - 4) >> 2, tok = wq * 32 + lane, et = tid - 128;
     const bool live = tok < p.M;
-    float* my_key = l_key + tok * kLmDenseListStride;
-    int* my_id = l_id + tok * kLmDenseListStride;
+    float* my_key = l_key + (half * 128 + tok) * kLmDenseListStride;
+    int* my_id = l_id + (half * 128 + tok) * kLmDenseListStride;
     pdl_wait();
     float rstd = 0.f;
     if (live) {  // the final RMSNorm's 1/rms from the previous kernel's sums of squares (same order everywhere)
@@ -570,47 +576,34 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const 
       rstd = 1.f / sqrtf(ssq / (float)p.Kd + p.rms_eps);
     }
     float m_run = -INFINITY, s_run = 0.f;
-    // The token's candidate list: up to 33 entries in this thread's shared-memory row.  An entry is appended when
-    // it may precede the threshold (the last-ranked entry kept by the latest compaction); when any row of the warp
-    // is full the whole warp compacts together -- keeps its best `topk`, renews its threshold -- so the 32 rows do
-    // their list work in step instead of one at a time.  An entry appended at temperature > 0 carries the plain
-    // logit and a pending mark: its exact perturbed key is computed at the next compaction.  (Keeping the kept
-    // part sorted and inserting the appended entries was slower: its shift loop is one dependent chain.)
+    // The token's candidates: a binary heap in this thread's shared-memory row, its root the last-ranked entry kept,
+    // i.e. the exact threshold a new logit has to precede.  An insertion is a walk of at most five levels, so a
+    // warp whose rows insert at different moments loses little (replace-the-worst rescanned all `topk` entries
+    // whenever any row inserted; append-and-compact paid ~4000 instructions per compaction).
     int n_list = 0;
-    bool have_thr = false;
-    float t_key = -INFINITY; int t_id = 0x7fffffff;
     const int topk = p.topk;
-    constexpr int kPending = 1 << 30;
-    auto compact = [&]() {
-      if (p.gumbel) {
-        for (int e = 0; e < n_list; ++e) {
-          const int ie = my_id[e];
-          if (ie & kPending) {
-            const int v = ie & ~kPending;
-            const uint4 rnd = philox4x32_10(make_uint4((uint32_t)v >> 2, (uint32_t)(tok % p.K), (uint32_t)(tok / p.K), p.step), p.seed_lo, p.seed_hi);
-            const uint32_t wsel = (v & 3) == 0 ? rnd.x : ((v & 3) == 1 ? rnd.y : ((v & 3) == 2 ? rnd.z : rnd.w));
-            my_key[e] += gumbel_from_bits(wsel);
-            my_id[e] = v;
-          }
+    auto worse = [&](int x, int y) { return cand_before(my_key[y], my_id[y], my_key[x], my_id[x]); };   // entry x ranks after entry y
+    auto heap_insert = [&](float ke, int ie) {
+      if (n_list < topk) {                       // grow: the new leaf rises while it ranks after its parent
+        int i = n_list++;
+        while (i > 0) {
+          const int up = (i - 1) >> 1;
+          if (!cand_before(my_key[up], my_id[up], ke, ie)) break;          // the parent does not rank before it: stop
+          my_key[i] = my_key[up]; my_id[i] = my_id[up];
+          i = up;
         }
-      }
-      while (n_list > topk) {                  // drop the last-ranked entry until topk are left
-        int worst = 0;
-        float wk = my_key[0]; int wi = my_id[0];
-        for (int e = 1; e < n_list; ++e) {
-          const float ke = my_key[e]; const int ie = my_id[e];
-          if (cand_before(wk, wi, ke, ie)) { wk = ke; wi = ie; worst = e; }
+        my_key[i] = ke; my_id[i] = ie;
+      } else if (cand_before(ke, ie, my_key[0], my_id[0])) {               // replace the root, sink it
+        int i = 0;
+        for (;;) {
+          int ch = 2 * i + 1;
+          if (ch >= topk) break;
+          if (ch + 1 < topk && worse(ch + 1, ch)) ++ch;                    // the later-ranked child
+          if (!cand_before(ke, ie, my_key[ch], my_id[ch])) break;          // the new entry ranks after both children
+          my_key[i] = my_key[ch]; my_id[i] = my_id[ch];
+          i = ch;
         }
-        --n_list;
-        my_key[worst] = my_key[n_list]; my_id[worst] = my_id[n_list];
-      }
-      if (n_list == topk) {                    // the threshold: the last-ranked of the kept entries
-        float wk = my_key[0]; int wi = my_id[0];
-        for (int e = 1; e < n_list; ++e) {
-          const float ke = my_key[e]; const int ie = my_id[e];
-          if (cand_before(wk, wi, ke, ie)) { wk = ke; wi = ie; }
-        }
-        t_key = wk; t_id = wi; have_thr = true;
+        my_key[i] = ke; my_id[i] = ie;
       }
     };
     int visit = 0;
@@ -631,16 +624,16 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const 
         }
         __threadfence();
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
       if (s_bad) break;
       tc_fence_after();
       const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + buf * 256;
 #pragma unroll 1
-      for (int cb = 0; cb < 256; cb += 16) {
+      for (int cb = half * 128; cb < half * 128 + 128; cb += 16) {
         uint32_t r[16];
         tmem_ld16(tbase + cb, r);
         tmem_ld_wait();
-        if (cb == 240) {  // the accumulator buffer is free once its last columns are in registers
+        if (cb == half * 128 + 112) {  // the accumulator buffer is free once both halves' last columns are in registers
           tc_fence_before();
           mbar_arrive(&acc_empty[buf]);
         }
@@ -684,65 +677,74 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const 
           for (int j = 0; j < 16; ++j) e4[j & 3] += expf(y[j] - m_run);
           s_run += (e4[0] + e4[1]) + (e4[2] + e4[3]);
         }
-        // which of the 16 logits may precede the threshold.  At temperature > 0 the key is y + G(u): a fast
-        // evaluation of G decides with a margin 10x its error bound (u in [2^-14, 1 - 2^-8]: |error| < 1.2e-4;
-        // outside that range the entry is simply kept as a candidate); exact keys come at the compaction.
+        // which of the 16 logits may precede the threshold (the heap's root once `topk` are kept).  At temperature
+        // > 0 the key is y + G(u): a fast evaluation of G decides with a margin 10x its error bound (u in
+        // [2^-14, 1 - 2^-8]: |error| < 1.2e-4; other u always pass); the exact fp32 G is computed for those only.
+        const bool full = n_list == topk;
+        const float t_key = full ? my_key[0] : -INFINITY;
+        const int t_id = full ? my_id[0] : 0x7fffffff;
         uint32_t may = 0u;
+        uint32_t bits[16];
         if (p.gumbel) {
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             const uint4 rnd = philox4x32_10(make_uint4((uint32_t)((v0 >> 2) + q4), (uint32_t)(tok % p.K), (uint32_t)(tok / p.K), p.step), p.seed_lo, p.seed_hi);
-            const uint32_t rw[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+            bits[4 * q4] = rnd.x; bits[4 * q4 + 1] = rnd.y; bits[4 * q4 + 2] = rnd.z; bits[4 * q4 + 3] = rnd.w;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              const uint32_t m = rw[q] >> 8;
+              const uint32_t m = bits[4 * q4 + q] >> 8;
               const float gq = -__logf(-__logf(((float)m + 0.5f) * (1.f / 16777216.f)));
               const bool safe = m >= 1024u && m <= (1u << 24) - 65536u;
-              if (!have_thr || !safe || y[4 * q4 + q] + gq + 1e-3f >= t_key) may |= 1u << (4 * q4 + q);
+              if (!full || !safe || y[4 * q4 + q] + gq + 1e-3f >= t_key) may |= 1u << (4 * q4 + q);
             }
           }
         } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (!have_thr || cand_before(y[j], v0 + j, t_key, t_id)) may |= 1u << j;
+          for (int j = 0; j < 16; ++j) {
+            bits[j] = 0u;
+            if (!full || cand_before(y[j], v0 + j, t_key, t_id)) may |= 1u << j;
+          }
         }
         if (!live) may = 0u;
 #pragma unroll 1
-        while (__any_sync(0xffffffffu, may != 0u)) {
-          if (may != 0u) {
-            const int j = __ffs(may) - 1;
-            may &= may - 1u;
-            float yj = y[0];
+        while (may != 0u) {                      // one candidate per round; rows of a warp go through their rounds together
+          const int j = __ffs(may) - 1;
+          may &= may - 1u;
+          float yj = y[0];
+          uint32_t bj = bits[0];
 #pragma unroll
-            for (int q = 1; q < 16; ++q) yj = q == j ? y[q] : yj;
-            my_key[n_list] = yj;
-            my_id[n_list] = (v0 + j) | (p.gumbel ? kPending : 0);
-            ++n_list;
-          }
-          if (__any_sync(0xffffffffu, n_list == kLmDenseListStride)) {
-            compact();
-            // entries of this chunk not yet appended are re-checked against the new threshold when keys are exact
-            if (!p.gumbel && have_thr) {
-              uint32_t keep = 0u;
-#pragma unroll
-              for (int q = 0; q < 16; ++q)
-                if (((may >> q) & 1u) && cand_before(y[q], v0 + q, t_key, t_id)) keep |= 1u << q;
-              may = keep;
-            }
-          }
+          for (int q = 1; q < 16; ++q) { yj = q == j ? y[q] : yj; bj = q == j ? bits[q] : bj; }
+          heap_insert(p.gumbel ? yj + gumbel_from_bits(bj) : yj, v0 + j);
         }
       }
       if (!owner) {
         __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (et == 0) *reinterpret_cast<volatile int*>(a.flags + c) = a.tag;
       }
       ++visit;
       u = ue;
     }
     // ---- this token's list, sorted (key desc, id asc), and its statistics
-    compact();                                      // exact keys for the pending entries, the best topk kept
-    if (live) {
+    // ---- the second half's statistics and list join the first half's (the ring is free by now: scratch)
+    float* x_m = reinterpret_cast<float*>(ring);
+    float* x_s = x_m + 128;
+    int* x_n = reinterpret_cast<int*>(x_s + 128);
+    if (half == 1) { x_m[tok] = m_run; x_s[tok] = s_run; x_n[tok] = n_list; }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (half == 0) {
+      const float m1 = x_m[tok], s1 = x_s[tok];
+      if (m1 != -INFINITY) {
+        const float mn = fmaxf(m_run, m1);
+        s_run = (m_run == -INFINITY ? 0.f : s_run * expf(m_run - mn)) + s1 * expf(m1 - mn);
+        m_run = mn;
+      }
+      const float* k1 = l_key + (128 + tok) * kLmDenseListStride;
+      const int* i1 = l_id + (128 + tok) * kLmDenseListStride;
+      const int n1 = x_n[tok];
+      for (int e1 = 0; e1 < n1; ++e1) heap_insert(k1[e1], i1[e1]);
+    }
+    if (live && half == 0) {
       for (int i = 1; i < n_list; ++i) {            // insertion sort of at most 32 entries
         const float ki = my_key[i]; const int ii = my_id[i];
         int j = i - 1;
@@ -777,11 +779,11 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_dense_kernel(const 
     for (int i = 0; i < 100; ++i) __nanosleep(1000);
   }
   // token rows past M leave empty lists (the merge reads MP = 128 rows per CTA)
-  for (int i = tid; i < (128 - p.M) * 32; i += kLmUmmaThreads) {
+  for (int i = tid; i < (128 - p.M) * 32; i += kLmDenseThreads) {
     const size_t o = ((size_t)c * 128 + p.M) * 32 + i;
     p.part_key[o] = -INFINITY; p.part_y[o] = 0.f; p.part_id[o] = 0x7fffffff;
   }
-  for (int i = tid; i < (128 - p.M) * 2; i += kLmUmmaThreads) p.part_stats[((size_t)c * 128 + p.M) * 2 + i] = (i & 1) ? 0.f : -INFINITY;
+  for (int i = tid; i < (128 - p.M) * 2; i += kLmDenseThreads) p.part_stats[((size_t)c * 128 + p.M) * 2 + i] = (i & 1) ? 0.f : -INFINITY;
 }
 
 cudaError_t launch_lm_head_dense(const LmParams& pin, const CUtensorMap& mapW256, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
@@ -795,7 +797,7 @@ cudaError_t launch_lm_head_dense(const LmParams& pin, const CUtensorMap& mapW256
   a.pieces = pieces; a.flags = flags; a.tag = tag; a.status = status;
   const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(lm_head_dense_kernel), kLmDenseSmem);
   if (e != cudaSuccess) return e;
-  return launch_pdl(lm_head_dense_kernel, dim3(a.p.grid), dim3(kLmUmmaThreads), kLmDenseSmem, st, a);
+  return launch_pdl(lm_head_dense_kernel, dim3(a.p.grid), dim3(kLmDenseThreads), kLmDenseSmem, st, a);
 }
 
 template <int NT, int NW>
