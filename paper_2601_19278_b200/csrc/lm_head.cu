@@ -459,7 +459,7 @@ constexpr int kLmDenseStages = 2;
 constexpr int kLmDenseThreads = 384;
 constexpr int kLmDenseStageBytes = 2 * 128 * 64 * 2 + 256 * 64 * 2;   // hi tokens, lo tokens, 256 vocabulary rows
 constexpr int kLmDenseListStride = 33;                                  // floats per token row of the lists (no bank conflicts)
-constexpr size_t kLmDenseSmem = (size_t)kLmDenseStages * kLmDenseStageBytes + 1024 + 2 * 2 * 128 * kLmDenseListStride * 4;
+constexpr size_t kLmDenseSmem = (size_t)kLmDenseStages * kLmDenseStageBytes + 1024 + 2 * 2 * 128 * kLmDenseListStride * 4 + 2 * 128 * 4;
 
 // (key, id) a precedes (key, id) b in the candidate order: larger key first, then smaller id
 __device__ __forceinline__ bool cand_before(float ka, int ia, float kb, int ib) { return ka > kb || (ka == kb && ia < ib); }
@@ -470,6 +470,7 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   float* l_key = reinterpret_cast<float*>(ring + (size_t)kLmDenseStages * kLmDenseStageBytes);   // [2 halves][128][33]
   int* l_id = reinterpret_cast<int*>(l_key + 2 * 128 * kLmDenseListStride);                       // [2 halves][128][33]
+  volatile float* l_thr = reinterpret_cast<volatile float*>(l_id + 2 * 128 * kLmDenseListStride);  // [2 halves][128] published thresholds
   __shared__ uint64_t full[kLmDenseStages], empty[kLmDenseStages], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base;
   __shared__ int abort_flag, s_bad;
@@ -580,6 +581,10 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
     // i.e. the exact threshold a new logit has to precede.  An insertion is a walk of at most five levels, so a
     // warp whose rows insert at different moments loses little (replace-the-worst rescanned all `topk` entries
     // whenever any row inserted; append-and-compact paid ~4000 instructions per compaction).
+    // Each half publishes the key of its heap's root once it holds `topk` entries: the other half of the same row
+    // may skip whatever is below it too (topk entries of the row's union are at least that large), which takes away
+    // close to half of the insertions.  A stale value only prunes less; the merged list does not depend on timing.
+    l_thr[half * 128 + tok] = -INFINITY;
     int n_list = 0;
     const int topk = p.topk;
     auto worse = [&](int x, int y) { return cand_before(my_key[y], my_id[y], my_key[x], my_id[x]); };   // entry x ranks after entry y
@@ -671,18 +676,20 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
           float cm = y[0];
 #pragma unroll
           for (int j = 1; j < 16; ++j) cm = fmaxf(cm, y[j]);
-          if (cm > m_run) { s_run *= expf(m_run - cm); m_run = cm; }
+          if (cm > m_run) { s_run *= __expf(m_run - cm); m_run = cm; }
           float e4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int j = 0; j < 16; ++j) e4[j & 3] += expf(y[j] - m_run);
+          for (int j = 0; j < 16; ++j) e4[j & 3] += __expf(y[j] - m_run);   // ex2.approx: ~2e-6 relative, far inside s_logit's tolerance
           s_run += (e4[0] + e4[1]) + (e4[2] + e4[3]);
         }
         // which of the 16 logits may precede the threshold (the heap's root once `topk` are kept).  At temperature
         // > 0 the key is y + G(u): a fast evaluation of G decides with a margin 10x its error bound (u in
         // [2^-14, 1 - 2^-8]: |error| < 1.2e-4; other u always pass); the exact fp32 G is computed for those only.
         const bool full = n_list == topk;
+        const float o_key = l_thr[(half ^ 1) * 128 + tok];             // the other half's threshold (or -inf)
         const float t_key = full ? my_key[0] : -INFINITY;
         const int t_id = full ? my_id[0] : 0x7fffffff;
+        if (full) l_thr[half * 128 + tok] = t_key;
         uint32_t may = 0u;
         uint32_t bits[16];
         if (p.gumbel) {
@@ -695,14 +702,15 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
               const uint32_t m = bits[4 * q4 + q] >> 8;
               const float gq = -__logf(-__logf(((float)m + 0.5f) * (1.f / 16777216.f)));
               const bool safe = m >= 1024u && m <= (1u << 24) - 65536u;
-              if (!full || !safe || y[4 * q4 + q] + gq + 1e-3f >= t_key) may |= 1u << (4 * q4 + q);
+              const float kq = y[4 * q4 + q] + gq + 1e-3f;
+              if ((!full || !safe || kq >= t_key) && (!safe || kq >= o_key)) may |= 1u << (4 * q4 + q);
             }
           }
         } else {
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             bits[j] = 0u;
-            if (!full || cand_before(y[j], v0 + j, t_key, t_id)) may |= 1u << j;
+            if ((!full || cand_before(y[j], v0 + j, t_key, t_id)) && y[j] >= o_key) may |= 1u << j;
           }
         }
         if (!live) may = 0u;
@@ -714,7 +722,8 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
           uint32_t bj = bits[0];
 #pragma unroll
           for (int q = 1; q < 16; ++q) { yj = q == j ? y[q] : yj; bj = q == j ? bits[q] : bj; }
-          heap_insert(p.gumbel ? yj + gumbel_from_bits(bj) : yj, v0 + j);
+          const float kj = p.gumbel ? yj + gumbel_from_bits(bj) : yj;
+          if (kj >= o_key) heap_insert(kj, v0 + j);
         }
       }
       if (!owner) {
