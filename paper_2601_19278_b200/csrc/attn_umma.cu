@@ -5,12 +5,13 @@
 // mma.sync pairs (tensor pipe 42 % busy at 2.1 TB/s on 16 sequences):
 //   * a CTA runs two (sequence, KV head, chunk) pipelines side by side -- two consecutive chunks of one sequence,
 //     which share the Q tiles -- each with its own producer thread (TMA, 128-byte swizzle, two K and two V stages
-//     of 64 keys), MMA issuer thread, and two softmax warps (query rows 0..63 = tensor-memory lanes 0..63);
-//   * S = Q_hi K^T + Q_lo K^T by tcgen05.mma 128 x 64 (k = 128) into one of two tensor-memory buffers (the M = 128
-//     instruction runs over 64 real query rows; the upper accumulator rows are never read);
+//     of 64 keys), MMA issuer thread, and four softmax warps;
+//   * S = Q_hi K^T + Q_lo K^T by tcgen05.mma 64 x 64 (k = 128) into one of two tensor-memory buffers.  An M = 64
+//     accumulator puts row r in lane 32 (r / 16) + r % 16, so each of the four softmax warps of a pipeline owns
+//     16 rows (lanes 0..15 of its lane quarter) and all four schedulers take part;
 //   * one thread per query row: exp2 against a reference maximum that only moves when exceeded by 2^8 (O rescaled
 //     in tensor memory then), P split into bf16 hi + lo tiles written in the operand layout;
-//   * O += P_hi V + P_lo V by tcgen05.mma 128 x 128 (k = 64) with the V tile as stored (MN-major B operand).
+//   * O += P_hi V + P_lo V by tcgen05.mma 64 x 128 (k = 64) with the V tile as stored (MN-major B operand).
 // The step's own K new rows are one more chunk: a 16-row side tile (rows 0..7 hi parts, 8..15 lo parts), so score
 // columns c and c + 8 add up to q.k and the weight of column c is repeated on column c + 8 for v_lo.
 // Every mbarrier wait is bounded; d_h = 128.
@@ -23,12 +24,11 @@ namespace dart {
 
 using namespace umma;
 
-constexpr int kAuThreads = 320;                 // warps 0/2: producers, 1/3: MMA issuers, 4-5 and 8-9: softmax, 6-7 idle
+constexpr int kAuThreads = 384;                 // warps 0/2: producers, 1/3: MMA issuers, 4-7 and 8-11: softmax
 constexpr int kAuQ = 64 * 128 * 2;              // 64 query rows x 128: two 64-column halves of 8 KB
 constexpr int kAuP = 64 * 64 * 2;               // 64 query rows x 64 keys
 constexpr int kAuKV = 64 * 128 * 2;             // 64 keys x 128: two 64-column halves
-// Q hi, Q lo | P [pipeline][buffer][hi, lo] | K [pipeline][stage] | V [pipeline][stage].  The A operands (Q, P) come
-// first: an M = 128 instruction reads 64 rows past a 64-row tile, which must still be inside the allocation.
+// Q hi, Q lo | P [pipeline][buffer][hi, lo] | K [pipeline][stage] | V [pipeline][stage].
 constexpr size_t kAuSmem = (size_t)2 * kAuQ + 8 * kAuP + 8 * kAuKV + 1024;
 
 __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_constant__ AttnUmmaArgs a) {
@@ -57,8 +57,8 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
     for (int pl = 0; pl < 2; ++pl)
       for (int s = 0; s < 2; ++s) {
         mbar_init(&k_full[pl][s], 1); mbar_init(&k_empty[pl][s], 1); mbar_init(&v_full[pl][s], 1); mbar_init(&v_empty[pl][s], 1);
-        mbar_init(&s_full[pl][s], 1); mbar_init(&s_empty[pl][s], 2);     // one arrival per softmax warp
-        mbar_init(&p_full[pl][s], 2); mbar_init(&pv_done[pl][s], 1);
+        mbar_init(&s_full[pl][s], 1); mbar_init(&s_empty[pl][s], 4);     // one arrival per softmax warp
+        mbar_init(&p_full[pl][s], 4); mbar_init(&pv_done[pl][s], 1);
       }
     abort_flag = 0;
     fence_barrier_init();
@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
     }
   } else if ((warp == 1 || warp == 3) && lane == 0 && pl_on) {
     // ---- MMA issuer of pipeline pl
-    constexpr uint32_t idesc_s = idesc_bf16(128, 64), idesc_o = idesc_bf16(128, 128) | kIdescBMnMajor;
+    constexpr uint32_t idesc_s = idesc_bf16(64, 64), idesc_o = idesc_bf16(64, 128) | kIdescBMnMajor;
     const uint64_t dqh0 = desc_sw128(smem_u32(sQ)), dqh1 = desc_sw128(smem_u32(sQ + kAuQ / 2));
     const uint64_t dql0 = desc_sw128(smem_u32(sQ + kAuQ)), dql1 = desc_sw128(smem_u32(sQ + kAuQ + kAuQ / 2));
     bool ok = ta_wait(&q_full, 0, &abort_flag);
@@ -156,9 +156,12 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       mma_commit(&pv_done[pl][s]);
       mma_commit(&v_empty[pl][s]);
     }
-  } else if (warp >= 4 && (warp & 3) < 2 && pl_on) {
-    // ---- softmax of pipeline pl: thread = query row = tensor-memory lane (rows 0..63)
-    const int wq = warp & 3, row = wq * 32 + lane;
+  } else if (warp >= 4 && pl_on) {
+    // ---- softmax of pipeline pl: lanes 0..15 of warp quarter wq own query rows 16 wq .. 16 wq + 15 (the M = 64
+    // accumulator layout); lanes 16..31 only take part in the warp-wide tensor-memory instructions
+    const int wq = warp & 3;
+    const bool act = lane < 16;
+    const int row = act ? wq * 16 + lane : 64;
     const uint32_t tb = tmem + ((uint32_t)(wq * 32) << 16) + pl * 256;
     const int r = row % p.K;             // position of the row inside its sequence's K-block
     const float c = rsqrtf(128.f) * 1.4426950408889634f;   // 1/sqrt(d_h) * log2(e)
@@ -210,7 +213,7 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       const int valid = is_new ? 16 : min(64, k_end - (k_begin + t * 64));
       if (valid < 64) {
         if (!ta_wait(&v_full[pl][s], (t >> 1) & 1, &abort_flag)) { ok = false; break; }
-        if (row >= valid) {
+        if (act && row >= valid) {
           uint8_t* vrow = sV + (pl * 2 + s) * kAuKV + row * 128;
 #pragma unroll
           for (int ch = 0; ch < 8; ++ch) {
@@ -237,10 +240,11 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       }
       // P as hi + lo A operands: [64 rows][64 keys] each, rows of 128 bytes, 16-byte chunk ch of row r stored at
       // chunk ch ^ (r & 7) (the 128-byte swizzle)
-      uint8_t* ph = sP + ((pl * 2 + s) * 2) * kAuP + row * 128;
+      uint8_t* ph = sP + ((pl * 2 + s) * 2) * kAuP + (row & 63) * 128;
       uint8_t* plo = ph + kAuP;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {
+        if (!act) break;
         uint32_t wh[4], wl[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -268,14 +272,14 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
         uint32_t rr[16];
         tmem_ld16(tb + 128 + cb, rr);
         tmem_ld_wait();
-        if (row < R) {
+        if (act && row < R) {
           float4* dst = reinterpret_cast<float4*>(p.o_part + slot * 128 + cb);
 #pragma unroll
           for (int q = 0; q < 4; ++q)
             dst[q] = make_float4(__uint_as_float(rr[4 * q]), __uint_as_float(rr[4 * q + 1]), __uint_as_float(rr[4 * q + 2]), __uint_as_float(rr[4 * q + 3]));
         }
       }
-      if (row < R) *reinterpret_cast<float2*>(p.ml_part + slot * 2) = make_float2(m_ref, l);
+      if (act && row < R) *reinterpret_cast<float2*>(p.ml_part + slot * 2) = make_float2(m_ref, l);
     }
   }
   tc_fence_before();
