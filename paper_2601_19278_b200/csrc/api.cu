@@ -484,8 +484,8 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   if (h->umma && cfg->head_dim == 128) {   // the attention's maps over the library's own buffers
     const unsigned long long q_rows = (unsigned long long)cfg->max_batch * cfg->n_q_heads * cfg->K;
     const unsigned long long n_rows16 = (unsigned long long)cfg->max_batch * cfg->n_kv_heads * 16;
-    INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapQhi, h->ws.q_hi, 128, q_rows, 256, 64, 64));
-    INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapQlo, h->ws.q_lo, 128, q_rows, 256, 64, 64));
+    INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapQhi, h->ws.q_hi, 128, q_rows, 256, 64, 16));
+    INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapQlo, h->ws.q_lo, 128, q_rows, 256, 64, 16));
     INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapKn, h->ws.k_new, 128, n_rows16, 256, 64, 64));
     INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapVn, h->ws.v_new, 128, n_rows16, 256, 64, 64));
   }

@@ -4,14 +4,19 @@
 // both; what changes is the data path, because at batch > 1 that kernel is bound by the issue rate of its
 // mma.sync pairs (tensor pipe 42 % busy at 2.1 TB/s on 16 sequences):
 //   * a CTA runs two (sequence, KV head, chunk) pipelines side by side -- two consecutive chunks of one sequence,
-//     which share the Q tiles -- each with its own producer thread (TMA, 128-byte swizzle, two K and two V stages
+//     which share the Q tile -- each with its own producer thread (TMA, 128-byte swizzle, two K and two V stages
 //     of 64 keys), MMA issuer thread, and four softmax warps;
-//   * S = Q_hi K^T + Q_lo K^T by tcgen05.mma 64 x 64 (k = 128) into one of two tensor-memory buffers.  An M = 64
-//     accumulator puts row r in lane 32 (r / 16) + r % 16, so each of the four softmax warps of a pipeline owns
-//     16 rows (lanes 0..15 of its lane quarter) and all four schedulers take part;
-//   * one thread per query row: exp2 against a reference maximum that only moves when exceeded by 2^8 (O rescaled
-//     in tensor memory then), P split into bf16 hi + lo tiles written in the operand layout;
-//   * O += P_hi V + P_lo V by tcgen05.mma 64 x 128 (k = 64) with the V tile as stored (MN-major B operand).
+//   * the hi and lo parts of an operand are stacked along M: rows 32 q + i of the 128-row Q tile hold Q_hi of query
+//     row 16 q + i, rows 32 q + 16 + i hold Q_lo of the same row (i < 16, q = warp quarter), so ONE tcgen05.mma
+//     128 x 64 (k = 128) leaves q_hi.k in tensor-memory lane 32 q + i and q_lo.k in lane 32 q + 16 + i: the two
+//     lanes belong to the same warp, and the score is their sum, exchanged by shuffles.  (The cost of an MMA here
+//     hardly depends on M, so stacking halves the tensor time against one MMA per part.)
+//   * two threads per query row: lane i of a warp takes key columns 0..31, lane 16 + i columns 32..63 (after the
+//     exchange each holds the full score of its columns); exp2 against a reference maximum shared by the pair that
+//     only moves when exceeded by 2^8 (O rescaled in tensor memory then); P is written as bf16 hi and lo rows of
+//     one 128-row operand tile laid out like Q;
+//   * O_hi / O_lo += P V by ONE tcgen05.mma 128 x 128 (k = 64) with the V tile as stored (MN-major B operand); the
+//     two accumulator rows of a query row are added once, when the chunk's partial is written.
 // The step's own K new rows are one more chunk: a 16-row side tile (rows 0..7 hi parts, 8..15 lo parts), so score
 // columns c and c + 8 add up to q.k and the weight of column c is repeated on column c + 8 for v_lo.
 // Every mbarrier wait is bounded; d_h = 128.
@@ -25,19 +30,19 @@ namespace dart {
 using namespace umma;
 
 constexpr int kAuThreads = 384;                 // warps 0/2: producers, 1/3: MMA issuers, 4-7 and 8-11: softmax
-constexpr int kAuQ = 64 * 128 * 2;              // 64 query rows x 128: two 64-column halves of 8 KB
-constexpr int kAuP = 64 * 64 * 2;               // 64 query rows x 64 keys
+constexpr int kAuQ = 128 * 128 * 2;             // 128 operand rows (hi and lo of 64 query rows) x 128: two 64-column halves
+constexpr int kAuP = 128 * 64 * 2;              // 128 operand rows (hi and lo of 64 query rows) x 64 keys
 constexpr int kAuKV = 64 * 128 * 2;             // 64 keys x 128: two 64-column halves
-// Q hi, Q lo | P [pipeline][buffer][hi, lo] | K [pipeline][stage] | V [pipeline][stage].
-constexpr size_t kAuSmem = (size_t)2 * kAuQ + 8 * kAuP + 8 * kAuKV + 1024;
+// Q | P [pipeline][buffer] | K [pipeline][stage] | V [pipeline][stage]
+constexpr size_t kAuSmem = (size_t)kAuQ + 4 * kAuP + 8 * kAuKV + 1024;
 
 __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_constant__ AttnUmmaArgs a) {
   const AttnParams& p = a.a.p;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = sm;                                    // hi, lo
-  uint8_t* sP = sm + 2 * kAuQ;
-  uint8_t* sK = sP + 8 * kAuP;
+  uint8_t* sQ = sm;
+  uint8_t* sP = sm + kAuQ;
+  uint8_t* sK = sP + 4 * kAuP;
   uint8_t* sV = sK + 4 * kAuKV;
   __shared__ uint64_t q_full, k_full[2][2], k_empty[2][2], v_full[2][2], v_empty[2][2];
   __shared__ uint64_t s_full[2][2], s_empty[2][2], p_full[2][2], pv_done[2][2];
@@ -101,11 +106,13 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
     pdl_wait();
     if (pl == 0) {
       const int q_row = (b * p.Hq + hk * G) * p.K;
-      mbar_expect_tx(&q_full, 2 * kAuQ);
-      tma_load_2d(sQ, &a.mapQhi, &q_full, 0, q_row);
-      tma_load_2d(sQ + kAuQ / 2, &a.mapQhi, &q_full, 64, q_row);
-      tma_load_2d(sQ + kAuQ, &a.mapQlo, &q_full, 0, q_row);
-      tma_load_2d(sQ + kAuQ + kAuQ / 2, &a.mapQlo, &q_full, 64, q_row);
+      mbar_expect_tx(&q_full, kAuQ);
+      for (int q4 = 0; q4 < 4; ++q4)        // 16 query rows per warp quarter: hi rows, then lo rows, per 64-column half
+        for (int ch = 0; ch < 2; ++ch) {
+          uint8_t* d = sQ + ch * (kAuQ / 2) + q4 * 32 * 128;
+          tma_load_2d(d, &a.mapQhi, &q_full, ch * 64, q_row + 16 * q4);
+          tma_load_2d(d + 16 * 128, &a.mapQlo, &q_full, ch * 64, q_row + 16 * q4);
+        }
     }
     for (; t < n_t; ++t) {
       const int s = t & 1;
@@ -117,11 +124,10 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
     }
   } else if ((warp == 1 || warp == 3) && lane == 0 && pl_on) {
     // ---- MMA issuer of pipeline pl
-    constexpr uint32_t idesc_s = idesc_bf16(64, 64), idesc_o = idesc_bf16(64, 128) | kIdescBMnMajor;
-    const uint64_t dqh0 = desc_sw128(smem_u32(sQ)), dqh1 = desc_sw128(smem_u32(sQ + kAuQ / 2));
-    const uint64_t dql0 = desc_sw128(smem_u32(sQ + kAuQ)), dql1 = desc_sw128(smem_u32(sQ + kAuQ + kAuQ / 2));
+    constexpr uint32_t idesc_s = idesc_bf16(128, 64), idesc_o = idesc_bf16(128, 128) | kIdescBMnMajor;
+    const uint64_t dq0 = desc_sw128(smem_u32(sQ)), dq1 = desc_sw128(smem_u32(sQ + kAuQ / 2));
     bool ok = ta_wait(&q_full, 0, &abort_flag);
-    auto issue_s = [&](int t) -> bool {      // S[t & 1] = (Q_hi + Q_lo) K_t^T
+    auto issue_s = [&](int t) -> bool {      // S[t & 1] = [Q_hi ; Q_lo] K_t^T
       const int s = t & 1;
       if (!ta_wait(&k_full[pl][s], (t >> 1) & 1, &abort_flag)) return false;
       if (t >= 2 && !ta_wait(&s_empty[pl][s], ((t >> 1) - 1) & 1, &abort_flag)) return false;
@@ -129,13 +135,9 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       const uint64_t dk0 = desc_sw128(smem_u32(sK + (pl * 2 + s) * kAuKV)), dk1 = desc_sw128(smem_u32(sK + (pl * 2 + s) * kAuKV + kAuKV / 2));
       const uint32_t acc = tmem + pl * 256 + s * 64;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(acc, dqh0 + 2 * k, dk0 + 2 * k, idesc_s, k > 0 ? 1u : 0u);
+      for (int k = 0; k < 4; ++k) mma_f16(acc, dq0 + 2 * k, dk0 + 2 * k, idesc_s, k > 0 ? 1u : 0u);
 #pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(acc, dqh1 + 2 * k, dk1 + 2 * k, idesc_s, 1u);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(acc, dql0 + 2 * k, dk0 + 2 * k, idesc_s, 1u);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(acc, dql1 + 2 * k, dk1 + 2 * k, idesc_s, 1u);
+      for (int k = 0; k < 4; ++k) mma_f16(acc, dq1 + 2 * k, dk1 + 2 * k, idesc_s, 1u);
       mma_commit(&s_full[pl][s]);
       mma_commit(&k_empty[pl][s]);
       return true;
@@ -148,50 +150,58 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       if (!ta_wait(&p_full[pl][s], (t >> 1) & 1, &abort_flag)) break;
       tc_fence_after();
       const uint64_t dv = desc_sw128_mn(smem_u32(sV + (pl * 2 + s) * kAuKV), kAuKV / 2);
-      const uint64_t dph = desc_sw128(smem_u32(sP + ((pl * 2 + s) * 2) * kAuP)), dpl = desc_sw128(smem_u32(sP + ((pl * 2 + s) * 2 + 1) * kAuP));
+      const uint64_t dp = desc_sw128(smem_u32(sP + (pl * 2 + s) * kAuP));
 #pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + pl * 256 + 128, dph + 2 * k, dv + 128 * k, idesc_o, (t > 0 || k > 0) ? 1u : 0u);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + pl * 256 + 128, dpl + 2 * k, dv + 128 * k, idesc_o, 1u);
+      for (int k = 0; k < 4; ++k) mma_f16(tmem + pl * 256 + 128, dp + 2 * k, dv + 128 * k, idesc_o, (t > 0 || k > 0) ? 1u : 0u);
       mma_commit(&pv_done[pl][s]);
       mma_commit(&v_empty[pl][s]);
     }
   } else if (warp >= 4 && pl_on) {
-    // ---- softmax of pipeline pl: lanes 0..15 of warp quarter wq own query rows 16 wq .. 16 wq + 15 (the M = 64
-    // accumulator layout); lanes 16..31 only take part in the warp-wide tensor-memory instructions
-    const int wq = warp & 3;
-    const bool act = lane < 16;
-    const int row = act ? wq * 16 + lane : 64;
+    // ---- softmax of pipeline pl.  Warp quarter wq owns query rows 16 wq .. 16 wq + 15; lane i < 16 sits on the
+    // tensor-memory lane of the row's hi part and takes key columns 0..31, lane 16 + i on the lo part's lane and
+    // takes columns 32..63.
+    const int wq = warp & 3, hh = lane >> 4;
+    const int row = wq * 16 + (lane & 15);          // query row
     const uint32_t tb = tmem + ((uint32_t)(wq * 32) << 16) + pl * 256;
     const int r = row % p.K;             // position of the row inside its sequence's K-block
     const float c = rsqrtf(128.f) * 1.4426950408889634f;   // 1/sqrt(d_h) * log2(e)
-    float m_ref = -INFINITY, l = 0.f;
+    float m_ref = -INFINITY, l = 0.f;    // l: this thread's half of the row sum
     bool ok = true;
     for (int t = 0; t < n_t; ++t) {
       const int s = t & 1;
       if (!ta_wait(&s_full[pl][s], (t >> 1) & 1, &abort_flag)) { ok = false; break; }
       tc_fence_after();
-      float sv[64];
-      tmem_ld64(tb + s * 64, sv);
+      float raw[64];
+      tmem_ld64(tb + s * 64, raw);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_empty[pl][s]);
+      // score of this thread's 32 columns = its own part + the partner lane's part of the same columns
+      float sv[32];
+#pragma unroll
+      for (int q = 0; q < 32; ++q) {
+        const float send = hh ? raw[q] : raw[32 + q];
+        const float got = __shfl_xor_sync(0xffffffffu, send, 16);
+        sv[q] = (hh ? raw[32 + q] : raw[q]) + got;
+      }
+      const int c0 = 32 * hh;            // first key column of this thread
       if (is_new) {      // columns c and c + 8 hold q.k_hi and q.k_lo of new row c; row r reads new rows c <= r
 #pragma unroll
-        for (int q = 0; q < 8; ++q) sv[q] = (q < p.K && q <= r) ? sv[q] + sv[q + 8] : -INFINITY;
+        for (int q = 0; q < 8; ++q) sv[q] = (hh == 0 && q < p.K && q <= r) ? sv[q] + sv[q + 8] : -INFINITY;
 #pragma unroll
-        for (int q = 8; q < 64; ++q) sv[q] = -INFINITY;
+        for (int q = 8; q < 32; ++q) sv[q] = -INFINITY;
       } else if (k_begin + t * 64 + 64 > k_end) {   // the chunk's last tile: keys past its end are hidden
-        const int hi = k_end - (k_begin + t * 64) - 1;
+        const int hi = k_end - (k_begin + t * 64) - 1 - c0;
 #pragma unroll
-        for (int q = 0; q < 64; ++q) sv[q] = q <= hi ? sv[q] : -INFINITY;
+        for (int q = 0; q < 32; ++q) sv[q] = q <= hi ? sv[q] : -INFINITY;
       }
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int q = 0; q < 64; ++q) mx[q & 3] = fmaxf(mx[q & 3], sv[q]);
-      const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;
+      for (int q = 0; q < 32; ++q) mx[q & 3] = fmaxf(mx[q & 3], sv[q]);
+      float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 16)) * c;   // the row's maximum over both halves
       float alpha = 1.f;
-      if (mt > m_ref + 8.f) {               // also the first visible tile (m_ref = -inf)
+      if (mt > m_ref + 8.f) {               // also the first visible tile (m_ref = -inf); the same in both lanes of a row
         alpha = m_ref == -INFINITY ? 1.f : ex2(m_ref - mt);
         m_ref = mt;
         l *= alpha;
@@ -199,7 +209,7 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int q = 0; q < 64; ++q) {
+      for (int q = 0; q < 32; ++q) {
         sv[q] = ex2(fmaf(sv[q], c, -m_use));   // ex2(-inf) = 0 for the hidden columns
         ls[q & 3] += sv[q];
       }
@@ -213,7 +223,7 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       const int valid = is_new ? 16 : min(64, k_end - (k_begin + t * 64));
       if (valid < 64) {
         if (!ta_wait(&v_full[pl][s], (t >> 1) & 1, &abort_flag)) { ok = false; break; }
-        if (act && row >= valid) {
+        if (hh == 0 && row >= valid) {      // 64 threads, one V row each
           uint8_t* vrow = sV + (pl * 2 + s) * kAuKV + row * 128;
 #pragma unroll
           for (int ch = 0; ch < 8; ++ch) {
@@ -224,7 +234,7 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       }
       // this P buffer was last read by the MMAs of tile t - 2
       if (t >= 2 && !ta_wait(&pv_done[pl][s], ((t >> 1) - 1) & 1, &abort_flag)) { ok = false; break; }
-      if (t > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rescale this warp's O rows in tensor memory
+      if (t > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rescale this warp's O rows (hi and lo parts) in tensor memory
         if (!ta_wait(&pv_done[pl][s ^ 1], ((t - 1) >> 1) & 1, &abort_flag)) { ok = false; break; }   // O holds tiles 0..t-1
         tc_fence_after();
 #pragma unroll 1
@@ -238,23 +248,24 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
         }
         tmem_st_wait();
       }
-      // P as hi + lo A operands: [64 rows][64 keys] each, rows of 128 bytes, 16-byte chunk ch of row r stored at
-      // chunk ch ^ (r & 7) (the 128-byte swizzle)
-      uint8_t* ph = sP + ((pl * 2 + s) * 2) * kAuP + (row & 63) * 128;
-      uint8_t* plo = ph + kAuP;
+      // P as one A operand of 128 rows x 64 keys laid out like Q: row 32 wq + i = hi parts of query row 16 wq + i,
+      // row 32 wq + 16 + i = lo parts; rows of 128 bytes, 16-byte chunk ch of operand row x stored at chunk
+      // ch ^ (x & 7) (the 128-byte swizzle).  This thread writes the 4 chunks of its 32 columns into both rows.
+      const int xrow = wq * 32 + (lane & 15);
+      uint8_t* ph = sP + (pl * 2 + s) * kAuP + xrow * 128;
+      uint8_t* plo = ph + 16 * 128;
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        if (!act) break;
+      for (int cq = 0; cq < 4; ++cq) {
         uint32_t wh[4], wl[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const float x0 = sv[ch * 8 + 2 * q], x1 = sv[ch * 8 + 2 * q + 1];
+          const float x0 = sv[cq * 8 + 2 * q], x1 = sv[cq * 8 + 2 * q + 1];
           const __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
           const __nv_bfloat162 l2 = __floats2bfloat162_rn(x0 - __low2float(h2), x1 - __high2float(h2));
           wh[q] = *reinterpret_cast<const uint32_t*>(&h2);
           wl[q] = *reinterpret_cast<const uint32_t*>(&l2);
         }
-        const int off = (ch ^ (row & 7)) << 4;
+        const int off = ((4 * hh + cq) ^ (xrow & 7)) << 4;     // (xrow + 16) & 7 == xrow & 7
         *reinterpret_cast<uint4*>(ph + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
         *reinterpret_cast<uint4*>(plo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
       }
@@ -265,21 +276,25 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
     }
     if (ok && ta_wait(&pv_done[pl][(n_t - 1) & 1], ((n_t - 1) >> 1) & 1, &abort_flag)) {
       tc_fence_after();
-      // the chunk's partial: (reference maximum, sum, un-normalised output), merged by attn_combine_kernel
+      // the chunk's partial: (reference maximum, sum, un-normalised output), merged by attn_combine_kernel.  The
+      // output row is the sum of the hi part's and the lo part's accumulator rows (this lane's and its partner's).
+      const float lt = l + __shfl_xor_sync(0xffffffffu, l, 16);
       const size_t slot = ((size_t)(a.a.chunk_base[b] + ci) * p.Hkv + hk) * 64 + row;
 #pragma unroll 1
       for (int cb = 0; cb < 128; cb += 16) {
         uint32_t rr[16];
         tmem_ld16(tb + 128 + cb, rr);
         tmem_ld_wait();
-        if (act && row < R) {
-          float4* dst = reinterpret_cast<float4*>(p.o_part + slot * 128 + cb);
+        float o[16];
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            dst[q] = make_float4(__uint_as_float(rr[4 * q]), __uint_as_float(rr[4 * q + 1]), __uint_as_float(rr[4 * q + 2]), __uint_as_float(rr[4 * q + 3]));
+        for (int q = 0; q < 16; ++q) o[q] = __uint_as_float(rr[q]) + __shfl_xor_sync(0xffffffffu, __uint_as_float(rr[q]), 16);
+        if (row < R) {                       // each lane of the pair stores half of the 16 columns
+          float4* dst = reinterpret_cast<float4*>(p.o_part + slot * 128 + cb + 8 * hh);
+          dst[0] = hh ? make_float4(o[8], o[9], o[10], o[11]) : make_float4(o[0], o[1], o[2], o[3]);
+          dst[1] = hh ? make_float4(o[12], o[13], o[14], o[15]) : make_float4(o[4], o[5], o[6], o[7]);
         }
       }
-      if (act && row < R) *reinterpret_cast<float2*>(p.ml_part + slot * 2) = make_float2(m_ref, l);
+      if (hh == 0 && row < R) *reinterpret_cast<float2*>(p.ml_part + slot * 2) = make_float2(m_ref, lt);
     }
   }
   tc_fence_before();

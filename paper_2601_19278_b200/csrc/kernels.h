@@ -226,8 +226,8 @@ struct AttnArgs {
   AttnParams p;
   int chunk_base[33];  // prefix sums of chunks per sequence (cache chunks + 1 new-rows chunk)
 };
-// The tensor-core split kernel (attn_umma.cu, d_h = 128): tensor maps over q_hi / q_lo [B*Hq*K][128], the caches
-// [B*Hkv*P_cap][128] and the new rows' side tiles [B*Hkv*16][128]; boxes of 64 rows x 64 columns.
+// The tensor-core split kernel (attn_umma.cu, d_h = 128): tensor maps over q_hi / q_lo [B*Hq*K][128] (boxes of 16
+// rows x 64 columns), the caches [B*Hkv*P_cap][128] and the new rows' side tiles [B*Hkv*16][128] (64 x 64).
 struct AttnUmmaMaps { CUtensorMap mapQhi, mapQlo, mapK, mapV, mapKn, mapVn; };
 struct AttnUmmaArgs {
   AttnArgs a;
