@@ -281,7 +281,7 @@ def run_ours(args):
             "stages_us": stages_us,
             "step_bytes": bytes_step, "step_gbs": step_gbs,
             "step_frac_of_hbm_peak": step_gbs / hbm_peak, "step_frac_of_8tbs": step_gbs / 8000.0,
-            "roofline": {"bound": "hbm", "kernel": "lm_head_umma_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+            "roofline": {"bound": "hbm", "kernel": "lm_head_dense_kernel" if w.batch * w.K > 32 else "lm_head_umma_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                          "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
                          "traffic": args.lm_traffic if args.lm_traffic is not None else lm_bytes * LM_READ_RATIO + LM_WRITE_BYTES,
                          "traffic_source": "ncu capture of a vocab-32768 launch (profiles/lm_head_umma_kernel_C3_vocab32768.txt), reads "
