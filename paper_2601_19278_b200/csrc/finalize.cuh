@@ -142,9 +142,17 @@ __device__ __forceinline__ void tile_rows_sum(int ft, float (&v)[NV], float* sh)
 // dry = true executes the same instructions without a single store to global memory (a measurement aid: a
 // second call on the same group takes 3 us instead of 5.5, because the pieces, written by SMs all over the
 // chip, are then close by - not because of the code: a dry pass ahead of time does not help).
-// One instantiation per epilogue mode, so each mode only carries its own instructions.
+// One instantiation per epilogue mode, so each mode only carries its own instructions.  A kernel that defines
+// DART_FINALIZE_INLINE before this header gets it inlined: its many reads of the arguments are then operands from
+// the constant bank; out of line they are dependent loads through a pointer (about 2 us more on the tail of every
+// projection), which the register-tight mma.sync kernels accept to keep their streaming loop free of spills.
+#ifdef DART_FINALIZE_INLINE
+#define DART_FINALIZE_ATTR __forceinline__
+#else
+#define DART_FINALIZE_ATTR __noinline__
+#endif
 template <int MODE, int NTHR, int BAR>
-static __device__ __noinline__ void finalize_group_t(int ft, const GemmArgs& p, int group, int MP, float* sh, float* s_rstd,
+static __device__ DART_FINALIZE_ATTR void finalize_group_t(int ft, const GemmArgs& p, int group, int MP, float* sh, float* s_rstd,
                                                      const int* s_pos, const GroupMeta* gm, FinSmem* fs, bool dry) {
   constexpr int NPAR = NTHR / 128;     // token classes: thread -> (row = ft & 127, class = ft >> 7)
   constexpr int NV = 8 / NPAR;         // tokens of an 8-token chunk per thread in the row-major modes

@@ -19,6 +19,7 @@
 #include "common.cuh"
 #include "kernels.h"
 #include "umma.cuh"
+#define DART_FINALIZE_INLINE
 #include "finalize.cuh"
 
 namespace dart {
