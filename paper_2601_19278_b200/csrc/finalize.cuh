@@ -334,4 +334,36 @@ static __device__ __noinline__ void embed_rows(const GemmArgs& p, float* sh, int
   }
 }
 
+// The same on a team of NTHR threads that synchronises on named barrier BAR (warps that idle while the projection
+// streams), with the arguments read from the kernel's constant bank.  red: NTHR / 32 floats of shared memory.
+template <int NTHR, int BAR>
+static __device__ __forceinline__ void embed_row_team(const EpiArgs& e, int ft, float* red, int ftok) {
+  const int orow = fresh_to_step_row(e, ftok);
+  const int id = min(max(e.tokens[ftok], 0), e.vocab - 1);
+  const int h = e.h;
+  const bf16* row = e.embed + (size_t)id * h;
+  float ss = 0.f;
+  for (int n = ft; n < h; n += NTHR) {
+    const float v = __bfloat162float(row[n]);
+    ss += v * v;
+  }
+  ss = warp_sum(ss);
+  if ((ft & 31) == 0) red[ft >> 5] = ss;
+  team_sync<NTHR, BAR>();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < NTHR / 32; ++w) tot += red[w];
+  const float rs = 1.f / sqrtf(tot / (float)h + e.eps);
+  bf16* out_hi = e.out_hi + (size_t)orow * e.ld_out + h;
+  bf16* out_lo = e.out_lo + (size_t)orow * e.ld_out + h;
+  const bf16* gam = e.gamma_e;
+  for (int n = ft; n < h; n += NTHR) {
+    bf16 hi, lo;
+    split_bf16(__bfloat162float(row[n]) * rs * __bfloat162float(gam[n]), hi, lo);
+    out_hi[n] = hi;
+    out_lo[n] = lo;
+  }
+  team_sync<NTHR, BAR>();   // red is free for the next row
+}
+
 }  // namespace dart

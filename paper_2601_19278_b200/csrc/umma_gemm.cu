@@ -72,6 +72,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
   __shared__ int abort_flag;
   __shared__ int s_cnt[4];
   __shared__ float sh[32];
+  __shared__ float s_emb[8];
   __shared__ float s_rstd[128];
   __shared__ int s_done[64];
   __shared__ int s_pos[128];
@@ -229,6 +230,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       ++visit;
       u = ue;
     }
+  } else if (warp >= 8 && p.epi.mode == EPI_FC) {
+    // ---- the warps with no part in the streaming: the fresh rows' shifted token embedding (its inputs are the
+    // step's; the wait orders its stores after every earlier reader of z)
+    pdl_wait();
+    for (int ftok = c; ftok < p.s.M; ftok += G) embed_row_team<256, 1>(p.epi, threadIdx.x - 256, s_emb, ftok);
   }
   pdl_wait();
   pdl_trigger();
@@ -244,8 +250,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
     __syncthreads();
     return;
   }
-  if (p.epi.mode == EPI_FC)
-    for (int ftok = c; ftok < p.s.M; ftok += G) embed_rows(p, sh, ftok);
   // fused finalize of the groups this CTA completed (the ring is idle now)
   const int n_done = s_done[0];
   FinSmem* fs = reinterpret_cast<FinSmem*>(ring);
