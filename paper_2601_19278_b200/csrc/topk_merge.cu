@@ -4,7 +4,7 @@
 // Input per CTA c and token row: (max, sum-exp) of its vocab slice and its best `topk` entries
 // (selection key, plain logit y, token id), sorted by (key desc, id asc).  One block per token row:
 //   1. log-sum-exp over the slices (fixed-order reductions, deterministic);
-//   2. all G lists are copied to shared memory with coalesced loads;
+//   2. all G lists (keys, ids, plain logits) are copied to shared memory with coalesced loads, all requested at once;
 //   3. a threshold T taken from the list *heads*: the heads are warp-sorted and T = the m-th best of
 //      the runs' p-th entries with m * (p + 1) >= topk, so at least topk heads are not after T and the
 //      global top-k lies among the entries that are not after T; each sorted list contributes a prefix;
@@ -19,13 +19,16 @@
 namespace dart {
 
 constexpr int kMergeThreads = 512;
+constexpr int kMergeYsMaxGrid = 256;   // up to this many lists their plain logits fit in shared memory beside the rest
 
 __global__ void __launch_bounds__(kMergeThreads) topk_merge_kernel(const LmParams p) {
   extern __shared__ __align__(16) unsigned char msm[];
   const int G = p.grid, MP = padded_tokens(p.M), tk = blockIdx.x, topk = p.topk;
   float* keys = reinterpret_cast<float*>(msm);                 // [G*32]
   int* ids = reinterpret_cast<int*>(keys + G * 32);            // [G*32]
-  Key* skey = reinterpret_cast<Key*>(ids + G * 32);            // [G*32] survivors' keys
+  const bool has_ys = G <= kMergeYsMaxGrid;
+  float* ys = reinterpret_cast<float*>(ids + G * 32);          // [G*32] plain logits (if they fit)
+  Key* skey = reinterpret_cast<Key*>(ys + (has_ys ? G * 32 : 0));   // [G*32] survivors' keys
   int* ssrc = reinterpret_cast<int*>(skey + G * 32);           // [G*32] survivors' positions c*32+e
   Key* xk = reinterpret_cast<Key*>(ssrc + G * 32);             // [16 warps][64] merge-tree scratch
   Key* hr = xk + 16 * 64;                                      // [32 runs][32] sorted heads
@@ -36,28 +39,50 @@ __global__ void __launch_bounds__(kMergeThreads) topk_merge_kernel(const LmParam
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_wait();
 
-  {  // coalesced copy of the G lists of this token row: 32 keys and 32 ids per list
+  // Every global load of the kernel is requested before any is used (the lists' keys, ids and plain logits with
+  // coalesced 16-byte loads, the slices' statistics), so the kernel pays one round trip to memory, not one per loop
+  // iteration or per phase.
+  float m = -INFINITY, s = 0.f;
+  {
     const float4* ksrc = reinterpret_cast<const float4*>(p.part_key);
+    const float4* ysrc = reinterpret_cast<const float4*>(p.part_y);
     const int4* isrc = reinterpret_cast<const int4*>(p.part_id);
-    for (int i = tid; i < G * 8; i += kMergeThreads) {
-      const int c = i >> 3, q = i & 7;
-      const size_t o = ((size_t)c * MP + tk) * 8 + q;
-      reinterpret_cast<float4*>(keys)[i] = ksrc[o];
-      reinterpret_cast<int4*>(ids)[i] = isrc[o];
+    constexpr int kBatch = 3;
+    for (int base = 0; base < G * 8; base += kBatch * kMergeThreads) {
+      float4 kr[kBatch], yr[kBatch];
+      int4 ir[kBatch];
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q) {
+        const int i = base + q * kMergeThreads + tid;
+        if (i < G * 8) {
+          const size_t o = ((size_t)(i >> 3) * MP + tk) * 8 + (i & 7);
+          kr[q] = ksrc[o];
+          if (has_ys) yr[q] = ysrc[o];
+          ir[q] = isrc[o];
+        }
+      }
+      float mc = -INFINITY, sc = 0.f;
+      // ---- log-sum-exp over the slices: per-thread online (max, sum), combined in a fixed order below
+      const int c0 = base / 8 + tid;   // the slices whose lists this pass copies: base/8 .. base/8 + kBatch*64 - 1
+      const bool has = tid < kBatch * (kMergeThreads / 8) && c0 < G;
+      if (has) { mc = p.part_stats[((size_t)c0 * MP + tk) * 2]; sc = p.part_stats[((size_t)c0 * MP + tk) * 2 + 1]; }
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q) {
+        const int i = base + q * kMergeThreads + tid;
+        if (i < G * 8) {
+          reinterpret_cast<float4*>(keys)[i] = kr[q];
+          if (has_ys) reinterpret_cast<float4*>(ys)[i] = yr[q];
+          reinterpret_cast<int4*>(ids)[i] = ir[q];
+        }
+      }
+      if (has && mc != -INFINITY) {
+        const float mn = fmaxf(m, mc);
+        s = s * expf(m - mn) + sc * expf(mc - mn);
+        m = mn;
+      }
     }
   }
   if (tid == 0) s_nsurv = 0;
-
-  // ---- log-sum-exp over the slices: per-thread online (max, sum), combined in a fixed order
-  float m = -INFINITY, s = 0.f;
-  for (int c = tid; c < G; c += kMergeThreads) {
-    const float mc = p.part_stats[((size_t)c * MP + tk) * 2], sc = p.part_stats[((size_t)c * MP + tk) * 2 + 1];
-    if (mc != -INFINITY) {
-      const float mn = fmaxf(m, mc);
-      s = s * expf(m - mn) + sc * expf(mc - mn);
-      m = mn;
-    }
-  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float mo = __shfl_xor_sync(0xffffffffu, m, o), so = __shfl_xor_sync(0xffffffffu, s, o);
@@ -124,8 +149,7 @@ __global__ void __launch_bounds__(kMergeThreads) topk_merge_kernel(const LmParam
       int src = -1;
       for (int o = 0; o < ns; ++o)
         if (skey[o] == x0) { src = ssrc[o]; break; }
-      const int c = src >> 5, e = src & 31;
-      const float y = p.part_y[((size_t)c * MP + tk) * 32 + e];
+      const float y = has_ys ? ys[src] : p.part_y[((size_t)(src >> 5) * MP + tk) * 32 + (src & 31)];
       p.out_ids[(size_t)tk * topk + lane] = ids[src];
       p.out_slogit[(size_t)tk * topk + lane] = logf(expf(y - lse) + p.eps_logit);
     }
@@ -136,8 +160,8 @@ __global__ void __launch_bounds__(kMergeThreads) topk_merge_kernel(const LmParam
       int rank = 0;
       for (int o = 0; o < ns; ++o) rank += skey[o] > me;
       if (rank < topk) {
-        const int src = ssrc[sidx], c = src >> 5, e = src & 31;
-        const float y = p.part_y[((size_t)c * MP + tk) * 32 + e];
+        const int src = ssrc[sidx];
+        const float y = has_ys ? ys[src] : p.part_y[((size_t)(src >> 5) * MP + tk) * 32 + (src & 31)];
         p.out_ids[(size_t)tk * topk + rank] = ids[src];
         p.out_slogit[(size_t)tk * topk + rank] = logf(expf(y - lse) + p.eps_logit);
       }
@@ -149,10 +173,11 @@ __global__ void __launch_bounds__(kMergeThreads) topk_merge_kernel(const LmParam
   }
 }
 
-static size_t merge_smem(int G) { return (size_t)G * 32 * (4 + 4 + 8 + 4) + (16 * 64 + 32 * 32) * 8 + 64; }
+static size_t merge_smem(int G) { return (size_t)G * 32 * (4 + 4 + (G <= kMergeYsMaxGrid ? 4 : 0) + 8 + 4) + (16 * 64 + 32 * 32) * 8 + 64; }
 
 cudaError_t topk_merge_setup(int max_grid) {
-  const size_t smem = merge_smem(max_grid);
+  size_t smem = merge_smem(max_grid);
+  if (max_grid > kMergeYsMaxGrid && merge_smem(kMergeYsMaxGrid) > smem) smem = merge_smem(kMergeYsMaxGrid);
   if (smem > 48 * 1024)
     return cudaFuncSetAttribute(topk_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   return cudaSuccess;
