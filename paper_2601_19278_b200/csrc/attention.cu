@@ -98,6 +98,7 @@ __global__ void __launch_bounds__(128) attn_splitkv_kernel(const __grid_constant
   if (!is_new) load_tile(0, 0);
   cp_async_commit();
   pdl_wait();
+  pdl_trigger();   // a short kernel: the next one may be scheduled and run its set-up now
   // Q tiles, hi and lo (rows >= R zero-filled)
   for (int i = tid; i < 64 * CH; i += 128) {
     const int row = i / CH, ch = i % CH;
@@ -258,6 +259,7 @@ __global__ void attn_combine_kernel(const AttnArgs a) {
   const int n_chunks = a.chunk_base[b + 1] - a.chunk_base[b];
   const size_t slot0 = ((size_t)a.chunk_base[b] * p.Hkv + hk) * 64 + rr, slot_step = (size_t)p.Hkv * 64;
   pdl_wait();
+  pdl_trigger();   // a short kernel: the next one may be scheduled and run its set-up now
   float l_c = 0.f;
   if (tid < n_chunks) {
     const float2 ml = *reinterpret_cast<const float2*>(p.ml_part + (slot0 + (size_t)tid * slot_step) * 2);

@@ -116,8 +116,10 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1
 // kernel's blocks are scheduled onto SMs as they drain and start their own weight stream early.
 // pdl_wait() returns once the predecessor grid has completed and its writes are visible; since every
 // kernel waits before it completes, completion is transitive along the stream.
-// (Measured on B200: triggering at kernel *start* instead doubled the step time -- the early-launched
-// successors crowd the running kernel -- so the trigger comes late.)
+// (Measured on B200: triggering at the *start* of the streaming kernels instead doubled the step time -- the
+// early-launched successors crowd the running kernel -- so there the trigger comes late.  The short kernels between
+// them -- attention split and combine, top-k merge, bigram sweep -- trigger right after their wait: their successors'
+// launch and set-up then overlap them, 1.3 us per step.)
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

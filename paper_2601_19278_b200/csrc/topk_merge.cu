@@ -38,6 +38,7 @@ __global__ void __launch_bounds__(kMergeThreads) topk_merge_kernel(const LmParam
   __shared__ int s_nsurv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_wait();
+  pdl_trigger();   // a short kernel: the next one may be scheduled and run its set-up now
 
   // Every global load of the kernel is requested before any is used (the lists' keys, ids and plain logits with
   // coalesced 16-byte loads, the slices' statistics), so the kernel pays one round trip to memory, not one per loop

@@ -176,6 +176,7 @@ __host__ __device__ inline size_t tree_layout(int k, int w, int budget, int L, u
 // gives log(eps).
 __global__ void __launch_bounds__(256) bigram_sweep_kernel(const TreeParams p) {
   pdl_wait();
+  pdl_trigger();   // a short kernel: the next one may be scheduled and run its set-up now
   const int k = p.topk, b = blockIdx.y;
   const int fr = p.first_rows[b], Lb = min(p.n_levels, p.K - fr);   // this sequence's level 0 row and levels
   const int n_bg = k + (p.n_levels - 1) * k * k;                   // layout stride: the launch's maximum
