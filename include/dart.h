@@ -214,10 +214,24 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
 int dart_draft_destroy(dart_handle* h);
 
 /* Device-side status word since the last call of this function: DART_OK or DART_ERR_TIMEOUT.
- * Synchronises `cuda_stream`. */
+ * Synchronises `cuda_stream`.  After DART_ERR_TIMEOUT the outputs of the calls since the previous check are void;
+ * the call has then also cleared the handle's internal work counters (a kernel that gives up on a wait leaves
+ * them half counted), so the handle stays usable: the next dart_draft_step starts from a clean state. */
 int dart_last_device_status(dart_handle* h, void* cuda_stream);
 
-/* The cudaError_t (as int) behind the last DART_ERR_CUDA of this handle (or of init when h is NULL). */
+/*
+ * Self-test of the time-out path (the paper has no counterpart).  Every device-side wait of this library is
+ * bounded: when it runs out the kernel records DART_ERR_TIMEOUT in the handle's status word and returns.  This call
+ * enqueues a one-block kernel that runs exactly that path on purpose -- a wait of `spin_limit` tries (1 .. 100000,
+ * each at most 2 microseconds) on a barrier that nothing signals -- so that a caller (or a test) can see the error
+ * arrive through dart_last_device_status and the handle recover.  leave_ticket != 0 additionally leaves one work
+ * counter of the QKV projection half counted, as a kernel that gave up mid-way would.  Faults nothing, hangs nothing.
+ * Asynchronous on `cuda_stream`.  Errors: INVALID_ARG, CUDA.
+ */
+int dart_selftest_bounded_wait(dart_handle* h, int32_t spin_limit, int32_t leave_ticket, void* cuda_stream);
+
+/* The cudaError_t (as int) behind the last DART_ERR_CUDA of this handle; with h = NULL, of the last call that has no
+ * handle (dart_draft_init, dart_train_attention_fwd, dart_topk_rows_noalloc). */
 int dart_last_cuda_error(const dart_handle* h);
 
 /* Human-readable name of a dart_status. */
@@ -293,8 +307,10 @@ int dart_tree_verify_inputs(dart_handle* h, const dart_verify_in* in, const dart
  * position and stores them.  Sequence b gets new_rows_host[b] rows at positions seq_lens_host[b] ..; their
  * features and next-token ids are packed in sequence order.  The caller then advances its sequence lengths and
  * runs dart_draft_step as usual (whose own fresh rows are appended by that call).  No logits are produced.
- * Asynchronous on `cuda_stream`; rows are processed in runs of up to 128 per pair of kernel launches.
- * Errors: INVALID_ARG, CAPACITY (batch > max_batch or seq_lens_host[b] + new_rows_host[b] > max_prefix).
+ * Asynchronous on `cuda_stream`; the packed rows are processed in passes of up to 4096 rows (three kernel launches
+ * per pass: token embeddings, feature FC, k / v projection), a sequence may straddle two passes.
+ * Errors: INVALID_ARG (also with feat_in = 0: the prefill needs the fusion matrix), CAPACITY (batch > max_batch or
+ * seq_lens_host[b] + new_rows_host[b] > max_prefix).
  */
 typedef struct dart_prefill_in {
   int32_t batch;                  /* B <= max_batch */
@@ -331,9 +347,11 @@ int dart_set_profile_events(dart_handle* h, int stage, void* start_event, void* 
  * loads the library holds until the process exits.  All calls on a GPU share it and it keeps the last
  * call's contents (every call overwrites what it reads, nothing needs clearing): calls that overlap on
  * the same GPU -- different streams or host threads -- race; serialise them.
- * The first call on each device (made with that device current) looks up the array's device address;
+ * The first call on each device (made with that device current) looks up the array's device address
+ * (two host threads making it together both cache the same address, which is harmless);
  * make that first call before any CUDA stream capture.  Calls cudaMalloc/cudaFree never.
- * Asynchronous on `cuda_stream`.  Errors: INVALID_ARG, CAPACITY, CUDA.
+ * Asynchronous on `cuda_stream`.  Errors: INVALID_ARG, CAPACITY, UNSUPPORTED_ARCH (not sm_100),
+ * CUDA (the cudaError_t is then returned by dart_last_cuda_error(NULL)).
  */
 int dart_topk_rows_noalloc(const float* logits, int32_t rows, int32_t vocab, int32_t topk, float eps_logit,
                            int32_t* out_ids, float* out_slogit, void* cuda_stream);

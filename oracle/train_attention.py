@@ -17,16 +17,19 @@ import numpy as np
 from .mask import training_visible
 
 
-def training_attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, prompt_len: int, draft_len: int, seq_len: int) -> np.ndarray:
+def training_attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, prompt_len: int, draft_len: int, seq_len: int,
+                       query_slots=None) -> np.ndarray:
     """q: [H_q, L, d_h]; k, v: [H_kv, L, d_h] with L = prompt_len * (1 + draft_len), fp64.
-    Returns softmax(q k^T / sqrt(d_h) over the visible slots) v, [H_q, L, d_h]."""
+    Returns softmax(q k^T / sqrt(d_h) over the visible slots) v, [H_q, L, d_h].
+    query_slots: compute only these query slots (the other rows of the result stay zero) -- rows are
+    independent of one another, so a long packed row can be checked on a sample of its slots."""
     Hq, L, dh = q.shape
     Hkv = k.shape[0]
     assert L == prompt_len * (1 + draft_len) and Hq % Hkv == 0
     G = Hq // Hkv
     scale = 1.0 / math.sqrt(dh)
     out = np.zeros((Hq, L, dh), dtype=np.float64)
-    for qi in range(L):
+    for qi in (range(L) if query_slots is None else query_slots):
         vis = np.array([training_visible(qi, ki, prompt_len, draft_len, seq_len) for ki in range(L)], dtype=bool)
         if not vis.any():
             continue

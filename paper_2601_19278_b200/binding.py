@@ -27,7 +27,7 @@ DART_ERR_INTERNAL = -6
 EXPORTS = [
     "dart_draft_init", "dart_draft_step", "dart_build_tree", "dart_draft_destroy", "dart_last_device_status",
     "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_ngram_bytes", "dart_train_attention_fwd", "dart_step_launch_count", "dart_draft_prefill", "dart_tree_verify_inputs",
-    "dart_set_profile_events", "dart_topk_rows_noalloc",
+    "dart_set_profile_events", "dart_topk_rows_noalloc", "dart_selftest_bounded_wait",
 ]
 
 
@@ -142,6 +142,8 @@ def lib() -> C.CDLL:
         L.dart_topk_rows_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
                                              C.c_void_p, C.c_void_p]
         L.dart_topk_rows_noalloc.restype = C.c_int
+        L.dart_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
+        L.dart_selftest_bounded_wait.restype = C.c_int
         _lib = L
     return _lib
 
@@ -257,6 +259,12 @@ class DartDraft:
 
     def device_status(self, stream=None) -> int:
         return lib().dart_last_device_status(self._h, self._stream(stream))
+
+    def selftest_bounded_wait(self, spin_limit: int, leave_ticket: bool = False, stream=None) -> None:
+        """dart_selftest_bounded_wait: enqueue a wait that runs out on purpose (device_status() then reports the time-out)."""
+        rc = lib().dart_selftest_bounded_wait(self._h, spin_limit, 1 if leave_ticket else 0, self._stream(stream))
+        if rc != DART_OK:
+            raise DartError(rc, "dart_selftest_bounded_wait", lib().dart_last_cuda_error(self._h))
 
     def set_profile_events(self, stage: int, start: torch.cuda.Event, stop: torch.cuda.Event) -> None:
         """dart_set_profile_events: bracket one stage of the next call with two torch CUDA events."""

@@ -47,6 +47,10 @@ struct Workspace {
 
 }  // namespace
 
+namespace dart {
+void record_global_cuda_error(cudaError_t e) { g_init_cuda_error = (int)e; }
+}  // namespace dart
+
 struct dart_handle {
   dart_config cfg;
   dart_weights w;
@@ -54,7 +58,6 @@ struct dart_handle {
   int n_sm = 0;
   int last_cuda_error = 0;
   GemmPlan plan_fc, plan_qkv, plan_o, plan_gu, plan_down;
-  bool umma = false;         // projections run on the tcgen05 / TMA kernels (tensor maps could be encoded)
   UmmaMaps maps_fc, maps_qkv, maps_o, maps_gu, maps_down;
   CUtensorMap pmap_fc, pmap_kv[4];   // prefill: W_fc, and the g-/e-half columns of W_k and W_v (boxes of 256 rows)
   CUtensorMap map_lm;        // the LM head's weight matrix (boxes of 128 rows)
@@ -115,65 +118,13 @@ struct PlanHost {
   std::vector<int> expected, meta;
 };
 
-// Cut the flattened (16-row tile, k-round) space of a projection into `grid_target` equal ranges.
+// Cut the flattened (128-row tile, 64-k block) space of a projection into `grid_target` equal ranges, one
+// persistent CTA per SM; a CTA's piece of a tile holds all 128 rows.  The piece table keeps the 16-row
+// granularity of the fused finalize: the j-th 16 rows of a 128-row piece at slot s are "piece" 8 s + j.
 void make_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int grid_target, int pair_offset) {
   GemmPlan& p = ph.plan;
   memset(&p, 0, sizeof(p));
   p.nseg = nseg;
-  int tiles = 0;
-  for (int i = 0; i < 6; ++i) {
-    if (i < nseg) {
-      p.seg[i] = segs[i];
-      p.seg[i].tile0 = tiles;
-      tiles += (segs[i].rows + 127) / 128;
-    } else {
-      p.seg[i] = p.seg[0];
-    }
-  }
-  p.Kd = Kd;
-  p.SK = (Kd + 63) / 64;
-  p.KR = (p.SK + 15) / 16;
-  p.n_tiles = tiles;
-  const int n_mt = tiles * 8;
-  p.U = (long long)n_mt * p.KR;
-  p.grid = (int)((long long)grid_target < p.U ? grid_target : p.U);
-  p.pair_offset = pair_offset;
-  p.n_groups = pair_offset > 0 ? pair_offset : tiles;
-  // CTA c streams units [c*U/grid, (c+1)*U/grid): every 16-row tile it touches gets one piece (one ticket).
-  // The piece table holds at most kMetaStride-1 pieces per tile; a tile of KR k-rounds is cut into at most
-  // ceil(KR / (U / grid)) + 1 of them, so (for very long reductions only) the grid shrinks until that fits.
-  while (p.grid > 1 && (p.KR + (p.U / p.grid) - 1) / (p.U / p.grid) + 1 > kMetaStride - 1) p.grid /= 2;
-  p.slots = 1;
-  p.meta_stride = kMetaStride;
-  ph.expected.assign(p.n_groups, 0);
-  ph.meta.assign((size_t)n_mt * kMetaStride, 0);
-  for (int c = 0; c < p.grid; ++c) {
-    const long long u0 = ((long long)c * p.U) / p.grid, u1 = ((long long)(c + 1) * p.U) / p.grid;
-    if (u0 >= u1) continue;
-    const int t0 = (int)(u0 / p.KR), t1 = (int)((u1 - 1) / p.KR);
-    if (t1 - t0 + 1 > p.slots) p.slots = t1 - t0 + 1;
-  }
-  for (int c = 0; c < p.grid; ++c) {
-    const long long u0 = ((long long)c * p.U) / p.grid, u1 = ((long long)(c + 1) * p.U) / p.grid;
-    if (u0 >= u1) continue;
-    const int t0 = (int)(u0 / p.KR), t1 = (int)((u1 - 1) / p.KR);
-    for (int t = t0; t <= t1; ++t) {
-      const int tile = t >> 3;
-      ph.expected[pair_offset > 0 ? tile % pair_offset : tile] += 1;
-      int& n = ph.meta[(size_t)t * kMetaStride];
-      if (n < kMetaStride - 1) ph.meta[(size_t)t * kMetaStride + 1 + n++] = c * p.slots + (t - t0);
-    }
-  }
-}
-
-// The same cut for the tcgen05 kernel: units are (128-row tile, 64-k block), one persistent CTA per SM, a
-// CTA's piece of a tile holds all 128 rows.  The piece table keeps the 16-row granularity of the fused
-// finalize: the j-th 16 rows of a 128-row piece at slot s are "piece" 8 s + j.
-void make_umma_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int grid_target, int pair_offset) {
-  GemmPlan& p = ph.plan;
-  memset(&p, 0, sizeof(p));
-  p.nseg = nseg;
-  p.umma = 1;
   int tiles = 0;
   for (int i = 0; i < 6; ++i) {
     if (i < nseg) {
@@ -217,7 +168,7 @@ void make_umma_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, in
   }
 }
 
-size_t part_floats(const GemmPlan& p, int MP) { return (size_t)p.grid * p.slots * (p.umma ? 128 : 16) * MP; }
+size_t part_floats(const GemmPlan& p, int MP) { return (size_t)p.grid * p.slots * 128 * MP; }
 
 struct Layout {
   size_t total = 0;
@@ -292,11 +243,8 @@ struct PlanSet {
   size_t part_max = 0;
 };
 
-void build_plans(const dart_config& c, const dart_weights* w, int n_sm, bool umma, PlanSet& ps) {
-  const int grid = umma ? n_sm : 2 * n_sm;
-  auto make_plan_host = [&](PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int g, int pair) {
-    if (umma) make_umma_plan_host(ph, segs, nseg, Kd, g, pair); else ::make_plan_host(ph, segs, nseg, Kd, g, pair);
-  };
+void build_plans(const dart_config& c, const dart_weights* w, int n_sm, PlanSet& ps) {
+  const int grid = n_sm;
   const int h = c.hidden, dq = c.n_q_heads * c.head_dim, dkv = c.n_kv_heads * c.head_dim;
   auto W = [&](const void* p, long long off) { return w ? static_cast<const bf16*>(p) + off : nullptr; };
   GemmSeg s[6];
@@ -329,12 +277,11 @@ void build_plans(const dart_config& c, const dart_weights* w, int n_sm, bool umm
   }
 }
 
-// Piece area that serves either kernel family (the choice is made at init, the size must not depend on it).
+// Floats of the piece area: the largest projection's pieces at the largest token-row padding.
 size_t part_capacity(const dart_config& c, int n_sm) {
-  PlanSet a, b;
-  build_plans(c, nullptr, n_sm, false, a);
-  build_plans(c, nullptr, n_sm, true, b);
-  return a.part_max > b.part_max ? a.part_max : b.part_max;
+  PlanSet a;
+  build_plans(c, nullptr, n_sm, a);
+  return a.part_max;
 }
 
 // Attention chunks: about two CTAs per SM, chunks of 128 .. 512 keys (longer chunks leave a CTA a long serial
@@ -426,16 +373,18 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
     return DART_ERR_CUDA;                                \
   }
 
-#ifndef DART_FORCE_LEGACY
   {
-    CUtensorMap probe;   // the encoder is there and accepts a weight matrix: use the tcgen05 / TMA kernels
-    h->umma = tmap_encode_bf16(&probe, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 128) == cudaSuccess;
+    // every kernel of the path is fed by TMA: a driver whose tensor-map encoder cannot be had is not supported
+    CUtensorMap probe;
+    if (tmap_encode_bf16(&probe, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 128) == cudaErrorNotSupported) {
+      delete h;
+      return DART_ERR_UNSUPPORTED_ARCH;
+    }
   }
-#endif
   PlanSet ps;
-  build_plans(*cfg, weights, n_sm, h->umma, ps);
+  build_plans(*cfg, weights, n_sm, ps);
   PlanHost* plans[5] = {&ps.fc, &ps.qkv, &ps.o, &ps.gu, &ps.down};
-  if (h->umma) {
+  {
     INIT_CHECK(tmap_encode_bf16(&h->map_lm, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 128));
     INIT_CHECK(tmap_encode_bf16(&h->map_lm256, weights->w_lm, cfg->hidden, cfg->vocab, (unsigned long long)cfg->hidden * 2, 64, 256));
     if (cfg->feat_in > 0) {
@@ -481,7 +430,7 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
   }
 
   INIT_CHECK(launch_rope_table(h->ws.rope_tab, cfg->max_prefix + cfg->K, cfg->head_dim, cfg->rope_theta, nullptr));
-  if (h->umma && cfg->head_dim == 128) {   // the attention's maps over the library's own buffers
+  if (cfg->head_dim == 128) {   // the attention's maps over the library's own buffers
     const unsigned long long q_rows = (unsigned long long)cfg->max_batch * cfg->n_q_heads * cfg->K;
     const unsigned long long n_rows16 = (unsigned long long)cfg->max_batch * cfg->n_kv_heads * 16;
     INIT_CHECK(tmap_encode_bf16(&h->attn_maps.mapQhi, h->ws.q_hi, 128, q_rows, 256, 64, 16));
@@ -607,7 +556,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   };
   EpiArgs ep;
   GemmInput gi;
-  if (h->umma && h->maps_M != M) {
+  if (h->maps_M != M) {
     // activation tensor maps: hi and lo buffers as one [M rows][2][width] tensor, box = 64 k x 2 x MP rows; rows past M
     // read as zeros
     struct { UmmaMaps* m; const bf16* hi; const bf16* lo; int width; } xin[4] = {
@@ -621,7 +570,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
     h->maps_M = M;
   }
   auto project = [&](const GemmPlan& plan, const UmmaMaps& maps) -> cudaError_t {
-    return h->umma ? launch_umma_rows(plan, maps, gi, ep, ws.part, ws.status, st) : launch_gemm_rows(plan, gi, ep, ws.part, st);
+    return launch_umma_rows(plan, maps, gi, ep, ws.part, ws.status, st);
   };
 
   // the <mask> rows of z are constant; they are (re)written only when the row pattern changes
@@ -648,7 +597,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
       if ((e = launch_prefused_rows(ep, static_cast<const bf16*>(in->feats), NF, st)) != cudaSuccess) return fail_cuda(h, e);
     } else {
     gi = {static_cast<const bf16*>(in->feats), nullptr, c.feat_in, NF};
-    if (h->umma && (h->maps_feats != in->feats || h->maps_fc_M != NF)) {
+    if ((h->maps_feats != in->feats || h->maps_fc_M != NF)) {
       // plain bf16 input: one box of 2 * MP rows, the rows past the fresh rows (the "lo" half among them) read as zeros
       if ((e = tmap_encode_bf16(&h->maps_fc.Xhi, in->feats, c.feat_in, NF, (unsigned long long)c.feat_in * 2, 64,
                                 2 * padded_tokens(NF))) != cudaSuccess)
@@ -691,7 +640,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
     if (pairs > h->attn_pairs_cap) return DART_ERR_INTERNAL;
   }
   const AttnUmmaMaps* amaps = nullptr;
-  if (h->umma && c.head_dim == 128 && (long long)c.max_batch * c.n_kv_heads * c.max_prefix < (1ll << 31)) {
+  if (c.head_dim == 128 && (long long)c.max_batch * c.n_kv_heads * c.max_prefix < (1ll << 31)) {
     // maps over the caller's caches are re-encoded only when the pointers change
     if (h->attn_k_ptr != in->k_cache || h->attn_v_ptr != in->v_cache) {
       const unsigned long long rows = (unsigned long long)c.max_batch * c.n_kv_heads * c.max_prefix;
@@ -749,7 +698,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   lp.part_stats = ws.lm_stats; lp.part_key = ws.lm_key; lp.part_y = ws.lm_y; lp.part_id = ws.lm_id;
   lp.out_ids = out->topk_ids; lp.out_slogit = out->topk_slogit;
   mark(6, true);
-  if (h->umma) {
+  {
     // one CTA per SM at most: the CTAs of this kernel wait on one another's pieces, so all must be resident
     const bool dense = MP == 128;   // many token rows: tokens on the MMA's M side, 256 vocabulary rows per tile
     const long long units = (long long)((c.vocab + (dense ? 255 : 127)) / (dense ? 256 : 128)) * ((hdim + 63) / 64);
@@ -765,8 +714,6 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
     } else {
       e = launch_lm_head_umma(lp, h->map_lm, h->maps_gu.Xhi, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
     }
-  } else {
-    e = launch_lm_head(lp, st);
   }
   if (e != cudaSuccess) return fail_cuda(h, e);
   mark(6, false);
@@ -847,7 +794,6 @@ int dart_draft_prefill(dart_handle* h, const dart_prefill_in* in, void* cuda_str
   }
   if (total == 0) return DART_OK;
   if (!aligned32(in->feats) || in->tokens == nullptr) return DART_ERR_INVALID_ARG;
-  if (!h->umma) return DART_ERR_UNSUPPORTED_ARCH;   // the dense kernels need the tensor-map encoder
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   Workspace& ws = h->ws;
   const bf16* feats = static_cast<const bf16*>(in->feats);
@@ -948,10 +894,23 @@ int dart_last_device_status(dart_handle* h, void* cuda_stream) {
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return fail_cuda(h, e);
   if (v != 0) {
+    // A kernel gave up on a wait: the step's outputs are void, and CTAs that left between their tickets and their
+    // finalize have left group counters behind.  Clear them with the status word, so that the handle's next
+    // step starts from the state dart_draft_init left.
     cudaMemsetAsync(h->ws.status, 0, sizeof(int), st);
-    cudaStreamSynchronize(st);
+    const GemmPlan* plans[5] = {&h->plan_fc, &h->plan_qkv, &h->plan_o, &h->plan_gu, &h->plan_down};
+    for (int i = 0; i < 5; ++i) cudaMemsetAsync(plans[i]->d_ctr, 0, sizeof(int) * (size_t)plans[i]->n_groups, st);
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return fail_cuda(h, e);
   }
   return v == 0 ? DART_OK : DART_ERR_TIMEOUT;
+}
+
+int dart_selftest_bounded_wait(dart_handle* h, int32_t spin_limit, int32_t leave_ticket, void* cuda_stream) {
+  if (h == nullptr || spin_limit < 1 || spin_limit > 100000) return DART_ERR_INVALID_ARG;
+  const cudaError_t e = launch_bounded_wait_probe(spin_limit, h->ws.status, leave_ticket ? h->plan_qkv.d_ctr : nullptr,
+                                                  static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? DART_OK : fail_cuda(h, e);
 }
 
 }  // extern "C"

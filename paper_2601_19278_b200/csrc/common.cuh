@@ -8,55 +8,6 @@ namespace dart {
 
 typedef __nv_bfloat16 bf16;
 
-// 16-byte streaming load of weights: read-only path, do not keep the line in L1
-// (every weight byte is used exactly once per step).
-__device__ __forceinline__ uint4 ld_stream16(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
-}
-
-// 16-byte load of activations: small, re-read by every warp of the SM, so let L1 keep it.
-__device__ __forceinline__ uint4 ld_act16(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.ca.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
-}
-
-// 32-byte (256-bit) loads, sm_100: a lane's two 16-byte chunks of a k-step are adjacent (see chunk_k0/1),
-// so one instruction fetches both.  Addresses must be 32-byte aligned.
-struct U8 { uint32_t v[8]; };
-__device__ __forceinline__ U8 ld_stream32(const void* p) {
-  U8 r;
-  asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]), "=r"(r.v[4]), "=r"(r.v[5]), "=r"(r.v[6]), "=r"(r.v[7])
-               : "l"(p));
-  return r;
-}
-__device__ __forceinline__ U8 ld_act32(const void* p) {
-  U8 r;
-  asm volatile("ld.global.ca.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]), "=r"(r.v[4]), "=r"(r.v[5]), "=r"(r.v[6]), "=r"(r.v[7])
-               : "l"(p));
-  return r;
-}
-
-// Element offsets, inside a 64-wide k-step, of the two 16-byte chunks that lane t (= lane & 3)
-// of a quad loads from a weight row (and, identically, from an activation row).  Mode 0: the
-// quad's four lanes take bytes [32t, 32t+16) in one instruction and [32t+16, 32t+32) in the next,
-// so each instruction touches all four 32-byte sectors of the row's 128-byte line; mode 1: one
-// instruction covers bytes [0,64) contiguously, the next [64,128).  Mode 0 measured faster on
-// B200 (the memory system sees whole-line requests).
-#ifndef DART_CHUNK_MODE
-#define DART_CHUNK_MODE 0
-#endif
-__device__ __forceinline__ int chunk_k0(int t) { return DART_CHUNK_MODE == 0 ? t * 16 : t * 8; }
-__device__ __forceinline__ int chunk_k1(int t) { return DART_CHUNK_MODE == 0 ? t * 16 + 8 : t * 8 + 32; }
-
 // D(16x8,f32) += A(16x16,bf16,row) * B(16x8,bf16,col)
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {

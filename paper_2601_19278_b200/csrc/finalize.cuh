@@ -1,4 +1,4 @@
-// Fused epilogues of the projections, shared by the mma.sync and the tcgen05 streaming kernels: the CTA
+// Fused epilogues of the projections (umma_gemm.cu): the CTA
 // that completes a 128-row group (or a pair of groups) adds up the stream-K pieces and applies the step's
 // elementwise work (Section 3.2: RMSNorm scales, RoPE, residual adds, SiLU gating, cache append).
 #pragma once
@@ -48,7 +48,7 @@ __device__ __forceinline__ void meta_prefetch(const GemmArgs& p, int group, Grou
 }
 
 // The finalize runs on a team of NTHR threads that synchronises on barrier BAR (0 = __syncthreads, NTHR = the
-// whole CTA: what both kernel families use; a 256-thread team of otherwise idle warps was measured slower).
+// whole CTA; a 256-thread team of otherwise idle warps was measured slower).
 // ft is the thread's index in the team.
 template <int NTHR, int BAR>
 __device__ __forceinline__ void team_sync() {
@@ -142,17 +142,11 @@ __device__ __forceinline__ void tile_rows_sum(int ft, float (&v)[NV], float* sh)
 // dry = true executes the same instructions without a single store to global memory (a measurement aid: a
 // second call on the same group takes 3 us instead of 5.5, because the pieces, written by SMs all over the
 // chip, are then close by - not because of the code: a dry pass ahead of time does not help).
-// One instantiation per epilogue mode, so each mode only carries its own instructions.  A kernel that defines
-// DART_FINALIZE_INLINE before this header gets it inlined: its many reads of the arguments are then operands from
-// the constant bank; out of line they are dependent loads through a pointer (about 2 us more on the tail of every
-// projection), which the register-tight mma.sync kernels accept to keep their streaming loop free of spills.
-#ifdef DART_FINALIZE_INLINE
-#define DART_FINALIZE_ATTR __forceinline__
-#else
-#define DART_FINALIZE_ATTR __noinline__
-#endif
+// One instantiation per epilogue mode, so each mode only carries its own instructions; always inlined into the
+// kernel, so that its many reads of the arguments are operands from the constant bank (out of line they were
+// dependent loads through a pointer: about 2 us more on the tail of every projection).
 template <int MODE, int NTHR, int BAR>
-static __device__ DART_FINALIZE_ATTR void finalize_group_t(int ft, const GemmArgs& p, int group, int MP, float* sh, float* s_rstd,
+static __device__ __forceinline__ void finalize_group_t(int ft, const GemmArgs& p, int group, int MP, float* sh, float* s_rstd,
                                                      const int* s_pos, const GroupMeta* gm, FinSmem* fs, bool dry) {
   constexpr int NPAR = NTHR / 128;     // token classes: thread -> (row = ft & 127, class = ft >> 7)
   constexpr int NV = 8 / NPAR;         // tokens of an 8-token chunk per thread in the row-major modes
@@ -312,30 +306,10 @@ static __device__ __forceinline__ void finalize_group(int ft, const GemmArgs& p,
   }
 }
 
-// Shifted token embedding of the fresh rows (Section 3.2): e = E[token], normalised (its 1/rms needs
-// nothing else) and written as the second half of the fresh row's z.  One CTA per fresh row.
-static __device__ __noinline__ void embed_rows(const GemmArgs& p, float* sh, int ftok) {
-  const EpiArgs& e = p.epi;
-  const int orow = fresh_to_step_row(e, ftok);   // z row of fresh row (b, r)
-  const int id = min(max(e.tokens[ftok], 0), e.vocab - 1);
-  const bf16* row = e.embed + (size_t)id * e.h;
-  float ss = 0.f;
-  for (int n = threadIdx.x; n < e.h; n += blockDim.x) {
-    const float v = __bfloat162float(row[n]);
-    ss += v * v;
-  }
-  ss = block_sum(ss, sh);
-  const float rs = 1.f / sqrtf(ss / (float)e.h + e.eps);
-  for (int n = threadIdx.x; n < e.h; n += blockDim.x) {
-    bf16 hi, lo;
-    split_bf16(__bfloat162float(row[n]) * rs * __bfloat162float(e.gamma_e[n]), hi, lo);
-    e.out_hi[(size_t)orow * e.ld_out + e.h + n] = hi;
-    e.out_lo[(size_t)orow * e.ld_out + e.h + n] = lo;
-  }
-}
-
-// The same on a team of NTHR threads that synchronises on named barrier BAR (warps that idle while the projection
-// streams), with the arguments read from the kernel's constant bank.  red: NTHR / 32 floats of shared memory.
+// Shifted token embedding of the fresh rows (Section 3.2): e = E[token], normalised (its 1/rms needs nothing
+// else) and written as the second half of the fresh row's z.  Runs on a team of NTHR threads that synchronises on
+// named barrier BAR (warps that idle while the projection streams), with the arguments read from the kernel's
+// constant bank.  red: NTHR / 32 floats of shared memory.
 template <int NTHR, int BAR>
 static __device__ __forceinline__ void embed_row_team(const EpiArgs& e, int ft, float* red, int ftok) {
   const int orow = fresh_to_step_row(e, ftok);

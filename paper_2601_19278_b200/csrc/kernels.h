@@ -39,6 +39,9 @@ inline cudaError_t allow_dynamic_smem(const void* fn, size_t bytes) {
   return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
+// The cudaError_t behind a DART_ERR_CUDA of a call that has no handle (dart_last_cuda_error(NULL) reads it; api.cu).
+void record_global_cuda_error(cudaError_t e);
+
 // Launch with programmatic stream serialization (see pdl_wait / pdl_trigger in common.cuh).
 template <class... KArgs, class... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
@@ -76,14 +79,13 @@ struct GemmPlan {
   int nseg;
   GemmSeg seg[6];
   int Kd;           // reduction length per segment, multiple of 16
-  int SK;           // ceil(Kd / 64) k-steps per row
-  int KR;           // ceil(SK / 16) k-rounds per 16-row tile (16 warps take one k-step each)
-  int n_tiles;      // 128-row tiles over all segments (8 16-row tiles each)
+  int SK;           // ceil(Kd / 64) k-blocks per row
+  int KR;           // k-blocks per 128-row tile (= SK)
+  int n_tiles;      // 128-row tiles over all segments
   int grid;         // CTAs
-  int slots;        // max 16-row tiles a CTA touches
-  long long U;      // n_tiles * 8 * KR work units
+  int slots;        // max tiles a CTA touches
+  long long U;      // n_tiles * KR work units
   int pair_offset;  // > 0: tiles T and T + pair_offset are finalized together (group = T % pair_offset)
-  int umma;         // 1: units are (128-row tile, 64-k block) for the tcgen05 kernel (KR = k-blocks per tile), pieces hold 128 rows
   int n_groups;
   int* d_ctr;         // DEVICE [n_groups] tickets taken (zero between launches)
   int* d_expected;    // DEVICE [n_groups] tickets that complete a group
@@ -128,13 +130,13 @@ struct EpiArgs {
   bf16* q_hi; bf16* q_lo; bf16* k_new; bf16* v_new; bf16* k_cache; bf16* v_cache; long long P_cap;
 };
 
-// What the shared streaming core (stream_core.cuh) needs to know about a launch.
+// The weight sub-matrices and the activations of one streaming launch.
 struct StreamArgs {
   GemmSeg seg[6];     // sub-matrices streamed by this launch; tile0 in 128-row tiles
   int nseg;
   int Kd;             // reduction length (multiple of 16)
-  int SK;             // 64-wide k-steps per row
-  int KR;             // k-rounds per 16-row tile = ceil(SK / warps per CTA)
+  int SK;             // 64-wide k-blocks per row
+  int KR;             // k-blocks per 128-row tile (= SK)
   const bf16* x_hi;   // activations [rows, ldx] hi part
   const bf16* x_lo;   // lo part (== x_hi when the input is plain bf16)
   long long ldx;
@@ -151,8 +153,7 @@ struct GemmArgs {
   EpiArgs epi;
 };
 
-// The same projections on the tcgen05 / TMA path (umma_gemm.cu): plan units are (128-row tile, 64-k block),
-// one persistent CTA per SM.  Tensor maps: one per weight segment; Xhi = the activations: hi + lo inputs as one
+// The projections (umma_gemm.cu): plan units are (128-row tile, 64-k block), one persistent CTA per SM.  Tensor maps: one per weight segment; Xhi = the activations: hi + lo inputs as one
 // 3-D map (box = 64 k x (hi, lo) x MP rows: accumulator column 2t is token t's hi part, 2t+1 its lo part); a
 // plain-bf16 input as a 2-D map with a box of 2*MP rows whose missing rows read 0 (column t is token t).
 struct UmmaMaps {
@@ -188,6 +189,10 @@ cudaError_t launch_umma_dense(const DenseArgs& a, int n_sm, cudaStream_t st);
 cudaError_t launch_prefill_embed(const int32_t* tokens, int T, int vocab, const bf16* embed, const bf16* gain_e, int h, float eps,
                                  bf16* z, long long ldz, cudaStream_t st);
 
+// Self-test of the bounded waits (selftest.cu): a wait of `limit` tries on a barrier nobody signals; on expiry the
+// status word becomes DEV_TIMEOUT.  ticket != NULL: one ticket is taken on that counter first.
+cudaError_t launch_bounded_wait_probe(int limit, int* status, int* ticket, cudaStream_t st);
+
 // 2-D bf16 tensor map [outer][inner] (row stride ld_bytes), box {box_inner, box_outer}, 128-byte swizzle, zero fill.
 cudaError_t tmap_encode_bf16(CUtensorMap* m, const void* base, unsigned long long inner, unsigned long long outer,
                              unsigned long long ld_bytes, unsigned box_inner, unsigned box_outer);
@@ -195,7 +200,6 @@ cudaError_t tmap_encode_bf16(CUtensorMap* m, const void* base, unsigned long lon
 cudaError_t tmap_encode_bf16_pair(CUtensorMap* m, const void* hi, unsigned long long pair_bytes, unsigned long long inner,
                                   unsigned long long rows, unsigned long long ld_bytes, unsigned box_rows);
 
-cudaError_t launch_gemm_rows(const GemmPlan& plan, const GemmInput& in, const EpiArgs& epi, float* part, cudaStream_t st);
 // (cos, sin) table of RoPE for positions 0 .. n_pos-1 (once, at init)
 cudaError_t launch_rope_table(float2* tab, int n_pos, int dh, float theta, cudaStream_t st);
 // Copies the <mask> row into every z row (b, r) with r >= F (when the batch size or F changes)
@@ -238,14 +242,15 @@ cudaError_t attn_umma_setup();  // once per device
 cudaError_t launch_attn_umma_split(const AttnUmmaArgs& a, int max_chunks, cudaStream_t st);
 cudaError_t attention_setup();  // once per device: opt in to the kernels' dynamic shared memory
 // seq_lens_host: the same lengths on the host (sizes the grid and the partial layout); B <= 32.  With `maps`
-// (d_h = 128) the split runs on the tcgen05 kernel, otherwise on the mma.sync one; the combine is the same.
+// (d_h = 128, batches with a few thousand key tiles) the split runs on the tcgen05 kernel, otherwise on the warp-MMA one
+// that a single sequence's few chunks are faster on; the combine is the same.
 cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, const AttnUmmaMaps* maps, int* status, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
 // LM head with fused log-softmax / top-k partials, and the merge that finishes them.
 // ---------------------------------------------------------------------------------------------
 struct LmParams {
-  StreamArgs s;  // filled by launch_lm_head
+  StreamArgs s;  // unused by the LM-head kernels (kept zero)
   const bf16* W; int V; int Kd;
   const bf16* x_hi; const bf16* x_lo; long long ldx; int M; int K;  // token m = b*K + r
   const float* ss_in; int ss_tiles; int ss_mp; float rms_eps;  // final RMSNorm's 1/rms, applied to the logits
@@ -256,8 +261,7 @@ struct LmParams {
   float* part_key; float* part_y; int32_t* part_id;  // [grid][MP][32]
   int32_t* out_ids; float* out_slogit;  // [M, topk]
 };
-cudaError_t launch_lm_head(const LmParams& p, cudaStream_t st);
-// The tcgen05 / TMA LM head (p.grid CTAs, at most one per SM so that all of them are resident at once).
+// The LM head for up to 32 token rows (p.grid CTAs, at most one per SM so that all of them are resident at once).
 // pieces: [grid][128][MP] fp32 partial logits of tiles cut between CTAs; flags: [grid] ints, a CTA's piece is
 // complete when its flag equals `tag` (a value no earlier launch used).
 struct LmUmmaArgs {

@@ -123,12 +123,19 @@ extern "C" int dart_topk_rows_noalloc(const float* logits, int32_t rows, int32_t
   if (logits == nullptr || out_ids == nullptr || out_slogit == nullptr) return DART_ERR_INVALID_ARG;
   if (rows < 1 || vocab < 1 || topk < 1 || topk > 32 || topk > vocab || !(eps_logit >= 0.f)) return DART_ERR_INVALID_ARG;
   if (rows > kMaxRows) return DART_ERR_CAPACITY;  // the static scratch holds at most kMaxRows rows
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DART_ERR_CUDA;
+  int dev = 0, major = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { record_global_cuda_error(e); return DART_ERR_CUDA; }
+  if (dev < 0 || dev >= 64) return DART_ERR_INVALID_ARG;   // the address cache below holds 64 devices
   if (g_scratch_ptr[dev] == nullptr) {
-    // first call on this device (it must be the current device): resolve the array's device address
+    // first call on this device (it must be the current device): check the architecture once and resolve the
+    // array's device address.  Two host threads that get here together both store the same address: benign.
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) { record_global_cuda_error(e); return DART_ERR_CUDA; }
+    if (major != 10) return DART_ERR_UNSUPPORTED_ARCH;
     float* ptr = nullptr;
-    if (cudaGetSymbolAddress((void**)&ptr, g_topk_scratch) != cudaSuccess || ptr == nullptr) return DART_ERR_CUDA;
+    e = cudaGetSymbolAddress((void**)&ptr, g_topk_scratch);
+    if (e != cudaSuccess || ptr == nullptr) { record_global_cuda_error(e); return DART_ERR_CUDA; }
     g_scratch_ptr[dev] = ptr;
   }
   float* base = g_scratch_ptr[dev];
@@ -143,7 +150,7 @@ extern "C" int dart_topk_rows_noalloc(const float* logits, int32_t rows, int32_t
   p.out_ids = out_ids; p.out_slogit = out_slogit;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   slice_partials_kernel<<<dim3(kSlices, rows), 256, 0, st>>>(logits, vocab, MP, topk, p.part_stats, p.part_key, p.part_y, p.part_id);
-  if (cudaGetLastError() != cudaSuccess) return DART_ERR_CUDA;
-  if (launch_topk_merge(p, st) != cudaSuccess) return DART_ERR_CUDA;
+  if ((e = cudaGetLastError()) != cudaSuccess) { record_global_cuda_error(e); return DART_ERR_CUDA; }
+  if ((e = launch_topk_merge(p, st)) != cudaSuccess) { record_global_cuda_error(e); return DART_ERR_CUDA; }
   return DART_OK;
 }

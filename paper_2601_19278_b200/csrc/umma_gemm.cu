@@ -11,15 +11,14 @@
 //     the next tile's MMAs overlap the previous tile's read-out); tcgen05.commit frees the stage;
 //   * four warps read the accumulator out of tensor memory (tcgen05.ld), add the hi and lo halves and write
 //     the CTA's fp32 piece of the tile;
-//   * stream-K: the flattened (128-row tile, 64-k block) space is cut into gridDim.x equal ranges, pieces
-//     and tickets exactly as in the mma.sync kernel, and the CTA that takes a group's last ticket runs the
-//     same fused finalize (finalize.cuh) once the whole CTA is past its streaming loop.
+//   * stream-K: the flattened (128-row tile, 64-k block) space is cut into gridDim.x equal ranges;
+//     a CTA writes one fp32 piece per tile it touches and takes a ticket on the tile's group, and the CTA that
+//     takes a group's last ticket runs the fused finalize (finalize.cuh) once it is past its streaming loop.
 // TMA zero-fills what lies outside a matrix, so ragged row counts, k tails and missing token rows need no
 // predicates here.
 #include "common.cuh"
 #include "kernels.h"
 #include "umma.cuh"
-#define DART_FINALIZE_INLINE
 #include "finalize.cuh"
 
 namespace dart {

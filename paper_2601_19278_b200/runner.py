@@ -11,7 +11,13 @@ import torch
 from . import binding, synthetic
 
 
+GUARD = 64   # sentinel elements in front of and behind every output buffer
+
+
 class DraftSession:
+    """Every output buffer sits between two runs of sentinel elements; check_guards() (called by tree_outputs() and
+    close()) fails if a kernel wrote outside the buffer it was given."""
+
     def __init__(self, w: synthetic.Workload, weights: Dict[str, torch.Tensor], ngram: Optional[Dict[str, np.ndarray]],
                  device: str = "cuda:0", want_logits: bool = False, **cfg_over):
         self.w = w
@@ -21,17 +27,35 @@ class DraftSession:
         self.weights = {k: v.to(self.dev) for k, v in weights.items()}
         self.draft = binding.DartDraft(self.cfg, self.weights, ngram)
         B, K, k, bud = w.batch, w.K, self.cfg.topk, self.cfg.tree_budget
-        i32 = dict(dtype=torch.int32, device=self.dev)
-        self.topk_ids = torch.full((B, K, k), -7, **i32)
-        self.topk_slogit = torch.zeros((B, K, k), dtype=torch.float32, device=self.dev)
-        self.logits = torch.zeros((B, K, w.vocab), dtype=torch.float32, device=self.dev) if want_logits else None
-        self.tokens = torch.full((B, bud), -7, **i32)
-        self.parents = torch.full((B, bud), -7, **i32)
-        self.depth = torch.full((B, bud), -7, **i32)
-        self.mask = torch.full((B, bud, bud), 9, dtype=torch.uint8, device=self.dev)
-        self.n_nodes = torch.zeros((B,), **i32)
-        self.scores = torch.zeros((B, bud), dtype=torch.float32, device=self.dev)
+        self._guards = []
+        self.topk_ids = self._guarded((B, K, k), torch.int32, -7)
+        self.topk_slogit = self._guarded((B, K, k), torch.float32, 0)
+        self.logits = self._guarded((B, K, w.vocab), torch.float32, 0) if want_logits else None
+        self.tokens = self._guarded((B, bud), torch.int32, -7)
+        self.parents = self._guarded((B, bud), torch.int32, -7)
+        self.depth = self._guarded((B, bud), torch.int32, -7)
+        self.mask = self._guarded((B, bud, bud), torch.uint8, 9)
+        self.n_nodes = self._guarded((B,), torch.int32, 0)
+        self.scores = self._guarded((B, bud), torch.float32, 0)
         self.inp = None
+
+    _SENTINEL = {torch.int32: 0x5A5A5A5A, torch.float32: 1.2345e30, torch.uint8: 0xA5}
+
+    def _guarded(self, shape, dtype, fill) -> torch.Tensor:
+        n = int(np.prod(shape))
+        buf = torch.full((n + 2 * GUARD,), self._SENTINEL[dtype], dtype=dtype, device=self.dev)
+        view = buf[GUARD:GUARD + n].view(shape)
+        view.fill_(fill)
+        self._guards.append((buf, n))
+        return view
+
+    def check_guards(self) -> None:
+        """The sentinels around every output buffer are intact: no kernel wrote before or behind its output."""
+        torch.cuda.synchronize(self.dev)
+        for buf, n in self._guards:
+            want = torch.tensor(self._SENTINEL[buf.dtype], dtype=buf.dtype, device=self.dev)
+            assert bool((buf[:GUARD] == want).all()) and bool((buf[GUARD + n:] == want).all()), \
+                f"a kernel wrote outside a {buf.dtype} output buffer of {n} elements"
 
     def load_inputs(self, inp: Dict[str, object]) -> None:
         """Copy one step's inputs (synthetic.make_step_inputs) to the device."""
@@ -110,10 +134,13 @@ class DraftSession:
                               n_nodes=self.n_nodes, scores=self.scores, first_row=fr, stream=stream)
 
     def tree_outputs(self) -> Dict[str, np.ndarray]:
-        torch.cuda.synchronize(self.dev)
+        self.check_guards()
         return {"tokens": self.tokens.cpu().numpy(), "parents": self.parents.cpu().numpy(),
                 "depth": self.depth.cpu().numpy(), "mask": self.mask.cpu().numpy(),
                 "n_nodes": self.n_nodes.cpu().numpy(), "scores": self.scores.cpu().numpy()}
 
     def close(self):
+        if self._guards:
+            self.check_guards()
+            self._guards = []
         self.draft.close()

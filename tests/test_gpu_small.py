@@ -121,7 +121,7 @@ def test_runs_are_bitwise_repeatable():
     w = CASES["dh128_k8"]
     wt, inp, rows, ses = _run(w)
     a = (ses.logits.clone(), ses.topk_ids.clone(), ses.topk_slogit.clone(), ses.tokens.clone(), ses.mask.clone())
-    for _ in range(5):
+    for _ in range(20):
         ses.step(step_counter=5)
         ses.tree()
         torch.cuda.synchronize()

@@ -67,6 +67,39 @@ def test_sharp_softmax_moves_the_reference_maximum():
     _run(1, 2, 1, 300, 4, [300], seed=5, q_scale=6.0)
 
 
+def test_long_packed_row_on_sampled_query_slots():
+    """A packed row of the size the kernel is timed on has tens of thousands of slots; the oracle (one visibility
+    test per slot pair) checks a seeded sample of query slots from every region of the mask: clean slots, the first
+    and last masked blocks, blocks in the middle, block boundaries, the last valid slots and slots past the length."""
+    B, Hq, Hkv, Lp, d, dh = 1, 10, 2, 1100, 8, 128          # groups of five query heads, as at the 14B shape
+    S = 1063                                                 # valid prompt slots: the tail of the row reads nothing
+    L = Lp * (1 + d)
+    g = torch.Generator().manual_seed(21)
+    q = torch.randn(B, Hq, L, dh, generator=g).to(torch.bfloat16)
+    k = torch.randn(B, Hkv, L, dh, generator=g).to(torch.bfloat16)
+    v = torch.randn(B, Hkv, L, dh, generator=g).to(torch.bfloat16)
+    dev = torch.device("cuda:0")
+    out = torch.full((B, Hq, L, dh), float("nan"), dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    binding.train_attention_fwd(q.to(dev), k.to(dev), v.to(dev), [S], Lp, d, out, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = out[0].float().cpu().numpy().astype(np.float64)
+    assert not np.isnan(got).any()
+    rng = np.random.default_rng(22)
+    block = lambda n: list(range(Lp + n * d, Lp + (n + 1) * d))
+    slots = [0, 1, 63, 64, 127, 128, 129, S - 1, S, Lp - 1]                                   # clean part, tile edges, length cut
+    slots += block(0) + block(1) + block(15) + block(16) + block(S - 1) + block(S) + block(Lp - 1)
+    slots += rng.integers(0, S, 24).tolist()                                                  # random clean slots
+    slots += [Lp + int(n) * d + int(r) for n, r in zip(rng.integers(0, S, 40), rng.integers(0, d, 40))]   # random block slots
+    slots = sorted(set(slots))
+    ref = ota.training_attention(q[0].double().numpy(), k[0].double().numpy(), v[0].double().numpy(), Lp, d, S, query_slots=slots)
+    err = np.abs(got[:, slots] - ref[:, slots])
+    assert np.all(err <= ATOL + RTOL * np.abs(ref[:, slots])), float(err.max())
+    assert np.abs(ref[:, slots]).max() > 0.1
+    assert np.all(got[:, S:Lp] == 0) and np.all(got[:, Lp + S * d:] == 0)
+
+
 def test_argument_errors():
     dev = torch.device("cuda:0")
     B, Hq, Hkv, Lp, d, dh = 1, 2, 1, 16, 8, 128
