@@ -33,7 +33,8 @@ struct Workspace {
   float* rstd_mask = nullptr;
   float* mask_res = nullptr;    // [h] g half of the <mask> representation as fp32
   float2* rope_tab = nullptr;   // [max_prefix + K][dh/2] (cos, sin)
-  float* bg = nullptr;          // [max_batch][topk + (K-1)*topk^2] bigram scores of the tree builder
+  float* sg = nullptr;          // [max_batch][tree_sg_floats] dense N-gram scores of the tree builder (hash layout)
+  float* bg = nullptr;          // [max_batch][topk + (K-1)*topk^2] bigram scores of the tree builder (trie layout)
   uint2* cx = nullptr;          // [max_batch][1 + topk + (K-2)*topk^2] child ranges of the 3-gram contexts (trie layout)
   float *o_part = nullptr, *ml_part = nullptr;
   float *lm_stats = nullptr, *lm_key = nullptr, *lm_y = nullptr;
@@ -219,6 +220,7 @@ size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_p
   TAKE(rstd_mask, float*, 256);
   TAKE(mask_res, float*, (size_t)c.hidden * sizeof(float));
   TAKE(rope_tab, float2*, (size_t)(c.max_prefix + c.K) * (c.head_dim / 2) * sizeof(float2));
+  TAKE(sg, float*, (size_t)c.max_batch * tree_sg_floats(c.topk, c.K) * sizeof(float));
   TAKE(bg, float*, (size_t)c.max_batch * (c.topk + (size_t)(c.K - 1) * c.topk * c.topk) * sizeof(float));
   TAKE(cx, uint2*, (size_t)c.max_batch * (1 + c.topk + (size_t)(c.K > 2 ? c.K - 2 : 0) * c.topk * c.topk) * sizeof(uint2));
   TAKE(o_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * c.head_dim * sizeof(float));
@@ -867,7 +869,7 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
   for (int i = 0; i < 8; ++i) { tp.wl[i] = h->wl[i]; tp.wv[i] = h->wv[i]; }
   tp.trie.bi_off = h->ng_trie.bi_off; tp.trie.bi_ent = h->ng_trie.bi_ent; tp.trie.tri_off = h->ng_trie.tri_off;
   tp.trie.tri_node = h->ng_trie.tri_node; tp.trie.tri_ent = h->ng_trie.tri_ent; tp.trie.nb8 = 8u * (uint32_t)((c.vocab + 479) / 480);
-  tp.wn = h->wn; tp.miss = h->miss; tp.bg = h->ws.bg; tp.cx = h->ws.cx;
+  tp.wn = h->wn; tp.miss = h->miss; tp.sg = h->ws.sg; tp.bg = h->ws.bg; tp.cx = h->ws.cx;
   tp.tokens = out->tokens; tp.parents = out->parents; tp.depth = out->depth; tp.mask = out->mask;
   tp.n_nodes = out->n_nodes; tp.scores = out->scores; tp.status = h->ws.status;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

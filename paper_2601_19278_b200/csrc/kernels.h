@@ -326,7 +326,8 @@ struct TreeParams {
   const int32_t* ids; const float* slogit; const int32_t* ctx_tail;
   NgramTable table;
   NgramTrie trie;   // used instead of `table` when trie.bi_off != nullptr
-  float* bg;   // [B][topk + (n_levels-1)*topk^2] bigram scores (workspace, written by the sweep kernel)
+  float* sg;   // [B][tree_sg_floats] dense s_ng table of the hash layout (workspace, written by ngram_sweep_kernel)
+  float* bg;   // [B][topk + (n_levels-1)*topk^2] bigram scores of the trie layout (workspace, written by trie_sweep_kernel)
   uint2* cx;   // [B][1 + topk + (n_levels-2)*topk^2] child ranges of the 3-gram contexts (trie layout only)
   float wl[8]; float wv[8]; float wn; float miss;
   int32_t* tokens; int32_t* parents; int32_t* depth; uint8_t* mask; int32_t* n_nodes; float* scores;
@@ -337,6 +338,7 @@ cudaError_t tree_setup(int topk, int beam, int budget, int max_levels);  // once
 cudaError_t launch_verify_inputs(int B, int budget, int max_levels, const int32_t* parents, const int32_t* depth, const int32_t* n_nodes,
                                  const int32_t* root_pos, int32_t* position_ids, int32_t* retrieve, int32_t* n_leaves, cudaStream_t st);
 size_t tree_smem_bytes(int topk, int beam, int budget, int n_levels);
+size_t tree_sg_floats(int topk, int levels);   // floats per sequence of TreeParams::sg
 cudaError_t launch_tree(const TreeParams& p, cudaStream_t st);
 
 // key packing shared by the host-side table builder and the device lookup

@@ -7,21 +7,20 @@
 // (__fmul_rn/__fadd_rn), in the same order as a sequential evaluation, so the tree is
 // bit-exact with one.
 //
-// Latency is what matters here (a few thousand candidates, a few hundred random 16-byte reads):
-//   * every bigram a level can ask for is known up front -- (token of S_{i-1}, token of S_i) --
-//     so all of them are looked up by a separate many-block kernel first (one SM cannot keep
-//     4400 random reads in flight; 13 us inside this kernel against ~2 us spread over the GPU);
-//     inside the level loop each candidate needs one trigram probe, whose context only exists
-//     once the previous level's beam is known;
-//   * selection is a bitonic merge tree held in registers.  Every warp sorts its 32 candidates
-//     with a shuffle network (total order: score desc, generation index asc); pairs of warps
-//     then merge their runs, keeping the best 64 (two per lane): C[p] = better(A[p], B[63-p])
-//     is a bitonic sequence holding the best 64 of A and B, which six compare-exchange stages
-//     sort.  After log2(warps) rounds warp 0 holds the level's best 64 in order: the first w
-//     are the next beam (w <= 32).  There are no data-dependent loops and the result does
-//     not depend on thread timing;
-//   * the final top-theta (theta <= 63) is kept the same way: warp 0 merges each level's best
-//     64 (by ancestor-clamped score, node index asc) into a running global best 64.
+// Latency is what matters here (a few thousand candidates, a few hundred random 16-byte reads per level if they
+// were made inside the level loop).  With the hash layout (ngram_sweep_kernel + tree_hash_kernel):
+//   * every N-gram score a level can ask for is known before the first level runs -- the context of a level-i
+//     candidate is (a token of S_{i-2}, a token of S_{i-1}) -- so a many-block sweep looks all of them up first
+//     (k + k^2 + (levels-2) k^3 lookups: 94 400 at k = 25 and 8 levels, a few hundred per SM, one round trip) and
+//     leaves the final s_ng (3-gram row, else 2-gram row, else log eps) in a dense table; the tree kernel copies
+//     one level's slice of it (k^3 floats) into shared memory while the previous level is being selected, so the
+//     level loop itself touches no global memory;
+//   * the per-level selection is block_select64 of select.cuh (histogram threshold + rank counting, four barriers);
+//   * the final top-theta (theta <= 63) is a running best 64 (by ancestor-clamped score, node index asc) that the
+//     block's last warp merges one level behind, while the other warps rank the next level's survivors.
+// With the trie layout (trie_sweep_kernel + tree_kernel) the 3-gram scores are read inside the level loop -- one warp
+// per beam entry walks its context's child list -- and the selection is the register merge tree of select.cuh.
+// Nothing depends on the order in which threads run.
 #include "common.cuh"
 #include "kernels.h"
 #include "select.cuh"
@@ -171,29 +170,60 @@ __host__ __device__ inline size_t tree_layout(int k, int w, int budget, int L, u
   return o;
 }
 
-// Bigram scores of every (level, previous candidate, candidate) triple, one lookup per thread:
-// bg[b][jt] = (ctx1, S_0[jt]) for e < k, bg[b][k + (i-1)k^2 + jb*k + jt] = (S_{i-1}[jb], S_i[jt]); a missing row
-// gives log(eps).
-__global__ void __launch_bounds__(256) bigram_sweep_kernel(const TreeParams p) {
+// ---- dense N-gram score table of one sequence (hash layout), written by ngram_sweep_kernel ----
+//   level 0          sg[j]                                   context (c_-2, c_-1),           candidate S_0[j]
+//   level 1          sg[o1 + j' k + j]                       context (c_-1, S_0[j']),        candidate S_1[j]
+//   level i >= 2     sg[o2 + (i-2) st3 + (j'' k + j') k + j] context (S_{i-2}[j''], S_{i-1}[j']), candidate S_i[j]
+// Offsets and strides are multiples of four floats so that slices can be copied with 16-byte cp.async.
+struct SgLayout { int o1, o2, st3, total; };
+__host__ __device__ inline SgLayout sg_layout(int k, int levels) {
+  SgLayout g;
+  g.o1 = (k + 3) & ~3;
+  g.o2 = (g.o1 + k * k + 3) & ~3;
+  g.st3 = (k * k * k + 3) & ~3;
+  g.total = g.o2 + (levels > 2 ? levels - 2 : 0) * g.st3;
+  return g;
+}
+size_t tree_sg_floats(int topk, int levels) { return (size_t)sg_layout(topk, levels).total; }
+
+// One thread per table entry: s_ng = the 3-gram row's score, else the 2-gram row's, else log(eps) (Algorithm 1
+// line 9, Appendix C / D).  Both first slots are requested before either is examined.
+__global__ void __launch_bounds__(256) ngram_sweep_kernel(const TreeParams p) {
   pdl_wait();
   pdl_trigger();   // a short kernel: the next one may be scheduled and run its set-up now
   const int k = p.topk, b = blockIdx.y;
   const int fr = p.first_rows[b], Lb = min(p.n_levels, p.K - fr);   // this sequence's level 0 row and levels
-  const int n_bg = k + (p.n_levels - 1) * k * k;                   // layout stride: the launch's maximum
+  const SgLayout g = sg_layout(k, p.n_levels);
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= k + (Lb - 1) * k * k) return;
   const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
-  int tb, tt;
-  if (e < k) { tb = p.ctx_tail[2 * b + 1]; tt = ids[e]; }
-  else { const int r = e - k, i = r / (k * k), q = r - i * k * k, jb = q / k; tb = ids[i * k + jb]; tt = ids[(i + 1) * k + q - jb * k]; }
-  float sc = p.miss;
-  if (p.table.slots != nullptr && tb >= 0) {
-    const unsigned long long key = ngram_key(2, -1, tb, tt);
-    const uint32_t hh = (uint32_t)ngram_hash(key) & p.table.mask;
-    float v;
-    if (probe_rest(p.table, key, hh, load_slot(p.table.slots + hh), v)) sc = v;
+  int ta, tb, tt, dst;
+  const int k2 = k * k, k3 = k2 * k;
+  if (e < k) {
+    ta = p.ctx_tail[2 * b]; tb = p.ctx_tail[2 * b + 1]; tt = ids[e]; dst = e;
+  } else if (e < k + k2) {
+    if (Lb < 2) return;
+    const int r = e - k, j1 = r / k;
+    ta = p.ctx_tail[2 * b + 1]; tb = ids[j1]; tt = ids[k + r - j1 * k]; dst = g.o1 + r;
+  } else {
+    const int r = e - k - k2, i = 2 + r / k3;
+    if (i >= Lb) return;
+    const int q = r - (i - 2) * k3, j2 = q / k2, j1 = (q - j2 * k2) / k;
+    ta = ids[(i - 2) * k + j2]; tb = ids[(i - 1) * k + j1]; tt = ids[i * k + q - j2 * k2 - j1 * k];
+    dst = g.o2 + (i - 2) * g.st3 + q;
   }
-  p.bg[(size_t)b * n_bg + e] = sc;
+  float sc = p.miss;
+  const NgramTable T = p.table;
+  if (T.slots != nullptr && tb >= 0) {
+    const bool tri = p.ngram_order >= 3 && ta >= 0;
+    const unsigned long long k2key = ngram_key(2, -1, tb, tt), k3key = ngram_key(3, tri ? ta : 0, tb, tt);
+    const uint32_t h2 = (uint32_t)ngram_hash(k2key) & T.mask, h3 = (uint32_t)ngram_hash(k3key) & T.mask;
+    const NgramSlot s2 = load_slot(T.slots + h2);
+    const NgramSlot s3 = tri ? load_slot(T.slots + h3) : s2;
+    float v;
+    if (probe_rest(T, k2key, h2, s2, v)) sc = v;
+    if (tri && probe_rest(T, k3key, h3, s3, v)) sc = v;
+  }
+  p.sg[(size_t)b * g.total + dst] = sc;
 }
 
 // The sweep for the trie layout: one warp per (level i, list kind, context position jb).  The context token x is
@@ -259,8 +289,10 @@ __global__ void __launch_bounds__(256) trie_sweep_kernel(const TreeParams p) {
   }
 }
 
+// The tree kernel of the trie layout.
 // MAXT: launch bound (512 leaves the compiler twice the registers; 1024 covers beam * topk up to 1024)
-// TRIE: the N-gram is the child-list trie (3-gram scores: search the context's children, located by the sweep).
+// TRIE: always true here (the hash layout runs tree_hash_kernel below); the N-gram is the child-list trie
+// (3-gram scores: search the context's children, located by the sweep).
 template <int MAXT, bool TRIE>
 __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
   extern __shared__ __align__(16) unsigned char tsm[];
@@ -274,9 +306,7 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
   pdl_wait();
   const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
   const float* sl = p.slogit + ((size_t)b * p.K + fr) * k;
-  const int ctx0 = p.ctx_tail[2 * b], ctx1 = p.ctx_tail[2 * b + 1];
-  const NgramTable T = p.table;
-  const bool have_table = T.slots != nullptr;
+  const int ctx1 = p.ctx_tail[2 * b + 1];
   const float* bg = p.bg + (size_t)b * sweep_bigrams(k, p.n_levels);  // bigram scores from the sweep kernel
   const uint2* cx = TRIE ? p.cx + (size_t)b * sweep_contexts(k, p.n_levels) : nullptr;
 
@@ -334,18 +364,11 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
     if (tid < ncand) {
       const int rho = tid / k, j = tid - rho * k;
       const int node = beam[rho];
-      const int tb = m.n_tok[node];
-      const int ta = node == 0 ? ctx0 : m.n_tok[m.n_par[node]];
       const int t = ids[i * k + j];
       float s_ng = __ldg(bg + (i == 0 ? j : k + (i - 1) * k * k + (int)m.n_j[node] * k + j));
       if (TRIE) {
         const int f = m.fj[i * k + j];
         if ((hit[rho] >> f) & 1u) s_ng = __uint_as_float(s3[rho * k + f]);
-      } else if (have_table && p.ngram_order >= 3 && ta >= 0 && tb >= 0) {
-        const unsigned long long k3 = ngram_key(3, ta, tb, t);
-        const uint32_t h3 = (uint32_t)ngram_hash(k3) & T.mask;
-        float v;
-        if (probe_rest(T, k3, h3, load_slot(T.slots + h3), v)) s_ng = v;
       }
       const float inc = __fmul_rn(__fadd_rn(__fmul_rn(p.wl[i], sl[i * k + j]), __fmul_rn(p.wn, s_ng)), p.wv[i]);
       s = __fadd_rn(m.n_score[node], inc);
@@ -432,6 +455,216 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------------
+// The tree kernel of the hash layout: Algorithm 1 over the dense score table of ngram_sweep_kernel.
+// ------------------------------------------------------------------------------------------------------
+struct HashTreeSmem {
+  float* n_score; float* n_clamp; int* n_tok; int* n_par;   // per node (the root is node 0)
+  int* c_ids; float* c_sl;                         // [L][k] the candidates' ids and s_logit, staged once
+  int* b_node; float* b_sc; float* b_cl; int* b_row;   // per beam entry: node, score, clamped score, row of its context in the level's slice
+  Key* lvl_sorted;                                 // [2][64] best of a level by clamped score (the running best lags one level behind)
+  int* sel; int* par_out; int* lvl_base;
+  SelectSmem* ss;
+  float* sg01; float* slice;                       // staged score table: levels 0 and 1; one level >= 2
+};
+__host__ __device__ inline size_t hash_tree_layout(int k, int w, int budget, int L, bool stage, unsigned char* base, HashTreeSmem* t) {
+  const int n_max = 1 + k + (L - 1) * w * k;
+  const SgLayout g = sg_layout(k, L);
+  size_t o = 0;
+  auto take = [&](size_t bytes) { const size_t r = o; o += (bytes + 15) & ~size_t(15); return r; };
+  const size_t o_sc = take((size_t)n_max * 4), o_cl = take((size_t)n_max * 4), o_tok = take((size_t)n_max * 4), o_par = take((size_t)n_max * 4),
+               o_ci = take((size_t)L * k * 4), o_cs = take((size_t)L * k * 4),
+               o_bn = take((size_t)w * 4), o_bs = take((size_t)w * 4), o_bc = take((size_t)w * 4), o_br = take((size_t)w * 4),
+               o_ls = take(2 * 64 * 8), o_sel = take((size_t)(budget + 1) * 4), o_po = take((size_t)budget * 4),
+               o_lb = take((size_t)(L + 1) * 4), o_ss = take(sizeof(SelectSmem)),
+               o_01 = take(stage ? (size_t)g.o2 * 4 : 0), o_sl = take(stage && L > 2 ? (size_t)g.st3 * 4 : 0);
+  if (t != nullptr) {
+    t->n_score = reinterpret_cast<float*>(base + o_sc);
+    t->n_clamp = reinterpret_cast<float*>(base + o_cl); t->n_tok = reinterpret_cast<int*>(base + o_tok);
+    t->n_par = reinterpret_cast<int*>(base + o_par);
+    t->c_ids = reinterpret_cast<int*>(base + o_ci); t->c_sl = reinterpret_cast<float*>(base + o_cs);
+    t->b_node = reinterpret_cast<int*>(base + o_bn); t->b_sc = reinterpret_cast<float*>(base + o_bs);
+    t->b_cl = reinterpret_cast<float*>(base + o_bc); t->b_row = reinterpret_cast<int*>(base + o_br);
+    t->lvl_sorted = reinterpret_cast<Key*>(base + o_ls);
+    t->sel = reinterpret_cast<int*>(base + o_sel); t->par_out = reinterpret_cast<int*>(base + o_po);
+    t->lvl_base = reinterpret_cast<int*>(base + o_lb); t->ss = reinterpret_cast<SelectSmem*>(base + o_ss);
+    t->sg01 = reinterpret_cast<float*>(base + o_01); t->slice = reinterpret_cast<float*>(base + o_sl);
+  }
+  return o;
+}
+
+// 16-byte asynchronous copies global -> shared by the whole block (n4 chunks), one commit group.
+__device__ __forceinline__ void copy_async16(float* dst, const float* src, int n4) {
+  for (int e = threadIdx.x; e < n4; e += blockDim.x) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(dst + 4 * e);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + 4 * e) : "memory");
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// STAGE: the score table's slices are staged in shared memory (they fit for the paper's k = 25); otherwise the
+// level loop reads the table where the sweep left it (L2).
+template <int MAXT, bool STAGE>
+__global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
+  extern __shared__ __align__(16) unsigned char tsm[];
+  const int k = p.topk, w = p.beam, theta = p.budget - 1;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x, last_warp = (nthr >> 5) - 1;
+  const int fr = p.first_rows[b], L = min(p.n_levels, p.K - fr);   // this sequence's level 0 row and levels
+  HashTreeSmem m;
+  hash_tree_layout(k, w, p.budget, p.n_levels, STAGE, tsm, &m);
+  __shared__ unsigned long long s_bits[64];
+  const SgLayout g = sg_layout(k, p.n_levels);
+#ifdef DART_TREE_TL
+  __shared__ long long s_tl[40];
+  int n_tl = 0;
+  const long long tl0 = clock64();
+#define TL_STAMP() do { if (tid == 0 && n_tl < 40) s_tl[n_tl] = clock64() - tl0; ++n_tl; } while (0)
+#else
+#define TL_STAMP() do {} while (0)
+#endif
+
+  if (tid == 0) { m.n_score[0] = 0.f; m.n_clamp[0] = INFINITY; m.n_par[0] = -1; m.b_node[0] = 0; m.b_sc[0] = 0.f; m.b_cl[0] = INFINITY; m.b_row[0] = 0; m.lvl_base[0] = 1; }
+  pdl_wait();
+  TL_STAMP();
+  const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
+  const float* sl = p.slogit + ((size_t)b * p.K + fr) * k;
+  const float* sg = p.sg + (size_t)b * g.total;
+  if (tid == 0) m.n_tok[0] = p.ctx_tail[2 * b + 1];
+  for (int e = tid; e < L * k; e += nthr) { m.c_ids[e] = ids[e]; m.c_sl[e] = sl[e]; }
+  if (STAGE) {
+    copy_async16(m.sg01, sg, g.o2 / 4);
+    asm volatile("cp.async.wait_all;" ::: "memory");    // the scores of levels 0 and 1
+  }
+  block_select_init(m.ss);
+  __syncthreads();
+  // running best 64 by (clamped score desc, node index asc): lives in the last warp's registers
+  Key g0 = kPadKey, g1 = kPadKey;
+  TL_STAMP();
+
+  int nb = 1;
+  for (int i = 0; i < L; ++i) {
+    const int ncand = nb * k;
+    const int base = m.lvl_base[i];
+    float s = -INFINITY, cl = -INFINITY;
+    if (tid < ncand) {
+      const int rho = tid / k, j = tid - rho * k;
+      const int t = m.c_ids[i * k + j];
+      const int at = m.b_row[rho] + j;
+      float s_ng;
+      if (STAGE) s_ng = i < 2 ? m.sg01[(i == 0 ? 0 : g.o1) + at] : m.slice[at];
+      else s_ng = __ldg(sg + (i == 0 ? 0 : i == 1 ? g.o1 : g.o2 + (i - 2) * g.st3) + at);
+      const float inc = __fmul_rn(__fadd_rn(__fmul_rn(p.wl[i], m.c_sl[i * k + j]), __fmul_rn(p.wn, s_ng)), p.wv[i]);
+      s = __fadd_rn(m.b_sc[rho], inc);
+      const float pc = m.b_cl[rho];
+      cl = s < pc ? s : pc;
+      const int n = base + tid;
+      m.n_score[n] = s; m.n_clamp[n] = cl; m.n_tok[n] = t; m.n_par[n] = m.b_node[rho];
+    }
+    // keys carry the node index base + tid, which orders candidates of one level like tid does
+    // best 64 by score -> next beam; `differs`: some clamped score is not its score (never, when increments <= 0)
+    TL_STAMP();
+    const bool more = STAGE && (i == 0 ? L > 2 : (i >= 2 && i + 1 < L));   // a slice to fetch while this level is selected
+    const int nb_next = ncand < w ? ncand : w;
+    const int pbase = i > 0 ? m.lvl_base[i - 1] : 0;
+    Key* lvl_out = m.lvl_sorted + (i & 1) * 64;
+    const int differs = block_select64(
+        tid < ncand ? make_key(s, base + tid) : kPadKey, s, tid < ncand && cl != s, m.ss,
+        [&](int r, Key key, int any) {
+          if (!any) lvl_out[r] = key;
+          if (r < nb_next) {
+            // beam entry r of the next level: its node, scores and the row of its context -- (the parent's candidate
+            // index, this node's candidate index) -- in the next level's slice of the score table
+            const int node = key_index(key), j = (node - base) % k;
+            m.b_node[r] = node;
+            m.b_sc[r] = m.n_score[node];
+            m.b_cl[r] = m.n_clamp[node];
+            m.b_row[r] = (i == 0 ? j : ((m.n_par[node] - pbase) % k) * k + j) * k;
+          }
+        },
+        [&]() {
+          // every thread has read what it needs of level i's slice: the next one may overwrite it (levels 0 and 1 use
+          // the small table, so level 2's slice is fetched during level 0 and nothing during level 1)
+          if (more) copy_async16(m.slice, sg + g.o2 + (i == 0 ? 0 : i - 1) * g.st3, g.st3 / 4);
+        },
+        [&]() {
+          // the running best takes in the previous level's best 64 while the first warps rank this level's survivors
+          if (warp == last_warp && i > 0) {
+            const Key* q = m.lvl_sorted + ((i - 1) & 1) * 64;
+            merge_keep64(g0, g1, q[lane], q[32 + lane], lane);
+          }
+          if (tid == 0) m.lvl_base[i + 1] = base + ncand;
+          if (STAGE && i >= 1) asm volatile("cp.async.wait_all;" ::: "memory");   // the next level's slice has landed
+        });
+    if (differs)   // the level's best 64 by clamped score are a different set: select again
+      block_select64(tid < ncand ? make_key(cl, base + tid) : kPadKey, cl, 0, m.ss, [&](int r, Key key, int) { lvl_out[r] = key; }, [] {}, [] {});
+    TL_STAMP();
+    nb = nb_next;
+  }
+  if (warp == last_warp && L > 0) {
+    const Key* q = m.lvl_sorted + ((L - 1) & 1) * 64;
+    merge_keep64(g0, g1, q[lane], q[32 + lane], lane);
+  }
+
+  // ---- the selected nodes: the first n_sel entries of the running best 64
+  const int total = m.lvl_base[L] - 1;
+  const int n_sel = total < theta ? total : theta;
+  if (warp == last_warp) {
+    if (lane < n_sel) m.sel[1 + lane] = key_index(g0);
+    if (32 + lane < n_sel) m.sel[33 + lane] = key_index(g1);
+    if (lane == 0) m.sel[0] = 0;
+  }
+  __syncthreads();
+
+  // ---- outputs
+  const int budget = p.budget;
+  int* slot_of = reinterpret_cast<int*>(m.n_score);   // node -> output slot (the scores are no longer needed)
+  for (int x = tid; x <= n_sel; x += nthr) slot_of[m.sel[x]] = x;
+  __syncthreads();
+  // the selection is closed under "parent of" (clamped scores never rise along a path), so every parent has a slot
+  for (int x = tid; x < budget; x += nthr) m.par_out[x] = (x >= 1 && x <= n_sel) ? slot_of[m.n_par[m.sel[x]]] : -1;
+  __syncthreads();
+  for (int x = tid; x < budget; x += nthr) {
+    const size_t o = (size_t)b * budget + x;
+    unsigned long long bits = 0ull;
+    if (x <= n_sel) {
+      const int n = m.sel[x];
+      int lev = 0;
+      if (x > 0) {
+        while (n >= m.lvl_base[lev + 1]) ++lev;
+        lev += 1;
+      }
+      p.tokens[o] = m.n_tok[n];
+      p.parents[o] = m.par_out[x];
+      p.depth[o] = lev;
+      if (p.scores) p.scores[o] = x == 0 ? 0.f : m.n_clamp[n];
+      int y = x;
+      for (int guard = 0; guard <= L + 1 && y >= 0; ++guard) { bits |= 1ull << y; y = m.par_out[y]; }
+    } else {
+      p.tokens[o] = -1; p.parents[o] = -1; p.depth[o] = -1;
+      if (p.scores) p.scores[o] = -INFINITY;
+    }
+    s_bits[x] = bits;
+  }
+  if (tid == 0) p.n_nodes[b] = 1 + n_sel;
+  __syncthreads();
+  uint8_t* mbase = p.mask + (size_t)b * budget * budget;
+  for (int e = tid; e < budget * budget; e += nthr) {
+    const int x = e / budget, y = e - x * budget;
+    mbase[e] = (uint8_t)((s_bits[x] >> y) & 1ull);
+  }
+#ifdef DART_TREE_TL
+  TL_STAMP();
+  __syncthreads();
+  if (tid == 0 && p.scores)
+  {
+    for (int e = 0; e < n_tl && e < 40 && 1 + e < budget; ++e) p.scores[(size_t)b * budget + 1 + e] = (float)s_tl[e];
+    for (int e = 0; e < 8 && 45 + e < budget; ++e) p.scores[(size_t)b * budget + 45 + e] = (float)g_sel_tl[e];
+  }
+#endif
+#undef TL_STAMP
+}
+
 // Verification inputs of one tree per block: thread x owns slot x (budget <= 64 threads' worth of slots).
 __global__ void __launch_bounds__(64) verify_inputs_kernel(int budget, int max_levels, const int32_t* parents, const int32_t* depth,
                                                            const int32_t* n_nodes, const int32_t* root_pos, int32_t* position_ids,
@@ -481,42 +714,60 @@ cudaError_t launch_verify_inputs(int B, int budget, int max_levels, const int32_
 size_t tree_smem_bytes(int topk, int beam, int budget, int n_levels) {
   return tree_layout(topk, beam, budget, n_levels, nullptr, nullptr) + 16;
 }
+// The hash-layout kernel stages the score table's slices in shared memory when they fit beside the nodes.
+constexpr size_t kTreeSmemMax = 200 * 1024;
+static bool hash_tree_stages(int topk, int beam, int budget, int n_levels) {
+  return hash_tree_layout(topk, beam, budget, n_levels, true, nullptr, nullptr) + 16 <= kTreeSmemMax;
+}
+static size_t hash_tree_smem_bytes(int topk, int beam, int budget, int n_levels) {
+  return hash_tree_layout(topk, beam, budget, n_levels, hash_tree_stages(topk, beam, budget, n_levels), nullptr, nullptr) + 16;
+}
 
 cudaError_t tree_setup(int topk, int beam, int budget, int max_levels) {
-  const size_t smem = tree_smem_bytes(topk, beam, budget, max_levels);
-  if (smem > 48 * 1024)
-  {
-    cudaError_t e = cudaFuncSetAttribute(tree_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<1024, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  size_t smem = tree_smem_bytes(topk, beam, budget, max_levels);
+  cudaError_t e = cudaSuccess;
+  if (smem > 48 * 1024) {
+    e = cudaFuncSetAttribute(tree_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<1024, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    return e;
   }
-  return cudaSuccess;
+  smem = hash_tree_smem_bytes(topk, beam, budget, max_levels);
+  if (e == cudaSuccess && smem > 48 * 1024) {
+    e = cudaFuncSetAttribute(tree_hash_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<1024, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<1024, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  }
+  return e;
 }
 
 cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
   const bool trie = p.trie.bi_off != nullptr;
-  {
-    const int n_bg = sweep_bigrams(p.topk, p.n_levels);
-    const int n_task = p.n_levels * 2 * p.topk;   // trie layout: one warp per (level, list kind, context position)
-    cudaError_t e = trie ? launch_pdl(trie_sweep_kernel, dim3((n_task + 7) / 8, p.B), dim3(256), 0, st, p)
-                         : launch_pdl(bigram_sweep_kernel, dim3((n_bg + 255) / 256, p.B), dim3(256), 0, st, p);
-    if (e != cudaSuccess) return e;
-  }
-  const size_t smem = tree_smem_bytes(p.topk, p.beam, p.budget, p.n_levels);
   // one thread per (beam entry, candidate) pair; a smaller block makes every barrier cheaper
   int need = p.beam * p.topk;
   if (p.budget > need) need = p.budget;
+  if (need < 64) need = 64;
   if (trie && 32 * p.beam > need) need = 32 * p.beam;   // one warp per beam entry reads its context's children
   int threads = (need + 31) / 32 * 32;
   if (threads > 1024) threads = 1024;
   if (trie) {
+    const int n_task = p.n_levels * 2 * p.topk;   // one warp per (level, list kind, context position)
+    const cudaError_t e = launch_pdl(trie_sweep_kernel, dim3((n_task + 7) / 8, p.B), dim3(256), 0, st, p);
+    if (e != cudaSuccess) return e;
+    const size_t smem = tree_smem_bytes(p.topk, p.beam, p.budget, p.n_levels);
     if (threads <= 512) return launch_pdl(tree_kernel<512, true>, dim3(p.B), dim3(threads), smem, st, p);
     return launch_pdl(tree_kernel<1024, true>, dim3(p.B), dim3(threads), smem, st, p);
   }
-  if (threads <= 512) return launch_pdl(tree_kernel<512, false>, dim3(p.B), dim3(threads), smem, st, p);
-  return launch_pdl(tree_kernel<1024, false>, dim3(p.B), dim3(threads), smem, st, p);
+  const int k = p.topk, n_sg = k + k * k + (p.n_levels > 2 ? (p.n_levels - 2) * k * k * k : 0);
+  const cudaError_t e = launch_pdl(ngram_sweep_kernel, dim3((n_sg + 255) / 256, p.B), dim3(256), 0, st, p);
+  if (e != cudaSuccess) return e;
+  const bool stage = hash_tree_stages(p.topk, p.beam, p.budget, p.n_levels);
+  const size_t smem = hash_tree_layout(p.topk, p.beam, p.budget, p.n_levels, stage, nullptr, nullptr) + 16;
+  if (stage) {
+    if (threads <= 512) return launch_pdl(tree_hash_kernel<512, true>, dim3(p.B), dim3(threads), smem, st, p);
+    return launch_pdl(tree_hash_kernel<1024, true>, dim3(p.B), dim3(threads), smem, st, p);
+  }
+  if (threads <= 512) return launch_pdl(tree_hash_kernel<512, false>, dim3(p.B), dim3(threads), smem, st, p);
+  return launch_pdl(tree_hash_kernel<1024, false>, dim3(p.B), dim3(threads), smem, st, p);
 }
 
 }  // namespace dart

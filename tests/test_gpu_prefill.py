@@ -20,7 +20,7 @@ CASES = {
     # the path the benchmark times: 4300 packed rows = two passes (the second sequence straddles the 4096-row pass
     # boundary), 33 token tiles x 10 feature tiles = 330 jobs of the feature FC for 148 persistent CTAs (every CTA
     # takes a second and a third tile: both accumulator buffers and their hand-over), 256 jobs of the k / v projection
-    "three_seqs_two_passes": (syn.small_variant(C1, batch=3, prefix=2300, hidden=2560, n_q_heads=20, n_kv_heads=8, head_dim=128,
+    "three_seqs_two_passes": (syn.small_variant(C1, batch=3, prefix=2300, hidden=2560, n_q_heads=16, n_kv_heads=8, head_dim=128,
                                                 mlp_inter=1376, vocab=4112, K=8, tree_budget=60), [3, 10, 0], [2100, 2050, 150]),
 }
 
