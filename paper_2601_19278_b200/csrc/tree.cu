@@ -460,7 +460,7 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
 // The tree kernel of the hash layout: Algorithm 1 over the dense score table of ngram_sweep_kernel.
 // ------------------------------------------------------------------------------------------------------
 struct HashTreeSmem {
-  float* n_score; float* n_clamp; int* n_tok; int* n_par;   // per node (the root is node 0)
+  float* n_score; float* n_clamp; int* n_tok; int* n_par; unsigned char* n_j;   // per node (the root is node 0); n_j: its candidate index
   int* c_ids; float* c_sl;                         // [L][k] the candidates' ids and s_logit, staged once
   int* b_node; float* b_sc; float* b_cl; int* b_row;   // per beam entry: node, score, clamped score, row of its context in the level's slice
   Key* lvl_sorted;                                 // [2][64] best of a level by clamped score (the running best lags one level behind)
@@ -474,6 +474,7 @@ __host__ __device__ inline size_t hash_tree_layout(int k, int w, int budget, int
   size_t o = 0;
   auto take = [&](size_t bytes) { const size_t r = o; o += (bytes + 15) & ~size_t(15); return r; };
   const size_t o_sc = take((size_t)n_max * 4), o_cl = take((size_t)n_max * 4), o_tok = take((size_t)n_max * 4), o_par = take((size_t)n_max * 4),
+               o_nj = take((size_t)n_max),
                o_ci = take((size_t)L * k * 4), o_cs = take((size_t)L * k * 4),
                o_bn = take((size_t)w * 4), o_bs = take((size_t)w * 4), o_bc = take((size_t)w * 4), o_br = take((size_t)w * 4),
                o_ls = take(2 * 64 * 8), o_sel = take((size_t)(budget + 1) * 4), o_po = take((size_t)budget * 4),
@@ -482,7 +483,7 @@ __host__ __device__ inline size_t hash_tree_layout(int k, int w, int budget, int
   if (t != nullptr) {
     t->n_score = reinterpret_cast<float*>(base + o_sc);
     t->n_clamp = reinterpret_cast<float*>(base + o_cl); t->n_tok = reinterpret_cast<int*>(base + o_tok);
-    t->n_par = reinterpret_cast<int*>(base + o_par);
+    t->n_par = reinterpret_cast<int*>(base + o_par); t->n_j = base + o_nj;
     t->c_ids = reinterpret_cast<int*>(base + o_ci); t->c_sl = reinterpret_cast<float*>(base + o_cs);
     t->b_node = reinterpret_cast<int*>(base + o_bn); t->b_sc = reinterpret_cast<float*>(base + o_bs);
     t->b_cl = reinterpret_cast<float*>(base + o_bc); t->b_row = reinterpret_cast<int*>(base + o_br);
@@ -511,6 +512,12 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
   const int k = p.topk, w = p.beam, theta = p.budget - 1;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x, last_warp = (nthr >> 5) - 1;
   const int fr = p.first_rows[b], L = min(p.n_levels, p.K - fr);   // this sequence's level 0 row and levels
+  // When the block has a warp beyond the candidates (the launch adds one where 1024 threads allow it), that warp takes
+  // no part in the selection: it keeps the running best 64, merging one level behind while the others select.
+  const bool spare = w * k <= nthr - 32 && p.budget <= nthr - 32 && nthr >= 128;
+  const bool idle = spare && warp == last_warp;
+  const int n_active = spare ? nthr - 32 : nthr;
+  const int my_rho = tid / k, my_j = tid - my_rho * k;              // this thread's (beam entry, candidate) pair at every level
   HashTreeSmem m;
   hash_tree_layout(k, w, p.budget, p.n_levels, STAGE, tsm, &m);
   __shared__ unsigned long long s_bits[64];
@@ -524,7 +531,7 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
 #define TL_STAMP() do {} while (0)
 #endif
 
-  if (tid == 0) { m.n_score[0] = 0.f; m.n_clamp[0] = INFINITY; m.n_par[0] = -1; m.b_node[0] = 0; m.b_sc[0] = 0.f; m.b_cl[0] = INFINITY; m.b_row[0] = 0; m.lvl_base[0] = 1; }
+  if (tid == 0) { m.n_score[0] = 0.f; m.n_clamp[0] = INFINITY; m.n_par[0] = -1; m.n_j[0] = 0; m.b_node[0] = 0; m.b_sc[0] = 0.f; m.b_cl[0] = INFINITY; m.b_row[0] = 0; m.lvl_base[0] = 1; }
   pdl_wait();
   TL_STAMP();
   const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
@@ -548,7 +555,7 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
     const int base = m.lvl_base[i];
     float s = -INFINITY, cl = -INFINITY;
     if (tid < ncand) {
-      const int rho = tid / k, j = tid - rho * k;
+      const int rho = my_rho, j = my_j;
       const int t = m.c_ids[i * k + j];
       const int at = m.b_row[rho] + j;
       float s_ng;
@@ -559,37 +566,40 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
       const float pc = m.b_cl[rho];
       cl = s < pc ? s : pc;
       const int n = base + tid;
-      m.n_score[n] = s; m.n_clamp[n] = cl; m.n_tok[n] = t; m.n_par[n] = m.b_node[rho];
+      m.n_score[n] = s; m.n_clamp[n] = cl; m.n_tok[n] = t; m.n_par[n] = m.b_node[rho]; m.n_j[n] = (unsigned char)j;
     }
     // keys carry the node index base + tid, which orders candidates of one level like tid does
     // best 64 by score -> next beam; `differs`: some clamped score is not its score (never, when increments <= 0)
     TL_STAMP();
     const bool more = STAGE && (i == 0 ? L > 2 : (i >= 2 && i + 1 < L));   // a slice to fetch while this level is selected
     const int nb_next = ncand < w ? ncand : w;
-    const int pbase = i > 0 ? m.lvl_base[i - 1] : 0;
     Key* lvl_out = m.lvl_sorted + (i & 1) * 64;
     const int differs = block_select64(
-        tid < ncand ? make_key(s, base + tid) : kPadKey, s, tid < ncand && cl != s, m.ss,
+        tid < ncand ? make_key(s, base + tid) : kPadKey, s, tid < ncand && cl != s, idle, n_active, m.ss,
         [&](int r, Key key, int any) {
           if (!any) lvl_out[r] = key;
           if (r < nb_next) {
             // beam entry r of the next level: its node, scores and the row of its context -- (the parent's candidate
             // index, this node's candidate index) -- in the next level's slice of the score table
-            const int node = key_index(key), j = (node - base) % k;
+            const int node = key_index(key), j = m.n_j[node];
             m.b_node[r] = node;
             m.b_sc[r] = m.n_score[node];
             m.b_cl[r] = m.n_clamp[node];
-            m.b_row[r] = (i == 0 ? j : ((m.n_par[node] - pbase) % k) * k + j) * k;
+            m.b_row[r] = (i == 0 ? j : (int)m.n_j[m.n_par[node]] * k + j) * k;
           }
         },
         [&]() {
           // every thread has read what it needs of level i's slice: the next one may overwrite it (levels 0 and 1 use
           // the small table, so level 2's slice is fetched during level 0 and nothing during level 1)
           if (more) copy_async16(m.slice, sg + g.o2 + (i == 0 ? 0 : i - 1) * g.st3, g.st3 / 4);
+          if (idle && i > 0) {   // the spare warp: the running best takes in the previous level's best 64
+            const Key* q = m.lvl_sorted + ((i - 1) & 1) * 64;
+            merge_keep64(g0, g1, q[lane], q[32 + lane], lane);
+          }
         },
         [&]() {
-          // the running best takes in the previous level's best 64 while the first warps rank this level's survivors
-          if (warp == last_warp && i > 0) {
+          // without a spare warp the last warp does that while the first warps rank this level's survivors
+          if (!spare && warp == last_warp && i > 0) {
             const Key* q = m.lvl_sorted + ((i - 1) & 1) * 64;
             merge_keep64(g0, g1, q[lane], q[32 + lane], lane);
           }
@@ -597,7 +607,7 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
           if (STAGE && i >= 1) asm volatile("cp.async.wait_all;" ::: "memory");   // the next level's slice has landed
         });
     if (differs)   // the level's best 64 by clamped score are a different set: select again
-      block_select64(tid < ncand ? make_key(cl, base + tid) : kPadKey, cl, 0, m.ss, [&](int r, Key key, int) { lvl_out[r] = key; }, [] {}, [] {});
+      block_select64(tid < ncand ? make_key(cl, base + tid) : kPadKey, cl, 0, idle, n_active, m.ss, [&](int r, Key key, int) { lvl_out[r] = key; }, [] {}, [] {});
     TL_STAMP();
     nb = nb_next;
   }
@@ -606,22 +616,18 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
     merge_keep64(g0, g1, q[lane], q[32 + lane], lane);
   }
 
-  // ---- the selected nodes: the first n_sel entries of the running best 64
+  // ---- the selected nodes: the first n_sel entries of the running best 64; slot_of: node -> output slot
   const int total = m.lvl_base[L] - 1;
   const int n_sel = total < theta ? total : theta;
+  int* slot_of = reinterpret_cast<int*>(m.n_score);   // the scores are no longer needed
   if (warp == last_warp) {
-    if (lane < n_sel) m.sel[1 + lane] = key_index(g0);
-    if (32 + lane < n_sel) m.sel[33 + lane] = key_index(g1);
-    if (lane == 0) m.sel[0] = 0;
+    if (lane < n_sel) { const int n = key_index(g0); m.sel[1 + lane] = n; slot_of[n] = 1 + lane; }
+    if (32 + lane < n_sel) { const int n = key_index(g1); m.sel[33 + lane] = n; slot_of[n] = 33 + lane; }
+    if (lane == 0) { m.sel[0] = 0; slot_of[0] = 0; }
   }
   __syncthreads();
-
-  // ---- outputs
-  const int budget = p.budget;
-  int* slot_of = reinterpret_cast<int*>(m.n_score);   // node -> output slot (the scores are no longer needed)
-  for (int x = tid; x <= n_sel; x += nthr) slot_of[m.sel[x]] = x;
-  __syncthreads();
   // the selection is closed under "parent of" (clamped scores never rise along a path), so every parent has a slot
+  const int budget = p.budget;
   for (int x = tid; x < budget; x += nthr) m.par_out[x] = (x >= 1 && x <= n_sel) ? slot_of[m.n_par[m.sel[x]]] : -1;
   __syncthreads();
   for (int x = tid; x < budget; x += nthr) {
@@ -629,17 +635,12 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
     unsigned long long bits = 0ull;
     if (x <= n_sel) {
       const int n = m.sel[x];
-      int lev = 0;
-      if (x > 0) {
-        while (n >= m.lvl_base[lev + 1]) ++lev;
-        lev += 1;
-      }
-      p.tokens[o] = m.n_tok[n];
-      p.parents[o] = m.par_out[x];
-      p.depth[o] = lev;
-      if (p.scores) p.scores[o] = x == 0 ? 0.f : m.n_clamp[n];
       int y = x;
       for (int guard = 0; guard <= L + 1 && y >= 0; ++guard) { bits |= 1ull << y; y = m.par_out[y]; }
+      p.tokens[o] = m.n_tok[n];
+      p.parents[o] = m.par_out[x];
+      p.depth[o] = __popcll(bits) - 1;                 // a node's depth = its ancestors, the root (depth 0) among them
+      if (p.scores) p.scores[o] = x == 0 ? 0.f : m.n_clamp[n];
     } else {
       p.tokens[o] = -1; p.parents[o] = -1; p.depth[o] = -1;
       if (p.scores) p.scores[o] = -INFINITY;
@@ -649,9 +650,9 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
   if (tid == 0) p.n_nodes[b] = 1 + n_sel;
   __syncthreads();
   uint8_t* mbase = p.mask + (size_t)b * budget * budget;
-  for (int e = tid; e < budget * budget; e += nthr) {
-    const int x = e / budget, y = e - x * budget;
-    mbase[e] = (uint8_t)((s_bits[x] >> y) & 1ull);
+  for (int x = warp; x < budget; x += nthr >> 5) {      // a warp per row of the mask
+    const unsigned long long bits = s_bits[x];
+    for (int y = lane; y < budget; y += 32) mbase[x * budget + y] = (uint8_t)((bits >> y) & 1ull);
   }
 #ifdef DART_TREE_TL
   TL_STAMP();
@@ -659,7 +660,7 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
   if (tid == 0 && p.scores)
   {
     for (int e = 0; e < n_tl && e < 40 && 1 + e < budget; ++e) p.scores[(size_t)b * budget + 1 + e] = (float)s_tl[e];
-    for (int e = 0; e < 8 && 45 + e < budget; ++e) p.scores[(size_t)b * budget + 45 + e] = (float)g_sel_tl[e];
+    for (int e = 0; e < 11 && 45 + e < budget; ++e) p.scores[(size_t)b * budget + 45 + e] = (float)g_sel_tl[e];
   }
 #endif
 #undef TL_STAMP
@@ -732,9 +733,9 @@ cudaError_t tree_setup(int topk, int beam, int budget, int max_levels) {
   }
   smem = hash_tree_smem_bytes(topk, beam, budget, max_levels);
   if (e == cudaSuccess && smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(tree_hash_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(tree_hash_kernel<576, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<1024, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<576, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<1024, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   }
   return e;
@@ -749,6 +750,7 @@ cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
   if (trie && 32 * p.beam > need) need = 32 * p.beam;   // one warp per beam entry reads its context's children
   int threads = (need + 31) / 32 * 32;
   if (threads > 1024) threads = 1024;
+  if (!trie && threads + 32 <= 1024) threads += 32;     // a spare warp that keeps the running best (see tree_hash_kernel)
   if (trie) {
     const int n_task = p.n_levels * 2 * p.topk;   // one warp per (level, list kind, context position)
     const cudaError_t e = launch_pdl(trie_sweep_kernel, dim3((n_task + 7) / 8, p.B), dim3(256), 0, st, p);
@@ -763,10 +765,10 @@ cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
   const bool stage = hash_tree_stages(p.topk, p.beam, p.budget, p.n_levels);
   const size_t smem = hash_tree_layout(p.topk, p.beam, p.budget, p.n_levels, stage, nullptr, nullptr) + 16;
   if (stage) {
-    if (threads <= 512) return launch_pdl(tree_hash_kernel<512, true>, dim3(p.B), dim3(threads), smem, st, p);
+    if (threads <= 576) return launch_pdl(tree_hash_kernel<576, true>, dim3(p.B), dim3(threads), smem, st, p);
     return launch_pdl(tree_hash_kernel<1024, true>, dim3(p.B), dim3(threads), smem, st, p);
   }
-  if (threads <= 512) return launch_pdl(tree_hash_kernel<512, false>, dim3(p.B), dim3(threads), smem, st, p);
+  if (threads <= 576) return launch_pdl(tree_hash_kernel<576, false>, dim3(p.B), dim3(threads), smem, st, p);
   return launch_pdl(tree_hash_kernel<1024, false>, dim3(p.B), dim3(threads), smem, st, p);
 }
 
