@@ -160,10 +160,12 @@ void make_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int gri
     if (u0 >= u1) continue;
     const int t0 = (int)(u0 / p.KR), t1 = (int)((u1 - 1) / p.KR);
     for (int t = t0; t <= t1; ++t) {
-      ph.expected[pair_offset > 0 ? t % pair_offset : t] += 1;
+      // t counts tiles in unit order: paired tiles alternate (T, T + pair_offset, T + 1, ...), see umma_gemm.cu
+      const int T = pair_offset > 0 ? (t & 1) * pair_offset + (t >> 1) : t;
+      ph.expected[pair_offset > 0 ? t >> 1 : t] += 1;
       for (int j = 0; j < 8; ++j) {
-        int& n = ph.meta[(size_t)(t * 8 + j) * kMetaStride];
-        if (n < kMetaStride - 1) ph.meta[(size_t)(t * 8 + j) * kMetaStride + 1 + n++] = (c * p.slots + (t - t0)) * 8 + j;
+        int& n = ph.meta[(size_t)(T * 8 + j) * kMetaStride];
+        if (n < kMetaStride - 1) ph.meta[(size_t)(T * 8 + j) * kMetaStride + 1 + n++] = (c * p.slots + (t - t0)) * 8 + j;
       }
     }
   }

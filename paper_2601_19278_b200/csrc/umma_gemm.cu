@@ -40,17 +40,26 @@ struct UmmaCfg {
 
 // Position of unit u = tile * KB + kb of the launch, advanced one unit at a time (the single producer
 // thread sits on the critical path of every stage, so it does no divisions in its loop).
+// With paired tiles (pair_offset > 0: QKV's g- and e-halves, gate and up) the units run over the tiles in the order
+// T, T + pair_offset, T + 1, T + 1 + pair_offset, ...: the two tiles of a group are streamed back to back, so a group is
+// complete where its 2 * KR consecutive units end, the groups' ends are spread evenly over the CTAs and no CTA finalizes
+// two groups in a row (in plain tile order every group ended in the second half of the CTAs).
+__host__ __device__ inline int actual_tile(int v, int pair_offset) { return pair_offset > 0 ? (v & 1) * pair_offset + (v >> 1) : v; }
+__host__ __device__ inline int group_of_unit_tile(int v, int pair_offset) { return pair_offset > 0 ? v >> 1 : v; }
+
 struct UnitPos {
-  int tile, kb, seg, row0, xoff;
+  int tile, kb, seg, row0, xoff, po;   // tile: position in unit order (see actual_tile)
   __device__ __forceinline__ void locate(const StreamArgs& a) {
+    const int T = actual_tile(tile, po);
     seg = 0;
 #pragma unroll
     for (int i = 1; i < 6; ++i)
-      if (i < a.nseg && tile >= a.seg[i].tile0) seg = i;
-    row0 = (tile - a.seg[seg].tile0) * 128;
+      if (i < a.nseg && T >= a.seg[i].tile0) seg = i;
+    row0 = (T - a.seg[seg].tile0) * 128;
     xoff = a.seg[seg].xoff;
   }
-  __device__ __forceinline__ void set(const StreamArgs& a, long long u) {
+  __device__ __forceinline__ void set(const StreamArgs& a, long long u, int pair_offset) {
+    po = pair_offset;
     tile = (int)(u / a.KR);
     kb = (int)(u - (long long)tile * a.KR);
     locate(a);
@@ -94,7 +103,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
     const int pre = n < C::Stages ? n : C::Stages;
     const uint64_t wpol = l2_policy_evict_first();
     UnitPos q;
-    if (n > 0) q.set(p.s, u0);
+    if (n > 0) q.set(p.s, u0, p.pair_offset);
     for (int it = 0; it < pre; ++it, q.next(p.s)) {
       mbar_expect_tx(&full[it], C::StageBytes);
       tma_load_2d_hint(ring + (size_t)it * C::StageBytes, &a.mapW[q.seg], &full[it], q.kb * 64, q.row0, wpol);
@@ -109,8 +118,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
   int cand[kMetaSlots] = {-1, -1};  // groups whose piece tables sit in s_meta
   if (u0 < u1) {
     const int t0 = (int)(u0 / KB), t1 = (int)((u1 - 1) / KB);
-    cand[0] = p.pair_offset > 0 ? t0 % p.pair_offset : t0;
-    cand[1] = p.pair_offset > 0 ? t1 % p.pair_offset : t1;
+    cand[0] = group_of_unit_tile(t0, p.pair_offset);
+    cand[1] = group_of_unit_tile(t1, p.pair_offset);
     meta_prefetch(p, cand[0], &s_meta[0]);
     if (cand[1] != cand[0]) meta_prefetch(p, cand[1], &s_meta[1]);
   }
@@ -126,7 +135,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
     const uint64_t wpol = l2_policy_evict_first();
     UnitPos q;
     pdl_wait();
-    q.set(p.s, u0);
+    q.set(p.s, u0, p.pair_offset);
     for (int it = 0; it < pre; ++it, q.next(p.s)) {
       uint8_t* xs = ring + (size_t)it * C::StageBytes + kWBytes;
       if (a.has_lo) tma_load_3d(xs, &a.mapXhi, &full[it], q.xoff + q.kb * 64, 0, 0);
@@ -220,7 +229,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       __syncwarp();
       if (lane == 0 && atomicAdd(&s_cnt[visit & 3], 1) == 3) {
         s_cnt[visit & 3] = 0;
-        const int group = p.pair_offset > 0 ? tile % p.pair_offset : tile;
+        const int group = group_of_unit_tile(tile, p.pair_offset);
         if (atomicAdd(&p.ctr[group], 1) + 1 == p.expected[group]) {
           __threadfence();  // acquire: the other CTAs' pieces are visible to whatever follows the next barrier
           s_done[++s_done[0]] = group;
