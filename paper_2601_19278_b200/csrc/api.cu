@@ -74,6 +74,7 @@ struct dart_handle {
   const void* attn_v_ptr = nullptr;
   int h_tiles = 0;         // 128-row tiles of a hidden-sized row
   Workspace ws;
+  void* ng_base = nullptr;       // the hash layout's allocation: fingerprint words, then slots
   NgramSlot* ng_slots = nullptr;
   uint32_t ng_mask = 0, ng_max_probe = 0;
   NgramTrieOwned ng_trie{};     // the child-list layout (ngram_layout = DART_NGRAM_TRIE)
@@ -470,31 +471,49 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
                                 cfg->ngram_order, &h->ng_trie));
     h->ng_bytes = h->ng_trie.bytes;
   } else if (n_rows > 0) {
-    // open-addressing table: linear probing, load <= 0.5
+    // open addressing over buckets of eight rows (NgramTable in kernels.h), linear probing over buckets, load <= 0.5
     size_t cap = 16;
     while (cap < (size_t)(2 * n_rows)) cap <<= 1;
     if (cap > (1ull << 31)) { dart_draft_destroy(h); return DART_ERR_INVALID_ARG; }
+    const size_t n_buckets = cap / 8;
     std::vector<NgramSlot> tab(cap);
+    std::vector<uint16_t> fps(cap, 0);
     memset(tab.data(), 0, cap * sizeof(NgramSlot));
-    const uint32_t mask = (uint32_t)(cap - 1);
+    const uint32_t mask = (uint32_t)(n_buckets - 1);
     uint32_t max_probe = 0;
     for (long long i = 0; i < n_rows; ++i) {
       const int ord = ngram->order[i];
       const int c0 = ngram->ctx0[i], c1 = ngram->ctx1[i], nx = ngram->next[i];
       if (ord == 3 && cfg->ngram_order < 3) continue;
-      const unsigned long long key = ngram_key(ord, c0, c1, nx);
-      uint32_t pos = (uint32_t)ngram_hash(key) & mask, d = 0;
-      while (tab[pos].key != 0ull && tab[pos].key != key) { pos = (pos + 1) & mask; ++d; }
-      if (tab[pos].key == key) continue;
-      tab[pos].key = key;
-      tab[pos].score = ngram->score[i];
-      if (d > max_probe) max_probe = d;
+      const unsigned long long key = ngram_key(ord, c0, c1, nx), hh = ngram_hash(key);
+      const uint16_t f = (uint16_t)ngram_fingerprint(hh);
+      uint32_t pos = (uint32_t)hh & mask, d = 0;
+      for (;; pos = (pos + 1) & mask, ++d) {
+        int slot = -1;
+        bool dup = false;
+        for (int q = 0; q < 8 && slot < 0 && !dup; ++q) {
+          if (fps[(size_t)pos * 8 + q] == 0) slot = q;                       // slots of a bucket fill in order: none is used after an empty one
+          else if (tab[(size_t)pos * 8 + q].key == key) dup = true;          // of duplicate rows the first wins
+        }
+        if (dup) break;
+        if (slot >= 0) {
+          tab[(size_t)pos * 8 + slot].key = key;
+          tab[(size_t)pos * 8 + slot].score = ngram->score[i];
+          fps[(size_t)pos * 8 + slot] = f;
+          if (d > max_probe) max_probe = d;
+          break;
+        }
+      }
     }
-    INIT_CHECK(cudaMalloc(&h->ng_slots, cap * sizeof(NgramSlot)));
-    INIT_CHECK(cudaMemcpy(h->ng_slots, tab.data(), cap * sizeof(NgramSlot), cudaMemcpyHostToDevice));
+    // one allocation: the fingerprint words first (16 bytes per bucket), then the slots
+    const size_t fp_bytes = align_up(n_buckets * 16, 256);
+    INIT_CHECK(cudaMalloc(&h->ng_base, fp_bytes + cap * sizeof(NgramSlot)));
+    INIT_CHECK(cudaMemcpy(h->ng_base, fps.data(), n_buckets * 16, cudaMemcpyHostToDevice));
+    INIT_CHECK(cudaMemcpy(static_cast<char*>(h->ng_base) + fp_bytes, tab.data(), cap * sizeof(NgramSlot), cudaMemcpyHostToDevice));
+    h->ng_slots = reinterpret_cast<NgramSlot*>(static_cast<char*>(h->ng_base) + fp_bytes);
     h->ng_mask = mask;
     h->ng_max_probe = max_probe;
-    h->ng_bytes = cap * sizeof(NgramSlot);
+    h->ng_bytes = fp_bytes + cap * sizeof(NgramSlot);
   }
 
   INIT_CHECK(topk_merge_setup(2 * n_sm));
@@ -510,7 +529,7 @@ int dart_draft_destroy(dart_handle* h) {
   if (h == nullptr) return DART_OK;
   for (void* p : h->owned) cudaFree(p);
   if (h->ws.base) cudaFree(h->ws.base);
-  if (h->ng_slots) cudaFree(h->ng_slots);
+  if (h->ng_base) cudaFree(h->ng_base);
   ngram_trie_free(&h->ng_trie);
   delete h;
   return DART_OK;
@@ -867,7 +886,7 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
     tp.first_rows[b] = (unsigned char)fr;
   }
   tp.ids = in->topk_ids; tp.slogit = in->topk_slogit; tp.ctx_tail = in->ctx_tail;
-  tp.table.slots = h->ng_slots; tp.table.mask = h->ng_mask; tp.table.max_probe = h->ng_max_probe;
+  tp.table.fp = static_cast<const uint4*>(h->ng_base); tp.table.slots = h->ng_slots; tp.table.mask = h->ng_mask; tp.table.max_probe = h->ng_max_probe;
   for (int i = 0; i < 8; ++i) { tp.wl[i] = h->wl[i]; tp.wv[i] = h->wv[i]; }
   tp.trie.bi_off = h->ng_trie.bi_off; tp.trie.bi_ent = h->ng_trie.bi_ent; tp.trie.tri_off = h->ng_trie.tri_off;
   tp.trie.tri_node = h->ng_trie.tri_node; tp.trie.tri_ent = h->ng_trie.tri_ent; tp.trie.nb8 = 8u * (uint32_t)((c.vocab + 479) / 480);

@@ -299,8 +299,20 @@ cudaError_t launch_train_attn(const TrainAttnArgs& a, cudaStream_t st);
 // ---------------------------------------------------------------------------------------------
 // N-gram hash table + tree pruning.
 // ---------------------------------------------------------------------------------------------
-struct NgramSlot { unsigned long long key; float score; uint32_t pad; };  // 16 bytes; key 0 = empty
-struct NgramTable { const NgramSlot* slots; uint32_t mask; uint32_t max_probe; };
+// Open addressing over buckets of eight rows.  A row lives in the bucket its key hashes to, or -- when that one was
+// full at build time -- in the next bucket with room (linear probing over buckets, the longest displacement recorded
+// as max_probe).  Per bucket there are eight 16-bit fingerprints of the keys in one 16-byte word (0 = empty slot) and,
+// in a second array, the eight {key, score} slots.  A lookup reads the fingerprint word -- ONE 16-byte request -- and a
+// slot only where a fingerprint matches: a miss ends at a word with an empty slot and no match, one request in all.
+// (The sweep makes ~10^5 lookups per tree, every lane of a warp in another line of the table: what bounds it is the
+// number of such scattered requests an SM can issue, not their latency.  Four requests per lookup -- a bucket's eight
+// full keys -- took 5.2 us per round of lookups; probing 16-byte slots one after the other took as long.)
+struct NgramSlot { unsigned long long key; float score; uint32_t pad; };  // 16 bytes
+struct NgramTable { const uint4* fp; const NgramSlot* slots; uint32_t mask; uint32_t max_probe; };   // mask: buckets - 1
+__host__ __device__ inline uint32_t ngram_fingerprint(unsigned long long hash) {
+  const uint32_t f = (uint32_t)(hash >> 48);
+  return f == 0u ? 1u : f;     // 0 marks an empty slot
+}
 // The same rows as child lists (Appendix C).  Every list is a run of {key, payload} slots in ascending key order:
 //   2-gram context b   -> bi_ent[bi_off[b] .. bi_off[b+1])             {next token, score bits}
 //   first token a      -> tri_node[tri_off[a] .. tri_off[a+1])         {second context token b, first child}, then a

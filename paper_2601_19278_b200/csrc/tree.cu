@@ -27,25 +27,6 @@
 
 namespace dart {
 
-__device__ __forceinline__ NgramSlot load_slot(const NgramSlot* p) {
-  const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
-  NgramSlot s;
-  s.key = ((unsigned long long)v.y << 32) | v.x;
-  s.score = __uint_as_float(v.z);
-  s.pad = v.w;
-  return s;
-}
-
-// Finish a lookup whose first slot has been loaded: follow the probe sequence (bounded).
-__device__ __forceinline__ bool probe_rest(const NgramTable& T, unsigned long long key, uint32_t h, NgramSlot s, float& score) {
-  for (uint32_t i = 0; i <= T.max_probe; ++i) {
-    if (s.key == key) { score = s.score; return true; }
-    if (s.key == 0ull) return false;
-    s = load_slot(T.slots + ((h + i + 1) & T.mask));
-  }
-  return false;
-}
-
 // The entry of token t in a long list (region ent[lo ..), nb8 bitmap slots first): read t's 64-byte bitmap block,
 // test its bit, count the entries before it, read the entry -- two dependent reads whatever the list's length.
 __device__ __forceinline__ bool long_find(const uint2* __restrict__ ent, uint32_t lo, uint32_t nb8, int t, uint32_t& payload, uint32_t& index) {
@@ -170,60 +151,108 @@ __host__ __device__ inline size_t tree_layout(int k, int w, int budget, int L, u
   return o;
 }
 
-// ---- dense N-gram score table of one sequence (hash layout), written by ngram_sweep_kernel ----
-//   level 0          sg[j]                                   context (c_-2, c_-1),           candidate S_0[j]
-//   level 1          sg[o1 + j' k + j]                       context (c_-1, S_0[j']),        candidate S_1[j]
-//   level i >= 2     sg[o2 + (i-2) st3 + (j'' k + j') k + j] context (S_{i-2}[j''], S_{i-1}[j']), candidate S_i[j]
-// Offsets and strides are multiples of four floats so that slices can be copied with 16-byte cp.async.
-struct SgLayout { int o1, o2, st3, total; };
+// ---- dense N-gram score tables of one sequence (hash layout), written by the sweep ----
+//   bg0  [j]                           2-gram (c_-1, S_0[j])
+//   t0   [j]                           3-gram (c_-2, c_-1, S_0[j])
+//   bg   [(i-1) k^2 + j' k + j]        2-gram (S_{i-1}[j'], S_i[j]), levels i >= 1
+//   t1   [j' k + j]                    3-gram (c_-1, S_0[j'], S_1[j])
+//   t3   [(i-2) st3 + (j'' k + j') k + j]   3-gram (S_{i-2}[j''], S_{i-1}[j'], S_i[j]), levels i >= 2: one slice per level
+// A 2-gram entry holds the row's score or log(eps); a 3-gram entry the row's score or kNoRow, in which case the
+// candidate's s_ng is its 2-gram entry (Algorithm 1 line 9 with Appendix C's back-off).  Offsets and strides are
+// multiples of four floats so that tables can be copied with 16-byte cp.async; everything before t3 ("the small
+// tables", 20 KB at k = 25 and 8 levels) is staged in shared memory once, t3 one slice at a time.
+constexpr uint32_t kNoRowBits = 0x7fc00000u;   // a NaN: no score is one
+struct SgLayout { int t0, bg, t1, small, st3, total; };
 __host__ __device__ inline SgLayout sg_layout(int k, int levels) {
   SgLayout g;
-  g.o1 = (k + 3) & ~3;
-  g.o2 = (g.o1 + k * k + 3) & ~3;
+  g.t0 = (k + 3) & ~3;
+  g.bg = (g.t0 + k + 3) & ~3;
+  g.t1 = (g.bg + (levels > 1 ? levels - 1 : 0) * k * k + 3) & ~3;
+  g.small = (g.t1 + k * k + 3) & ~3;
   g.st3 = (k * k * k + 3) & ~3;
-  g.total = g.o2 + (levels > 2 ? levels - 2 : 0) * g.st3;
+  g.total = g.small + (levels > 2 ? levels - 2 : 0) * g.st3;
   return g;
 }
 size_t tree_sg_floats(int topk, int levels) { return (size_t)sg_layout(topk, levels).total; }
 
-// One thread per table entry: s_ng = the 3-gram row's score, else the 2-gram row's, else log(eps) (Algorithm 1
-// line 9, Appendix C / D).  Both first slots are requested before either is examined.
+// One lookup (see NgramTable): the fingerprint word of the key's home bucket; a slot is read (and its key compared)
+// only where a fingerprint matches; a word with an empty slot and no matching row ends the search (a miss), a full one
+// sends it on to the next bucket, at most max_probe times.
+__device__ __noinline__ bool table_find(const NgramTable T, unsigned long long key, float* score) {
+  const unsigned long long hh = ngram_hash(key);
+  const uint32_t f = ngram_fingerprint(hh);
+  uint32_t h = (uint32_t)hh & T.mask;
+  for (uint32_t i = 0; i <= T.max_probe; ++i, h = (h + 1) & T.mask) {
+    const uint4 w = __ldg(T.fp + h);
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+    bool has_empty = false;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const uint32_t g = (ww[q >> 1] >> ((q & 1) * 16)) & 0xffffu;
+      has_empty = has_empty || g == 0u;
+      if (g == f) {
+        const uint4 sl = __ldg(reinterpret_cast<const uint4*>(T.slots + (size_t)h * 8 + q));
+        if ((((unsigned long long)sl.y << 32) | sl.x) == key) { *score = __uint_as_float(sl.z); return true; }
+      }
+    }
+    if (has_empty) return false;
+  }
+  return false;
+}
+
+// The sweep's unit of work is one row of k entries, a warp per row and a lane per candidate of the level, so that the
+// row's context tokens, its place in the tables and the level are worked out once per warp (one thread per entry spent
+// most of its time on the divisions that take an entry's index apart: the sweep is bound by instructions, not by its
+// reads -- the same 7.7 us with a table fresh in L2 as with a cold one).
+//   small rows  r = 0: bg0 and t0;  r = 1 + (i-1) k + j', i >= 1: bg of (level i, j'), and for i = 1 also t1 of j'
+//   slice rows  (level i >= 2, r' = j'' k + j'): t3
+__host__ __device__ inline int sweep_small_rows(int k, int levels) { return 1 + (levels > 1 ? levels - 1 : 0) * k; }
+
+__device__ __forceinline__ void sweep_lookup2(const TreeParams& p, int ta, int tb, int tt, float* dst2, float* dst3) {
+  // dst2 (may be null): the 2-gram entry (tb, tt); dst3 (may be null): the 3-gram entry (ta, tb, tt)
+  const bool have = p.table.slots != nullptr && tb >= 0;
+  float v;
+  if (dst2 != nullptr) *dst2 = (have && table_find(p.table, ngram_key(2, -1, tb, tt), &v)) ? v : p.miss;
+  if (dst3 != nullptr)
+    *dst3 = (have && p.ngram_order >= 3 && ta >= 0 && table_find(p.table, ngram_key(3, ta, tb, tt), &v))
+                ? v : __uint_as_float(kNoRowBits);
+}
+__device__ __forceinline__ void sweep_small_row(const TreeParams& p, int b, int Lb, const SgLayout& g, int r, int lane) {
+  const int k = p.topk;
+  if (lane >= k) return;
+  const int* ids = p.ids + ((size_t)b * p.K + p.first_rows[b]) * k;
+  float* sg = p.sg + (size_t)b * g.total;
+  if (r == 0) {
+    sweep_lookup2(p, p.ctx_tail[2 * b], p.ctx_tail[2 * b + 1], ids[lane], sg + lane, sg + g.t0 + lane);
+  } else {
+    const int i = 1 + (r - 1) / k, j1 = (r - 1) - (i - 1) * k;
+    if (i >= Lb) return;
+    sweep_lookup2(p, i == 1 ? p.ctx_tail[2 * b + 1] : -1, ids[(i - 1) * k + j1], ids[i * k + lane], sg + g.bg + (i - 1) * k * k + j1 * k + lane,
+                  i == 1 ? sg + g.t1 + j1 * k + lane : nullptr);
+  }
+}
+__device__ __forceinline__ void sweep_slice_row(const TreeParams& p, int b, int Lb, const SgLayout& g, int i, int r, int lane) {
+  const int k = p.topk;
+  if (lane >= k || i >= Lb) return;
+  const int* ids = p.ids + ((size_t)b * p.K + p.first_rows[b]) * k;
+  const int j2 = r / k, j1 = r - j2 * k;
+  sweep_lookup2(p, ids[(i - 2) * k + j2], ids[(i - 1) * k + j1], ids[i * k + lane], nullptr,
+                p.sg + (size_t)b * g.total + g.small + (i - 2) * g.st3 + r * k + lane);
+}
+
+// The sweep as a kernel of its own (batches whose fused launch would not fit the GPU): one warp per row.
 __global__ void __launch_bounds__(256) ngram_sweep_kernel(const TreeParams p) {
   pdl_wait();
   pdl_trigger();   // a short kernel: the next one may be scheduled and run its set-up now
-  const int k = p.topk, b = blockIdx.y;
-  const int fr = p.first_rows[b], Lb = min(p.n_levels, p.K - fr);   // this sequence's level 0 row and levels
+  const int b = blockIdx.y, k = p.topk, lane = threadIdx.x & 31;
+  const int Lb = min(p.n_levels, p.K - p.first_rows[b]);   // this sequence's levels
   const SgLayout g = sg_layout(k, p.n_levels);
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
-  int ta, tb, tt, dst;
-  const int k2 = k * k, k3 = k2 * k;
-  if (e < k) {
-    ta = p.ctx_tail[2 * b]; tb = p.ctx_tail[2 * b + 1]; tt = ids[e]; dst = e;
-  } else if (e < k + k2) {
-    if (Lb < 2) return;
-    const int r = e - k, j1 = r / k;
-    ta = p.ctx_tail[2 * b + 1]; tb = ids[j1]; tt = ids[k + r - j1 * k]; dst = g.o1 + r;
-  } else {
-    const int r = e - k - k2, i = 2 + r / k3;
-    if (i >= Lb) return;
-    const int q = r - (i - 2) * k3, j2 = q / k2, j1 = (q - j2 * k2) / k;
-    ta = ids[(i - 2) * k + j2]; tb = ids[(i - 1) * k + j1]; tt = ids[i * k + q - j2 * k2 - j1 * k];
-    dst = g.o2 + (i - 2) * g.st3 + q;
+  const int n_small = sweep_small_rows(k, p.n_levels), row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row < n_small) sweep_small_row(p, b, Lb, g, row, lane);
+  else {
+    const int rr = row - n_small, i = 2 + rr / (k * k);
+    if (i < p.n_levels) sweep_slice_row(p, b, Lb, g, i, rr - (i - 2) * k * k, lane);
   }
-  float sc = p.miss;
-  const NgramTable T = p.table;
-  if (T.slots != nullptr && tb >= 0) {
-    const bool tri = p.ngram_order >= 3 && ta >= 0;
-    const unsigned long long k2key = ngram_key(2, -1, tb, tt), k3key = ngram_key(3, tri ? ta : 0, tb, tt);
-    const uint32_t h2 = (uint32_t)ngram_hash(k2key) & T.mask, h3 = (uint32_t)ngram_hash(k3key) & T.mask;
-    const NgramSlot s2 = load_slot(T.slots + h2);
-    const NgramSlot s3 = tri ? load_slot(T.slots + h3) : s2;
-    float v;
-    if (probe_rest(T, k2key, h2, s2, v)) sc = v;
-    if (tri && probe_rest(T, k3key, h3, s3, v)) sc = v;
-  }
-  p.sg[(size_t)b * g.total + dst] = sc;
 }
 
 // The sweep for the trie layout: one warp per (level i, list kind, context position jb).  The context token x is
@@ -462,11 +491,11 @@ __global__ void __launch_bounds__(MAXT) tree_kernel(const TreeParams p) {
 struct HashTreeSmem {
   float* n_score; float* n_clamp; int* n_tok; int* n_par; unsigned char* n_j;   // per node (the root is node 0); n_j: its candidate index
   int* c_ids; float* c_sl;                         // [L][k] the candidates' ids and s_logit, staged once
-  int* b_node; float* b_sc; float* b_cl; int* b_row;   // per beam entry: node, score, clamped score, row of its context in the level's slice
+  int* b_node; float* b_sc; float* b_cl; int* b_row; int* b_bg;   // per beam entry: node, score, clamped score, rows of its context in the level's 3-gram and 2-gram tables
   Key* lvl_sorted;                                 // [2][64] best of a level by clamped score (the running best lags one level behind)
   int* sel; int* par_out; int* lvl_base;
   SelectSmem* ss;
-  float* sg01; float* slice;                       // staged score table: levels 0 and 1; one level >= 2
+  float* sg01; float* slice;                       // staged score tables: the small ones; one level's slice of t3
 };
 __host__ __device__ inline size_t hash_tree_layout(int k, int w, int budget, int L, bool stage, unsigned char* base, HashTreeSmem* t) {
   const int n_max = 1 + k + (L - 1) * w * k;
@@ -476,17 +505,17 @@ __host__ __device__ inline size_t hash_tree_layout(int k, int w, int budget, int
   const size_t o_sc = take((size_t)n_max * 4), o_cl = take((size_t)n_max * 4), o_tok = take((size_t)n_max * 4), o_par = take((size_t)n_max * 4),
                o_nj = take((size_t)n_max),
                o_ci = take((size_t)L * k * 4), o_cs = take((size_t)L * k * 4),
-               o_bn = take((size_t)w * 4), o_bs = take((size_t)w * 4), o_bc = take((size_t)w * 4), o_br = take((size_t)w * 4),
+               o_bn = take((size_t)w * 4), o_bs = take((size_t)w * 4), o_bc = take((size_t)w * 4), o_br = take((size_t)w * 4), o_bb = take((size_t)w * 4),
                o_ls = take(2 * 64 * 8), o_sel = take((size_t)(budget + 1) * 4), o_po = take((size_t)budget * 4),
                o_lb = take((size_t)(L + 1) * 4), o_ss = take(sizeof(SelectSmem)),
-               o_01 = take(stage ? (size_t)g.o2 * 4 : 0), o_sl = take(stage && L > 2 ? (size_t)g.st3 * 4 : 0);
+               o_01 = take(stage ? (size_t)g.small * 4 : 0), o_sl = take(stage && L > 2 ? (size_t)g.st3 * 4 : 0);
   if (t != nullptr) {
     t->n_score = reinterpret_cast<float*>(base + o_sc);
     t->n_clamp = reinterpret_cast<float*>(base + o_cl); t->n_tok = reinterpret_cast<int*>(base + o_tok);
     t->n_par = reinterpret_cast<int*>(base + o_par); t->n_j = base + o_nj;
     t->c_ids = reinterpret_cast<int*>(base + o_ci); t->c_sl = reinterpret_cast<float*>(base + o_cs);
     t->b_node = reinterpret_cast<int*>(base + o_bn); t->b_sc = reinterpret_cast<float*>(base + o_bs);
-    t->b_cl = reinterpret_cast<float*>(base + o_bc); t->b_row = reinterpret_cast<int*>(base + o_br);
+    t->b_cl = reinterpret_cast<float*>(base + o_bc); t->b_row = reinterpret_cast<int*>(base + o_br); t->b_bg = reinterpret_cast<int*>(base + o_bb);
     t->lvl_sorted = reinterpret_cast<Key*>(base + o_ls);
     t->sel = reinterpret_cast<int*>(base + o_sel); t->par_out = reinterpret_cast<int*>(base + o_po);
     t->lvl_base = reinterpret_cast<int*>(base + o_lb); t->ss = reinterpret_cast<SelectSmem*>(base + o_ss);
@@ -510,7 +539,9 @@ template <int MAXT, bool STAGE>
 __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
   extern __shared__ __align__(16) unsigned char tsm[];
   const int k = p.topk, w = p.beam, theta = p.budget - 1;
-  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x, last_warp = (nthr >> 5) - 1;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x, last_warp = (nthr >> 5) - 1;
+  const SgLayout g = sg_layout(k, p.n_levels);
+  const int b = blockIdx.x;
   const int fr = p.first_rows[b], L = min(p.n_levels, p.K - fr);   // this sequence's level 0 row and levels
   // When the block has a warp beyond the candidates (the launch adds one where 1024 threads allow it), that warp takes
   // no part in the selection: it keeps the running best 64, merging one level behind while the others select.
@@ -521,7 +552,6 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
   HashTreeSmem m;
   hash_tree_layout(k, w, p.budget, p.n_levels, STAGE, tsm, &m);
   __shared__ unsigned long long s_bits[64];
-  const SgLayout g = sg_layout(k, p.n_levels);
 #ifdef DART_TREE_TL
   __shared__ long long s_tl[40];
   int n_tl = 0;
@@ -531,7 +561,7 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
 #define TL_STAMP() do {} while (0)
 #endif
 
-  if (tid == 0) { m.n_score[0] = 0.f; m.n_clamp[0] = INFINITY; m.n_par[0] = -1; m.n_j[0] = 0; m.b_node[0] = 0; m.b_sc[0] = 0.f; m.b_cl[0] = INFINITY; m.b_row[0] = 0; m.lvl_base[0] = 1; }
+  if (tid == 0) { m.n_score[0] = 0.f; m.n_clamp[0] = INFINITY; m.n_par[0] = -1; m.n_j[0] = 0; m.b_node[0] = 0; m.b_sc[0] = 0.f; m.b_cl[0] = INFINITY; m.b_row[0] = 0; m.b_bg[0] = 0; m.lvl_base[0] = 1; }
   pdl_wait();
   TL_STAMP();
   const int* ids = p.ids + ((size_t)b * p.K + fr) * k;
@@ -540,8 +570,8 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
   if (tid == 0) m.n_tok[0] = p.ctx_tail[2 * b + 1];
   for (int e = tid; e < L * k; e += nthr) { m.c_ids[e] = ids[e]; m.c_sl[e] = sl[e]; }
   if (STAGE) {
-    copy_async16(m.sg01, sg, g.o2 / 4);
-    asm volatile("cp.async.wait_all;" ::: "memory");    // the scores of levels 0 and 1
+    copy_async16(m.sg01, sg, g.small / 4);
+    asm volatile("cp.async.wait_all;" ::: "memory");    // the small tables
   }
   block_select_init(m.ss);
   __syncthreads();
@@ -557,10 +587,13 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
     if (tid < ncand) {
       const int rho = my_rho, j = my_j;
       const int t = m.c_ids[i * k + j];
-      const int at = m.b_row[rho] + j;
-      float s_ng;
-      if (STAGE) s_ng = i < 2 ? m.sg01[(i == 0 ? 0 : g.o1) + at] : m.slice[at];
-      else s_ng = __ldg(sg + (i == 0 ? 0 : i == 1 ? g.o1 : g.o2 + (i - 2) * g.st3) + at);
+      // the candidate's 3-gram entry, or -- no such row -- its 2-gram entry
+      const int at3 = (i == 0 ? g.t0 : i == 1 ? g.t1 : g.small + (i - 2) * g.st3) + m.b_row[rho] + j;
+      const int at2 = (i == 0 ? 0 : g.bg + (i - 1) * k * k) + m.b_bg[rho] + j;
+      float s3, s2;
+      if (STAGE) { s3 = i < 2 ? m.sg01[at3] : m.slice[at3 - g.small - (i - 2) * g.st3]; s2 = m.sg01[at2]; }
+      else { s3 = __ldg(sg + at3); s2 = __ldg(sg + at2); }
+      const float s_ng = __float_as_uint(s3) == kNoRowBits ? s2 : s3;
       const float inc = __fmul_rn(__fadd_rn(__fmul_rn(p.wl[i], m.c_sl[i * k + j]), __fmul_rn(p.wn, s_ng)), p.wv[i]);
       s = __fadd_rn(m.b_sc[rho], inc);
       const float pc = m.b_cl[rho];
@@ -571,7 +604,7 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
     // keys carry the node index base + tid, which orders candidates of one level like tid does
     // best 64 by score -> next beam; `differs`: some clamped score is not its score (never, when increments <= 0)
     TL_STAMP();
-    const bool more = STAGE && (i == 0 ? L > 2 : (i >= 2 && i + 1 < L));   // a slice to fetch while this level is selected
+    const int fetch = i == 0 ? (L > 2 ? 2 : -1) : ((i >= 2 && i + 1 < L) ? i + 1 : -1);   // the level whose slice is fetched while this one is selected
     const int nb_next = ncand < w ? ncand : w;
     Key* lvl_out = m.lvl_sorted + (i & 1) * 64;
     const int differs = block_select64(
@@ -586,12 +619,13 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
             m.b_sc[r] = m.n_score[node];
             m.b_cl[r] = m.n_clamp[node];
             m.b_row[r] = (i == 0 ? j : (int)m.n_j[m.n_par[node]] * k + j) * k;
+            m.b_bg[r] = j * k;
           }
         },
         [&]() {
           // every thread has read what it needs of level i's slice: the next one may overwrite it (levels 0 and 1 use
           // the small table, so level 2's slice is fetched during level 0 and nothing during level 1)
-          if (more) copy_async16(m.slice, sg + g.o2 + (i == 0 ? 0 : i - 1) * g.st3, g.st3 / 4);
+          if (STAGE && fetch >= 0) copy_async16(m.slice, sg + g.small + (fetch - 2) * g.st3, g.st3 / 4);
           if (idle && i > 0) {   // the spare warp: the running best takes in the previous level's best 64
             const Key* q = m.lvl_sorted + ((i - 1) & 1) * 64;
             merge_keep64(g0, g1, q[lane], q[32 + lane], lane);
@@ -724,21 +758,27 @@ static size_t hash_tree_smem_bytes(int topk, int beam, int budget, int n_levels)
   return hash_tree_layout(topk, beam, budget, n_levels, hash_tree_stages(topk, beam, budget, n_levels), nullptr, nullptr) + 16;
 }
 
+template <class K>
+static cudaError_t allow_smem(K kernel, size_t smem) {
+  return smem > 48 * 1024 ? cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) : cudaSuccess;
+}
+
 cudaError_t tree_setup(int topk, int beam, int budget, int max_levels) {
   size_t smem = tree_smem_bytes(topk, beam, budget, max_levels);
-  cudaError_t e = cudaSuccess;
-  if (smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(tree_kernel<512, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<1024, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  }
+  cudaError_t e = allow_smem(tree_kernel<512, true>, smem);
+  if (e == cudaSuccess) e = allow_smem(tree_kernel<1024, true>, smem);
   smem = hash_tree_smem_bytes(topk, beam, budget, max_levels);
-  if (e == cudaSuccess && smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(tree_hash_kernel<576, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<1024, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<576, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_hash_kernel<1024, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  }
+  if (e == cudaSuccess) e = allow_smem(tree_hash_kernel<576, true>, smem);
+  if (e == cudaSuccess) e = allow_smem(tree_hash_kernel<1024, true>, smem);
+  if (e == cudaSuccess) e = allow_smem(tree_hash_kernel<576, false>, smem);
+  if (e == cudaSuccess) e = allow_smem(tree_hash_kernel<1024, false>, smem);
   return e;
+}
+
+template <bool STAGE>
+static cudaError_t launch_hash_tree(const TreeParams& p, int threads, size_t smem, cudaStream_t st) {
+  if (threads <= 576) return launch_pdl(tree_hash_kernel<576, STAGE>, dim3(p.B), dim3(threads), smem, st, p);
+  return launch_pdl(tree_hash_kernel<1024, STAGE>, dim3(p.B), dim3(threads), smem, st, p);
 }
 
 cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
@@ -759,17 +799,17 @@ cudaError_t launch_tree(const TreeParams& p, cudaStream_t st) {
     if (threads <= 512) return launch_pdl(tree_kernel<512, true>, dim3(p.B), dim3(threads), smem, st, p);
     return launch_pdl(tree_kernel<1024, true>, dim3(p.B), dim3(threads), smem, st, p);
   }
-  const int k = p.topk, n_sg = k + k * k + (p.n_levels > 2 ? (p.n_levels - 2) * k * k * k : 0);
-  const cudaError_t e = launch_pdl(ngram_sweep_kernel, dim3((n_sg + 255) / 256, p.B), dim3(256), 0, st, p);
+  // (Sweep and tree as one launch -- sweep blocks that count themselves done, a tree block that waits for the count of a
+  // slice before fetching it -- was built and measured slower, 41.7 against 35.8 us at the 14B shape: the fence, the
+  // count and the poll cost more than the launch they replace.)
+  const int n3 = p.n_levels > 2 ? p.n_levels - 2 : 0;
+  const int n_rows = sweep_small_rows(p.topk, p.n_levels) + n3 * p.topk * p.topk;
+  const cudaError_t e = launch_pdl(ngram_sweep_kernel, dim3((n_rows + 7) / 8, p.B), dim3(256), 0, st, p);
   if (e != cudaSuccess) return e;
   const bool stage = hash_tree_stages(p.topk, p.beam, p.budget, p.n_levels);
   const size_t smem = hash_tree_layout(p.topk, p.beam, p.budget, p.n_levels, stage, nullptr, nullptr) + 16;
-  if (stage) {
-    if (threads <= 576) return launch_pdl(tree_hash_kernel<576, true>, dim3(p.B), dim3(threads), smem, st, p);
-    return launch_pdl(tree_hash_kernel<1024, true>, dim3(p.B), dim3(threads), smem, st, p);
-  }
-  if (threads <= 576) return launch_pdl(tree_hash_kernel<576, false>, dim3(p.B), dim3(threads), smem, st, p);
-  return launch_pdl(tree_hash_kernel<1024, false>, dim3(p.B), dim3(threads), smem, st, p);
+  return stage ? launch_hash_tree<true>(p, threads, smem, st) : launch_hash_tree<false>(p, threads, smem, st);
 }
+
 
 }  // namespace dart
