@@ -8,9 +8,8 @@
 //   3. a threshold T taken from the list *heads*: the heads are warp-sorted and T = the m-th best of
 //      the runs' p-th entries with m * (p + 1) >= topk, so at least topk heads are not after T and the
 //      global top-k lies among the entries that are not after T; each sorted list contributes a prefix;
-//   4. the survivors (typically a few dozen) go through the register merge tree of select.cuh, whose
-//      first topk entries are the answer in order.  More than 1024 survivors (massive ties) fall back
-//      to rank counting.
+//   4. every survivor (typically a few dozen) counts the survivors that precede it: its rank, and, below topk,
+//      its place in the output.
 // Nothing here depends on the order in which threads run.
 #include "common.cuh"
 #include "kernels.h"
@@ -142,24 +141,14 @@ __global__ void __launch_bounds__(kMergeThreads) topk_merge_kernel(const LmParam
   const float lse = s_lse;
   const int filled = ns < topk ? ns : topk;
 
-  if (ns <= kMergeThreads) {
-    // ---- best 64 of the survivors, in order, via the register merge tree
-    Key x0, x1;
-    block_best64(tid < ns ? skey[tid] : kPadKey, (ns + 31) >> 5, xk, 0, x0, x1);
-    if (warp == 0 && lane < filled) {
-      int src = -1;
-      for (int o = 0; o < ns; ++o)
-        if (skey[o] == x0) { src = ssrc[o]; break; }
-      const float y = has_ys ? ys[src] : p.part_y[((size_t)(src >> 5) * MP + tk) * 32 + (src & 31)];
-      p.out_ids[(size_t)tk * topk + lane] = ids[src];
-      p.out_slogit[(size_t)tk * topk + lane] = logf(expf(y - lse) + p.eps_logit);
-    }
-  } else {
-    // ---- massive ties: rank every survivor by counting the survivors that precede it
+  {
+    // ---- rank every survivor by counting the survivors that precede it (typically a few dozen of them: the count is
+    // a short loop of broadcast reads on two or three warps; a sort network over the block cost several times that)
     for (int sidx = tid; sidx < ns; sidx += kMergeThreads) {
       const Key me = skey[sidx];
       int rank = 0;
-      for (int o = 0; o < ns; ++o) rank += skey[o] > me;
+#pragma unroll 4
+      for (int o = 0; o < ns; ++o) rank += skey[o] > me ? 1 : 0;
       if (rank < topk) {
         const int src = ssrc[sidx];
         const float y = has_ys ? ys[src] : p.part_y[((size_t)(src >> 5) * MP + tk) * 32 + (src & 31)];
