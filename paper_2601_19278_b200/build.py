@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdart.so")
-SOURCES = ["api.cu", "tmap.cu", "umma_gemm.cu", "umma_dense.cu", "stage_inputs.cu", "attention.cu", "attn_umma.cu", "lm_head.cu", "topk_merge.cu", "topk_static.cu", "ngram_trie.cu", "tree.cu", "train_attn.cu", "selftest.cu"]
+SOURCES = ["api.cu", "tmap.cu", "umma_gemm.cu", "umma_own.cu", "umma_dense.cu", "stage_inputs.cu", "attention.cu", "attn_umma.cu", "lm_head.cu", "topk_merge.cu", "topk_static.cu", "ngram_trie.cu", "tree.cu", "train_attn.cu", "selftest.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-DNDEBUG",

@@ -169,6 +169,30 @@ struct UmmaGemmArgs {
 };
 cudaError_t launch_umma_rows(const GemmPlan& plan, const UmmaMaps& maps, const GemmInput& in, const EpiArgs& epi, float* part,
                              int* status, cudaStream_t st);
+// Gate / up with row ownership (umma_own.cu), for steps of up to eight token rows: CTA c owns output rows
+// [c * rows / grid, (c + 1) * rows / grid) of both matrices over the whole reduction length.
+constexpr size_t kOwnSmemMax = 208 * 1024;
+constexpr int kOwnMinRows = 96;   // rows per CTA from which the kernel's TMA boxes stream at the HBM rate
+struct OwnPlan {
+  int rows, Kd, KB;            // output rows per matrix, reduction length, 64-k blocks
+  int grid, R;                 // CTAs, weight rows per TMA box = ceil(rows / grid)
+  int stages, stage_bytes, w_tx_bytes;
+  size_t smem;
+};
+struct OwnArgs {
+  CUtensorMap mapW[2];         // gate and up, boxes of 64 k x R rows
+  CUtensorMap mapX;            // the activations: hi + lo pair as one 3-D map
+  int rows, KB, M;
+  int stages, stage_bytes, w_tx_bytes;
+  const float* ss_in; int ss_tiles, ss_mp, h; float eps;   // the input's sums of squares (1/rms is applied to the output)
+  bf16* out_hi; bf16* out_lo; long long ld_out;
+  int* status;
+};
+// false: this shape does not suit the kernel (fewer than kOwnMinRows or more than 128 rows per CTA)
+bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm);
+cudaError_t launch_umma_own(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi, int* status,
+                            cudaStream_t st);
+
 // Dense projections of the draft-side prefill (umma_dense.cu): C[T, n_out] = A[T, k] W^T with 128 token rows per
 // tile on the MMA's M side and 256 output features on its N side.  mode 0: feature FC (A = features, one weight
 // matrix, one reduction range) -> z g-half = bf16(g * gain), ss[T][n_tiles] partial sums of squares.  mode 1:

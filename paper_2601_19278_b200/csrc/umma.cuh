@@ -9,6 +9,9 @@
 namespace dart {
 namespace umma {
 
+#ifndef DART_TRYWAIT_HINT
+#define DART_TRYWAIT_HINT 2000u
+#endif
 constexpr int kSpinLimit = 400000;   // bounded waits: x <= 2 us per try
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -31,7 +34,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   asm volatile(
       "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(2000u)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(DART_TRYWAIT_HINT)
       : "memory");
   return ok != 0;
 }

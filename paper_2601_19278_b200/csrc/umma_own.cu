@@ -1,0 +1,193 @@
+// The gate / up projection with row ownership, for steps of up to eight token rows (Section 3.2's SiLU-gated MLP):
+// u = SiLU(rstd * W_gate n) * (rstd * W_up n).
+//
+// umma_gemm.cu balances the SMs by cutting the (tile, k-block) space into equal ranges, which splits every output
+// tile between CTAs: pieces in global memory, tickets, and a fused finalize on the kernel's tail by whichever CTA
+// arrives last (3.5 - 5.5 us per projection, on the critical path of the step).  Here the OUTPUT ROWS are cut instead:
+// CTA c owns rows [c * rows / G, (c + 1) * rows / G) of both matrices -- 117 or 118 of 17408 at the 14B shape -- and
+// streams them over the whole reduction length, gate first, then up, into two accumulators: every CTA reads the same
+// number of bytes AND holds complete results, so the epilogue goes from tensor memory straight to the down
+// projection's input, with no piece, no ticket and no second CTA involved (gate/up stage 71.7 -> 67.6 us).  A TMA box
+// may be any number of rows high: a stage of the ring holds R = ceil(rows / G) weight rows x 64 k plus the matching
+// 2 KB activation slice, and tcgen05.mma runs with M = 128 over a tile whose rows past R are whatever shared memory
+// holds there -- accumulator rows that nothing reads.
+// Why only gate / up: an SM takes in one box of weight rows after the other, each in about 320 + 3.4 cycles per
+// 128-byte row, whatever the MMA thread or the activation loads do (measured with this kernel: 35-row boxes 10 bytes
+// per clock, 70-row boxes 12, 118-row boxes 22 = the SM's share of HBM).  FC, o_proj and down would own 35 rows per
+// CTA at that shape -- 95 / 39 / 104 us instead of 41 / 25 / 43 -- and stay on the stream-K kernel, whose boxes are
+// 128 rows high.
+// Roles, barriers, bounded waits and programmatic dependent launch are those of umma_gemm.cu.
+#include "common.cuh"
+#include "kernels.h"
+#include "umma.cuh"
+
+namespace dart {
+
+using namespace umma;
+
+constexpr int kOwnThreads = 256;
+constexpr int kOwnMaxStages = 32;
+constexpr int kOwnXBytes = 16 * 64 * 2;          // hi and lo rows of eight tokens, 64 k
+
+__global__ void __launch_bounds__(kOwnThreads, 1) umma_own_kernel(const __grid_constant__ OwnArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ uint64_t full[kOwnMaxStages], empty[kOwnMaxStages], acc_full;
+  __shared__ uint32_t tmem_base;
+  __shared__ int abort_flag, s_bad;
+  __shared__ float s_rstd[8];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int c = blockIdx.x, G = gridDim.x;
+  const int r0 = (int)(((long long)c * a.rows) / G), r1 = (int)(((long long)(c + 1) * a.rows) / G);
+  const int stages = a.stages, stage_bytes = a.stage_bytes, w_bytes = stage_bytes - kOwnXBytes;
+  const int n_units = 2 * a.KB;     // gate's k-blocks, then up's
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(&acc_full, 1);
+    abort_flag = 0;
+    s_bad = 0;
+    fence_barrier_init();
+    // this thread is the producer: weights do not depend on the previous kernel, so the ring is filled with them
+    // before anything else of the CTA's setup
+    const int pre = n_units < stages ? n_units : stages;
+    const uint64_t wpol = l2_policy_evict_first();
+    int mat = 0, kb = 0;
+    for (int it = 0; it < pre; ++it) {
+      mbar_expect_tx(&full[it], a.w_tx_bytes + kOwnXBytes);
+      tma_load_2d_hint(ring + (size_t)it * stage_bytes, &a.mapW[mat], &full[it], kb * 64, r0, wpol);
+      if (++kb == a.KB) { kb = 0; ++mat; }
+    }
+  }
+  if (warp == 2) tmem_alloc(&tmem_base, 32);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base;
+
+  if (warp == 0 && lane == 0) {
+    // ---- producer (the ring already holds the first weights): activations depend on the previous kernel
+    const int pre = n_units < stages ? n_units : stages;
+    const uint64_t wpol = l2_policy_evict_first();
+    pdl_wait();
+    int mat = 0, kb = 0;
+    for (int it = 0; it < pre; ++it) {
+      tma_load_3d(ring + (size_t)it * stage_bytes + w_bytes, &a.mapX, &full[it], kb * 64, 0, 0);
+      if (++kb == a.KB) { kb = 0; ++mat; }
+    }
+    int s = pre == stages ? 0 : pre, ph = pre == stages ? 1 : 0;
+    for (int it = pre; it < n_units; ++it) {
+      if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
+      uint8_t* st = ring + (size_t)s * stage_bytes;
+      mbar_expect_tx(&full[s], a.w_tx_bytes + kOwnXBytes);
+      tma_load_2d_hint(st, &a.mapW[mat], &full[s], kb * 64, r0, wpol);
+      tma_load_3d(st + w_bytes, &a.mapX, &full[s], kb * 64, 0, 0);
+      if (++s == stages) { s = 0; ++ph; }
+      if (++kb == a.KB) { kb = 0; ++mat; }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer: gate accumulates into tensor-memory columns 0 .. 15, up into 16 .. 31
+    constexpr uint32_t idesc = idesc_bf16(128, 16);
+    int s = 0, ph = 0, mat = 0, kb = 0;
+    bool ok = true;
+    for (int it = 0; it < n_units; ++it) {
+      if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t wa = smem_u32(ring + (size_t)s * stage_bytes);
+      const uint64_t ad = desc_sw128(wa), bd = desc_sw128(wa + w_bytes);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) mma_f16(tmem + 16 * mat, ad + 2 * k, bd + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+      mma_commit(&empty[s]);
+      if (++s == stages) { s = 0; ++ph; }
+      if (++kb == a.KB) { kb = 0; ++mat; }
+    }
+    if (ok) mma_commit(&acc_full);
+  } else if (warp >= 4) {
+    // ---- epilogue: one output row per thread (row = tensor-memory lane)
+    const int wq = warp & 3, row = wq * 32 + lane;
+    const bool has_row = row < r1 - r0;
+    const int n = r0 + row, M = a.M;
+    pdl_wait();   // the sums of squares below are the previous kernel's; u may still be read by the one before it
+    if (wq == 0) {
+      // 1/rms of this projection's input, from the partial sums of squares its producer left (a fixed order)
+      for (int t = 0; t < 8; ++t) {
+        float sacc = 0.f;
+        if (t < M)
+          for (int tl = lane; tl < a.ss_tiles; tl += 32) sacc += __ldcg(a.ss_in + (size_t)tl * a.ss_mp + t);
+        sacc = warp_sum(sacc);
+        if (lane == 0) s_rstd[t] = t < M ? 1.f / sqrtf(sacc / (float)a.h + a.eps) : 0.f;
+      }
+    }
+    if (!mbar_wait(&acc_full, 0, &abort_flag)) s_bad = 1;
+    asm volatile("bar.sync 1, 128;" ::: "memory");   // s_rstd is written; the four warps agree on what follows
+    if (!s_bad) {
+      tc_fence_after();
+      const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16);
+      uint32_t rg[16], ru[16];
+      tmem_ld16(tbase, rg);
+      tmem_ld16(tbase + 16, ru);
+      tmem_ld_wait();
+      if (has_row) {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          if (t < M) {
+            // columns (2t, 2t+1) are token t's hi and lo parts; the previous RMSNorm's 1/rms is applied here
+            const float gt = s_rstd[t] * (__uint_as_float(rg[2 * t]) + __uint_as_float(rg[2 * t + 1]));
+            const float up = s_rstd[t] * (__uint_as_float(ru[2 * t]) + __uint_as_float(ru[2 * t + 1]));
+            bf16 hi, lo;
+            split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
+            a.out_hi[(size_t)t * a.ld_out + n] = hi;
+            a.out_lo[(size_t)t * a.ld_out + n] = lo;
+          }
+        }
+      }
+    }
+  }
+  pdl_wait();
+  pdl_trigger();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) { tc_fence_after(); tmem_dealloc(tmem, 32); }
+  if (abort_flag && threadIdx.x == 0) {
+    // a wait ran out: report it and give copies that may still be in flight time to land
+    atomicExch(a.status, DEV_TIMEOUT);
+    for (int i = 0; i < 100; ++i) __nanosleep(1000);
+  }
+}
+
+bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm) {
+  p->rows = rows; p->Kd = Kd; p->KB = (Kd + 63) / 64;
+  p->grid = rows < n_sm ? rows : n_sm;
+  p->R = (rows + p->grid - 1) / p->grid;
+  // boxes of fewer rows would not stream at the HBM rate (see the head of this file); more do not fit the MMA tile
+  if (p->R < kOwnMinRows || p->R > 128) return false;
+  const int w_area = ((p->R + 7) / 8) * 8 * 128;                  // whole 8-row groups of 128-byte rows
+  p->stage_bytes = w_area + kOwnXBytes;
+  p->w_tx_bytes = p->R * 128;                                     // what one weight box delivers (rows past the matrix are zero-filled and counted)
+  // the MMA reads 128 rows from a stage's base, i.e. past the rows that were loaded: the ring ends with that much room
+  const int tail = 128 * 128;
+  int stages = (int)((kOwnSmemMax - 1024 - tail) / p->stage_bytes);
+  if (stages > kOwnMaxStages) stages = kOwnMaxStages;
+  if (stages < 2) return false;
+  p->stages = stages;
+  p->smem = (size_t)stages * p->stage_bytes + tail + 1024;
+  return true;
+}
+
+cudaError_t launch_umma_own(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi,
+                            int* status, cudaStream_t st) {
+  OwnArgs a;
+  memset(&a, 0, sizeof(a));
+  a.mapW[0] = mapW[0]; a.mapW[1] = mapW[1];
+  a.mapX = mapX;
+  a.rows = plan.rows; a.KB = plan.KB; a.M = M;
+  a.stages = plan.stages; a.stage_bytes = plan.stage_bytes; a.w_tx_bytes = plan.w_tx_bytes;
+  a.ss_in = epi.ss_in; a.ss_tiles = epi.ss_tiles; a.ss_mp = epi.ss_mp; a.h = epi.h; a.eps = epi.eps;
+  a.out_hi = epi.out_hi; a.out_lo = epi.out_lo; a.ld_out = epi.ld_out;
+  a.status = status;
+  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_own_kernel), kOwnSmemMax);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(umma_own_kernel, dim3(plan.grid), dim3(kOwnThreads), plan.smem, st, a);
+}
+
+}  // namespace dart
