@@ -14,7 +14,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdart.so")
+# DART_LIB: load another build of the same library instead (the tests run once against the -DDART_DEBUG build)
+LIB_PATH = os.environ.get("DART_LIB") or os.path.join(_HERE, "libdart.so")
 
 DART_OK = 0
 DART_ERR_INVALID_ARG = -1

@@ -614,7 +614,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   }
   auto set_epi = [&](int mode) {
     memset(&ep, 0, sizeof(ep));
-    ep.mode = mode; ep.K = K; ep.h = hdim; ep.eps = c.rms_eps; ep.B = B;
+    ep.mode = mode; ep.K = K; ep.h = hdim; ep.eps = c.rms_eps; ep.B = B; ep.status = ws.status;
     memcpy(ep.foff, fo.v, sizeof(ep.foff));
   };
 
@@ -938,7 +938,7 @@ int dart_last_device_status(dart_handle* h, void* cuda_stream) {
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return fail_cuda(h, e);
   }
-  return v == 0 ? DART_OK : DART_ERR_TIMEOUT;
+  return v == 0 ? DART_OK : (v == DART_ERR_INTERNAL ? DART_ERR_INTERNAL : DART_ERR_TIMEOUT);
 }
 
 int dart_selftest_bounded_wait(dart_handle* h, int32_t spin_limit, int32_t leave_ticket, void* cuda_stream) {

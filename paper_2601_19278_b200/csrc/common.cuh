@@ -75,6 +75,16 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Device status word values (mirrors dart_status for the device-detectable errors).
-enum : int { DEV_OK = 0, DEV_TIMEOUT = -5 };
+enum : int { DEV_OK = 0, DEV_TIMEOUT = -5, DEV_BAD_INDEX = -6 };
+
+// Index checks of the debug build (-DDART_DEBUG): `DART_CHECK(cond, status) statement;` runs the statement only when
+// cond holds and otherwise records DEV_BAD_INDEX in the status word (never traps, never faults); the release build
+// compiles the statement alone.  The checks stand in for a memory sanitizer: they guard the stores whose indices
+// come from the caller's lengths, counts and plans.
+#ifdef DART_DEBUG
+#define DART_CHECK(cond, status) if (!(cond)) { if ((status) != nullptr) atomicExch((status), (int)DEV_BAD_INDEX); } else
+#else
+#define DART_CHECK(cond, status)
+#endif
 
 }  // namespace dart

@@ -229,11 +229,13 @@ static __device__ __forceinline__ void finalize_group_t(int ft, const GemmArgs& 
         // the FC's token index counts fresh rows only; its z row is the step's row (b, r)
         const int o = MODE == EPI_FC ? fresh_to_step_row(e, t < M ? t : 0) : t;
         if (row < rows_valid && t < M && !dry) {
-          if (resw != nullptr) resw[(size_t)t * e.h + n] = x[k];
-          bf16 hi, lo;
-          split_bf16(x[k] * gam, hi, lo);
-          e.out_hi[(size_t)o * e.ld_out + n] = hi;
-          e.out_lo[(size_t)o * e.ld_out + n] = lo;
+          DART_CHECK(n < e.h && o >= 0 && o < e.B * e.K, e.status) {
+            if (resw != nullptr) resw[(size_t)t * e.h + n] = x[k];
+            bf16 hi, lo;
+            split_bf16(x[k] * gam, hi, lo);
+            e.out_hi[(size_t)o * e.ld_out + n] = hi;
+            e.out_lo[(size_t)o * e.ld_out + n] = lo;
+          }
         }
         if (row == 0 && t < M && !dry) e.ss_out[(size_t)Ta * MP + t] = q[k];
       }
@@ -246,8 +248,10 @@ static __device__ __forceinline__ void finalize_group_t(int ft, const GemmArgs& 
           const float gt = s_rstd[tok] * fs->xs[0][row][tl], up = s_rstd[tok] * fs->xs[1][row][tl];
           bf16 hi, lo;
           split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
-          e.out_hi[(size_t)tok * e.ld_out + n] = hi;
-          e.out_lo[(size_t)tok * e.ld_out + n] = lo;
+          DART_CHECK(n < e.ld_out && tok < e.B * e.K, e.status) {
+            e.out_hi[(size_t)tok * e.ld_out + n] = hi;
+            e.out_lo[(size_t)tok * e.ld_out + n] = lo;
+          }
         }
       }
     } else if (MODE == EPI_QKV) {
@@ -276,16 +280,20 @@ static __device__ __forceinline__ void finalize_group_t(int ft, const GemmArgs& 
           const int head = (row_base / dh) + hl;
           if (kind == 0) {
             const size_t o = (((size_t)b * e.Hq + head) * K + r) * dh;
-            e.q_hi[o + i] = h1; e.q_hi[o + i + half] = h2;
-            e.q_lo[o + i] = l1; e.q_lo[o + i + half] = l2;
+            DART_CHECK(head < e.Hq && b < e.B, e.status) {
+              e.q_hi[o + i] = h1; e.q_hi[o + i + half] = h2;
+              e.q_lo[o + i] = l1; e.q_lo[o + i + half] = l2;
+            }
           } else {
             bf16* side = (kind == 1 ? e.k_new : e.v_new) + ((size_t)b * e.Hkv + head) * 16 * dh;
             side[(size_t)r * dh + i] = h1; side[(size_t)r * dh + i + half] = h2;
             side[(size_t)(8 + r) * dh + i] = l1; side[(size_t)(8 + r) * dh + i + half] = l2;
             if (fresh_index(e, b, r) >= 0) {
               bf16* dst = (kind == 1 ? e.k_cache : e.v_cache) + (((size_t)b * e.Hkv + head) * e.P_cap + s_pos[tok]) * dh;
-              dst[i] = h1;
-              dst[i + half] = h2;
+              DART_CHECK(s_pos[tok] >= 0 && s_pos[tok] < e.P_cap && head < e.Hkv, e.status) {   // the append stays inside the sequence's cache rows
+                dst[i] = h1;
+                dst[i + half] = h2;
+              }
             }
           }
         }

@@ -128,6 +128,7 @@ struct EpiArgs {
   // EPI_QKV
   int Hq, Hkv, dh; const int32_t* seq_lens; const float2* rope_tab;  // [positions][dh/2] (cos, sin)
   bf16* q_hi; bf16* q_lo; bf16* k_new; bf16* v_new; bf16* k_cache; bf16* v_cache; long long P_cap;
+  int* status;   // device status word (the debug build's index checks report here)
 };
 
 // The weight sub-matrices and the activations of one streaming launch.

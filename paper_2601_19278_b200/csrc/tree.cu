@@ -599,7 +599,9 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
       const float pc = m.b_cl[rho];
       cl = s < pc ? s : pc;
       const int n = base + tid;
-      m.n_score[n] = s; m.n_clamp[n] = cl; m.n_tok[n] = t; m.n_par[n] = m.b_node[rho]; m.n_j[n] = (unsigned char)j;
+      DART_CHECK(n < 1 + k + (p.n_levels - 1) * w * k, p.status) {   // inside the node arrays
+        m.n_score[n] = s; m.n_clamp[n] = cl; m.n_tok[n] = t; m.n_par[n] = m.b_node[rho]; m.n_j[n] = (unsigned char)j;
+      }
     }
     // keys carry the node index base + tid, which orders candidates of one level like tid does
     // best 64 by score -> next beam; `differs`: some clamped score is not its score (never, when increments <= 0)
@@ -610,6 +612,7 @@ __global__ void __launch_bounds__(MAXT) tree_hash_kernel(const TreeParams p) {
     const int differs = block_select64(
         tid < ncand ? make_key(s, base + tid) : kPadKey, s, tid < ncand && cl != s, idle, n_active, m.ss,
         [&](int r, Key key, int any) {
+          DART_CHECK(r >= 0 && r < 64, p.status)
           if (!any) lvl_out[r] = key;
           if (r < nb_next) {
             // beam entry r of the next level: its node, scores and the row of its context -- (the parent's candidate

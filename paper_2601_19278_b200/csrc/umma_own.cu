@@ -136,8 +136,10 @@ __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_kernel(const __grid_c
             const float up = s_rstd[t] * (__uint_as_float(ru[2 * t]) + __uint_as_float(ru[2 * t + 1]));
             bf16 hi, lo;
             split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
-            a.out_hi[(size_t)t * a.ld_out + n] = hi;
-            a.out_lo[(size_t)t * a.ld_out + n] = lo;
+            DART_CHECK(n < a.rows && n < a.ld_out, a.status) {
+              a.out_hi[(size_t)t * a.ld_out + n] = hi;
+              a.out_lo[(size_t)t * a.ld_out + n] = lo;
+            }
           }
         }
       }
