@@ -9,10 +9,7 @@
 namespace dart {
 namespace umma {
 
-#ifndef DART_TRYWAIT_HINT
-#define DART_TRYWAIT_HINT 2000u
-#endif
-constexpr int kSpinLimit = 400000;   // bounded waits: x <= 2 us per try
+constexpr int kSpinLimit = 4000000;   // bounded waits: polls of ~60 cycles each, i.e. about a tenth of a second in all
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -29,20 +26,24 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+// One non-blocking look at the barrier.  (mbarrier.try_wait, which may suspend the thread until the phase completes,
+// reacted later: the single-thread producer and MMA loops are on every stage's critical path, and polling with
+// test_wait took 5 us off the LM head at the 14B shape and 2 us off each large projection.  The poll must not be
+// tighter than this one -- a look, then a shared-memory read of the abort flag: 64 looks between two reads of the
+// flag, with 130 threads of a CTA waiting at a time, cost the LM head 30 us.)
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(DART_TRYWAIT_HINT)
-      : "memory");
+  asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+               : "=r"(ok)
+               : "r"(smem_u32(bar)), "r"(parity)
+               : "memory");
   return ok != 0;
 }
 // Bounded wait.  On time-out (or when another role has given up) sets *abort_flag and returns false.
 // `limit`: tries before giving up (the kernels use the default; the self-test kernel passes a small one).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int limit = kSpinLimit) {
   for (int it = 0; it < limit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_test_wait(bar, parity)) return true;
     if (*abort_flag) return false;
   }
   *abort_flag = 1;

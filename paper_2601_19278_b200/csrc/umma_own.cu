@@ -11,11 +11,13 @@
 // may be any number of rows high: a stage of the ring holds R = ceil(rows / G) weight rows x 64 k plus the matching
 // 2 KB activation slice, and tcgen05.mma runs with M = 128 over a tile whose rows past R are whatever shared memory
 // holds there -- accumulator rows that nothing reads.
-// Why only gate / up: an SM takes in one box of weight rows after the other, each in about 320 + 3.4 cycles per
-// 128-byte row, whatever the MMA thread or the activation loads do (measured with this kernel: 35-row boxes 10 bytes
-// per clock, 70-row boxes 12, 118-row boxes 22 = the SM's share of HBM).  FC, o_proj and down would own 35 rows per
-// CTA at that shape -- 95 / 39 / 104 us instead of 41 / 25 / 43 -- and stay on the stream-K kernel, whose boxes are
-// 128 rows high.
+// Why only gate / up: a stage of the ring costs the same ~650 cycles whatever it holds.  Cycle counters in this kernel:
+// the MMA-issuing thread spends ~370 cycles per stage on the fence, four MMAs and the commit and ~270 waiting for the
+// stage; the producer ~220 on the expect-tx and two TMA issues and ~360 waiting for a free stage; the period equals the
+// sum of the two issue times, with 4 stages in the ring as with 27, with or without the activation loads, with one
+// commit per stage or per four.  118 rows x 64 k per stage is then 22 bytes per clock -- an SM's share of HBM; FC,
+// o_proj and down would own 35 rows per CTA at the 14B shape and stream at 10 (95 / 39 / 104 us instead of 41 / 25 /
+// 43: measured), so they stay on the stream-K kernel, whose stages hold 128 rows.
 // Roles, barriers, bounded waits and programmatic dependent launch are those of umma_gemm.cu.
 #include "common.cuh"
 #include "kernels.h"
