@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
       if (ue > u1) ue = u1;
       const bool owner = ka == 0, whole = owner && ue == (long long)(tile + 1) * KB;
       const int buf = visit & 1;
-      if (!mbar_wait(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) s_bad = 1;
+      if (!mbar_wait_relaxed(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) s_bad = 1;
       if (owner && !whole && et == 0) {
         // the rest of this tile comes from the next CTAs, for which it was the first thing to do
         for (int cc = c + 1; cc < G && ((long long)cc * a.U) / G < (long long)(tile + 1) * KB; ++cc) {
@@ -530,7 +530,7 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
       if (ue > u1) ue = u1;
       const bool owner = ka == 0, whole = owner && ue == (long long)(tile + 1) * KB;
       const int buf = visit & 1;
-      if (!mbar_wait(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) s_bad = 1;
+      if (!mbar_wait_relaxed(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) s_bad = 1;
       if (owner && !whole && et == 0) {
         for (int cc = c + 1; cc < G && ((long long)cc * a.U) / G < (long long)(tile + 1) * KB; ++cc) {
           int it = 0;

@@ -9,6 +9,9 @@
 namespace dart {
 namespace umma {
 
+#ifndef DART_RELAX_NS
+#define DART_RELAX_NS 200
+#endif
 constexpr int kSpinLimit = 4000000;   // bounded waits: polls of ~60 cycles each, i.e. about a tenth of a second in all
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -45,6 +48,18 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   for (int it = 0; it < limit; ++it) {
     if (mbar_test_wait(bar, parity)) return true;
     if (*abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+// The same for waits that last a whole tile (the read-out warps waiting for an accumulator): a pause between two
+// looks, so that 128 waiting threads leave the shared-memory pipe to the copy engine and the MMAs.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int limit = kSpinLimit / 4) {
+  for (int it = 0; it < limit; ++it) {
+    if (mbar_test_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    __nanosleep(DART_RELAX_NS);
   }
   *abort_flag = 1;
   return false;

@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       long long ue = (long long)(tile + 1) * KB;
       if (ue > u1) ue = u1;
       const int buf = visit & 1;
-      if (!mbar_wait(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) break;
+      if (!mbar_wait_relaxed(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) break;
       tc_fence_after();
       if (!waited) { pdl_wait(); waited = true; }   // the piece area may still be read by the previous kernel
       float* dst = p.part + (((size_t)c * p.slots + visit) * 128 + row) * MP;

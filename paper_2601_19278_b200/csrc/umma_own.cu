@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_kernel(const __grid_c
         if (lane == 0) s_rstd[t] = t < M ? 1.f / sqrtf(sacc / (float)a.h + a.eps) : 0.f;
       }
     }
-    if (!mbar_wait(&acc_full, 0, &abort_flag)) s_bad = 1;
+    if (!mbar_wait_relaxed(&acc_full, 0, &abort_flag)) s_bad = 1;
     asm volatile("bar.sync 1, 128;" ::: "memory");   // s_rstd is written; the four warps agree on what follows
     if (!s_bad) {
       tc_fence_after();
