@@ -106,7 +106,7 @@ __device__ __forceinline__ void fold_token(const LmParams& p, const float* srow,
 // ------------------------------------------------------------------------------------------------------
 using namespace umma;
 
-constexpr int kLmUmmaThreads = 256;
+constexpr int kLmUmmaThreads = 512;   // producer, MMA issuer, TMEM owner, one idle warp; four read-out and eight more fold warps
 
 template <int MP>
 struct LmUmmaCfg {
@@ -114,9 +114,9 @@ struct LmUmmaCfg {
   static constexpr int XBytes = N * 64 * 2;
   static constexpr int StageBytes = 128 * 64 * 2 + XBytes;
   static constexpr int TmemCols = 2 * N < 32 ? 32 : 2 * N;
-  // epilogue shared memory: stage [8][129] floats, lists 3 x [MP][32], statistics [MP][2], 1/rms [MP]
-  static constexpr size_t EpiBytes = sizeof(float) * (8 * 129 + 3 * MP * 32 + 3 * MP);
-  static constexpr int Stages = MP == 8 ? 11 : (MP == 32 ? 7 : 3);
+  // epilogue shared memory: stage [MP][129] floats, lists 3 x [MP][32], statistics [MP][2], 1/rms [MP]
+  static constexpr size_t EpiBytes = sizeof(float) * (MP * 129 + 3 * MP * 32 + 3 * MP);
+  static constexpr int Stages = MP == 8 ? 11 : 7;
   static constexpr size_t SmemBytes = (size_t)Stages * StageBytes + 1024 + EpiBytes;
 };
 
@@ -127,8 +127,8 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
   const LmParams& p = a.p;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  float* stage = reinterpret_cast<float*>(ring + (size_t)C::Stages * C::StageBytes);   // [8][SROW]
-  float* st_key = stage + 8 * SROW;          // [MP][32]
+  float* stage = reinterpret_cast<float*>(ring + (size_t)C::Stages * C::StageBytes);   // [MP][SROW]
+  float* st_key = stage + MP * SROW;         // [MP][32]
   float* st_y = st_key + MP * 32;
   int* st_id = reinterpret_cast<int*>(st_y + MP * 32);
   float* st_ms = reinterpret_cast<float*>(st_id + MP * 32);  // [MP][2]
@@ -221,18 +221,28 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
     }
     if (ok && tile >= 0) mma_commit(&acc_full[buf]);
   } else if (warp >= 4) {
-    // ---- read-out and fold: TMEM lane = vocabulary row of the tile.  The four warps agree on every exit
-    // through s_bad before a barrier of their own (id 1), so a wait that ran out cannot strand the others.
+    // ---- read-out (warps 4-7: TMEM lane = vocabulary row of the tile) and fold (warps 4-15: one token row per warp
+    // at a time).  A fold costs ~6000 cycles -- a CTA sees ~1000 vocabulary rows per token, so its running threshold
+    // never gets selective and one value in seven is inserted -- and with 32 token rows on four warps that was 47000
+    // cycles per tile against the 54000 the tile takes to stream: the MMA thread waited for a free accumulator a fifth
+    // of the time (cycle counters).  On twelve warps it is three folds per tile and warp.
+    // Every visit ends with the same two barriers for all twelve warps, and s_bad is only written between the second
+    // of one visit and the first of the next, so a wait that ran out takes all of them out at the same place.
+    const int fw = warp - 4;
+    const bool reader = fw < 4;
+    const int fi = reader ? fw + 8 : fw - 4;     // fold order: the warps that do not read out take the first rows
     const int wq = warp & 3, row = wq * 32 + lane, et = tid - 128;
     pdl_wait();
-    // the final RMSNorm's per-token 1/rms comes from the previous kernel's sums of squares
-    for (int i = et; i < MP; i += 128) {
-      float ssq = 0.f;
-      if (i < p.M)
-        for (int tl = 0; tl < p.ss_tiles; ++tl) ssq += p.ss_in[(size_t)tl * p.ss_mp + i];
-      s_rstd[i] = i < p.M ? 1.f / sqrtf(ssq / (float)p.Kd + p.rms_eps) : 0.f;
+    if (reader) {
+      // the final RMSNorm's per-token 1/rms comes from the previous kernel's sums of squares
+      for (int i = et; i < MP; i += 128) {
+        float ssq = 0.f;
+        if (i < p.M)
+          for (int tl = 0; tl < p.ss_tiles; ++tl) ssq += p.ss_in[(size_t)tl * p.ss_mp + i];
+        s_rstd[i] = i < p.M ? 1.f / sqrtf(ssq / (float)p.Kd + p.rms_eps) : 0.f;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
     }
-    asm volatile("bar.sync 1, 128;" ::: "memory");
     int visit = 0;
     long long u = u0;
     while (u < u1) {
@@ -241,68 +251,71 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
       long long ue = (long long)(tile + 1) * KB;
       if (ue > u1) ue = u1;
       const bool owner = ka == 0, whole = owner && ue == (long long)(tile + 1) * KB;
-      const int buf = visit & 1;
-      if (!mbar_wait_relaxed(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) s_bad = 1;
-      if (owner && !whole && et == 0) {
-        // the rest of this tile comes from the next CTAs, for which it was the first thing to do
-        for (int cc = c + 1; cc < G && ((long long)cc * a.U) / G < (long long)(tile + 1) * KB; ++cc) {
-          int it = 0;
-          while (*reinterpret_cast<volatile int*>(a.flags + cc) != a.tag && it < kSpinLimit) { __nanosleep(200); ++it; }
-          if (it >= kSpinLimit) { s_bad = 1; abort_flag = 1; }
-        }
-        __threadfence();
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (s_bad) break;
-      tc_fence_after();
-      const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + buf * C::N;
       const int rows_here = min(128, p.V - tile * 128);
-#pragma unroll 1
-      for (int ch = 0; ch < MP / 8; ++ch) {
-        uint32_t r[16];   // columns (2t, 2t+1) are token t's hi and lo parts
-        tmem_ld16(tbase + ch * 16, r);
-        tmem_ld_wait();
-        float y[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) y[j] = __uint_as_float(r[2 * j]) + __uint_as_float(r[2 * j + 1]);
-        if (ch == MP / 8 - 1) {  // the accumulator buffer is free once its last columns are in registers
-          tc_fence_before();
-          mbar_arrive(&acc_empty[buf]);
-        }
-        if (!owner) {
-          float* dst = a.pieces + (((size_t)c * 128 + row) * MP + ch * 8);
-          reinterpret_cast<float4*>(dst)[0] = make_float4(y[0], y[1], y[2], y[3]);
-          reinterpret_cast<float4*>(dst)[1] = make_float4(y[4], y[5], y[6], y[7]);
-          continue;
-        }
-        if (!whole) {
+      if (reader) {
+        const int buf = visit & 1;
+        if (!mbar_wait_relaxed(&acc_full[buf], (visit >> 1) & 1, &abort_flag)) s_bad = 1;
+        if (owner && !whole && et == 0) {
+          // the rest of this tile comes from the next CTAs, for which it was the first thing to do
           for (int cc = c + 1; cc < G && ((long long)cc * a.U) / G < (long long)(tile + 1) * KB; ++cc) {
-            const float* src = a.pieces + (((size_t)cc * 128 + row) * MP + ch * 8);
-            const float4 q0 = __ldcg(reinterpret_cast<const float4*>(src)), q1 = __ldcg(reinterpret_cast<const float4*>(src) + 1);
-            y[0] += q0.x; y[1] += q0.y; y[2] += q0.z; y[3] += q0.w;
-            y[4] += q1.x; y[5] += q1.y; y[6] += q1.z; y[7] += q1.w;
+            int it = 0;
+            while (*reinterpret_cast<volatile int*>(a.flags + cc) != a.tag && it < kSpinLimit) { __nanosleep(200); ++it; }
+            if (it >= kSpinLimit) { s_bad = 1; abort_flag = 1; }
+          }
+          __threadfence();
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (!s_bad) {
+          tc_fence_after();
+          const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + buf * C::N;
+#pragma unroll 1
+          for (int ch = 0; ch < MP / 8; ++ch) {
+            uint32_t r[16];   // columns (2t, 2t+1) are token t's hi and lo parts
+            tmem_ld16(tbase + ch * 16, r);
+            tmem_ld_wait();
+            float y[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) y[j] = __uint_as_float(r[2 * j]) + __uint_as_float(r[2 * j + 1]);
+            if (ch == MP / 8 - 1) {  // the accumulator buffer is free once its last columns are in registers
+              tc_fence_before();
+              mbar_arrive(&acc_empty[buf]);
+            }
+            if (!owner) {
+              float* dst = a.pieces + (((size_t)c * 128 + row) * MP + ch * 8);
+              reinterpret_cast<float4*>(dst)[0] = make_float4(y[0], y[1], y[2], y[3]);
+              reinterpret_cast<float4*>(dst)[1] = make_float4(y[4], y[5], y[6], y[7]);
+              continue;
+            }
+            if (!whole) {
+              for (int cc = c + 1; cc < G && ((long long)cc * a.U) / G < (long long)(tile + 1) * KB; ++cc) {
+                const float* src = a.pieces + (((size_t)cc * 128 + row) * MP + ch * 8);
+                const float4 q0 = __ldcg(reinterpret_cast<const float4*>(src)), q1 = __ldcg(reinterpret_cast<const float4*>(src) + 1);
+                y[0] += q0.x; y[1] += q0.y; y[2] += q0.z; y[3] += q0.w;
+                y[4] += q1.x; y[5] += q1.y; y[6] += q1.z; y[7] += q1.w;
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int tok = ch * 8 + j;
+              const float v = y[j] * s_rstd[tok];
+              stage[tok * SROW + row] = v;
+              if (p.logits_out != nullptr && tok < p.M && row < rows_here) p.logits_out[(size_t)tok * p.V + tile * 128 + row] = v;
+            }
+          }
+          if (!owner) {
+            // release the piece: every thread fences its part, then one thread raises this CTA's flag
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (et == 0) *reinterpret_cast<volatile int*>(a.flags + c) = a.tag;
           }
         }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int tok = ch * 8 + j;
-          const float v = y[j] * s_rstd[tok];
-          stage[j * SROW + row] = v;
-          if (p.logits_out != nullptr && tok < p.M && row < rows_here) p.logits_out[(size_t)tok * p.V + tile * 128 + row] = v;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        for (int j = wq; j < 8; j += 4) {
-          const int tk = ch * 8 + j;
-          if (tk < p.M) fold_token(p, stage + j * SROW, rows_here, tile * 128, tk, lane, st_key, st_y, st_id, st_ms);
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
       }
-      if (!owner) {
-        // release the piece: every thread fences its part, then one thread raises this CTA's flag
-        __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (et == 0) *reinterpret_cast<volatile int*>(a.flags + c) = a.tag;
-      }
+      asm volatile("bar.sync 2, 384;" ::: "memory");   // the tile's logits are staged (or a wait ran out)
+      const bool bad = s_bad != 0;
+      if (!bad && owner)
+        for (int tk = fi; tk < p.M; tk += 12) fold_token(p, stage + tk * SROW, rows_here, tile * 128, tk, lane, st_key, st_y, st_id, st_ms);
+      asm volatile("bar.sync 3, 384;" ::: "memory");   // the staging rows are free again
+      if (bad) break;
       ++visit;
       u = ue;
     }
@@ -347,7 +360,7 @@ cudaError_t launch_lm_head_umma(const LmParams& pin, const CUtensorMap& mapW, co
   const int MP = padded_tokens(pin.M);
   if (MP == 8) return launch_lm_umma_t<8>(a, st);
   if (MP == 32) return launch_lm_umma_t<32>(a, st);
-  return launch_lm_umma_t<128>(a, st);
+  return cudaErrorInvalidValue;   // more token rows go to lm_head_dense_kernel
 }
 
 // ------------------------------------------------------------------------------------------------------
