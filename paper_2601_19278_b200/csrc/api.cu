@@ -292,8 +292,9 @@ size_t part_capacity(const dart_config& c, int n_sm) {
   return a.part_max;
 }
 
-// Attention chunks: about two CTAs per SM, chunks of 128 .. 512 keys (longer chunks leave a CTA a long serial
-// loop of 64-key tiles; measured at batch 16: 1792-key chunks 218 us, 448-key chunks 190 us).
+// Attention chunks of the one-chunk-per-CTA split: about two CTAs per SM, chunks of 128 .. 512 keys (longer chunks
+// leave a CTA a long serial loop of 64-key tiles; measured at batch 16: 1792-key chunks 218 us, 448-key chunks 190 us).
+// The tcgen05 split picks longer ones (attn_umma_chunk_keys), which need fewer partial slots than this bound.
 constexpr int kAttnMaxChunk = 512;
 int attn_pairs_capacity(const dart_config& c, int n_sm) {
   const long long by_sm = (2 * n_sm) / c.n_kv_heads, by_len = ((long long)c.max_batch * c.max_prefix + kAttnMaxChunk - 1) / kAttnMaxChunk;
@@ -660,19 +661,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ap.B = B; ap.K = K; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.dh = c.head_dim;
   ap.seq_lens = in->seq_lens; ap.q_hi = ws.q_hi; ap.q_lo = ws.q_lo; ap.k_new = ws.k_new; ap.v_new = ws.v_new;
   ap.k_cache = static_cast<const bf16*>(in->k_cache); ap.v_cache = static_cast<const bf16*>(in->v_cache); ap.P_cap = c.max_prefix;
-  {
-    long long per = (total_keys * c.n_kv_heads + 2 * h->n_sm - 1) / (2 * h->n_sm);
-    long long chunk = ((per + 63) / 64) * 64;
-    if (chunk < 128) chunk = 128;
-    if (chunk > kAttnMaxChunk) chunk = kAttnMaxChunk;
-    ap.chunk_keys = (int)chunk;
-  }
   ap.o_part = ws.o_part; ap.ml_part = ws.ml_part; ap.a_hi = ws.a_hi; ap.a_lo = ws.a_lo;
-  {
-    long long pairs = 0;
-    for (int b = 0; b < B; ++b) pairs += (in->seq_lens_host[b] + ap.chunk_keys - 1) / ap.chunk_keys + 1;
-    if (pairs > h->attn_pairs_cap) return DART_ERR_INTERNAL;
-  }
   const AttnUmmaMaps* amaps = nullptr;
   if (c.head_dim == 128 && (long long)c.max_batch * c.n_kv_heads * c.max_prefix < (1ll << 31)) {
     // maps over the caller's caches are re-encoded only when the pointers change
@@ -684,6 +673,21 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
       h->attn_k_ptr = in->k_cache; h->attn_v_ptr = in->v_cache;
     }
     amaps = &h->attn_maps;
+  }
+  {
+    // one chunk per CTA, about two CTAs per SM, 128 .. 512 keys; the tcgen05 split has its own rule
+    long long per = (total_keys * c.n_kv_heads + 2 * h->n_sm - 1) / (2 * h->n_sm);
+    long long chunk = ((per + 63) / 64) * 64;
+    if (chunk < 128) chunk = 128;
+    if (chunk > kAttnMaxChunk) chunk = kAttnMaxChunk;
+    if (attn_uses_umma(B, c.n_kv_heads, c.head_dim, in->seq_lens_host, amaps != nullptr)) {
+      const int uc = attn_umma_chunk_keys(B, c.n_kv_heads, in->seq_lens_host, h->n_sm, h->attn_pairs_cap);
+      if (uc > 0) chunk = uc;
+    }
+    ap.chunk_keys = (int)chunk;
+    long long pairs = 0;
+    for (int b = 0; b < B; ++b) pairs += (in->seq_lens_host[b] + ap.chunk_keys - 1) / ap.chunk_keys + 1;
+    if (pairs > h->attn_pairs_cap) return DART_ERR_INTERNAL;
   }
   if ((e = launch_attention(ap, in->seq_lens_host, amaps, ws.status, st)) != cudaSuccess) return fail_cuda(h, e);
   mark(2, false);

@@ -306,6 +306,53 @@ cudaError_t attention_setup() {
   return e != cudaSuccess ? e : attn_umma_setup();
 }
 
+// Whether the step's attention runs on the tcgen05 split (attn_umma.cu).  It pays a few microseconds of set-up per
+// CTA (barriers, tensor memory, first loads) and wins from a few thousand 64-key tiles on (batch 4 x 8192 keys: 75 vs
+// 89 us; batch 1 x 4096 keys: 23.6 vs 21.1 us).
+bool attn_uses_umma(int B, int Hkv, int dh, const int* seq_lens_host, bool have_maps) {
+  long long key_tiles = 0;
+  for (int b = 0; b < B; ++b) key_tiles += (seq_lens_host[b] + 63) / 64;
+  return have_maps && dh == 128 && key_tiles * Hkv >= 2048;
+}
+
+// Chunk length for the tcgen05 split, whose CTAs take two consecutive chunks of a sequence each and stay alone on
+// their SM.  Short chunks mean several waves of CTAs, each paying its set-up, and more partials for the combine; long
+// ones leave SMs idle or one CTA with a long tail.  The estimate below -- a CTA costs its first chunk's 64-key tiles
+// plus six tiles' worth of set-up; one wave lasts as long as its longest CTA, more waves as long as the work spread
+// over the SMs plus half a CTA -- reproduces the measured order (4 x 8192 keys, 8 KV heads: 1216 keys 48 us, 1024:
+// 52, 512: 58; 16 ragged sequences: 1408 keys 103 us, 1024: 107, 512: 120, 4096: 146).  Candidates are the multiples
+// of 64 from 128 to 2048 whose chunk count fits `pairs_cap`; returns 0 if none does.
+int attn_umma_chunk_keys(int B, int Hkv, const int* seq_lens_host, int n_sm, int pairs_cap) {
+  constexpr int kSetupTiles = 6;
+  int best = 0;
+  double best_t = 0.0;
+  for (int chunk = 128; chunk <= 2048; chunk += 64) {
+    long long ctas = 0, total = 0, pairs = 0;
+    int longest = 0, most = 0;
+    for (int b = 0; b < B; ++b) {
+      const int P = seq_lens_host[b];
+      const int ncc = (P + chunk - 1) / chunk;            // cache chunks; chunk ncc is the new rows
+      const int n_full = ncc > 0 ? ncc / 2 : 0;           // CTAs whose first chunk is a whole one: 2x < ncc - 1
+      const int full_cost = chunk / 64 + kSetupTiles;
+      // the last CTA starts with the sequence's last cache chunk (ncc odd) or with the new rows (ncc even)
+      const int last_tiles = (ncc & 1) ? (P - (ncc - 1) * chunk + 63) / 64 : 1;
+      const int last_cost = last_tiles + kSetupTiles;
+      ctas += n_full + 1;
+      total += (long long)n_full * full_cost + last_cost;
+      if (n_full > 0 && full_cost > longest) longest = full_cost;
+      if (last_cost > longest) longest = last_cost;
+      pairs += ncc + 1;
+      if (ncc + 1 > most) most = ncc + 1;
+    }
+    if (pairs > pairs_cap || most > kMaxChunks) continue;
+    ctas *= Hkv; total *= Hkv;
+    const double spread = (double)total / n_sm + 0.5 * longest;
+    const double t = ctas <= n_sm ? (double)longest : (spread > longest ? spread : (double)longest);
+    if (best == 0 || t < best_t) { best = chunk; best_t = t; }
+  }
+  return best;
+}
+
 cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, const AttnUmmaMaps* maps, int* status, cudaStream_t st) {
   AttnArgs a;
   a.p = p;
@@ -320,11 +367,7 @@ cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, cons
   if (max_chunks > kMaxChunks) return cudaErrorInvalidValue;
   dim3 grid(max_chunks, p.Hkv, p.B);
   cudaError_t e;
-  // The tcgen05 split pays a few microseconds of set-up per CTA (barriers, tensor memory, first loads): it wins
-  // from a few thousand 64-key tiles on (batch 4 x 8192 keys: 75 vs 89 us; batch 1 x 4096 keys: 23.6 vs 21.1 us).
-  long long key_tiles = 0;
-  for (int b = 0; b < p.B; ++b) key_tiles += (seq_lens_host[b] + 63) / 64;
-  if (maps != nullptr && p.dh == 128 && key_tiles * p.Hkv >= 2048) {
+  if (attn_uses_umma(p.B, p.Hkv, p.dh, seq_lens_host, maps != nullptr)) {
     AttnUmmaArgs u;
     u.a = a;
     u.mapQhi = maps->mapQhi; u.mapQlo = maps->mapQlo; u.mapK = maps->mapK; u.mapV = maps->mapV; u.mapKn = maps->mapKn; u.mapVn = maps->mapVn;

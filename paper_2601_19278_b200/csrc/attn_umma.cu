@@ -4,8 +4,10 @@
 // both; what changes is the data path, because at batch > 1 that kernel is bound by the issue rate of its
 // mma.sync pairs (tensor pipe 42 % busy at 2.1 TB/s on 16 sequences):
 //   * a CTA runs two (sequence, KV head, chunk) pipelines side by side -- two consecutive chunks of one sequence,
-//     which share the Q tile -- each with its own producer thread (TMA, 128-byte swizzle, two K and two V stages
-//     of 64 keys), MMA issuer thread, and four softmax warps;
+//     which share the Q tile -- each with its own producer thread (TMA, 128-byte swizzle, three K and two V stages
+//     of 64 keys, loaded independently: a K stage is free once its scores are in tensor memory, a full tile earlier
+//     than the V stage of the same keys, and its refill has to cover the HBM latency before the next-but-one score
+//     MMA), MMA issuer thread, and four softmax warps;
 //   * the hi and lo parts of an operand are stacked along M: rows 32 q + i of the 128-row Q tile hold Q_hi of query
 //     row 16 q + i, rows 32 q + 16 + i hold Q_lo of the same row (i < 16, q = warp quarter), so ONE tcgen05.mma
 //     128 x 64 (k = 128) leaves q_hi.k in tensor-memory lane 32 q + i and q_lo.k in lane 32 q + 16 + i: the two
@@ -33,8 +35,10 @@ constexpr int kAuThreads = 384;                 // warps 0/2: producers, 1/3: MM
 constexpr int kAuQ = 128 * 128 * 2;             // 128 operand rows (hi and lo of 64 query rows) x 128: two 64-column halves
 constexpr int kAuP = 128 * 64 * 2;              // 128 operand rows (hi and lo of 64 query rows) x 64 keys
 constexpr int kAuKV = 64 * 128 * 2;             // 64 keys x 128: two 64-column halves
-// Q | P [pipeline][buffer] | K [pipeline][stage] | V [pipeline][stage]
-constexpr size_t kAuSmem = (size_t)kAuQ + 4 * kAuP + 8 * kAuKV + 1024;
+constexpr int kAuKStages = 3, kAuVStages = 2;
+// Q | P [pipeline] | K [pipeline][stage] | V [pipeline][stage].  One P tile per pipeline is enough: the MMAs that
+// read it finish a few hundred cycles after it is complete, long before the next tile's weights exist.
+constexpr size_t kAuSmem = (size_t)kAuQ + 2 * kAuP + 2 * (kAuKStages + kAuVStages) * kAuKV + 1024;
 
 __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_constant__ AttnUmmaArgs a) {
   const AttnParams& p = a.a.p;
@@ -42,10 +46,10 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = sm;
   uint8_t* sP = sm + kAuQ;
-  uint8_t* sK = sP + 4 * kAuP;
-  uint8_t* sV = sK + 4 * kAuKV;
-  __shared__ uint64_t q_full, k_full[2][2], k_empty[2][2], v_full[2][2], v_empty[2][2];
-  __shared__ uint64_t s_full[2][2], s_empty[2][2], p_full[2][2], pv_done[2][2];
+  uint8_t* sK = sP + 2 * kAuP;
+  uint8_t* sV = sK + 2 * kAuKStages * kAuKV;
+  __shared__ uint64_t q_full, k_full[2][kAuKStages], k_empty[2][kAuKStages], v_full[2][2], v_empty[2][2];
+  __shared__ uint64_t s_full[2][2], s_empty[2][2], p_full[2], pv_done[2];
   __shared__ uint32_t tmem_base;
   __shared__ int abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -59,12 +63,14 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
 
   if (threadIdx.x == 0) {
     mbar_init(&q_full, 1);
-    for (int pl = 0; pl < 2; ++pl)
+    for (int pl = 0; pl < 2; ++pl) {
+      for (int s = 0; s < kAuKStages; ++s) { mbar_init(&k_full[pl][s], 1); mbar_init(&k_empty[pl][s], 1); }
       for (int s = 0; s < 2; ++s) {
-        mbar_init(&k_full[pl][s], 1); mbar_init(&k_empty[pl][s], 1); mbar_init(&v_full[pl][s], 1); mbar_init(&v_empty[pl][s], 1);
+        mbar_init(&v_full[pl][s], 1); mbar_init(&v_empty[pl][s], 1);
         mbar_init(&s_full[pl][s], 1); mbar_init(&s_empty[pl][s], 4);     // one arrival per softmax warp
-        mbar_init(&p_full[pl][s], 4); mbar_init(&pv_done[pl][s], 1);
       }
+      mbar_init(&p_full[pl], 4); mbar_init(&pv_done[pl], 1);
+    }
     abort_flag = 0;
     fence_barrier_init();
   }
@@ -89,20 +95,24 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
     const int row0 = is_new ? (b * p.Hkv + hk) * 16 : (int)(((long long)b * p.Hkv + hk) * p.P_cap) + k_begin;
     const CUtensorMap* mk = is_new ? &a.mapKn : &a.mapK;
     const CUtensorMap* mv = is_new ? &a.mapVn : &a.mapV;
-    auto load_tile = [&](int t) {
-      const int s = t & 1;
-      uint8_t* kd = sK + (pl * 2 + s) * kAuKV;
-      uint8_t* vd = sV + (pl * 2 + s) * kAuKV;
+    auto load_k = [&](int t, int s) {
+      uint8_t* kd = sK + (pl * kAuKStages + s) * kAuKV;
       mbar_expect_tx(&k_full[pl][s], kAuKV);
       tma_load_2d(kd, mk, &k_full[pl][s], 0, row0 + t * 64);
       tma_load_2d(kd + kAuKV / 2, mk, &k_full[pl][s], 64, row0 + t * 64);
+    };
+    auto load_v = [&](int t) {
+      const int s = t & 1;
+      uint8_t* vd = sV + (pl * 2 + s) * kAuKV;
       mbar_expect_tx(&v_full[pl][s], kAuKV);
       tma_load_2d(vd, mv, &v_full[pl][s], 0, row0 + t * 64);
       tma_load_2d(vd + kAuKV / 2, mv, &v_full[pl][s], 64, row0 + t * 64);
     };
-    int t = 0;
-    if (!is_new)
-      for (; t < n_t && t < 2; ++t) load_tile(t);
+    // the first tiles (K 0, 1, 2 and V 0, 1) find their stages free
+    if (!is_new) {
+      for (int t = 0; t < n_t && t < kAuKStages; ++t) load_k(t, t);
+      for (int t = 0; t < n_t && t < 2; ++t) load_v(t);
+    }
     pdl_wait();
     if (pl == 0) {
       const int q_row = (b * p.Hq + hk * G) * p.K;
@@ -114,32 +124,42 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
           tma_load_2d(d + 16 * 128, &a.mapQlo, &q_full, ch * 64, q_row + 16 * q4);
         }
     }
-    for (; t < n_t; ++t) {
-      const int s = t & 1;
-      if (t >= 2) {
-        if (!ta_wait(&k_empty[pl][s], ((t >> 1) - 1) & 1, &abort_flag)) break;
-        if (!ta_wait(&v_empty[pl][s], ((t >> 1) - 1) & 1, &abort_flag)) break;
+    if (is_new) { load_k(0, 0); load_v(0); }     // one tile, written by the QKV kernel
+    // then, in the order in which the stages come free: K of tile t + 1 (after the scores of tile t - 2), V of tile t
+    // (after the P V product of tile t - 2)
+    int ks = 0, kph = 0;      // stage and round of K tile t + 1
+    for (int t = 2; t < n_t; ++t) {
+      if (t + 1 < n_t) {
+        if (!ta_wait(&k_empty[pl][ks], kph & 1, &abort_flag)) break;
+        load_k(t + 1, ks);
+        if (++ks == kAuKStages) { ks = 0; ++kph; }
       }
-      load_tile(t);
+      if (t < n_t) {
+        if (!ta_wait(&v_empty[pl][t & 1], ((t >> 1) - 1) & 1, &abort_flag)) break;
+        load_v(t);
+      }
     }
   } else if ((warp == 1 || warp == 3) && lane == 0 && pl_on) {
     // ---- MMA issuer of pipeline pl
     constexpr uint32_t idesc_s = idesc_bf16(128, 64), idesc_o = idesc_bf16(128, 128) | kIdescBMnMajor;
     const uint64_t dq0 = desc_sw128(smem_u32(sQ)), dq1 = desc_sw128(smem_u32(sQ + kAuQ / 2));
     bool ok = ta_wait(&q_full, 0, &abort_flag);
+    int ks = 0, kph = 0;                     // stage and round of the next K tile
     auto issue_s = [&](int t) -> bool {      // S[t & 1] = [Q_hi ; Q_lo] K_t^T
       const int s = t & 1;
-      if (!ta_wait(&k_full[pl][s], (t >> 1) & 1, &abort_flag)) return false;
+      if (!ta_wait(&k_full[pl][ks], kph & 1, &abort_flag)) return false;
       if (t >= 2 && !ta_wait(&s_empty[pl][s], ((t >> 1) - 1) & 1, &abort_flag)) return false;
       tc_fence_after();
-      const uint64_t dk0 = desc_sw128(smem_u32(sK + (pl * 2 + s) * kAuKV)), dk1 = desc_sw128(smem_u32(sK + (pl * 2 + s) * kAuKV + kAuKV / 2));
+      const uint32_t ka = smem_u32(sK + (pl * kAuKStages + ks) * kAuKV);
+      const uint64_t dk0 = desc_sw128(ka), dk1 = desc_sw128(ka + kAuKV / 2);
       const uint32_t acc = tmem + pl * 256 + s * 64;
 #pragma unroll
       for (int k = 0; k < 4; ++k) mma_f16(acc, dq0 + 2 * k, dk0 + 2 * k, idesc_s, k > 0 ? 1u : 0u);
 #pragma unroll
       for (int k = 0; k < 4; ++k) mma_f16(acc, dq1 + 2 * k, dk1 + 2 * k, idesc_s, 1u);
       mma_commit(&s_full[pl][s]);
-      mma_commit(&k_empty[pl][s]);
+      mma_commit(&k_empty[pl][ks]);
+      if (++ks == kAuKStages) { ks = 0; ++kph; }
       return true;
     };
     if (ok) ok = issue_s(0);
@@ -147,13 +167,13 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       const int s = t & 1;
       if (t + 1 < n_t && !issue_s(t + 1)) break;
       if (!ta_wait(&v_full[pl][s], (t >> 1) & 1, &abort_flag)) break;
-      if (!ta_wait(&p_full[pl][s], (t >> 1) & 1, &abort_flag)) break;
+      if (!ta_wait(&p_full[pl], t & 1, &abort_flag)) break;
       tc_fence_after();
       const uint64_t dv = desc_sw128_mn(smem_u32(sV + (pl * 2 + s) * kAuKV), kAuKV / 2);
-      const uint64_t dp = desc_sw128(smem_u32(sP + (pl * 2 + s) * kAuP));
+      const uint64_t dp = desc_sw128(smem_u32(sP + pl * kAuP));
 #pragma unroll
       for (int k = 0; k < 4; ++k) mma_f16(tmem + pl * 256 + 128, dp + 2 * k, dv + 128 * k, idesc_o, (t > 0 || k > 0) ? 1u : 0u);
-      mma_commit(&pv_done[pl][s]);
+      mma_commit(&pv_done[pl]);
       mma_commit(&v_empty[pl][s]);
     }
   } else if (warp >= 4 && pl_on) {
@@ -232,10 +252,9 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
           }
         }
       }
-      // this P buffer was last read by the MMAs of tile t - 2
-      if (t >= 2 && !ta_wait(&pv_done[pl][s], ((t >> 1) - 1) & 1, &abort_flag)) { ok = false; break; }
+      // the P tile was last read by the MMAs of tile t - 1, after which O holds tiles 0 .. t - 1
+      if (t >= 1 && !ta_wait(&pv_done[pl], (t - 1) & 1, &abort_flag)) { ok = false; break; }
       if (t > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rescale this warp's O rows (hi and lo parts) in tensor memory
-        if (!ta_wait(&pv_done[pl][s ^ 1], ((t - 1) >> 1) & 1, &abort_flag)) { ok = false; break; }   // O holds tiles 0..t-1
         tc_fence_after();
 #pragma unroll 1
         for (int cb = 0; cb < 128; cb += 16) {
@@ -252,7 +271,7 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       // row 32 wq + 16 + i = lo parts; rows of 128 bytes, 16-byte chunk ch of operand row x stored at chunk
       // ch ^ (x & 7) (the 128-byte swizzle).  This thread writes the 4 chunks of its 32 columns into both rows.
       const int xrow = wq * 32 + (lane & 15);
-      uint8_t* ph = sP + (pl * 2 + s) * kAuP + xrow * 128;
+      uint8_t* ph = sP + pl * kAuP + xrow * 128;
       uint8_t* plo = ph + 16 * 128;
 #pragma unroll
       for (int cq = 0; cq < 4; ++cq) {
@@ -272,9 +291,9 @@ __global__ void __launch_bounds__(kAuThreads, 1) attn_umma_kernel(const __grid_c
       fence_async_smem();
       tc_fence_before();
       __syncwarp();                          // every lane's P chunks and fences precede the warp's one arrival
-      if (lane == 0) mbar_arrive(&p_full[pl][s]);
+      if (lane == 0) mbar_arrive(&p_full[pl]);
     }
-    if (ok && ta_wait(&pv_done[pl][(n_t - 1) & 1], ((n_t - 1) >> 1) & 1, &abort_flag)) {
+    if (ok && ta_wait(&pv_done[pl], (n_t - 1) & 1, &abort_flag)) {
       tc_fence_after();
       // the chunk's partial: (reference maximum, sum, un-normalised output), merged by attn_combine_kernel.  The
       // output row is the sum of the hi part's and the lo part's accumulator rows (this lane's and its partner's).

@@ -270,6 +270,9 @@ cudaError_t attention_setup();  // once per device: opt in to the kernels' dynam
 // (d_h = 128, batches with a few thousand key tiles) the split runs on the tcgen05 kernel, otherwise on the warp-MMA one
 // that a single sequence's few chunks are faster on; the combine is the same.
 cudaError_t launch_attention(const AttnParams& p, const int* seq_lens_host, const AttnUmmaMaps* maps, int* status, cudaStream_t st);
+// which split kernel launch_attention picks, and the chunk length that suits the tcgen05 one (0: none fits pairs_cap)
+bool attn_uses_umma(int B, int Hkv, int dh, const int* seq_lens_host, bool have_maps);
+int attn_umma_chunk_keys(int B, int Hkv, const int* seq_lens_host, int n_sm, int pairs_cap);
 
 // ---------------------------------------------------------------------------------------------
 // LM head with fused log-softmax / top-k partials, and the merge that finishes them.
