@@ -44,6 +44,7 @@ struct Workspace {
   float* pss = nullptr;         // prefill: per-row partial sums of squares of g [kPrefillPassRows, h/256]
   float* lm_pieces = nullptr;   // [SMs][128][MPmax] partial logits of vocabulary tiles cut between CTAs
   int* lm_flags = nullptr;      // [SMs] launch tag of each CTA's piece
+  unsigned long long* lm_bound = nullptr;   // [128][kLmBoundSlots] lower bounds the LM head's CTAs share (many token rows)
 };
 
 }  // namespace
@@ -233,6 +234,7 @@ size_t layout_workspace(const dart_config& c, size_t part_max_floats, int attn_p
   TAKE(ml_part, float*, (size_t)attn_pairs_cap * c.n_kv_heads * 64 * 2 * sizeof(float));
   TAKE(lm_pieces, float*, (size_t)lm_grid * 128 * MPmax * sizeof(float));
   TAKE(lm_flags, int*, (size_t)lm_grid * sizeof(int));
+  TAKE(lm_bound, unsigned long long*, (size_t)128 * kLmBoundSlots * sizeof(unsigned long long));
   TAKE(lm_stats, float*, (size_t)lm_grid * MPmax * 2 * sizeof(float));
   TAKE(lm_key, float*, (size_t)lm_grid * MPmax * 32 * sizeof(float));
   TAKE(lm_y, float*, (size_t)lm_grid * MPmax * 32 * sizeof(float));
@@ -749,7 +751,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
           return fail_cuda(h, e);
         h->lmx_M = M;
       }
-      e = launch_lm_head_dense(lp, h->map_lm256, h->lmx_hi, h->lmx_lo, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
+      e = launch_lm_head_dense(lp, h->map_lm256, h->lmx_hi, h->lmx_lo, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, ws.lm_bound, st);
     } else {
       e = launch_lm_head_umma(lp, h->map_lm, h->maps_gu.Xhi, ws.lm_pieces, ws.lm_flags, ++h->lm_tag, ws.status, st);
     }

@@ -298,14 +298,17 @@ struct LmUmmaArgs {
   int KB; long long U;
   float* pieces; int* flags; int tag;
   int* status;
+  unsigned long long* bound;   // lm_head_dense_kernel: [128 token rows][kLmBoundSlots] shared lower bounds (tag << 32 | ordered key)
 };
+constexpr int kLmBoundSlots = 40;   // topk + 7 of them are used
 cudaError_t launch_lm_head_umma(const LmParams& p, const CUtensorMap& mapW, const CUtensorMap& mapX,
                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st);
 // The LM head for 33..128 token rows with the operands swapped (token rows on the MMA's M side; lm_head.cu).
 // mapW256: the weight matrix with boxes of 256 rows; mapXhi / mapXlo: 2-D maps [M][Kd], boxes of 128 rows;
 // pieces: [grid][128][256] fp32.  The per-CTA results are laid out for MP = 128 token rows.
+// bound: kLmBoundSlots 64-bit words per token row, zero before the first launch; tags must differ between launches.
 cudaError_t launch_lm_head_dense(const LmParams& p, const CUtensorMap& mapW256, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
-                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st);
+                                 float* pieces, int* flags, int tag, int* status, unsigned long long* bound, cudaStream_t st);
 cudaError_t topk_merge_setup(int max_grid);  // once per device
 cudaError_t launch_topk_merge(const LmParams& p, cudaStream_t st);
 

@@ -16,6 +16,7 @@
 #include "common.cuh"
 #include "kernels.h"
 #include "umma.cuh"
+#include "select.cuh"
 
 namespace dart {
 
@@ -510,6 +511,33 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
     l_thr[half * 128 + tok] = -INFINITY;
     int n_list = 0;
     const int topk = p.topk;
+    // A bound shared by all CTAs.  A CTA sees ~1000 vocabulary rows of a token, so its own thresholds let one logit
+    // in five through, and the insertions (~2300 cycles per warp round: cycle counters) were 4/5 of this role's time.
+    // Every (CTA, half) publishes the largest key it has met so far for the token -- at temperature > 0 a lower
+    // bound of it -- into slot (2 c + half) mod (topk + 7) of the token's row of `bound` (atomic max; the launch's
+    // tag in the upper word makes older launches' values invalid without a reset).  The slots hold keys of distinct
+    // vocabulary rows, so the topk-th largest slot -- the 8th smallest -- is at most the topk-th largest key of the
+    // whole vocabulary: whatever is below it cannot be in the result.  After one 16-logit chunk per thread that is
+    // already the 99th percentile.  A stale or missing value only prunes less: which candidates a CTA keeps depends
+    // on timing, the merged top list does not.
+    const int n_slots = topk + 7;
+    unsigned long long* g_row = a.bound + (size_t)tok * kLmBoundSlots;
+    const int g_slot = (2 * c + half) % n_slots;
+    const unsigned long long g_tag = (unsigned long long)(uint32_t)a.tag << 32;
+    float tau = -INFINITY, pub = -INFINITY;
+    int n_own = 0;                               // chunks of owned tiles folded so far
+    auto refresh_tau = [&]() {
+      float s8[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) s8[q] = INFINITY;
+      for (int i = 0; i < n_slots; ++i) {
+        const unsigned long long w = __ldcg(g_row + i);
+        float v = (w >> 32) == (g_tag >> 32) ? float_unorder((uint32_t)w) : -INFINITY;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) { const float lo = fminf(s8[q], v); v = fmaxf(s8[q], v); s8[q] = lo; }
+      }
+      tau = s8[7];
+    };
     auto worse = [&](int x, int y) { return cand_before(my_key[y], my_id[y], my_key[x], my_id[x]); };   // entry x ranks after entry y
     auto heap_insert = [&](float ke, int ie) {
       if (n_list < topk) {                       // grow: the new leaf rises while it ranks after its parent
@@ -609,12 +637,13 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
         // > 0 the key is y + G(u): a fast evaluation of G decides with a margin 10x its error bound (u in
         // [2^-14, 1 - 2^-8]: |error| < 1.2e-4; other u always pass); the exact fp32 G is computed for those only.
         const bool full = n_list == topk;
-        const float o_key = l_thr[(half ^ 1) * 128 + tok];             // the other half's threshold (or -inf)
+        const float o_key = fmaxf(l_thr[(half ^ 1) * 128 + tok], tau);   // the other half's threshold and the shared bound (or -inf)
         const float t_key = full ? my_key[0] : -INFINITY;
         const int t_id = full ? my_id[0] : 0x7fffffff;
         if (full) l_thr[half * 128 + tok] = t_key;
         uint32_t may = 0u;
         uint32_t bits[16];
+        float kmax = -INFINITY;                  // a lower bound of the chunk's largest key
         if (p.gumbel) {
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
@@ -626,6 +655,7 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
               const float gq = -__logf(-__logf(((float)m + 0.5f) * (1.f / 16777216.f)));
               const bool safe = m >= 1024u && m <= (1u << 24) - 65536u;
               const float kq = y[4 * q4 + q] + gq + 1e-3f;
+              if (safe) kmax = fmaxf(kmax, kq - 2e-3f);
               if ((!full || !safe || kq >= t_key) && (!safe || kq >= o_key)) may |= 1u << (4 * q4 + q);
             }
           }
@@ -633,10 +663,15 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             bits[j] = 0u;
+            kmax = fmaxf(kmax, y[j]);
             if ((!full || cand_before(y[j], v0 + j, t_key, t_id)) && y[j] >= o_key) may |= 1u << j;
           }
         }
         if (!live) may = 0u;
+        if (live && kmax > pub) {
+          atomicMax(g_row + g_slot, g_tag | float_order(kmax));
+          pub = kmax;
+        }
 #pragma unroll 1
         while (may != 0u) {                      // one candidate per round; rows of a warp go through their rounds together
           const int j = __ffs(may) - 1;
@@ -648,6 +683,9 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
           const float kj = p.gumbel ? yj + gumbel_from_bits(bj) : yj;
           if (kj >= o_key) heap_insert(kj, v0 + j);
         }
+        // the shared bound is read again after 1, 2, 4, 8 chunks and then once per tile half
+        ++n_own;
+        if (live && (n_own <= 8 ? (n_own & (n_own - 1)) == 0 : (n_own & 7) == 0)) refresh_tau();
       }
       if (!owner) {
         __threadfence();
@@ -719,10 +757,11 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
 }
 
 cudaError_t launch_lm_head_dense(const LmParams& pin, const CUtensorMap& mapW256, const CUtensorMap& mapXhi, const CUtensorMap& mapXlo,
-                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st) {
+                                 float* pieces, int* flags, int tag, int* status, unsigned long long* bound, cudaStream_t st) {
   LmUmmaArgs a;
   memset(&a, 0, sizeof(a));
   a.p = pin;
+  a.bound = bound;
   a.mapW = mapW256; a.mapXhi = mapXhi; a.mapXlo = mapXlo;
   a.KB = (pin.Kd + 63) / 64;
   a.U = (long long)((pin.V + 255) / 256) * a.KB;
