@@ -377,13 +377,16 @@ cudaError_t launch_lm_head_umma(const LmParams& pin, const CUtensorMap& mapW, co
 // ------------------------------------------------------------------------------------------------------
 // Two read-out threads per token row, one per half of a tile's 256 columns (warps 4-7 and 8-11), each with its own
 // statistics and list: one warp per scheduler ran the fold at several cycles per instruction and was the longest
-// part of the kernel; two halve that.  The second set of lists takes the shared memory of the ring's third stage
-// (three stages without the fold: 320 us; two: 372 us; fold on one warp set: 748 us).
-constexpr int kLmDenseStages = 2;
+// part of the kernel; two halve that (fold on one warp set: 748 us).  The two sets of lists leave room for 160 KB of
+// stages: three of weights and two of activations, in rings of their own (see the producer).
+constexpr int kLmDenseWStages = 3, kLmDenseXStages = 2;
 constexpr int kLmDenseThreads = 384;
-constexpr int kLmDenseStageBytes = 2 * 128 * 64 * 2 + 256 * 64 * 2;   // hi tokens, lo tokens, 256 vocabulary rows
-constexpr int kLmDenseListStride = 33;                                  // floats per token row of the lists (no bank conflicts)
-constexpr size_t kLmDenseSmem = (size_t)kLmDenseStages * kLmDenseStageBytes + 1024 + 2 * 2 * 128 * kLmDenseListStride * 4 + 2 * 128 * 4;
+constexpr int kLmDenseXBytes = 2 * 128 * 64 * 2;   // a stage of activations: hi tokens, lo tokens
+constexpr int kLmDenseWBytes = 256 * 64 * 2;       // a stage of weights: 256 vocabulary rows
+constexpr int kLmDenseRingBytes = kLmDenseXStages * kLmDenseXBytes + kLmDenseWStages * kLmDenseWBytes;
+// lists: entry e of token row t of half h at [h][e][t] -- a thread's entries are 128 floats apart, so whichever
+// entries the lanes of a warp touch, they touch 32 different banks
+constexpr size_t kLmDenseSmem = (size_t)kLmDenseRingBytes + 1024 + 2 * 2 * 32 * 128 * 4 + 2 * 128 * 4;
 
 // (key, id) a precedes (key, id) b in the candidate order: larger key first, then smaller id
 __device__ __forceinline__ bool cand_before(float ka, int ia, float kb, int ib) { return ka > kb || (ka == kb && ia < ib); }
@@ -392,10 +395,13 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
   const LmParams& p = a.p;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  float* l_key = reinterpret_cast<float*>(ring + (size_t)kLmDenseStages * kLmDenseStageBytes);   // [2 halves][128][33]
-  int* l_id = reinterpret_cast<int*>(l_key + 2 * 128 * kLmDenseListStride);                       // [2 halves][128][33]
-  volatile float* l_thr = reinterpret_cast<volatile float*>(l_id + 2 * 128 * kLmDenseListStride);  // [2 halves][128] published thresholds
-  __shared__ uint64_t full[kLmDenseStages], empty[kLmDenseStages], acc_full[2], acc_empty[2];
+  uint8_t* ring_x = ring;                                                  // [2][hi | lo]
+  uint8_t* ring_w = ring + kLmDenseXStages * kLmDenseXBytes;               // [3]
+  float* l_key = reinterpret_cast<float*>(ring + kLmDenseRingBytes);       // [2 halves][32][128]
+  int* l_id = reinterpret_cast<int*>(l_key + 2 * 32 * 128);                // [2 halves][32][128]
+  volatile float* l_thr = reinterpret_cast<volatile float*>(l_id + 2 * 32 * 128);  // [2 halves][128] published thresholds
+  __shared__ uint64_t full_w[kLmDenseWStages], empty_w[kLmDenseWStages], full_x[kLmDenseXStages], empty_x[kLmDenseXStages];
+  __shared__ uint64_t acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base;
   __shared__ int abort_flag, s_bad;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
@@ -405,19 +411,20 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
   constexpr int kXBytes = 128 * 64 * 2;
 
   if (tid == 0) {
-    for (int s = 0; s < kLmDenseStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < kLmDenseWStages; ++s) { mbar_init(&full_w[s], 1); mbar_init(&empty_w[s], 1); }
+    for (int s = 0; s < kLmDenseXStages; ++s) { mbar_init(&full_x[s], 1); mbar_init(&empty_x[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 256); }
     abort_flag = 0;
     s_bad = 0;
     fence_barrier_init();
-    // the producer fills the ring's weight slots before anything else of the CTA's setup
+    // the producer fills the weight stages before anything else of the CTA's setup
     const int n = (int)(u1 - u0);
-    const int pre = n < kLmDenseStages ? n : kLmDenseStages;
+    const int pre = n < kLmDenseWStages ? n : kLmDenseWStages;
     const uint64_t wpol = l2_policy_evict_first();
     int tile = (int)(u0 / KB), kb = (int)(u0 % KB);
     for (int it = 0; it < pre; ++it) {
-      mbar_expect_tx(&full[it], kLmDenseStageBytes);
-      tma_load_2d_hint(ring + (size_t)it * kLmDenseStageBytes + 2 * kXBytes, &a.mapW, &full[it], kb * 64, tile * 256, wpol);
+      mbar_expect_tx(&full_w[it], kLmDenseWBytes);
+      tma_load_2d_hint(ring_w + (size_t)it * kLmDenseWBytes, &a.mapW, &full_w[it], kb * 64, tile * 256, wpol);
       if (++kb == KB) { kb = 0; ++tile; }
     }
   }
@@ -428,36 +435,47 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
   const uint32_t tmem = tmem_base;
 
   if (warp == 0 && lane == 0) {
-    // ---- producer
+    // ---- producer.  Weights and activations have rings of their own: three weight stages, so that a refill has two
+    // stages' worth of MMAs to arrive from HBM, and two for the activation slices, which come from L2.  Unit it reads
+    // weight stage it mod 3 and activation stage it mod 2.  Cycle counters at 128 token rows: the MMA thread spends
+    // ~960 cycles per stage issuing (the eight MMAs of a stage take 1024 on the tensor pipe) and waits 270 for weights
+    // and 620 for activations (985 with two stages of both).  The launch did not get shorter for it: it runs under the
+    // power cap (600 000 cycles in 368 us on the global timer -- 1.6 GHz -- in a run of three steps, fewer MHz still
+    // in a long one), where fewer stalled cycles buy a lower clock.
     const int n = (int)(u1 - u0);
-    const int pre = n < kLmDenseStages ? n : kLmDenseStages;
     const uint64_t wpol = l2_policy_evict_first();
-    int tile, kb;
     pdl_wait();
-    tile = (int)(u0 / KB); kb = (int)(u0 % KB);
-    for (int it = 0; it < pre; ++it) {
-      uint8_t* st = ring + (size_t)it * kLmDenseStageBytes;
-      tma_load_2d(st, &a.mapXhi, &full[it], kb * 64, 0);
-      tma_load_2d(st + kXBytes, &a.mapXlo, &full[it], kb * 64, 0);
-      if (++kb == KB) { kb = 0; ++tile; }
-    }
-    int s = pre == kLmDenseStages ? 0 : pre, ph = pre == kLmDenseStages ? 1 : 0;
-    for (int it = pre; it < n; ++it) {
-      if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
-      uint8_t* st = ring + (size_t)s * kLmDenseStageBytes;
-      mbar_expect_tx(&full[s], kLmDenseStageBytes);
-      tma_load_2d_hint(st + 2 * kXBytes, &a.mapW, &full[s], kb * 64, tile * 256, wpol);
-      tma_load_2d(st, &a.mapXhi, &full[s], kb * 64, 0);
-      tma_load_2d(st + kXBytes, &a.mapXlo, &full[s], kb * 64, 0);
-      if (++s == kLmDenseStages) { s = 0; ++ph; }
-      if (++kb == KB) { kb = 0; ++tile; }
+    int xkb = (int)(u0 % KB);                                  // k-block of the next activation slice
+    int wt = (int)(u0 / KB), wkb = (int)(u0 % KB);             // tile and k-block of the next weight stage
+    auto load_x = [&](int s) {
+      uint8_t* st = ring_x + (size_t)s * kLmDenseXBytes;
+      mbar_expect_tx(&full_x[s], kLmDenseXBytes);
+      tma_load_2d(st, &a.mapXhi, &full_x[s], xkb * 64, 0);
+      tma_load_2d(st + kXBytes, &a.mapXlo, &full_x[s], xkb * 64, 0);
+      if (++xkb == KB) xkb = 0;
+    };
+    for (int it = 0; it < n && it < kLmDenseXStages; ++it) load_x(it);
+    for (int it = 0; it < n && it < kLmDenseWStages; ++it)     // already requested above
+      if (++wkb == KB) { wkb = 0; ++wt; }
+    // from unit 2 on, both refills wait for the MMAs of unit it - 2: weights of unit it + 1, activations of unit it
+    int ws = 0, wph = 0;
+    for (int it = 2; it < n; ++it) {
+      if (it + 1 < n) {
+        if (!mbar_wait(&empty_w[ws], wph & 1, &abort_flag)) break;
+        mbar_expect_tx(&full_w[ws], kLmDenseWBytes);
+        tma_load_2d_hint(ring_w + (size_t)ws * kLmDenseWBytes, &a.mapW, &full_w[ws], wkb * 64, wt * 256, wpol);
+        if (++wkb == KB) { wkb = 0; ++wt; }
+        if (++ws == kLmDenseWStages) { ws = 0; ++wph; }
+      }
+      if (!mbar_wait(&empty_x[it & 1], ((it >> 1) - 1) & 1, &abort_flag)) break;
+      load_x(it & 1);
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer: D[token, vocabulary row] += (X_hi + X_lo)[token, k] * W[vocabulary row, k]
     constexpr uint32_t idesc = idesc_bf16(128, 256);
     const int n = (int)(u1 - u0);
     int visit = -1, buf = 0, tile = -1;
-    int t = (int)(u0 / KB), kb = (int)(u0 % KB), s = 0, ph = 0;
+    int t = (int)(u0 / KB), kb = (int)(u0 % KB), ws = 0, wph = 0;
     bool ok = true;
     for (int it = 0; it < n && ok; ++it) {
       bool first = false;
@@ -472,17 +490,20 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
           tc_fence_after();
         }
       }
-      if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
+      const int xs = it & 1;
+      if (!mbar_wait(&full_w[ws], wph & 1, &abort_flag)) { ok = false; break; }
+      if (!mbar_wait(&full_x[xs], (it >> 1) & 1, &abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const uint32_t sa = smem_u32(ring + (size_t)s * kLmDenseStageBytes);
-      const uint64_t hd = desc_sw128(sa), ld = desc_sw128(sa + kXBytes), wd = desc_sw128(sa + 2 * kXBytes);
+      const uint32_t xa = smem_u32(ring_x + (size_t)xs * kLmDenseXBytes);
+      const uint64_t hd = desc_sw128(xa), ld = desc_sw128(xa + kXBytes), wd = desc_sw128(smem_u32(ring_w + (size_t)ws * kLmDenseWBytes));
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         mma_f16(tmem + buf * 256, hd + 2 * k, wd + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
         mma_f16(tmem + buf * 256, ld + 2 * k, wd + 2 * k, idesc, 1u);
       }
-      mma_commit(&empty[s]);
-      if (++s == kLmDenseStages) { s = 0; ++ph; }
+      mma_commit(&empty_w[ws]);
+      mma_commit(&empty_x[xs]);
+      if (++ws == kLmDenseWStages) { ws = 0; ++wph; }
       if (++kb == KB) { kb = 0; ++t; }
     }
     if (ok && tile >= 0) mma_commit(&acc_full[buf]);
@@ -491,8 +512,8 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
     // every tile, with statistics and a list of its own (the two halves are merged at the end)
     const int wq = warp & 3, half = (warp - 4) >> 2, tok = wq * 32 + lane, et = tid - 128;
     const bool live = tok < p.M;
-    float* my_key = l_key + (half * 128 + tok) * kLmDenseListStride;
-    int* my_id = l_id + (half * 128 + tok) * kLmDenseListStride;
+    float* my_key = l_key + half * 32 * 128 + tok;      // entry e at my_key[(e * 128) * 128]
+    int* my_id = l_id + half * 32 * 128 + tok;
     pdl_wait();
     float rstd = 0.f;
     if (live) {  // the final RMSNorm's 1/rms from the previous kernel's sums of squares (same order everywhere)
@@ -538,28 +559,28 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
       }
       tau = s8[7];
     };
-    auto worse = [&](int x, int y) { return cand_before(my_key[y], my_id[y], my_key[x], my_id[x]); };   // entry x ranks after entry y
+    auto worse = [&](int x, int y) { return cand_before(my_key[(y) * 128], my_id[(y) * 128], my_key[(x) * 128], my_id[(x) * 128]); };   // entry x ranks after entry y
     auto heap_insert = [&](float ke, int ie) {
       if (n_list < topk) {                       // grow: the new leaf rises while it ranks after its parent
         int i = n_list++;
         while (i > 0) {
           const int up = (i - 1) >> 1;
-          if (!cand_before(my_key[up], my_id[up], ke, ie)) break;          // the parent does not rank before it: stop
-          my_key[i] = my_key[up]; my_id[i] = my_id[up];
+          if (!cand_before(my_key[(up) * 128], my_id[(up) * 128], ke, ie)) break;          // the parent does not rank before it: stop
+          my_key[(i) * 128] = my_key[(up) * 128]; my_id[(i) * 128] = my_id[(up) * 128];
           i = up;
         }
-        my_key[i] = ke; my_id[i] = ie;
-      } else if (cand_before(ke, ie, my_key[0], my_id[0])) {               // replace the root, sink it
+        my_key[(i) * 128] = ke; my_id[(i) * 128] = ie;
+      } else if (cand_before(ke, ie, my_key[(0) * 128], my_id[(0) * 128])) {               // replace the root, sink it
         int i = 0;
         for (;;) {
           int ch = 2 * i + 1;
           if (ch >= topk) break;
           if (ch + 1 < topk && worse(ch + 1, ch)) ++ch;                    // the later-ranked child
-          if (!cand_before(ke, ie, my_key[ch], my_id[ch])) break;          // the new entry ranks after both children
-          my_key[i] = my_key[ch]; my_id[i] = my_id[ch];
+          if (!cand_before(ke, ie, my_key[(ch) * 128], my_id[(ch) * 128])) break;          // the new entry ranks after both children
+          my_key[(i) * 128] = my_key[(ch) * 128]; my_id[(i) * 128] = my_id[(ch) * 128];
           i = ch;
         }
-        my_key[i] = ke; my_id[i] = ie;
+        my_key[(i) * 128] = ke; my_id[(i) * 128] = ie;
       }
     };
     int visit = 0;
@@ -638,8 +659,8 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
         // [2^-14, 1 - 2^-8]: |error| < 1.2e-4; other u always pass); the exact fp32 G is computed for those only.
         const bool full = n_list == topk;
         const float o_key = fmaxf(l_thr[(half ^ 1) * 128 + tok], tau);   // the other half's threshold and the shared bound (or -inf)
-        const float t_key = full ? my_key[0] : -INFINITY;
-        const int t_id = full ? my_id[0] : 0x7fffffff;
+        const float t_key = full ? my_key[(0) * 128] : -INFINITY;
+        const int t_id = full ? my_id[(0) * 128] : 0x7fffffff;
         if (full) l_thr[half * 128 + tok] = t_key;
         uint32_t may = 0u;
         uint32_t bits[16];
@@ -709,23 +730,23 @@ __global__ void __launch_bounds__(kLmDenseThreads, 1) lm_head_dense_kernel(const
         s_run = (m_run == -INFINITY ? 0.f : s_run * expf(m_run - mn)) + s1 * expf(m1 - mn);
         m_run = mn;
       }
-      const float* k1 = l_key + (128 + tok) * kLmDenseListStride;
-      const int* i1 = l_id + (128 + tok) * kLmDenseListStride;
+      const float* k1 = l_key + 32 * 128 + tok;
+      const int* i1 = l_id + 32 * 128 + tok;
       const int n1 = x_n[tok];
-      for (int e1 = 0; e1 < n1; ++e1) heap_insert(k1[e1], i1[e1]);
+      for (int e1 = 0; e1 < n1; ++e1) heap_insert(k1[e1 * 128], i1[e1 * 128]);
     }
     if (live && half == 0) {
       for (int i = 1; i < n_list; ++i) {            // insertion sort of at most 32 entries
-        const float ki = my_key[i]; const int ii = my_id[i];
+        const float ki = my_key[(i) * 128]; const int ii = my_id[(i) * 128];
         int j = i - 1;
-        while (j >= 0 && cand_before(ki, ii, my_key[j], my_id[j])) { my_key[j + 1] = my_key[j]; my_id[j + 1] = my_id[j]; --j; }
-        my_key[j + 1] = ki; my_id[j + 1] = ii;
+        while (j >= 0 && cand_before(ki, ii, my_key[(j) * 128], my_id[(j) * 128])) { my_key[(j + 1) * 128] = my_key[(j) * 128]; my_id[(j + 1) * 128] = my_id[(j) * 128]; --j; }
+        my_key[(j + 1) * 128] = ki; my_id[(j + 1) * 128] = ii;
       }
       const size_t o = ((size_t)c * 128 + tok) * 32;
       for (int e = 0; e < 32; ++e) {
         const bool have = e < n_list;
-        const float key = have ? my_key[e] : -INFINITY;
-        const int id = have ? my_id[e] : 0x7fffffff;
+        const float key = have ? my_key[(e) * 128] : -INFINITY;
+        const int id = have ? my_id[(e) * 128] : 0x7fffffff;
         float yv = key;                                   // the un-perturbed logit / T of the entry
         if (have && p.gumbel) {
           const uint4 rnd = philox4x32_10(make_uint4((uint32_t)id >> 2, (uint32_t)(tok % p.K), (uint32_t)(tok / p.K), p.step), p.seed_lo, p.seed_hi);
