@@ -307,12 +307,13 @@ cudaError_t attention_setup() {
 }
 
 // Whether the step's attention runs on the tcgen05 split (attn_umma.cu).  It pays a few microseconds of set-up per
-// CTA (barriers, tensor memory, first loads) and wins from a few thousand 64-key tiles on (batch 4 x 8192 keys: 75 vs
-// 89 us; batch 1 x 4096 keys: 23.6 vs 21.1 us).
+// CTA (barriers, tensor memory, first loads) and wins from about 512 (64-key tile, KV head) pairs on (attention stage,
+// split and combine: batch 1 x 4096 keys x 8 heads 21.5 vs 23.6 us; 2048 keys 21.7 vs 21.5; batch 4 x 8192 keys 49.6
+// vs 89).
 bool attn_uses_umma(int B, int Hkv, int dh, const int* seq_lens_host, bool have_maps) {
   long long key_tiles = 0;
   for (int b = 0; b < B; ++b) key_tiles += (seq_lens_host[b] + 63) / 64;
-  return have_maps && dh == 128 && key_tiles * Hkv >= 2048;
+  return have_maps && dh == 128 && key_tiles * Hkv >= 512;
 }
 
 // Chunk length for the tcgen05 split, whose CTAs take two consecutive chunks of a sequence each and stay alone on

@@ -29,12 +29,15 @@ CASES = {
     # with row ownership: every CTA forms its own rows of SiLU(gate) * up from two accumulators
     "wide_mlp_row_ownership": syn.small_variant(C1, mlp_inter=14224, K=8, tree_budget=60, n_fresh=2),
     "hot_b4": syn.small_variant(C1, batch=4, ragged_lo=20, prefix=160, temperature=1.0),
-    # enough 64-key tiles (sum over sequences x KV heads >= 2048) for the tensor-core split-KV attention: ragged
-    # lengths (partial last tiles, sequences with fewer chunks), 16 and 40 query rows per KV head
+    # enough 64-key tiles (sum over sequences x KV heads >= 512) for the tensor-core split-KV attention: ragged
+    # lengths (partial last tiles, sequences with fewer chunks), 16 and 40 query rows per KV head; one long sequence
+    # just above that bound, cut into many short chunks
     "attn_tiles_g2": syn.small_variant(C1, hidden=512, n_q_heads=32, n_kv_heads=16, head_dim=128, mlp_inter=1376,
                                        vocab=2064, batch=8, ragged_lo=900, prefix=2000, K=8, tree_budget=60),
     "attn_tiles_g5": syn.small_variant(C1, hidden=512, n_q_heads=40, n_kv_heads=8, head_dim=128, mlp_inter=1376,
                                        vocab=2064, batch=8, ragged_lo=2100, prefix=3000, K=8, tree_budget=60),
+    "attn_tiles_b1": syn.small_variant(C1, hidden=512, n_q_heads=40, n_kv_heads=8, head_dim=128, mlp_inter=1376,
+                                       vocab=2064, batch=1, prefix=4100, K=8, tree_budget=60),
 }
 
 
