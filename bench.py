@@ -225,17 +225,12 @@ def run_ours(args):
     lm_ms += [a.elapsed_time(b) for a, b in extra]
     clocks = sampler.stop() if rank == 0 else None
 
-    # ---- end to end through the C ABI with host buffers: pinned inputs in, tree out, every step.  The session
-    # keeps the step's small inputs in one device buffer and the tree outputs in another, so a step costs one
-    # copy each way.
+    # ---- end to end through the C ABI with host buffers: dart_draft_step_host takes the step's small inputs from
+    # one pinned host buffer (one copy in), runs the forward pass and the tree, and leaves the tree in another (one
+    # copy out) before it returns.
     in_host, in_dev, out_host, out_dev, _ = ses.pack_io()
     h2d, d2h = in_host.numel(), out_host.numel()
-
-    def e2e_step(i):
-        in_dev.copy_(in_host, non_blocking=True)
-        step(i)
-        out_host.copy_(out_dev, non_blocking=True)
-        stream.synchronize()                     # the caller needs the tree before it can verify
+    e2e_step = ses.host_step(in_host, in_dev, out_host, out_dev, stream=stream)
 
     for i in range(args.warmup):
         e2e_step(i)

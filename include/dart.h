@@ -210,6 +210,27 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
  */
 int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out* out, void* cuda_stream);
 
+/*
+ * One whole draft step for a caller whose step inputs and tree outputs live in HOST memory (Section 3.2 followed by
+ * Algorithm 1, as one call): copies `in_bytes` from `in_host` to `in_dev`, runs dart_draft_step(in, out) and
+ * dart_build_tree(tree_in, tree_out), copies `out_bytes` from `out_dev` to `out_host` and waits for `cuda_stream`.
+ * The device pointers of `in` / `tree_in` (feats, tokens, seq_lens, ctx_tail) are expected to point into
+ * [in_dev, in_dev + in_bytes) and those of `tree_out` into [out_dev, out_dev + out_bytes): the layout inside the two
+ * buffers is the caller's.  Host buffers should be page-locked (pageable memory works, more slowly).  All buffers
+ * are caller-owned; nothing is allocated.  Synchronous: on return the tree is in `out_host`.
+ * Errors: those of the two calls; INVALID_ARG for a NULL buffer with a non-zero size; CUDA if a copy or the wait fails.
+ */
+typedef struct dart_host_io {
+  const void* in_host;   /* HOST   step inputs, in_bytes */
+  void* in_dev;          /* DEVICE their home on the device */
+  size_t in_bytes;
+  const void* out_dev;   /* DEVICE tree outputs, out_bytes */
+  void* out_host;        /* HOST   where the caller reads them */
+  size_t out_bytes;
+} dart_host_io;
+int dart_draft_step_host(dart_handle* h, const dart_host_io* io, const dart_step_in* in, const dart_step_out* out,
+                         const dart_tree_in* tree_in, const dart_tree_out* tree_out, void* cuda_stream);
+
 /* Free the workspace and the N-gram table.  The caller's buffers are untouched. */
 int dart_draft_destroy(dart_handle* h);
 

@@ -28,7 +28,7 @@ DART_ERR_INTERNAL = -6
 EXPORTS = [
     "dart_draft_init", "dart_draft_step", "dart_build_tree", "dart_draft_destroy", "dart_last_device_status",
     "dart_last_cuda_error", "dart_status_string", "dart_workspace_bytes", "dart_ngram_bytes", "dart_train_attention_fwd", "dart_step_launch_count", "dart_draft_prefill", "dart_tree_verify_inputs",
-    "dart_set_profile_events", "dart_topk_rows_noalloc", "dart_selftest_bounded_wait",
+    "dart_set_profile_events", "dart_topk_rows_noalloc", "dart_selftest_bounded_wait", "dart_draft_step_host",
 ]
 
 
@@ -100,6 +100,11 @@ class DartTreeOut(C.Structure):
                 ("n_nodes", C.c_void_p), ("scores", C.c_void_p)]
 
 
+class DartHostIo(C.Structure):
+    _fields_ = [("in_host", C.c_void_p), ("in_dev", C.c_void_p), ("in_bytes", C.c_size_t),
+                ("out_dev", C.c_void_p), ("out_host", C.c_void_p), ("out_bytes", C.c_size_t)]
+
+
 _lib = None
 
 
@@ -118,6 +123,9 @@ def lib() -> C.CDLL:
         L.dart_draft_step.restype = C.c_int
         L.dart_build_tree.argtypes = [C.c_void_p, C.POINTER(DartTreeIn), C.POINTER(DartTreeOut), C.c_void_p]
         L.dart_build_tree.restype = C.c_int
+        L.dart_draft_step_host.argtypes = [C.c_void_p, C.POINTER(DartHostIo), C.POINTER(DartStepIn), C.POINTER(DartStepOut),
+                                           C.POINTER(DartTreeIn), C.POINTER(DartTreeOut), C.c_void_p]
+        L.dart_draft_step_host.restype = C.c_int
         L.dart_draft_destroy.argtypes = [C.c_void_p]
         L.dart_draft_destroy.restype = C.c_int
         L.dart_last_device_status.argtypes = [C.c_void_p, C.c_void_p]
@@ -227,6 +235,19 @@ class DartDraft:
         if rc != DART_OK:
             raise DartError(rc, "dart_draft_step", lib().dart_last_cuda_error(self._h))
 
+    def host_step(self, *, in_host, in_dev, out_host, out_dev, feats, tokens, seq_lens, seq_lens_host, k_cache, v_cache,
+                  n_fresh, topk_ids, topk_slogit, ctx_tail, tree_tokens, parents, depth, mask, n_nodes, scores=None,
+                  logits=None, first_row=0, n_levels: Optional[int] = None, stream=None) -> "HostStep":
+        """dart_draft_step_host with its argument structures built once: the returned object is called with the
+        step counter and runs copy in, forward pass, tree, copy out, wait.  in_host / out_host are (pinned) host byte
+        tensors, in_dev / out_dev the device buffers that the device tensors passed here are views of."""
+        return HostStep(self, dict(in_host=in_host, in_dev=in_dev, out_host=out_host, out_dev=out_dev, feats=feats,
+                                   tokens=tokens, seq_lens=seq_lens, seq_lens_host=seq_lens_host, k_cache=k_cache,
+                                   v_cache=v_cache, n_fresh=n_fresh, topk_ids=topk_ids, topk_slogit=topk_slogit,
+                                   ctx_tail=ctx_tail, tree_tokens=tree_tokens, parents=parents, depth=depth, mask=mask,
+                                   n_nodes=n_nodes, scores=scores, logits=logits, first_row=first_row,
+                                   n_levels=n_levels), stream)
+
     def prefill(self, *, feats, tokens, seq_lens_host, new_rows_host, k_cache, v_cache, stream=None) -> None:
         """dart_draft_prefill: append the k, v of new prefix rows (packed features / next-token ids) to the caches."""
         slh = np.ascontiguousarray(seq_lens_host, dtype=np.int32)
@@ -310,3 +331,39 @@ def train_attention_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_l
 
 def workspace_bytes(cfg: DartConfig) -> int:
     return lib().dart_workspace_bytes(C.byref(cfg))
+
+
+class HostStep:
+    """One prepared dart_draft_step_host call (argument marshalling only; see DartDraft.host_step)."""
+
+    def __init__(self, draft: "DartDraft", a: dict, stream) -> None:
+        self._draft, self._keep = draft, a
+        self._slh = np.ascontiguousarray(a["seq_lens_host"], dtype=np.int32)
+        nf = a["n_fresh"]
+        self._counts = None if isinstance(nf, (int, np.integer)) else np.ascontiguousarray(nf, dtype=np.int32)
+        fr = a["first_row"]
+        self._rows = None if isinstance(fr, (int, np.integer)) else np.ascontiguousarray(fr, dtype=np.int32)
+        B = len(self._slh)
+        any_fresh = (int(nf) if self._counts is None else int(self._counts.max(initial=0))) > 0
+        self.io = DartHostIo(_ptr(a["in_host"]), _ptr(a["in_dev"]), a["in_host"].numel() * a["in_host"].element_size(),
+                             _ptr(a["out_dev"]), _ptr(a["out_host"]), a["out_host"].numel() * a["out_host"].element_size())
+        self.sin = DartStepIn(B, int(nf) if self._counts is None else int(self._counts.max(initial=0)),
+                              _ptr(a["feats"]) if any_fresh else None, _ptr(a["tokens"]) if any_fresh else None,
+                              _ptr(a["seq_lens"]), self._slh.ctypes.data, _ptr(a["k_cache"]), _ptr(a["v_cache"]), 0,
+                              None if self._counts is None else self._counts.ctypes.data)
+        self.sout = DartStepOut(_ptr(a["topk_ids"]), _ptr(a["topk_slogit"]), _ptr(a["logits"]))
+        f0 = int(fr) if self._rows is None else int(self._rows.min())
+        self.tin = DartTreeIn(B, f0, draft.cfg.K - f0 if a["n_levels"] is None else a["n_levels"], _ptr(a["topk_ids"]),
+                              _ptr(a["topk_slogit"]), _ptr(a["ctx_tail"]), None if self._rows is None else self._rows.ctypes.data)
+        self.tout = DartTreeOut(_ptr(a["tree_tokens"]), _ptr(a["parents"]), _ptr(a["depth"]), _ptr(a["mask"]),
+                                _ptr(a["n_nodes"]), _ptr(a["scores"]))
+        self._st = draft._stream(stream)
+        self._fn = lib().dart_draft_step_host
+        self._args = (draft._h, C.byref(self.io), C.byref(self.sin), C.byref(self.sout), C.byref(self.tin), C.byref(self.tout),
+                      self._st)
+
+    def __call__(self, step_counter: int = 0) -> None:
+        self.sin.step_counter = step_counter
+        rc = self._fn(*self._args)
+        if rc != DART_OK:
+            raise DartError(rc, "dart_draft_step_host", lib().dart_last_cuda_error(self._draft._h))

@@ -919,6 +919,26 @@ int dart_build_tree(dart_handle* h, const dart_tree_in* in, const dart_tree_out*
   return DART_OK;
 }
 
+int dart_draft_step_host(dart_handle* h, const dart_host_io* io, const dart_step_in* in, const dart_step_out* out,
+                         const dart_tree_in* tree_in, const dart_tree_out* tree_out, void* cuda_stream) {
+  if (h == nullptr || io == nullptr) return DART_ERR_INVALID_ARG;
+  if ((io->in_bytes > 0 && (io->in_host == nullptr || io->in_dev == nullptr)) ||
+      (io->out_bytes > 0 && (io->out_host == nullptr || io->out_dev == nullptr)))
+    return DART_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e;
+  if (io->in_bytes > 0 && (e = cudaMemcpyAsync(io->in_dev, io->in_host, io->in_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return fail_cuda(h, e);
+  int rc = dart_draft_step(h, in, out, cuda_stream);
+  if (rc == DART_OK) rc = dart_build_tree(h, tree_in, tree_out, cuda_stream);
+  if (rc == DART_OK && io->out_bytes > 0 &&
+      (e = cudaMemcpyAsync(io->out_host, io->out_dev, io->out_bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+    rc = fail_cuda(h, e);
+  // whatever was enqueued is waited for, also after an error: the caller's buffers are quiet on return
+  if ((e = cudaStreamSynchronize(st)) != cudaSuccess && rc == DART_OK) rc = fail_cuda(h, e);
+  return rc;
+}
+
 int dart_set_profile_events(dart_handle* h, int stage, void* start_event, void* stop_event) {
   if (h == nullptr || stage < 0 || stage > 8 || start_event == nullptr || stop_event == nullptr) return DART_ERR_INVALID_ARG;
   h->prof_stage = stage;

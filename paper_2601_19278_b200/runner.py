@@ -133,6 +133,17 @@ class DraftSession:
                               tokens=self.tokens, parents=self.parents, depth=self.depth, mask=self.mask,
                               n_nodes=self.n_nodes, scores=self.scores, first_row=fr, stream=stream)
 
+    def host_step(self, in_host, in_dev, out_host, out_dev, stream=None):
+        """A prepared dart_draft_step_host call over the buffers pack_io returned: call it with the step counter."""
+        i, nf = self.inp, self.inp["n_fresh"]
+        fr = max(nf, 1) - 1 if isinstance(nf, int) else [max(int(f), 1) - 1 for f in nf]
+        return self.draft.host_step(in_host=in_host, in_dev=in_dev, out_host=out_host, out_dev=out_dev, feats=i["feats"],
+                                    tokens=i["tokens"], seq_lens=i["seq_lens"], seq_lens_host=i["seq_lens_host"],
+                                    k_cache=i["k_cache"], v_cache=i["v_cache"], n_fresh=nf, topk_ids=self.topk_ids,
+                                    topk_slogit=self.topk_slogit, ctx_tail=i["ctx_tail"], tree_tokens=self.tokens,
+                                    parents=self.parents, depth=self.depth, mask=self.mask, n_nodes=self.n_nodes,
+                                    scores=self.scores, logits=self.logits, first_row=fr, stream=stream)
+
     def tree_outputs(self) -> Dict[str, np.ndarray]:
         self.check_guards()
         return {"tokens": self.tokens.cpu().numpy(), "parents": self.parents.cpu().numpy(),

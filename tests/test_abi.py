@@ -42,16 +42,17 @@ def test_header_is_plain_c_and_layouts_match_ctypes(binding, tmp_path):
     src = tmp_path / "sz.c"
     src.write_text(
         '#include <stdio.h>\n#include <stddef.h>\n#include "dart.h"\n'
-        "int main(void){printf(\"%zu %zu %zu %zu %zu %zu %zu %zu %zu %zu\\n\", sizeof(dart_config), sizeof(dart_weights),"
+        "int main(void){printf(\"%zu %zu %zu %zu %zu %zu %zu %zu %zu %zu %zu %zu\\n\", sizeof(dart_config), sizeof(dart_weights),"
         " sizeof(dart_ngram_host), sizeof(dart_step_in), sizeof(dart_step_out), sizeof(dart_tree_in), sizeof(dart_tree_out),"
-        " offsetof(dart_config, philox_seed), offsetof(dart_step_in, step_counter), offsetof(dart_tree_in, topk_ids));return 0;}\n")
+        " offsetof(dart_config, philox_seed), offsetof(dart_step_in, step_counter), offsetof(dart_tree_in, topk_ids),"
+        " sizeof(dart_host_io), offsetof(dart_host_io, out_dev));return 0;}\n")
     exe = tmp_path / "sz"
     subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
     got = [int(x) for x in subprocess.check_output([str(exe)]).split()]
     b = binding
     want = [C.sizeof(b.DartConfig), C.sizeof(b.DartWeights), C.sizeof(b.DartNgramHost), C.sizeof(b.DartStepIn),
             C.sizeof(b.DartStepOut), C.sizeof(b.DartTreeIn), C.sizeof(b.DartTreeOut), b.DartConfig.philox_seed.offset,
-            b.DartStepIn.step_counter.offset, b.DartTreeIn.topk_ids.offset]
+            b.DartStepIn.step_counter.offset, b.DartTreeIn.topk_ids.offset, C.sizeof(b.DartHostIo), b.DartHostIo.out_dev.offset]
     assert got == want
 
 
