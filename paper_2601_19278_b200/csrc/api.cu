@@ -839,7 +839,7 @@ int dart_draft_prefill(dart_handle* h, const dart_prefill_in* in, void* cuda_str
   Workspace& ws = h->ws;
   const bf16* feats = static_cast<const bf16*>(in->feats);
   cudaError_t e;
-  // passes of up to kPrefillPassRows packed rows: embeddings -> z e-half, feature FC -> z g-half, k / v -> caches
+  // passes of up to kPrefillPassRows packed rows: feature FC -> z g-half, beside it embeddings -> z e-half, then k / v -> caches
   for (long long done = 0; done < total; done += kPrefillPassRows) {
     const int T = (int)(total - done < kPrefillPassRows ? total - done : kPrefillPassRows);
     DenseArgs a;
@@ -860,9 +860,6 @@ int dart_draft_prefill(dart_handle* h, const dart_prefill_in* in, void* cuda_str
       a.seq_off[b + 1] = (int)(a.seq_off[b] + (hi - lo));
     }
     for (int b = B + 1; b < 33; ++b) a.seq_off[b] = a.seq_off[B];
-    if ((e = launch_prefill_embed(in->tokens + done, T, c.vocab, static_cast<const bf16*>(h->w.embed),
-                                  static_cast<const bf16*>(h->w.norm_e), hdim, c.rms_eps, ws.pz, 2 * hdim, st)) != cudaSuccess)
-      return fail_cuda(h, e);
     DenseArgs fc = a;
     fc.mode = 0; fc.n_w = 1; fc.n_tiles_per_w = prefill_fc_tiles(c); fc.n_out = hdim;
     fc.KB[0] = (c.feat_in + 63) / 64; fc.KB[1] = 0; fc.a_koff[0] = 0; fc.a_koff[1] = 0;
@@ -871,6 +868,9 @@ int dart_draft_prefill(dart_handle* h, const dart_prefill_in* in, void* cuda_str
     if ((e = tmap_encode_bf16(&fc.mapA, feats + (size_t)done * c.feat_in, c.feat_in, T, (unsigned long long)c.feat_in * 2, 64, 128)) != cudaSuccess)
       return fail_cuda(h, e);
     if ((e = launch_umma_dense(fc, h->n_sm, st)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = launch_prefill_embed(in->tokens + done, T, c.vocab, static_cast<const bf16*>(h->w.embed),
+                                  static_cast<const bf16*>(h->w.norm_e), hdim, c.rms_eps, ws.pz, 2 * hdim, h->n_sm, st)) != cudaSuccess)
+      return fail_cuda(h, e);
     DenseArgs kv = a;
     kv.mode = 1; kv.n_w = 2; kv.n_tiles_per_w = (c.n_kv_heads * c.head_dim + 255) / 256; kv.n_out = c.n_kv_heads * c.head_dim;
     kv.KB[0] = kv.KB[1] = (hdim + 63) / 64; kv.a_koff[0] = 0; kv.a_koff[1] = hdim;

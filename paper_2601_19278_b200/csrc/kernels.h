@@ -202,6 +202,7 @@ cudaError_t launch_umma_own(const OwnPlan& plan, const CUtensorMap* mapW, const 
 struct DenseArgs {
   CUtensorMap mapA, mapW[4];
   int T, mode, n_w, n_tiles_per_w, n_out;
+  int pair_waves;                                  // set by launch_umma_dense: waves of two-token-tile items (mode 0)
   int KB[2], a_koff[2];
   int h; float eps;
   const bf16* gain; bf16* z; long long ldz;       // mode 0 outputs
@@ -211,8 +212,9 @@ struct DenseArgs {
   int* status;
 };
 cudaError_t launch_umma_dense(const DenseArgs& a, int n_sm, cudaStream_t st);
+// to be launched right after the feature FC of the same pass (see the kernel)
 cudaError_t launch_prefill_embed(const int32_t* tokens, int T, int vocab, const bf16* embed, const bf16* gain_e, int h, float eps,
-                                 bf16* z, long long ldz, cudaStream_t st);
+                                 bf16* z, long long ldz, int n_sm, cudaStream_t st);
 
 // Self-test of the bounded waits (selftest.cu): a wait of `limit` tries on a barrier nobody signals; on expiry the
 // status word becomes DEV_TIMEOUT.  ticket != NULL: one ticket is taken on that counter first.

@@ -4,10 +4,11 @@
 // for T new prefix rows at once.  Unlike the drafting step (8..128 token rows against the whole model, HBM-bound)
 // this is a compute-bound GEMM, so the operands swap sides: 128 token rows are the M side of tcgen05.mma, 256
 // output features its N side, K = 16, four per 64-k stage; both operand tiles arrive by TMA (128-byte swizzle) in
-// a four-stage shared-memory ring (16 KB + 32 KB per stage), the fp32 accumulators sit in tensor memory (FC: two
-// buffers of 256 columns, so a tile's read-out overlaps the next tile's MMAs; k/v: one buffer per half of z,
-// because the two halves carry different 1/rms factors), and four warps read them out, one token row per thread.
-// One persistent CTA per SM walks the (token tile, feature tile) space; every mbarrier wait is bounded.
+// a shared-memory ring (16 KB + 32 KB per stage, four stages; the FC's pair items: 2 x 16 KB + 32 KB, three), the
+// fp32 accumulators sit in tensor memory (FC: two buffers of 256 columns -- a single tile's read-out overlaps the
+// next tile's MMAs, a pair item fills both; k/v: one buffer per half of z, because the two halves carry different
+// 1/rms factors), and four warps read them out, one token row per thread.
+// One persistent CTA per SM walks its list of work items (below); every mbarrier wait is bounded.
 #include "common.cuh"
 #include "kernels.h"
 #include "umma.cuh"
@@ -17,9 +18,40 @@ namespace dart {
 using namespace umma;
 
 constexpr int kDenseThreads = 256;
-constexpr int kDenseStages = 4;
-constexpr int kDenseABytes = 128 * 64 * 2, kDenseBBytes = 256 * 64 * 2, kDenseStageBytes = kDenseABytes + kDenseBBytes;
-constexpr size_t kDenseSmem = (size_t)kDenseStages * kDenseStageBytes + 1024;
+constexpr int kDenseABytes = 128 * 64 * 2, kDenseBBytes = 256 * 64 * 2;
+// The ring holds 192 KB either way: four stages of one token tile + one weight tile (48 KB), or -- feature FC with
+// pairs of token tiles -- three of two token tiles + one weight tile (64 KB).
+constexpr int kDenseRingBytes = 192 * 1024;
+constexpr size_t kDenseSmem = (size_t)kDenseRingBytes + 1024;
+
+// Work items.  A 128 x 256 tile asks for 48 KB of operands per 512 cycles of MMAs, more than an SM is delivered, so
+// the feature FC (mode 0) runs whole waves of PAIR items first: two token tiles that share the weight tile of a stage
+// (64 KB per 1024 cycles of MMAs), one accumulator each -- which leaves no second buffer to overlap the read-out with
+// the next item, a few per cent of an item with K = 3h.  What does not fill a wave of pairs runs as single tiles.
+// CTA c takes pair items c, c + G, ... of the first `pair_waves` * G pairs, then single tiles c, c + G, ... of the rest:
+// the two halves of every remaining pair (neighbouring CTAs share its weight tile in L2), then an odd last row of
+// token tiles.  Every role of a CTA walks the same list.
+struct DenseItem { int mt, nm, nt; };
+__device__ __forceinline__ bool dense_item(const DenseArgs& a, int i, int m_tiles, int n_tiles, DenseItem& it) {
+  const int G = gridDim.x, c = blockIdx.x;
+  const int pairs = (m_tiles >> 1) * n_tiles, n_pair = a.pair_waves * G;     // host: n_pair <= pairs
+  if (i < a.pair_waves) {
+    const int bi = i * G + c;
+    it.mt = 2 * (bi / n_tiles); it.nm = 2; it.nt = bi % n_tiles;
+    return true;
+  }
+  const int si = (i - a.pair_waves) * G + c, split = 2 * (pairs - n_pair);
+  if (si < split) {
+    const int bi = n_pair + (si >> 1);
+    it.mt = 2 * (bi / n_tiles) + (si & 1); it.nm = 1; it.nt = bi % n_tiles;
+    return true;
+  }
+  if ((m_tiles & 1) && si - split < n_tiles) {
+    it.mt = m_tiles - 1; it.nm = 1; it.nt = si - split;
+    return true;
+  }
+  return false;
+}
 
 // Cache slab and absolute position of packed row t (rows of sequence b are seq_off[b] .. seq_off[b+1]-1).
 __device__ __forceinline__ void row_place(const DenseArgs& a, int t, int& slab, int& pos) {
@@ -32,16 +64,18 @@ __device__ __forceinline__ void row_place(const DenseArgs& a, int t, int& slab, 
 __global__ void __launch_bounds__(kDenseThreads, 1) umma_dense_kernel(const __grid_constant__ DenseArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  __shared__ uint64_t full[kDenseStages], empty[kDenseStages], acc_full[2], acc_empty[2];
+  __shared__ uint64_t full[4], empty[4], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base;
   __shared__ int abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m_tiles = (a.T + 127) >> 7, n_tiles = a.n_w * a.n_tiles_per_w, tiles = m_tiles * n_tiles;
+  const int m_tiles = (a.T + 127) >> 7, n_tiles = a.n_w * a.n_tiles_per_w;
   const int KBt = a.KB[0] + a.KB[1];            // k-blocks per tile (k/v: g half then e half)
   const bool two_acc = a.mode == 1;             // k/v: one accumulator per half of z, no double buffering
+  const int stages = a.pair_waves > 0 ? 3 : 4;
+  const int stage_bytes = kDenseRingBytes / stages, w_off = stage_bytes - kDenseBBytes;   // [A0 | (A1) | W]
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kDenseStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < 4; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
     abort_flag = 0;
     fence_barrier_init();
@@ -52,58 +86,83 @@ __global__ void __launch_bounds__(kDenseThreads, 1) umma_dense_kernel(const __gr
   tc_fence_after();
   const uint32_t tmem = tmem_base;
   pdl_wait();   // every operand of this kernel is produced by the kernels before it
+  // The feature FC lets its successor start at once: that is prefill_embed_kernel, a few small blocks per SM that fit
+  // beside this CTA, share nothing with it (the other half of z) and wait for this grid before they exit.
+  if (a.mode == 0) pdl_trigger();
 
+  // Accumulator buffers of an item, the same in the MMA thread and the read-out warps: k/v items use both halves
+  // under buffer 0's barriers; a pair item takes buffers 0 and 1; a single FC tile takes them in turn.
   if (warp == 0 && lane == 0) {
     // ---- producer
     int s = 0, ph = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
-      const int mt = t / n_tiles, nt = t - mt * n_tiles;
-      const int w = nt / a.n_tiles_per_w, nrow = (nt - w * a.n_tiles_per_w) * 256;
+    DenseItem it;
+    for (int i = 0; ok && dense_item(a, i, m_tiles, n_tiles, it); ++i) {
+      const int w = it.nt / a.n_tiles_per_w, nrow = (it.nt - w * a.n_tiles_per_w) * 256;
       for (int kb = 0; kb < KBt; ++kb) {
         if (ph > 0 && !mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) { ok = false; break; }
         const int half = kb < a.KB[0] ? 0 : 1, kk = (half ? kb - a.KB[0] : kb) * 64;
-        uint8_t* st = ring + (size_t)s * kDenseStageBytes;
-        mbar_expect_tx(&full[s], kDenseStageBytes);
-        tma_load_2d(st, &a.mapA, &full[s], a.a_koff[half] + kk, mt * 128);
-        tma_load_2d(st + kDenseABytes, &a.mapW[w * 2 + half], &full[s], kk, nrow);
-        if (++s == kDenseStages) { s = 0; ++ph; }
+        uint8_t* st = ring + (size_t)s * stage_bytes;
+        mbar_expect_tx(&full[s], it.nm * kDenseABytes + kDenseBBytes);
+        tma_load_2d(st, &a.mapA, &full[s], a.a_koff[half] + kk, it.mt * 128);
+        if (it.nm == 2) tma_load_2d(st + kDenseABytes, &a.mapA, &full[s], a.a_koff[half] + kk, (it.mt + 1) * 128);
+        tma_load_2d(st + w_off, &a.mapW[w * 2 + half], &full[s], kk, nrow);
+        if (++s == stages) { s = 0; ++ph; }
       }
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer
     constexpr uint32_t idesc = idesc_bf16(128, 256);
-    int s = 0, ph = 0, it = 0;
+    int s = 0, ph = 0, use[2] = {0, 0}, tog = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
-      const int buf = two_acc ? 0 : (it & 1), use = two_acc ? it : (it >> 1);
-      if (use > 0) {
-        if (!mbar_wait(&acc_empty[buf], (use - 1) & 1, &abort_flag)) break;
-        tc_fence_after();
-      }
+    DenseItem it;
+    for (int i = 0; ok && dense_item(a, i, m_tiles, n_tiles, it); ++i) {
+      const int b0 = (two_acc || it.nm == 2) ? 0 : tog, nb = (!two_acc && it.nm == 2) ? 2 : 1;
+      if (!two_acc && it.nm == 1) tog ^= 1;
+      for (int b = b0; b < b0 + nb && ok; ++b)
+        if (use[b] > 0) {
+          if (!mbar_wait(&acc_empty[b], (use[b] - 1) & 1, &abort_flag)) ok = false;
+        }
+      if (!ok) break;
+      tc_fence_after();
       for (int kb = 0; kb < KBt; ++kb) {
         if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
         tc_fence_after();
         const int half = kb < a.KB[0] ? 0 : 1;
         const bool first = kb == 0 || kb == a.KB[0];
-        const uint32_t acc = tmem + (two_acc ? half * 256 : buf * 256);
-        const uint32_t wa = smem_u32(ring + (size_t)s * kDenseStageBytes);
-        const uint64_t ad = desc_sw128(wa), bd = desc_sw128(wa + kDenseABytes);
+        const uint32_t acc = tmem + (two_acc ? half * 256 : b0 * 256);
+        const uint32_t wa = smem_u32(ring + (size_t)s * stage_bytes);
+        const uint64_t ad = desc_sw128(wa), bd = desc_sw128(wa + w_off);
+        if (it.nm == 2) {
+          const uint64_t ad1 = desc_sw128(wa + kDenseABytes);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) mma_f16(acc, ad + 2 * k, bd + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+          for (int k = 0; k < 4; ++k) {
+            mma_f16(acc, ad + 2 * k, bd + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+            mma_f16(acc + 256, ad1 + 2 * k, bd + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mma_f16(acc, ad + 2 * k, bd + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+        }
         mma_commit(&empty[s]);
-        if (++s == kDenseStages) { s = 0; ++ph; }
+        if (++s == stages) { s = 0; ++ph; }
       }
-      if (ok) mma_commit(&acc_full[buf]);
+      if (ok)
+        for (int b = b0; b < b0 + nb; ++b) { mma_commit(&acc_full[b]); ++use[b]; }
     }
   } else if (warp >= 4) {
     // ---- read-out: TMEM lane = token row of the tile, columns = output features
     const int wq = warp & 3, row = wq * 32 + lane;
-    int it = 0;
-    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
-      const int mt = t / n_tiles, nt = t - mt * n_tiles;
-      const int buf = two_acc ? 0 : (it & 1), use = two_acc ? it : (it >> 1);
-      if (!mbar_wait(&acc_full[buf], use & 1, &abort_flag)) break;
+    int use[2] = {0, 0}, tog = 0;
+    bool ok = true;
+    DenseItem it;
+    for (int i = 0; ok && dense_item(a, i, m_tiles, n_tiles, it); ++i) {
+      const int b0 = (two_acc || it.nm == 2) ? 0 : tog, nb = (!two_acc && it.nm == 2) ? 2 : 1;
+      if (!two_acc && it.nm == 1) tog ^= 1;
+     for (int buf = b0; buf < b0 + nb; ++buf) {
+      const int mt = it.mt + (buf - b0), nt = it.nt;
+      if (!mbar_wait(&acc_full[buf], use[buf] & 1, &abort_flag)) { ok = false; break; }
+      ++use[buf];
       tc_fence_after();
       const int tok = mt * 128 + row;
       const bool live = tok < a.T;
@@ -187,6 +246,7 @@ __global__ void __launch_bounds__(kDenseThreads, 1) umma_dense_kernel(const __gr
       }
       tc_fence_before();
       mbar_arrive(&acc_empty[buf]);
+     }
     }
   }
   pdl_trigger();
@@ -198,37 +258,89 @@ __global__ void __launch_bounds__(kDenseThreads, 1) umma_dense_kernel(const __gr
   }
 }
 
-// z e-half of the prefill rows: RMSNorm of the next token's embedding, gain-scaled, bf16.  One block per row.
+// z e-half of the prefill rows: RMSNorm of the next token's embedding, gain-scaled, bf16.  A row is read and written
+// 16 bytes per thread and request when h is a multiple of 8 (two-byte requests made this kernel 64 us for 4096 rows
+// of 5120: a tenth of the prefill).  Launched right AFTER the feature FC, which triggers its dependents at once: a
+// few blocks per SM walk the rows while the FC's CTAs compute (its inputs are the caller's; the half of z it writes
+// is read by the k / v kernel only, and the previous pass's k / v kernel was complete before the FC triggered).  It
+// waits for the FC's grid at its END, so that the k / v kernel, which waits for this grid, finds both halves of z.
 __global__ void __launch_bounds__(256) prefill_embed_kernel(const int32_t* tokens, int T, int vocab, const bf16* embed, const bf16* gain_e,
                                                             int h, float eps, bf16* z, long long ldz) {
   __shared__ float sh[32];
-  pdl_wait();
-  const int t = blockIdx.x;
+ for (int t = blockIdx.x; t < T; t += gridDim.x) {
   const int id = min(max(tokens[t], 0), vocab - 1);
   const bf16* row = embed + (size_t)id * h;
+  bf16* out = z + (size_t)t * ldz + h;
+  const bool vec = (h & 7) == 0 && ((reinterpret_cast<uintptr_t>(row) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(gain_e)) & 15) == 0;
   float ss = 0.f;
-  for (int n = threadIdx.x; n < h; n += blockDim.x) {
-    const float v = __bfloat162float(row[n]);
-    ss += v * v;
+  if (vec) {
+    for (int n = threadIdx.x; n < (h >> 3); n += blockDim.x) {
+      const uint4 q = __ldg(reinterpret_cast<const uint4*>(row) + n);
+      const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&q);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(p2[j]);
+        ss += f.x * f.x + f.y * f.y;
+      }
+    }
+  } else {
+    for (int n = threadIdx.x; n < h; n += blockDim.x) {
+      const float v = __bfloat162float(row[n]);
+      ss += v * v;
+    }
   }
   ss = block_sum(ss, sh);
   const float rs = 1.f / sqrtf(ss / (float)h + eps);
-  for (int n = threadIdx.x; n < h; n += blockDim.x)
-    z[(size_t)t * ldz + h + n] = __float2bfloat16(__bfloat162float(row[n]) * rs * __bfloat162float(gain_e[n]));
+  if (vec) {
+    for (int n = threadIdx.x; n < (h >> 3); n += blockDim.x) {
+      const uint4 q = __ldg(reinterpret_cast<const uint4*>(row) + n), g = __ldg(reinterpret_cast<const uint4*>(gain_e) + n);
+      const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&q);
+      const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&g);
+      uint32_t w[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(p2[j]), gg = __bfloat1622float2(g2[j]);
+        // the same products, in the same order, as the element-wise form: (x * rs) * gain, rounded once
+        const __nv_bfloat162 v = __floats2bfloat162_rn(f.x * rs * gg.x, f.y * rs * gg.y);
+        w[j] = *reinterpret_cast<const uint32_t*>(&v);
+      }
+      reinterpret_cast<uint4*>(out)[n] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  } else {
+    for (int n = threadIdx.x; n < h; n += blockDim.x)
+      out[n] = __float2bfloat16(__bfloat162float(row[n]) * rs * __bfloat162float(gain_e[n]));
+  }
+  __syncthreads();    // sh is reused by the next row's sum
+ }
+  pdl_wait();
   pdl_trigger();
 }
 
 cudaError_t launch_prefill_embed(const int32_t* tokens, int T, int vocab, const bf16* embed, const bf16* gain_e, int h, float eps,
-                                 bf16* z, long long ldz, cudaStream_t st) {
-  return launch_pdl(prefill_embed_kernel, dim3(T), dim3(256), 0, st, tokens, T, vocab, embed, gain_e, h, eps, z, ldz);
+                                 bf16* z, long long ldz, int n_sm, cudaStream_t st) {
+  const int blocks = T < 2 * n_sm ? T : 2 * n_sm;   // what fits beside a CTA of the feature FC (registers)
+  return launch_pdl(prefill_embed_kernel, dim3(blocks), dim3(256), 0, st, tokens, T, vocab, embed, gain_e, h, eps, z, ldz);
 }
 
 cudaError_t launch_umma_dense(const DenseArgs& a, int n_sm, cudaStream_t st) {
   const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_dense_kernel), kDenseSmem);
   if (e != cudaSuccess) return e;
-  const int tiles = ((a.T + 127) / 128) * a.n_w * a.n_tiles_per_w;
+  const int m_tiles = (a.T + 127) / 128, n_tiles = a.n_w * a.n_tiles_per_w, tiles = m_tiles * n_tiles;
   const int grid = tiles < n_sm ? tiles : n_sm;
-  return launch_pdl(umma_dense_kernel, dim3(grid), dim3(kDenseThreads), kDenseSmem, st, a);
+  DenseArgs b = a;
+  b.pair_waves = 0;
+  if (a.mode == 0) {
+    // whole waves of pair items, as many as make the estimate smallest: a pair item costs two single tiles' MMAs,
+    // a single tile a quarter more than its own (the operands arrive more slowly than the MMAs take them)
+    const int pairs = (m_tiles / 2) * n_tiles;
+    double best = 0.0;
+    for (int pw = 0; pw <= pairs / grid; ++pw) {
+      const int singles = tiles - 2 * pw * grid;
+      const double t = 2.0 * pw + 1.25 * ((singles + grid - 1) / grid);
+      if (pw == 0 || t < best) { best = t; b.pair_waves = pw; }
+    }
+  }
+  return launch_pdl(umma_dense_kernel, dim3(grid), dim3(kDenseThreads), kDenseSmem, st, b);
 }
 
 }  // namespace dart
