@@ -805,7 +805,7 @@ int dart_train_attention_fwd(const dart_train_attn_in* in, void* cuda_stream) {
   TrainAttnArgs a;
   memset(&a, 0, sizeof(a));
   if ((e = tmap_encode_bf16(&a.mapQ, in->q, 128, (unsigned long long)B * Hq * L, 256, 64, 128)) != cudaSuccess ||
-      (e = tmap_encode_bf16(&a.mapK, in->k, 128, (unsigned long long)B * Hkv * L, 256, 64, 64)) != cudaSuccess ||
+      (e = tmap_encode_bf16(&a.mapK, in->k, 128, (unsigned long long)B * Hkv * L, 256, 64, 128)) != cudaSuccess ||
       (e = tmap_encode_bf16(&a.mapV, in->v, 128, (unsigned long long)B * Hkv * L, 256, 64, 64)) != cudaSuccess)
     return e == cudaErrorNotSupported ? DART_ERR_UNSUPPORTED_ARCH : fail_cuda(nullptr, e);
   a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.prompt_len = Lp; a.draft_len = d; a.n_clean_tiles = (Lp + 127) / 128;
