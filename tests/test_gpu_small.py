@@ -137,6 +137,34 @@ def test_runs_are_bitwise_repeatable():
     ses.close()
 
 
+def test_runs_with_128_token_rows_and_noise_are_bitwise_repeatable():
+    """At 33..128 token rows the LM head's CTAs prune against a bound they share through global memory, so which
+    candidates a CTA keeps depends on timing; the merged candidates, their log-probabilities and the trees must not.
+    A vocabulary wide enough for every SM to hold several tiles, temperature 1 (the bound then uses a lower bound of
+    the noisy keys), 12 runs."""
+    w = syn.small_variant(C1, batch=16, K=8, ragged_lo=10, prefix=300, vocab=80000, tree_budget=60, temperature=1.0)
+    wt = syn.make_weights(w)
+    inp = syn.make_step_inputs(w)
+    rows = syn.make_ngram_rows(w.vocab, 20000, w.ngram_mode)
+    ses = runner.DraftSession(w, wt, rows, want_logits=True, philox_seed=parity.PHILOX_SEED)
+    ses.load_inputs(inp)
+    ses.step(step_counter=5)
+    ses.tree()
+    torch.cuda.synchronize()
+    assert ses.draft.device_status() == 0
+    ref = parity.oracle_forward(w, wt, inp)
+    stats = parity.check_logits(ses.logits.cpu().numpy(), ref["logits"])
+    assert stats["max_abs"] < parity.TOL_ABS
+    a = (ses.topk_ids.clone(), ses.topk_slogit.clone(), ses.tokens.clone(), ses.parents.clone(), ses.mask.clone())
+    for _ in range(12):
+        ses.step(step_counter=5)
+        ses.tree()
+        torch.cuda.synchronize()
+        for x, y in zip(a, (ses.topk_ids, ses.topk_slogit, ses.tokens, ses.parents, ses.mask)):
+            assert torch.equal(x, y)
+    ses.close()
+
+
 def test_packed_io_moves_a_step_with_one_copy_each_way():
     """The end-to-end path of the benchmark: inputs in one pinned buffer, one copy in, one copy out."""
     w = CASES["ragged_b2"]
