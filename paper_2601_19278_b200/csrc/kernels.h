@@ -193,6 +193,10 @@ struct OwnArgs {
 bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm);
 cudaError_t launch_umma_own(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi, int* status,
                             cudaStream_t st);
+// The same for 33 .. 128 token rows (umma_own_wide_kernel): gate and up advance together and share each activation slice.
+bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm);
+cudaError_t launch_umma_own_wide(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi,
+                                 int* status, cudaStream_t st);
 
 // Dense projections of the draft-side prefill (umma_dense.cu): C[T, n_out] = A[T, k] W^T with 128 token rows per
 // tile on the MMA's M side and 256 output features on its N side.  mode 0: feature FC (A = features, one weight

@@ -159,6 +159,177 @@ __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_kernel(const __grid_c
   }
 }
 
+// ------------------------------------------------------------------------------------------------------
+// The same ownership for 33 .. 128 token rows.  There the activation slice of a 64-k block is 32 KB (hi and lo rows of
+// 128 tokens) against 16 KB of weights per 128 rows, and the stream-K kernel, which fetches it once per weight tile,
+// is bound by the L2 -> SM path (3 bytes per weight byte: gate / up 111 us for 54 us of bytes at 128 rows of the 14B
+// shape).  Here a stage holds the CTA's rows of BOTH matrices for one k-block and ONE activation slice; gate and up
+// advance together, each into an accumulator of its own (2 x 256 columns: all of tensor memory, which is fine because
+// a CTA has one read-out, at the end), so the slice is fetched once per two weight boxes: 2 bytes per weight byte.
+// Accumulator column 2 t (2 t + 1) of either matrix is token t's hi (lo) part.
+// ------------------------------------------------------------------------------------------------------
+constexpr int kOwnWideX = 256 * 64 * 2;           // hi and lo rows of 128 tokens, 64 k
+
+__global__ void __launch_bounds__(kOwnThreads, 1) umma_own_wide_kernel(const __grid_constant__ OwnArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ uint64_t full[4], empty[4], acc_full;
+  __shared__ uint32_t tmem_base;
+  __shared__ int abort_flag, s_bad;
+  __shared__ float s_rstd[128];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int c = blockIdx.x, G = gridDim.x;
+  const int r0 = (int)(((long long)c * a.rows) / G), r1 = (int)(((long long)(c + 1) * a.rows) / G);
+  const int stages = a.stages, stage_bytes = a.stage_bytes, w_area = (stage_bytes - kOwnWideX) / 2;   // [gate | up | x]
+  const int KB = a.KB;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(&acc_full, 1);
+    abort_flag = 0;
+    s_bad = 0;
+    fence_barrier_init();
+    // this thread is the producer: the weights of the first stages are requested before anything else of the set-up
+    const int pre = KB < stages ? KB : stages;
+    const uint64_t wpol = l2_policy_evict_first();
+    for (int it = 0; it < pre; ++it) {
+      uint8_t* st = ring + (size_t)it * stage_bytes;
+      mbar_expect_tx(&full[it], 2 * a.w_tx_bytes + kOwnWideX);
+      tma_load_2d_hint(st, &a.mapW[0], &full[it], it * 64, r0, wpol);
+      tma_load_2d_hint(st + w_area, &a.mapW[1], &full[it], it * 64, r0, wpol);
+    }
+  }
+  if (warp == 2) tmem_alloc(&tmem_base, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base;
+
+  if (warp == 0 && lane == 0) {
+    // ---- producer: activations depend on the previous kernel
+    const int pre = KB < stages ? KB : stages;
+    const uint64_t wpol = l2_policy_evict_first();
+    pdl_wait();
+    for (int it = 0; it < pre; ++it)
+      tma_load_3d(ring + (size_t)it * stage_bytes + 2 * w_area, &a.mapX, &full[it], it * 64, 0, 0);
+    int s = pre == stages ? 0 : pre, ph = pre == stages ? 1 : 0;
+    for (int kb = pre; kb < KB; ++kb) {
+      if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
+      uint8_t* st = ring + (size_t)s * stage_bytes;
+      mbar_expect_tx(&full[s], 2 * a.w_tx_bytes + kOwnWideX);
+      tma_load_2d_hint(st, &a.mapW[0], &full[s], kb * 64, r0, wpol);
+      tma_load_2d_hint(st + w_area, &a.mapW[1], &full[s], kb * 64, r0, wpol);
+      tma_load_3d(st + 2 * w_area, &a.mapX, &full[s], kb * 64, 0, 0);
+      if (++s == stages) { s = 0; ++ph; }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer: gate into tensor-memory columns 0 .. 255, up into 256 .. 511
+    constexpr uint32_t idesc = idesc_bf16(128, 256);
+    int s = 0, ph = 0;
+    bool ok = true;
+    for (int kb = 0; kb < KB; ++kb) {
+      if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t wa = smem_u32(ring + (size_t)s * stage_bytes);
+      const uint64_t gd = desc_sw128(wa), ud = desc_sw128(wa + w_area), xd = desc_sw128(wa + 2 * w_area);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        mma_f16(tmem, gd + 2 * k, xd + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+        mma_f16(tmem + 256, ud + 2 * k, xd + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+      }
+      mma_commit(&empty[s]);
+      if (++s == stages) { s = 0; ++ph; }
+    }
+    if (ok) mma_commit(&acc_full);
+  } else if (warp >= 4) {
+    // ---- epilogue: one output row per thread (row = tensor-memory lane), eight tokens at a time
+    const int wq = warp & 3, row = wq * 32 + lane;
+    const bool has_row = row < r1 - r0;
+    const int n = r0 + row, M = a.M;
+    pdl_wait();   // the sums of squares below are the previous kernel's; u may still be read by the one before it
+    for (int t = wq * 32; t < wq * 32 + 32; ++t) {     // 1/rms of this projection's input, 32 tokens per warp
+      float sacc = 0.f;
+      if (t < M)
+        for (int tl = lane; tl < a.ss_tiles; tl += 32) sacc += __ldcg(a.ss_in + (size_t)tl * a.ss_mp + t);
+      sacc = warp_sum(sacc);
+      if (lane == 0) s_rstd[t] = t < M ? 1.f / sqrtf(sacc / (float)a.h + a.eps) : 0.f;
+    }
+    if (!mbar_wait_relaxed(&acc_full, 0, &abort_flag)) s_bad = 1;
+    asm volatile("bar.sync 1, 128;" ::: "memory");   // s_rstd is written; the four warps agree on what follows
+    if (!s_bad) {
+      tc_fence_after();
+      const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16);
+#pragma unroll 1
+      for (int ch = 0; ch < 16 && ch * 8 < M; ++ch) {
+        uint32_t rg[16], ru[16];
+        tmem_ld16(tbase + 16 * ch, rg);
+        tmem_ld16(tbase + 256 + 16 * ch, ru);
+        tmem_ld_wait();
+        if (has_row) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int t = ch * 8 + j;
+            if (t < M) {
+              const float gt = s_rstd[t] * (__uint_as_float(rg[2 * j]) + __uint_as_float(rg[2 * j + 1]));
+              const float up = s_rstd[t] * (__uint_as_float(ru[2 * j]) + __uint_as_float(ru[2 * j + 1]));
+              bf16 hi, lo;
+              split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
+              DART_CHECK(n < a.rows && n < a.ld_out, a.status) {
+                a.out_hi[(size_t)t * a.ld_out + n] = hi;
+                a.out_lo[(size_t)t * a.ld_out + n] = lo;
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+  pdl_wait();
+  pdl_trigger();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+  if (abort_flag && threadIdx.x == 0) {
+    atomicExch(a.status, DEV_TIMEOUT);
+    for (int i = 0; i < 100; ++i) __nanosleep(1000);
+  }
+}
+
+// Plan of the kernel above: at least kOwnMinRows and at most 128 rows per CTA, two to four stages.
+bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm) {
+  p->rows = rows; p->Kd = Kd; p->KB = (Kd + 63) / 64;
+  p->grid = rows < n_sm ? rows : n_sm;
+  p->R = (rows + p->grid - 1) / p->grid;
+  if (p->R < kOwnMinRows || p->R > 128) return false;
+  const int w_area = ((p->R + 7) / 8) * 8 * 128;
+  p->stage_bytes = 2 * w_area + kOwnWideX;
+  p->w_tx_bytes = p->R * 128;
+  // the MMA reads 128 rows from a weight box's base: past gate's rows it reads up's, past up's the activation slice,
+  // all inside the stage (2 * w_area + 32 KB >= w_area + 16 KB)
+  int stages = (int)((kOwnSmemMax - 1024) / p->stage_bytes);
+  if (stages > 4) stages = 4;
+  if (stages < 2) return false;
+  p->stages = stages;
+  p->smem = (size_t)stages * p->stage_bytes + 1024;
+  return true;
+}
+
+cudaError_t launch_umma_own_wide(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi,
+                                 int* status, cudaStream_t st) {
+  OwnArgs a;
+  memset(&a, 0, sizeof(a));
+  a.mapW[0] = mapW[0]; a.mapW[1] = mapW[1];
+  a.mapX = mapX;
+  a.rows = plan.rows; a.KB = plan.KB; a.M = M;
+  a.stages = plan.stages; a.stage_bytes = plan.stage_bytes; a.w_tx_bytes = plan.w_tx_bytes;
+  a.ss_in = epi.ss_in; a.ss_tiles = epi.ss_tiles; a.ss_mp = epi.ss_mp; a.h = epi.h; a.eps = epi.eps;
+  a.out_hi = epi.out_hi; a.out_lo = epi.out_lo; a.ld_out = epi.ld_out;
+  a.status = status;
+  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_own_wide_kernel), kOwnSmemMax);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(umma_own_wide_kernel, dim3(plan.grid), dim3(kOwnThreads), plan.smem, st, a);
+}
+
 bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm) {
   p->rows = rows; p->Kd = Kd; p->KB = (Kd + 63) / 64;
   p->grid = rows < n_sm ? rows : n_sm;

@@ -28,6 +28,10 @@ CASES = {
     # an MLP wide enough (97 rows per SM on a 148-SM GPU, 96 on its last ones) for the gate / up projection to run
     # with row ownership: every CTA forms its own rows of SiLU(gate) * up from two accumulators
     "wide_mlp_row_ownership": syn.small_variant(C1, mlp_inter=14224, K=8, tree_budget=60, n_fresh=2),
+    # the same at 128 token rows: gate and up advance together and share each activation slice (eight k-blocks through
+    # a ring of three stages)
+    "wide_mlp_row_ownership_b16": syn.small_variant(C1, hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, mlp_inter=14224,
+                                                    vocab=2064, batch=16, K=8, ragged_lo=10, prefix=120, tree_budget=60),
     "hot_b4": syn.small_variant(C1, batch=4, ragged_lo=20, prefix=160, temperature=1.0),
     # enough 64-key tiles (sum over sequences x KV heads >= 512) for the tensor-core split-KV attention: ragged
     # lengths (partial last tiles, sequences with fewer chunks), 16 and 40 query rows per KV head; one long sequence
