@@ -193,8 +193,9 @@ struct OwnArgs {
 bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm);
 cudaError_t launch_umma_own(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi, int* status,
                             cudaStream_t st);
-// The same for 33 .. 128 token rows (umma_own_wide_kernel): gate and up advance together and share each activation slice.
-bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm);
+// The same for 9 .. 32 and 33 .. 128 token rows (umma_own_wide_kernel): gate and up advance together and share each
+// activation slice; a plan per padding (MP = 32: up to 256 rows per CTA, MP = 128: up to 128).
+bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm, int MP);
 cudaError_t launch_umma_own_wide(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi,
                                  int* status, cudaStream_t st);
 

@@ -168,19 +168,26 @@ __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_kernel(const __grid_c
 // a CTA has one read-out, at the end), so the slice is fetched once per two weight boxes: 2 bytes per weight byte.
 // Accumulator column 2 t (2 t + 1) of either matrix is token t's hi (lo) part.
 // ------------------------------------------------------------------------------------------------------
-constexpr int kOwnWideX = 256 * 64 * 2;           // hi and lo rows of 128 tokens, 64 k
+// The kernel is written for two shapes: 128 token rows (accumulators of 256 columns, up to 128 weight rows per CTA and
+// matrix) and 32 token rows (64 columns; up to 256 weight rows per CTA and matrix as two halves of 128, each with an
+// accumulator of its own: a 32B-shaped MLP is 173 rows per SM).  At 32 token rows the point is the one of
+// umma_own_kernel -- no pieces, no tickets, no finalize -- rather than the activation traffic.
+constexpr size_t kOwnWideSmemMax = 220 * 1024;
 
+template <int MP, int H>
 __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_wide_kernel(const __grid_constant__ OwnArgs a) {
+  constexpr int N = 2 * MP, XB = N * 64 * 2, TC = 2 * H * N;      // accumulator columns, bytes of a slice, tensor-memory columns
+  static_assert(TC == 128 || TC == 256 || TC == 512, "tensor-memory columns: a power of two");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ uint64_t full[4], empty[4], acc_full;
   __shared__ uint32_t tmem_base;
   __shared__ int abort_flag, s_bad;
-  __shared__ float s_rstd[128];
+  __shared__ float s_rstd[MP];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = blockIdx.x, G = gridDim.x;
   const int r0 = (int)(((long long)c * a.rows) / G), r1 = (int)(((long long)(c + 1) * a.rows) / G);
-  const int stages = a.stages, stage_bytes = a.stage_bytes, w_area = (stage_bytes - kOwnWideX) / 2;   // [gate | up | x]
+  const int stages = a.stages, stage_bytes = a.stage_bytes, w_area = (stage_bytes - XB) / 2;   // [gate | up | x]
   const int KB = a.KB;
 
   if (threadIdx.x == 0) {
@@ -194,12 +201,12 @@ __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_wide_kernel(const __g
     const uint64_t wpol = l2_policy_evict_first();
     for (int it = 0; it < pre; ++it) {
       uint8_t* st = ring + (size_t)it * stage_bytes;
-      mbar_expect_tx(&full[it], 2 * a.w_tx_bytes + kOwnWideX);
+      mbar_expect_tx(&full[it], 2 * a.w_tx_bytes + XB);
       tma_load_2d_hint(st, &a.mapW[0], &full[it], it * 64, r0, wpol);
       tma_load_2d_hint(st + w_area, &a.mapW[1], &full[it], it * 64, r0, wpol);
     }
   }
-  if (warp == 2) tmem_alloc(&tmem_base, 512);
+  if (warp == 2) tmem_alloc(&tmem_base, TC);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -216,38 +223,38 @@ __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_wide_kernel(const __g
     for (int kb = pre; kb < KB; ++kb) {
       if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
       uint8_t* st = ring + (size_t)s * stage_bytes;
-      mbar_expect_tx(&full[s], 2 * a.w_tx_bytes + kOwnWideX);
+      mbar_expect_tx(&full[s], 2 * a.w_tx_bytes + XB);
       tma_load_2d_hint(st, &a.mapW[0], &full[s], kb * 64, r0, wpol);
       tma_load_2d_hint(st + w_area, &a.mapW[1], &full[s], kb * 64, r0, wpol);
       tma_load_3d(st + 2 * w_area, &a.mapX, &full[s], kb * 64, 0, 0);
       if (++s == stages) { s = 0; ++ph; }
     }
   } else if (warp == 1 && lane == 0) {
-    // ---- MMA issuer: gate into tensor-memory columns 0 .. 255, up into 256 .. 511
-    constexpr uint32_t idesc = idesc_bf16(128, 256);
+    // ---- MMA issuer: accumulator (matrix g, row half hh) at tensor-memory columns (g H + hh) N
+    constexpr uint32_t idesc = idesc_bf16(128, N);
     int s = 0, ph = 0;
     bool ok = true;
     for (int kb = 0; kb < KB; ++kb) {
       if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t wa = smem_u32(ring + (size_t)s * stage_bytes);
-      const uint64_t gd = desc_sw128(wa), ud = desc_sw128(wa + w_area), xd = desc_sw128(wa + 2 * w_area);
+      const uint64_t xd = desc_sw128(wa + 2 * w_area);
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        mma_f16(tmem, gd + 2 * k, xd + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-        mma_f16(tmem + 256, ud + 2 * k, xd + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-      }
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int g = 0; g < 2; ++g)
+#pragma unroll
+          for (int hh = 0; hh < H; ++hh)      // rows 128 hh .. of the box: 16 KB further on
+            mma_f16(tmem + (g * H + hh) * N, desc_sw128(wa + g * w_area + hh * 16384) + 2 * k, xd + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
       mma_commit(&empty[s]);
       if (++s == stages) { s = 0; ++ph; }
     }
     if (ok) mma_commit(&acc_full);
   } else if (warp >= 4) {
-    // ---- epilogue: one output row per thread (row = tensor-memory lane), eight tokens at a time
-    const int wq = warp & 3, row = wq * 32 + lane;
-    const bool has_row = row < r1 - r0;
-    const int n = r0 + row, M = a.M;
+    // ---- epilogue: one output row per thread and row half (row = tensor-memory lane), eight tokens at a time
+    const int wq = warp & 3, M = a.M;
     pdl_wait();   // the sums of squares below are the previous kernel's; u may still be read by the one before it
-    for (int t = wq * 32; t < wq * 32 + 32; ++t) {     // 1/rms of this projection's input, 32 tokens per warp
+    for (int t = wq * (MP / 4); t < (wq + 1) * (MP / 4); ++t) {     // 1/rms of this projection's input, a quarter of the tokens per warp
       float sacc = 0.f;
       if (t < M)
         for (int tl = lane; tl < a.ss_tiles; tl += 32) sacc += __ldcg(a.ss_in + (size_t)tl * a.ss_mp + t);
@@ -260,23 +267,28 @@ __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_wide_kernel(const __g
       tc_fence_after();
       const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16);
 #pragma unroll 1
-      for (int ch = 0; ch < 16 && ch * 8 < M; ++ch) {
-        uint32_t rg[16], ru[16];
-        tmem_ld16(tbase + 16 * ch, rg);
-        tmem_ld16(tbase + 256 + 16 * ch, ru);
-        tmem_ld_wait();
-        if (has_row) {
+      for (int hh = 0; hh < H; ++hh) {
+        const int row = hh * 128 + wq * 32 + lane, n = r0 + row;
+        const bool has_row = row < r1 - r0;
+#pragma unroll 1
+        for (int ch = 0; ch < MP / 8 && ch * 8 < M; ++ch) {
+          uint32_t rg[16], ru[16];
+          tmem_ld16(tbase + hh * N + 16 * ch, rg);
+          tmem_ld16(tbase + (H + hh) * N + 16 * ch, ru);
+          tmem_ld_wait();
+          if (has_row) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int t = ch * 8 + j;
-            if (t < M) {
-              const float gt = s_rstd[t] * (__uint_as_float(rg[2 * j]) + __uint_as_float(rg[2 * j + 1]));
-              const float up = s_rstd[t] * (__uint_as_float(ru[2 * j]) + __uint_as_float(ru[2 * j + 1]));
-              bf16 hi, lo;
-              split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
-              DART_CHECK(n < a.rows && n < a.ld_out, a.status) {
-                a.out_hi[(size_t)t * a.ld_out + n] = hi;
-                a.out_lo[(size_t)t * a.ld_out + n] = lo;
+            for (int j = 0; j < 8; ++j) {
+              const int t = ch * 8 + j;
+              if (t < M) {
+                const float gt = s_rstd[t] * (__uint_as_float(rg[2 * j]) + __uint_as_float(rg[2 * j + 1]));
+                const float up = s_rstd[t] * (__uint_as_float(ru[2 * j]) + __uint_as_float(ru[2 * j + 1]));
+                bf16 hi, lo;
+                split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
+                DART_CHECK(n < a.rows && n < a.ld_out, a.status) {
+                  a.out_hi[(size_t)t * a.ld_out + n] = hi;
+                  a.out_lo[(size_t)t * a.ld_out + n] = lo;
+                }
               }
             }
           }
@@ -288,30 +300,41 @@ __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_wide_kernel(const __g
   pdl_trigger();
   tc_fence_before();
   __syncthreads();
-  if (warp == 2) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+  if (warp == 2) { tc_fence_after(); tmem_dealloc(tmem, TC); }
   if (abort_flag && threadIdx.x == 0) {
     atomicExch(a.status, DEV_TIMEOUT);
     for (int i = 0; i < 100; ++i) __nanosleep(1000);
   }
 }
 
-// Plan of the kernel above: at least kOwnMinRows and at most 128 rows per CTA, two to four stages.
-bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm) {
+// Plan of the kernel above for MP = 32 or 128 token rows: at least kOwnMinRows rows per CTA, at most 128 (MP = 128) or
+// 256 (MP = 32); two to four stages.
+bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm, int MP) {
   p->rows = rows; p->Kd = Kd; p->KB = (Kd + 63) / 64;
   p->grid = rows < n_sm ? rows : n_sm;
   p->R = (rows + p->grid - 1) / p->grid;
-  if (p->R < kOwnMinRows || p->R > 128) return false;
+  if (p->R < kOwnMinRows || p->R > (MP == 128 ? 128 : 256)) return false;
+  const int H = p->R > 128 ? 2 : 1, xb = 2 * MP * 128;
   const int w_area = ((p->R + 7) / 8) * 8 * 128;
-  p->stage_bytes = 2 * w_area + kOwnWideX;
+  p->stage_bytes = 2 * w_area + xb;
   p->w_tx_bytes = p->R * 128;
-  // the MMA reads 128 rows from a weight box's base: past gate's rows it reads up's, past up's the activation slice,
-  // all inside the stage (2 * w_area + 32 KB >= w_area + 16 KB)
-  int stages = (int)((kOwnSmemMax - 1024) / p->stage_bytes);
+  // the MMAs read H x 128 rows from a weight box's base: past gate's rows they read up's, past up's the activation
+  // slice and, in the ring's last stage, this much beyond it
+  int tail = H * 16384 - w_area - xb;
+  tail = tail > 0 ? ((tail + 1023) / 1024) * 1024 : 0;
+  int stages = (int)((kOwnWideSmemMax - 1024 - tail) / p->stage_bytes);
   if (stages > 4) stages = 4;
   if (stages < 2) return false;
   p->stages = stages;
-  p->smem = (size_t)stages * p->stage_bytes + 1024;
+  p->smem = (size_t)stages * p->stage_bytes + tail + 1024;
   return true;
+}
+
+template <int MP, int H>
+static cudaError_t launch_own_wide_t(const OwnPlan& plan, const OwnArgs& a, cudaStream_t st) {
+  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_own_wide_kernel<MP, H>), kOwnWideSmemMax);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(umma_own_wide_kernel<MP, H>, dim3(plan.grid), dim3(kOwnThreads), plan.smem, st, a);
 }
 
 cudaError_t launch_umma_own_wide(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi,
@@ -325,9 +348,10 @@ cudaError_t launch_umma_own_wide(const OwnPlan& plan, const CUtensorMap* mapW, c
   a.ss_in = epi.ss_in; a.ss_tiles = epi.ss_tiles; a.ss_mp = epi.ss_mp; a.h = epi.h; a.eps = epi.eps;
   a.out_hi = epi.out_hi; a.out_lo = epi.out_lo; a.ld_out = epi.ld_out;
   a.status = status;
-  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_own_wide_kernel), kOwnSmemMax);
-  if (e != cudaSuccess) return e;
-  return launch_pdl(umma_own_wide_kernel, dim3(plan.grid), dim3(kOwnThreads), plan.smem, st, a);
+  const int MP = padded_tokens(M);
+  if (MP == 128) return launch_own_wide_t<128, 1>(plan, a, st);
+  if (MP == 32) return plan.R > 128 ? launch_own_wide_t<32, 2>(plan, a, st) : launch_own_wide_t<32, 1>(plan, a, st);
+  return cudaErrorInvalidValue;
 }
 
 bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm) {

@@ -32,6 +32,9 @@ CASES = {
     # a ring of three stages)
     "wide_mlp_row_ownership_b16": syn.small_variant(C1, hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, mlp_inter=14224,
                                                     vocab=2064, batch=16, K=8, ragged_lo=10, prefix=120, tree_budget=60),
+    # ... and at 32 token rows with 151 rows per SM: two row halves per matrix, four accumulators
+    "tall_mlp_row_ownership_b4": syn.small_variant(C1, hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, mlp_inter=22208,
+                                                   vocab=2064, batch=4, K=8, ragged_lo=10, prefix=120, tree_budget=60),
     "hot_b4": syn.small_variant(C1, batch=4, ragged_lo=20, prefix=160, temperature=1.0),
     # enough 64-key tiles (sum over sequences x KV heads >= 512) for the tensor-core split-KV attention: ragged
     # lengths (partial last tiles, sequences with fewer chunks), 16 and 40 query rows per KV head; one long sequence
