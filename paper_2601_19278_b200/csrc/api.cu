@@ -61,12 +61,10 @@ struct dart_handle {
   int last_cuda_error = 0;
   GemmPlan plan_fc, plan_qkv, plan_o, plan_gu, plan_down;
   UmmaMaps maps_fc, maps_qkv, maps_o, maps_gu, maps_down;
-  bool own_ok = false;       // gate / up runs with row ownership on steps of up to eight token rows (the shape suits it)
-  OwnPlan own_gu;
-  CUtensorMap own_w_gu[2];
-  bool own_wide_ok[2] = {false, false};  // the same at 9 .. 32 [0] and 33 .. 128 [1] token rows (gate and up share each slice)
-  OwnPlan own_gu_wide[2];
-  CUtensorMap own_w_gu_wide[2][2];
+  // gate / up with row ownership where the shape suits it, at up to 8 [0], 32 [1] and 128 [2] token rows
+  bool own_ok[3] = {false, false, false};
+  OwnPlan own_gu[3];
+  CUtensorMap own_w_gu[3][2];
   CUtensorMap pmap_fc, pmap_kv[4];   // prefill: W_fc, and the g-/e-half columns of W_k and W_v (boxes of 256 rows)
   CUtensorMap map_lm;        // the LM head's weight matrix (boxes of 128 rows)
   CUtensorMap map_lm256;     // the same with boxes of 256 rows, for the swapped-operand kernel (33..128 token rows)
@@ -419,18 +417,12 @@ int dart_draft_init(const dart_config* cfg, const dart_weights* weights, const d
     }
   }
   // gate / up with row ownership (umma_own.cu): weight maps with boxes of 64 k x R rows
-  h->own_ok = n_sm <= 256 && own_plan_make(&h->own_gu, cfg->mlp_inter, cfg->hidden, n_sm);
-  if (h->own_ok) {
-    const unsigned long long hh = cfg->hidden;
-    INIT_CHECK(tmap_encode_bf16(&h->own_w_gu[0], weights->w_gate, hh, cfg->mlp_inter, hh * 2, 64, h->own_gu.R));
-    INIT_CHECK(tmap_encode_bf16(&h->own_w_gu[1], weights->w_up, hh, cfg->mlp_inter, hh * 2, 64, h->own_gu.R));
-  }
-  for (int i = 0; i < 2; ++i) {     // the wide form at 32 and at 128 token rows, each with weight boxes of its own height
-    h->own_wide_ok[i] = n_sm <= 256 && own_wide_plan_make(&h->own_gu_wide[i], cfg->mlp_inter, cfg->hidden, n_sm, i == 0 ? 32 : 128);
-    if (h->own_wide_ok[i]) {
+  for (int i = 0; i < 3; ++i) {     // a plan and weight boxes of their own height per token-row padding
+    h->own_ok[i] = n_sm <= 256 && own_plan_make(&h->own_gu[i], cfg->mlp_inter, cfg->hidden, n_sm, i == 0 ? 8 : (i == 1 ? 32 : 128));
+    if (h->own_ok[i]) {
       const unsigned long long hh = cfg->hidden;
-      INIT_CHECK(tmap_encode_bf16(&h->own_w_gu_wide[i][0], weights->w_gate, hh, cfg->mlp_inter, hh * 2, 64, h->own_gu_wide[i].R));
-      INIT_CHECK(tmap_encode_bf16(&h->own_w_gu_wide[i][1], weights->w_up, hh, cfg->mlp_inter, hh * 2, 64, h->own_gu_wide[i].R));
+      INIT_CHECK(tmap_encode_bf16(&h->own_w_gu[i][0], weights->w_gate, hh, cfg->mlp_inter, hh * 2, 64, h->own_gu[i].R));
+      INIT_CHECK(tmap_encode_bf16(&h->own_w_gu[i][1], weights->w_up, hh, cfg->mlp_inter, hh * 2, 64, h->own_gu[i].R));
     }
   }
   for (int i = 0; i < 5; ++i) {
@@ -619,9 +611,8 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   auto project = [&](const GemmPlan& plan, const UmmaMaps& maps) -> cudaError_t {
     return launch_umma_rows(plan, maps, gi, ep, ws.part, ws.status, st);
   };
-  const bool own_gu = h->own_ok && M <= 8;   // gate / up with row ownership: no pieces, no finalize
-  const int wide_i = MP == 32 ? 0 : 1;
-  const bool own_gu_wide = !own_gu && MP >= 32 && h->own_wide_ok[wide_i];
+  const int own_i = MP == 8 ? 0 : (MP == 32 ? 1 : 2);
+  const bool own_gu = h->own_ok[own_i];      // gate / up with row ownership: no pieces, no finalize
 
   // the <mask> rows of z are constant; they are (re)written only when the row pattern changes
   if (h->z_B != B || memcmp(h->z_foff.v, fo.v, sizeof(fo.v)) != 0) {
@@ -723,8 +714,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   ep.ss_in = ws.ss_1; ep.ss_tiles = h->h_tiles; ep.ss_mp = MP;
   ep.out_hi = ws.u_hi; ep.out_lo = ws.u_lo; ep.ld_out = c.mlp_inter;
   gi = {ws.n_hi, ws.n_lo, hdim, M};
-  if (own_gu) e = launch_umma_own(h->own_gu, h->own_w_gu, h->maps_gu.Xhi, M, ep, ws.status, st);
-  else if (own_gu_wide) e = launch_umma_own_wide(h->own_gu_wide[wide_i], h->own_w_gu_wide[wide_i], h->maps_gu.Xhi, M, ep, ws.status, st);
+  if (own_gu) e = launch_umma_own(h->own_gu[own_i], h->own_w_gu[own_i], h->maps_gu.Xhi, M, ep, ws.status, st);
   else e = project(h->plan_gu, h->maps_gu);
   if (e != cudaSuccess) return fail_cuda(h, e);
   mark(4, false);

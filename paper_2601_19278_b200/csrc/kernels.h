@@ -170,10 +170,9 @@ struct UmmaGemmArgs {
 };
 cudaError_t launch_umma_rows(const GemmPlan& plan, const UmmaMaps& maps, const GemmInput& in, const EpiArgs& epi, float* part,
                              int* status, cudaStream_t st);
-// Gate / up with row ownership (umma_own.cu), for steps of up to eight token rows: CTA c owns output rows
-// [c * rows / grid, (c + 1) * rows / grid) of both matrices over the whole reduction length.
-constexpr size_t kOwnSmemMax = 208 * 1024;
-constexpr int kOwnMinRows = 96;   // rows per CTA from which the kernel's TMA boxes stream at the HBM rate
+// Gate / up with row ownership (umma_own.cu): CTA c owns output rows [c * rows / grid, (c + 1) * rows / grid) of both
+// matrices over the whole reduction length; a stage holds its rows of both for one k-block and one activation slice.
+constexpr int kOwnMinRows = 96;   // rows per stage (both matrices together) from which the TMA boxes stream at the HBM rate
 struct OwnPlan {
   int rows, Kd, KB;            // output rows per matrix, reduction length, 64-k blocks
   int grid, R;                 // CTAs, weight rows per TMA box = ceil(rows / grid)
@@ -189,15 +188,11 @@ struct OwnArgs {
   bf16* out_hi; bf16* out_lo; long long ld_out;
   int* status;
 };
-// false: this shape does not suit the kernel (fewer than kOwnMinRows or more than 128 rows per CTA)
-bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm);
+// A plan per token-row padding MP = 8, 32, 128 (the activation slice's size decides the stage count).  false: the shape
+// does not suit the kernel (fewer than kOwnMinRows / 2 rows per CTA and matrix, or more than 256 -- 128 at MP = 128).
+bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm, int MP);
 cudaError_t launch_umma_own(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi, int* status,
                             cudaStream_t st);
-// The same for 9 .. 32 and 33 .. 128 token rows (umma_own_wide_kernel): gate and up advance together and share each
-// activation slice; a plan per padding (MP = 32: up to 256 rows per CTA, MP = 128: up to 128).
-bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm, int MP);
-cudaError_t launch_umma_own_wide(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi,
-                                 int* status, cudaStream_t st);
 
 // Dense projections of the draft-side prefill (umma_dense.cu): C[T, n_out] = A[T, k] W^T with 128 token rows per
 // tile on the MMA's M side and 256 output features on its N side.  mode 0: feature FC (A = features, one weight

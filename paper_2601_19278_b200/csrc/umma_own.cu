@@ -1,23 +1,30 @@
-// The gate / up projection with row ownership, for steps of up to eight token rows (Section 3.2's SiLU-gated MLP):
-// u = SiLU(rstd * W_gate n) * (rstd * W_up n).
+// The gate / up projection with row ownership (Section 3.2's SiLU-gated MLP): u = SiLU(rstd * W_gate n) * (rstd * W_up n).
 //
 // umma_gemm.cu balances the SMs by cutting the (tile, k-block) space into equal ranges, which splits every output
 // tile between CTAs: pieces in global memory, tickets, and a fused finalize on the kernel's tail by whichever CTA
 // arrives last (3.5 - 5.5 us per projection, on the critical path of the step).  Here the OUTPUT ROWS are cut instead:
 // CTA c owns rows [c * rows / G, (c + 1) * rows / G) of both matrices -- 117 or 118 of 17408 at the 14B shape -- and
-// streams them over the whole reduction length, gate first, then up, into two accumulators: every CTA reads the same
-// number of bytes AND holds complete results, so the epilogue goes from tensor memory straight to the down
-// projection's input, with no piece, no ticket and no second CTA involved (gate/up stage 71.7 -> 67.6 us).  A TMA box
-// may be any number of rows high: a stage of the ring holds R = ceil(rows / G) weight rows x 64 k plus the matching
-// 2 KB activation slice, and tcgen05.mma runs with M = 128 over a tile whose rows past R are whatever shared memory
-// holds there -- accumulator rows that nothing reads.
-// Why only gate / up: a stage of the ring costs the same ~650 cycles whatever it holds.  Cycle counters in this kernel:
-// the MMA-issuing thread spends ~370 cycles per stage on the fence, four MMAs and the commit and ~270 waiting for the
-// stage; the producer ~220 on the expect-tx and two TMA issues and ~360 waiting for a free stage; the period equals the
-// sum of the two issue times, with 4 stages in the ring as with 27, with or without the activation loads, with one
-// commit per stage or per four.  118 rows x 64 k per stage is then 22 bytes per clock -- an SM's share of HBM; FC,
-// o_proj and down would own 35 rows per CTA at the 14B shape and stream at 10 (95 / 39 / 104 us instead of 41 / 25 /
-// 43: measured), so they stay on the stream-K kernel, whose stages hold 128 rows.
+// streams them over the whole reduction length: every CTA reads the same number of bytes AND holds complete results,
+// so the epilogue goes from tensor memory straight to the down projection's input, with no piece, no ticket and no
+// second CTA involved.  A TMA box may be any number of rows high: a stage of the ring holds the CTA's R rows x 64 k of
+// W_gate, the same of W_up, and ONE activation slice; gate and up advance together, each into accumulators of its
+// own, and tcgen05.mma runs with M = 128 over a tile whose rows past R are whatever shared memory holds there --
+// accumulator rows that nothing reads.
+// Why gate and up share a stage.  A stage of the ring costs the same ~650 cycles whatever it holds (cycle counters: the
+// MMA-issuing thread spends ~370 cycles per stage on the fence, four MMAs and the commit and ~270 waiting for the
+// stage; the producer ~220 on the expect-tx and two TMA issues and ~360 waiting for a free stage; the period equals
+// the sum of the two issue times, with 4 stages in the ring as with 27, with or without the activation loads, with one
+// commit per stage or per four).  The first form of this kernel streamed gate, then up, 118 rows x 64 k per stage:
+// 22 bytes per clock, just an SM's share of HBM (gate / up stage 71.7 -> 65.6 us at the 14B shape).  With both boxes
+// in a stage it is 30 KB per ~770 cycles (61.6 us; 45.1 -> 41.5 us at the 8B shape, whose 83 rows per SM were too few
+// to stream alone).  And at 33 .. 128 token rows, where the activation slice (32 KB) is twice a weight tile and the
+// stream-K kernel, which fetches it once per 128 weight rows, is bound by the L2 -> SM path (3 bytes per weight
+// byte), the slice is fetched once per two weight boxes: 2 bytes per weight byte (111 -> 86 us at 16 x 8 token rows).
+// Why only gate / up: FC, o_proj and down would own 35 rows per CTA at the 14B shape and stream at 10 bytes per clock
+// (95 / 39 / 104 us instead of 41 / 25 / 43: measured), so they stay on the stream-K kernel, whose stages hold 128 rows.
+// Shapes: MP = 8, 32 or 128 token rows (accumulators of 2 MP columns: column 2 t is token t's hi part, 2 t + 1 its lo
+// part); up to 128 weight rows per CTA and matrix, or -- MP <= 32 -- up to 256 as two halves of 128 with an accumulator
+// each (a 32B-shaped MLP is 173 rows per SM; the second half's MMAs read 16 KB further into the weight box).
 // Roles, barriers, bounded waits and programmatic dependent launch are those of umma_gemm.cu.
 #include "common.cuh"
 #include "kernels.h"
@@ -28,159 +35,15 @@ namespace dart {
 using namespace umma;
 
 constexpr int kOwnThreads = 256;
-constexpr int kOwnMaxStages = 32;
-constexpr int kOwnXBytes = 16 * 64 * 2;          // hi and lo rows of eight tokens, 64 k
-
-__global__ void __launch_bounds__(kOwnThreads, 1) umma_own_kernel(const __grid_constant__ OwnArgs a) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  __shared__ uint64_t full[kOwnMaxStages], empty[kOwnMaxStages], acc_full;
-  __shared__ uint32_t tmem_base;
-  __shared__ int abort_flag, s_bad;
-  __shared__ float s_rstd[8];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int c = blockIdx.x, G = gridDim.x;
-  const int r0 = (int)(((long long)c * a.rows) / G), r1 = (int)(((long long)(c + 1) * a.rows) / G);
-  const int stages = a.stages, stage_bytes = a.stage_bytes, w_bytes = stage_bytes - kOwnXBytes;
-  const int n_units = 2 * a.KB;     // gate's k-blocks, then up's
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(&acc_full, 1);
-    abort_flag = 0;
-    s_bad = 0;
-    fence_barrier_init();
-    // this thread is the producer: weights do not depend on the previous kernel, so the ring is filled with them
-    // before anything else of the CTA's setup
-    const int pre = n_units < stages ? n_units : stages;
-    const uint64_t wpol = l2_policy_evict_first();
-    int mat = 0, kb = 0;
-    for (int it = 0; it < pre; ++it) {
-      mbar_expect_tx(&full[it], a.w_tx_bytes + kOwnXBytes);
-      tma_load_2d_hint(ring + (size_t)it * stage_bytes, &a.mapW[mat], &full[it], kb * 64, r0, wpol);
-      if (++kb == a.KB) { kb = 0; ++mat; }
-    }
-  }
-  if (warp == 2) tmem_alloc(&tmem_base, 32);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = tmem_base;
-
-  if (warp == 0 && lane == 0) {
-    // ---- producer (the ring already holds the first weights): activations depend on the previous kernel
-    const int pre = n_units < stages ? n_units : stages;
-    const uint64_t wpol = l2_policy_evict_first();
-    pdl_wait();
-    int mat = 0, kb = 0;
-    for (int it = 0; it < pre; ++it) {
-      tma_load_3d(ring + (size_t)it * stage_bytes + w_bytes, &a.mapX, &full[it], kb * 64, 0, 0);
-      if (++kb == a.KB) { kb = 0; ++mat; }
-    }
-    int s = pre == stages ? 0 : pre, ph = pre == stages ? 1 : 0;
-    for (int it = pre; it < n_units; ++it) {
-      if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
-      uint8_t* st = ring + (size_t)s * stage_bytes;
-      mbar_expect_tx(&full[s], a.w_tx_bytes + kOwnXBytes);
-      tma_load_2d_hint(st, &a.mapW[mat], &full[s], kb * 64, r0, wpol);
-      tma_load_3d(st + w_bytes, &a.mapX, &full[s], kb * 64, 0, 0);
-      if (++s == stages) { s = 0; ++ph; }
-      if (++kb == a.KB) { kb = 0; ++mat; }
-    }
-  } else if (warp == 1 && lane == 0) {
-    // ---- MMA issuer: gate accumulates into tensor-memory columns 0 .. 15, up into 16 .. 31
-    constexpr uint32_t idesc = idesc_bf16(128, 16);
-    int s = 0, ph = 0, mat = 0, kb = 0;
-    bool ok = true;
-    for (int it = 0; it < n_units; ++it) {
-      if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
-      tc_fence_after();
-      const uint32_t wa = smem_u32(ring + (size_t)s * stage_bytes);
-      const uint64_t ad = desc_sw128(wa), bd = desc_sw128(wa + w_bytes);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + 16 * mat, ad + 2 * k, bd + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-      mma_commit(&empty[s]);
-      if (++s == stages) { s = 0; ++ph; }
-      if (++kb == a.KB) { kb = 0; ++mat; }
-    }
-    if (ok) mma_commit(&acc_full);
-  } else if (warp >= 4) {
-    // ---- epilogue: one output row per thread (row = tensor-memory lane)
-    const int wq = warp & 3, row = wq * 32 + lane;
-    const bool has_row = row < r1 - r0;
-    const int n = r0 + row, M = a.M;
-    pdl_wait();   // the sums of squares below are the previous kernel's; u may still be read by the one before it
-    if (wq == 0) {
-      // 1/rms of this projection's input, from the partial sums of squares its producer left (a fixed order)
-      for (int t = 0; t < 8; ++t) {
-        float sacc = 0.f;
-        if (t < M)
-          for (int tl = lane; tl < a.ss_tiles; tl += 32) sacc += __ldcg(a.ss_in + (size_t)tl * a.ss_mp + t);
-        sacc = warp_sum(sacc);
-        if (lane == 0) s_rstd[t] = t < M ? 1.f / sqrtf(sacc / (float)a.h + a.eps) : 0.f;
-      }
-    }
-    if (!mbar_wait_relaxed(&acc_full, 0, &abort_flag)) s_bad = 1;
-    asm volatile("bar.sync 1, 128;" ::: "memory");   // s_rstd is written; the four warps agree on what follows
-    if (!s_bad) {
-      tc_fence_after();
-      const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16);
-      uint32_t rg[16], ru[16];
-      tmem_ld16(tbase, rg);
-      tmem_ld16(tbase + 16, ru);
-      tmem_ld_wait();
-      if (has_row) {
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-          if (t < M) {
-            // columns (2t, 2t+1) are token t's hi and lo parts; the previous RMSNorm's 1/rms is applied here
-            const float gt = s_rstd[t] * (__uint_as_float(rg[2 * t]) + __uint_as_float(rg[2 * t + 1]));
-            const float up = s_rstd[t] * (__uint_as_float(ru[2 * t]) + __uint_as_float(ru[2 * t + 1]));
-            bf16 hi, lo;
-            split_bf16(gt / (1.f + expf(-gt)) * up, hi, lo);
-            DART_CHECK(n < a.rows && n < a.ld_out, a.status) {
-              a.out_hi[(size_t)t * a.ld_out + n] = hi;
-              a.out_lo[(size_t)t * a.ld_out + n] = lo;
-            }
-          }
-        }
-      }
-    }
-  }
-  pdl_wait();
-  pdl_trigger();
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 2) { tc_fence_after(); tmem_dealloc(tmem, 32); }
-  if (abort_flag && threadIdx.x == 0) {
-    // a wait ran out: report it and give copies that may still be in flight time to land
-    atomicExch(a.status, DEV_TIMEOUT);
-    for (int i = 0; i < 100; ++i) __nanosleep(1000);
-  }
-}
-
-// ------------------------------------------------------------------------------------------------------
-// The same ownership for 33 .. 128 token rows.  There the activation slice of a 64-k block is 32 KB (hi and lo rows of
-// 128 tokens) against 16 KB of weights per 128 rows, and the stream-K kernel, which fetches it once per weight tile,
-// is bound by the L2 -> SM path (3 bytes per weight byte: gate / up 111 us for 54 us of bytes at 128 rows of the 14B
-// shape).  Here a stage holds the CTA's rows of BOTH matrices for one k-block and ONE activation slice; gate and up
-// advance together, each into an accumulator of its own (2 x 256 columns: all of tensor memory, which is fine because
-// a CTA has one read-out, at the end), so the slice is fetched once per two weight boxes: 2 bytes per weight byte.
-// Accumulator column 2 t (2 t + 1) of either matrix is token t's hi (lo) part.
-// ------------------------------------------------------------------------------------------------------
-// The kernel is written for two shapes: 128 token rows (accumulators of 256 columns, up to 128 weight rows per CTA and
-// matrix) and 32 token rows (64 columns; up to 256 weight rows per CTA and matrix as two halves of 128, each with an
-// accumulator of its own: a 32B-shaped MLP is 173 rows per SM).  At 32 token rows the point is the one of
-// umma_own_kernel -- no pieces, no tickets, no finalize -- rather than the activation traffic.
-constexpr size_t kOwnWideSmemMax = 220 * 1024;
+constexpr size_t kOwnSmemLimit = 220 * 1024;
 
 template <int MP, int H>
-__global__ void __launch_bounds__(kOwnThreads, 1) umma_own_wide_kernel(const __grid_constant__ OwnArgs a) {
+__global__ void __launch_bounds__(kOwnThreads, 1) umma_own_kernel(const __grid_constant__ OwnArgs a) {
   constexpr int N = 2 * MP, XB = N * 64 * 2, TC = 2 * H * N;      // accumulator columns, bytes of a slice, tensor-memory columns
-  static_assert(TC == 128 || TC == 256 || TC == 512, "tensor-memory columns: a power of two");
+  static_assert(TC == 32 || TC == 64 || TC == 128 || TC == 256 || TC == 512, "tensor-memory columns: a power of two");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  __shared__ uint64_t full[4], empty[4], acc_full;
+  __shared__ uint64_t full[8], empty[8], acc_full;
   __shared__ uint32_t tmem_base;
   __shared__ int abort_flag, s_bad;
   __shared__ float s_rstd[MP];
@@ -307,13 +170,13 @@ __global__ void __launch_bounds__(kOwnThreads, 1) umma_own_wide_kernel(const __g
   }
 }
 
-// Plan of the kernel above for MP = 32 or 128 token rows: at least kOwnMinRows rows per CTA, at most 128 (MP = 128) or
-// 256 (MP = 32); two to four stages.
-bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm, int MP) {
+// Plan of the kernel above for MP = 8, 32 or 128 token rows: at least kOwnMinRows / 2 rows per CTA and matrix (two
+// boxes to a stage: enough bytes to stream), at most 128 (MP = 128) or 256; two to eight stages.
+bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm, int MP) {
   p->rows = rows; p->Kd = Kd; p->KB = (Kd + 63) / 64;
   p->grid = rows < n_sm ? rows : n_sm;
   p->R = (rows + p->grid - 1) / p->grid;
-  if (p->R < kOwnMinRows || p->R > (MP == 128 ? 128 : 256)) return false;
+  if (p->R < kOwnMinRows / 2 || p->R > (MP == 128 ? 128 : 256)) return false;
   const int H = p->R > 128 ? 2 : 1, xb = 2 * MP * 128;
   const int w_area = ((p->R + 7) / 8) * 8 * 128;
   p->stage_bytes = 2 * w_area + xb;
@@ -322,8 +185,8 @@ bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm, int MP) {
   // slice and, in the ring's last stage, this much beyond it
   int tail = H * 16384 - w_area - xb;
   tail = tail > 0 ? ((tail + 1023) / 1024) * 1024 : 0;
-  int stages = (int)((kOwnWideSmemMax - 1024 - tail) / p->stage_bytes);
-  if (stages > 4) stages = 4;
+  int stages = (int)((kOwnSmemLimit - 1024 - tail) / p->stage_bytes);
+  if (stages > 8) stages = 8;
   if (stages < 2) return false;
   p->stages = stages;
   p->smem = (size_t)stages * p->stage_bytes + tail + 1024;
@@ -331,13 +194,13 @@ bool own_wide_plan_make(OwnPlan* p, int rows, int Kd, int n_sm, int MP) {
 }
 
 template <int MP, int H>
-static cudaError_t launch_own_wide_t(const OwnPlan& plan, const OwnArgs& a, cudaStream_t st) {
-  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_own_wide_kernel<MP, H>), kOwnWideSmemMax);
+static cudaError_t launch_own_t(const OwnPlan& plan, const OwnArgs& a, cudaStream_t st) {
+  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_own_kernel<MP, H>), kOwnSmemLimit);
   if (e != cudaSuccess) return e;
-  return launch_pdl(umma_own_wide_kernel<MP, H>, dim3(plan.grid), dim3(kOwnThreads), plan.smem, st, a);
+  return launch_pdl(umma_own_kernel<MP, H>, dim3(plan.grid), dim3(kOwnThreads), plan.smem, st, a);
 }
 
-cudaError_t launch_umma_own_wide(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi,
+cudaError_t launch_umma_own(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi,
                                  int* status, cudaStream_t st) {
   OwnArgs a;
   memset(&a, 0, sizeof(a));
@@ -349,44 +212,10 @@ cudaError_t launch_umma_own_wide(const OwnPlan& plan, const CUtensorMap* mapW, c
   a.out_hi = epi.out_hi; a.out_lo = epi.out_lo; a.ld_out = epi.ld_out;
   a.status = status;
   const int MP = padded_tokens(M);
-  if (MP == 128) return launch_own_wide_t<128, 1>(plan, a, st);
-  if (MP == 32) return plan.R > 128 ? launch_own_wide_t<32, 2>(plan, a, st) : launch_own_wide_t<32, 1>(plan, a, st);
+  if (MP == 128) return launch_own_t<128, 1>(plan, a, st);
+  if (MP == 32) return plan.R > 128 ? launch_own_t<32, 2>(plan, a, st) : launch_own_t<32, 1>(plan, a, st);
+  if (MP == 8) return plan.R > 128 ? launch_own_t<8, 2>(plan, a, st) : launch_own_t<8, 1>(plan, a, st);
   return cudaErrorInvalidValue;
-}
-
-bool own_plan_make(OwnPlan* p, int rows, int Kd, int n_sm) {
-  p->rows = rows; p->Kd = Kd; p->KB = (Kd + 63) / 64;
-  p->grid = rows < n_sm ? rows : n_sm;
-  p->R = (rows + p->grid - 1) / p->grid;
-  // boxes of fewer rows would not stream at the HBM rate (see the head of this file); more do not fit the MMA tile
-  if (p->R < kOwnMinRows || p->R > 128) return false;
-  const int w_area = ((p->R + 7) / 8) * 8 * 128;                  // whole 8-row groups of 128-byte rows
-  p->stage_bytes = w_area + kOwnXBytes;
-  p->w_tx_bytes = p->R * 128;                                     // what one weight box delivers (rows past the matrix are zero-filled and counted)
-  // the MMA reads 128 rows from a stage's base, i.e. past the rows that were loaded: the ring ends with that much room
-  const int tail = 128 * 128;
-  int stages = (int)((kOwnSmemMax - 1024 - tail) / p->stage_bytes);
-  if (stages > kOwnMaxStages) stages = kOwnMaxStages;
-  if (stages < 2) return false;
-  p->stages = stages;
-  p->smem = (size_t)stages * p->stage_bytes + tail + 1024;
-  return true;
-}
-
-cudaError_t launch_umma_own(const OwnPlan& plan, const CUtensorMap* mapW, const CUtensorMap& mapX, int M, const EpiArgs& epi,
-                            int* status, cudaStream_t st) {
-  OwnArgs a;
-  memset(&a, 0, sizeof(a));
-  a.mapW[0] = mapW[0]; a.mapW[1] = mapW[1];
-  a.mapX = mapX;
-  a.rows = plan.rows; a.KB = plan.KB; a.M = M;
-  a.stages = plan.stages; a.stage_bytes = plan.stage_bytes; a.w_tx_bytes = plan.w_tx_bytes;
-  a.ss_in = epi.ss_in; a.ss_tiles = epi.ss_tiles; a.ss_mp = epi.ss_mp; a.h = epi.h; a.eps = epi.eps;
-  a.out_hi = epi.out_hi; a.out_lo = epi.out_lo; a.ld_out = epi.ld_out;
-  a.status = status;
-  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_own_kernel), kOwnSmemMax);
-  if (e != cudaSuccess) return e;
-  return launch_pdl(umma_own_kernel, dim3(plan.grid), dim3(kOwnThreads), plan.smem, st, a);
 }
 
 }  // namespace dart

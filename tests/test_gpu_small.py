@@ -25,8 +25,8 @@ CASES = {
                                  vocab=3088, prefix=150, K=8, tree_budget=60, batch=2, ragged_lo=3),
     "b16_k8_pad128": syn.small_variant(C1, batch=16, K=8, ragged_lo=10, prefix=300, vocab=2048, tree_budget=60),
     "empty_prefix": syn.small_variant(C1, prefix=0),
-    # an MLP wide enough (97 rows per SM on a 148-SM GPU, 96 on its last ones) for the gate / up projection to run
-    # with row ownership: every CTA forms its own rows of SiLU(gate) * up from two accumulators
+    # an MLP wide enough (97 rows per SM on a 148-SM GPU, 96 on its last ones; from 48 on) for the gate / up projection
+    # to run with row ownership: every CTA forms its own rows of SiLU(gate) * up from two accumulators
     "wide_mlp_row_ownership": syn.small_variant(C1, mlp_inter=14224, K=8, tree_budget=60, n_fresh=2),
     # the same at 128 token rows: gate and up advance together and share each activation slice (eight k-blocks through
     # a ring of three stages)
@@ -35,6 +35,9 @@ CASES = {
     # ... and at 32 token rows with 151 rows per SM: two row halves per matrix, four accumulators
     "tall_mlp_row_ownership_b4": syn.small_variant(C1, hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, mlp_inter=22208,
                                                    vocab=2064, batch=4, K=8, ragged_lo=10, prefix=120, tree_budget=60),
+    # the remaining shapes of that kernel: 32 token rows with one row half, 8 token rows with two
+    "wide_mlp_row_ownership_b4": syn.small_variant(C1, mlp_inter=14224, batch=4, K=8, ragged_lo=10, prefix=120, tree_budget=60),
+    "tall_mlp_row_ownership_b1": syn.small_variant(C1, mlp_inter=22208, K=8, tree_budget=60, n_fresh=2),
     "hot_b4": syn.small_variant(C1, batch=4, ragged_lo=20, prefix=160, temperature=1.0),
     # enough 64-key tiles (sum over sequences x KV heads >= 512) for the tensor-core split-KV attention: ragged
     # lengths (partial last tiles, sequences with fewer chunks), 16 and 40 query rows per KV head; one long sequence
