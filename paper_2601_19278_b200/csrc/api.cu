@@ -747,7 +747,7 @@ int dart_draft_step(dart_handle* h, const dart_step_in* in, const dart_step_out*
   {
     // one CTA per SM at most: the CTAs of this kernel wait on one another's pieces, so all must be resident
     const bool dense = MP == 128;   // many token rows: tokens on the MMA's M side, 256 vocabulary rows per tile
-    const long long units = (long long)((c.vocab + (dense ? 255 : 127)) / (dense ? 256 : 128)) * ((hdim + 63) / 64);
+    const long long units = lm_head_units(c.vocab, hdim, dense);
     lp.grid = (int)(units < h->n_sm ? units : h->n_sm);
     if (dense) {
       if (h->lmx_M != M) {

@@ -303,6 +303,8 @@ struct LmUmmaArgs {
   unsigned long long* bound;   // lm_head_dense_kernel: [128 token rows][kLmBoundSlots] shared lower bounds (tag << 32 | ordered key)
 };
 constexpr int kLmBoundSlots = 40;   // topk + 7 of them are used
+// units of work of an LM-head launch; its grid must not exceed them (nor the SM count: the CTAs wait on one another)
+long long lm_head_units(int V, int Kd, bool dense);
 cudaError_t launch_lm_head_umma(const LmParams& p, const CUtensorMap& mapW, const CUtensorMap& mapX,
                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st);
 // The LM head for 33..128 token rows with the operands swapped (token rows on the MMA's M side; lm_head.cu).

@@ -113,11 +113,18 @@ template <int MP>
 struct LmUmmaCfg {
   static constexpr int N = 2 * MP;
   static constexpr int XBytes = N * 64 * 2;
-  static constexpr int StageBytes = 128 * 64 * 2 + XBytes;
+#ifndef LM_KS
+#define LM_KS 2
+#endif
+  // A stage holds KS consecutive 64-k blocks of a vocabulary tile: KS weight boxes, then KS activation slices.  A
+  // stage of the ring costs about the same ~690 cycles whatever it holds, and with one block (16 KB of weights) that
+  // is 23 bytes per clock: just an SM's share of HBM.
+  static constexpr int KS = LM_KS;
+  static constexpr int StageBytes = KS * (128 * 64 * 2 + XBytes);
   static constexpr int TmemCols = 2 * N < 32 ? 32 : 2 * N;
   // epilogue shared memory: stage [MP][129] floats, lists 3 x [MP][32], statistics [MP][2], 1/rms [MP]
   static constexpr size_t EpiBytes = sizeof(float) * (MP * 129 + 3 * MP * 32 + 3 * MP);
-  static constexpr int Stages = MP == 8 ? 11 : 7;
+  static constexpr int Stages = (MP == 8 ? 11 : 7) / KS + (KS > 1 && MP == 32 ? 1 : 0);
   static constexpr size_t SmemBytes = (size_t)Stages * StageBytes + 1024 + EpiBytes;
 };
 
@@ -155,7 +162,9 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
     int tile = (int)(u0 / KB), kb = (int)(u0 % KB);
     for (int it = 0; it < pre; ++it) {
       mbar_expect_tx(&full[it], C::StageBytes);
-      tma_load_2d_hint(ring + (size_t)it * C::StageBytes, &a.mapW, &full[it], kb * 64, tile * 128, wpol);
+#pragma unroll
+      for (int q = 0; q < C::KS; ++q)
+        tma_load_2d_hint(ring + (size_t)it * C::StageBytes + q * (128 * 64 * 2), &a.mapW, &full[it], (kb * C::KS + q) * 64, tile * 128, wpol);
       if (++kb == KB) { kb = 0; ++tile; }
     }
   }
@@ -176,8 +185,9 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
     pdl_wait();
     tile = (int)(u0 / KB); kb = (int)(u0 % KB);
     for (int it = 0; it < pre; ++it) {
-      uint8_t* xs = ring + (size_t)it * C::StageBytes + 128 * 64 * 2;
-      tma_load_3d(xs, &a.mapXhi, &full[it], kb * 64, 0, 0);
+      uint8_t* xs = ring + (size_t)it * C::StageBytes + C::KS * (128 * 64 * 2);
+#pragma unroll
+      for (int q = 0; q < C::KS; ++q) tma_load_3d(xs + q * C::XBytes, &a.mapXhi, &full[it], (kb * C::KS + q) * 64, 0, 0);
       if (++kb == KB) { kb = 0; ++tile; }
     }
     int s = pre == C::Stages ? 0 : pre, ph = pre == C::Stages ? 1 : 0;
@@ -185,8 +195,11 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
       if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
       uint8_t* st = ring + (size_t)s * C::StageBytes;
       mbar_expect_tx(&full[s], C::StageBytes);
-      tma_load_2d_hint(st, &a.mapW, &full[s], kb * 64, tile * 128, wpol);
-      tma_load_3d(st + 128 * 64 * 2, &a.mapXhi, &full[s], kb * 64, 0, 0);
+#pragma unroll
+      for (int q = 0; q < C::KS; ++q) {
+        tma_load_2d_hint(st + q * (128 * 64 * 2), &a.mapW, &full[s], (kb * C::KS + q) * 64, tile * 128, wpol);
+        tma_load_3d(st + C::KS * (128 * 64 * 2) + q * C::XBytes, &a.mapXhi, &full[s], (kb * C::KS + q) * 64, 0, 0);
+      }
       if (++s == C::Stages) { s = 0; ++ph; }
       if (++kb == KB) { kb = 0; ++tile; }
     }
@@ -213,9 +226,12 @@ __global__ void __launch_bounds__(kLmUmmaThreads, 1) lm_head_umma_kernel(const _
       if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t wa = smem_u32(ring + (size_t)s * C::StageBytes);
-      const uint64_t ad = desc_sw128(wa), bd = desc_sw128(wa + 128 * 64 * 2);
 #pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + buf * C::N, ad + 2 * k, bd + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+      for (int q = 0; q < C::KS; ++q) {
+        const uint64_t ad = desc_sw128(wa + q * (128 * 64 * 2)), bd = desc_sw128(wa + C::KS * (128 * 64 * 2) + q * C::XBytes);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mma_f16(tmem + buf * C::N, ad + 2 * k, bd + 2 * k, idesc, (!first || q > 0 || k > 0) ? 1u : 0u);
+      }
       mma_commit(&empty[s]);
       if (++s == C::Stages) { s = 0; ++ph; }
       if (++kb == KB) { kb = 0; ++t; }
@@ -349,13 +365,19 @@ static cudaError_t launch_lm_umma_t(const LmUmmaArgs& a, cudaStream_t st) {
   return launch_pdl(lm_head_umma_kernel<MP>, dim3(a.p.grid), dim3(kLmUmmaThreads), C::SmemBytes, st, a);
 }
 
+// Units of work of a launch (what the grid is cut over): vocabulary tiles x ring stages per tile.
+long long lm_head_units(int V, int Kd, bool dense) {
+  const int kb = (Kd + 63) / 64;
+  return dense ? (long long)((V + 255) / 256) * kb : (long long)((V + 127) / 128) * ((kb + LM_KS - 1) / LM_KS);
+}
+
 cudaError_t launch_lm_head_umma(const LmParams& pin, const CUtensorMap& mapW, const CUtensorMap& mapX,
                                 float* pieces, int* flags, int tag, int* status, cudaStream_t st) {
   LmUmmaArgs a;
   memset(&a, 0, sizeof(a));
   a.p = pin;
   a.mapW = mapW; a.mapXhi = mapX;
-  a.KB = (pin.Kd + 63) / 64;
+  a.KB = ((pin.Kd + 63) / 64 + LM_KS - 1) / LM_KS;   // stages per vocabulary tile (a k tail reads as zeros)
   a.U = (long long)((pin.V + 127) / 128) * a.KB;
   a.pieces = pieces; a.flags = flags; a.tag = tag; a.status = status;
   const int MP = padded_tokens(pin.M);
