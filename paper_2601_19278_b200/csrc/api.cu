@@ -144,7 +144,7 @@ void make_plan_host(PlanHost& ph, const GemmSeg* segs, int nseg, int Kd, int gri
   }
   p.Kd = Kd;
   p.SK = (Kd + 63) / 64;
-  p.KR = p.SK;
+  p.KR = (p.SK + kUmmaKS - 1) / kUmmaKS;   // a work unit = one ring stage = kUmmaKS k-blocks (a k tail reads as zeros)
   p.n_tiles = tiles;
   p.U = (long long)tiles * p.KR;
   p.grid = (int)((long long)grid_target < p.U ? grid_target : p.U);

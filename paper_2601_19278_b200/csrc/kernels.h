@@ -73,6 +73,7 @@ struct GemmSeg {
   int xoff;       // column offset into the activation rows for this segment
 };
 
+constexpr int kUmmaKS = 2;         // 64-k blocks per ring stage of the stream-K projections = per work unit of their plans
 constexpr int kMetaStride = 36;   // ints per 16-row tile in the piece table: count + up to 35 offsets
 
 struct GemmPlan {
@@ -80,7 +81,7 @@ struct GemmPlan {
   GemmSeg seg[6];
   int Kd;           // reduction length per segment, multiple of 16
   int SK;           // ceil(Kd / 64) k-blocks per row
-  int KR;           // k-blocks per 128-row tile (= SK)
+  int KR;           // ring stages (work units) per 128-row tile = ceil(SK / kUmmaKS)
   int n_tiles;      // 128-row tiles over all segments
   int grid;         // CTAs
   int slots;        // max tiles a CTA touches
@@ -137,7 +138,7 @@ struct StreamArgs {
   int nseg;
   int Kd;             // reduction length (multiple of 16)
   int SK;             // 64-wide k-blocks per row
-  int KR;             // k-blocks per 128-row tile (= SK)
+  int KR;             // ring stages (work units) per 128-row tile = ceil(SK / kUmmaKS)
   const bf16* x_hi;   // activations [rows, ldx] hi part
   const bf16* x_lo;   // lo part (== x_hi when the input is plain bf16)
   long long ldx;

@@ -32,8 +32,16 @@ template <int MP>
 struct UmmaCfg {
   static constexpr int N = 2 * MP;                       // hi rows + lo rows
   static constexpr int XBytes = N * 64 * 2;
-  static constexpr int StageBytes = kWBytes + XBytes;
-  static constexpr int Stages = MP == 8 ? 11 : (MP == 32 ? 8 : 4);
+  // A stage holds kUmmaKS consecutive 64-k blocks of a tile (the weight boxes, then the activation slices): a stage
+  // of the ring costs about the same ~690 cycles whatever it holds, and one block -- 16 KB of weights -- per stage is
+  // just an SM's share of HBM.  The plans count their units in stages (GemmPlan::KR).
+  static constexpr int KS = kUmmaKS;
+  static constexpr int StageBytes = KS * (kWBytes + XBytes);
+#ifdef UMMA_STAGES8
+  static constexpr int Stages = MP == 8 ? UMMA_STAGES8 : (MP == 32 ? 4 : 2);
+#else
+  static constexpr int Stages = MP == 8 ? 5 : (MP == 32 ? 4 : 2);
+#endif
   static constexpr int TmemCols = 2 * N < 32 ? 32 : 2 * N;
   static constexpr size_t SmemBytes = (size_t)Stages * StageBytes + 1024;
 };
@@ -106,7 +114,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
     if (n > 0) q.set(p.s, u0, p.pair_offset);
     for (int it = 0; it < pre; ++it, q.next(p.s)) {
       mbar_expect_tx(&full[it], C::StageBytes);
-      tma_load_2d_hint(ring + (size_t)it * C::StageBytes, &a.mapW[q.seg], &full[it], q.kb * 64, q.row0, wpol);
+#pragma unroll
+      for (int j = 0; j < C::KS; ++j)
+        tma_load_2d_hint(ring + (size_t)it * C::StageBytes + j * kWBytes, &a.mapW[q.seg], &full[it], (q.kb * C::KS + j) * 64, q.row0, wpol);
     }
   }
   if (warp == 2) tmem_alloc(&tmem_base, C::TmemCols);
@@ -137,18 +147,25 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
     pdl_wait();
     q.set(p.s, u0, p.pair_offset);
     for (int it = 0; it < pre; ++it, q.next(p.s)) {
-      uint8_t* xs = ring + (size_t)it * C::StageBytes + kWBytes;
-      if (a.has_lo) tma_load_3d(xs, &a.mapXhi, &full[it], q.xoff + q.kb * 64, 0, 0);
-      else tma_load_2d(xs, &a.mapXhi, &full[it], q.xoff + q.kb * 64, 0);
+      uint8_t* xs = ring + (size_t)it * C::StageBytes + C::KS * kWBytes;
+#pragma unroll
+      for (int j = 0; j < C::KS; ++j) {
+        if (a.has_lo) tma_load_3d(xs + j * C::XBytes, &a.mapXhi, &full[it], q.xoff + (q.kb * C::KS + j) * 64, 0, 0);
+        else tma_load_2d(xs + j * C::XBytes, &a.mapXhi, &full[it], q.xoff + (q.kb * C::KS + j) * 64, 0);
+      }
     }
     int s = pre == C::Stages ? 0 : pre, ph = pre == C::Stages ? 1 : 0;
     for (int it = pre; it < n; ++it, q.next(p.s)) {
       if (!mbar_wait(&empty[s], (ph - 1) & 1, &abort_flag)) break;
       uint8_t* st = ring + (size_t)s * C::StageBytes;
       mbar_expect_tx(&full[s], C::StageBytes);
-      tma_load_2d_hint(st, &a.mapW[q.seg], &full[s], q.kb * 64, q.row0, wpol);
-      if (a.has_lo) tma_load_3d(st + kWBytes, &a.mapXhi, &full[s], q.xoff + q.kb * 64, 0, 0);
-      else tma_load_2d(st + kWBytes, &a.mapXhi, &full[s], q.xoff + q.kb * 64, 0);
+#pragma unroll
+      for (int j = 0; j < C::KS; ++j) {
+        const int k0 = (q.kb * C::KS + j) * 64;
+        tma_load_2d_hint(st + j * kWBytes, &a.mapW[q.seg], &full[s], k0, q.row0, wpol);
+        if (a.has_lo) tma_load_3d(st + C::KS * kWBytes + j * C::XBytes, &a.mapXhi, &full[s], q.xoff + k0, 0, 0);
+        else tma_load_2d(st + C::KS * kWBytes + j * C::XBytes, &a.mapXhi, &full[s], q.xoff + k0, 0);
+      }
       if (++s == C::Stages) { s = 0; ++ph; }
     }
   } else if (warp == 1 && lane == 0) {
@@ -174,9 +191,12 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       if (!mbar_wait(&full[s], ph & 1, &abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t wa = smem_u32(ring + (size_t)s * C::StageBytes);
-      const uint64_t ad = desc_sw128(wa), bd = desc_sw128(wa + kWBytes);
 #pragma unroll
-      for (int k = 0; k < 4; ++k) mma_f16(tmem + buf * C::N, ad + 2 * k, bd + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+      for (int j = 0; j < C::KS; ++j) {
+        const uint64_t ad = desc_sw128(wa + j * kWBytes), bd = desc_sw128(wa + C::KS * kWBytes + j * C::XBytes);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mma_f16(tmem + buf * C::N, ad + 2 * k, bd + 2 * k, idesc, (!first || j > 0 || k > 0) ? 1u : 0u);
+      }
       mma_commit(&empty[s]);
       if (++s == C::Stages) { s = 0; ++ph; }
       if (++kb == KB) { kb = 0; ++t; }
