@@ -35,13 +35,12 @@ struct UmmaCfg {
   // A stage holds kUmmaKS consecutive 64-k blocks of a tile (the weight boxes, then the activation slices): a stage
   // of the ring costs about the same ~690 cycles whatever it holds, and one block -- 16 KB of weights -- per stage is
   // just an SM's share of HBM.  The plans count their units in stages (GemmPlan::KR).
-  static constexpr int KS = kUmmaKS;
+  // At 128 token rows a block pair would be a 96 KB stage, two to the ring (measured slower than four of 48 KB): there
+  // a unit is SPU = 2 stages of one block each.
+  static constexpr int KS = MP == 128 ? 1 : kUmmaKS;      // 64-k blocks per stage
+  static constexpr int SPU = kUmmaKS / KS;                // stages per work unit
   static constexpr int StageBytes = KS * (kWBytes + XBytes);
-#ifdef UMMA_STAGES8
-  static constexpr int Stages = MP == 8 ? UMMA_STAGES8 : (MP == 32 ? 4 : 2);
-#else
-  static constexpr int Stages = MP == 8 ? 5 : (MP == 32 ? 4 : 2);
-#endif
+  static constexpr int Stages = MP == 8 ? 5 : 4;
   static constexpr int TmemCols = 2 * N < 32 ? 32 : 2 * N;
   static constexpr size_t SmemBytes = (size_t)Stages * StageBytes + 1024;
 };
@@ -76,6 +75,17 @@ struct UnitPos {
     if (++kb == a.KR) { kb = 0; ++tile; locate(a); }
   }
 };
+// Walks the ring stages of a range of units: SPU stages per unit, KS k-blocks per stage.
+template <int SPU, int KS>
+struct StagePos {
+  UnitPos q;
+  int sub;
+  __device__ __forceinline__ void set(const StreamArgs& a, long long u, int pair_offset) { q.set(a, u, pair_offset); sub = 0; }
+  __device__ __forceinline__ int k0(int j) const { return ((q.kb * SPU + sub) * KS + j) * 64; }   // first k of the stage's block j
+  __device__ __forceinline__ void next(const StreamArgs& a) {
+    if (++sub == SPU) { sub = 0; q.next(a); }
+  }
+};
 
 template <int MP>
 __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid_constant__ UmmaGemmArgs a) {
@@ -107,16 +117,16 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
     fence_barrier_init();
     // this thread is the producer: weights do not depend on the previous kernel, so the ring is filled with
     // them before anything else of the CTA's setup
-    const int n = (int)(u1 - u0);
+    const int n = (int)(u1 - u0) * C::SPU;           // stages of this CTA's range
     const int pre = n < C::Stages ? n : C::Stages;
     const uint64_t wpol = l2_policy_evict_first();
-    UnitPos q;
+    StagePos<C::SPU, C::KS> q;
     if (n > 0) q.set(p.s, u0, p.pair_offset);
     for (int it = 0; it < pre; ++it, q.next(p.s)) {
       mbar_expect_tx(&full[it], C::StageBytes);
 #pragma unroll
       for (int j = 0; j < C::KS; ++j)
-        tma_load_2d_hint(ring + (size_t)it * C::StageBytes + j * kWBytes, &a.mapW[q.seg], &full[it], (q.kb * C::KS + j) * 64, q.row0, wpol);
+        tma_load_2d_hint(ring + (size_t)it * C::StageBytes + j * kWBytes, &a.mapW[q.q.seg], &full[it], q.k0(j), q.q.row0, wpol);
     }
   }
   if (warp == 2) tmem_alloc(&tmem_base, C::TmemCols);
@@ -140,18 +150,18 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
 
   if (warp == 0 && lane == 0) {
     // ---- producer (the ring already holds the first weights): activations depend on the previous kernel
-    const int n = (int)(u1 - u0);
+    const int n = (int)(u1 - u0) * C::SPU;
     const int pre = n < C::Stages ? n : C::Stages;
     const uint64_t wpol = l2_policy_evict_first();
-    UnitPos q;
+    StagePos<C::SPU, C::KS> q;
     pdl_wait();
     q.set(p.s, u0, p.pair_offset);
     for (int it = 0; it < pre; ++it, q.next(p.s)) {
       uint8_t* xs = ring + (size_t)it * C::StageBytes + C::KS * kWBytes;
 #pragma unroll
       for (int j = 0; j < C::KS; ++j) {
-        if (a.has_lo) tma_load_3d(xs + j * C::XBytes, &a.mapXhi, &full[it], q.xoff + (q.kb * C::KS + j) * 64, 0, 0);
-        else tma_load_2d(xs + j * C::XBytes, &a.mapXhi, &full[it], q.xoff + (q.kb * C::KS + j) * 64, 0);
+        if (a.has_lo) tma_load_3d(xs + j * C::XBytes, &a.mapXhi, &full[it], q.q.xoff + q.k0(j), 0, 0);
+        else tma_load_2d(xs + j * C::XBytes, &a.mapXhi, &full[it], q.q.xoff + q.k0(j), 0);
       }
     }
     int s = pre == C::Stages ? 0 : pre, ph = pre == C::Stages ? 1 : 0;
@@ -161,19 +171,19 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       mbar_expect_tx(&full[s], C::StageBytes);
 #pragma unroll
       for (int j = 0; j < C::KS; ++j) {
-        const int k0 = (q.kb * C::KS + j) * 64;
-        tma_load_2d_hint(st + j * kWBytes, &a.mapW[q.seg], &full[s], k0, q.row0, wpol);
-        if (a.has_lo) tma_load_3d(st + C::KS * kWBytes + j * C::XBytes, &a.mapXhi, &full[s], q.xoff + k0, 0, 0);
-        else tma_load_2d(st + C::KS * kWBytes + j * C::XBytes, &a.mapXhi, &full[s], q.xoff + k0, 0);
+        const int k0 = q.k0(j);
+        tma_load_2d_hint(st + j * kWBytes, &a.mapW[q.q.seg], &full[s], k0, q.q.row0, wpol);
+        if (a.has_lo) tma_load_3d(st + C::KS * kWBytes + j * C::XBytes, &a.mapXhi, &full[s], q.q.xoff + k0, 0, 0);
+        else tma_load_2d(st + C::KS * kWBytes + j * C::XBytes, &a.mapXhi, &full[s], q.q.xoff + k0, 0);
       }
       if (++s == C::Stages) { s = 0; ++ph; }
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer
     constexpr uint32_t idesc = idesc_bf16(128, C::N);
-    const int n = (int)(u1 - u0);
+    const int n = (int)(u1 - u0) * C::SPU;
     int visit = -1, buf = 0, tile = -1;
-    int t = (int)(u0 / KB), kb = (int)(u0 % KB), s = 0, ph = 0;
+    int t = (int)(u0 / KB), kb = (int)(u0 % KB), sub = 0, s = 0, ph = 0;
     bool ok = true;
     for (int it = 0; it < n && ok; ++it) {
       bool first = false;                            // first block of this visit: overwrite the accumulator
@@ -199,7 +209,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
       }
       mma_commit(&empty[s]);
       if (++s == C::Stages) { s = 0; ++ph; }
-      if (++kb == KB) { kb = 0; ++t; }
+      if (++sub == C::SPU) {
+        sub = 0;
+        if (++kb == KB) { kb = 0; ++t; }
+      }
     }
     if (ok && tile >= 0) mma_commit(&acc_full[buf]);
   } else if (warp >= 4 && warp < 8) {
