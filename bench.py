@@ -491,8 +491,8 @@ def cpu_baseline(w, wt, inp, rows, gpu_tree=None):
 
 # DRAM traffic of one LM-head launch, from the committed ncu capture of the vocab-32768 case of the same
 # kernel: dram__bytes_read / algorithmic bytes, and dram__bytes_write (per-CTA results, independent of vocab).
-LM_READ_RATIO = 336.96e6 / 335.544e6
-LM_WRITE_BYTES = 3.5e6
+LM_READ_RATIO = 335.78e6 / 335.544e6
+LM_WRITE_BYTES = 4.0e6
 LM_EVERY = 8      # timed steps between two event-bracketed LM-head launches
 
 
