@@ -28,7 +28,7 @@ using namespace umma;
 constexpr int kUmmaThreads = 512;
 constexpr int kWBytes = 128 * 64 * 2;
 
-template <int MP>
+template <int MP, bool ONE = (MP == 128)>      // ONE: one 64-k block per stage (a work unit is then two stages)
 struct UmmaCfg {
   static constexpr int N = 2 * MP;                       // hi rows + lo rows
   static constexpr int XBytes = N * 64 * 2;
@@ -36,11 +36,12 @@ struct UmmaCfg {
   // of the ring costs about the same ~690 cycles whatever it holds, and one block -- 16 KB of weights -- per stage is
   // just an SM's share of HBM.  The plans count their units in stages (GemmPlan::KR).
   // At 128 token rows a block pair would be a 96 KB stage, two to the ring (measured slower than four of 48 KB): there
-  // a unit is SPU = 2 stages of one block each.
-  static constexpr int KS = MP == 128 ? 1 : kUmmaKS;      // 64-k blocks per stage
+  // a unit is SPU = 2 stages of one block each.  So it is for QKV at 32 token rows (59.7 us against 64.3 with block
+  // pairs at a 32B shape, where o_proj and down gain from the pairs: 34.8 and 59.4 us against 36.9 and 63.5).
+  static constexpr int KS = ONE ? 1 : kUmmaKS;            // 64-k blocks per stage
   static constexpr int SPU = kUmmaKS / KS;                // stages per work unit
   static constexpr int StageBytes = KS * (kWBytes + XBytes);
-  static constexpr int Stages = MP == 8 ? 5 : 4;
+  static constexpr int Stages = MP == 8 ? 5 : (MP == 32 && ONE ? 8 : 4);
   static constexpr int TmemCols = 2 * N < 32 ? 32 : 2 * N;
   static constexpr size_t SmemBytes = (size_t)Stages * StageBytes + 1024;
 };
@@ -87,9 +88,9 @@ struct StagePos {
   }
 };
 
-template <int MP>
+template <int MP, bool ONE>
 __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid_constant__ UmmaGemmArgs a) {
-  using C = UmmaCfg<MP>;
+  using C = UmmaCfg<MP, ONE>;
   const GemmArgs& p = a.g;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -311,12 +312,12 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) umma_rows_kernel(const __grid
   }
 }
 
-template <int MP>
+template <int MP, bool ONE>
 static cudaError_t launch_umma_t(const UmmaGemmArgs& a, int grid, cudaStream_t st) {
-  using C = UmmaCfg<MP>;
-  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_rows_kernel<MP>), C::SmemBytes);
+  using C = UmmaCfg<MP, ONE>;
+  const cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(umma_rows_kernel<MP, ONE>), C::SmemBytes);
   if (e != cudaSuccess) return e;
-  return launch_pdl(umma_rows_kernel<MP>, dim3(grid), dim3(kUmmaThreads), C::SmemBytes, st, a);
+  return launch_pdl(umma_rows_kernel<MP, ONE>, dim3(grid), dim3(kUmmaThreads), C::SmemBytes, st, a);
 }
 
 cudaError_t launch_umma_rows(const GemmPlan& plan, const UmmaMaps& maps, const GemmInput& in, const EpiArgs& epi, float* part,
@@ -335,9 +336,9 @@ cudaError_t launch_umma_rows(const GemmPlan& plan, const UmmaMaps& maps, const G
   a.mapXhi = maps.Xhi; a.has_lo = in.x_lo != nullptr ? 1 : 0;
   a.status = status;
   const int MP = padded_tokens(in.M);
-  if (MP == 8) return launch_umma_t<8>(a, plan.grid, st);
-  if (MP == 32) return launch_umma_t<32>(a, plan.grid, st);
-  return launch_umma_t<128>(a, plan.grid, st);
+  if (MP == 8) return launch_umma_t<8, false>(a, plan.grid, st);
+  if (MP == 32) return epi.mode == EPI_QKV ? launch_umma_t<32, true>(a, plan.grid, st) : launch_umma_t<32, false>(a, plan.grid, st);
+  return launch_umma_t<128, true>(a, plan.grid, st);
 }
 
 }  // namespace dart
